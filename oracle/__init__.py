@@ -1,0 +1,11 @@
+"""CPU oracle for placement scoring.  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg import this package.
+It compiles oracle/maaso_oracle.c with gcc on first use and calls it through ctypes;
+it imports nothing from the CUDA package.
+"""
+from .binding import (build, eval_placements, eval_placements_parallel, topk,
+                      FLAG_PRED_OPTIMISTIC, STATUS)
+
+__all__ = ["build", "eval_placements", "eval_placements_parallel", "topk",
+           "FLAG_PRED_OPTIMISTIC", "STATUS"]

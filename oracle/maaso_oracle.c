@@ -1,0 +1,399 @@
+/*
+ * CPU oracle for placement scoring by trace replay.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-threaded discrete-event simulation of what the placer's
+ * simulator computes for ONE candidate placement: requests are taken in trace
+ * order, the SLO-aware distributor picks an instance (or blocks, or rejects), every
+ * instance runs continuous batching with at most B virtual slots, and decode-step
+ * times come from the profiler's latency tables.  Nothing here is tuned; nothing
+ * here is shared with the CUDA library (own structs, own constants, own helpers).
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg call it.
+ *
+ * Passages followed (paper section / equation):
+ *   - "Simulator Implementation" (Sec. V-A): virtual slots = inference batch size;
+ *     "map" puts a request into a free slot, "reduce" advances instance clocks when
+ *     no slot is free and retries, until the request is accommodated or rejected.
+ *   - Distributor, Sec. IV-F steps 1-3: sub-cluster mapping (class mask), capability
+ *     check + choice among capable instances, overflow protection with the
+ *     worst-case throughput F(M,P,B_I).
+ *   - Profiler, Sec. IV-B Eq. 1: decode rate depends on min(B, W); here as a table
+ *     step_us[w] = time of one decode step with w running requests, w <= B.
+ *   - Sec. II-A "Inference Batch Size": at most B running requests, others wait.
+ *   - Sec. IV-C: L_r = L_q + L_d, SLO indicator [L_q + L_d <= tau_r] (objective
+ *     Phi_S), constraints (b)-(d).
+ *   - Sec. V-A "Evaluation Metrics": SLO attainment, decoding throughput, response
+ *     latency = time to first token.
+ *
+ * Readings taken where the paper is silent or ambiguous (all integer microseconds):
+ *   - Prefill of a request runs alone at a decode-step boundary of its instance and
+ *     stalls the running decodes; the first token appears when it ends.
+ *       prefill = base + ((q16 * in_tokens + 32768) >> 16)
+ *   - Decode speed is dynamic: one step for all w running requests takes step_us[w];
+ *     admissions and completions happen only at step boundaries.
+ *   - One FIFO at the dispatcher (head-of-line): a blocked request holds back later
+ *     ones; `now` only moves forward.
+ *   - Choice among feasible instances: free slot first, then earliest predicted first
+ *     token, then lowest instance index.
+ *   - "Block" = defer while some full instance is still predicted feasible at the exact
+ *     time its next slot frees; reject once none is.
+ *   - A request with one output token completes at the end of its prefill and never
+ *     occupies a slot.
+ *   - TBT limit is on the mean gap: finish - first_token <= (S-1) * tbt.
+ *
+ * Parity pins (tests/, marker "not gpu"): hand-worked timelines under tests/golden/,
+ * the single-server FIFO (Lindley) closed form for B = 1, the no-contention closed
+ * form, a token-by-token re-formulation, conservation / monotonicity invariants,
+ * mask algebra, the no-cascade special case with zero prefill, and brute-force
+ * ranking.  Agreement with the paper's figures is "parity unpinned": the figures,
+ * measured profiles and traces are not available.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_WMAX 64
+#define ORC_MAX_INST 128
+#define ORC_ATTEMPT_CAP (2u + ORC_MAX_INST * ORC_WMAX)
+
+/* candidate status bits */
+#define ORC_EBUDGET 1u   /* devices used exceed the budget: constraint (c) */
+#define ORC_EMEMFIT 2u   /* an instance has fewer devices than its model needs: (d) */
+#define ORC_ETOOMANY 4u  /* more than ORC_MAX_INST instances */
+#define ORC_EBADINST 8u  /* unknown model / strategy, batch cap outside 1..64, reserved bits */
+#define ORC_ETIMEOUT 16u /* never set by the oracle */
+#define ORC_ELOOP 32u    /* attempt cap hit (cannot happen if the termination argument holds) */
+#define ORC_EINVARIANT 0x80000000u /* an internal invariant failed: the oracle is wrong */
+
+#define ORC_FLAG_PRED_OPTIMISTIC 1u
+
+typedef struct {
+    int64_t arrival_us;
+    uint32_t in_tokens;
+    uint16_t out_tokens;
+    uint8_t cls;
+    uint8_t model;
+} orc_request;
+
+typedef struct {
+    int64_t ttft_us, tbt_us, e2e_us; /* negative = no limit */
+} orc_slo;
+
+typedef struct {
+    uint32_t n_models, n_strategies, wmax;
+    const int32_t *devices;         /* [S] */
+    const int32_t *min_devices;     /* [M] */
+    const int32_t *prefill_base_us; /* [M][S] */
+    const int32_t *prefill_q16;     /* [M][S] */
+    const int32_t *step_us;         /* [M][S][wmax], entry w-1 = step time at running count w */
+} orc_profile;
+
+typedef struct {
+    uint32_t status, n_counted, n_served, n_hit, n_rejected, n_cascade;
+    uint32_t hit_by_class[8];
+    int64_t sum_ttft_us, max_ttft_us, sum_e2e_us, max_e2e_us, makespan_us;
+    uint64_t tokens_out, checksum, attempts, reserved;
+} orc_result;
+
+typedef struct {
+    int used;
+    uint32_t req;
+    int64_t arrival, first_tok;
+    int64_t fin_idx; /* value of the instance's step counter at which this request ends */
+    uint32_t S;
+    uint32_t cls;
+} slot_t;
+
+typedef struct {
+    uint32_t model, strat, B;
+    const int32_t *step; /* step[w-1] */
+    int64_t pre_base;
+    int64_t pre_q16;
+    int64_t T; /* clock; always a step boundary */
+    int64_t K; /* decode steps done so far */
+    uint32_t w; /* running requests */
+    slot_t slots[ORC_WMAX];
+} inst_t;
+
+typedef struct {
+    const orc_slo *classes;
+    orc_result *res;
+    int64_t *dump_finish; /* [n] or NULL */
+    int64_t *dump_first;
+    int32_t *dump_inst;
+    int bad; /* invariant violated */
+} ctx_t;
+
+/* SplitMix64 output mixer (public domain, Steele/Lea/Flood) */
+static uint64_t mix64(uint64_t z) {
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+    z ^= z >> 27; z *= 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    return z;
+}
+static uint64_t rotl64(uint64_t x, int r) { return (x << r) | (x >> (64 - r)); }
+
+/* A request leaves the system served: Phi_S indicator, latency and throughput sums. */
+static void complete(ctx_t *c, uint32_t inst_idx, uint32_t req, int64_t arrival, int64_t first_tok,
+                     int64_t t_fin, uint32_t S, uint32_t cls) {
+    const orc_slo *k = &c->classes[cls];
+    int64_t ttft = first_tok - arrival, e2e = t_fin - arrival, span = t_fin - first_tok;
+    int hit = (k->ttft_us < 0 || ttft <= k->ttft_us) &&
+              (k->tbt_us < 0 || span <= (int64_t)(S - 1) * k->tbt_us) &&
+              (k->e2e_us < 0 || e2e <= k->e2e_us);
+    orc_result *r = c->res;
+    if (ttft < 0 || span < 0) c->bad = 1;
+    r->n_served++;
+    if (hit) { r->n_hit++; r->hit_by_class[cls < 7 ? cls : 7]++; } else r->n_cascade++;
+    r->sum_ttft_us += ttft; if (ttft > r->max_ttft_us) r->max_ttft_us = ttft;
+    r->sum_e2e_us += e2e;   if (e2e > r->max_e2e_us) r->max_e2e_us = e2e;
+    r->tokens_out += S;
+    if (t_fin > r->makespan_us) r->makespan_us = t_fin;
+    r->checksum += mix64((uint64_t)req * 0x9E3779B97F4A7C15ull ^ (uint64_t)t_fin ^
+                         rotl64((uint64_t)first_tok, 32) ^ ((uint64_t)inst_idx << 56));
+    if (c->dump_finish) c->dump_finish[req] = t_fin;
+    if (c->dump_first) c->dump_first[req] = first_tok;
+    if (c->dump_inst) c->dump_inst[req] = (int32_t)inst_idx;
+}
+
+static int64_t min_fin(const inst_t *in) {
+    int64_t m = INT64_MAX;
+    for (uint32_t j = 0; j < in->B; j++)
+        if (in->slots[j].used && in->slots[j].fin_idx < m) m = in->slots[j].fin_idx;
+    return m;
+}
+
+/* "reduce": run whole decode steps until the clock reaches t (t < 0 means: until empty). */
+static void advance(ctx_t *c, inst_t *in, uint32_t inst_idx, int64_t t) {
+    int drain = t < 0;
+    while (in->w > 0 && (drain || in->T < t)) {
+        int64_t s = in->step[in->w - 1];
+        int64_t kfin = min_fin(in) - in->K;
+        int64_t k = kfin;
+        if (kfin < 1) c->bad = 1;
+        if (!drain) {
+            int64_t need = (t - in->T + s - 1) / s; /* ceil */
+            if (need < k) k = need;
+        }
+        in->T += k * s;
+        in->K += k;
+        for (uint32_t j = 0; j < in->B; j++) {
+            slot_t *sl = &in->slots[j];
+            if (sl->used && sl->fin_idx == in->K) {
+                complete(c, inst_idx, sl->req, sl->arrival, sl->first_tok, in->T, sl->S, sl->cls);
+                sl->used = 0;
+                in->w--;
+            }
+        }
+    }
+    if (!drain && in->w == 0 && in->T < t) in->T = t; /* an idle instance starts at once */
+}
+
+static int64_t prefill_us(const inst_t *in, uint32_t in_tokens) {
+    return in->pre_base + (int64_t)(((uint64_t)in->pre_q16 * in_tokens + 32768u) >> 16);
+}
+
+/* Validate the instance list against constraints (c), (d) and the table ranges. */
+static uint32_t validate(const orc_profile *p, const uint32_t *inst, uint32_t n_inst, uint32_t budget) {
+    uint32_t status = 0;
+    uint64_t devsum = 0;
+    if (n_inst > ORC_MAX_INST) return ORC_ETOOMANY;
+    for (uint32_t i = 0; i < n_inst; i++) {
+        uint32_t word = inst[i];
+        uint32_t m = word & 0xF, s = (word >> 4) & 0xFF, b = (word >> 12) & 0xFF;
+        if ((word >> 20) != 0 || m >= p->n_models || s >= p->n_strategies || b < 1 || b > p->wmax ||
+            b > ORC_WMAX) {
+            status |= ORC_EBADINST;
+            continue;
+        }
+        devsum += (uint64_t)p->devices[s];
+        if (p->devices[s] < p->min_devices[m]) status |= ORC_EMEMFIT;
+    }
+    if (devsum > budget) status |= ORC_EBUDGET;
+    return status;
+}
+
+/*
+ * Score one candidate.  inst[n_inst]: packed words (model bits 0-3, strategy 4-11, batch
+ * cap 12-19).  has_mask/class_mask: requests whose class bit is clear are not part of the
+ * request subset R_x this placement is scored on (ignored when n_classes > 32).
+ * dump_* (each [n] or NULL): per request finish time / first-token time / instance;
+ * -1 = rejected, -2 = not counted.
+ * Returns 0; the outcome is in out->status.
+ */
+int orc_eval_candidate(const orc_profile *p, const orc_request *reqs, uint64_t n,
+                       const orc_slo *classes, uint32_t n_classes, const uint32_t *inst,
+                       uint32_t n_inst, int has_mask, uint32_t class_mask, uint32_t budget,
+                       uint32_t flags, orc_result *out, int64_t *dump_finish, int64_t *dump_first,
+                       int32_t *dump_inst) {
+    ctx_t c;
+    memset(out, 0, sizeof(*out));
+    c.classes = classes; c.res = out; c.bad = 0;
+    c.dump_finish = dump_finish; c.dump_first = dump_first; c.dump_inst = dump_inst;
+    for (uint64_t r = 0; r < n; r++) {
+        if (dump_finish) dump_finish[r] = -2;
+        if (dump_first) dump_first[r] = -2;
+        if (dump_inst) dump_inst[r] = -2;
+    }
+    out->status = validate(p, inst, n_inst, budget);
+    if (out->status) return 0;
+    if (n_classes > 32) has_mask = 0;
+
+    inst_t *I = (inst_t *)calloc(n_inst ? n_inst : 1, sizeof(inst_t));
+    if (!I) return -1;
+    for (uint32_t i = 0; i < n_inst; i++) {
+        uint32_t word = inst[i];
+        I[i].model = word & 0xF; I[i].strat = (word >> 4) & 0xFF; I[i].B = (word >> 12) & 0xFF;
+        size_t row = (size_t)I[i].model * p->n_strategies + I[i].strat;
+        I[i].step = p->step_us + row * p->wmax;
+        I[i].pre_base = p->prefill_base_us[row];
+        I[i].pre_q16 = (int64_t)(uint32_t)p->prefill_q16[row];
+    }
+
+    int64_t now = 0;
+    for (uint64_t r = 0; r < n && !out->status; r++) {
+        const orc_request *q = &reqs[r];
+        if (has_mask && !((class_mask >> q->cls) & 1u)) continue; /* not in R_x */
+        const orc_slo *k = &classes[q->cls];
+        int64_t S = q->out_tokens;
+        out->n_counted++;
+        if (q->arrival_us > now) now = q->arrival_us; /* pending time: never back in time */
+        for (uint32_t attempt = 0;; attempt++) {
+            if (attempt >= ORC_ATTEMPT_CAP) { out->status = ORC_ELOOP; break; }
+            out->attempts++;
+            for (uint32_t i = 0; i < n_inst; i++) {
+                int64_t before = I[i].T;
+                advance(&c, &I[i], i, now);
+                if (I[i].T < before || I[i].w > I[i].B) c.bad = 1;
+            }
+            int have = 0; int best_tier = 0; int64_t best_first = 0, best_t0 = 0; uint32_t best_i = 0;
+            for (uint32_t i = 0; i < n_inst; i++) {
+                inst_t *in = &I[i];
+                if (in->model != q->model) continue;
+                int tier; int64_t t0;
+                if (in->w < in->B) { tier = 0; t0 = in->T; }             /* a free virtual slot */
+                else { tier = 1; t0 = in->T + (min_fin(in) - in->K) * (int64_t)in->step[in->w - 1]; }
+                int64_t pre = prefill_us(in, q->in_tokens);
+                int64_t sB = in->step[in->B - 1];                        /* worst case F(M,P,B_I) */
+                if ((flags & ORC_FLAG_PRED_OPTIMISTIC) && tier == 0) {
+                    uint32_t wn = in->w + 1 < in->B ? in->w + 1 : in->B;
+                    sB = in->step[wn - 1];
+                }
+                int64_t first = t0 + pre, fin = first + (S - 1) * sB;
+                int feasible = (k->ttft_us < 0 || first - q->arrival_us <= k->ttft_us) &&
+                               (k->tbt_us < 0 || S == 1 || sB <= k->tbt_us) &&
+                               (k->e2e_us < 0 || fin - q->arrival_us <= k->e2e_us);
+                if (!feasible) continue;
+                if (!have || tier < best_tier || (tier == best_tier && first < best_first)) {
+                    have = 1; best_tier = tier; best_first = first; best_t0 = t0; best_i = i;
+                }
+            }
+            if (!have) { /* overflow protection: no instance can meet the deadline */
+                out->n_rejected++;
+                out->checksum += mix64((uint64_t)r * 0x9E3779B97F4A7C15ull ^ ~0ull);
+                if (dump_finish) dump_finish[r] = -1;
+                if (dump_first) dump_first[r] = -1;
+                if (dump_inst) dump_inst[r] = -1;
+                break;
+            }
+            if (best_tier == 0) { /* "map": prefill at the boundary, then occupy a slot */
+                inst_t *in = &I[best_i];
+                in->T += prefill_us(in, q->in_tokens);
+                if (S == 1) {
+                    complete(&c, best_i, (uint32_t)r, q->arrival_us, in->T, in->T, 1, q->cls);
+                } else {
+                    uint32_t j = 0;
+                    while (j < in->B && in->slots[j].used) j++;
+                    if (j >= in->B) { c.bad = 1; break; }
+                    slot_t *sl = &in->slots[j];
+                    sl->used = 1; sl->req = (uint32_t)r; sl->arrival = q->arrival_us;
+                    sl->first_tok = in->T; sl->fin_idx = in->K + S - 1; sl->S = (uint32_t)S;
+                    sl->cls = q->cls;
+                    in->w++;
+                }
+                break;
+            }
+            if (best_t0 <= now) c.bad = 1; /* a wait must move time strictly forward */
+            now = best_t0;                 /* wait until that slot frees, then try again */
+        }
+    }
+    if (!out->status)
+        for (uint32_t i = 0; i < n_inst; i++) advance(&c, &I[i], i, -1); /* drain */
+    free(I);
+
+    if (!out->status) {
+        if (out->n_counted != out->n_served + out->n_rejected) c.bad = 1; /* conservation */
+        if (out->n_cascade != out->n_served - out->n_hit) c.bad = 1;
+    }
+    if (c.bad) out->status |= ORC_EINVARIANT;
+    if (out->status) { /* invalid candidates carry a status and nothing else */
+        uint32_t st = out->status;
+        memset(out, 0, sizeof(*out));
+        out->status = st;
+    }
+    return 0;
+}
+
+/* Score a batch: CSR offsets[n_cand+1] into inst[]; class_mask may be NULL.
+ * dump_idx[dump_n] picks candidates whose per-request times are written to
+ * dump_finish / dump_first / dump_inst, each [dump_n][n] (any may be NULL). */
+int orc_eval_batch(const orc_profile *p, const orc_request *reqs, uint64_t n, const orc_slo *classes,
+                   uint32_t n_classes, const uint32_t *offsets, const uint32_t *inst,
+                   const uint32_t *class_mask, uint64_t n_cand, uint32_t budget, uint32_t flags,
+                   orc_result *out, const uint32_t *dump_idx, uint32_t dump_n, int64_t *dump_finish,
+                   int64_t *dump_first, int32_t *dump_inst) {
+    for (uint64_t c = 0; c < n_cand; c++) {
+        int64_t *df = NULL, *d1 = NULL; int32_t *di = NULL;
+        for (uint32_t d = 0; d < dump_n; d++)
+            if (dump_idx[d] == c) {
+                if (dump_finish) df = dump_finish + (size_t)d * n;
+                if (dump_first) d1 = dump_first + (size_t)d * n;
+                if (dump_inst) di = dump_inst + (size_t)d * n;
+            }
+        int rc = orc_eval_candidate(p, reqs, n, classes, n_classes, inst + offsets[c],
+                                    offsets[c + 1] - offsets[c], class_mask != NULL,
+                                    class_mask ? class_mask[c] : 0, budget, flags, &out[c], df, d1, di);
+        if (rc) return rc;
+    }
+    return 0;
+}
+
+/*
+ * Ranking used for "keep the best placements" (order 0): valid candidates first; more SLO
+ * hits first; then lower mean time-to-first-token, sum/n_served compared exactly by
+ * cross-multiplication in 128 bits (a candidate that served nothing ranks after any that
+ * served something); then lower candidate index.
+ */
+static const orc_result *g_res;
+static int before(uint32_t a, uint32_t b) {
+    const orc_result *x = &g_res[a], *y = &g_res[b];
+    int vx = x->status == 0, vy = y->status == 0;
+    if (vx != vy) return vx > vy;
+    if (vx) {
+        if (x->n_hit != y->n_hit) return x->n_hit > y->n_hit;
+        int sx = x->n_served > 0, sy = y->n_served > 0;
+        if (sx != sy) return sx > sy;
+        if (sx) {
+            unsigned __int128 l = (unsigned __int128)(uint64_t)x->sum_ttft_us * y->n_served;
+            unsigned __int128 r = (unsigned __int128)(uint64_t)y->sum_ttft_us * x->n_served;
+            if (l != r) return l < r;
+        }
+    }
+    return a < b;
+}
+static int cmp(const void *pa, const void *pb) {
+    uint32_t a = *(const uint32_t *)pa, b = *(const uint32_t *)pb;
+    if (a == b) return 0;
+    return before(a, b) ? -1 : 1;
+}
+/* out_idx[min(k, n)] = indices of the k best candidates, best first. */
+int orc_topk(const orc_result *res, uint64_t n, uint32_t k, uint32_t order, uint32_t *out_idx) {
+    if (order != 0) return -1;
+    uint32_t *idx = (uint32_t *)malloc((n ? n : 1) * sizeof(uint32_t));
+    if (!idx) return -1;
+    for (uint64_t i = 0; i < n; i++) idx[i] = (uint32_t)i;
+    g_res = res;
+    qsort(idx, n, sizeof(uint32_t), cmp);
+    for (uint64_t i = 0; i < k && i < n; i++) out_idx[i] = idx[i];
+    free(idx);
+    return 0;
+}

@@ -1,0 +1,320 @@
+"""Pins for the CPU oracle: things fixed by the paper's rules and by mathematics, none of
+them produced by the oracle itself."""
+import numpy as np
+import pytest
+
+import gen
+from golden_cases import all_cases, check_against_expect, SCALAR_KEYS
+from stepwise_sim import simulate
+
+NONE3 = [(None, None, None)]
+
+
+def one_instance_profile(step1=9150, steps=None, base=2000, q16=7864):
+    table = np.full((1, 1, gen.WMAX), step1, dtype=np.int32)
+    if steps is not None:
+        table[0, 0, : len(steps)] = steps
+        table[0, 0, len(steps):] = steps[-1]
+    return {"n_models": 1, "n_strategies": 1, "wmax": gen.WMAX,
+            "devices": np.array([1], dtype=np.int32), "min_devices": np.array([1], dtype=np.int32),
+            "prefill_base_us": np.array([[base]], dtype=np.int32),
+            "prefill_q16": np.array([[q16]], dtype=np.int32), "step_us": table}
+
+
+def run_one(oracle, profile, trace, classes, instances, budget=128, mask=None, flags=0):
+    offsets, inst = gen.candidates_from_lists([instances])
+    cm = None if mask is None else np.array([mask], dtype=np.uint32)
+    res, dumps = oracle.eval_placements(profile, trace, classes, offsets, inst, budget, cm, flags,
+                                        dump_idx=[0])
+    return res[0], {k: v[0] for k, v in dumps.items()}
+
+
+# ---- P1: hand-worked timelines -------------------------------------------------------------
+@pytest.mark.parametrize("case", all_cases(), ids=lambda c: c["name"])
+def test_hand_timelines(oracle_mod, case):
+    for flags, expect in case["runs"]:
+        res, dumps = oracle_mod.eval_placements(case["profile"], case["trace"], case["classes"],
+                                                case["offsets"], case["inst"], case["budget"],
+                                                None, flags, dump_idx=[0])
+        check_against_expect(res[0], {k: v[0] for k, v in dumps.items()}, expect)
+
+
+# ---- P2: B = 1, one instance, no SLO limits = single-server FIFO (Lindley recursion) --------
+def test_single_server_closed_form(oracle_mod):
+    prof = gen.profile_tiny()
+    trace = gen.make_trace(400, 3.0, 11)
+    classes = gen.make_classes(NONE3 * 3)
+    res, d = run_one(oracle_mod, prof, trace, classes, [(0, 1, 1)])
+    base, q16, s1 = int(prof["prefill_base_us"][0, 1]), int(prof["prefill_q16"][0, 1]), int(prof["step_us"][0, 1, 0])
+    prev = 0
+    fin, first = [], []
+    for q in trace:
+        start = max(int(q["arrival_us"]), prev)
+        f1 = start + base + ((q16 * int(q["in_tokens"]) + 32768) >> 16)
+        prev = f1 + (int(q["out_tokens"]) - 1) * s1
+        first.append(f1)
+        fin.append(prev)
+    assert d["finish_us"].tolist() == fin
+    assert d["first_us"].tolist() == first
+    assert int(res["n_served"]) == 400 and int(res["n_hit"]) == 400 and int(res["n_rejected"]) == 0
+    arr = trace["arrival_us"].astype(np.int64)
+    assert int(res["sum_e2e_us"]) == int((np.array(fin) - arr).sum())
+    assert int(res["sum_ttft_us"]) == int((np.array(first) - arr).sum())
+    assert int(res["max_ttft_us"]) == int((np.array(first) - arr).max())
+    assert int(res["makespan_us"]) == fin[-1]
+    assert int(res["tokens_out"]) == int(trace["out_tokens"].astype(np.int64).sum())
+
+
+# ---- P3: no contention: every request alone in the system ---------------------------------
+def test_no_contention_closed_form(oracle_mod):
+    prof = gen.profile_tiny()
+    trace = gen.make_trace(60, 1.0, 5)
+    trace["arrival_us"] = np.arange(60, dtype=np.int64) * 400_000_000  # 400 s apart
+    classes = gen.make_classes(NONE3 * 3)
+    # instance 2 (tp4) has the smallest prefill; instances 0 and 1 are identical tp2 rows
+    res, d = run_one(oracle_mod, prof, trace, classes, [(0, 1, 4), (0, 1, 8), (0, 2, 2), (0, 0, 16)])
+    base, q16, s1 = int(prof["prefill_base_us"][0, 2]), int(prof["prefill_q16"][0, 2]), int(prof["step_us"][0, 2, 0])
+    for k, q in enumerate(trace):
+        f1 = int(q["arrival_us"]) + base + ((q16 * int(q["in_tokens"]) + 32768) >> 16)
+        assert int(d["first_us"][k]) == f1
+        assert int(d["finish_us"][k]) == f1 + (int(q["out_tokens"]) - 1) * s1
+        assert int(d["inst"][k]) == 2
+    # ties go to the lowest index
+    res, d = run_one(oracle_mod, prof, trace, classes, [(0, 1, 4), (0, 1, 8)])
+    assert set(d["inst"].tolist()) == {0}
+
+
+# ---- P8: token-by-token re-formulation on tiny inputs -------------------------------------
+@pytest.mark.parametrize("seed", range(12))
+def test_against_token_by_token(oracle_mod, seed):
+    rng = np.random.default_rng(1000 + seed)
+    if seed % 3 == 2:
+        prof = gen.profile_multimodel(seed)
+        model_mix = (0.5, 0.3, 0.2)
+    else:
+        prof = gen.profile_node(seed)
+        model_mix = (1.0,)
+    M, S = prof["n_models"], prof["n_strategies"]
+    trace = gen.make_trace(120, float(rng.choice([4.0, 20.0, 80.0])), seed, cv=float(rng.choice([1.0, 3.0])),
+                           model_mix=model_mix, out_dist=("lognormal", 3.0, 1.0, 1, 300),
+                           doc_out=(200, 400))
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None),
+                                (None, None, 8_000_000)])
+    n_inst = int(rng.integers(1, 7))
+    instances = []
+    for _ in range(n_inst):
+        m = int(rng.integers(M))
+        ok = np.nonzero(prof["devices"] >= prof["min_devices"][m])[0]
+        instances.append((m, int(rng.choice(ok)), int(rng.choice([1, 2, 3, 4, 8, 16, 64]))))
+    mask = None if seed % 4 else 0b101
+    flags = seed % 2
+    res, d = run_one(oracle_mod, prof, trace, classes, instances, mask=mask, flags=flags)
+    ref = simulate(prof, trace, classes, instances, class_mask=mask, optimistic=bool(flags))
+    for key in SCALAR_KEYS:
+        assert int(res[key]) == ref[key], key
+    assert d["finish_us"].tolist() == ref["finish_us"]
+    assert d["first_us"].tolist() == ref["first_us"]
+    assert d["inst"].tolist() == ref["inst"]
+
+
+# ---- P4: invariants -----------------------------------------------------------------------
+def test_invariants_on_tiny_config(oracle_mod):
+    cfg = gen.make_config("tiny")
+    n = len(cfg["traces"][0])
+    idx = np.arange(0, 143, 7, dtype=np.uint32)
+    res, dumps = oracle_mod.eval_placements(cfg["profile"], cfg["traces"][0], cfg["classes"],
+                                            cfg["offsets"], cfg["inst"], cfg["budget"], dump_idx=idx)
+    assert (res["status"] == 0).all()          # includes the oracle's own invariant flag
+    assert (res["n_counted"] == n).all()
+    assert (res["n_served"] + res["n_rejected"] == n).all()      # conservation
+    assert (res["n_cascade"] == res["n_served"] - res["n_hit"]).all()
+    assert (res["hit_by_class"].sum(axis=1) == res["n_hit"]).all()
+    arr = cfg["traces"][0]["arrival_us"].astype(np.int64)
+    S = cfg["traces"][0]["out_tokens"].astype(np.int64)
+    for row, c in enumerate(idx):
+        fin, first, where = dumps["finish_us"][row], dumps["first_us"][row], dumps["inst"][row]
+        served = fin >= 0
+        assert served.sum() == res["n_served"][c]
+        assert ((fin == -1) == (where == -1)).all()
+        assert (first[served] >= arr[served]).all() and (fin[served] >= first[served]).all()
+        assert int((first[served] - arr[served]).sum()) == int(res["sum_ttft_us"][c])
+        assert int((fin[served] - arr[served]).sum()) == int(res["sum_e2e_us"][c])
+        assert int(S[served].sum()) == int(res["tokens_out"][c])
+        # batch cap: at any first-token instant, running requests on that instance <= B
+        lo, hi = int(cfg["offsets"][c]), int(cfg["offsets"][c + 1])
+        caps = ((cfg["inst"][lo:hi] >> 12) & 0xFF).astype(np.int64)
+        for i, cap in enumerate(caps):
+            on = served & (where == i) & (S > 1)
+            f1, f2 = first[on], fin[on]
+            for t in f1:
+                assert ((f1 <= t) & (f2 > t)).sum() <= cap
+        # first tokens on one instance are strictly ordered by request index (FIFO dispatcher)
+        for i in range(hi - lo):
+            on = served & (where == i)
+            assert (np.diff(first[on]) > 0).all()
+
+
+# ---- P6: worst-case prediction + zero prefill + monotone table => no cascaded misses --------
+@pytest.mark.parametrize("seed", range(4))
+def test_no_cascade_without_prefill(oracle_mod, seed):
+    prof = gen.profile_node(seed)
+    prof["prefill_base_us"][:] = 0
+    prof["prefill_q16"][:] = 0
+    prof["step_us"][:] = np.maximum.accumulate(prof["step_us"], axis=2)
+    trace = gen.make_trace(1500, 40.0, seed, cv=2.0, out_dist=("lognormal", 4.0, 1.0, 1, 600),
+                           doc_out=(500, 900))
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None),
+                                (None, None, 20_000_000)])
+    offsets, inst = gen.enumerate_node(prof["devices"], 4, batches=(2, 16, 64))
+    res = oracle_mod.eval_placements(prof, trace, classes, offsets, inst, 8)
+    assert (res["status"] == 0).all()
+    assert res["n_served"].sum() > 0 and res["n_rejected"].sum() > 0
+    assert (res["n_cascade"] == 0).all()
+    # the optimistic estimate must show cascades somewhere (what overflow protection prevents)
+    res2 = oracle_mod.eval_placements(prof, trace, classes, offsets, inst, 8, flags=oracle_mod.FLAG_PRED_OPTIMISTIC)
+    assert res2["n_cascade"].sum() > 0
+
+
+# ---- P7: mask algebra ---------------------------------------------------------------------
+def test_mask_algebra(oracle_mod):
+    cfg = gen.make_config("tiny")
+    tr = cfg["traces"][0]
+    off, inst = cfg["offsets"], cfg["inst"]
+    C = len(off) - 1
+    a = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 4, np.full(C, 0b011, np.uint32))
+    b = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 4, np.full(C, 0b100, np.uint32))
+    full = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 4, np.full(C, 0b111, np.uint32))
+    nomask = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 4)
+    assert (a["n_counted"] + b["n_counted"] == len(tr)).all()
+    assert (a["n_counted"] == (tr["cls"] < 2).sum()).all()
+    assert full.tobytes() == nomask.tobytes()
+    # a masked run equals a run on the filtered trace except for request numbering (checksum)
+    sub = tr[tr["cls"] == 2]
+    c = oracle_mod.eval_placements(cfg["profile"], sub, cfg["classes"], off, inst, 4)
+    for key in SCALAR_KEYS:
+        assert (b[key] == c[key]).all(), key
+
+
+# ---- constraints (c), (d) and malformed instances -------------------------------------------
+def test_candidate_validation(oracle_mod):
+    prof = gen.profile_multimodel(0)
+    tr = gen.make_trace(50, 8.0, 0, model_mix=(0.6, 0.3, 0.1))
+    classes = gen.make_classes(NONE3 * 3)
+    lists = [
+        [(0, 6, 4), (0, 6, 4)],          # 16 devices > budget 8
+        [(2, 0, 4)],                      # 70B-like on one device
+        [(0, 0, 4)] * 129,                # too many
+        [(3, 0, 4)],                      # unknown model
+        [(0, 10, 4)],                     # unknown strategy
+        [(0, 0, 0)],                      # batch cap 0
+        [(0, 0, 65)],                     # batch cap too large
+        [(0, 0, 4), (2, 3, 8)],           # fine
+        [],                               # empty placement: everything is rejected
+    ]
+    off, inst = gen.candidates_from_lists(lists)
+    inst = inst.copy()
+    res = oracle_mod.eval_placements(prof, tr, classes, off, inst, 8)
+    E = oracle_mod.STATUS
+    assert res["status"].tolist() == [E["EBUDGET"], E["EMEMFIT"], E["ETOOMANY"], E["EBADINST"],
+                                      E["EBADINST"], E["EBADINST"], E["EBADINST"], 0, 0]
+    bad = res[res["status"] != 0]
+    for key in SCALAR_KEYS:
+        assert (bad[key] == 0).all()
+    assert int(res["n_rejected"][8]) == 50 and int(res["n_served"][8]) == 0
+    inst2 = inst.copy()
+    inst2[off[7]] |= 1 << 20                  # reserved bit set
+    res2 = oracle_mod.eval_placements(prof, tr, classes, off, inst2, 8)
+    assert int(res2["status"][7]) == E["EBADINST"]
+
+
+# ---- batch composition cannot matter ------------------------------------------------------
+def test_alone_in_batch_duplicated(oracle_mod):
+    cfg = gen.make_config("tiny")
+    tr, off, inst = cfg["traces"][0], cfg["offsets"], cfg["inst"]
+    full = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 4)
+    for c in (0, 57, 142):
+        words = inst[off[c]:off[c + 1]]
+        o2 = np.array([0, len(words), 2 * len(words)], dtype=np.uint32)
+        two = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], o2, np.concatenate([words, words]), 4)
+        assert two[0].tobytes() == full[c].tobytes() and two[1].tobytes() == full[c].tobytes()
+    par = oracle_mod.eval_placements_parallel(cfg["profile"], tr, cfg["classes"], off, inst, 4, workers=2)
+    assert par.tobytes() == full.tobytes()
+
+
+# ---- qualitative claims of the paper's batch-size study (Sec. III-B) ------------------------
+def test_batch_cap_tradeoff(oracle_mod):
+    prof = gen.profile_tiny()
+    trace = gen.make_trace(300, 6.0, 3, out_dist=("lognormal", 4.0, 0.5, 2, 400), doc_class=None)
+    classes = gen.make_classes(NONE3 * 3)
+    r4, d4 = run_one(oracle_mod, prof, trace, classes, [(0, 0, 4)])
+    r8, d8 = run_one(oracle_mod, prof, trace, classes, [(0, 0, 8)])
+    assert int(r4["n_served"]) == int(r8["n_served"]) == 300
+    # a larger cap relieves queuing ...
+    assert int(r8["sum_ttft_us"]) < int(r4["sum_ttft_us"])
+    # ... at the price of slower decoding per request
+    span4 = (d4["finish_us"] - d4["first_us"]).sum()
+    span8 = (d8["finish_us"] - d8["first_us"]).sum()
+    assert span4 < span8
+
+
+# ---- P5: ranking by brute force with exact rationals ----------------------------------------
+def test_topk_brute_force(oracle_mod):
+    from fractions import Fraction
+    cfg = gen.make_config("tiny")
+    res = oracle_mod.eval_placements(cfg["profile"], cfg["traces"][0], cfg["classes"], cfg["offsets"],
+                                     cfg["inst"], cfg["budget"])
+    res = res.copy()
+    res["status"][5] = 1           # invalid candidates go last
+    res["n_served"][9] = 0         # nothing served ranks after anything served, same hits
+    res["n_hit"][9] = res["n_hit"][10]
+    res["n_hit"][20] = res["n_hit"][21]  # force a tie on hits, decided by mean TTFT
+
+    def key(i):
+        r = res[i]
+        if r["status"] != 0:
+            return (1, 0, 0, 0, i)
+        served = int(r["n_served"])
+        mean = Fraction(int(r["sum_ttft_us"]), served) if served else Fraction(0)
+        return (0, -int(r["n_hit"]), 0 if served else 1, mean, i)
+
+    want = sorted(range(len(res)), key=key)
+    for k in (1, 7, 64, 143, 500):
+        got = oracle_mod.topk(res, k).tolist()
+        assert got == want[:k]
+
+
+def test_topk_exact_fraction_compare(oracle_mod):
+    """Means that differ by less than a double can resolve must still be ordered exactly."""
+    res = np.zeros(3, dtype=gen.RESULT_DTYPE)
+    big = (1 << 62) - 57
+    res["n_hit"] = 5
+    res["n_served"] = [1_000_003, 1_000_003, 1_000_002]
+    res["sum_ttft_us"] = [big, big - 1, big - 1_000_000_000_000]
+    # mean1 < mean0 by 1e-6/1e6; candidate 2: (big - 1e12)/1000002 vs big/1000003
+    from fractions import Fraction
+    want = sorted(range(3), key=lambda i: (Fraction(int(res["sum_ttft_us"][i]), int(res["n_served"][i])), i))
+    assert oracle_mod.topk(res, 3).tolist() == want
+
+
+# ---- generators -----------------------------------------------------------------------------
+def test_generator_counts_and_layout():
+    off, inst = gen.enumerate_tiny()
+    assert len(off) - 1 == 143
+    prof = gen.profile_node(0)
+    off, inst = gen.enumerate_node(prof["devices"], 8)
+    assert len(off) - 1 == 10864
+    tr = gen.make_trace(1000, 16.0, 0)
+    assert tr.dtype.itemsize == 16 and (np.diff(tr["arrival_us"]) >= 0).all()
+    assert tr["out_tokens"].min() >= 1
+    doc = tr["cls"] == 2
+    assert tr["out_tokens"][doc].min() >= 2048 and tr["out_tokens"][~doc].max() <= 2048
+    pm = gen.profile_multimodel(0)
+    off, inst = gen.sample_candidates(2000, 1, 32, pm)
+    m, s, b = gen.unpack_inst(inst)
+    cand = np.repeat(np.arange(2000), np.diff(off.astype(np.int64)))
+    used = np.bincount(cand, weights=pm["devices"][s], minlength=2000)
+    assert used.max() <= 32 and (np.diff(off.astype(np.int64)) >= 1).all()
+    assert (pm["devices"][s] >= pm["min_devices"][m]).all()
+    a = gen.make_trace(100, 8.0, 7)
+    b2 = gen.make_trace(100, 8.0, 7)
+    assert a.tobytes() == b2.tobytes()
