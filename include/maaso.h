@@ -1,0 +1,210 @@
+/*
+ * maaso.h — C ABI of the placement-scoring library.
+ *
+ * The library scores many candidate placements of heterogeneous model instances against
+ * one request trace, the inner loop of a simulator-guided placer (paper: Alg. 1 evaluates
+ * Phi(I', R_x) once per tentative instance list; the simulator is described in Sec. V-A
+ * "Simulator Implementation", the distributor in Sec. IV-F, the profiler model in
+ * Sec. IV-B Eq. 1).  Everything runs in CUDA kernels on one GPU; there is no CPU fallback.
+ *
+ * Conventions
+ *   - All times are int64 microseconds.  All results are integers; the same inputs give
+ *     byte-identical outputs whatever the launch shape, stream or mapping.
+ *   - "host" / "device" below says where a pointer must live.  The caller owns every
+ *     buffer it passes; the library copies what it keeps (profile, trace) and never frees
+ *     or retains caller memory beyond the stream work of the call.
+ *   - Every function returns 0 on success or a negative MAASO_E* code; maaso_strerror()
+ *     gives a text.  Nothing throws, aborts or traps.  A bad *candidate* never fails a
+ *     call: its record carries a non-zero `status` (MAASO_CAND_*) and zeroed statistics.
+ *   - Calls on one context are not thread-safe.  maaso_eval_placements / maaso_topk only
+ *     enqueue work on the given stream; outputs are valid once that stream is synchronised.
+ *     Successive calls on one context share its scratch memory, so their device work must
+ *     not overlap: use one stream, or synchronise between calls on different streams.
+ */
+#ifndef MAASO_H
+#define MAASO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define MAASO_API __attribute__((visibility("default")))
+#else
+#define MAASO_API
+#endif
+
+#define MAASO_WMAX 64           /* largest batch cap; latency tables have this many columns */
+#define MAASO_MAX_INSTANCES 128 /* most instances in one candidate */
+#define MAASO_MAX_MODELS 16
+#define MAASO_MAX_STRATEGIES 256
+#define MAASO_MAX_ROWS 256      /* n_models * n_strategies */
+#define MAASO_MAX_CLASSES 256
+#define MAASO_MAX_STEP_US (1 << 30)
+#define MAASO_MAX_TOPK 1024
+
+/* return codes */
+#define MAASO_OK 0
+#define MAASO_EINVAL (-1) /* null pointer, size or range violation, unsorted trace, unknown model/class */
+#define MAASO_ESTATE (-2) /* profile not loaded, trace belongs to another context, ... */
+#define MAASO_ENOMEM (-3)
+#define MAASO_ECUDA (-4)  /* a CUDA runtime call failed; text via maaso_last_error() */
+
+/* per-candidate status bits (maaso_result.status) */
+#define MAASO_CAND_EBUDGET 1u   /* devices used exceed the budget: constraint (c), Sec. IV-C */
+#define MAASO_CAND_EMEMFIT 2u   /* an instance has fewer devices than its model needs: constraint (d) */
+#define MAASO_CAND_ETOOMANY 4u  /* more than MAASO_MAX_INSTANCES instances */
+#define MAASO_CAND_EBADINST 8u  /* unknown model/strategy, batch cap outside 1..64, reserved bits set */
+#define MAASO_CAND_ETIMEOUT 16u /* a bounded device-side wait ran out; the candidate was not scored */
+#define MAASO_CAND_ELOOP 32u    /* more than 2 + 128*64 distributor attempts for one request */
+
+/* maaso_eval_opts.flags */
+#define MAASO_FLAG_PRED_OPTIMISTIC 1u /* distributor predicts with the step time right after admission
+                                         instead of the worst case F(M,P,B_I) of Sec. IV-F step 3 */
+
+/* maaso_eval_opts.mapping */
+#define MAASO_MAP_AUTO 0u  /* lanes-per-instance groups for <= 32 instances, one block otherwise */
+#define MAASO_MAP_BLOCK 1u /* one thread block per candidate, one warp per instance, lanes = slots */
+#define MAASO_MAP_GROUP 2u /* same as AUTO */
+
+typedef struct maaso_ctx maaso_ctx;
+typedef struct maaso_trace maaso_trace;
+
+/* One request of the trace (16 bytes).  Requests are sorted by arrival; equal arrivals
+ * are served in index order.  out_tokens >= 1 (S_r, the decode length of Sec. IV-C). */
+typedef struct {
+    int64_t arrival_us;
+    uint32_t in_tokens;
+    uint16_t out_tokens;
+    uint8_t cls;   /* index into the SLO class table */
+    uint8_t model; /* which model the request is for */
+} maaso_request;
+
+/* One SLO class; a negative limit means "no limit".  The deadline tau_r = d_r*theta_r*theta
+ * of Sec. III-C is the tbt term: finish - first_token <= (S-1) * tbt_us. */
+typedef struct {
+    int64_t ttft_us; /* first token - arrival */
+    int64_t tbt_us;  /* mean time between tokens */
+    int64_t e2e_us;  /* finish - arrival */
+} maaso_slo_class;
+
+/* Latency tables, all host pointers, int32, copied by maaso_load_profile.
+ * Row (m, s) = model m under parallelism strategy s. */
+typedef struct {
+    uint32_t n_models;     /* 1..MAASO_MAX_MODELS */
+    uint32_t n_strategies; /* 1..MAASO_MAX_STRATEGIES, n_models*n_strategies <= MAASO_MAX_ROWS */
+    uint32_t wmax;         /* must be MAASO_WMAX */
+    const int32_t *devices;         /* [S]  N(P): devices one instance occupies, >= 1 */
+    const int32_t *min_devices;     /* [M]  fewest devices a model fits in */
+    const int32_t *prefill_base_us; /* [M][S] >= 0 */
+    const int32_t *prefill_q16;     /* [M][S] >= 0, microseconds per input token in Q16 */
+    const int32_t *step_us;         /* [M][S][wmax]: one decode step with w running requests is
+                                       entry w-1, 1..MAASO_MAX_STEP_US (Eq. 1 as a table:
+                                       step = 1 / F(M,P,B,W) at W = w <= B) */
+} maaso_profile_desc;
+
+/* A batch of candidates in CSR form; device pointers (host pointers for the *_host call).
+ * inst word: bits 0-3 model, 4-11 strategy, 12-19 batch cap B, 20-31 zero.
+ * class_mask (may be NULL): bit k set = requests of class k belong to the request subset
+ * this placement is scored on (sub-cluster mapping, Sec. IV-F step 1); ignored when the
+ * trace has more than 32 classes. */
+typedef struct {
+    const uint32_t *offsets;    /* [n_cand + 1], offsets[0] = 0, non-decreasing */
+    const uint32_t *inst;       /* [n_inst] */
+    const uint32_t *class_mask; /* [n_cand] or NULL */
+    uint64_t n_cand;
+    uint64_t n_inst;            /* = offsets[n_cand] */
+    uint32_t budget;            /* modeled devices available, N(G) */
+    uint32_t reserved;
+} maaso_cand_batch;
+
+/* Options; NULL means all zero.  The dump buffers (device, each [dump_n][n_requests], any
+ * may be NULL) receive per-request times for the candidates listed in dump_cand_idx
+ * (device, [dump_n], distinct): finish time, first-token time, serving instance;
+ * -1 = rejected, -2 = not counted (masked out, or the candidate is invalid). */
+typedef struct {
+    uint32_t flags;
+    uint32_t mapping;
+    uint32_t dump_n;
+    uint32_t reserved;
+    const uint32_t *dump_cand_idx;
+    int64_t *dump_finish_us;
+    int64_t *dump_first_us;
+    int32_t *dump_inst;
+} maaso_eval_opts;
+
+/* Per-candidate result (128 bytes).  Statistics are over served requests unless noted. */
+typedef struct {
+    uint32_t status;      /* 0 = scored */
+    uint32_t n_counted;   /* requests of the subset (after class_mask) */
+    uint32_t n_served;
+    uint32_t n_hit;       /* Phi_S: served within every limit of their class */
+    uint32_t n_rejected;  /* blocked by overflow protection; count as SLO misses */
+    uint32_t n_cascade;   /* admitted as feasible but finished late (cascaded timeout, Sec. III-B) */
+    uint32_t hit_by_class[8]; /* classes >= 7 share the last bin */
+    int64_t sum_ttft_us, max_ttft_us; /* response latency = time to first token (Sec. V-A) */
+    int64_t sum_e2e_us, max_e2e_us;
+    int64_t makespan_us;  /* last completion time */
+    uint64_t tokens_out;  /* decode throughput = tokens_out / makespan */
+    uint64_t checksum;    /* order-independent hash of (request, instance, first token, finish) */
+    uint64_t attempts;    /* distributor attempts over all counted requests */
+    uint64_t reserved;
+} maaso_result;
+
+/* Create / destroy a context bound to one CUDA device.  maaso_destroy frees the profile,
+ * every trace loaded through the context and its scratch memory. */
+MAASO_API int maaso_create(maaso_ctx **out, int cuda_device);
+MAASO_API void maaso_destroy(maaso_ctx *ctx);
+
+/* Copy and validate the latency tables (profiler output, Sec. IV-B).  Replaces any earlier
+ * profile; traces loaded before stay valid only if n_models did not shrink below their
+ * largest model index (checked at eval).  Synchronous. */
+MAASO_API int maaso_load_profile(maaso_ctx *ctx, const maaso_profile_desc *desc);
+
+/* Copy and validate a trace (R_x of Alg. 1) with its SLO class table.  `reqs` may be a host
+ * or a device pointer, `classes` is a host pointer.  Checks: n >= 0, n < 2^32, arrivals
+ * non-negative and non-decreasing, out_tokens >= 1, cls < n_classes, model < n_models of
+ * the loaded profile (MAASO_ESTATE if none).  Synchronous.  *out must be released with
+ * maaso_free_trace (or by maaso_destroy). */
+MAASO_API int maaso_load_trace(maaso_ctx *ctx, const maaso_request *reqs, uint64_t n,
+                     const maaso_slo_class *classes, uint32_t n_classes, maaso_trace **out);
+MAASO_API void maaso_free_trace(maaso_ctx *ctx, maaso_trace *trace);
+
+/* Score every candidate of `cands` (device pointers) against `trace`: replay the trace
+ * through the distributor (Sec. IV-F) and per-instance continuous batching with virtual
+ * slots (Sec. V-A), and write one record per candidate to out_results (device,
+ * [n_cand]).  Work is enqueued on `cuda_stream` (a cudaStream_t, NULL = default stream).
+ * The context's scratch memory grows on demand (this may allocate and synchronise on the
+ * first call or when a batch is larger than any before). */
+MAASO_API int maaso_eval_placements(maaso_ctx *ctx, const maaso_trace *trace, const maaso_cand_batch *cands,
+                          const maaso_eval_opts *opts, maaso_result *out_results, void *cuda_stream);
+
+/* Same scoring with HOST buffers: copies the candidate batch to the device, scores it,
+ * copies the records back into out_results (host, [n_cand]) and synchronises.  Dump
+ * buffers are not supported here (opts->dump_n must be 0). */
+MAASO_API int maaso_eval_placements_host(maaso_ctx *ctx, const maaso_trace *trace, const maaso_cand_batch *cands,
+                               const maaso_eval_opts *opts, maaso_result *out_results);
+
+/* Select the k best records (the "keep the best solution per GPU count" step of Alg. 1,
+ * and the argmax of a sweep).  order 0: scored candidates before invalid ones; more n_hit first; then lower
+ * mean time to first token, sum_ttft_us / n_served compared exactly by 128-bit
+ * cross-multiplication (a candidate that served nothing ranks after one that served
+ * something); then lower index.  out_idx (device, [k]) gets candidate indices, best
+ * first, padded with 0xFFFFFFFF when k > n_cand; out_res (device, [k], may be NULL) the
+ * matching records (zeroed padding).  k <= MAASO_MAX_TOPK.  Enqueued on cuda_stream. */
+MAASO_API int maaso_topk(maaso_ctx *ctx, const maaso_result *results, uint64_t n_cand, uint32_t k,
+               uint32_t order, uint32_t *out_idx, maaso_result *out_res, void *cuda_stream);
+
+/* Number of kernels this context has launched so far (for accounting in benchmarks). */
+MAASO_API uint64_t maaso_launch_count(const maaso_ctx *ctx);
+
+/* Text for a return code; for MAASO_ECUDA the context keeps the CUDA error string. */
+MAASO_API const char *maaso_strerror(int code);
+MAASO_API const char *maaso_last_error(const maaso_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MAASO_H */

@@ -1,0 +1,22 @@
+"""B200-native scoring of candidate model-instance placements by trace replay.
+
+Thin Python binding over the C ABI in include/maaso.h (libmaaso.so, CUDA kernels for
+sm_100a).  The binding only marshals arguments: every step of the computation runs in the
+library's kernels.  Importing this package fails loudly if the library cannot be loaded.
+"""
+from .binding import (
+    MaasoError, Context, Trace,
+    maaso_create, maaso_destroy, maaso_load_profile, maaso_load_trace, maaso_free_trace,
+    maaso_eval_placements, maaso_eval_placements_host, maaso_topk, maaso_launch_count,
+    maaso_strerror, maaso_last_error, lib_path,
+    REQUEST_DTYPE, SLO_DTYPE, RESULT_DTYPE,
+    FLAG_PRED_OPTIMISTIC, MAP_AUTO, MAP_BLOCK, MAP_GROUP, CAND_STATUS,
+)
+
+__all__ = [
+    "MaasoError", "Context", "Trace", "maaso_create", "maaso_destroy", "maaso_load_profile",
+    "maaso_load_trace", "maaso_free_trace", "maaso_eval_placements", "maaso_eval_placements_host",
+    "maaso_topk", "maaso_launch_count", "maaso_strerror", "maaso_last_error", "lib_path",
+    "REQUEST_DTYPE", "SLO_DTYPE", "RESULT_DTYPE", "FLAG_PRED_OPTIMISTIC", "MAP_AUTO", "MAP_BLOCK",
+    "MAP_GROUP", "CAND_STATUS",
+]

@@ -1,0 +1,290 @@
+"""ctypes binding of libmaaso.so: same names as the C entry points, marshalling only.
+
+Device buffers are torch tensors (torch is used for device memory and streams, nothing
+else); host buffers are numpy arrays.  There is no CPU path: if the shared library is
+missing it is built with nvcc, and if that fails the import raises.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+REQUEST_DTYPE = np.dtype([("arrival_us", "<i8"), ("in_tokens", "<u4"), ("out_tokens", "<u2"),
+                          ("cls", "u1"), ("model", "u1")])
+SLO_DTYPE = np.dtype([("ttft_us", "<i8"), ("tbt_us", "<i8"), ("e2e_us", "<i8")])
+RESULT_DTYPE = np.dtype([
+    ("status", "<u4"), ("n_counted", "<u4"), ("n_served", "<u4"), ("n_hit", "<u4"),
+    ("n_rejected", "<u4"), ("n_cascade", "<u4"), ("hit_by_class", "<u4", (8,)),
+    ("sum_ttft_us", "<i8"), ("max_ttft_us", "<i8"), ("sum_e2e_us", "<i8"), ("max_e2e_us", "<i8"),
+    ("makespan_us", "<i8"), ("tokens_out", "<u8"), ("checksum", "<u8"), ("attempts", "<u8"),
+    ("reserved", "<u8")])
+assert REQUEST_DTYPE.itemsize == 16 and SLO_DTYPE.itemsize == 24 and RESULT_DTYPE.itemsize == 128
+
+FLAG_PRED_OPTIMISTIC = 1
+MAP_AUTO, MAP_BLOCK, MAP_GROUP = 0, 1, 2
+CAND_STATUS = {"EBUDGET": 1, "EMEMFIT": 2, "ETOOMANY": 4, "EBADINST": 8, "ETIMEOUT": 16, "ELOOP": 32}
+
+
+class MaasoError(RuntimeError):
+    def __init__(self, code, where, detail=""):
+        self.code = code
+        super().__init__(f"{where}: {maaso_strerror(code)} ({code}) {detail}".strip())
+
+
+class _ProfileDesc(C.Structure):
+    _fields_ = [("n_models", C.c_uint32), ("n_strategies", C.c_uint32), ("wmax", C.c_uint32),
+                ("devices", C.c_void_p), ("min_devices", C.c_void_p), ("prefill_base_us", C.c_void_p),
+                ("prefill_q16", C.c_void_p), ("step_us", C.c_void_p)]
+
+
+class _CandBatch(C.Structure):
+    _fields_ = [("offsets", C.c_void_p), ("inst", C.c_void_p), ("class_mask", C.c_void_p),
+                ("n_cand", C.c_uint64), ("n_inst", C.c_uint64), ("budget", C.c_uint32),
+                ("reserved", C.c_uint32)]
+
+
+class _EvalOpts(C.Structure):
+    _fields_ = [("flags", C.c_uint32), ("mapping", C.c_uint32), ("dump_n", C.c_uint32),
+                ("reserved", C.c_uint32), ("dump_cand_idx", C.c_void_p), ("dump_finish_us", C.c_void_p),
+                ("dump_first_us", C.c_void_p), ("dump_inst", C.c_void_p)]
+
+
+def lib_path():
+    return _build.LIB
+
+
+def _load():
+    path = _build.LIB
+    if not os.path.exists(path) or _build.stale():
+        path = _build.build()          # raises if nvcc is missing or the build fails
+    lib = C.CDLL(path)
+    vp, u64, u32 = C.c_void_p, C.c_uint64, C.c_uint32
+    lib.maaso_create.argtypes = [C.POINTER(vp), C.c_int]
+    lib.maaso_destroy.argtypes = [vp]
+    lib.maaso_destroy.restype = None
+    lib.maaso_load_profile.argtypes = [vp, C.POINTER(_ProfileDesc)]
+    lib.maaso_load_trace.argtypes = [vp, vp, u64, vp, u32, C.POINTER(vp)]
+    lib.maaso_free_trace.argtypes = [vp, vp]
+    lib.maaso_free_trace.restype = None
+    lib.maaso_eval_placements.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp, vp]
+    lib.maaso_eval_placements_host.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp]
+    lib.maaso_topk.argtypes = [vp, vp, u64, u32, u32, vp, vp, vp]
+    lib.maaso_launch_count.argtypes = [vp]
+    lib.maaso_launch_count.restype = u64
+    lib.maaso_strerror.argtypes = [C.c_int]
+    lib.maaso_strerror.restype = C.c_char_p
+    lib.maaso_last_error.argtypes = [vp]
+    lib.maaso_last_error.restype = C.c_char_p
+    for name in ("maaso_create", "maaso_load_profile", "maaso_load_trace", "maaso_eval_placements",
+                 "maaso_eval_placements_host", "maaso_topk"):
+        getattr(lib, name).restype = C.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def maaso_strerror(code):
+    return _lib.maaso_strerror(int(code)).decode()
+
+
+def maaso_last_error(ctx):
+    return _lib.maaso_last_error(ctx).decode()
+
+
+def _check(rc, where, ctx=None):
+    if rc != 0:
+        raise MaasoError(rc, where, maaso_last_error(ctx) if ctx else "")
+
+
+def _ptr(x):
+    """device pointer of a torch tensor, host pointer of a numpy array, or NULL"""
+    if x is None:
+        return None
+    if isinstance(x, np.ndarray):
+        assert x.flags["C_CONTIGUOUS"]
+        return x.ctypes.data
+    assert x.is_contiguous()
+    return x.data_ptr()
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return getattr(stream, "cuda_stream", stream)
+
+
+# ---- entry points, one per C function ---------------------------------------------------------
+def maaso_create(cuda_device=0):
+    ctx = C.c_void_p()
+    _check(_lib.maaso_create(C.byref(ctx), int(cuda_device)), "maaso_create")
+    return ctx
+
+
+def maaso_destroy(ctx):
+    _lib.maaso_destroy(ctx)
+
+
+def maaso_load_profile(ctx, profile):
+    """profile: dict with n_models, n_strategies, wmax and the int32 tables (host arrays)."""
+    keep = {k: np.ascontiguousarray(profile[k], dtype=np.int32)
+            for k in ("devices", "min_devices", "prefill_base_us", "prefill_q16", "step_us")}
+    M, S, W = int(profile["n_models"]), int(profile["n_strategies"]), int(profile["wmax"])
+    if keep["devices"].size != S or keep["min_devices"].size != M or \
+            keep["prefill_base_us"].size != M * S or keep["prefill_q16"].size != M * S or \
+            keep["step_us"].size != M * S * W:
+        raise MaasoError(-1, "maaso_load_profile", "table sizes do not match n_models/n_strategies/wmax")
+    d = _ProfileDesc(M, S, W, *(keep[k].ctypes.data for k in
+                               ("devices", "min_devices", "prefill_base_us", "prefill_q16", "step_us")))
+    _check(_lib.maaso_load_profile(ctx, C.byref(d)), "maaso_load_profile", ctx)
+
+
+def maaso_load_trace(ctx, reqs, classes):
+    """reqs: numpy array of REQUEST_DTYPE (host) or a torch uint8 CUDA tensor of 16-byte records;
+    classes: numpy array of SLO_DTYPE (host).  Returns the trace handle."""
+    classes = np.ascontiguousarray(classes, dtype=SLO_DTYPE)
+    if isinstance(reqs, np.ndarray):
+        reqs = np.ascontiguousarray(reqs, dtype=REQUEST_DTYPE)
+        n = len(reqs)
+    else:
+        assert reqs.dtype.itemsize == 1 and reqs.numel() % 16 == 0
+        n = reqs.numel() // 16
+    out = C.c_void_p()
+    _check(_lib.maaso_load_trace(ctx, _ptr(reqs), n, classes.ctypes.data, len(classes), C.byref(out)),
+           "maaso_load_trace", ctx)
+    return out
+
+
+def maaso_free_trace(ctx, trace):
+    _lib.maaso_free_trace(ctx, trace)
+
+
+def _batch(offsets, inst, class_mask, budget):
+    n_cand = int(offsets.shape[0]) - 1
+    n_inst = int(inst.shape[0]) if inst is not None else 0
+    return _CandBatch(_ptr(offsets), _ptr(inst) if n_inst else None, _ptr(class_mask), n_cand, n_inst,
+                      int(budget), 0)
+
+
+def maaso_eval_placements(ctx, trace, offsets, inst, budget, out_results, class_mask=None, flags=0,
+                          mapping=MAP_AUTO, dump_cand_idx=None, dump_finish_us=None, dump_first_us=None,
+                          dump_inst=None, stream=None):
+    """All array arguments are CUDA tensors (int32 views of the uint32 words; out_results a
+    uint8 tensor of n_cand*128 bytes).  Work is enqueued on `stream` (default: torch's current)."""
+    b = _batch(offsets, inst, class_mask, budget)
+    o = _EvalOpts(int(flags), int(mapping), 0 if dump_cand_idx is None else int(dump_cand_idx.shape[0]), 0,
+                  _ptr(dump_cand_idx), _ptr(dump_finish_us), _ptr(dump_first_us), _ptr(dump_inst))
+    _check(_lib.maaso_eval_placements(ctx, trace, C.byref(b), C.byref(o), _ptr(out_results),
+                                      _stream_ptr(stream)), "maaso_eval_placements", ctx)
+
+
+def maaso_eval_placements_host(ctx, trace, offsets, inst, budget, out_results, class_mask=None, flags=0,
+                               mapping=MAP_AUTO):
+    """Host (numpy) buffers in and out; copies happen inside the call, which synchronises."""
+    b = _batch(offsets, inst, class_mask, budget)
+    o = _EvalOpts(int(flags), int(mapping), 0, 0, None, None, None, None)
+    _check(_lib.maaso_eval_placements_host(ctx, trace, C.byref(b), C.byref(o), _ptr(out_results)),
+           "maaso_eval_placements_host", ctx)
+
+
+def maaso_topk(ctx, results, n_cand, k, out_idx, out_res=None, order=0, stream=None):
+    _check(_lib.maaso_topk(ctx, _ptr(results), int(n_cand), int(k), int(order), _ptr(out_idx), _ptr(out_res),
+                           _stream_ptr(stream)), "maaso_topk", ctx)
+
+
+def maaso_launch_count(ctx):
+    return int(_lib.maaso_launch_count(ctx))
+
+
+# ---- convenience wrappers (allocation of outputs only) -------------------------------------------
+class Trace:
+    def __init__(self, ctx, handle, n):
+        self.ctx, self.handle, self.n = ctx, handle, n
+
+
+class Context:
+    """Owns a library context on one CUDA device; allocates output tensors for the calls."""
+
+    def __init__(self, device=0):
+        import torch
+        self.torch = torch
+        self.device = torch.device("cuda", device)
+        self.handle = maaso_create(device)
+
+    def close(self):
+        if self.handle is not None:
+            maaso_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def load_profile(self, profile):
+        maaso_load_profile(self.handle, profile)
+
+    def load_trace(self, reqs, classes):
+        n = len(reqs) if isinstance(reqs, np.ndarray) else reqs.numel() // 16
+        return Trace(self, maaso_load_trace(self.handle, reqs, classes), n)
+
+    def free_trace(self, trace):
+        maaso_free_trace(self.handle, trace.handle)
+        trace.handle = None
+
+    def to_device(self, words):
+        """uint32 numpy words -> int32 CUDA tensor with the same bits"""
+        t = self.torch.from_numpy(np.ascontiguousarray(words, dtype=np.uint32).view(np.int32))
+        return t.to(self.device)
+
+    def eval_placements(self, trace, offsets, inst, budget, class_mask=None, flags=0, mapping=MAP_AUTO,
+                        dump_idx=None, out=None, stream=None):
+        """offsets / inst / class_mask: CUDA int32 tensors (see to_device).  Returns the uint8
+        result tensor [n_cand, 128] and, if dump_idx is given, a dict of dump tensors."""
+        torch = self.torch
+        n_cand = int(offsets.shape[0]) - 1
+        if out is None:
+            out = torch.empty((n_cand, 128), dtype=torch.uint8, device=self.device)
+        dumps = None
+        kw = {}
+        if dump_idx is not None:
+            d = self.to_device(np.asarray(dump_idx, dtype=np.uint32))
+            dumps = {"finish_us": torch.empty((len(dump_idx), trace.n), dtype=torch.int64, device=self.device),
+                     "first_us": torch.empty((len(dump_idx), trace.n), dtype=torch.int64, device=self.device),
+                     "inst": torch.empty((len(dump_idx), trace.n), dtype=torch.int32, device=self.device)}
+            kw = dict(dump_cand_idx=d, dump_finish_us=dumps["finish_us"], dump_first_us=dumps["first_us"],
+                      dump_inst=dumps["inst"])
+        maaso_eval_placements(self.handle, trace.handle, offsets, inst, budget, out, class_mask, flags,
+                              mapping, stream=stream, **kw)
+        return (out, dumps) if dump_idx is not None else out
+
+    def eval_placements_host(self, trace, offsets, inst, budget, class_mask=None, flags=0,
+                             mapping=MAP_AUTO, out=None):
+        offsets = np.ascontiguousarray(offsets, dtype=np.uint32)
+        inst = np.ascontiguousarray(inst, dtype=np.uint32)
+        if class_mask is not None:
+            class_mask = np.ascontiguousarray(class_mask, dtype=np.uint32)
+        if out is None:
+            out = np.empty(len(offsets) - 1, dtype=RESULT_DTYPE)
+        maaso_eval_placements_host(self.handle, trace.handle, offsets, inst, budget, out, class_mask,
+                                   flags, mapping)
+        return out
+
+    def topk(self, results, k, order=0, with_records=True, stream=None):
+        torch = self.torch
+        n_cand = int(results.shape[0])
+        idx = torch.empty(k, dtype=torch.int32, device=self.device)
+        rec = torch.empty((k, 128), dtype=torch.uint8, device=self.device) if with_records else None
+        maaso_topk(self.handle, results, n_cand, k, idx, rec, order, stream)
+        return idx, rec
+
+    def launch_count(self):
+        return maaso_launch_count(self.handle)
+
+    @staticmethod
+    def results_to_numpy(t):
+        return t.cpu().numpy().reshape(-1).view(RESULT_DTYPE)

@@ -1,0 +1,463 @@
+// C ABI of the placement-scoring library: handles, validation, host<->device copies and
+// kernel launches.  Semantics of every entry point are documented in include/maaso.h.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+namespace maaso {
+cudaError_t launch_prep(const EvalParams& P, const uint32_t* dump_idx, cudaStream_t stream, int* launches);
+cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, cudaStream_t stream);
+int occupancy_eval_group(const EvalParams& P, int tile_recs);
+cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
+int occupancy_eval_block(const EvalParams& P, int bucket, int tile_recs);
+size_t block_payload_per_cta(int bucket);
+size_t topk_scratch_bytes(uint64_t n_cand, uint32_t k);
+cudaError_t launch_topk(const maaso_result* results, uint64_t n_cand, uint32_t k, void* scratch,
+                        uint32_t* out_idx, maaso_result* out_res, cudaStream_t stream, int* launches);
+}  // namespace maaso
+
+using namespace maaso;
+
+struct maaso_trace {
+    maaso_ctx* owner;
+    uint4* d_reqs;
+    int64_t* d_classes;
+    uint64_t n;
+    uint32_t n_classes;
+    uint32_t max_model;
+};
+
+struct maaso_ctx {
+    int device;
+    int sm_count;
+    bool has_profile;
+    uint32_t n_models, n_strategies, n_rows;
+    int32_t* d_rows;
+    int32_t* d_devices;
+    int32_t* d_min_devices;
+    std::vector<maaso_trace*> traces;
+    void* scratch;
+    size_t scratch_bytes;
+    void* topk_scratch;
+    size_t topk_scratch_bytes;
+    // staging for the host-buffer entry point
+    void* stage;
+    size_t stage_bytes;
+    cudaStream_t own_stream;
+    uint64_t launches;
+    int tile_recs;
+    std::string last_error;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev;
+    bool ok;
+    explicit DeviceGuard(int dev) : prev(-1), ok(true) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+int cuda_fail(maaso_ctx* ctx, cudaError_t e, const char* what) {
+    if (ctx) ctx->last_error = std::string(what) + ": " + cudaGetErrorString(e);
+    cudaGetLastError();  // clear the sticky-free error state
+    return e == cudaErrorMemoryAllocation ? MAASO_ENOMEM : MAASO_ECUDA;
+}
+
+int fail(maaso_ctx* ctx, int code, const char* what) {
+    if (ctx) ctx->last_error = what;
+    return code;
+}
+
+int grow(maaso_ctx* ctx, void** buf, size_t* have, size_t need) {
+    if (need <= *have) return MAASO_OK;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "synchronize before growing scratch");
+    if (*buf) cudaFree(*buf);
+    *buf = nullptr;
+    *have = 0;
+    need = (need + (size_t)(1 << 20) - 1) & ~((size_t)(1 << 20) - 1);
+    e = cudaMalloc(buf, need);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "scratch allocation");
+    *have = need;
+    return MAASO_OK;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
+    if (!out) return MAASO_EINVAL;
+    *out = nullptr;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaGetDeviceCount");
+    if (cuda_device < 0 || cuda_device >= count) return MAASO_EINVAL;
+    maaso_ctx* ctx = new (std::nothrow) maaso_ctx();
+    if (!ctx) return MAASO_ENOMEM;
+    ctx->device = cuda_device;
+    ctx->has_profile = false;
+    ctx->d_rows = ctx->d_devices = ctx->d_min_devices = nullptr;
+    ctx->scratch = ctx->topk_scratch = ctx->stage = nullptr;
+    ctx->scratch_bytes = ctx->topk_scratch_bytes = ctx->stage_bytes = 0;
+    ctx->launches = 0;
+    ctx->tile_recs = 256;
+    ctx->own_stream = nullptr;
+    DeviceGuard g(cuda_device);
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, cuda_device);
+    if (e != cudaSuccess || !g.ok) {
+        delete ctx;
+        return cuda_fail(nullptr, e, "cudaGetDeviceProperties");
+    }
+    if (prop.major < 10) {  // the kernels are built for sm_100a only
+        delete ctx;
+        return MAASO_ESTATE;
+    }
+    ctx->sm_count = prop.multiProcessorCount;
+    e = cudaStreamCreateWithFlags(&ctx->own_stream, cudaStreamNonBlocking);
+    if (e != cudaSuccess) {
+        delete ctx;
+        return cuda_fail(nullptr, e, "cudaStreamCreate");
+    }
+    const char* env = getenv("MAASO_TILE_RECS");
+    if (env) {
+        int v = atoi(env);
+        if (v >= 16 && v <= 2048) ctx->tile_recs = v;
+    }
+    *out = ctx;
+    return MAASO_OK;
+}
+
+MAASO_API void maaso_free_trace(maaso_ctx* ctx, maaso_trace* trace) {
+    if (!ctx || !trace || trace->owner != ctx) return;
+    DeviceGuard g(ctx->device);
+    cudaDeviceSynchronize();
+    for (size_t i = 0; i < ctx->traces.size(); i++)
+        if (ctx->traces[i] == trace) {
+            ctx->traces.erase(ctx->traces.begin() + i);
+            break;
+        }
+    if (trace->d_reqs) cudaFree(trace->d_reqs);
+    if (trace->d_classes) cudaFree(trace->d_classes);
+    delete trace;
+}
+
+MAASO_API void maaso_destroy(maaso_ctx* ctx) {
+    if (!ctx) return;
+    DeviceGuard g(ctx->device);
+    cudaDeviceSynchronize();
+    while (!ctx->traces.empty()) maaso_free_trace(ctx, ctx->traces.back());
+    if (ctx->d_rows) cudaFree(ctx->d_rows);
+    if (ctx->d_devices) cudaFree(ctx->d_devices);
+    if (ctx->d_min_devices) cudaFree(ctx->d_min_devices);
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->topk_scratch) cudaFree(ctx->topk_scratch);
+    if (ctx->stage) cudaFree(ctx->stage);
+    if (ctx->own_stream) cudaStreamDestroy(ctx->own_stream);
+    delete ctx;
+}
+
+MAASO_API int maaso_load_profile(maaso_ctx* ctx, const maaso_profile_desc* d) {
+    if (!ctx || !d) return MAASO_EINVAL;
+    if (!d->devices || !d->min_devices || !d->prefill_base_us || !d->prefill_q16 || !d->step_us)
+        return fail(ctx, MAASO_EINVAL, "profile: null table");
+    if (d->n_models < 1 || d->n_models > MAASO_MAX_MODELS || d->n_strategies < 1 ||
+        d->n_strategies > MAASO_MAX_STRATEGIES || d->n_models * d->n_strategies > MAASO_MAX_ROWS ||
+        d->wmax != MAASO_WMAX)
+        return fail(ctx, MAASO_EINVAL, "profile: table shape out of range");
+    const uint32_t M = d->n_models, S = d->n_strategies, R = M * S;
+    for (uint32_t s = 0; s < S; s++)
+        if (d->devices[s] < 1) return fail(ctx, MAASO_EINVAL, "profile: devices[s] < 1");
+    for (uint32_t m = 0; m < M; m++)
+        if (d->min_devices[m] < 0) return fail(ctx, MAASO_EINVAL, "profile: min_devices[m] < 0");
+    std::vector<int32_t> rows((size_t)R * kRowStride);
+    for (uint32_t r = 0; r < R; r++) {
+        if (d->prefill_base_us[r] < 0 || d->prefill_q16[r] < 0)
+            return fail(ctx, MAASO_EINVAL, "profile: negative prefill cost");
+        rows[(size_t)r * kRowStride + 0] = d->prefill_base_us[r];
+        rows[(size_t)r * kRowStride + 1] = d->prefill_q16[r];
+        for (uint32_t w = 0; w < MAASO_WMAX; w++) {
+            const int32_t v = d->step_us[(size_t)r * MAASO_WMAX + w];
+            if (v < 1 || v > MAASO_MAX_STEP_US) return fail(ctx, MAASO_EINVAL, "profile: step_us out of range");
+            rows[(size_t)r * kRowStride + 2 + w] = v;
+        }
+    }
+    DeviceGuard g(ctx->device);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "synchronize");
+    if (ctx->d_rows) cudaFree(ctx->d_rows);
+    if (ctx->d_devices) cudaFree(ctx->d_devices);
+    if (ctx->d_min_devices) cudaFree(ctx->d_min_devices);
+    ctx->d_rows = ctx->d_devices = ctx->d_min_devices = nullptr;
+    ctx->has_profile = false;
+    if ((e = cudaMalloc(&ctx->d_rows, rows.size() * 4)) != cudaSuccess) return cuda_fail(ctx, e, "profile alloc");
+    if ((e = cudaMalloc(&ctx->d_devices, S * 4)) != cudaSuccess) return cuda_fail(ctx, e, "profile alloc");
+    if ((e = cudaMalloc(&ctx->d_min_devices, M * 4)) != cudaSuccess) return cuda_fail(ctx, e, "profile alloc");
+    if ((e = cudaMemcpy(ctx->d_rows, rows.data(), rows.size() * 4, cudaMemcpyHostToDevice)) != cudaSuccess ||
+        (e = cudaMemcpy(ctx->d_devices, d->devices, S * 4, cudaMemcpyHostToDevice)) != cudaSuccess ||
+        (e = cudaMemcpy(ctx->d_min_devices, d->min_devices, M * 4, cudaMemcpyHostToDevice)) != cudaSuccess)
+        return cuda_fail(ctx, e, "profile copy");
+    ctx->n_models = M;
+    ctx->n_strategies = S;
+    ctx->n_rows = R;
+    ctx->has_profile = true;
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64_t n, const maaso_slo_class* classes,
+                     uint32_t n_classes, maaso_trace** out) {
+    if (!ctx || !out) return MAASO_EINVAL;
+    *out = nullptr;
+    if (!ctx->has_profile) return fail(ctx, MAASO_ESTATE, "trace: load a profile first");
+    if ((!reqs && n) || !classes || n_classes < 1 || n_classes > MAASO_MAX_CLASSES || n >= 0xFFFFFFFFull)
+        return fail(ctx, MAASO_EINVAL, "trace: null pointer or size out of range");
+    const int64_t kLimMax = (int64_t)1 << 40;
+    std::vector<int64_t> cls((size_t)n_classes * 3);
+    for (uint32_t k = 0; k < n_classes; k++) {
+        const int64_t v[3] = {classes[k].ttft_us, classes[k].tbt_us, classes[k].e2e_us};
+        for (int j = 0; j < 3; j++) {
+            if (v[j] > kLimMax) return fail(ctx, MAASO_EINVAL, "trace: SLO limit above 2^40 us");
+            cls[(size_t)k * 3 + j] = v[j] < 0 ? -1 : v[j];
+        }
+    }
+    DeviceGuard g(ctx->device);
+    // the requests may live on the host or on the device; validate on a host copy
+    const maaso_request* host = reqs;
+    std::vector<maaso_request> tmp;
+    bool on_device = false;
+    if (n) {
+        cudaPointerAttributes attr;
+        cudaError_t pe = cudaPointerGetAttributes(&attr, reqs);
+        if (pe != cudaSuccess) cudaGetLastError();
+        on_device = pe == cudaSuccess && (attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged);
+        if (on_device) {
+            tmp.resize(n);
+            cudaError_t e = cudaMemcpy(tmp.data(), reqs, n * sizeof(maaso_request), cudaMemcpyDeviceToHost);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "trace copy to host");
+            host = tmp.data();
+        }
+    }
+    int64_t prev = 0;
+    uint32_t max_model = 0;
+    const int64_t kArrMax = (int64_t)1 << 50;
+    for (uint64_t r = 0; r < n; r++) {
+        const maaso_request& q = host[r];
+        if (q.arrival_us < prev || q.arrival_us > kArrMax)
+            return fail(ctx, MAASO_EINVAL, "trace: arrivals must be non-negative, non-decreasing, below 2^50");
+        prev = q.arrival_us;
+        if (q.out_tokens < 1) return fail(ctx, MAASO_EINVAL, "trace: out_tokens must be >= 1");
+        if (q.cls >= n_classes) return fail(ctx, MAASO_EINVAL, "trace: unknown SLO class");
+        if (q.model >= ctx->n_models) return fail(ctx, MAASO_EINVAL, "trace: unknown model");
+        if (q.model > max_model) max_model = q.model;
+    }
+    maaso_trace* t = new (std::nothrow) maaso_trace();
+    if (!t) return MAASO_ENOMEM;
+    t->owner = ctx;
+    t->d_reqs = nullptr;
+    t->d_classes = nullptr;
+    t->n = n;
+    t->n_classes = n_classes;
+    t->max_model = max_model;
+    cudaError_t e = cudaMalloc(&t->d_reqs, (n ? n : 1) * sizeof(maaso_request));
+    if (e == cudaSuccess) e = cudaMalloc(&t->d_classes, cls.size() * 8);
+    if (e == cudaSuccess && n)
+        e = cudaMemcpy(t->d_reqs, reqs, n * sizeof(maaso_request),
+                       on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(t->d_classes, cls.data(), cls.size() * 8, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        if (t->d_reqs) cudaFree(t->d_reqs);
+        if (t->d_classes) cudaFree(t->d_classes);
+        delete t;
+        return cuda_fail(ctx, e, "trace upload");
+    }
+    ctx->traces.push_back(t);
+    *out = t;
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, const maaso_cand_batch* cands,
+                          const maaso_eval_opts* opts, maaso_result* out_results, void* cuda_stream) {
+    if (!ctx || !trace || !cands) return MAASO_EINVAL;
+    if (!ctx->has_profile) return fail(ctx, MAASO_ESTATE, "eval: no profile loaded");
+    if (trace->owner != ctx) return fail(ctx, MAASO_ESTATE, "eval: trace belongs to another context");
+    if (trace->n && trace->max_model >= ctx->n_models)
+        return fail(ctx, MAASO_ESTATE, "eval: trace refers to a model the current profile lacks");
+    if (cands->n_cand == 0) return MAASO_OK;
+    if (!cands->offsets || !out_results || (cands->n_inst && !cands->inst) || cands->n_cand >= 0xFFFFFFFFull ||
+        cands->n_inst >= 0xFFFFFFFFull)
+        return fail(ctx, MAASO_EINVAL, "eval: null pointer or size out of range");
+    maaso_eval_opts o;
+    memset(&o, 0, sizeof(o));
+    if (opts) o = *opts;
+    if (o.mapping > MAASO_MAP_GROUP) return fail(ctx, MAASO_EINVAL, "eval: unknown mapping");
+    if (o.dump_n && !o.dump_cand_idx) return fail(ctx, MAASO_EINVAL, "eval: dump_n without dump_cand_idx");
+    if (o.flags & ~MAASO_FLAG_PRED_OPTIMISTIC) return fail(ctx, MAASO_EINVAL, "eval: unknown flag");
+
+    DeviceGuard g(ctx->device);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const uint32_t C = (uint32_t)cands->n_cand;
+    const int tile = ctx->tile_recs;
+
+    EvalParams P;
+    memset(&P, 0, sizeof(P));
+    P.reqs = trace->d_reqs;
+    P.n_req = (uint32_t)trace->n;
+    P.n_classes = trace->n_classes;
+    P.classes = trace->d_classes;
+    P.rows = ctx->d_rows;
+    P.devices = ctx->d_devices;
+    P.min_devices = ctx->d_min_devices;
+    P.n_rows = ctx->n_rows;
+    P.n_models = ctx->n_models;
+    P.n_strategies = ctx->n_strategies;
+    P.budget = cands->budget;
+    P.offsets = cands->offsets;
+    P.inst = cands->inst;
+    P.class_mask = cands->class_mask;
+    P.n_cand = C;
+    P.n_inst = (uint32_t)cands->n_inst;
+    P.flags = o.flags;
+    P.mapping = o.mapping;
+    P.out = out_results;
+    P.dump_n = o.dump_n;
+    P.dump_finish = o.dump_finish_us;
+    P.dump_first = o.dump_first_us;
+    P.dump_inst = o.dump_inst;
+
+    // launch shapes: persistent grids bounded by what the batch can use
+    const int occ_g = occupancy_eval_group(P, tile);
+    int grid_g = ctx->sm_count * occ_g;
+    const uint64_t max_items_g = (uint64_t)C / 4 + 6;  // at most one work item per 4 candidates + bucket tails
+    if ((uint64_t)grid_g > max_items_g) grid_g = (int)max_items_g;
+    int grid_b[3];
+    size_t pay_entries = (size_t)grid_g * kGroupThreads * MAASO_WMAX;
+    for (int b = 6; b <= 8; b++) {
+        // without the block mapping only candidates with more than 32 instances go to a block kernel
+        const bool used = o.mapping == MAASO_MAP_BLOCK || (b == 8 && cands->n_inst > 32);
+        grid_b[b - 6] = 0;
+        if (!used) continue;
+        int gb = ctx->sm_count * occupancy_eval_block(P, b, tile);
+        if ((uint64_t)gb > C) gb = (int)C;
+        grid_b[b - 6] = gb;
+        const size_t need = (size_t)gb * block_payload_per_cta(b);
+        if (need > pay_entries) pay_entries = need;
+    }
+
+    // scratch layout: counters | bucket lists | dump rows | payload
+    size_t off = 0;
+    const size_t off_counters = off; off = align_up(off + 64 * 4, 256);
+    const size_t off_lists = off;    off = align_up(off + (size_t)kNumBuckets * C * 4, 256);
+    const size_t off_dump = off;     off = align_up(off + (o.dump_n ? (size_t)C * 4 : 0), 256);
+    const size_t off_pay = off;      off = align_up(off + pay_entries * sizeof(Payload), 256);
+    int rc = grow(ctx, &ctx->scratch, &ctx->scratch_bytes, off);
+    if (rc != MAASO_OK) return rc;
+    unsigned char* sb = static_cast<unsigned char*>(ctx->scratch);
+    P.bucket_count = reinterpret_cast<uint32_t*>(sb + off_counters);
+    P.work_ctr = P.bucket_count + 16;
+    P.bucket_list = reinterpret_cast<uint32_t*>(sb + off_lists);
+    P.dump_row = o.dump_n ? reinterpret_cast<int32_t*>(sb + off_dump) : nullptr;
+    P.payload = reinterpret_cast<Payload*>(sb + off_pay);
+
+    cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, 64 * 4, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "memset");
+    int launches = 0;
+    e = launch_prep(P, o.dump_cand_idx, stream, &launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "prep launch");
+    if (o.mapping != MAASO_MAP_BLOCK) {
+        e = launch_eval_group(P, grid_g, tile, stream);
+        launches++;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "group kernel launch");
+    }
+    for (int b = 6; b <= 8; b++) {
+        if (grid_b[b - 6] == 0) continue;
+        e = launch_eval_block(P, b, grid_b[b - 6], tile, stream);
+        launches++;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "block kernel launch");
+    }
+    ctx->launches += (uint64_t)launches;
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_eval_placements_host(maaso_ctx* ctx, const maaso_trace* trace, const maaso_cand_batch* cands,
+                               const maaso_eval_opts* opts, maaso_result* out_results) {
+    if (!ctx || !trace || !cands) return MAASO_EINVAL;
+    if (opts && opts->dump_n) return fail(ctx, MAASO_EINVAL, "eval_host: dump buffers are not supported");
+    if (cands->n_cand == 0) return MAASO_OK;
+    if (!cands->offsets || !out_results || (cands->n_inst && !cands->inst) || cands->n_cand >= 0xFFFFFFFFull ||
+        cands->n_inst >= 0xFFFFFFFFull)
+        return fail(ctx, MAASO_EINVAL, "eval_host: null pointer or size out of range");
+    DeviceGuard g(ctx->device);
+    const size_t C = cands->n_cand, NI = cands->n_inst;
+    size_t off = 0;
+    const size_t o_off = off; off = align_up(off + (C + 1) * 4, 256);
+    const size_t o_inst = off; off = align_up(off + (NI ? NI : 1) * 4, 256);
+    const size_t o_mask = off; off = align_up(off + C * 4, 256);
+    const size_t o_res = off;  off = align_up(off + C * sizeof(maaso_result), 256);
+    int rc = grow(ctx, &ctx->stage, &ctx->stage_bytes, off);
+    if (rc != MAASO_OK) return rc;
+    unsigned char* sb = static_cast<unsigned char*>(ctx->stage);
+    cudaStream_t st = ctx->own_stream;
+    cudaError_t e = cudaMemcpyAsync(sb + o_off, cands->offsets, (C + 1) * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && NI) e = cudaMemcpyAsync(sb + o_inst, cands->inst, NI * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && cands->class_mask)
+        e = cudaMemcpyAsync(sb + o_mask, cands->class_mask, C * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "eval_host: upload");
+    maaso_cand_batch dev = *cands;
+    dev.offsets = reinterpret_cast<const uint32_t*>(sb + o_off);
+    dev.inst = reinterpret_cast<const uint32_t*>(sb + o_inst);
+    dev.class_mask = cands->class_mask ? reinterpret_cast<const uint32_t*>(sb + o_mask) : nullptr;
+    rc = maaso_eval_placements(ctx, trace, &dev, opts, reinterpret_cast<maaso_result*>(sb + o_res), st);
+    if (rc != MAASO_OK) return rc;
+    e = cudaMemcpyAsync(out_results, sb + o_res, C * sizeof(maaso_result), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "eval_host: download");
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_topk(maaso_ctx* ctx, const maaso_result* results, uint64_t n_cand, uint32_t k, uint32_t order,
+               uint32_t* out_idx, maaso_result* out_res, void* cuda_stream) {
+    if (!ctx) return MAASO_EINVAL;
+    if (k == 0) return MAASO_OK;
+    if (!out_idx || (!results && n_cand) || k > MAASO_MAX_TOPK || order != 0 || n_cand >= 0xFFFFFFFFull)
+        return fail(ctx, MAASO_EINVAL, "topk: null pointer, k or order out of range");
+    DeviceGuard g(ctx->device);
+    int rc = grow(ctx, &ctx->topk_scratch, &ctx->topk_scratch_bytes, topk_scratch_bytes(n_cand, k));
+    if (rc != MAASO_OK) return rc;
+    int launches = 0;
+    cudaError_t e = launch_topk(results, n_cand, k, ctx->topk_scratch, out_idx, out_res,
+                                (cudaStream_t)cuda_stream, &launches);
+    ctx->launches += (uint64_t)launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "topk launch");
+    return MAASO_OK;
+}
+
+MAASO_API uint64_t maaso_launch_count(const maaso_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+MAASO_API const char* maaso_strerror(int code) {
+    switch (code) {
+        case MAASO_OK: return "ok";
+        case MAASO_EINVAL: return "invalid argument";
+        case MAASO_ESTATE: return "wrong state (no profile, foreign trace, unsupported device)";
+        case MAASO_ENOMEM: return "out of memory";
+        case MAASO_ECUDA: return "CUDA runtime error";
+        default: return "unknown error";
+    }
+}
+
+MAASO_API const char* maaso_last_error(const maaso_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+}  // extern "C"

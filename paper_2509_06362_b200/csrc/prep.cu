@@ -1,0 +1,81 @@
+// Candidate decode + validation (constraints (c) and (d) of Sec. IV-C, table ranges) and
+// sorting of valid candidates into launch buckets; helpers for the per-request dump buffers.
+#include "common.cuh"
+
+namespace maaso {
+
+__global__ void prep_kernel(const EvalParams P) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= P.n_cand) return;
+    const uint32_t lo = P.offsets[c], hi = P.offsets[c + 1];
+    uint32_t status = 0, n = 0;
+    if (hi < lo || hi > P.n_inst) {
+        status = MAASO_CAND_EBADINST;  // malformed CSR row
+    } else {
+        n = hi - lo;
+        if (n > MAASO_MAX_INSTANCES) {
+            status = MAASO_CAND_ETOOMANY;
+        } else {
+            uint64_t devsum = 0;
+            for (uint32_t i = 0; i < n; i++) {
+                const uint32_t word = P.inst[lo + i];
+                const uint32_t m = word & 0xFu, s = (word >> 4) & 0xFFu, b = (word >> 12) & 0xFFu;
+                if ((word >> 20) != 0 || m >= P.n_models || s >= P.n_strategies || b < 1 || b > MAASO_WMAX) {
+                    status |= MAASO_CAND_EBADINST;
+                    continue;
+                }
+                devsum += (uint64_t)P.devices[s];
+                if (P.devices[s] < P.min_devices[m]) status |= MAASO_CAND_EMEMFIT;
+            }
+            if (devsum > P.budget) status |= MAASO_CAND_EBUDGET;
+        }
+    }
+    if (P.dump_row) P.dump_row[c] = -1;
+    if (status) {
+        uint4* o = reinterpret_cast<uint4*>(P.out + c);
+        o[0] = make_uint4(status, 0, 0, 0);
+        for (int i = 1; i < 8; i++) o[i] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    int b;
+    if (P.mapping == MAASO_MAP_BLOCK) b = n <= 2 ? 6 : (n <= 8 ? 7 : 8);
+    else if (n <= 32) b = n <= 1 ? 0 : 32 - __clz((int)(n - 1));
+    else b = 8;
+    const uint32_t pos = atomicAdd(&P.bucket_count[b], 1u);
+    P.bucket_list[(size_t)b * P.n_cand + pos] = c;
+}
+
+__global__ void dump_map_kernel(const EvalParams P, const uint32_t* dump_idx) {
+    const uint32_t d = blockIdx.x * blockDim.x + threadIdx.x;
+    if (d >= P.dump_n) return;
+    const uint32_t c = dump_idx[d];
+    if (c < P.n_cand) P.dump_row[c] = (int32_t)d;
+}
+
+__global__ void dump_fill_kernel(int64_t* finish, int64_t* first, int32_t* inst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        if (finish) finish[i] = -2;
+        if (first) first[i] = -2;
+        if (inst) inst[i] = -2;
+    }
+}
+
+cudaError_t launch_prep(const EvalParams& P, const uint32_t* dump_idx, cudaStream_t stream, int* launches) {
+    if (P.dump_n) {
+        const size_t n = (size_t)P.dump_n * P.n_req;
+        if (n) {
+            dump_fill_kernel<<<(unsigned)min((size_t)4096, (n + 255) / 256), 256, 0, stream>>>(
+                P.dump_finish, P.dump_first, P.dump_inst, n);
+            (*launches)++;
+        }
+    }
+    prep_kernel<<<(P.n_cand + 255) / 256, 256, 0, stream>>>(P);
+    (*launches)++;
+    if (P.dump_n) {
+        dump_map_kernel<<<(P.dump_n + 255) / 256, 256, 0, stream>>>(P, dump_idx);
+        (*launches)++;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace maaso

@@ -1,0 +1,243 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle: bit-exact records,
+per-request times and ranking."""
+import numpy as np
+import pytest
+
+import gen
+from golden_cases import all_cases, check_against_expect
+from gpu_common import gpu_eval, assert_records_equal
+
+pytestmark = pytest.mark.gpu
+
+MAPPINGS = [0, 1]  # lane groups (auto), block layout
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2509_06362_b200 as m
+    c = m.Context(0)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+@pytest.mark.parametrize("case", all_cases(), ids=lambda c: c["name"])
+def test_hand_timelines_on_gpu(ctx, case, mapping):
+    for flags, expect in case["runs"]:
+        res, dumps = gpu_eval(ctx, case["profile"], case["trace"], case["classes"], case["offsets"],
+                              case["inst"], case["budget"], None, flags, mapping, dump_idx=[0])
+        check_against_expect(res[0], {k: v[0] for k, v in dumps.items()}, expect)
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+@pytest.mark.parametrize("flags", [0, 1])
+def test_tiny_config_full(ctx, oracle_mod, mapping, flags):
+    cfg = gen.make_config("tiny")
+    tr = cfg["traces"][0]
+    idx = np.arange(0, 143, 5, dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"],
+                                          cfg["budget"], None, flags, dump_idx=idx)
+    got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], cfg["budget"],
+                       None, flags, mapping, dump_idx=idx)
+    assert_records_equal(got, want, "tiny")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_node_config_subset(ctx, oracle_mod, mapping):
+    # ragged sizes: 1777 requests = 6 tiles of 256 + a tail; candidates span every group width
+    cfg = gen.make_config("node", n_req=1777)
+    sel = np.arange(0, 10864, 23)
+    lists = []
+    for c in sel:
+        w = cfg["inst"][cfg["offsets"][c]:cfg["offsets"][c + 1]]
+        m, s, b = gen.unpack_inst(w)
+        lists.append(list(zip(m.tolist(), s.tolist(), b.tolist())))
+    off, inst = gen.candidates_from_lists(lists)
+    tr = cfg["traces"][0]
+    idx = np.arange(0, len(sel), 37, dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 8, dump_idx=idx)
+    got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 8, mapping=mapping, dump_idx=idx)
+    assert_records_equal(got, want, "node subset")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_multimodel_subset_with_masks(ctx, oracle_mod, mapping):
+    cfg = gen.make_config("multimodel", n_cand=600, n_req=3000)
+    tr = cfg["traces"][0]
+    rng = np.random.default_rng(5)
+    mask = rng.integers(1, 8, size=600).astype(np.uint32)
+    want = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 32, mask)
+    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 32, mask,
+                      mapping=mapping)
+    assert_records_equal(got, want, "multimodel masks")
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_bursty_optimistic_shows_cascades(ctx, oracle_mod, mapping):
+    cfg = gen.make_config("bursty", n_req=1500)
+    sel = slice(0, 10864, 61)
+    off_full, inst_full = cfg["offsets"], cfg["inst"]
+    lists = []
+    for c in range(0, 10864, 61):
+        m, s, b = gen.unpack_inst(inst_full[off_full[c]:off_full[c + 1]])
+        lists.append(list(zip(m.tolist(), s.tolist(), b.tolist())))
+    off, inst = gen.candidates_from_lists(lists)
+    total_cascade = 0
+    for j in (3, 9, 15):
+        tr = cfg["traces"][j]
+        for flags in (0, 1):
+            want = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 8, None, flags)
+            got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 8, None, flags, mapping)
+            assert_records_equal(got, want, f"bursty trace {j} flags {flags}")
+            total_cascade += int(got["n_cascade"].sum())
+    assert total_cascade > 0
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_large_placements_over_32_instances(ctx, oracle_mod, mapping):
+    """Candidates with up to 128 instances (budget 128): the strided block path."""
+    prof = gen.profile_multimodel(0)
+    rng = np.random.default_rng(3)
+    lists = []
+    for n_i in (33, 40, 64, 97, 128, 128, 5, 32, 1):
+        lst = []
+        for _ in range(n_i):
+            m = int(rng.integers(3))
+            s = 3 if m == 2 else 0
+            lst.append((m, s, int(rng.choice([1, 2, 4, 8, 16, 32, 64]))))
+        lists.append(lst)
+    off, inst = gen.candidates_from_lists(lists)
+    tr = gen.make_trace(4000, 400.0, 9, model_mix=(0.6, 0.3, 0.1), class_mix=(0.45, 0.27, 0.18, 0.10))
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None),
+                                (None, None, 180_000_000), (30_000_000, None, 600_000_000)])
+    idx = np.array([1, 4, 6], dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(prof, tr, classes, off, inst, 1024, dump_idx=idx)
+    got, gd = gpu_eval(ctx, prof, tr, classes, off, inst, 1024, mapping=mapping, dump_idx=idx)
+    assert (want["status"] == 0).all()
+    assert_records_equal(got, want, "large placements")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_edge_cases(ctx, oracle_mod, mapping):
+    prof = gen.profile_multimodel(0)
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 180_000_000)])
+    lists = [
+        [(0, 6, 4), (0, 6, 4)], [(2, 0, 4)], [(0, 0, 4)] * 129, [(3, 0, 4)], [(0, 10, 4)], [(0, 0, 0)],
+        [(0, 0, 65)], [(0, 0, 4), (2, 3, 8)], [], [(1, 1, 64)],
+    ]
+    off, inst = gen.candidates_from_lists(lists)
+    tr = gen.make_trace(700, 30.0, 4, model_mix=(0.6, 0.3, 0.1))
+    tr["out_tokens"][::7] = 1          # single-token requests never occupy a slot
+    tr["arrival_us"][100:140] = tr["arrival_us"][100]   # simultaneous arrivals
+    want = oracle_mod.eval_placements(prof, tr, classes, off, inst, 8)
+    got, _ = gpu_eval(ctx, prof, tr, classes, off, inst, 8, mapping=mapping)
+    assert_records_equal(got, want, "edge cases")
+    # empty trace: every valid candidate gets an all-zero record
+    empty = tr[:0]
+    want = oracle_mod.eval_placements(prof, empty, classes, off, inst, 8)
+    got, _ = gpu_eval(ctx, prof, empty, classes, off, inst, 8, mapping=mapping)
+    assert_records_equal(got, want, "empty trace")
+    # one request, one candidate
+    want = oracle_mod.eval_placements(prof, tr[:1], classes, off[7:9] - off[7], inst[off[7]:off[8]], 8)
+    got, _ = gpu_eval(ctx, prof, tr[:1], classes, off[7:9] - off[7], inst[off[7]:off[8]], 8, mapping=mapping)
+    assert_records_equal(got, want, "single")
+
+
+def test_determinism_and_mapping_independence(ctx):
+    cfg = gen.make_config("node", n_cand=700, n_req=2000)
+    tr = cfg["traces"][0]
+    a, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=0)
+    b, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=0)
+    c, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=1)
+    assert a.tobytes() == b.tobytes() == c.tobytes()
+
+
+def test_host_entry_point_matches_device_entry_point(ctx, oracle_mod):
+    cfg = gen.make_config("tiny")
+    tr = cfg["traces"][0]
+    ctx.load_profile(cfg["profile"])
+    t = ctx.load_trace(tr, cfg["classes"])
+    host = ctx.eval_placements_host(t, cfg["offsets"], cfg["inst"], 4)
+    ctx.free_trace(t)
+    want = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 4)
+    assert_records_equal(host, want, "host entry")
+
+
+def test_topk_matches_oracle_ranking(ctx, oracle_mod):
+    import torch
+    cfg = gen.make_config("node", n_cand=9000, n_req=600)
+    tr = cfg["traces"][0]
+    ctx.load_profile(cfg["profile"])
+    t = ctx.load_trace(tr, cfg["classes"])
+    res = ctx.eval_placements(t, ctx.to_device(cfg["offsets"]), ctx.to_device(cfg["inst"]), 8)
+    torch.cuda.synchronize()
+    rec = ctx.results_to_numpy(res)
+    want_rec = oracle_mod.eval_placements_parallel(cfg["profile"], tr, cfg["classes"], cfg["offsets"],
+                                                   cfg["inst"], 8)
+    assert_records_equal(rec, want_rec, "topk input")
+    for k in (1, 64, 1000):
+        idx, out = ctx.topk(res, k)
+        torch.cuda.synchronize()
+        want = oracle_mod.topk(want_rec, k)
+        got = idx.cpu().numpy().view(np.uint32)
+        assert got.tolist() == want.tolist(), k
+        assert ctx.results_to_numpy(out).tobytes() == want_rec[want].tobytes()
+    # doctored records: invalid ones last, exact mean comparison, padding when k > n
+    doctored = want_rec[:100].copy()
+    doctored["status"][3] = 8
+    doctored["n_hit"][:] = 7
+    doctored["n_served"][:] = 1_000_003
+    doctored["sum_ttft_us"][:] = (1 << 62) - np.arange(100, dtype=np.int64) % 5
+    doctored["n_served"][10] = 0
+    d = torch.from_numpy(doctored.view(np.uint8).reshape(100, 128)).cuda()
+    idx, _ = ctx.topk(d, 128)
+    torch.cuda.synchronize()
+    got = idx.cpu().numpy().view(np.uint32)
+    want = oracle_mod.topk(doctored, 128)
+    assert got[:100].tolist() == want.tolist()
+    assert (got[100:] == 0xFFFFFFFF).all()
+    ctx.free_trace(t)
+
+
+def test_api_errors(ctx):
+    import paper_2509_06362_b200 as m
+    cfg = gen.make_config("tiny")
+    ctx.load_profile(cfg["profile"])
+    bad = cfg["traces"][0].copy()
+    bad["arrival_us"][5] = bad["arrival_us"][4] - 1
+    with pytest.raises(m.MaasoError):
+        ctx.load_trace(bad, cfg["classes"])
+    bad = cfg["traces"][0].copy()
+    bad["model"][0] = 3
+    with pytest.raises(m.MaasoError):
+        ctx.load_trace(bad, cfg["classes"])
+    bad = cfg["traces"][0].copy()
+    bad["cls"][0] = 9
+    with pytest.raises(m.MaasoError):
+        ctx.load_trace(bad, cfg["classes"])
+    bad = cfg["traces"][0].copy()
+    bad["out_tokens"][0] = 0
+    with pytest.raises(m.MaasoError):
+        ctx.load_trace(bad, cfg["classes"])
+    p = dict(cfg["profile"])
+    p["step_us"] = cfg["profile"]["step_us"].copy()
+    p["step_us"][0, 0, 3] = 0
+    with pytest.raises(m.MaasoError):
+        ctx.load_profile(p)
+    fresh = m.Context(0)
+    with pytest.raises(m.MaasoError):
+        fresh.load_trace(cfg["traces"][0], cfg["classes"])    # no profile yet
+    fresh.close()
+    # a device-resident trace loads as well
+    import torch
+    ctx.load_profile(cfg["profile"])
+    dev = torch.from_numpy(cfg["traces"][0].view(np.uint8)).cuda()
+    t = ctx.load_trace(dev, cfg["classes"])
+    assert t.n == 500
+    ctx.free_trace(t)
