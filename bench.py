@@ -1,0 +1,303 @@
+#!/usr/bin/env python
+"""Throughput benchmark of the placement-scoring path.
+
+One step = one pass of the whole path over one batch: candidate validation, trace replay
+for every candidate (distributor + continuous batching) and the top-64 selection, on the
+single-node sweep (10,864 placements of <= 8 devices x a 10,000-request trace).
+Prints ONE JSON line.  `--impl reference` times the CPU oracle instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "candidate x request evaluations per second"
+UNIT = "evals/s"
+TOPK = 64
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t_begin, t_end):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        rows = [r for r in self.rows if t_begin - 0.05 <= r[0] <= t_end + 0.15] or self.rows
+        for _, line in rows:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(cfg, evals):
+    """Effective bytes of one pass: a 16-byte trace record per evaluation, the candidate
+    words and offsets, one 128-byte record per candidate, the latency tables once."""
+    n_cand = len(cfg["offsets"]) - 1
+    prof = cfg["profile"]
+    prof_bytes = prof["step_us"].nbytes + prof["prefill_base_us"].nbytes + prof["prefill_q16"].nbytes
+    return evals * 16 + 4 * len(cfg["inst"]) + 8 * n_cand + 128 * n_cand + prof_bytes
+
+
+def oracle_pass(oracle, cfg):
+    res = oracle.eval_placements(cfg["profile"], cfg["traces"][0], cfg["classes"], cfg["offsets"],
+                                 cfg["inst"], cfg["budget"])
+    oracle.topk(res, TOPK)
+    return int(res["n_counted"][res["status"] == 0].astype(np.int64).sum())
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, one thread, on a bounded sample per step."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import gen
+    import oracle
+    oracle.build()
+    sample_cands = 1024
+    cfg = gen.make_config(args.workload, n_cand=sample_cands, n_req=args.n_req)
+    times, evals = [], 0
+    for step in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        ev = oracle_pass(oracle, cfg)
+        dt = time.perf_counter() - t0
+        if step >= args.warmup:
+            times.append(dt)
+            evals = ev
+    value = evals * len(times) / sum(times)
+    sample = (f"first {sample_cands} placements of the sweep x all {len(cfg['traces'][0])} requests "
+              f"per step, 1 thread")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+        "data": "synthetic", "config": {"workload": f"{cfg['name']} sweep (sampled)", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def cpu_baseline(args):
+    """Oracle throughput on this host, one thread, on a bounded sample of the same workload."""
+    import gen
+    import oracle
+    oracle.build()
+    sample_cands = 2048
+    cfg = gen.make_config(args.workload, n_cand=sample_cands, n_req=args.n_req)
+    t0 = time.perf_counter()
+    evals = oracle_pass(oracle, cfg)
+    dt = time.perf_counter() - t0
+    return {"value": evals / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {sample_cands} placements of the sweep x all {len(cfg['traces'][0])} "
+                      f"requests, {dt:.1f} s, 1 thread"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mapping", type=int, default=0, help="0 auto (lane groups), 1 block layout")
+    ap.add_argument("--workload", default="node", help="node (default) or another configuration name")
+    ap.add_argument("--n-cand", type=int, default=None)
+    ap.add_argument("--n-req", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import gen
+    import paper_2509_06362_b200 as m
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    cfg = gen.make_config(args.workload, n_cand=args.n_cand, n_req=args.n_req)
+    trace_np = cfg["traces"][0]
+    n_cand = len(cfg["offsets"]) - 1
+    ctx = m.Context(local)
+    ctx.load_profile(cfg["profile"])
+    trace = ctx.load_trace(trace_np, cfg["classes"])
+    d_off, d_inst = ctx.to_device(cfg["offsets"]), ctx.to_device(cfg["inst"])
+    results = torch.empty((n_cand, 128), dtype=torch.uint8, device=ctx.device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=ctx.device)  # > L2 (126 MB)
+    stream = torch.cuda.current_stream()
+    ctx.set_timing(True)
+
+    def step():
+        ctx.eval_placements(trace, d_off, d_inst, cfg["budget"], mapping=args.mapping, out=results,
+                            stream=stream)
+        return ctx.topk(results, TOPK, stream=stream)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.fill_(1)
+        step()
+    sync_all()
+    rec = ctx.results_to_numpy(results)
+    evals_per_step = int(rec["n_counted"][rec["status"] == 0].astype(np.int64).sum())
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = ctx.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    kernel_ms = []
+    sync_all()
+    t_begin = time.time()
+    for a, b in ev:
+        flush.fill_(2)               # L2 flush between timed iterations (not timed)
+        a.record(stream)
+        step()
+        b.record(stream)
+        b.synchronize()
+        kernel_ms.append(ctx.get_timing())
+    sync_all()
+    t_end = time.time()
+    launches = ctx.launch_count() - launches0
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device=ctx.device)
+    if dist is not None:
+        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
+    total_ms = float(total_ms.item())
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
+
+    # end to end through the host-buffer entry point: H2D of the candidates from pinned memory,
+    # scoring, D2H of the records, every step
+    off_pin = torch.from_numpy(cfg["offsets"].view(np.int32)).pin_memory()
+    inst_pin = torch.from_numpy(cfg["inst"].view(np.int32)).pin_memory()
+    out_pin = torch.empty((n_cand, 128), dtype=torch.uint8).pin_memory()
+    off_h, inst_h = off_pin.numpy().view(np.uint32), inst_pin.numpy().view(np.uint32)
+    out_h = out_pin.numpy().reshape(-1).view(m.RESULT_DTYPE)
+    for _ in range(2):
+        ctx.eval_placements_host(trace, off_h, inst_h, cfg["budget"], mapping=args.mapping, out=out_h)
+    sync_all()
+    e2e_steps = max(3, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        ctx.eval_placements_host(trace, off_h, inst_h, cfg["budget"], mapping=args.mapping, out=out_h)
+    torch.cuda.synchronize()
+    e2e_s = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=ctx.device)
+    if dist is not None:
+        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
+    e2e_value = evals_per_step * world * e2e_steps / float(e2e_s.item())
+    assert out_h.tobytes() == rec.tobytes(), "host entry point disagrees with the device entry point"
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    value = evals_per_step * world * args.steps / (total_ms * 1e-3)
+    peak, peak_kind = measured_peak()
+    dom = "group_ms" if args.mapping == 0 else "block_ms"
+    dom_ms = statistics.mean(k[dom] for k in kernel_ms)
+    abytes = algorithmic_bytes(cfg, evals_per_step)
+    achieved = abytes / (dom_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": f"{cfg['name']} sweep: {n_cand} placements x {len(trace_np)} requests, "
+                               f"budget {cfg['budget']}, top-{TOPK}",
+                   "evals_per_step": evals_per_step, "mapping": "lane groups" if args.mapping == 0 else "block",
+                   "l2": "flushed between timed steps (256 MB write)", "per_gpu": "same sweep on every rank"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": int(cfg["offsets"].nbytes + cfg["inst"].nbytes),
+                "d2h_bytes_per_step": int(n_cand * 128)},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "eval_group_kernel" if args.mapping == 0 else "eval_block_kernel",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": abytes, "kernel_ms": dom_ms,
+                     "note": "effective bytes (16 B trace record per evaluation); the path is bound by "
+                             "integer issue of a dependent event chain, not by DRAM"},
+        "kernel_ms": {k: statistics.mean(x[k] for x in kernel_ms) for k in kernel_ms[0]},
+    }
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(args)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -197,6 +197,19 @@ MAASO_API int maaso_eval_placements_host(maaso_ctx *ctx, const maaso_trace *trac
 MAASO_API int maaso_topk(maaso_ctx *ctx, const maaso_result *results, uint64_t n_cand, uint32_t k,
                uint32_t order, uint32_t *out_idx, maaso_result *out_res, void *cuda_stream);
 
+/* Optional device timing.  While enabled, maaso_eval_placements and maaso_topk record CUDA
+ * events on the caller's stream around each kernel family; maaso_get_timing waits for the
+ * events of the most recent calls and reports milliseconds (0 for a family that did not
+ * run).  Off by default; costs a few event records per call when on. */
+typedef struct {
+    float prep_ms;  /* validation + bucket sort (+ dump buffer fill) */
+    float group_ms; /* lane-group scoring kernel */
+    float block_ms; /* block-layout scoring kernels */
+    float topk_ms;  /* all passes of the last maaso_topk */
+} maaso_timing;
+MAASO_API int maaso_set_timing(maaso_ctx *ctx, int enabled);
+MAASO_API int maaso_get_timing(maaso_ctx *ctx, maaso_timing *out);
+
 /* Number of kernels this context has launched so far (for accounting in benchmarks). */
 MAASO_API uint64_t maaso_launch_count(const maaso_ctx *ctx);
 

@@ -51,6 +51,11 @@ class _EvalOpts(C.Structure):
                 ("dump_first_us", C.c_void_p), ("dump_inst", C.c_void_p)]
 
 
+class _Timing(C.Structure):
+    _fields_ = [("prep_ms", C.c_float), ("group_ms", C.c_float), ("block_ms", C.c_float),
+                ("topk_ms", C.c_float)]
+
+
 def lib_path():
     return _build.LIB
 
@@ -71,6 +76,8 @@ def _load():
     lib.maaso_eval_placements.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp, vp]
     lib.maaso_eval_placements_host.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp]
     lib.maaso_topk.argtypes = [vp, vp, u64, u32, u32, vp, vp, vp]
+    lib.maaso_set_timing.argtypes = [vp, C.c_int]
+    lib.maaso_get_timing.argtypes = [vp, C.POINTER(_Timing)]
     lib.maaso_launch_count.argtypes = [vp]
     lib.maaso_launch_count.restype = u64
     lib.maaso_strerror.argtypes = [C.c_int]
@@ -78,7 +85,7 @@ def _load():
     lib.maaso_last_error.argtypes = [vp]
     lib.maaso_last_error.restype = C.c_char_p
     for name in ("maaso_create", "maaso_load_profile", "maaso_load_trace", "maaso_eval_placements",
-                 "maaso_eval_placements_host", "maaso_topk"):
+                 "maaso_eval_placements_host", "maaso_topk", "maaso_set_timing", "maaso_get_timing"):
         getattr(lib, name).restype = C.c_int
     return lib
 
@@ -195,6 +202,17 @@ def maaso_topk(ctx, results, n_cand, k, out_idx, out_res=None, order=0, stream=N
                            _stream_ptr(stream)), "maaso_topk", ctx)
 
 
+def maaso_set_timing(ctx, enabled):
+    _check(_lib.maaso_set_timing(ctx, 1 if enabled else 0), "maaso_set_timing", ctx)
+
+
+def maaso_get_timing(ctx):
+    """milliseconds per kernel family of the most recent eval / topk calls (waits for them)"""
+    t = _Timing()
+    _check(_lib.maaso_get_timing(ctx, C.byref(t)), "maaso_get_timing", ctx)
+    return {"prep_ms": t.prep_ms, "group_ms": t.group_ms, "block_ms": t.block_ms, "topk_ms": t.topk_ms}
+
+
 def maaso_launch_count(ctx):
     return int(_lib.maaso_launch_count(ctx))
 
@@ -281,6 +299,12 @@ class Context:
         rec = torch.empty((k, 128), dtype=torch.uint8, device=self.device) if with_records else None
         maaso_topk(self.handle, results, n_cand, k, idx, rec, order, stream)
         return idx, rec
+
+    def set_timing(self, enabled):
+        maaso_set_timing(self.handle, enabled)
+
+    def get_timing(self):
+        return maaso_get_timing(self.handle)
 
     def launch_count(self):
         return maaso_launch_count(self.handle)

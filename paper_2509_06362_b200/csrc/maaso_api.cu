@@ -51,6 +51,9 @@ struct maaso_ctx {
     cudaStream_t own_stream;
     uint64_t launches;
     int tile_recs;
+    bool timing;
+    cudaEvent_t ev[6];   // eval: start, after prep, after group, after block; topk: start, end
+    bool ev_eval, ev_topk;
     std::string last_error;
 };
 
@@ -116,6 +119,9 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
     ctx->launches = 0;
     ctx->tile_recs = 256;
     ctx->own_stream = nullptr;
+    ctx->timing = false;
+    ctx->ev_eval = ctx->ev_topk = false;
+    for (int i = 0; i < 6; i++) ctx->ev[i] = nullptr;
     DeviceGuard g(cuda_device);
     cudaDeviceProp prop;
     e = cudaGetDeviceProperties(&prop, cuda_device);
@@ -168,6 +174,8 @@ MAASO_API void maaso_destroy(maaso_ctx* ctx) {
     if (ctx->topk_scratch) cudaFree(ctx->topk_scratch);
     if (ctx->stage) cudaFree(ctx->stage);
     if (ctx->own_stream) cudaStreamDestroy(ctx->own_stream);
+    for (int i = 0; i < 6; i++)
+        if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
     delete ctx;
 }
 
@@ -375,18 +383,25 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, 64 * 4, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "memset");
     int launches = 0;
+    if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
     e = launch_prep(P, o.dump_cand_idx, stream, &launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "prep launch");
+    if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
     if (o.mapping != MAASO_MAP_BLOCK) {
         e = launch_eval_group(P, grid_g, tile, stream);
         launches++;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "group kernel launch");
     }
+    if (ctx->timing) cudaEventRecord(ctx->ev[2], stream);
     for (int b = 6; b <= 8; b++) {
         if (grid_b[b - 6] == 0) continue;
         e = launch_eval_block(P, b, grid_b[b - 6], tile, stream);
         launches++;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "block kernel launch");
+    }
+    if (ctx->timing) {
+        cudaEventRecord(ctx->ev[3], stream);
+        ctx->ev_eval = true;
     }
     ctx->launches += (uint64_t)launches;
     return MAASO_OK;
@@ -438,10 +453,49 @@ MAASO_API int maaso_topk(maaso_ctx* ctx, const maaso_result* results, uint64_t n
     int rc = grow(ctx, &ctx->topk_scratch, &ctx->topk_scratch_bytes, topk_scratch_bytes(n_cand, k));
     if (rc != MAASO_OK) return rc;
     int launches = 0;
+    if (ctx->timing) cudaEventRecord(ctx->ev[4], (cudaStream_t)cuda_stream);
     cudaError_t e = launch_topk(results, n_cand, k, ctx->topk_scratch, out_idx, out_res,
                                 (cudaStream_t)cuda_stream, &launches);
+    if (ctx->timing) {
+        cudaEventRecord(ctx->ev[5], (cudaStream_t)cuda_stream);
+        ctx->ev_topk = true;
+    }
     ctx->launches += (uint64_t)launches;
     if (e != cudaSuccess) return cuda_fail(ctx, e, "topk launch");
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_set_timing(maaso_ctx* ctx, int enabled) {
+    if (!ctx) return MAASO_EINVAL;
+    DeviceGuard g(ctx->device);
+    if (enabled)
+        for (int i = 0; i < 6; i++)
+            if (!ctx->ev[i]) {
+                cudaError_t e = cudaEventCreate(&ctx->ev[i]);
+                if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventCreate");
+            }
+    ctx->timing = enabled != 0;
+    ctx->ev_eval = ctx->ev_topk = false;
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_get_timing(maaso_ctx* ctx, maaso_timing* out) {
+    if (!ctx || !out) return MAASO_EINVAL;
+    memset(out, 0, sizeof(*out));
+    if (!ctx->timing) return fail(ctx, MAASO_ESTATE, "timing is not enabled");
+    DeviceGuard g(ctx->device);
+    cudaError_t e = cudaSuccess;
+    if (ctx->ev_eval) {
+        e = cudaEventSynchronize(ctx->ev[3]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->prep_ms, ctx->ev[0], ctx->ev[1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->group_ms, ctx->ev[1], ctx->ev[2]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->block_ms, ctx->ev[2], ctx->ev[3]);
+    }
+    if (e == cudaSuccess && ctx->ev_topk) {
+        e = cudaEventSynchronize(ctx->ev[5]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->topk_ms, ctx->ev[4], ctx->ev[5]);
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "timing events");
     return MAASO_OK;
 }
 
