@@ -8,7 +8,6 @@
 namespace maaso {
 
 constexpr int kStages = 3;
-constexpr int kKeyStride = 72;  // uint16 per lane: 64 keys + pad so 16-byte rows spread over banks
 
 __device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t v, int off, uint32_t mask) {
     uint32_t lo = __shfl_xor_sync(mask, (uint32_t)v, off);
@@ -45,18 +44,19 @@ __host__ __device__ inline size_t group_smem_bytes(uint32_t n_rows, uint32_t n_c
 __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows, uint32_t n_classes,
                                            int tile_recs) {
     GroupSmem s;
+    // 16-byte aligned parts first (tiles, slot keys are read as 16-byte words)
     s.tiles = reinterpret_cast<uint4*>(base);
     base += (size_t)kStages * tile_recs * 16;
+    s.keys = reinterpret_cast<uint16_t*>(base);
+    base += (size_t)kGroupThreads * kKeyStride * 2;
+    s.hbc = reinterpret_cast<uint32_t*>(base);
+    base += (size_t)kGroupThreads * 8 * 4;
     s.classes = reinterpret_cast<int64_t*>(base);
     base += (size_t)n_classes * 24;
     s.full_bar = reinterpret_cast<uint64_t*>(base);
     base += kStages * 8;
     s.steps = reinterpret_cast<int32_t*>(base);
     base += (size_t)n_rows * 64 * 4;
-    s.keys = reinterpret_cast<uint16_t*>(base);
-    base += (size_t)kGroupThreads * kKeyStride * 2;
-    s.hbc = reinterpret_cast<uint32_t*>(base);
-    base += (size_t)kGroupThreads * 8 * 4;
     s.empty_cnt = reinterpret_cast<uint32_t*>(base);
     base += kStages * 4;
     s.work = reinterpret_cast<uint32_t*>(base);
@@ -84,9 +84,12 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
     }
     __syncthreads();
 
-    uint16_t* const keys = sm.keys + tid * kKeyStride;
-    uint32_t* const hbc = sm.hbc + tid * 8;
-    Payload* const pay = P.payload + ((size_t)blockIdx.x * kGroupThreads + tid) * MAASO_WMAX;
+    LaneEnv env;
+    env.keys = sm.keys + tid * kKeyStride;
+    env.hbc = sm.hbc + tid * 8;
+    env.pay = P.payload + ((size_t)blockIdx.x * kGroupThreads + tid) * MAASO_WMAX;
+    env.classes = sm.classes;
+    uint32_t* const hbc = env.hbc;
     const bool optimistic = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
     const uint32_t n_tiles = (P.n_req + tile_recs - 1) / tile_recs;
@@ -113,14 +116,18 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
         const uint32_t sub = tid & (G - 1u);
         const uint32_t pos = wi * per + (tid >> b);
         const bool valid = pos < P.bucket_count[b];
-        const uint32_t cand = valid ? P.bucket_list[(size_t)b * P.n_cand + pos] : 0u;
+        // neighbouring candidates of a sweep cost about the same; a multiplicative shuffle of the
+        // bucket order spreads the expensive ones over warps and blocks
+        const uint32_t cnt = P.bucket_count[b];
+        const uint32_t mult = (cnt % 1000003u) ? 1000003u : 999983u;
+        const uint32_t cand = valid ? P.bucket_list[(size_t)b * P.n_cand + (uint32_t)(((uint64_t)pos * mult) % cnt)] : 0u;
         const uint32_t gmask = (G == 32u) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(G - 1u)));
 
         uint32_t n_i = 0, lo = 0;
         if (valid) { lo = P.offsets[cand]; n_i = P.offsets[cand + 1] - lo; }
         const bool has = valid && sub < n_i;
         LaneInst in;
-        in.T = 0; in.K = 0; in.w = 0; in.kmin = 0; in.mask = 0;
+        in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = 0; in.sw = 1; in.mask = 0;
         in.B = 1; in.model = 0xFFFFFFFFu; in.step = sm.steps; in.stepB = 1; in.pre_base = 0; in.pre_q16 = 0;
         if (has) {
             const uint32_t word = P.inst[lo + sub];
@@ -135,6 +142,8 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
         const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
         Dump dump{nullptr, nullptr, nullptr};
         if (valid) dump = dump_for(P, cand);
+        env.dump = dump;
+        env.inst_idx = sub;
         Stats st; st.clear();
         for (int i = 0; i < 8; i++) hbc[i] = 0;
         int64_t now = 0;
@@ -184,7 +193,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                         uint64_t key = kKeyInf;
                         int64_t t0 = 0;
                         if (elig) {
-                            lane_advance(in, now, false, keys, pay, st, hbc, sm.classes, sub, dump);
+                            lane_advance(in, now, false, env, st);
                             key = lane_predict(in, q, pre, lim_ttft, lim_tbt, lim_e2e, optimistic, t0);
                         }
                         uint64_t best = key;
@@ -205,7 +214,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                             const int winner = __ffs((int)votes) - 1;  // lowest instance index wins ties
                             if ((best >> 63) == 0) {
                                 if ((int)lane == winner)
-                                    lane_admit(in, q, req, pre, keys, pay, st, hbc, sm.classes, sub, dump);
+                                    lane_admit(in, q, req, pre, env, st);
                                 pending = false;
                             } else {
                                 // every capable instance is full: wait until the chosen slot frees
@@ -237,7 +246,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
         }
 
         // drain, reduce over the group, write the record
-        if (has && status == 0) lane_advance(in, 0, true, keys, pay, st, hbc, sm.classes, sub, dump);
+        if (has && status == 0) lane_advance(in, 0, true, env, st);
         for (uint32_t off = 1; off < G; off <<= 1) {
             st.served += __shfl_xor_sync(gmask, st.served, (int)off);
             st.hit += __shfl_xor_sync(gmask, st.hit, (int)off);
