@@ -51,6 +51,7 @@ extern "C" {
 #define MAASO_ESTATE (-2) /* profile not loaded, trace belongs to another context, ... */
 #define MAASO_ENOMEM (-3)
 #define MAASO_ECUDA (-4)  /* a CUDA runtime call failed; text via maaso_last_error() */
+#define MAASO_ETOOBIG (-5) /* size beyond the fixed capacity of an entry point that cannot allocate */
 
 /* per-candidate status bits (maaso_result.status) */
 #define MAASO_CAND_EBUDGET 1u   /* devices used exceed the budget: constraint (c), Sec. IV-C */
@@ -196,6 +197,26 @@ MAASO_API int maaso_eval_placements_host(maaso_ctx *ctx, const maaso_trace *trac
  * matching records (zeroed padding).  k <= MAASO_MAX_TOPK.  Enqueued on cuda_stream. */
 MAASO_API int maaso_topk(maaso_ctx *ctx, const maaso_result *results, uint64_t n_cand, uint32_t k,
                uint32_t order, uint32_t *out_idx, maaso_result *out_res, void *cuda_stream);
+
+/* Top-k without any allocation.  (The paper has no counterpart; this is a deployment
+ * variant of maaso_topk.)  It is meant for callers that must not allocate device memory
+ * while they run: code inside a memory-pool or arena framework that owns all device memory,
+ * a latency-critical serving loop where an allocation would synchronise the device, or a
+ * process that is already close to its memory limit.  Same inputs, outputs and ordering
+ * as maaso_topk, no context needed; the partial lists of the selection passes live in a
+ * fixed array of about 0.8 MB inside the library image (every GPU that loads the library
+ * holds it until the process exits) instead of context scratch memory.
+ * Limits: n_cand <= MAASO_NOALLOC_MAX_CAND and k <= MAASO_NOALLOC_MAX_K; anything larger
+ * returns MAASO_ETOOBIG and does nothing.  The call uses the current CUDA device and calls
+ * no cudaMalloc / cudaFree or other allocating routine.  The first call on a device looks
+ * up the array's device address; make that first call before starting any stream capture.
+ * All calls on a device share the one array: two calls whose kernels may overlap on the
+ * GPU (different streams, no ordering between them) race on it, so order them.  Nothing
+ * in the array needs clearing between calls: each pass overwrites what the next one reads. */
+#define MAASO_NOALLOC_MAX_CAND (1u << 20)
+#define MAASO_NOALLOC_MAX_K 64
+MAASO_API int maaso_topk_noalloc(const maaso_result *results, uint64_t n_cand, uint32_t k, uint32_t order,
+                                 uint32_t *out_idx, maaso_result *out_res, void *cuda_stream);
 
 /* Optional device timing.  While enabled, maaso_eval_placements and maaso_topk record CUDA
  * events on the caller's stream around each kernel family; maaso_get_timing waits for the

@@ -76,6 +76,8 @@ def _load():
     lib.maaso_eval_placements.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp, vp]
     lib.maaso_eval_placements_host.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp]
     lib.maaso_topk.argtypes = [vp, vp, u64, u32, u32, vp, vp, vp]
+    lib.maaso_topk_noalloc.argtypes = [vp, u64, u32, u32, vp, vp, vp]
+    lib.maaso_topk_noalloc.restype = C.c_int
     lib.maaso_set_timing.argtypes = [vp, C.c_int]
     lib.maaso_get_timing.argtypes = [vp, C.POINTER(_Timing)]
     lib.maaso_launch_count.argtypes = [vp]
@@ -200,6 +202,19 @@ def maaso_eval_placements_host(ctx, trace, offsets, inst, budget, out_results, c
 def maaso_topk(ctx, results, n_cand, k, out_idx, out_res=None, order=0, stream=None):
     _check(_lib.maaso_topk(ctx, _ptr(results), int(n_cand), int(k), int(order), _ptr(out_idx), _ptr(out_res),
                            _stream_ptr(stream)), "maaso_topk", ctx)
+
+
+NOALLOC_MAX_CAND = 1 << 20
+NOALLOC_MAX_K = 64
+
+
+def maaso_topk_noalloc(results, n_cand, k, out_idx, out_res=None, order=0, stream=None):
+    """Top-k for callers that may not allocate device memory (pool-managed or latency-critical
+    code): same result as maaso_topk, no context, scratch in a fixed array of the library;
+    n_cand <= NOALLOC_MAX_CAND, k <= NOALLOC_MAX_K.  Returns the C return code unchanged so
+    that the caller can tell a capacity refusal (-5) from other errors."""
+    return int(_lib.maaso_topk_noalloc(_ptr(results), int(n_cand), int(k), int(order), _ptr(out_idx),
+                                       _ptr(out_res), _stream_ptr(stream)))
 
 
 def maaso_set_timing(ctx, enabled):

@@ -508,6 +508,7 @@ MAASO_API const char* maaso_strerror(int code) {
         case MAASO_ESTATE: return "wrong state (no profile, foreign trace, unsupported device)";
         case MAASO_ENOMEM: return "out of memory";
         case MAASO_ECUDA: return "CUDA runtime error";
+        case MAASO_ETOOBIG: return "size beyond the fixed capacity of this entry point";
         default: return "unknown error";
     }
 }

@@ -135,4 +135,56 @@ cudaError_t launch_topk(const maaso_result* results, uint64_t n_cand, uint32_t k
     return cudaGetLastError();
 }
 
+// ---- top-k for callers that cannot allocate ---------------------------------------------------
+// The partial lists of the passes live in a fixed array inside the library image instead of
+// memory obtained at run time.  Every pass writes each entry the next pass reads, so nothing
+// in the array has to be cleared between calls.
+constexpr uint64_t kNoAllocMaxCand = MAASO_NOALLOC_MAX_CAND;
+constexpr uint32_t kNoAllocMaxK = MAASO_NOALLOC_MAX_K;
+constexpr size_t kNoAllocBytes =
+    ((((kNoAllocMaxCand + kChunk - 1) / kChunk) * kNoAllocMaxK * sizeof(Entry) * 2 + 64) + 255) / 256 * 256;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_noalloc_ptr[kMaxDevices];  // device address of the array, per device, once resolved
+
+// Resolves (once per device, with that device current) the device address of the array:
+// its name is only a host-side handle and must not be handed to a kernel.
+static cudaError_t noalloc_scratch(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
+}
+
 }  // namespace maaso
+
+extern "C" MAASO_API int maaso_topk_noalloc(const maaso_result* results, uint64_t n_cand, uint32_t k,
+                                            uint32_t order, uint32_t* out_idx, maaso_result* out_res,
+                                            void* cuda_stream) {
+    using namespace maaso;
+    if (k == 0) return MAASO_OK;
+    if (!out_idx || (!results && n_cand) || order != 0) return MAASO_EINVAL;
+    if (n_cand > kNoAllocMaxCand || k > kNoAllocMaxK) return MAASO_ETOOBIG;  // beyond the fixed scratch
+    void* scratch = nullptr;
+    if (noalloc_scratch(&scratch) != cudaSuccess) {
+        cudaGetLastError();
+        return MAASO_ECUDA;
+    }
+    int launches = 0;
+    const cudaError_t e = launch_topk(results, n_cand, k, scratch, out_idx, out_res, (cudaStream_t)cuda_stream,
+                                      &launches);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return MAASO_ECUDA;
+    }
+    return MAASO_OK;
+}
