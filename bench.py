@@ -194,10 +194,18 @@ def main():
     stream = torch.cuda.current_stream()
     ctx.set_timing(True)
 
+    from paper_2509_06362_b200.distributed import global_topk
+
+    def rank_topk(rec, k):
+        return ctx.topk(rec, k, stream=stream)
+
     def step():
         ctx.eval_placements(trace, d_off, d_inst, cfg["budget"], mapping=args.mapping, out=results,
                             stream=stream)
-        return ctx.topk(results, TOPK, stream=stream)
+        if world == 1:
+            return ctx.topk(results, TOPK, stream=stream)
+        # every rank holds its own copy of the sweep: global index = rank * n_cand + local index
+        return global_topk(rank_topk, rank_topk, results, rank * n_cand, TOPK)
 
     def sync_all():
         torch.cuda.synchronize()

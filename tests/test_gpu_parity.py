@@ -149,6 +149,64 @@ def test_edge_cases(ctx, oracle_mod, mapping):
     assert_records_equal(got, want, "single")
 
 
+def _subset(cfg, sel):
+    lists = []
+    for c in sel:
+        m, s, b = gen.unpack_inst(cfg["inst"][cfg["offsets"][c]:cfg["offsets"][c + 1]])
+        lists.append(list(zip(m.tolist(), s.tolist(), b.tolist())))
+    return gen.candidates_from_lists(lists)
+
+
+def test_node_config_full_size_as_benchmarked(ctx, oracle_mod):
+    """The benchmark's workload and launch configuration: all 10,864 placements x 10,000 requests."""
+    cfg = gen.make_config("node")
+    tr = cfg["traces"][0]
+    want = oracle_mod.eval_placements_parallel(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8)
+    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=0)
+    assert_records_equal(got, want, "node full")
+    assert (want["status"] == 0).all() and (want["n_counted"] == 10000).all()
+    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=1)
+    assert_records_equal(got, want, "node full, block mapping")
+
+
+def test_multimodel_full_trace_sampled_candidates(ctx, oracle_mod):
+    cfg = gen.make_config("multimodel")
+    tr = cfg["traces"][0]
+    n_i = np.diff(cfg["offsets"].astype(np.int64))
+    sel = sorted(set(np.arange(0, 100_000, 400).tolist() + np.argsort(n_i)[-6:].tolist()))
+    off, inst = _subset(cfg, sel)
+    idx = np.array([0, len(sel) - 1], dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 32, dump_idx=idx)
+    got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 32, dump_idx=idx)
+    assert_records_equal(got, want, "multimodel full trace")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+
+
+def test_scale_full_trace_sampled_candidates(ctx, oracle_mod):
+    """10^6-request trace, four SLO classes, candidates sampled from the 10^6-candidate set
+    including the ones with the most instances (over 32: block path)."""
+    cfg = gen.make_config("scale")
+    tr = cfg["traces"][0]
+    n_i = np.diff(cfg["offsets"].astype(np.int64))
+    sel = sorted(set(np.arange(0, 1_000_000, 40_000).tolist() + np.argsort(n_i)[-4:].tolist()))
+    off, inst = _subset(cfg, sel)
+    want = oracle_mod.eval_placements_parallel(cfg["profile"], tr, cfg["classes"], off, inst, 128, workers=8)
+    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 128)
+    assert (want["status"] == 0).all() and n_i.max() > 32
+    assert_records_equal(got, want, "scale full trace")
+
+
+def test_bursty_all_traces_full_length(ctx, oracle_mod):
+    cfg = gen.make_config("bursty")
+    off, inst = _subset(cfg, range(0, 10864, 97))
+    for j, tr in enumerate(cfg["traces"]):
+        flags = j % 2
+        want = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 8, None, flags)
+        got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 8, None, flags)
+        assert_records_equal(got, want, f"bursty trace {j}")
+
+
 def test_determinism_and_mapping_independence(ctx):
     cfg = gen.make_config("node", n_cand=700, n_req=2000)
     tr = cfg["traces"][0]
