@@ -20,6 +20,40 @@ __device__ __forceinline__ uint64_t shfl_u64(uint64_t v, int src, uint32_t mask)
     return ((uint64_t)hi << 32) | lo;
 }
 
+struct ArgMin {
+    bool found;
+    uint32_t tier;
+    int winner;  // lane
+};
+
+// Distributor's choice inside a lane group: smallest (tier, predicted first token), lowest lane
+// among equals.  Predicted times are at or after `now`; when every finite key is within 2^31 us
+// of it the minimum is a 32-bit shuffle butterfly, otherwise a 64-bit one.
+__device__ __forceinline__ ArgMin group_argmin(uint64_t key, int64_t now, uint32_t gmask, uint32_t G) {
+    // Called by all 32 lanes; every operation uses the full mask and stays inside the group
+    // because xor offsets are below the group width.
+    ArgMin r;
+    const bool finite = key != kKeyInf;
+    const uint64_t d = (key & ~(1ull << 63)) - (uint64_t)now;
+    const bool wide = finite && d >= 0x7FFFFFFFull;
+    if (!__any_sync(0xFFFFFFFFu, wide)) {
+        const uint32_t k32 = finite ? ((uint32_t)(key >> 63) << 31) | (uint32_t)d : 0xFFFFFFFFu;
+        uint32_t best = k32;
+        for (uint32_t off = 1; off < G; off <<= 1) best = min(best, __shfl_xor_sync(0xFFFFFFFFu, best, (int)off));
+        r.found = best != 0xFFFFFFFFu;
+        r.tier = best >> 31;
+        r.winner = __ffs((int)(__ballot_sync(0xFFFFFFFFu, k32 == best) & gmask)) - 1;
+    } else {
+        uint64_t best = key;
+        for (uint32_t off = 1; off < G; off <<= 1) best = min(best, shfl_xor_u64(best, (int)off, 0xFFFFFFFFu));
+        r.found = best != kKeyInf;
+        r.tier = (uint32_t)(best >> 63);
+        r.winner = __ffs((int)(__ballot_sync(0xFFFFFFFFu, key == best) & gmask)) - 1;
+    }
+    if (!r.found) r.winner = (int)(threadIdx.x & 31u);  // any valid source lane for the shuffle that follows
+    return r;
+}
+
 struct GroupSmem {
     uint4* tiles;        // [kStages][tile_recs]
     int32_t* steps;      // [n_rows][64]
@@ -63,6 +97,8 @@ __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows,
     return s;
 }
 
+// OPT: the distributor predicts with the step time right after admission (optimistic estimate)
+template <bool OPT>
 __global__ void __launch_bounds__(kGroupThreads)
 eval_group_kernel(const EvalParams P, const int tile_recs) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -90,7 +126,6 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
     env.pay = P.payload + ((size_t)blockIdx.x * kGroupThreads + tid) * MAASO_WMAX;
     env.classes = sm.classes;
     uint32_t* const hbc = env.hbc;
-    const bool optimistic = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
     const uint32_t n_tiles = (P.n_req + tile_recs - 1) / tile_recs;
     uint32_t tile_seq = 0;  // tiles consumed so far by this warp (same in every warp)
@@ -173,6 +208,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
             const uint4* tile = sm.tiles + (size_t)s * tile_recs;
             const uint32_t recs = min((uint32_t)tile_recs, P.n_req - t * tile_recs);
             for (uint32_t ri = 0; ri < recs; ri++) {
+                // All 32 lanes walk the trace together and every warp-level operation below uses
+                // the full mask (segmented by the group width), so the groups of a warp share one
+                // instruction stream; only events (retire, admit) diverge.
                 const Request q = decode_request(tile[ri]);
                 const uint32_t req = t * tile_recs + ri;
                 bool pending = valid && status == 0 && ((cmask >> (q.cls & 31u)) & 1u);
@@ -186,20 +224,21 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                 const int64_t lim_tbt = sm.classes[q.cls * 3 + 1];
                 const int64_t lim_e2e = sm.classes[q.cls * 3 + 2];
                 uint32_t tries = 0;
-                while (__any_sync(0xFFFFFFFFu, pending)) {
+                do {
+                    uint64_t key = kKeyInf;
+                    int64_t t0 = 0;
                     if (pending) {
                         attempts++;
                         tries++;
-                        uint64_t key = kKeyInf;
-                        int64_t t0 = 0;
                         if (elig) {
                             lane_advance(in, now, false, env, st);
-                            key = lane_predict(in, q, pre, lim_ttft, lim_tbt, lim_e2e, optimistic, t0);
+                            key = lane_predict(in, q, pre, lim_ttft, lim_tbt, lim_e2e, OPT, t0);
                         }
-                        uint64_t best = key;
-                        for (uint32_t off = 1; off < G; off <<= 1)
-                            best = min(best, shfl_xor_u64(best, (int)off, gmask));
-                        if (best == kKeyInf) {
+                    }
+                    const ArgMin am = group_argmin(key, now, gmask, G);
+                    const int64_t t0w = (int64_t)shfl_u64((uint64_t)t0, am.winner, 0xFFFFFFFFu);
+                    if (pending) {
+                        if (!am.found) {
                             // overflow protection: nobody can meet the deadline -> rejected
                             n_rejected++;
                             if (sub == 0) {
@@ -209,21 +248,30 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                                 if (dump.inst) dump.inst[req] = -1;
                             }
                             pending = false;
+                        } else if (am.tier == 0) {
+                            if ((int)lane == am.winner) lane_admit(in, q, req, pre, env, st);
+                            pending = false;
                         } else {
-                            const uint32_t votes = __ballot_sync(gmask, key == best) & gmask;
-                            const int winner = __ffs((int)votes) - 1;  // lowest instance index wins ties
-                            if ((best >> 63) == 0) {
-                                if ((int)lane == winner)
+                            // every capable instance is full: wait until the chosen slot frees
+                            now = t0w;
+                            if (!OPT) {
+                                // With the worst-case estimate the next round cannot choose differently:
+                                // at that time the winner has a free slot with the same predicted first
+                                // token, and no other instance's prediction can have become earlier or
+                                // feasible.  The second round is only counted; other clocks catch up lazily.
+                                attempts++;
+                                if ((int)lane == am.winner) {
+                                    lane_advance(in, now, false, env, st);
                                     lane_admit(in, q, req, pre, env, st);
+                                }
                                 pending = false;
-                            } else {
-                                // every capable instance is full: wait until the chosen slot frees
-                                now = (int64_t)shfl_u64((uint64_t)t0, winner, gmask);
-                                if (tries >= kAttemptCap) { status = MAASO_CAND_ELOOP; pending = false; }
+                            } else if (tries >= kAttemptCap) {
+                                status = MAASO_CAND_ELOOP;
+                                pending = false;
                             }
                         }
                     }
-                }
+                } while (OPT && __any_sync(0xFFFFFFFFu, pending));
             }
             // release the stage; the warp that arrives last refills it
             __syncwarp();
@@ -247,18 +295,20 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
 
         // drain, reduce over the group, write the record
         if (has && status == 0) lane_advance(in, 0, true, env, st);
+        __syncwarp();
+        constexpr uint32_t kFull = 0xFFFFFFFFu;
         for (uint32_t off = 1; off < G; off <<= 1) {
-            st.served += __shfl_xor_sync(gmask, st.served, (int)off);
-            st.hit += __shfl_xor_sync(gmask, st.hit, (int)off);
-            st.sum_ttft += (int64_t)shfl_xor_u64((uint64_t)st.sum_ttft, (int)off, gmask);
-            st.sum_e2e += (int64_t)shfl_xor_u64((uint64_t)st.sum_e2e, (int)off, gmask);
-            st.tokens += shfl_xor_u64(st.tokens, (int)off, gmask);
-            st.checksum += shfl_xor_u64(st.checksum, (int)off, gmask);
-            st.max_ttft = max(st.max_ttft, (int64_t)shfl_xor_u64((uint64_t)st.max_ttft, (int)off, gmask));
-            st.max_e2e = max(st.max_e2e, (int64_t)shfl_xor_u64((uint64_t)st.max_e2e, (int)off, gmask));
-            st.makespan = max(st.makespan, (int64_t)shfl_xor_u64((uint64_t)st.makespan, (int)off, gmask));
+            st.served += __shfl_xor_sync(kFull, st.served, (int)off);
+            st.hit += __shfl_xor_sync(kFull, st.hit, (int)off);
+            st.sum_ttft += (int64_t)shfl_xor_u64((uint64_t)st.sum_ttft, (int)off, kFull);
+            st.sum_e2e += (int64_t)shfl_xor_u64((uint64_t)st.sum_e2e, (int)off, kFull);
+            st.tokens += shfl_xor_u64(st.tokens, (int)off, kFull);
+            st.checksum += shfl_xor_u64(st.checksum, (int)off, kFull);
+            st.max_ttft = max(st.max_ttft, (int64_t)shfl_xor_u64((uint64_t)st.max_ttft, (int)off, kFull));
+            st.max_e2e = max(st.max_e2e, (int64_t)shfl_xor_u64((uint64_t)st.max_e2e, (int)off, kFull));
+            st.makespan = max(st.makespan, (int64_t)shfl_xor_u64((uint64_t)st.makespan, (int)off, kFull));
         }
-        __syncwarp(gmask);
+        __syncwarp();
         if (valid && sub == 0) {
             uint32_t h[8];
             for (int i = 0; i < 8; i++) h[i] = 0;
@@ -271,20 +321,21 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
 
 cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, cudaStream_t stream) {
     const size_t smem = group_smem_bytes(P.n_rows, P.n_classes, tile_recs);
-    cudaError_t e = cudaFuncSetAttribute(eval_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    const bool opt = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
+    auto kernel = opt ? eval_group_kernel<true> : eval_group_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    eval_group_kernel<<<grid, kGroupThreads, smem, stream>>>(P, tile_recs);
+    kernel<<<grid, kGroupThreads, smem, stream>>>(P, tile_recs);
     return cudaGetLastError();
 }
 
 int occupancy_eval_group(const EvalParams& P, int tile_recs) {
     const size_t smem = group_smem_bytes(P.n_rows, P.n_classes, tile_recs);
-    cudaFuncSetAttribute(eval_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const bool opt = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
+    auto kernel = opt ? eval_group_kernel<true> : eval_group_kernel<false>;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, eval_group_kernel, kGroupThreads, smem) !=
-        cudaSuccess)
-        return 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kGroupThreads, smem) != cudaSuccess) return 1;
     return n < 1 ? 1 : n;
 }
 
