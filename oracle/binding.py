@@ -118,6 +118,10 @@ def eval_placements_parallel(profile, trace, classes, offsets, inst, budget, cla
     inst = np.asarray(inst, dtype=np.uint32)
     n_cand = len(offsets) - 1
     workers = workers or min(os.cpu_count() or 1, 32)
+    import sys
+    main = sys.modules.get("__main__")
+    if pool is None and not hasattr(main, "__file__"):
+        workers = 1   # a spawn pool cannot re-import a __main__ that came from stdin
     if n_cand < 2 * workers or workers <= 1:
         return eval_placements(profile, trace, classes, offsets, inst, budget, class_mask, flags)
     n_chunks = min(n_cand, workers * 8)

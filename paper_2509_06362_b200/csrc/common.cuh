@@ -16,6 +16,8 @@ constexpr long long kWaitCycles = 4000000000ll;  // bound on any device-side wai
 // 0..5: lane groups of 1,2,4,8,16,32 lanes (one lane per instance)
 // 6..8: block layout with 2, 8, 32 warps (one warp per instance, strided above 32)
 constexpr int kNumBuckets = 9;
+constexpr int kCostBins = 256;   // bin 0 = most expensive (largest total batch cap)
+constexpr int kCounterWords = 8192;  // counters | work counters | histograms + cursors, cleared per call
 constexpr int kGroupThreads = 128;
 
 struct Request {
@@ -123,6 +125,17 @@ __device__ __forceinline__ uint32_t ceil_div_steps(int64_t dt, uint32_t s) {
     return (uint32_t)(((uint64_t)dt - 1ull) / s) + 1u;
 }
 
+// ceil(dt / s) when the quotient is known to be below 2^16 and rs = 1/s rounded to float:
+// the float estimate is then within one of the true quotient and is fixed up exactly.
+__device__ __forceinline__ uint32_t ceil_div_small(int64_t dt, uint32_t s, float rs) {
+    if (((uint64_t)dt >> 32) != 0) return (uint32_t)(((uint64_t)dt - 1ull) / s) + 1u;
+    uint32_t q = (uint32_t)(__uint2float_rz((uint32_t)dt) * rs);
+    int64_t r = dt - (int64_t)q * (int64_t)s;
+    if (r < 0) { q--; r += s; }
+    else if (r >= (int64_t)s) { q++; r -= s; }
+    return q + (r > 0 ? 1u : 0u);
+}
+
 __device__ __forceinline__ int64_t prefill_us(uint32_t base, uint32_t q16, uint32_t in_tokens) {
     return (int64_t)base + (int64_t)(((uint64_t)q16 * in_tokens + 32768u) >> 16);
 }
@@ -194,8 +207,11 @@ struct EvalParams {
     uint32_t mapping;
     maaso_result* out;
     uint32_t* bucket_count;  // [kNumBuckets]
-    uint32_t* bucket_list;   // [kNumBuckets][n_cand]
+    uint32_t* bucket_list;   // [kNumBuckets][n_cand], each bucket sorted by decreasing cost estimate
     uint32_t* work_ctr;      // [4]
+    uint32_t* hist;          // [2][kNumBuckets][kCostBins]: candidates per cost bin, then write cursors
+    uint32_t* code;          // [n_cand] bucket << 8 | cost bin, 0xFFFFFFFF for invalid candidates
+    uint32_t group_warps;    // warps the lane-group grid keeps resident (capacity for promotions)
     int32_t* dump_row;       // [n_cand] or null
     uint32_t dump_n;
     int64_t* dump_finish;

@@ -130,12 +130,13 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
     const uint32_t n_tiles = (P.n_req + tile_recs - 1) / tile_recs;
     uint32_t tile_seq = 0;  // tiles consumed so far by this warp (same in every warp)
 
-    // how many work items each bucket contributes (largest groups first)
+    // how many work items (4 warps each) every bucket contributes (largest groups first)
     uint32_t items[6];
     uint32_t total_items = 0;
     for (int b = 5; b >= 0; b--) {
-        const uint32_t per = kGroupThreads >> b;
-        items[b] = (P.bucket_count[b] + per - 1) / per;
+        const uint32_t gpw = 32u >> b;                                 // groups per warp
+        const uint32_t n_warps = (P.bucket_count[b] + gpw - 1) / gpw;
+        items[b] = (n_warps + kWarps - 1) / kWarps;
         total_items += items[b];
     }
 
@@ -147,22 +148,26 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
         if (wi >= total_items) break;
         int b = 5;
         while (wi >= items[b]) { wi -= items[b]; b--; }
-        const uint32_t G = 1u << b, per = kGroupThreads >> b;
+        const uint32_t G = 1u << b;
         const uint32_t sub = tid & (G - 1u);
-        const uint32_t pos = wi * per + (tid >> b);
-        const bool valid = pos < P.bucket_count[b];
-        // neighbouring candidates of a sweep cost about the same; a multiplicative shuffle of the
-        // bucket order spreads the expensive ones over warps and blocks
+        // The bucket list is sorted by decreasing cost estimate.  Group slot j of warp x takes
+        // position j * n_warps + x: every warp gets one candidate of each cost quantile, so the
+        // expensive ones (whose events serialise inside a warp) are dealt one per warp, and the
+        // most expensive warps start first.
         const uint32_t cnt = P.bucket_count[b];
-        const uint32_t mult = (cnt % 1000003u) ? 1000003u : 999983u;
-        const uint32_t cand = valid ? P.bucket_list[(size_t)b * P.n_cand + (uint32_t)(((uint64_t)pos * mult) % cnt)] : 0u;
+        const uint32_t gpw = 32u >> b;
+        const uint32_t n_warps = (cnt + gpw - 1) / gpw;
+        const uint32_t warp_x = wi * kWarps + (tid >> 5);
+        const uint32_t pos = (lane >> b) * n_warps + warp_x;
+        const bool valid = warp_x < n_warps && pos < cnt;
+        const uint32_t cand = valid ? P.bucket_list[(size_t)b * P.n_cand + pos] : 0u;
         const uint32_t gmask = (G == 32u) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(G - 1u)));
 
         uint32_t n_i = 0, lo = 0;
         if (valid) { lo = P.offsets[cand]; n_i = P.offsets[cand + 1] - lo; }
         const bool has = valid && sub < n_i;
         LaneInst in;
-        in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = 0; in.sw = 1; in.mask = 0;
+        in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = 0; in.sw = 1; in.rsw = 1.0f; in.mask = 0;
         in.B = 1; in.model = 0xFFFFFFFFu; in.step = sm.steps; in.stepB = 1; in.pre_base = 0; in.pre_q16 = 0;
         if (has) {
             const uint32_t word = P.inst[lo + sub];
@@ -207,11 +212,14 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
             }
             const uint4* tile = sm.tiles + (size_t)s * tile_recs;
             const uint32_t recs = min((uint32_t)tile_recs, P.n_req - t * tile_recs);
+            uint4 raw_next = tile[0];
             for (uint32_t ri = 0; ri < recs; ri++) {
+                const uint4 raw = raw_next;
+                raw_next = tile[min(ri + 1, recs - 1)];  // read the next record ahead of its use
                 // All 32 lanes walk the trace together and every warp-level operation below uses
                 // the full mask (segmented by the group width), so the groups of a warp share one
                 // instruction stream; only events (retire, admit) diverge.
-                const Request q = decode_request(tile[ri]);
+                const Request q = decode_request(raw);
                 const uint32_t req = t * tile_recs + ri;
                 bool pending = valid && status == 0 && ((cmask >> (q.cls & 31u)) & 1u);
                 if (pending) {

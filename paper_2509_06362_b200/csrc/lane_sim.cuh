@@ -24,6 +24,7 @@ struct LaneInst {
     uint32_t B;       // batch cap = number of virtual slots
     uint32_t kmin;    // low 16 bits of the smallest completion index among running requests
     uint32_t sw;      // step[w-1]: length of one decode step at the current level (valid while w > 0)
+    float rsw;        // 1 / sw
     uint64_t mask;    // occupied slots
     const int32_t* step;  // shared-memory row: step[w-1] = one decode step with w running
     uint32_t stepB;   // step[B-1]
@@ -95,6 +96,7 @@ __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, St
     in.kmin = (K16 + nd) & 0xFFFFu;
     if (in.w > 0) {
         in.sw = (uint32_t)in.step[in.w - 1];
+        in.rsw = __frcp_rn((float)in.sw);
         in.tc = in.T + (int64_t)nd * (int64_t)in.sw;
     }
 }
@@ -109,7 +111,8 @@ __device__ __forceinline__ void lane_advance(LaneInst& in, int64_t now, bool dra
         if (!drain && now <= in.tc - (int64_t)in.sw) {
             // the clock reaches `now` before anything completes
             if (in.w < in.B) {
-                const uint32_t k = ceil_div_steps(now - in.T, in.sw);
+                // fewer than kfin <= 65535 steps: the quotient fits the fast exact division
+                const uint32_t k = ceil_div_small(now - in.T, in.sw, in.rsw);
                 in.T += (int64_t)k * (int64_t)in.sw;
                 in.K += k;
             }
@@ -168,6 +171,7 @@ __device__ __forceinline__ void lane_admit(LaneInst& in, const Request& q, uint3
     in.mask |= 1ull << slot;
     in.w++;
     in.sw = (uint32_t)in.step[in.w - 1];
+    in.rsw = __frcp_rn((float)in.sw);
     in.tc = in.T + (int64_t)((in.kmin - in.K) & 0xFFFFu) * (int64_t)in.sw;
 }
 

@@ -367,7 +367,8 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
 
     // scratch layout: counters | bucket lists | dump rows | payload
     size_t off = 0;
-    const size_t off_counters = off; off = align_up(off + 64 * 4, 256);
+    const size_t off_counters = off; off = align_up(off + kCounterWords * 4, 256);
+    const size_t off_code = off;     off = align_up(off + (size_t)C * 4, 256);
     const size_t off_lists = off;    off = align_up(off + (size_t)kNumBuckets * C * 4, 256);
     const size_t off_dump = off;     off = align_up(off + (o.dump_n ? (size_t)C * 4 : 0), 256);
     const size_t off_pay = off;      off = align_up(off + pay_entries * sizeof(Payload), 256);
@@ -376,11 +377,15 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     unsigned char* sb = static_cast<unsigned char*>(ctx->scratch);
     P.bucket_count = reinterpret_cast<uint32_t*>(sb + off_counters);
     P.work_ctr = P.bucket_count + 16;
+    P.hist = P.bucket_count + 64;
+    P.code = reinterpret_cast<uint32_t*>(sb + off_code);
     P.bucket_list = reinterpret_cast<uint32_t*>(sb + off_lists);
     P.dump_row = o.dump_n ? reinterpret_cast<int32_t*>(sb + off_dump) : nullptr;
     P.payload = reinterpret_cast<Payload*>(sb + off_pay);
 
-    cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, 64 * 4, stream);
+    static_assert(64 + 2 * kNumBuckets * kCostBins <= kCounterWords, "counter region");
+    P.group_warps = (uint32_t)grid_g * (kGroupThreads / 32);
+    cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, kCounterWords * 4, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "memset");
     int launches = 0;
     if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);

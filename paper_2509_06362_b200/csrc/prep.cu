@@ -8,7 +8,7 @@ __global__ void prep_kernel(const EvalParams P) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= P.n_cand) return;
     const uint32_t lo = P.offsets[c], hi = P.offsets[c + 1];
-    uint32_t status = 0, n = 0;
+    uint32_t status = 0, n = 0, sum_b = 0;
     if (hi < lo || hi > P.n_inst) {
         status = MAASO_CAND_EBADINST;  // malformed CSR row
     } else {
@@ -24,6 +24,7 @@ __global__ void prep_kernel(const EvalParams P) {
                     status |= MAASO_CAND_EBADINST;
                     continue;
                 }
+                sum_b += b;
                 devsum += (uint64_t)P.devices[s];
                 if (P.devices[s] < P.min_devices[m]) status |= MAASO_CAND_EMEMFIT;
             }
@@ -35,13 +36,66 @@ __global__ void prep_kernel(const EvalParams P) {
         uint4* o = reinterpret_cast<uint4*>(P.out + c);
         o[0] = make_uint4(status, 0, 0, 0);
         for (int i = 1; i < 8; i++) o[i] = make_uint4(0, 0, 0, 0);
+        P.code[c] = 0xFFFFFFFFu;
         return;
     }
     int b;
     if (P.mapping == MAASO_MAP_BLOCK) b = n <= 2 ? 6 : (n <= 8 ? 7 : 8);
     else if (n <= 32) b = n <= 1 ? 0 : 32 - __clz((int)(n - 1));
     else b = 8;
-    const uint32_t pos = atomicAdd(&P.bucket_count[b], 1u);
+    // Cost estimate: the total batch cap (how many requests the placement can have in flight;
+    // it tracks the number of served requests and so the number of simulation events).
+    const uint32_t bin = (kCostBins - 1) - min((uint32_t)(kCostBins - 1), sum_b / 8u);
+    atomicAdd(&P.bucket_count[b], 1u);
+    atomicAdd(&P.hist[b * kCostBins + bin], 1u);
+    P.code[c] = ((uint32_t)b << 8) | bin;
+}
+
+// One thread: (1) if the resident grid has warps to spare, promote the most expensive
+// candidates of the narrower lane-group buckets to a warp of their own (bucket 5) so that
+// their event handling is not serialised with other candidates' in the same warp; (2) turn
+// the per-bin histograms into write cursors (bins in decreasing cost order).
+__global__ void plan_kernel(const EvalParams P) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    uint32_t cut = 0;  // bins below `cut` are promoted
+    if (P.mapping != MAASO_MAP_BLOCK) {
+        uint32_t need = 0;
+        for (int b = 0; b <= 5; b++) need += (P.bucket_count[b] + (32u >> b) - 1) / (32u >> b);
+        uint32_t spare = P.group_warps > need ? P.group_warps - need : 0, promoted = 0;
+        for (int bin = 0; bin < kCostBins; bin++) {
+            uint32_t n = 0;
+            for (int b = 0; b < 5; b++) n += P.hist[b * kCostBins + bin];
+            if (promoted + n > spare) break;
+            promoted += n;
+            cut = bin + 1;
+        }
+    }
+    P.bucket_count[15] = cut;
+    for (int b = 0; b < kNumBuckets; b++) {
+        uint32_t run = 0;
+        for (int bin = 0; bin < kCostBins; bin++) {
+            uint32_t v = P.hist[b * kCostBins + bin];
+            if (b < 5 && (uint32_t)bin < cut) v = 0;
+            if (b == 5 && (uint32_t)bin < cut)
+                for (int o = 0; o < 5; o++) v += P.hist[o * kCostBins + bin];
+            // buckets are processed in increasing b, so the counts of buckets 0..4 are still intact
+            // when bucket 5 reads them; they are overwritten below only for the current bucket
+            P.hist[(kNumBuckets + b) * kCostBins + bin] = run;
+            run += v;
+        }
+        P.bucket_count[b] = run;
+    }
+}
+
+__global__ void scatter_kernel(const EvalParams P) {
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= P.n_cand) return;
+    const uint32_t code = P.code[c];
+    if (code == 0xFFFFFFFFu) return;
+    uint32_t b = code >> 8;
+    const uint32_t bin = code & 0xFFu;
+    if (b < 5 && bin < P.bucket_count[15]) b = 5;
+    const uint32_t pos = atomicAdd(&P.hist[(kNumBuckets + b) * kCostBins + bin], 1u);
     P.bucket_list[(size_t)b * P.n_cand + pos] = c;
 }
 
@@ -70,7 +124,9 @@ cudaError_t launch_prep(const EvalParams& P, const uint32_t* dump_idx, cudaStrea
         }
     }
     prep_kernel<<<(P.n_cand + 255) / 256, 256, 0, stream>>>(P);
-    (*launches)++;
+    plan_kernel<<<1, 32, 0, stream>>>(P);
+    scatter_kernel<<<(P.n_cand + 255) / 256, 256, 0, stream>>>(P);
+    (*launches) += 3;
     if (P.dump_n) {
         dump_map_kernel<<<(P.dump_n + 255) / 256, 256, 0, stream>>>(P, dump_idx);
         (*launches)++;
