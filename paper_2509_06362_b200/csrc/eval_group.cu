@@ -31,8 +31,11 @@ struct ArgMin {
 // of it the minimum is a 32-bit shuffle butterfly, otherwise a 64-bit one.
 __device__ __forceinline__ ArgMin group_argmin(uint64_t key, int64_t now, uint32_t gmask, uint32_t G) {
     // Called by all 32 lanes; every operation uses the full mask and stays inside the group
-    // because xor offsets are below the group width.
+    // because xor offsets are below the group width.  G may be smaller than the group (only the
+    // first G lanes hold instances): the result is then taken from the group's first lane.
     ArgMin r;
+    const int base = __ffs((int)gmask) - 1;
+    const bool narrow = G < 32u && ((gmask >> base) >> G) != 0;  // group wider than G
     const bool finite = key != kKeyInf;
     const uint64_t d = (key & ~(1ull << 63)) - (uint64_t)now;
     const bool wide = finite && d >= 0x7FFFFFFFull;
@@ -40,12 +43,14 @@ __device__ __forceinline__ ArgMin group_argmin(uint64_t key, int64_t now, uint32
         const uint32_t k32 = finite ? ((uint32_t)(key >> 63) << 31) | (uint32_t)d : 0xFFFFFFFFu;
         uint32_t best = k32;
         for (uint32_t off = 1; off < G; off <<= 1) best = min(best, __shfl_xor_sync(0xFFFFFFFFu, best, (int)off));
+        if (narrow) best = __shfl_sync(0xFFFFFFFFu, best, base);
         r.found = best != 0xFFFFFFFFu;
         r.tier = best >> 31;
         r.winner = __ffs((int)(__ballot_sync(0xFFFFFFFFu, k32 == best) & gmask)) - 1;
     } else {
         uint64_t best = key;
         for (uint32_t off = 1; off < G; off <<= 1) best = min(best, shfl_xor_u64(best, (int)off, 0xFFFFFFFFu));
+        if (narrow) best = shfl_u64(best, base, 0xFFFFFFFFu);
         r.found = best != kKeyInf;
         r.tier = (uint32_t)(best >> 63);
         r.winner = __ffs((int)(__ballot_sync(0xFFFFFFFFu, key == best) & gmask)) - 1;
@@ -179,6 +184,10 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
             in.pre_base = (uint32_t)P.rows[row * kRowStride + 0];
             in.pre_q16 = (uint32_t)P.rows[row * kRowStride + 1];
         }
+        // A warp that holds a single candidate (bucket 5, possibly promoted there with few
+        // instances) only needs as many butterfly rounds as it has instances.
+        const uint32_t n_i_warp = __shfl_sync(0xFFFFFFFFu, n_i, 0);
+        const uint32_t Geff = b == 5 ? (n_i_warp <= 1 ? 1u : 1u << (32 - __clz((int)(n_i_warp - 1)))) : G;
         const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
         Dump dump{nullptr, nullptr, nullptr};
         if (valid) dump = dump_for(P, cand);
@@ -238,12 +247,12 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                     if (pending) {
                         attempts++;
                         tries++;
-                        if (elig) {
-                            lane_advance(in, now, false, env, st);
-                            key = lane_predict(in, q, pre, lim_ttft, lim_tbt, lim_e2e, OPT, t0);
-                        }
                     }
-                    const ArgMin am = group_argmin(key, now, gmask, G);
+                    if (pending && elig) {
+                        lane_advance(in, now, false, env, st);
+                        key = lane_predict(in, q, pre, lim_ttft, lim_tbt, lim_e2e, OPT, t0);
+                    }
+                    const ArgMin am = group_argmin(key, now, gmask, Geff);
                     const int64_t t0w = (int64_t)shfl_u64((uint64_t)t0, am.winner, 0xFFFFFFFFu);
                     if (pending) {
                         if (!am.found) {
