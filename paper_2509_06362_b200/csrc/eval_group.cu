@@ -27,35 +27,18 @@ struct ArgMin {
 };
 
 // Distributor's choice inside a lane group: smallest (tier, predicted first token), lowest lane
-// among equals.  Predicted times are at or after `now`; when every finite key is within 2^31 us
-// of it the minimum is a 32-bit shuffle butterfly, otherwise a 64-bit one.
-__device__ __forceinline__ ArgMin group_argmin(uint64_t key, int64_t now, uint32_t gmask, uint32_t G) {
-    // Called by all 32 lanes; every operation uses the full mask and stays inside the group
-    // because xor offsets are below the group width.  G may be smaller than the group (only the
-    // first G lanes hold instances): the result is then taken from the group's first lane.
+// among equals.  Called by all 32 lanes; every operation uses the full mask and stays inside
+// the group because xor offsets are below G.  G may be smaller than the group when only its
+// first G lanes hold instances: the other lanes then see "nothing found", which is harmless
+// because only lanes with instances and the group's first lane act on the result.
+__device__ __forceinline__ ArgMin group_argmin(uint64_t key, uint32_t gmask, uint32_t G) {
     ArgMin r;
-    const int base = __ffs((int)gmask) - 1;
-    const bool narrow = G < 32u && ((gmask >> base) >> G) != 0;  // group wider than G
-    const bool finite = key != kKeyInf;
-    const uint64_t d = (key & ~(1ull << 63)) - (uint64_t)now;
-    const bool wide = finite && d >= 0x7FFFFFFFull;
-    if (!__any_sync(0xFFFFFFFFu, wide)) {
-        const uint32_t k32 = finite ? ((uint32_t)(key >> 63) << 31) | (uint32_t)d : 0xFFFFFFFFu;
-        uint32_t best = k32;
-        for (uint32_t off = 1; off < G; off <<= 1) best = min(best, __shfl_xor_sync(0xFFFFFFFFu, best, (int)off));
-        if (narrow) best = __shfl_sync(0xFFFFFFFFu, best, base);
-        r.found = best != 0xFFFFFFFFu;
-        r.tier = best >> 31;
-        r.winner = __ffs((int)(__ballot_sync(0xFFFFFFFFu, k32 == best) & gmask)) - 1;
-    } else {
-        uint64_t best = key;
-        for (uint32_t off = 1; off < G; off <<= 1) best = min(best, shfl_xor_u64(best, (int)off, 0xFFFFFFFFu));
-        if (narrow) best = shfl_u64(best, base, 0xFFFFFFFFu);
-        r.found = best != kKeyInf;
-        r.tier = (uint32_t)(best >> 63);
-        r.winner = __ffs((int)(__ballot_sync(0xFFFFFFFFu, key == best) & gmask)) - 1;
-    }
-    if (!r.found) r.winner = (int)(threadIdx.x & 31u);  // any valid source lane for the shuffle that follows
+    uint64_t best = key;
+    for (uint32_t off = 1; off < G; off <<= 1) best = min(best, shfl_xor_u64(best, (int)off, 0xFFFFFFFFu));
+    r.found = best != kKeyInf;
+    r.tier = (uint32_t)(best >> 63);
+    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, key == best) & gmask;
+    r.winner = r.found ? __ffs((int)votes) - 1 : (int)(threadIdx.x & 31u);
     return r;
 }
 
@@ -172,7 +155,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
         if (valid) { lo = P.offsets[cand]; n_i = P.offsets[cand + 1] - lo; }
         const bool has = valid && sub < n_i;
         LaneInst in;
-        in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = 0; in.sw = 1; in.rsw = 1.0f; in.mask = 0;
+        in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = 0; in.sw = 1; in.rsw = 1.0f; in.bslots = 0; in.mask = 0;
         in.B = 1; in.model = 0xFFFFFFFFu; in.step = sm.steps; in.stepB = 1; in.pre_base = 0; in.pre_q16 = 0;
         if (has) {
             const uint32_t word = P.inst[lo + sub];
@@ -252,7 +235,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                         lane_advance(in, now, false, env, st);
                         key = lane_predict(in, q, pre, lim_ttft, lim_tbt, lim_e2e, OPT, t0);
                     }
-                    const ArgMin am = group_argmin(key, now, gmask, Geff);
+                    const ArgMin am = group_argmin(key, gmask, Geff);
                     const int64_t t0w = (int64_t)shfl_u64((uint64_t)t0, am.winner, 0xFFFFFFFFu);
                     if (pending) {
                         if (!am.found) {

@@ -25,6 +25,7 @@ struct LaneInst {
     uint32_t kmin;    // low 16 bits of the smallest completion index among running requests
     uint32_t sw;      // step[w-1]: length of one decode step at the current level (valid while w > 0)
     float rsw;        // 1 / sw
+    uint32_t bslots;  // 3 bits per block: which of its 8 slots holds the block minimum
     uint64_t mask;    // occupied slots
     const int32_t* step;  // shared-memory row: step[w-1] = one decode step with w running
     uint32_t stepB;   // step[B-1]
@@ -41,6 +42,11 @@ struct LaneEnv {
     Dump dump;
 };
 
+// Bring the payload of the request that will complete next into L1 ahead of its use.
+__device__ __forceinline__ void prefetch_l1(const void* p) {
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
+}
+
 __device__ __forceinline__ uint32_t half_of(const uint4& v, int j) {  // j static after unrolling
     const uint32_t word = (j >> 1) == 0 ? v.x : ((j >> 1) == 1 ? v.y : ((j >> 1) == 2 ? v.z : v.w));
     return (j & 1) ? (word >> 16) : (word & 0xFFFFu);
@@ -51,30 +57,32 @@ __device__ __forceinline__ uint32_t half_of(const uint4& v, int j) {  // j stati
 __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, Stats& st) {
     const uint32_t K16 = in.K & 0xFFFFu;
     const uint4 bm = *reinterpret_cast<const uint4*>(env.keys + 64);
-    uint32_t hit_blocks = 0, nd = 0x10000u;
+    uint32_t hit_blocks = 0, nd = 0x10000u, nb = 0;
 #pragma unroll
-    for (int b = 0; b < 8; b++) {
-        const uint32_t occ = (uint32_t)(in.mask >> (8 * b)) & 0xFFu;
-        const uint32_t d = (half_of(bm, b) - K16) & 0xFFFFu;
-        if (occ) {
-            if (d == 0) hit_blocks |= 1u << b;
-            else nd = min(nd, d);
-        }
+    for (int b = 0; b < 8; b++) {  // branch-free: empty blocks count as infinitely far
+        const bool occ = ((uint32_t)(in.mask >> (8 * b)) & 0xFFu) != 0;
+        const uint32_t d = occ ? ((half_of(bm, b) - K16) & 0xFFFFu) : 0x10000u;
+        hit_blocks |= (d == 0 ? 1u : 0u) << b;
+        const uint32_t dd = d == 0 ? 0x10000u : d;
+        nb = dd < nd ? (uint32_t)b : nb;
+        nd = min(nd, dd);
     }
     while (hit_blocks) {
         const int b = __ffs((int)hit_blocks) - 1;
         hit_blocks &= hit_blocks - 1;
         const uint32_t occ = (uint32_t)(in.mask >> (8 * b)) & 0xFFu;
         const uint4 kv = *reinterpret_cast<const uint4*>(env.keys + 8 * b);
-        uint32_t done = 0, bd = 0x10000u;
+        uint32_t done = 0, bd = 0x10000u, bj = 0;
 #pragma unroll
         for (int j = 0; j < 8; j++) {
-            const uint32_t d = (half_of(kv, j) - K16) & 0xFFFFu;
-            if ((occ >> j) & 1u) {
-                if (d == 0) done |= 1u << j;
-                else bd = min(bd, d);
-            }
+            const uint32_t d = ((occ >> j) & 1u) ? ((half_of(kv, j) - K16) & 0xFFFFu) : 0x10000u;
+            done |= (d == 0 ? 1u : 0u) << j;
+            const uint32_t dd = d == 0 ? 0x10000u : d;
+            bj = dd < bd ? (uint32_t)j : bj;
+            bd = min(bd, dd);
         }
+        in.bslots = (in.bslots & ~(7u << (3 * b))) | (bj << (3 * b));
+        nb = bd < nd ? (uint32_t)b : nb;
         in.mask &= ~((uint64_t)done << (8 * b));
         in.w -= __popc(done);
         env.keys[64 + b] = (uint16_t)(K16 + bd);
@@ -98,6 +106,7 @@ __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, St
         in.sw = (uint32_t)in.step[in.w - 1];
         in.rsw = __frcp_rn((float)in.sw);
         in.tc = in.T + (int64_t)nd * (int64_t)in.sw;
+        prefetch_l1(env.pay + 8 * nb + ((in.bslots >> (3 * nb)) & 7u));
     }
 }
 
@@ -166,8 +175,14 @@ __device__ __forceinline__ void lane_admit(LaneInst& in, const Request& q, uint3
     env.keys[slot] = (uint16_t)key;
     store_payload(env.pay + slot, in.T, q.arrival, req, q.S, q.cls);
     const uint32_t occ = (uint32_t)(in.mask >> (8 * b)) & 0xFFu;
-    if (occ == 0 || dist < (((uint32_t)env.keys[64 + b] - in.K) & 0xFFFFu)) env.keys[64 + b] = (uint16_t)key;
-    if (in.w == 0 || dist < ((in.kmin - in.K) & 0xFFFFu)) in.kmin = key;
+    if (occ == 0 || dist < (((uint32_t)env.keys[64 + b] - in.K) & 0xFFFFu)) {
+        env.keys[64 + b] = (uint16_t)key;
+        in.bslots = (in.bslots & ~(7u << (3 * b))) | ((uint32_t)(slot & 7) << (3 * b));
+    }
+    if (in.w == 0 || dist < ((in.kmin - in.K) & 0xFFFFu)) {
+        in.kmin = key;
+        prefetch_l1(env.pay + slot);
+    }
     in.mask |= 1ull << slot;
     in.w++;
     in.sw = (uint32_t)in.step[in.w - 1];

@@ -51,40 +51,48 @@ __global__ void prep_kernel(const EvalParams P) {
     P.code[c] = ((uint32_t)b << 8) | bin;
 }
 
-// One thread: (1) if the resident grid has warps to spare, promote the most expensive
-// candidates of the narrower lane-group buckets to a warp of their own (bucket 5) so that
-// their event handling is not serialised with other candidates' in the same warp; (2) turn
-// the per-bin histograms into write cursors (bins in decreasing cost order).
-__global__ void plan_kernel(const EvalParams P) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+// One block, one thread per cost bin: (1) if the resident grid has warps to spare, promote
+// the most expensive candidates of the narrower lane-group buckets to a warp of their own
+// (bucket 5) so that their event handling is not serialised with other candidates' in the
+// same warp; (2) turn the per-bin histograms into write cursors (bins in decreasing cost order).
+__device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t v, uint32_t* buf) {
+    const int t = threadIdx.x;
+    buf[t] = v;
+    __syncthreads();
+    for (int off = 1; off < kCostBins; off <<= 1) {
+        const uint32_t add = t >= off ? buf[t - off] : 0u;
+        __syncthreads();
+        buf[t] += add;
+        __syncthreads();
+    }
+    const uint32_t r = buf[t];
+    __syncthreads();
+    return r;
+}
+
+__global__ void __launch_bounds__(kCostBins) plan_kernel(const EvalParams P) {
+    __shared__ uint32_t buf[kCostBins];
+    const int bin = threadIdx.x;
     uint32_t cut = 0;  // bins below `cut` are promoted
+    uint32_t narrow = 0;
+    for (int b = 0; b < 5; b++) narrow += P.hist[b * kCostBins + bin];
     if (P.mapping != MAASO_MAP_BLOCK) {
         uint32_t need = 0;
         for (int b = 0; b <= 5; b++) need += (P.bucket_count[b] + (32u >> b) - 1) / (32u >> b);
-        uint32_t spare = P.group_warps > need ? P.group_warps - need : 0, promoted = 0;
-        for (int bin = 0; bin < kCostBins; bin++) {
-            uint32_t n = 0;
-            for (int b = 0; b < 5; b++) n += P.hist[b * kCostBins + bin];
-            if (promoted + n > spare) break;
-            promoted += n;
-            cut = bin + 1;
-        }
+        const uint32_t spare = P.group_warps > need ? P.group_warps - need : 0;
+        const uint32_t incl = block_inclusive_scan(narrow, buf);
+        cut = (uint32_t)__syncthreads_count(incl <= spare);  // prefix sums are monotone
     }
-    P.bucket_count[15] = cut;
+    __syncthreads();
     for (int b = 0; b < kNumBuckets; b++) {
-        uint32_t run = 0;
-        for (int bin = 0; bin < kCostBins; bin++) {
-            uint32_t v = P.hist[b * kCostBins + bin];
-            if (b < 5 && (uint32_t)bin < cut) v = 0;
-            if (b == 5 && (uint32_t)bin < cut)
-                for (int o = 0; o < 5; o++) v += P.hist[o * kCostBins + bin];
-            // buckets are processed in increasing b, so the counts of buckets 0..4 are still intact
-            // when bucket 5 reads them; they are overwritten below only for the current bucket
-            P.hist[(kNumBuckets + b) * kCostBins + bin] = run;
-            run += v;
-        }
-        P.bucket_count[b] = run;
+        uint32_t v = P.hist[b * kCostBins + bin];
+        if (b < 5 && (uint32_t)bin < cut) v = 0;
+        if (b == 5 && (uint32_t)bin < cut) v += narrow;
+        const uint32_t incl = block_inclusive_scan(v, buf);
+        P.hist[(kNumBuckets + b) * kCostBins + bin] = incl - v;
+        if (bin == kCostBins - 1) P.bucket_count[b] = incl;
     }
+    if (bin == 0) P.bucket_count[15] = cut;
 }
 
 __global__ void scatter_kernel(const EvalParams P) {
@@ -124,7 +132,7 @@ cudaError_t launch_prep(const EvalParams& P, const uint32_t* dump_idx, cudaStrea
         }
     }
     prep_kernel<<<(P.n_cand + 255) / 256, 256, 0, stream>>>(P);
-    plan_kernel<<<1, 32, 0, stream>>>(P);
+    plan_kernel<<<1, kCostBins, 0, stream>>>(P);
     scatter_kernel<<<(P.n_cand + 255) / 256, 256, 0, stream>>>(P);
     (*launches) += 3;
     if (P.dump_n) {
