@@ -212,6 +212,9 @@ struct EvalParams {
     uint32_t* hist;          // [2][kNumBuckets][kCostBins]: candidates per cost bin, then write cursors
     uint32_t* code;          // [n_cand] bucket << 8 | cost bin, 0xFFFFFFFF for invalid candidates
     uint32_t group_warps;    // warps the lane-group grid keeps resident (capacity for promotions)
+    uint32_t* sm_ctr;        // [n_sm] next work item of each SM's share (lane-group kernel)
+    uint32_t n_sm;
+    uint32_t promote_pct;
     int32_t* dump_row;       // [n_cand] or null
     uint32_t dump_n;
     int64_t* dump_finish;

@@ -130,7 +130,26 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
 
     for (;;) {
         __syncthreads();  // everyone is done with the previous batch (tiles, work slot)
-        if (tid == 0) sm.work[0] = sm.work[1] ? 0xFFFFFFFFu : atomicAdd(P.work_ctr, 1u);
+        if (tid == 0) {
+            // Work items are ordered from expensive to cheap.  SM s owns items s, s + n_sm, ...:
+            // every SM gets the same share of each cost class however blocks were placed; a
+            // block whose SM has run out takes from the other SMs' shares.
+            uint32_t item = 0xFFFFFFFFu;
+            if (!sm.work[1]) {
+                uint32_t my_sm;
+                asm volatile("mov.u32 %0, %%smid;" : "=r"(my_sm));
+                for (uint32_t k = 0; k < P.n_sm && item == 0xFFFFFFFFu; k++) {
+                    const uint32_t s = (my_sm + k) % P.n_sm;
+                    if (*(volatile uint32_t*)&P.sm_ctr[s] * P.n_sm >= total_items) continue;  // exhausted
+                    // snake order: odd rounds run backwards, so the SM that got the most expensive
+                    // item of one round gets the cheapest of the next
+                    const uint32_t j = atomicAdd(&P.sm_ctr[s], 1u);
+                    const uint32_t it = j * P.n_sm + ((j & 1u) ? P.n_sm - 1u - s : s);
+                    if (it < total_items) item = it;
+                }
+            }
+            sm.work[0] = item;
+        }
         __syncthreads();
         uint32_t wi = sm.work[0];
         if (wi >= total_items) break;

@@ -51,6 +51,7 @@ struct maaso_ctx {
     cudaStream_t own_stream;
     uint64_t launches;
     int tile_recs;
+    int promote_pct;  // share of the spare resident warps the planner may use for promotions
     bool timing;
     cudaEvent_t ev[6];   // eval: start, after prep, after group, after block; topk: start, end
     bool ev_eval, ev_topk;
@@ -138,6 +139,12 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
     if (e != cudaSuccess) {
         delete ctx;
         return cuda_fail(nullptr, e, "cudaStreamCreate");
+    }
+    ctx->promote_pct = 100;
+    const char* pp = getenv("MAASO_PROMOTE_PCT");
+    if (pp) {
+        int v = atoi(pp);
+        if (v >= 0 && v <= 100) ctx->promote_pct = v;
     }
     const char* env = getenv("MAASO_TILE_RECS");
     if (env) {
@@ -378,13 +385,16 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.bucket_count = reinterpret_cast<uint32_t*>(sb + off_counters);
     P.work_ctr = P.bucket_count + 16;
     P.hist = P.bucket_count + 64;
+    P.sm_ctr = P.hist + 2 * kNumBuckets * kCostBins;
+    P.n_sm = (uint32_t)(ctx->sm_count < 1024 ? ctx->sm_count : 1024);
     P.code = reinterpret_cast<uint32_t*>(sb + off_code);
     P.bucket_list = reinterpret_cast<uint32_t*>(sb + off_lists);
     P.dump_row = o.dump_n ? reinterpret_cast<int32_t*>(sb + off_dump) : nullptr;
     P.payload = reinterpret_cast<Payload*>(sb + off_pay);
 
-    static_assert(64 + 2 * kNumBuckets * kCostBins <= kCounterWords, "counter region");
+    static_assert(64 + 2 * kNumBuckets * kCostBins + 1024 <= kCounterWords, "counter region");
     P.group_warps = (uint32_t)grid_g * (kGroupThreads / 32);
+    P.promote_pct = (uint32_t)ctx->promote_pct;
     cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, kCounterWords * 4, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "memset");
     int launches = 0;

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(kCostBins) plan_kernel(const EvalParams P) {
     if (P.mapping != MAASO_MAP_BLOCK) {
         uint32_t need = 0;
         for (int b = 0; b <= 5; b++) need += (P.bucket_count[b] + (32u >> b) - 1) / (32u >> b);
-        const uint32_t spare = P.group_warps > need ? P.group_warps - need : 0;
+        const uint32_t spare = P.group_warps > need ? (uint32_t)((uint64_t)(P.group_warps - need) * P.promote_pct / 100) : 0;
         const uint32_t incl = block_inclusive_scan(narrow, buf);
         cut = (uint32_t)__syncthreads_count(incl <= spare);  // prefix sums are monotone
     }
