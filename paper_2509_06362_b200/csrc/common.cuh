@@ -193,6 +193,7 @@ struct EvalParams {
     uint32_t n_req;
     uint32_t n_classes;
     const int64_t* classes;  // [n_classes][3]
+    const uint64_t* rej_hash;  // [n_req] checksum term of "request r was rejected" (same for every candidate)
     const int32_t* rows;     // [n_rows][kRowStride]
     const int32_t* devices;
     const int32_t* min_devices;

@@ -45,7 +45,8 @@ __device__ __forceinline__ ArgMin group_argmin(uint64_t key, uint32_t gmask, uin
 struct GroupSmem {
     uint4* tiles;        // [kStages][tile_recs]
     int32_t* steps;      // [n_rows][64]
-    int64_t* classes;    // [n_classes][3]
+    int64_t* classes;    // [n_classes][3], negative = no limit (completion accounting)
+    int64_t* plimits;    // [n_classes][3], INT64_MAX = no limit (distributor prediction)
     uint16_t* keys;      // [kGroupThreads][kKeyStride]
     uint32_t* hbc;       // [kGroupThreads][8]
     uint64_t* full_bar;  // [kStages]
@@ -56,7 +57,7 @@ struct GroupSmem {
 __host__ __device__ inline size_t group_smem_bytes(uint32_t n_rows, uint32_t n_classes, int tile_recs) {
     size_t b = (size_t)kStages * tile_recs * 16;
     b += (size_t)n_rows * 64 * 4;
-    b += (size_t)n_classes * 24;
+    b += (size_t)n_classes * 48;
     b += (size_t)kGroupThreads * kKeyStride * 2;
     b += (size_t)kGroupThreads * 8 * 4;
     b += kStages * 8 + kStages * 4 + 8 + 32;
@@ -74,6 +75,8 @@ __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows,
     s.hbc = reinterpret_cast<uint32_t*>(base);
     base += (size_t)kGroupThreads * 8 * 4;
     s.classes = reinterpret_cast<int64_t*>(base);
+    base += (size_t)n_classes * 24;
+    s.plimits = reinterpret_cast<int64_t*>(base);
     base += (size_t)n_classes * 24;
     s.full_bar = reinterpret_cast<uint64_t*>(base);
     base += kStages * 8;
@@ -97,7 +100,11 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
     // profile residency: decode-step tables and SLO classes into shared memory
     for (uint32_t i = tid; i < P.n_rows * 64u; i += kGroupThreads)
         sm.steps[i] = P.rows[(i >> 6) * kRowStride + 2 + (i & 63u)];
-    for (uint32_t i = tid; i < P.n_classes * 3u; i += kGroupThreads) sm.classes[i] = P.classes[i];
+    for (uint32_t i = tid; i < P.n_classes * 3u; i += kGroupThreads) {
+        const int64_t v = P.classes[i];
+        sm.classes[i] = v;
+        sm.plimits[i] = v < 0 ? INT64_MAX : v;
+    }
     if (tid == 0) {
         for (int s = 0; s < kStages; s++) {
             mbar_init(&sm.full_bar[s], 1);
@@ -239,9 +246,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                 }
                 const int64_t pre = prefill_us(in.pre_base, in.pre_q16, q.in_tokens);
                 const bool elig = has && in.model == q.model;
-                const int64_t lim_ttft = sm.classes[q.cls * 3 + 0];
-                const int64_t lim_tbt = sm.classes[q.cls * 3 + 1];
-                const int64_t lim_e2e = sm.classes[q.cls * 3 + 2];
+                const int64_t lim_ttft = sm.plimits[q.cls * 3 + 0];
+                const int64_t lim_tbt = sm.plimits[q.cls * 3 + 1];
+                const int64_t lim_e2e = sm.plimits[q.cls * 3 + 2];
                 uint32_t tries = 0;
                 do {
                     uint64_t key = kKeyInf;
@@ -261,7 +268,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                             // overflow protection: nobody can meet the deadline -> rejected
                             n_rejected++;
                             if (sub == 0) {
-                                st.checksum += rejected_hash(req);
+                                st.checksum += __ldg(P.rej_hash + req);
                                 if (dump.finish) dump.finish[req] = -1;
                                 if (dump.first) dump.first[req] = -1;
                                 if (dump.inst) dump.inst[req] = -1;

@@ -136,7 +136,8 @@ __device__ __forceinline__ void lane_advance(LaneInst& in, int64_t now, bool dra
 
 // Distributor prediction for one instance (Sec. IV-F steps 2-3).  Returns the 64-bit
 // choice key (tier << 63 | predicted first-token time) or kKeyInf if the request cannot
-// meet its SLO there; t0 = time the request could start its prefill.
+// meet its SLO there; t0 = time the request could start its prefill.  Limits: "no limit" is
+// passed as INT64_MAX here (all compared quantities are far below it).
 __device__ __forceinline__ uint64_t lane_predict(const LaneInst& in, const Request& q, int64_t pre,
                                                  int64_t lim_ttft, int64_t lim_tbt, int64_t lim_e2e,
                                                  bool optimistic, int64_t& t0) {
@@ -152,9 +153,7 @@ __device__ __forceinline__ uint64_t lane_predict(const LaneInst& in, const Reque
     }
     const int64_t first = t0 + pre;
     const int64_t fin = first + (int64_t)(q.S - 1) * sB;
-    const bool ok = (lim_ttft < 0 || first - q.arrival <= lim_ttft) &&
-                    (lim_tbt < 0 || q.S == 1 || sB <= lim_tbt) &&
-                    (lim_e2e < 0 || fin - q.arrival <= lim_e2e);
+    const bool ok = first - q.arrival <= lim_ttft && (q.S == 1 || sB <= lim_tbt) && fin - q.arrival <= lim_e2e;
     return ok ? ((tier << 63) | (uint64_t)first) : kKeyInf;
 }
 

@@ -11,6 +11,7 @@
 
 namespace maaso {
 cudaError_t launch_prep(const EvalParams& P, const uint32_t* dump_idx, cudaStream_t stream, int* launches);
+cudaError_t launch_rej_hash(uint64_t* out, uint32_t n);
 cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, cudaStream_t stream);
 int occupancy_eval_group(const EvalParams& P, int tile_recs);
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
@@ -27,6 +28,7 @@ struct maaso_trace {
     maaso_ctx* owner;
     uint4* d_reqs;
     int64_t* d_classes;
+    uint64_t* d_rej_hash;
     uint64_t n;
     uint32_t n_classes;
     uint32_t max_model;
@@ -166,6 +168,7 @@ MAASO_API void maaso_free_trace(maaso_ctx* ctx, maaso_trace* trace) {
         }
     if (trace->d_reqs) cudaFree(trace->d_reqs);
     if (trace->d_classes) cudaFree(trace->d_classes);
+    if (trace->d_rej_hash) cudaFree(trace->d_rej_hash);
     delete trace;
 }
 
@@ -284,11 +287,15 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     t->owner = ctx;
     t->d_reqs = nullptr;
     t->d_classes = nullptr;
+    t->d_rej_hash = nullptr;
     t->n = n;
     t->n_classes = n_classes;
     t->max_model = max_model;
     cudaError_t e = cudaMalloc(&t->d_reqs, (n ? n : 1) * sizeof(maaso_request));
     if (e == cudaSuccess) e = cudaMalloc(&t->d_classes, cls.size() * 8);
+    if (e == cudaSuccess) e = cudaMalloc(&t->d_rej_hash, (n ? n : 1) * 8);
+    if (e == cudaSuccess) e = launch_rej_hash(t->d_rej_hash, (uint32_t)n);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e == cudaSuccess && n)
         e = cudaMemcpy(t->d_reqs, reqs, n * sizeof(maaso_request),
                        on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice);
@@ -296,6 +303,7 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     if (e != cudaSuccess) {
         if (t->d_reqs) cudaFree(t->d_reqs);
         if (t->d_classes) cudaFree(t->d_classes);
+        if (t->d_rej_hash) cudaFree(t->d_rej_hash);
         delete t;
         return cuda_fail(ctx, e, "trace upload");
     }
@@ -333,6 +341,7 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.n_req = (uint32_t)trace->n;
     P.n_classes = trace->n_classes;
     P.classes = trace->d_classes;
+    P.rej_hash = trace->d_rej_hash;
     P.rows = ctx->d_rows;
     P.devices = ctx->d_devices;
     P.min_devices = ctx->d_min_devices;

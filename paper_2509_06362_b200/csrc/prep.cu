@@ -122,6 +122,16 @@ __global__ void dump_fill_kernel(int64_t* finish, int64_t* first, int32_t* inst,
     }
 }
 
+// The checksum term of a rejected request depends on the request alone: computed once per trace.
+__global__ void rej_hash_kernel(uint64_t* out, uint32_t n) {
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < n) out[r] = rejected_hash(r);
+}
+cudaError_t launch_rej_hash(uint64_t* out, uint32_t n) {
+    if (n) rej_hash_kernel<<<(n + 255) / 256, 256>>>(out, n);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_prep(const EvalParams& P, const uint32_t* dump_idx, cudaStream_t stream, int* launches) {
     if (P.dump_n) {
         const size_t n = (size_t)P.dump_n * P.n_req;
