@@ -49,6 +49,8 @@ def _load():
         _lib = C.CDLL(build())
         _lib.orc_eval_batch.restype = C.c_int
         _lib.orc_topk.restype = C.c_int
+        _lib.orc_score.restype = C.c_int
+        _lib.orc_topk_scores.restype = C.c_int
     return _lib
 
 
@@ -145,6 +147,33 @@ def eval_placements_parallel(profile, trace, classes, offsets, inst, budget, cla
             pool.close()
             pool.join()
     return np.concatenate(parts)
+
+
+class _ScoreParams(C.Structure):
+    _fields_ = [("alpha", C.c_double), ("beta", C.c_double), ("gamma_t", C.c_double), ("gamma_l", C.c_double)]
+
+
+def score(results, alpha, beta, gamma_t, gamma_l):
+    """Composite serving score of every record (see orc_score)."""
+    lib = _load()
+    results = np.ascontiguousarray(results, dtype=_RES)
+    out = np.zeros(len(results), dtype=np.float64)
+    p = _ScoreParams(alpha, beta, gamma_t, gamma_l)
+    rc = lib.orc_score(_ptr(results), C.c_uint64(len(results)), C.byref(p), _ptr(out))
+    if rc != 0:
+        raise RuntimeError(f"oracle score failed with code {rc}")
+    return out
+
+
+def topk_scores(scores, k):
+    """Indices of the k highest scores, ties to the lower index, NaN last."""
+    lib = _load()
+    scores = np.ascontiguousarray(scores, dtype=np.float64)
+    out = np.zeros(min(k, len(scores)), dtype=np.uint32)
+    rc = lib.orc_topk_scores(_ptr(scores), C.c_uint64(len(scores)), C.c_uint32(k), _ptr(out))
+    if rc != 0:
+        raise RuntimeError(f"oracle topk_scores failed with code {rc}")
+    return out
 
 
 def topk(results, k, order=0):

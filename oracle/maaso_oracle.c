@@ -358,6 +358,65 @@ int orc_eval_batch(const orc_profile *p, const orc_request *reqs, uint64_t n, co
 }
 
 /*
+ * Composite serving score of Sec. IV-D:
+ *   Phi = alpha * PhiS_n + beta * PhiT_n + (1 - beta) * PhiL_n
+ *   PhiS_n = SLO satisfaction ratio            = n_hit / n_counted
+ *   PhiT_n = min(PhiT, gamma_T) / gamma_T      PhiT = decoding throughput = tokens / makespan [tokens/s]
+ *   PhiL_n = max(gamma_L - PhiL, 0) / gamma_L  PhiL = response latency = mean time to first token [s]
+ * ("Evaluation Metrics", Sec. V-A, define throughput and response latency).
+ * Readings: a placement that counted no request has PhiS_n = 0; one that served nothing has
+ * PhiT_n = PhiL_n = 0; an invalid candidate scores -1.  Plain IEEE double arithmetic in the
+ * order written, no fused operations.
+ */
+typedef struct { double alpha, beta, gamma_t, gamma_l; } orc_score_params;
+
+int orc_score(const orc_result *res, uint64_t n, const orc_score_params *p, double *out) {
+    for (uint64_t i = 0; i < n; i++) {
+        const orc_result *r = &res[i];
+        if (r->status != 0) { out[i] = -1.0; continue; }
+        double phis = 0.0, phit = 0.0, phil = 0.0;
+        if (r->n_counted > 0) phis = (double)r->n_hit / (double)r->n_counted;
+        if (r->n_served > 0 && r->makespan_us > 0) {
+            double thr = (double)r->tokens_out / ((double)r->makespan_us * 1e-6);
+            double capped = thr < p->gamma_t ? thr : p->gamma_t;
+            phit = capped / p->gamma_t;
+        }
+        if (r->n_served > 0) {
+            double lat = ((double)r->sum_ttft_us / (double)r->n_served) * 1e-6;
+            double room = p->gamma_l - lat;
+            if (room < 0.0) room = 0.0;
+            phil = room / p->gamma_l;
+        }
+        double a = p->alpha * phis;
+        double b = p->beta * phit;
+        double c = (1.0 - p->beta) * phil;
+        out[i] = (a + b) + c;
+    }
+    return 0;
+}
+
+/* Ranking by score (order 1): higher score first, then lower index; NaN scores last. */
+static const double *g_score;
+static int cmp_score(const void *pa, const void *pb) {
+    uint32_t a = *(const uint32_t *)pa, b = *(const uint32_t *)pb;
+    double x = g_score[a], y = g_score[b];
+    int nx = x != x, ny = y != y;
+    if (nx != ny) return nx ? 1 : -1;
+    if (!nx && x != y) return x > y ? -1 : 1;
+    return a < b ? -1 : (a > b ? 1 : 0);
+}
+int orc_topk_scores(const double *scores, uint64_t n, uint32_t k, uint32_t *out_idx) {
+    uint32_t *idx = (uint32_t *)malloc((n ? n : 1) * sizeof(uint32_t));
+    if (!idx) return -1;
+    for (uint64_t i = 0; i < n; i++) idx[i] = (uint32_t)i;
+    g_score = scores;
+    qsort(idx, n, sizeof(uint32_t), cmp_score);
+    for (uint64_t i = 0; i < k && i < n; i++) out_idx[i] = idx[i];
+    free(idx);
+    return 0;
+}
+
+/*
  * Ranking used for "keep the best placements" (order 0): valid candidates first; more SLO
  * hits first; then lower mean time-to-first-token, sum/n_served compared exactly by
  * cross-multiplication in 128 bits (a candidate that served nothing ranks after any that

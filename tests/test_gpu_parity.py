@@ -263,6 +263,29 @@ def test_topk_matches_oracle_ranking(ctx, oracle_mod):
     ctx.free_trace(t)
 
 
+def test_topk_million_records_three_passes(ctx, oracle_mod):
+    """Selection at the scale configuration's size: 10^6 records, k = 64 (three passes of the
+    grid-level reduction), many ties on the hit count so that the exact mean comparison and
+    the index tie-break decide."""
+    import torch
+    n = 1_000_000
+    rng = np.random.default_rng(11)
+    rec = np.zeros(n, dtype=gen.RESULT_DTYPE)
+    rec["status"] = (rng.random(n) < 0.01) * 2
+    rec["n_hit"] = rng.integers(900, 1000, n)
+    rec["n_served"] = rng.integers(1, 1200, n)
+    rec["sum_ttft_us"] = rng.integers(1, 1 << 44, n)
+    dup = rng.integers(0, n, 2000)                      # exact duplicates: index decides
+    rec[dup[:1000]] = rec[dup[1000:]]
+    dev = torch.from_numpy(rec.view(np.uint8).reshape(n, 128)).cuda()
+    for k in (64, 1024):
+        idx, out = ctx.topk(dev, k)
+        torch.cuda.synchronize()
+        want = oracle_mod.topk(rec, k)
+        assert idx.cpu().numpy().view(np.uint32).tolist() == want.tolist()
+        assert ctx.results_to_numpy(out).tobytes() == rec[want].tobytes()
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")

@@ -318,3 +318,53 @@ def test_generator_counts_and_layout():
     a = gen.make_trace(100, 8.0, 7)
     b2 = gen.make_trace(100, 8.0, 7)
     assert a.tobytes() == b2.tobytes()
+
+
+# ---- composite serving score (Sec. IV-D) ----------------------------------------------------
+def _rec(**kw):
+    r = np.zeros(1, dtype=gen.RESULT_DTYPE)
+    for k, v in kw.items():
+        r[k] = v
+    return r
+
+
+def test_score_worked_values(oracle_mod):
+    # 50 of 100 requests hit; 1000 tokens in 1 s -> 1000 tok/s of gamma_T = 2000 -> 0.5;
+    # mean TTFT 0.5 s of gamma_L = 2 s -> 0.75;  4*0.5 + 0.3*0.5 + 0.7*0.75 = 2.675
+    r = _rec(n_counted=100, n_served=80, n_hit=50, tokens_out=1000, makespan_us=1_000_000,
+             sum_ttft_us=80 * 500_000)
+    assert oracle_mod.score(r, 4.0, 0.3, 2000.0, 2.0)[0] == pytest.approx(2.675, abs=1e-12)
+    # throughput above the threshold is capped, latency beyond the threshold earns nothing
+    r = _rec(n_counted=10, n_served=10, n_hit=10, tokens_out=10_000_000, makespan_us=1_000_000,
+             sum_ttft_us=10 * 9_000_000)
+    assert oracle_mod.score(r, 10.0, 0.25, 2000.0, 2.0)[0] == pytest.approx(10.0 + 0.25, abs=1e-12)
+    # nothing served: only the (zero) SLO term; invalid: -1; nothing counted: 0
+    assert oracle_mod.score(_rec(n_counted=7), 4.0, 0.3, 1.0, 1.0)[0] == 0.0
+    assert oracle_mod.score(_rec(status=2), 4.0, 0.3, 1.0, 1.0)[0] == -1.0
+    assert oracle_mod.score(_rec(), 4.0, 0.3, 1.0, 1.0)[0] == 0.0
+
+
+def test_score_properties_and_ranking(oracle_mod):
+    cfg = gen.make_config("tiny")
+    res = oracle_mod.eval_placements(cfg["profile"], cfg["traces"][0], cfg["classes"], cfg["offsets"],
+                                     cfg["inst"], cfg["budget"])
+    a4 = oracle_mod.score(res, 4.0, 0.3, 500.0, 5.0)
+    a10 = oracle_mod.score(res, 10.0, 0.3, 500.0, 5.0)
+    ratio = res["n_hit"] / res["n_counted"]
+    # alpha only weighs the SLO term (MaaSO vs MaaSO*: alpha = 4 vs 10)
+    assert np.allclose(a10 - a4, 6.0 * ratio, atol=1e-12)
+    assert (a4 >= 4.0 * ratio - 1e-12).all() and (a4 <= 4.0 * ratio + 1.0 + 1e-12).all()
+    # beta = 1: throughput only; beta = 0: latency only
+    t_only = oracle_mod.score(res, 0.0, 1.0, 500.0, 5.0)
+    thr = np.where(res["n_served"] > 0, res["tokens_out"] / (res["makespan_us"] * 1e-6), 0.0)
+    assert np.allclose(t_only, np.minimum(thr, 500.0) / 500.0, atol=1e-12)
+    l_only = oracle_mod.score(res, 0.0, 0.0, 500.0, 5.0)
+    lat = np.where(res["n_served"] > 0, res["sum_ttft_us"] / np.maximum(res["n_served"], 1) * 1e-6, 5.0)
+    assert np.allclose(l_only, np.maximum(5.0 - lat, 0.0) / 5.0, atol=1e-12)
+    # ranking by score: brute force
+    s = a4.copy()
+    s[3] = s[77]                 # a tie decided by the index
+    s[5] = np.nan                # NaN goes last
+    want = sorted(range(len(s)), key=lambda i: (np.isnan(s[i]), -s[i] if not np.isnan(s[i]) else 0.0, i))
+    assert oracle_mod.topk_scores(s, 143).tolist() == want
+    assert oracle_mod.topk_scores(s, 10).tolist() == want[:10]
