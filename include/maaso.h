@@ -198,6 +198,27 @@ MAASO_API int maaso_eval_placements_host(maaso_ctx *ctx, const maaso_trace *trac
 MAASO_API int maaso_topk(maaso_ctx *ctx, const maaso_result *results, uint64_t n_cand, uint32_t k,
                uint32_t order, uint32_t *out_idx, maaso_result *out_res, void *cuda_stream);
 
+/* Composite serving score of Sec. IV-D, one double per record (device, [n_cand]):
+ *   Phi = alpha * PhiS_n + beta * PhiT_n + (1 - beta) * PhiL_n
+ *   PhiS_n = n_hit / n_counted (SLO satisfaction ratio),
+ *   PhiT_n = min(tokens_out / makespan [tokens/s], gamma_t) / gamma_t,
+ *   PhiL_n = max(gamma_l - mean time to first token [s], 0) / gamma_l.
+ * A record that counted nothing has PhiS_n = 0, one that served nothing has PhiT_n = PhiL_n = 0,
+ * an invalid candidate scores -1.  Computed in IEEE double without fused operations.
+ * gamma_t, gamma_l must be positive and finite.  (The paper uses alpha = 4, beta = 0.3, and
+ * alpha = 10 for its MaaSO* variant, Sec. V-A.)  Enqueued on cuda_stream. */
+typedef struct {
+    double alpha, beta, gamma_t, gamma_l;
+} maaso_score_params;
+MAASO_API int maaso_score(maaso_ctx *ctx, const maaso_result *results, uint64_t n_cand,
+                          const maaso_score_params *params, double *out_scores, void *cuda_stream);
+
+/* Top-k by score (the "if phi > Phi*[k]" selection of Alg. 1 over a batch): higher score first,
+ * then lower index; NaN scores rank last.  Outputs as maaso_topk. */
+MAASO_API int maaso_topk_scores(maaso_ctx *ctx, const maaso_result *results, const double *scores,
+                                uint64_t n_cand, uint32_t k, uint32_t *out_idx, maaso_result *out_res,
+                                void *cuda_stream);
+
 /* Top-k without any allocation.  (The paper has no counterpart; this is a deployment
  * variant of maaso_topk.)  It is meant for callers that must not allocate device memory
  * while they run: code inside a memory-pool or arena framework that owns all device memory,

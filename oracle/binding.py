@@ -37,7 +37,7 @@ def build(force=False):
     """Compile the oracle with gcc -O2 (plain C, single thread)."""
     if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
         tmp = _SO + f".{os.getpid()}.tmp"
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-Wall", "-Wextra",
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fPIC", "-shared", "-Wall", "-Wextra",
                                "-o", tmp, _SRC])
         os.replace(tmp, _SO)
     return _SO

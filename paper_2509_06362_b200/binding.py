@@ -51,6 +51,10 @@ class _EvalOpts(C.Structure):
                 ("dump_first_us", C.c_void_p), ("dump_inst", C.c_void_p)]
 
 
+class _ScoreParams(C.Structure):
+    _fields_ = [("alpha", C.c_double), ("beta", C.c_double), ("gamma_t", C.c_double), ("gamma_l", C.c_double)]
+
+
 class _Timing(C.Structure):
     _fields_ = [("prep_ms", C.c_float), ("group_ms", C.c_float), ("block_ms", C.c_float),
                 ("topk_ms", C.c_float)]
@@ -76,6 +80,8 @@ def _load():
     lib.maaso_eval_placements.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp, vp]
     lib.maaso_eval_placements_host.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp]
     lib.maaso_topk.argtypes = [vp, vp, u64, u32, u32, vp, vp, vp]
+    lib.maaso_score.argtypes = [vp, vp, u64, C.POINTER(_ScoreParams), vp, vp]
+    lib.maaso_topk_scores.argtypes = [vp, vp, vp, u64, u32, vp, vp, vp]
     lib.maaso_topk_noalloc.argtypes = [vp, u64, u32, u32, vp, vp, vp]
     lib.maaso_topk_noalloc.restype = C.c_int
     lib.maaso_set_timing.argtypes = [vp, C.c_int]
@@ -87,7 +93,8 @@ def _load():
     lib.maaso_last_error.argtypes = [vp]
     lib.maaso_last_error.restype = C.c_char_p
     for name in ("maaso_create", "maaso_load_profile", "maaso_load_trace", "maaso_eval_placements",
-                 "maaso_eval_placements_host", "maaso_topk", "maaso_set_timing", "maaso_get_timing"):
+                 "maaso_eval_placements_host", "maaso_topk", "maaso_set_timing", "maaso_get_timing",
+                 "maaso_score", "maaso_topk_scores"):
         getattr(lib, name).restype = C.c_int
     return lib
 
@@ -204,6 +211,17 @@ def maaso_topk(ctx, results, n_cand, k, out_idx, out_res=None, order=0, stream=N
                            _stream_ptr(stream)), "maaso_topk", ctx)
 
 
+def maaso_score(ctx, results, n_cand, alpha, beta, gamma_t, gamma_l, out_scores, stream=None):
+    p = _ScoreParams(float(alpha), float(beta), float(gamma_t), float(gamma_l))
+    _check(_lib.maaso_score(ctx, _ptr(results), int(n_cand), C.byref(p), _ptr(out_scores), _stream_ptr(stream)),
+           "maaso_score", ctx)
+
+
+def maaso_topk_scores(ctx, results, scores, n_cand, k, out_idx, out_res=None, stream=None):
+    _check(_lib.maaso_topk_scores(ctx, _ptr(results), _ptr(scores), int(n_cand), int(k), _ptr(out_idx),
+                                  _ptr(out_res), _stream_ptr(stream)), "maaso_topk_scores", ctx)
+
+
 NOALLOC_MAX_CAND = 1 << 20
 NOALLOC_MAX_K = 64
 
@@ -313,6 +331,18 @@ class Context:
         idx = torch.empty(k, dtype=torch.int32, device=self.device)
         rec = torch.empty((k, 128), dtype=torch.uint8, device=self.device) if with_records else None
         maaso_topk(self.handle, results, n_cand, k, idx, rec, order, stream)
+        return idx, rec
+
+    def score(self, results, alpha, beta, gamma_t, gamma_l, stream=None):
+        out = self.torch.empty(int(results.shape[0]), dtype=self.torch.float64, device=self.device)
+        maaso_score(self.handle, results, int(results.shape[0]), alpha, beta, gamma_t, gamma_l, out, stream)
+        return out
+
+    def topk_scores(self, results, scores, k, with_records=True, stream=None):
+        torch = self.torch
+        idx = torch.empty(k, dtype=torch.int32, device=self.device)
+        rec = torch.empty((k, 128), dtype=torch.uint8, device=self.device) if with_records else None
+        maaso_topk_scores(self.handle, results, scores, int(results.shape[0]), k, idx, rec, stream)
         return idx, rec
 
     def set_timing(self, enabled):

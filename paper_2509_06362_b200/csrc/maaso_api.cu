@@ -19,7 +19,10 @@ int occupancy_eval_block(const EvalParams& P, int bucket, int tile_recs);
 size_t block_payload_per_cta(int bucket);
 size_t topk_scratch_bytes(uint64_t n_cand, uint32_t k);
 cudaError_t launch_topk(const maaso_result* results, uint64_t n_cand, uint32_t k, void* scratch,
-                        uint32_t* out_idx, maaso_result* out_res, cudaStream_t stream, int* launches);
+                        uint32_t* out_idx, maaso_result* out_res, cudaStream_t stream, int* launches,
+                        const double* scores);
+cudaError_t launch_score(const maaso_result* res, uint64_t n, const maaso_score_params& p, double* out,
+                         cudaStream_t stream);
 }  // namespace maaso
 
 using namespace maaso;
@@ -479,13 +482,45 @@ MAASO_API int maaso_topk(maaso_ctx* ctx, const maaso_result* results, uint64_t n
     int launches = 0;
     if (ctx->timing) cudaEventRecord(ctx->ev[4], (cudaStream_t)cuda_stream);
     cudaError_t e = launch_topk(results, n_cand, k, ctx->topk_scratch, out_idx, out_res,
-                                (cudaStream_t)cuda_stream, &launches);
+                                (cudaStream_t)cuda_stream, &launches, nullptr);
     if (ctx->timing) {
         cudaEventRecord(ctx->ev[5], (cudaStream_t)cuda_stream);
         ctx->ev_topk = true;
     }
     ctx->launches += (uint64_t)launches;
     if (e != cudaSuccess) return cuda_fail(ctx, e, "topk launch");
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_score(maaso_ctx* ctx, const maaso_result* results, uint64_t n_cand,
+                          const maaso_score_params* params, double* out_scores, void* cuda_stream) {
+    if (!ctx || !params) return MAASO_EINVAL;
+    if (n_cand == 0) return MAASO_OK;
+    if (!results || !out_scores || !(params->gamma_t > 0.0) || !(params->gamma_l > 0.0) ||
+        params->gamma_t > 1e300 || params->gamma_l > 1e300)
+        return fail(ctx, MAASO_EINVAL, "score: null pointer or non-positive threshold");
+    DeviceGuard g(ctx->device);
+    cudaError_t e = launch_score(results, n_cand, *params, out_scores, (cudaStream_t)cuda_stream);
+    ctx->launches++;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "score launch");
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_topk_scores(maaso_ctx* ctx, const maaso_result* results, const double* scores,
+                                uint64_t n_cand, uint32_t k, uint32_t* out_idx, maaso_result* out_res,
+                                void* cuda_stream) {
+    if (!ctx) return MAASO_EINVAL;
+    if (k == 0) return MAASO_OK;
+    if (!out_idx || ((!results || !scores) && n_cand) || k > MAASO_MAX_TOPK || n_cand >= 0xFFFFFFFFull)
+        return fail(ctx, MAASO_EINVAL, "topk_scores: null pointer or k out of range");
+    DeviceGuard g(ctx->device);
+    int rc = grow(ctx, &ctx->topk_scratch, &ctx->topk_scratch_bytes, topk_scratch_bytes(n_cand, k));
+    if (rc != MAASO_OK) return rc;
+    int launches = 0;
+    cudaError_t e = launch_topk(results, n_cand, k, ctx->topk_scratch, out_idx, out_res,
+                                (cudaStream_t)cuda_stream, &launches, scores);
+    ctx->launches += (uint64_t)launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "topk_scores launch");
     return MAASO_OK;
 }
 

@@ -38,13 +38,21 @@ __device__ __forceinline__ bool ranks_before(const Entry& a, const Entry& b) {
     return a.idx < b.idx;
 }
 
+// Order 1 ranks by a score: the entry carries the bit pattern of the score mapped so that
+// unsigned order = descending score (as sum_ttft with n_served = 1, n_hit = 0), NaN = not valid.
+__device__ __forceinline__ uint64_t descending_key(double s) {
+    const uint64_t b = (uint64_t)__double_as_longlong(s);
+    const uint64_t ascending = (b >> 63) ? ~b : (b | (1ull << 63));
+    return ~ascending;
+}
+
 // src_res != null: first pass, entries are built from records [0, n).  Otherwise entries
 // come from src_ent[0, n).  Block b sorts its chunk and writes its k best to dst_ent[b*k ..]
 // or, when `final`, candidate indices / records to out_idx / out_res.
 __global__ void __launch_bounds__(kTopkThreads)
 topk_pass_kernel(const maaso_result* src_res, const Entry* src_ent, uint64_t n, uint32_t k,
                  Entry* dst_ent, int final_pass, const maaso_result* all_res, uint32_t* out_idx,
-                 maaso_result* out_res) {
+                 maaso_result* out_res, const double* scores) {
     extern __shared__ __align__(16) unsigned char topk_smem[];
     Entry* e = reinterpret_cast<Entry*>(topk_smem);
     const uint64_t base = (uint64_t)blockIdx.x * kChunk;
@@ -61,6 +69,13 @@ topk_pass_kernel(const maaso_result* src_res, const Entry* src_ent, uint64_t n, 
                 v.n_served = a.z;
                 v.n_hit = a.w;
                 v.sum_ttft = ((uint64_t)d.w << 32) | d.z;
+                if (scores) {
+                    const double sc = scores[g];
+                    v.valid = sc == sc ? 1u : 0u;
+                    v.n_hit = 0;
+                    v.n_served = 1;
+                    v.sum_ttft = descending_key(sc);
+                }
             } else {
                 v = src_ent[g];
             }
@@ -107,7 +122,8 @@ size_t topk_scratch_bytes(uint64_t n_cand, uint32_t k) {
 
 // scratch: at least topk_scratch_bytes(n_cand, k), 16-byte aligned.
 cudaError_t launch_topk(const maaso_result* results, uint64_t n_cand, uint32_t k, void* scratch,
-                        uint32_t* out_idx, maaso_result* out_res, cudaStream_t stream, int* launches) {
+                        uint32_t* out_idx, maaso_result* out_res, cudaStream_t stream, int* launches,
+                        const double* scores) {
     const size_t smem = (size_t)kChunk * sizeof(Entry);
     cudaError_t err = cudaFuncSetAttribute(topk_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem);
@@ -124,7 +140,7 @@ cudaError_t launch_topk(const maaso_result* results, uint64_t n_cand, uint32_t k
         const uint64_t blocks = n == 0 ? 1 : (n + kChunk - 1) / kChunk;
         const int final_pass = blocks == 1;
         topk_pass_kernel<<<(unsigned)blocks, kTopkThreads, smem, stream>>>(
-            src_res, src_ent, n, k, buf[which], final_pass, results, out_idx, out_res);
+            src_res, src_ent, n, k, buf[which], final_pass, results, out_idx, out_res, scores);
         (*launches)++;
         if (final_pass) break;
         src_res = nullptr;
@@ -181,7 +197,7 @@ extern "C" MAASO_API int maaso_topk_noalloc(const maaso_result* results, uint64_
     }
     int launches = 0;
     const cudaError_t e = launch_topk(results, n_cand, k, scratch, out_idx, out_res, (cudaStream_t)cuda_stream,
-                                      &launches);
+                                      &launches, nullptr);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return MAASO_ECUDA;

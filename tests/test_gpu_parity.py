@@ -286,6 +286,48 @@ def test_topk_million_records_three_passes(ctx, oracle_mod):
         assert ctx.results_to_numpy(out).tobytes() == rec[want].tobytes()
 
 
+def test_score_and_ranking_by_score(ctx, oracle_mod):
+    """Composite serving score (Sec. IV-D) in double precision: the kernel uses explicitly rounded
+    operations in the oracle's order, so values are expected to be identical; the test allows
+    4 ulp.  Ranking by score takes its decisions on the same doubles on both sides."""
+    import torch
+    cfg = gen.make_config("node", n_cand=6000, n_req=800)
+    tr = cfg["traces"][0]
+    ctx.load_profile(cfg["profile"])
+    t = ctx.load_trace(tr, cfg["classes"])
+    res = ctx.eval_placements(t, ctx.to_device(cfg["offsets"]), ctx.to_device(cfg["inst"]), 8)
+    torch.cuda.synchronize()
+    rec = ctx.results_to_numpy(res).copy()
+    rec["status"][17] = 4
+    rec["n_served"][23] = 0
+    rec["n_counted"][29] = 0
+    dev = torch.from_numpy(rec.view(np.uint8).reshape(-1, 128)).cuda()
+    for (alpha, beta, gt, gl) in [(4.0, 0.3, 800.0, 10.0), (10.0, 0.3, 800.0, 10.0), (2.5, 0.0, 50.0, 0.5),
+                                  (1.0, 1.0, 1e9, 1e-9)]:
+        got = ctx.score(dev, alpha, beta, gt, gl).cpu().numpy()
+        want = oracle_mod.score(rec, alpha, beta, gt, gl)
+        ulp = np.spacing(np.maximum(np.abs(want), 1e-300))
+        assert (np.abs(got - want) <= 4 * ulp).all(), np.abs(got - want).max()
+        for k in (1, 64, 1000):
+            idx, out = ctx.topk_scores(dev, torch.from_numpy(want).cuda(), k)
+            torch.cuda.synchronize()
+            w = oracle_mod.topk_scores(want, k)
+            assert idx.cpu().numpy().view(np.uint32).tolist() == w.tolist()
+            assert ctx.results_to_numpy(out).tobytes() == rec[w].tobytes()
+    s = oracle_mod.score(rec, 4.0, 0.3, 800.0, 10.0)
+    s[5] = np.nan
+    s[100] = s[200] = s.max() + 1.0
+    idx, _ = ctx.topk_scores(dev, torch.from_numpy(s).cuda(), 1024)
+    torch.cuda.synchronize()
+    assert idx.cpu().numpy().view(np.uint32).tolist() == oracle_mod.topk_scores(s, 1024).tolist()
+    # NaN ranks last: a tiny set where k covers everything
+    small = torch.from_numpy(rec[:8].view(np.uint8).reshape(8, 128)).cuda()
+    idx, _ = ctx.topk_scores(small, torch.from_numpy(s[:8]).cuda(), 8)
+    torch.cuda.synchronize()
+    assert idx.cpu().numpy().view(np.uint32).tolist() == oracle_mod.topk_scores(s[:8], 8).tolist()
+    ctx.free_trace(t)
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")
