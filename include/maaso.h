@@ -134,6 +134,8 @@ typedef struct {
     int64_t *dump_finish_us;
     int64_t *dump_first_us;
     int32_t *dump_inst;
+    uint32_t *rejected_by_model; /* device, [n_cand][MAASO_MAX_MODELS] or NULL: requests of each model
+                                    the placement left unserved (R_res of Alg. 1); zero for invalid ones */
 } maaso_eval_opts;
 
 /* Per-candidate result (128 bytes).  Statistics are over served requests unless noted. */
@@ -218,6 +220,29 @@ MAASO_API int maaso_score(maaso_ctx *ctx, const maaso_result *results, uint64_t 
 MAASO_API int maaso_topk_scores(maaso_ctx *ctx, const maaso_result *results, const double *scores,
                                 uint64_t n_cand, uint32_t k, uint32_t *out_idx, maaso_result *out_res,
                                 void *cuda_stream);
+
+/* Alg. 1, "Simulator-Based Instance Configuration": greedy instance deployment for one
+ * sub-cluster of `gpus` devices, scored on the requests of `trace` whose class bit is set in
+ * class_mask (all requests if use_mask == 0).  For every configuration (strategy, batch cap) of the
+ * caller's (already pruned) list, starting from the empty placement: while devices remain and a
+ * model is not saturated, add an instance of the non-saturated model with the most unserved
+ * requests (ties: lowest index), evaluate the tentative placement (maaso_eval_placements +
+ * maaso_score), accept it if the score improved, else mark the model saturated; the best score
+ * and placement per device count are kept.  All configurations advance together, so each greedy
+ * step is ONE batch of tentative placements on the GPU.  As printed in the paper, the device count
+ * k that indexes the outputs is that of the placement before the tentative instance is added.
+ * A tentative placement that violates a constraint scores -1 and is never accepted.
+ * Host pointers: configs[n_configs]; outputs phi_star[gpus+1], istar_len[gpus+1],
+ * istar_inst[(gpus+1) * MAASO_MAX_INSTANCES] (packed instance words).  Synchronous; uses the
+ * context's own stream and scratch memory.  gpus <= 4096. */
+typedef struct {
+    uint32_t strategy;
+    uint32_t batch;
+} maaso_config;
+MAASO_API int maaso_ins_deploy(maaso_ctx *ctx, const maaso_trace *trace, uint32_t gpus,
+                               const maaso_config *configs, uint32_t n_configs, int use_mask,
+                               uint32_t class_mask, const maaso_score_params *score, uint32_t flags,
+                               double *phi_star, uint32_t *istar_len, uint32_t *istar_inst);
 
 /* Top-k without any allocation.  (The paper has no counterpart; this is a deployment
  * variant of maaso_topk.)  It is meant for callers that must not allocate device memory

@@ -51,6 +51,8 @@ def _load():
         _lib.orc_topk.restype = C.c_int
         _lib.orc_score.restype = C.c_int
         _lib.orc_topk_scores.restype = C.c_int
+        _lib.orc_rejected_by_model.restype = C.c_int
+        _lib.orc_ins_deploy.restype = C.c_int
     return _lib
 
 
@@ -163,6 +165,49 @@ def score(results, alpha, beta, gamma_t, gamma_l):
     if rc != 0:
         raise RuntimeError(f"oracle score failed with code {rc}")
     return out
+
+
+def rejected_by_model(profile, trace, classes, offsets, inst, budget, class_mask=None, flags=0):
+    """[n_cand][16] requests of each model that every candidate left unserved."""
+    lib = _load()
+    p, keep = _profile_struct(profile)
+    trace = np.ascontiguousarray(trace, dtype=_REQ)
+    classes = np.ascontiguousarray(classes, dtype=_SLO)
+    offsets = np.ascontiguousarray(offsets, dtype=np.uint32)
+    inst = np.ascontiguousarray(inst, dtype=np.uint32)
+    if inst.size == 0:
+        inst = np.zeros(1, dtype=np.uint32)
+    mask = None if class_mask is None else np.ascontiguousarray(class_mask, dtype=np.uint32)
+    out = np.zeros((len(offsets) - 1, 16), dtype=np.uint32)
+    rc = lib.orc_rejected_by_model(C.byref(p), _ptr(trace), C.c_uint64(len(trace)), _ptr(classes),
+                                   C.c_uint32(len(classes)), _ptr(offsets), _ptr(inst), _ptr(mask),
+                                   C.c_uint64(len(offsets) - 1), C.c_uint32(budget), C.c_uint32(flags), _ptr(out))
+    if rc != 0:
+        raise RuntimeError(f"oracle rejected_by_model failed with code {rc}")
+    del keep
+    return out
+
+
+def ins_deploy(profile, trace, classes, gpus, configs, alpha, beta, gamma_t, gamma_l, class_mask=None, flags=0):
+    """Alg. 1 (see orc_ins_deploy).  configs: list of (strategy, batch).  Returns (phi_star[gpus+1],
+    list of gpus+1 instance-word arrays)."""
+    lib = _load()
+    p, keep = _profile_struct(profile)
+    trace = np.ascontiguousarray(trace, dtype=_REQ)
+    classes = np.ascontiguousarray(classes, dtype=_SLO)
+    cfg = np.ascontiguousarray(np.asarray(configs, dtype=np.uint32).reshape(-1, 2))
+    sp = _ScoreParams(alpha, beta, gamma_t, gamma_l)
+    phi = np.zeros(gpus + 1, dtype=np.float64)
+    ilen = np.zeros(gpus + 1, dtype=np.uint32)
+    iinst = np.zeros((gpus + 1, 128), dtype=np.uint32)
+    rc = lib.orc_ins_deploy(C.byref(p), _ptr(trace), C.c_uint64(len(trace)), _ptr(classes), C.c_uint32(len(classes)),
+                            C.c_int(0 if class_mask is None else 1), C.c_uint32(class_mask or 0), C.c_uint32(gpus),
+                            _ptr(cfg), C.c_uint32(len(cfg)), C.byref(sp), C.c_uint32(flags), _ptr(phi), _ptr(ilen),
+                            _ptr(iinst))
+    if rc != 0:
+        raise RuntimeError(f"oracle ins_deploy failed with code {rc}")
+    del keep
+    return phi, [iinst[k, :ilen[k]].copy() for k in range(gpus + 1)]
 
 
 def topk_scores(scores, k):

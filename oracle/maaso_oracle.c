@@ -395,6 +395,94 @@ int orc_score(const orc_result *res, uint64_t n, const orc_score_params *p, doub
     return 0;
 }
 
+/* Requests of each model left unserved (rejected) by every candidate: counted from the
+ * per-request outcome, out[c][16]. */
+int orc_rejected_by_model(const orc_profile *p, const orc_request *reqs, uint64_t n, const orc_slo *classes,
+                          uint32_t n_classes, const uint32_t *offsets, const uint32_t *inst,
+                          const uint32_t *class_mask, uint64_t n_cand, uint32_t budget, uint32_t flags,
+                          uint32_t *out) {
+    int32_t *where = (int32_t *)malloc((n ? n : 1) * sizeof(int32_t));
+    if (!where) return -1;
+    for (uint64_t c = 0; c < n_cand; c++) {
+        orc_result r;
+        int rc = orc_eval_candidate(p, reqs, n, classes, n_classes, inst + offsets[c], offsets[c + 1] - offsets[c],
+                                    class_mask != NULL, class_mask ? class_mask[c] : 0, budget, flags, &r, NULL,
+                                    NULL, where);
+        if (rc) { free(where); return rc; }
+        for (int m = 0; m < 16; m++) out[c * 16 + m] = 0;
+        for (uint64_t q = 0; q < n; q++)
+            if (where[q] == -1) out[c * 16 + reqs[q].model]++;
+    }
+    free(where);
+    return 0;
+}
+
+/*
+ * Alg. 1, "Simulator-Based Instance Configuration", taken literally.  For every configuration
+ * (P, B) of the (already pruned) list: start from the empty placement; while GPUs remain and
+ * some model is not saturated, add an instance (m', P, B) of the model m' with the most
+ * unserved requests among the non-saturated ones (ties: lowest model index), evaluate the
+ * serving score of the tentative placement on R_x with the simulator, accept it if the score
+ * improved, otherwise mark m' saturated; record the best score and placement per GPU count.
+ * As printed, k is the GPU count of the placement BEFORE the tentative instance is added;
+ * that reading is kept.  A tentative placement that violates a constraint (budget, memory fit,
+ * instance limit) scores -1 and is therefore never accepted.
+ * R_x = requests whose class bit is set in class_mask (all if has_mask == 0).
+ * Outputs: phi_star[gpus + 1], istar_len[gpus + 1], istar_inst[gpus + 1][128] (packed words).
+ */
+typedef struct { uint32_t strategy, batch; } orc_config;
+
+int orc_ins_deploy(const orc_profile *p, const orc_request *reqs, uint64_t n, const orc_slo *classes,
+                   uint32_t n_classes, int has_mask, uint32_t class_mask, uint32_t gpus,
+                   const orc_config *configs, uint32_t n_configs, const orc_score_params *sp, uint32_t flags,
+                   double *phi_star, uint32_t *istar_len, uint32_t *istar_inst) {
+    int32_t *where = (int32_t *)malloc((n ? n : 1) * sizeof(int32_t));
+    if (!where) return -1;
+    if (n_classes > 32) has_mask = 0;
+    for (uint32_t k = 0; k <= gpus; k++) { phi_star[k] = 0.0; istar_len[k] = 0; }
+    for (uint32_t c = 0; c < n_configs; c++) {
+        uint32_t I[ORC_MAX_INST + 1], nI = 0;
+        int sat[16] = {0};
+        uint32_t unserved[16] = {0};
+        double phi = 0.0;
+        const uint32_t dev = (uint32_t)p->devices[configs[c].strategy];
+        for (uint64_t q = 0; q < n; q++)  /* R_res = R_x: nothing is served yet */
+            if (!has_mask || ((class_mask >> reqs[q].cls) & 1u)) unserved[reqs[q].model]++;
+        for (;;) {
+            if (nI * dev >= gpus) break;                      /* gpuCount(I) < |G_x| */
+            int mp = -1;                                      /* mostUnservedModel over M \ M_sat */
+            for (uint32_t m = 0; m < p->n_models; m++)
+                if (!sat[m] && (mp < 0 || unserved[m] > unserved[mp])) mp = (int)m;
+            if (mp < 0) break;                                /* M_sat == M */
+            if (nI > ORC_MAX_INST) break;
+            I[nI] = ((uint32_t)mp & 0xF) | ((configs[c].strategy & 0xFF) << 4) | ((configs[c].batch & 0xFF) << 12);
+            const uint32_t k = nI * dev;                      /* gpuCount(I), before the addition */
+            orc_result r;
+            int rc = orc_eval_candidate(p, reqs, n, classes, n_classes, I, nI + 1, has_mask, class_mask, gpus,
+                                        flags, &r, NULL, NULL, where);
+            if (rc) { free(where); return rc; }
+            double phi2;
+            orc_score(&r, 1, sp, &phi2);
+            if (phi2 > phi) {                                 /* accept the new instance */
+                phi = phi2;
+                nI++;
+                for (int m = 0; m < 16; m++) unserved[m] = 0;
+                for (uint64_t q = 0; q < n; q++)
+                    if (where[q] == -1) unserved[reqs[q].model]++;
+            } else {
+                sat[mp] = 1;                                  /* stop deploying m' */
+            }
+            if (phi > phi_star[k]) {
+                phi_star[k] = phi;
+                istar_len[k] = nI;
+                for (uint32_t i = 0; i < nI; i++) istar_inst[(size_t)k * ORC_MAX_INST + i] = I[i];
+            }
+        }
+    }
+    free(where);
+    return 0;
+}
+
 /* Ranking by score (order 1): higher score first, then lower index; NaN scores last. */
 static const double *g_score;
 static int cmp_score(const void *pa, const void *pb) {

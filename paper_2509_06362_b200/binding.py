@@ -48,7 +48,7 @@ class _CandBatch(C.Structure):
 class _EvalOpts(C.Structure):
     _fields_ = [("flags", C.c_uint32), ("mapping", C.c_uint32), ("dump_n", C.c_uint32),
                 ("reserved", C.c_uint32), ("dump_cand_idx", C.c_void_p), ("dump_finish_us", C.c_void_p),
-                ("dump_first_us", C.c_void_p), ("dump_inst", C.c_void_p)]
+                ("dump_first_us", C.c_void_p), ("dump_inst", C.c_void_p), ("rejected_by_model", C.c_void_p)]
 
 
 class _ScoreParams(C.Structure):
@@ -82,6 +82,8 @@ def _load():
     lib.maaso_topk.argtypes = [vp, vp, u64, u32, u32, vp, vp, vp]
     lib.maaso_score.argtypes = [vp, vp, u64, C.POINTER(_ScoreParams), vp, vp]
     lib.maaso_topk_scores.argtypes = [vp, vp, vp, u64, u32, vp, vp, vp]
+    lib.maaso_ins_deploy.argtypes = [vp, vp, u32, vp, u32, C.c_int, u32, C.POINTER(_ScoreParams), u32, vp, vp, vp]
+    lib.maaso_ins_deploy.restype = C.c_int
     lib.maaso_topk_noalloc.argtypes = [vp, u64, u32, u32, vp, vp, vp]
     lib.maaso_topk_noalloc.restype = C.c_int
     lib.maaso_set_timing.argtypes = [vp, C.c_int]
@@ -187,12 +189,13 @@ def _batch(offsets, inst, class_mask, budget):
 
 def maaso_eval_placements(ctx, trace, offsets, inst, budget, out_results, class_mask=None, flags=0,
                           mapping=MAP_AUTO, dump_cand_idx=None, dump_finish_us=None, dump_first_us=None,
-                          dump_inst=None, stream=None):
+                          dump_inst=None, rejected_by_model=None, stream=None):
     """All array arguments are CUDA tensors (int32 views of the uint32 words; out_results a
     uint8 tensor of n_cand*128 bytes).  Work is enqueued on `stream` (default: torch's current)."""
     b = _batch(offsets, inst, class_mask, budget)
     o = _EvalOpts(int(flags), int(mapping), 0 if dump_cand_idx is None else int(dump_cand_idx.shape[0]), 0,
-                  _ptr(dump_cand_idx), _ptr(dump_finish_us), _ptr(dump_first_us), _ptr(dump_inst))
+                  _ptr(dump_cand_idx), _ptr(dump_finish_us), _ptr(dump_first_us), _ptr(dump_inst),
+                  _ptr(rejected_by_model))
     _check(_lib.maaso_eval_placements(ctx, trace, C.byref(b), C.byref(o), _ptr(out_results),
                                       _stream_ptr(stream)), "maaso_eval_placements", ctx)
 
@@ -201,7 +204,7 @@ def maaso_eval_placements_host(ctx, trace, offsets, inst, budget, out_results, c
                                mapping=MAP_AUTO):
     """Host (numpy) buffers in and out; copies happen inside the call, which synchronises."""
     b = _batch(offsets, inst, class_mask, budget)
-    o = _EvalOpts(int(flags), int(mapping), 0, 0, None, None, None, None)
+    o = _EvalOpts(int(flags), int(mapping), 0, 0, None, None, None, None, None)
     _check(_lib.maaso_eval_placements_host(ctx, trace, C.byref(b), C.byref(o), _ptr(out_results)),
            "maaso_eval_placements_host", ctx)
 
@@ -220,6 +223,20 @@ def maaso_score(ctx, results, n_cand, alpha, beta, gamma_t, gamma_l, out_scores,
 def maaso_topk_scores(ctx, results, scores, n_cand, k, out_idx, out_res=None, stream=None):
     _check(_lib.maaso_topk_scores(ctx, _ptr(results), _ptr(scores), int(n_cand), int(k), _ptr(out_idx),
                                   _ptr(out_res), _stream_ptr(stream)), "maaso_topk_scores", ctx)
+
+
+def maaso_ins_deploy(ctx, trace, gpus, configs, alpha, beta, gamma_t, gamma_l, class_mask=None, flags=0):
+    """Alg. 1 on the GPU.  configs: sequence of (strategy, batch).  Returns (phi_star[gpus+1] as a
+    numpy array, list of gpus+1 arrays of packed instance words)."""
+    cfg = np.ascontiguousarray(np.asarray(configs, dtype=np.uint32).reshape(-1, 2))
+    p = _ScoreParams(float(alpha), float(beta), float(gamma_t), float(gamma_l))
+    phi = np.zeros(gpus + 1, dtype=np.float64)
+    ilen = np.zeros(gpus + 1, dtype=np.uint32)
+    iinst = np.zeros((gpus + 1, 128), dtype=np.uint32)
+    _check(_lib.maaso_ins_deploy(ctx, trace, int(gpus), cfg.ctypes.data, len(cfg), 0 if class_mask is None else 1,
+                                 int(class_mask or 0), C.byref(p), int(flags), phi.ctypes.data, ilen.ctypes.data,
+                                 iinst.ctypes.data), "maaso_ins_deploy", ctx)
+    return phi, [iinst[k, :ilen[k]].copy() for k in range(gpus + 1)]
 
 
 NOALLOC_MAX_CAND = 1 << 20
@@ -292,8 +309,12 @@ class Context:
         t = self.torch.from_numpy(np.ascontiguousarray(words, dtype=np.uint32).view(np.int32))
         return t.to(self.device)
 
+    def ins_deploy(self, trace, gpus, configs, alpha, beta, gamma_t, gamma_l, class_mask=None, flags=0):
+        return maaso_ins_deploy(self.handle, trace.handle, gpus, configs, alpha, beta, gamma_t, gamma_l,
+                                class_mask, flags)
+
     def eval_placements(self, trace, offsets, inst, budget, class_mask=None, flags=0, mapping=MAP_AUTO,
-                        dump_idx=None, out=None, stream=None):
+                        dump_idx=None, out=None, stream=None, rejected_by_model=None):
         """offsets / inst / class_mask: CUDA int32 tensors (see to_device).  Returns the uint8
         result tensor [n_cand, 128] and, if dump_idx is given, a dict of dump tensors."""
         torch = self.torch
@@ -310,7 +331,7 @@ class Context:
             kw = dict(dump_cand_idx=d, dump_finish_us=dumps["finish_us"], dump_first_us=dumps["first_us"],
                       dump_inst=dumps["inst"])
         maaso_eval_placements(self.handle, trace.handle, offsets, inst, budget, out, class_mask, flags,
-                              mapping, stream=stream, **kw)
+                              mapping, stream=stream, rejected_by_model=rejected_by_model, **kw)
         return (out, dumps) if dump_idx is not None else out
 
     def eval_placements_host(self, trace, offsets, inst, budget, class_mask=None, flags=0,

@@ -222,6 +222,7 @@ struct EvalParams {
     int64_t* dump_first;
     int32_t* dump_inst;
     Payload* payload;        // scratch for running requests
+    uint32_t* rej_by_model;  // [n_cand][MAASO_MAX_MODELS] or null
 };
 
 __device__ __forceinline__ Dump dump_for(const EvalParams& P, uint32_t cand) {

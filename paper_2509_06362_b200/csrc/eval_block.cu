@@ -263,6 +263,8 @@ eval_block_kernel(const EvalParams P, const int tile_recs, const int bucket) {
                         if (tid == 0) {
                             n_rejected++;
                             st.checksum += rejected_hash(req);
+                            if (P.rej_by_model)
+                                atomicAdd(&P.rej_by_model[(size_t)cand * MAASO_MAX_MODELS + q.model], 1u);
                             if (dump.finish) dump.finish[req] = -1;
                             if (dump.first) dump.first[req] = -1;
                             if (dump.inst) dump.inst[req] = -1;

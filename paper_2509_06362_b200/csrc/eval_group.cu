@@ -269,6 +269,8 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                             n_rejected++;
                             if (sub == 0) {
                                 st.checksum += __ldg(P.rej_hash + req);
+                                if (P.rej_by_model)
+                                    atomicAdd(&P.rej_by_model[(size_t)cand * MAASO_MAX_MODELS + q.model], 1u);
                                 if (dump.finish) dump.finish[req] = -1;
                                 if (dump.first) dump.first[req] = -1;
                                 if (dump.inst) dump.inst[req] = -1;

@@ -45,6 +45,7 @@ struct maaso_ctx {
     int32_t* d_rows;
     int32_t* d_devices;
     int32_t* d_min_devices;
+    std::vector<int32_t> h_devices;  // host copy for the Alg. 1 driver
     std::vector<maaso_trace*> traces;
     void* scratch;
     size_t scratch_bytes;
@@ -53,6 +54,8 @@ struct maaso_ctx {
     // staging for the host-buffer entry point
     void* stage;
     size_t stage_bytes;
+    void* deploy;
+    size_t deploy_bytes;
     cudaStream_t own_stream;
     uint64_t launches;
     int tile_recs;
@@ -120,8 +123,8 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
     ctx->device = cuda_device;
     ctx->has_profile = false;
     ctx->d_rows = ctx->d_devices = ctx->d_min_devices = nullptr;
-    ctx->scratch = ctx->topk_scratch = ctx->stage = nullptr;
-    ctx->scratch_bytes = ctx->topk_scratch_bytes = ctx->stage_bytes = 0;
+    ctx->scratch = ctx->topk_scratch = ctx->stage = ctx->deploy = nullptr;
+    ctx->scratch_bytes = ctx->topk_scratch_bytes = ctx->stage_bytes = ctx->deploy_bytes = 0;
     ctx->launches = 0;
     ctx->tile_recs = 256;
     ctx->own_stream = nullptr;
@@ -186,6 +189,7 @@ MAASO_API void maaso_destroy(maaso_ctx* ctx) {
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->topk_scratch) cudaFree(ctx->topk_scratch);
     if (ctx->stage) cudaFree(ctx->stage);
+    if (ctx->deploy) cudaFree(ctx->deploy);
     if (ctx->own_stream) cudaStreamDestroy(ctx->own_stream);
     for (int i = 0; i < 6; i++)
         if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
@@ -232,6 +236,7 @@ MAASO_API int maaso_load_profile(maaso_ctx* ctx, const maaso_profile_desc* d) {
         (e = cudaMemcpy(ctx->d_devices, d->devices, S * 4, cudaMemcpyHostToDevice)) != cudaSuccess ||
         (e = cudaMemcpy(ctx->d_min_devices, d->min_devices, M * 4, cudaMemcpyHostToDevice)) != cudaSuccess)
         return cuda_fail(ctx, e, "profile copy");
+    ctx->h_devices.assign(d->devices, d->devices + S);
     ctx->n_models = M;
     ctx->n_strategies = S;
     ctx->n_rows = R;
@@ -364,6 +369,7 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.dump_finish = o.dump_finish_us;
     P.dump_first = o.dump_first_us;
     P.dump_inst = o.dump_inst;
+    P.rej_by_model = o.rejected_by_model;
 
     // launch shapes: persistent grids bounded by what the batch can use
     const int occ_g = occupancy_eval_group(P, tile);
@@ -521,6 +527,154 @@ MAASO_API int maaso_topk_scores(maaso_ctx* ctx, const maaso_result* results, con
                                 (cudaStream_t)cuda_stream, &launches, scores);
     ctx->launches += (uint64_t)launches;
     if (e != cudaSuccess) return cuda_fail(ctx, e, "topk_scores launch");
+    return MAASO_OK;
+}
+
+// Alg. 1 as a host driver: every configuration runs its own greedy chain; the tentative
+// placements of all chains in one greedy step are one candidate batch on the GPU.
+MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_t gpus,
+                               const maaso_config* configs, uint32_t n_configs, int use_mask,
+                               uint32_t class_mask, const maaso_score_params* score, uint32_t flags,
+                               double* phi_star, uint32_t* istar_len, uint32_t* istar_inst) {
+    if (!ctx || !trace || !score || !phi_star || !istar_len || !istar_inst || (n_configs && !configs) ||
+        gpus > 4096 || n_configs > (1u << 20))
+        return MAASO_EINVAL;
+    if (!ctx->has_profile) return fail(ctx, MAASO_ESTATE, "ins_deploy: no profile loaded");
+    for (uint32_t c = 0; c < n_configs; c++)
+        if (configs[c].strategy >= ctx->n_strategies || configs[c].batch < 1 || configs[c].batch > MAASO_WMAX)
+            return fail(ctx, MAASO_EINVAL, "ins_deploy: configuration out of range");
+    for (uint32_t k = 0; k <= gpus; k++) { phi_star[k] = 0.0; istar_len[k] = 0; }
+    if (n_configs == 0) return MAASO_OK;
+    DeviceGuard g(ctx->device);
+
+    // device staging: offsets | inst | mask | results | scores | rejected-by-model
+    const size_t C = n_configs, cap_inst = C * (MAASO_MAX_INSTANCES + 1);
+    size_t off = 0;
+    const size_t o_off = off;  off = align_up(off + (C + 1) * 4, 256);
+    const size_t o_inst = off; off = align_up(off + cap_inst * 4, 256);
+    const size_t o_mask = off; off = align_up(off + C * 4, 256);
+    const size_t o_res = off;  off = align_up(off + C * sizeof(maaso_result), 256);
+    const size_t o_sc = off;   off = align_up(off + C * 8, 256);
+    const size_t o_rbm = off;  off = align_up(off + C * MAASO_MAX_MODELS * 4, 256);
+    int rc = grow(ctx, &ctx->deploy, &ctx->deploy_bytes, off);
+    if (rc != MAASO_OK) return rc;
+    unsigned char* sb = static_cast<unsigned char*>(ctx->deploy);
+    cudaStream_t st = ctx->own_stream;
+
+    std::vector<uint32_t> h_off(C + 1), h_inst, h_mask(C, class_mask), h_rbm(C * MAASO_MAX_MODELS);
+    std::vector<double> h_sc(C);
+    auto run_batch = [&](uint32_t n_cand) -> int {
+        cudaError_t e = cudaMemcpyAsync(sb + o_off, h_off.data(), (n_cand + 1) * 4, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && !h_inst.empty())
+            e = cudaMemcpyAsync(sb + o_inst, h_inst.data(), h_inst.size() * 4, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess && use_mask)
+            e = cudaMemcpyAsync(sb + o_mask, h_mask.data(), n_cand * 4, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "ins_deploy: upload");
+        maaso_cand_batch b;
+        memset(&b, 0, sizeof(b));
+        b.offsets = reinterpret_cast<const uint32_t*>(sb + o_off);
+        b.inst = reinterpret_cast<const uint32_t*>(sb + o_inst);
+        b.class_mask = use_mask ? reinterpret_cast<const uint32_t*>(sb + o_mask) : nullptr;
+        b.n_cand = n_cand;
+        b.n_inst = h_inst.size();
+        b.budget = gpus;
+        maaso_eval_opts o;
+        memset(&o, 0, sizeof(o));
+        o.flags = flags;
+        o.rejected_by_model = reinterpret_cast<uint32_t*>(sb + o_rbm);
+        int r = maaso_eval_placements(ctx, trace, &b, &o, reinterpret_cast<maaso_result*>(sb + o_res), st);
+        if (r != MAASO_OK) return r;
+        r = maaso_score(ctx, reinterpret_cast<const maaso_result*>(sb + o_res), n_cand, score,
+                        reinterpret_cast<double*>(sb + o_sc), st);
+        if (r != MAASO_OK) return r;
+        e = cudaMemcpyAsync(h_sc.data(), sb + o_sc, n_cand * 8, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(h_rbm.data(), sb + o_rbm, (size_t)n_cand * MAASO_MAX_MODELS * 4,
+                                cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "ins_deploy: download");
+        return MAASO_OK;
+    };
+
+    // R_res = R_x before anything is deployed: the empty placement rejects every request of R_x
+    h_off[0] = 0;
+    h_off[1] = 0;
+    rc = run_batch(1);
+    if (rc != MAASO_OK) return rc;
+
+    struct Step {
+        uint32_t k;    // device count of the placement before the tentative instance was added
+        uint32_t len;  // instances of the accepted placement after the step
+        double phi;    // its score after the step
+    };
+    struct Chain {
+        std::vector<uint32_t> inst;  // accepted placement I (instances are only ever appended)
+        std::vector<Step> steps;
+        bool sat[MAASO_MAX_MODELS];
+        uint32_t unserved[MAASO_MAX_MODELS];
+        double phi;
+        uint32_t dev;
+        int tentative;  // model of the tentative instance, -1 = chain finished
+    };
+    std::vector<Chain> chains(C);
+    for (uint32_t c = 0; c < C; c++) {
+        Chain& ch = chains[c];
+        memset(ch.sat, 0, sizeof(ch.sat));
+        memcpy(ch.unserved, h_rbm.data(), sizeof(ch.unserved));
+        ch.phi = 0.0;
+        ch.dev = (uint32_t)ctx->h_devices[configs[c].strategy];
+        ch.tentative = 0;
+    }
+    std::vector<uint32_t> batch_chain;
+    for (;;) {
+        // every unfinished chain proposes its next tentative placement I' = I + (m', P, B)
+        batch_chain.clear();
+        h_inst.clear();
+        for (uint32_t c = 0; c < C; c++) {
+            Chain& ch = chains[c];
+            if (ch.tentative < 0) continue;
+            int mp = -1;  // model with the most unserved requests among the non-saturated ones
+            if ((uint64_t)ch.inst.size() * ch.dev < gpus && ch.inst.size() <= MAASO_MAX_INSTANCES)
+                for (uint32_t m = 0; m < ctx->n_models; m++)
+                    if (!ch.sat[m] && (mp < 0 || ch.unserved[m] > ch.unserved[mp])) mp = (int)m;
+            ch.tentative = mp;
+            if (mp < 0) continue;
+            h_off[batch_chain.size()] = (uint32_t)h_inst.size();
+            h_inst.insert(h_inst.end(), ch.inst.begin(), ch.inst.end());
+            h_inst.push_back(((uint32_t)mp & 0xFu) | ((configs[c].strategy & 0xFFu) << 4) |
+                             ((configs[c].batch & 0xFFu) << 12));
+            batch_chain.push_back(c);
+        }
+        if (batch_chain.empty()) break;
+        h_off[batch_chain.size()] = (uint32_t)h_inst.size();
+        rc = run_batch((uint32_t)batch_chain.size());
+        if (rc != MAASO_OK) return rc;
+        for (size_t j = 0; j < batch_chain.size(); j++) {
+            Chain& ch = chains[batch_chain[j]];
+            Step sp;
+            sp.k = (uint32_t)ch.inst.size() * ch.dev;
+            if (h_sc[j] > ch.phi) {  // accept the new instance
+                ch.phi = h_sc[j];
+                ch.inst.push_back(h_inst[h_off[j + 1] - 1]);
+                memcpy(ch.unserved, h_rbm.data() + j * MAASO_MAX_MODELS, sizeof(ch.unserved));
+            } else {
+                ch.sat[ch.tentative] = true;  // stop deploying this model
+            }
+            sp.len = (uint32_t)ch.inst.size();
+            sp.phi = ch.phi;
+            ch.steps.push_back(sp);
+        }
+    }
+    // Phi*[k] / I*[k]: replay the steps configuration by configuration, as the sequential algorithm
+    // would have met them ("first strictly better wins")
+    for (uint32_t c = 0; c < C; c++)
+        for (const Step& sp : chains[c].steps)
+            if (sp.k <= gpus && sp.phi > phi_star[sp.k]) {
+                phi_star[sp.k] = sp.phi;
+                istar_len[sp.k] = sp.len;
+                for (uint32_t i = 0; i < sp.len && i < MAASO_MAX_INSTANCES; i++)
+                    istar_inst[(size_t)sp.k * MAASO_MAX_INSTANCES + i] = chains[c].inst[i];
+            }
     return MAASO_OK;
 }
 

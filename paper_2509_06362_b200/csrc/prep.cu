@@ -32,6 +32,8 @@ __global__ void prep_kernel(const EvalParams P) {
         }
     }
     if (P.dump_row) P.dump_row[c] = -1;
+    if (P.rej_by_model)
+        for (int m = 0; m < MAASO_MAX_MODELS; m++) P.rej_by_model[(size_t)c * MAASO_MAX_MODELS + m] = 0;
     if (status) {
         uint4* o = reinterpret_cast<uint4*>(P.out + c);
         o[0] = make_uint4(status, 0, 0, 0);

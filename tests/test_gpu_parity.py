@@ -328,6 +328,49 @@ def test_score_and_ranking_by_score(ctx, oracle_mod):
     ctx.free_trace(t)
 
 
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_rejected_by_model(ctx, oracle_mod, mapping):
+    import torch
+    cfg = gen.make_config("multimodel", n_cand=300, n_req=2500)
+    tr = cfg["traces"][0]
+    lists = [[(2, 0, 4)], []]                       # an invalid candidate and the empty placement
+    off2, inst2 = gen.candidates_from_lists(lists)
+    off = np.concatenate([cfg["offsets"], cfg["offsets"][-1] + off2[1:]]).astype(np.uint32)
+    inst = np.concatenate([cfg["inst"], inst2]).astype(np.uint32)
+    mask = np.random.default_rng(2).integers(1, 8, size=len(off) - 1).astype(np.uint32)
+    ctx.load_profile(cfg["profile"])
+    t = ctx.load_trace(tr, cfg["classes"])
+    rbm = torch.full((len(off) - 1, 16), 77, dtype=torch.int32, device="cuda")
+    ctx.eval_placements(t, ctx.to_device(off), ctx.to_device(inst), 32, ctx.to_device(mask), mapping=mapping,
+                        rejected_by_model=rbm)
+    torch.cuda.synchronize()
+    want = oracle_mod.rejected_by_model(cfg["profile"], tr, cfg["classes"], off, inst, 32, mask)
+    assert (rbm.cpu().numpy().view(np.uint32) == want).all()
+    ctx.free_trace(t)
+
+
+def test_ins_deploy_matches_oracle(ctx, oracle_mod):
+    """Alg. 1 driven on the GPU (one batch of tentative placements per greedy step) against the
+    sequential oracle: identical scores (same doubles) and identical placements per device count."""
+    prof = gen.profile_multimodel(0)
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 180_000_000)])
+    ctx.load_profile(prof)
+    cases = [
+        (gen.make_trace(3000, 30.0, 3, model_mix=(0.2, 0.7, 0.1)), 16, [(0, 8), (1, 16), (3, 8), (3, 64), (6, 16), (0, 1)], None),
+        (gen.make_trace(2000, 60.0, 4, cv=2.0, model_mix=(0.6, 0.3, 0.1)), 24,
+         [(s, b) for s in (0, 1, 3, 6) for b in (4, 16, 64)], 0b011),
+        (gen.make_trace(500, 5.0, 5, model_mix=(1.0, 0.0, 0.0)), 3, [(6, 16), (0, 2)], None),
+    ]
+    for tr, gpus, configs, mask in cases:
+        t = ctx.load_trace(tr, classes)
+        for alpha in (4.0, 10.0):
+            phi, I = ctx.ins_deploy(t, gpus, configs, alpha, 0.3, 3000.0, 5.0, class_mask=mask)
+            wphi, wI = oracle_mod.ins_deploy(prof, tr, classes, gpus, configs, alpha, 0.3, 3000.0, 5.0, class_mask=mask)
+            assert phi.tolist() == wphi.tolist()
+            assert [x.tolist() for x in I] == [x.tolist() for x in wI]
+        ctx.free_trace(t)
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")

@@ -368,3 +368,67 @@ def test_score_properties_and_ranking(oracle_mod):
     want = sorted(range(len(s)), key=lambda i: (np.isnan(s[i]), -s[i] if not np.isnan(s[i]) else 0.0, i))
     assert oracle_mod.topk_scores(s, 143).tolist() == want
     assert oracle_mod.topk_scores(s, 10).tolist() == want[:10]
+
+
+# ---- Alg. 1: simulator-based instance configuration -------------------------------------------
+def test_ins_deploy_worked_example(oracle_mod):
+    """Requests 400 s apart on a one-model profile: one instance serves everything, a second one
+    changes nothing, so the score does not improve, the model saturates and the search stops.
+    With k = device count before the addition (as printed), slot 0 gets the one-instance placement
+    in the first step and slot 1 gets the same placement in the second."""
+    prof = gen.profile_tiny()
+    tr = gen.make_trace(40, 1.0, 5, doc_class=None)
+    tr["arrival_us"] = np.arange(40, dtype=np.int64) * 400_000_000
+    classes = gen.make_classes(NONE3 * 3)
+    phi, I = oracle_mod.ins_deploy(prof, tr, classes, 3, [(0, 4)], 4.0, 0.3, 1000.0, 10.0)
+    # closed form of the score: every request is a hit, first token = arrival + prefill
+    base, q16, s1 = int(prof["prefill_base_us"][0, 0]), int(prof["prefill_q16"][0, 0]), int(prof["step_us"][0, 0, 0])
+    pre = base + ((q16 * tr["in_tokens"].astype(np.int64) + 32768) >> 16)
+    fin = tr["arrival_us"] + pre + (tr["out_tokens"].astype(np.int64) - 1) * s1
+    thr = tr["out_tokens"].astype(np.int64).sum() / (fin.max() * 1e-6)
+    lat = pre.sum() / 40 * 1e-6
+    want = 4.0 * 1.0 + 0.3 * min(thr, 1000.0) / 1000.0 + 0.7 * max(10.0 - lat, 0.0) / 10.0
+    assert phi[0] == pytest.approx(want, rel=1e-12) and phi[1] == phi[0]
+    assert phi[2] == 0.0 and phi[3] == 0.0
+    assert I[0].tolist() == [int(gen.pack_inst(0, 0, 4))] and I[1].tolist() == I[0].tolist()
+    assert len(I[2]) == 0 and len(I[3]) == 0
+
+
+def test_ins_deploy_properties(oracle_mod):
+    prof = gen.profile_multimodel(0)
+    tr = gen.make_trace(1200, 25.0, 3, model_mix=(0.2, 0.7, 0.1))
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 180_000_000)])
+    configs = [(0, 8), (1, 16), (3, 8), (3, 64), (6, 16)]
+    gpus = 12
+    phi, I = oracle_mod.ins_deploy(prof, tr, classes, gpus, configs, 4.0, 0.3, 2000.0, 5.0)
+    assert (phi >= 0).all() and phi.max() > 0
+    for k in range(gpus + 1):
+        if len(I[k]) == 0:
+            assert phi[k] == 0.0
+            continue
+        m, s, b = gen.unpack_inst(I[k])
+        assert len(set(zip(s.tolist(), b.tolist()))) == 1 and (int(s[0]), int(b[0])) in configs  # one (P, B) per solution
+        assert prof["devices"][s].sum() <= gpus
+        assert (prof["devices"][s] >= prof["min_devices"][m]).all()
+        # the stored score is the score of the stored placement
+        off = np.array([0, len(I[k])], dtype=np.uint32)
+        rec = oracle_mod.eval_placements(prof, tr, classes, off, I[k], gpus)
+        assert oracle_mod.score(rec, 4.0, 0.3, 2000.0, 5.0)[0] == phi[k]
+    # the first instance of every chain serves the model with the most requests (model 1 here)
+    assert int(gen.unpack_inst(I[0])[0][0]) == 1
+    # a strategy that needs more devices than the sub-cluster has can never be deployed
+    phi2, I2 = oracle_mod.ins_deploy(prof, tr, classes, 4, [(6, 16)], 4.0, 0.3, 2000.0, 5.0)
+    assert (phi2 == 0).all() and all(len(x) == 0 for x in I2)
+    # the SLO weight only rescales: with alpha = 10 (MaaSO*) no slot scores less than with alpha = 4
+    phi10, _ = oracle_mod.ins_deploy(prof, tr, classes, gpus, configs, 10.0, 0.3, 2000.0, 5.0)
+    assert (phi10 >= phi - 1e-12).all()
+
+
+def test_rejected_by_model_matches_dumps(oracle_mod):
+    cfg = gen.make_config("multimodel", n_cand=40, n_req=1500)
+    tr = cfg["traces"][0]
+    rbm = oracle_mod.rejected_by_model(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 32)
+    res = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 32)
+    assert (rbm.sum(axis=1) == res["n_rejected"]).all()
+    assert (rbm[:, 3:] == 0).all()
+    assert (rbm <= np.bincount(tr["model"], minlength=16)[None, :]).all()
