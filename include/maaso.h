@@ -244,6 +244,20 @@ MAASO_API int maaso_ins_deploy(maaso_ctx *ctx, const maaso_trace *trace, uint32_
                                uint32_t class_mask, const maaso_score_params *score, uint32_t flags,
                                double *phi_star, uint32_t *istar_len, uint32_t *istar_inst);
 
+/* Alg. 2, "Dynamic Resource Partition", for two sub-clusters: R_t / R_l are the requests whose
+ * class bit is set in mask_t / mask_l.  G'_l = floor(|R_l| * gpus / (|R_t| + |R_l|));
+ * maaso_ins_deploy on (R_l, G'_l) and on (R_t, gpus); Phi_opt starts at the best score of
+ * maaso_ins_deploy on (R_t + R_l, gpus) if `baseline` is non-zero (homogeneous fallback), else
+ * at 0; then g_l = 1..G'_l, g_t = gpus - g_l, keeping the pair with the largest
+ * Phi_t*[g_t] + Phi_l*[g_l] if it is strictly better.  Host outputs: out_g[2] = (g_t, g_l), both 0
+ * when no partition beat Phi_opt; *out_phi; the two placements (packed words, up to
+ * MAASO_MAX_INSTANCES each) with their lengths.  Synchronous. */
+MAASO_API int maaso_partition(maaso_ctx *ctx, const maaso_trace *trace, uint32_t mask_t, uint32_t mask_l,
+                              uint32_t gpus, const maaso_config *configs, uint32_t n_configs,
+                              const maaso_score_params *score, uint32_t flags, int baseline, uint32_t *out_g,
+                              double *out_phi, uint32_t *len_t, uint32_t *inst_t, uint32_t *len_l,
+                              uint32_t *inst_l);
+
 /* Top-k without any allocation.  (The paper has no counterpart; this is a deployment
  * variant of maaso_topk.)  It is meant for callers that must not allocate device memory
  * while they run: code inside a memory-pool or arena framework that owns all device memory,

@@ -53,6 +53,7 @@ def _load():
         _lib.orc_topk_scores.restype = C.c_int
         _lib.orc_rejected_by_model.restype = C.c_int
         _lib.orc_ins_deploy.restype = C.c_int
+        _lib.orc_partition.restype = C.c_int
     return _lib
 
 
@@ -208,6 +209,30 @@ def ins_deploy(profile, trace, classes, gpus, configs, alpha, beta, gamma_t, gam
         raise RuntimeError(f"oracle ins_deploy failed with code {rc}")
     del keep
     return phi, [iinst[k, :ilen[k]].copy() for k in range(gpus + 1)]
+
+
+def partition(profile, trace, classes, mask_t, mask_l, gpus, configs, alpha, beta, gamma_t, gamma_l, flags=0,
+              baseline=False):
+    """Alg. 2 (see orc_partition).  Returns dict(g_t, g_l, phi, inst_t, inst_l)."""
+    lib = _load()
+    p, keep = _profile_struct(profile)
+    trace = np.ascontiguousarray(trace, dtype=_REQ)
+    classes = np.ascontiguousarray(classes, dtype=_SLO)
+    cfg = np.ascontiguousarray(np.asarray(configs, dtype=np.uint32).reshape(-1, 2))
+    sp = _ScoreParams(alpha, beta, gamma_t, gamma_l)
+    g = np.zeros(2, dtype=np.uint32)
+    phi = C.c_double(0.0)
+    lt, ll = C.c_uint32(0), C.c_uint32(0)
+    it, il = np.zeros(128, dtype=np.uint32), np.zeros(128, dtype=np.uint32)
+    rc = lib.orc_partition(C.byref(p), _ptr(trace), C.c_uint64(len(trace)), _ptr(classes), C.c_uint32(len(classes)),
+                           C.c_uint32(mask_t), C.c_uint32(mask_l), C.c_uint32(gpus), _ptr(cfg), C.c_uint32(len(cfg)),
+                           C.byref(sp), C.c_uint32(flags), C.c_int(1 if baseline else 0), _ptr(g), C.byref(phi),
+                           C.byref(lt), _ptr(it), C.byref(ll), _ptr(il))
+    if rc != 0:
+        raise RuntimeError(f"oracle partition failed with code {rc}")
+    del keep
+    return {"g_t": int(g[0]), "g_l": int(g[1]), "phi": phi.value, "inst_t": it[:lt.value].copy(),
+            "inst_l": il[:ll.value].copy()}
 
 
 def topk_scores(scores, k):

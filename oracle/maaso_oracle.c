@@ -483,6 +483,59 @@ int orc_ins_deploy(const orc_profile *p, const orc_request *reqs, uint64_t n, co
     return 0;
 }
 
+/*
+ * Alg. 2, "Dynamic Resource Partition", taken literally.  R_t / R_l = requests whose class bit
+ * is set in mask_t / mask_l (byRequestSLO); G'_l = floor(|R_l| / |R| * |G|) with |R| = |R_t| + |R_l|
+ * (integer arithmetic); Alg. 1 on (R_l, G'_l) and on (R_t, G); Phi_opt starts at the best
+ * homogeneous score max_k Phi*[k] of Alg. 1 on (R, G) if `baseline` is set, else at 0; then for
+ * g_l = 1 .. G'_l with g_t = |G| - g_l the pair maximising Phi_t*[g_t] + Phi_l*[g_l] is kept
+ * (strictly better only).  Outputs: out_g[2] = (g_t, g_l), both 0 if no partition beat Phi_opt;
+ * *out_phi = Phi_opt; placements of the chosen pair (lengths 0 if none).
+ */
+int orc_partition(const orc_profile *p, const orc_request *reqs, uint64_t n, const orc_slo *classes,
+                  uint32_t n_classes, uint32_t mask_t, uint32_t mask_l, uint32_t gpus, const orc_config *configs,
+                  uint32_t n_configs, const orc_score_params *sp, uint32_t flags, int baseline, uint32_t *out_g,
+                  double *out_phi, uint32_t *len_t, uint32_t *inst_t, uint32_t *len_l, uint32_t *inst_l) {
+    uint64_t n_t = 0, n_l = 0;
+    for (uint64_t q = 0; q < n; q++) {
+        if ((mask_t >> reqs[q].cls) & 1u) n_t++;
+        if ((mask_l >> reqs[q].cls) & 1u) n_l++;
+    }
+    const uint32_t gl_max = (n_t + n_l) ? (uint32_t)((n_l * (uint64_t)gpus) / (n_t + n_l)) : 0;
+    size_t cells = (size_t)gpus + 1;
+    double *phi_t = (double *)malloc(cells * sizeof(double)), *phi_l = (double *)malloc(cells * sizeof(double));
+    double *phi_h = (double *)malloc(cells * sizeof(double));
+    uint32_t *ln_t = (uint32_t *)malloc(cells * 4), *ln_l = (uint32_t *)malloc(cells * 4), *ln_h = (uint32_t *)malloc(cells * 4);
+    uint32_t *in_t = (uint32_t *)malloc(cells * ORC_MAX_INST * 4), *in_l = (uint32_t *)malloc(cells * ORC_MAX_INST * 4);
+    uint32_t *in_h = (uint32_t *)malloc(cells * ORC_MAX_INST * 4);
+    int rc = -1;
+    if (phi_t && phi_l && phi_h && ln_t && ln_l && ln_h && in_t && in_l && in_h) {
+        rc = orc_ins_deploy(p, reqs, n, classes, n_classes, 1, mask_l, gl_max, configs, n_configs, sp, flags, phi_l, ln_l, in_l);
+        if (!rc) rc = orc_ins_deploy(p, reqs, n, classes, n_classes, 1, mask_t, gpus, configs, n_configs, sp, flags, phi_t, ln_t, in_t);
+        double phi_opt = 0.0;
+        if (!rc && baseline) {
+            rc = orc_ins_deploy(p, reqs, n, classes, n_classes, 1, mask_t | mask_l, gpus, configs, n_configs, sp, flags, phi_h, ln_h, in_h);
+            for (uint32_t k = 0; !rc && k <= gpus; k++) if (phi_h[k] > phi_opt) phi_opt = phi_h[k];
+        }
+        if (!rc) {
+            out_g[0] = out_g[1] = 0; *len_t = *len_l = 0;
+            for (uint32_t gl = 1; gl <= gl_max; gl++) {
+                const uint32_t gt = gpus - gl;
+                if (phi_t[gt] + phi_l[gl] > phi_opt) {
+                    phi_opt = phi_t[gt] + phi_l[gl];
+                    out_g[0] = gt; out_g[1] = gl;
+                    *len_t = ln_t[gt]; *len_l = ln_l[gl];
+                    memcpy(inst_t, in_t + (size_t)gt * ORC_MAX_INST, ln_t[gt] * 4);
+                    memcpy(inst_l, in_l + (size_t)gl * ORC_MAX_INST, ln_l[gl] * 4);
+                }
+            }
+            *out_phi = phi_opt;
+        }
+    }
+    free(phi_t); free(phi_l); free(phi_h); free(ln_t); free(ln_l); free(ln_h); free(in_t); free(in_l); free(in_h);
+    return rc;
+}
+
 /* Ranking by score (order 1): higher score first, then lower index; NaN scores last. */
 static const double *g_score;
 static int cmp_score(const void *pa, const void *pb) {

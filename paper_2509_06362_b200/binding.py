@@ -84,6 +84,9 @@ def _load():
     lib.maaso_topk_scores.argtypes = [vp, vp, vp, u64, u32, vp, vp, vp]
     lib.maaso_ins_deploy.argtypes = [vp, vp, u32, vp, u32, C.c_int, u32, C.POINTER(_ScoreParams), u32, vp, vp, vp]
     lib.maaso_ins_deploy.restype = C.c_int
+    lib.maaso_partition.argtypes = [vp, vp, u32, u32, u32, vp, u32, C.POINTER(_ScoreParams), u32, C.c_int, vp,
+                                    C.POINTER(C.c_double), C.POINTER(u32), vp, C.POINTER(u32), vp]
+    lib.maaso_partition.restype = C.c_int
     lib.maaso_topk_noalloc.argtypes = [vp, u64, u32, u32, vp, vp, vp]
     lib.maaso_topk_noalloc.restype = C.c_int
     lib.maaso_set_timing.argtypes = [vp, C.c_int]
@@ -239,6 +242,22 @@ def maaso_ins_deploy(ctx, trace, gpus, configs, alpha, beta, gamma_t, gamma_l, c
     return phi, [iinst[k, :ilen[k]].copy() for k in range(gpus + 1)]
 
 
+def maaso_partition(ctx, trace, mask_t, mask_l, gpus, configs, alpha, beta, gamma_t, gamma_l, flags=0,
+                    baseline=False):
+    """Alg. 2 for two sub-clusters.  Returns dict(g_t, g_l, phi, inst_t, inst_l)."""
+    cfg = np.ascontiguousarray(np.asarray(configs, dtype=np.uint32).reshape(-1, 2))
+    p = _ScoreParams(float(alpha), float(beta), float(gamma_t), float(gamma_l))
+    g = np.zeros(2, dtype=np.uint32)
+    phi = C.c_double(0.0)
+    lt, ll = C.c_uint32(0), C.c_uint32(0)
+    it, il = np.zeros(128, dtype=np.uint32), np.zeros(128, dtype=np.uint32)
+    _check(_lib.maaso_partition(ctx, trace, int(mask_t), int(mask_l), int(gpus), cfg.ctypes.data, len(cfg),
+                                C.byref(p), int(flags), 1 if baseline else 0, g.ctypes.data, C.byref(phi),
+                                C.byref(lt), it.ctypes.data, C.byref(ll), il.ctypes.data), "maaso_partition", ctx)
+    return {"g_t": int(g[0]), "g_l": int(g[1]), "phi": phi.value, "inst_t": it[:lt.value].copy(),
+            "inst_l": il[:ll.value].copy()}
+
+
 NOALLOC_MAX_CAND = 1 << 20
 NOALLOC_MAX_K = 64
 
@@ -308,6 +327,11 @@ class Context:
         """uint32 numpy words -> int32 CUDA tensor with the same bits"""
         t = self.torch.from_numpy(np.ascontiguousarray(words, dtype=np.uint32).view(np.int32))
         return t.to(self.device)
+
+    def partition(self, trace, mask_t, mask_l, gpus, configs, alpha, beta, gamma_t, gamma_l, flags=0,
+                  baseline=False):
+        return maaso_partition(self.handle, trace.handle, mask_t, mask_l, gpus, configs, alpha, beta, gamma_t,
+                               gamma_l, flags, baseline)
 
     def ins_deploy(self, trace, gpus, configs, alpha, beta, gamma_t, gamma_l, class_mask=None, flags=0):
         return maaso_ins_deploy(self.handle, trace.handle, gpus, configs, alpha, beta, gamma_t, gamma_l,

@@ -678,6 +678,77 @@ MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_
     return MAASO_OK;
 }
 
+// Alg. 2 for two sub-clusters on top of maaso_ins_deploy.
+MAASO_API int maaso_partition(maaso_ctx* ctx, const maaso_trace* trace, uint32_t mask_t, uint32_t mask_l,
+                              uint32_t gpus, const maaso_config* configs, uint32_t n_configs,
+                              const maaso_score_params* score, uint32_t flags, int baseline, uint32_t* out_g,
+                              double* out_phi, uint32_t* len_t, uint32_t* inst_t, uint32_t* len_l,
+                              uint32_t* inst_l) {
+    if (!ctx || !trace || !out_g || !out_phi || !len_t || !inst_t || !len_l || !inst_l || gpus > 4096)
+        return MAASO_EINVAL;
+    if (trace->owner != ctx) return fail(ctx, MAASO_ESTATE, "partition: trace belongs to another context");
+    // |R_t|, |R_l|: what the empty placement counts under each mask
+    DeviceGuard g(ctx->device);
+    int rc = grow(ctx, &ctx->deploy, &ctx->deploy_bytes, 4096);
+    if (rc != MAASO_OK) return rc;
+    unsigned char* sb = static_cast<unsigned char*>(ctx->deploy);
+    const uint32_t h_off[3] = {0, 0, 0}, h_mask[2] = {mask_t, mask_l};
+    maaso_result h_res[2];
+    cudaStream_t st = ctx->own_stream;
+    cudaError_t e = cudaMemcpyAsync(sb, h_off, sizeof(h_off), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sb + 256, h_mask, sizeof(h_mask), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "partition: upload");
+    maaso_cand_batch b;
+    memset(&b, 0, sizeof(b));
+    b.offsets = reinterpret_cast<const uint32_t*>(sb);
+    b.inst = reinterpret_cast<const uint32_t*>(sb + 512);
+    b.class_mask = reinterpret_cast<const uint32_t*>(sb + 256);
+    b.n_cand = 2;
+    b.budget = gpus;
+    rc = maaso_eval_placements(ctx, trace, &b, nullptr, reinterpret_cast<maaso_result*>(sb + 1024), st);
+    if (rc != MAASO_OK) return rc;
+    e = cudaMemcpyAsync(h_res, sb + 1024, sizeof(h_res), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "partition: download");
+    const uint64_t n_t = h_res[0].n_counted, n_l = h_res[1].n_counted;
+    const uint32_t gl_max = (n_t + n_l) ? (uint32_t)((n_l * (uint64_t)gpus) / (n_t + n_l)) : 0;
+
+    const size_t cells = (size_t)gpus + 1;
+    std::vector<double> phi_t(cells), phi_l(cells), phi_h(cells);
+    std::vector<uint32_t> ln_t(cells), ln_l(cells), ln_h(cells);
+    std::vector<uint32_t> in_t(cells * MAASO_MAX_INSTANCES), in_l(cells * MAASO_MAX_INSTANCES),
+        in_h(cells * MAASO_MAX_INSTANCES);
+    rc = maaso_ins_deploy(ctx, trace, gl_max, configs, n_configs, 1, mask_l, score, flags, phi_l.data(),
+                          ln_l.data(), in_l.data());
+    if (rc == MAASO_OK)
+        rc = maaso_ins_deploy(ctx, trace, gpus, configs, n_configs, 1, mask_t, score, flags, phi_t.data(),
+                              ln_t.data(), in_t.data());
+    double phi_opt = 0.0;
+    if (rc == MAASO_OK && baseline) {  // homogeneous deployment as the fallback
+        rc = maaso_ins_deploy(ctx, trace, gpus, configs, n_configs, 1, mask_t | mask_l, score, flags, phi_h.data(),
+                              ln_h.data(), in_h.data());
+        for (uint32_t k = 0; rc == MAASO_OK && k <= gpus; k++)
+            if (phi_h[k] > phi_opt) phi_opt = phi_h[k];
+    }
+    if (rc != MAASO_OK) return rc;
+    out_g[0] = out_g[1] = 0;
+    *len_t = *len_l = 0;
+    for (uint32_t gl = 1; gl <= gl_max; gl++) {
+        const uint32_t gt = gpus - gl;
+        if (phi_t[gt] + phi_l[gl] > phi_opt) {
+            phi_opt = phi_t[gt] + phi_l[gl];
+            out_g[0] = gt;
+            out_g[1] = gl;
+            *len_t = ln_t[gt];
+            *len_l = ln_l[gl];
+            memcpy(inst_t, in_t.data() + (size_t)gt * MAASO_MAX_INSTANCES, ln_t[gt] * 4);
+            memcpy(inst_l, in_l.data() + (size_t)gl * MAASO_MAX_INSTANCES, ln_l[gl] * 4);
+        }
+    }
+    *out_phi = phi_opt;
+    return MAASO_OK;
+}
+
 MAASO_API int maaso_set_timing(maaso_ctx* ctx, int enabled) {
     if (!ctx) return MAASO_EINVAL;
     DeviceGuard g(ctx->device);

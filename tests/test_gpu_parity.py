@@ -371,6 +371,22 @@ def test_ins_deploy_matches_oracle(ctx, oracle_mod):
         ctx.free_trace(t)
 
 
+def test_partition_matches_oracle(ctx, oracle_mod):
+    prof = gen.profile_multimodel(0)
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 180_000_000)])
+    ctx.load_profile(prof)
+    tr = gen.make_trace(2500, 30.0, 6, cv=2.0, model_mix=(0.6, 0.3, 0.1))
+    t = ctx.load_trace(tr, classes)
+    configs = [(s, b) for s in (0, 1, 3) for b in (4, 16, 64)]
+    for (mt, ml, base) in [(0b001, 0b110, False), (0b011, 0b100, True), (0b111, 0, False)]:
+        got = ctx.partition(t, mt, ml, 16, configs, 4.0, 0.3, 3000.0, 5.0, baseline=base)
+        want = oracle_mod.partition(prof, tr, classes, mt, ml, 16, configs, 4.0, 0.3, 3000.0, 5.0, baseline=base)
+        assert (got["g_t"], got["g_l"], got["phi"]) == (want["g_t"], want["g_l"], want["phi"])
+        assert got["inst_t"].tolist() == want["inst_t"].tolist()
+        assert got["inst_l"].tolist() == want["inst_l"].tolist()
+    ctx.free_trace(t)
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")

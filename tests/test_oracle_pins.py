@@ -432,3 +432,32 @@ def test_rejected_by_model_matches_dumps(oracle_mod):
     assert (rbm.sum(axis=1) == res["n_rejected"]).all()
     assert (rbm[:, 3:] == 0).all()
     assert (rbm <= np.bincount(tr["model"], minlength=16)[None, :]).all()
+
+
+# ---- Alg. 2: dynamic resource partition -----------------------------------------------------
+def test_partition_scan(oracle_mod):
+    prof = gen.profile_multimodel(0)
+    tr = gen.make_trace(1500, 20.0, 3, model_mix=(0.6, 0.3, 0.1))
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 180_000_000)])
+    configs = [(0, 8), (1, 16), (3, 8), (3, 64)]
+    gpus, mt, ml = 12, 0b001, 0b110
+    args = (4.0, 0.3, 2000.0, 5.0)
+    got = oracle_mod.partition(prof, tr, classes, mt, ml, gpus, configs, *args)
+    n_l = int(((ml >> tr["cls"]) & 1).sum())
+    gl_max = n_l * gpus // len(tr)
+    phi_l, I_l = oracle_mod.ins_deploy(prof, tr, classes, gl_max, configs, *args, class_mask=ml)
+    phi_t, I_t = oracle_mod.ins_deploy(prof, tr, classes, gpus, configs, *args, class_mask=mt)
+    best, arg = 0.0, (0, 0)
+    for gl in range(1, gl_max + 1):            # brute-force scan, first strictly better wins
+        if phi_t[gpus - gl] + phi_l[gl] > best:
+            best, arg = phi_t[gpus - gl] + phi_l[gl], (gpus - gl, gl)
+    assert (got["g_t"], got["g_l"]) == arg and got["phi"] == best
+    assert got["g_t"] + got["g_l"] == gpus
+    assert got["inst_t"].tolist() == I_t[arg[0]].tolist() and got["inst_l"].tolist() == I_l[arg[1]].tolist()
+    # homogeneous fallback: an unbeatable baseline leaves the cluster unpartitioned
+    phi_h, _ = oracle_mod.ins_deploy(prof, tr, classes, gpus, configs, *args, class_mask=mt | ml)
+    with_base = oracle_mod.partition(prof, tr, classes, mt, ml, gpus, configs, *args, baseline=True)
+    assert with_base["phi"] == max(best, phi_h.max())
+    # no latency-tolerant requests -> G'_l = 0 -> nothing to scan
+    none = oracle_mod.partition(prof, tr, classes, 0b111, 0, gpus, configs, *args)
+    assert (none["g_t"], none["g_l"], none["phi"]) == (0, 0, 0.0) and len(none["inst_t"]) == 0
