@@ -24,6 +24,13 @@ METRIC = "candidate x request evaluations per second"
 UNIT = "evals/s"
 TOPK = 64
 
+# ncu counters of eval_group_kernel on the default workload (profiles/eval_group_kernel_node_sweep.md).
+# They describe the kernel as committed with that summary; set to None when the kernel changes.
+PROFILED = {"workload": "node", "mapping": 0,
+            "dram_bytes_per_launch": 11_255_040 + 3_470_336,
+            "warp_inst_per_launch": 6_513_415_397}
+SM_COUNT, ISSUE_PER_SM = 148, 4   # B200: 148 SMs x 4 warp schedulers, one warp instruction per cycle each
+
 
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -279,6 +286,17 @@ def main():
     dom_ms = statistics.mean(k[dom] for k in kernel_ms)
     abytes = algorithmic_bytes(cfg, evals_per_step)
     achieved = abytes / (dom_ms * 1e-3) / 1e9
+    profiled = (PROFILED if PROFILED and args.workload == PROFILED["workload"] and args.mapping == PROFILED["mapping"]
+                and args.n_cand is None and args.n_req is None else None)
+    sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    alu_peak = SM_COUNT * ISSUE_PER_SM * sm_mhz * 1e6
+    alu = None
+    if profiled:
+        ach = profiled["warp_inst_per_launch"] / (dom_ms * 1e-3)
+        alu = {"bound": "alu", "kernel": "eval_group_kernel", "achieved": ach / 1e9, "peak": alu_peak / 1e9,
+               "unit": "G warp-instructions/s", "frac": ach / alu_peak,
+               "peak_kind": f"{SM_COUNT} SMs x {ISSUE_PER_SM} issue slots x {sm_mhz:.0f} MHz sampled during the run",
+               "warp_inst_per_eval": profiled["warp_inst_per_launch"] / evals_per_step}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -294,10 +312,12 @@ def main():
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "eval_group_kernel" if args.mapping == 0 else "eval_block_kernel",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "peak_kind": f"of {peak_kind}",
+                     "traffic": profiled["dram_bytes_per_launch"] if profiled else None,
                      "algorithmic_bytes_per_launch": abytes, "kernel_ms": dom_ms,
                      "note": "effective bytes (16 B trace record per evaluation); the path is bound by "
                              "integer issue of a dependent event chain, not by DRAM"},
+        "roofline_alu": alu,
         "kernel_ms": {k: statistics.mean(x[k] for x in kernel_ms) for k in kernel_ms[0]},
     }
     if not args.no_cpu_baseline:
