@@ -65,6 +65,11 @@ extern "C" {
 #define MAASO_FLAG_PRED_OPTIMISTIC 1u /* distributor predicts with the step time right after admission
                                          instead of the worst case F(M,P,B_I) of Sec. IV-F step 3 */
 
+#define MAASO_FLAG_TEST_STALL 0x80000000u /* test hook for the bounded device-side waits: the trace copies
+                                             are never issued and every wait is limited to about 0.1 s, so
+                                             each valid candidate must come back with MAASO_CAND_ETIMEOUT
+                                             and the call must return normally */
+
 /* maaso_eval_opts.mapping */
 #define MAASO_MAP_AUTO 0u  /* lanes-per-instance groups for <= 32 instances, one block otherwise */
 #define MAASO_MAP_BLOCK 1u /* one thread block per candidate, one warp per instance, lanes = slots */

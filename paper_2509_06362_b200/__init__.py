@@ -10,7 +10,7 @@ from .binding import (
     maaso_eval_placements, maaso_eval_placements_host, maaso_topk, maaso_ins_deploy, maaso_partition, maaso_score, maaso_topk_scores, maaso_topk_noalloc, NOALLOC_MAX_CAND, NOALLOC_MAX_K, maaso_launch_count, maaso_set_timing, maaso_get_timing,
     maaso_strerror, maaso_last_error, lib_path,
     REQUEST_DTYPE, SLO_DTYPE, RESULT_DTYPE,
-    FLAG_PRED_OPTIMISTIC, MAP_AUTO, MAP_BLOCK, MAP_GROUP, CAND_STATUS,
+    FLAG_PRED_OPTIMISTIC, FLAG_TEST_STALL, MAP_AUTO, MAP_BLOCK, MAP_GROUP, CAND_STATUS,
 )
 
 __all__ = [

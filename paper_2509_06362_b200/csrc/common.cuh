@@ -169,11 +169,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: false if the barrier did not complete within kWaitCycles.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
     return true;
 }
@@ -216,6 +216,8 @@ struct EvalParams {
     uint32_t* sm_ctr;        // [n_sm] next work item of each SM's share (lane-group kernel)
     uint32_t n_sm;
     uint32_t promote_pct;
+    long long wait_cycles;   // bound of every device-side wait
+    uint32_t stall_test;     // test hook: never issue the trace copies
     int32_t* dump_row;       // [n_cand] or null
     uint32_t dump_n;
     int64_t* dump_finish;

@@ -131,7 +131,7 @@ eval_block_kernel(const EvalParams P, const int tile_recs, const int bucket) {
         int64_t now = 0;
         uint32_t n_counted = 0, n_rejected = 0, status = 0, buf = 0;
         uint64_t attempts = 0;
-        if (tid == 0) {
+        if (tid == 0 && !P.stall_test) {
             for (uint32_t j = 0; j < (uint32_t)kBStages && j < n_tiles; j++) {
                 const uint32_t s = (tile_seq + j) % kBStages;
                 const uint32_t recs = min((uint32_t)tile_recs, P.n_req - j * tile_recs);
@@ -205,9 +205,9 @@ eval_block_kernel(const EvalParams P, const int tile_recs, const int bucket) {
 
         for (uint32_t t = 0; t < n_tiles; t++) {
             const uint32_t s = tile_seq % kBStages, parity = (tile_seq / kBStages) & 1u;
-            bool ok = mbar_wait_bounded(&full_bar[s], parity);
+            bool ok = mbar_wait_bounded(&full_bar[s], parity, P.wait_cycles);
             if (!__all_sync(0xFFFFFFFFu, ok)) {
-                mbar_wait_bounded(&full_bar[s], parity);
+                mbar_wait_bounded(&full_bar[s], parity, P.wait_cycles);
                 status = MAASO_CAND_ETIMEOUT;
                 work[1] = 1;  // the block stops taking work
             }

@@ -209,7 +209,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
         uint64_t attempts = 0;
 
         // trace staging: first tiles of this batch
-        if (tid == 0) {
+        if (tid == 0 && !P.stall_test) {
             for (uint32_t j = 0; j < (uint32_t)kStages && j < n_tiles; j++) {
                 const uint32_t s = (tile_seq + j) % kStages;
                 const uint32_t recs = min((uint32_t)tile_recs, P.n_req - j * tile_recs);
@@ -221,9 +221,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
 
         for (uint32_t t = 0; t < n_tiles; t++) {
             const uint32_t s = tile_seq % kStages, parity = (tile_seq / kStages) & 1u;
-            const bool arrived = mbar_wait_bounded(&sm.full_bar[s], parity);
+            const bool arrived = mbar_wait_bounded(&sm.full_bar[s], parity, P.wait_cycles);
             if (!__all_sync(0xFFFFFFFFu, arrived)) {
-                mbar_wait_bounded(&sm.full_bar[s], parity);  // give copies in flight one more bounded chance
+                mbar_wait_bounded(&sm.full_bar[s], parity, P.wait_cycles);  // give copies in flight one more bounded chance
                 status = MAASO_CAND_ETIMEOUT;
                 sm.work[1] = 1;
                 break;

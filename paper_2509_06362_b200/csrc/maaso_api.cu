@@ -336,7 +336,7 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     if (opts) o = *opts;
     if (o.mapping > MAASO_MAP_GROUP) return fail(ctx, MAASO_EINVAL, "eval: unknown mapping");
     if (o.dump_n && !o.dump_cand_idx) return fail(ctx, MAASO_EINVAL, "eval: dump_n without dump_cand_idx");
-    if (o.flags & ~MAASO_FLAG_PRED_OPTIMISTIC) return fail(ctx, MAASO_EINVAL, "eval: unknown flag");
+    if (o.flags & ~(MAASO_FLAG_PRED_OPTIMISTIC | MAASO_FLAG_TEST_STALL)) return fail(ctx, MAASO_EINVAL, "eval: unknown flag");
 
     DeviceGuard g(ctx->device);
     cudaStream_t stream = (cudaStream_t)cuda_stream;
@@ -362,7 +362,9 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.class_mask = cands->class_mask;
     P.n_cand = C;
     P.n_inst = (uint32_t)cands->n_inst;
-    P.flags = o.flags;
+    P.flags = o.flags & ~MAASO_FLAG_TEST_STALL;
+    P.stall_test = (o.flags & MAASO_FLAG_TEST_STALL) ? 1u : 0u;
+    P.wait_cycles = P.stall_test ? 200000000ll : kWaitCycles;
     P.mapping = o.mapping;
     P.out = out_results;
     P.dump_n = o.dump_n;

@@ -34,10 +34,15 @@ __global__ void prep_kernel(const EvalParams P) {
     if (P.dump_row) P.dump_row[c] = -1;
     if (P.rej_by_model)
         for (int m = 0; m < MAASO_MAX_MODELS; m++) P.rej_by_model[(size_t)c * MAASO_MAX_MODELS + m] = 0;
-    if (status) {
+    {
+        // Invalid candidates get their final record here.  Valid ones are pre-marked "not scored"
+        // (ETIMEOUT); the scoring kernel overwrites the record when it finishes the candidate, so a
+        // kernel that gave up on a bounded wait leaves no record undefined.
         uint4* o = reinterpret_cast<uint4*>(P.out + c);
-        o[0] = make_uint4(status, 0, 0, 0);
+        o[0] = make_uint4(status ? status : MAASO_CAND_ETIMEOUT, 0, 0, 0);
         for (int i = 1; i < 8; i++) o[i] = make_uint4(0, 0, 0, 0);
+    }
+    if (status) {
         P.code[c] = 0xFFFFFFFFu;
         return;
     }

@@ -387,6 +387,36 @@ def test_partition_matches_oracle(ctx, oracle_mod):
     ctx.free_trace(t)
 
 
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_bounded_waits_give_up_cleanly(ctx, mapping):
+    """Failure path without a fault: with the stall hook the trace copies are never issued, so every
+    device-side wait runs into its bound.  The call must return, every valid candidate must carry
+    ETIMEOUT (and nothing else), invalid ones keep their own status, and the context must score the
+    same batch correctly right afterwards."""
+    import torch
+    import paper_2509_06362_b200 as m
+    cfg = gen.make_config("node", n_cand=3000, n_req=700)
+    lists = [[(0, 12, 4)]]
+    off2, inst2 = gen.candidates_from_lists(lists)
+    off = np.concatenate([cfg["offsets"], cfg["offsets"][-1] + off2[1:]]).astype(np.uint32)
+    inst = np.concatenate([cfg["inst"], inst2]).astype(np.uint32)
+    ctx.load_profile(cfg["profile"])
+    t = ctx.load_trace(cfg["traces"][0], cfg["classes"])
+    d_off, d_inst = ctx.to_device(off), ctx.to_device(inst)
+    res = ctx.eval_placements(t, d_off, d_inst, 8, flags=m.FLAG_TEST_STALL, mapping=mapping)
+    torch.cuda.synchronize()
+    rec = ctx.results_to_numpy(res)
+    assert (rec["status"][:-1] == m.CAND_STATUS["ETIMEOUT"]).all()
+    assert rec["status"][-1] == m.CAND_STATUS["EBADINST"]
+    for name in ("n_counted", "n_served", "n_hit", "n_rejected", "checksum", "attempts"):
+        assert (rec[name] == 0).all()
+    good = ctx.eval_placements(t, d_off, d_inst, 8, mapping=mapping)
+    torch.cuda.synchronize()
+    g = ctx.results_to_numpy(good)
+    assert (g["status"][:-1] == 0).all() and (g["n_counted"][:-1] == 700).all()
+    ctx.free_trace(t)
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")
