@@ -53,6 +53,24 @@ def _build(strategies, model_scale, min_devices, rng, pp_bubble, jitter):
     }
 
 
+def profile_decay(strategies=None, model_scale=(1.0, 1.9, 9.0), min_devices=(1, 1, 4)):
+    """Tables generated from the throughput decay function of the paper's profiler (Eq. 1):
+    F(M,P,B,W) = T0(M,P) * (1 - delta_P * ln(eps_P + min(B, W))) tokens/s per request, so one decode
+    step at level w takes 1e6 / F microseconds.  T0 = tp / (9 ms * model scale), reduced by 15 % per
+    extra pipeline stage; delta_P = 0.08 + 0.02 * log2(tp * pp) (higher-degree strategies decay faster,
+    as the paper observes); eps_P = 1.  Prefill as in the other profiles, without jitter."""
+    strategies = STRATEGIES_NODE if strategies is None else strategies
+    prof = _build(strategies, list(model_scale), list(min_devices), None, 0.15, 0.0)
+    w = np.arange(1, WMAX + 1, dtype=np.float64)
+    for m, scale in enumerate(model_scale):
+        for s, (tp, pp) in enumerate(strategies):
+            t0 = tp / (0.009 * scale) / (1.0 + 0.15 * (pp - 1))
+            delta = 0.08 + 0.02 * np.log2(tp * pp)
+            f = t0 * (1.0 - delta * np.log(1.0 + w))
+            prof["step_us"][m, s] = np.maximum(1, _rhu(1e6 / f))
+    return prof
+
+
 def profile_tiny():
     """One 7B-like model, tp in {1,2,4}; exact affine tables, no jitter."""
     return _build([(1, 1), (2, 1), (4, 1)], [1.0], [1], None, 0.0, 0.0)

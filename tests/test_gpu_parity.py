@@ -417,6 +417,23 @@ def test_bounded_waits_give_up_cleanly(ctx, mapping):
     ctx.free_trace(t)
 
 
+@pytest.mark.parametrize("trace_no", [1, 4])
+def test_table1_workload(ctx, oracle_mod, trace_no):
+    """Paper-shaped workload: 17,000 arrivals per hour with CV 2, 71 SLO classes (more than 32, so
+    class masks are ignored and classes >= 7 share the last per-class bin), Eq.-1 tables, 24 devices."""
+    cfg = gen.make_config(f"table1-{trace_no}", n_cand=800)
+    tr = cfg["traces"][0]
+    mask = np.full(800, 0b1, dtype=np.uint32)          # must be ignored: 71 classes
+    idx = np.array([3, 500], dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 24,
+                                          mask, dump_idx=idx)
+    got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 24, mask, dump_idx=idx)
+    assert (want["n_counted"] == 17000).all() and want["n_hit"].sum() > 0
+    assert_records_equal(got, want, f"table1-{trace_no}")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")

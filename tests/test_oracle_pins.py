@@ -461,3 +461,26 @@ def test_partition_scan(oracle_mod):
     # no latency-tolerant requests -> G'_l = 0 -> nothing to scan
     none = oracle_mod.partition(prof, tr, classes, 0b111, 0, gpus, configs, *args)
     assert (none["g_t"], none["g_l"], none["phi"]) == (0, 0, 0.0) and len(none["inst_t"]) == 0
+
+
+# ---- paper-shaped workload (Table I) and Eq.-1 tables ----------------------------------------
+def test_table1_generator_shapes():
+    cfg = gen.make_config("table1-4", n_cand=50, n_req=4000)
+    tr = cfg["traces"][0]
+    assert len(cfg["classes"]) == 71 and (cfg["classes"]["ttft_us"] < 0).all()
+    theta = int(cfg["profile"]["step_us"][0, 0, 0])
+    f = 0.80 + 0.01 * tr["cls"]
+    short = tr["out_tokens"] <= 500
+    assert ((tr["out_tokens"] >= 300) & (tr["out_tokens"] <= 1000)).all()
+    assert (f[short] <= 1.0 + 1e-9).all() and (f[~short] >= 1.2 - 1e-9).all()      # trace 4 pairs them
+    assert abs(short.mean() - 0.5) < 0.05
+    assert (cfg["classes"]["tbt_us"] == np.floor((0.80 + 0.01 * np.arange(71)) * theta + 0.5)).all()
+    # Eq. 1: per-request decode rate decays with the level and is truncated at the batch cap by use
+    step = cfg["profile"]["step_us"]
+    assert (np.diff(step, axis=2) >= 0).all()
+    rate = 1e6 / step[0, 0]
+    t0 = rate[0] / (1.0 - 0.08 * np.log(2.0))
+    assert np.allclose(rate, t0 * (1.0 - 0.08 * np.log(1.0 + np.arange(1, 65))), rtol=2e-4)
+    # gamma arrivals with CV 2: squared CV of the gaps near 4
+    gaps = np.diff(tr["arrival_us"].astype(np.float64))
+    assert 2.5 < gaps.var() / gaps.mean() ** 2 < 6.0
