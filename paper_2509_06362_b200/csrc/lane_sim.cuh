@@ -59,7 +59,8 @@ __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, St
     const uint4 bm = *reinterpret_cast<const uint4*>(env.keys + 64);
     uint32_t hit_blocks = 0, nd = 0x10000u, nb = 0;
 #pragma unroll
-    for (int b = 0; b < 8; b++) {  // branch-free: empty blocks count as infinitely far
+    for (int b = 0; b < 8; b++) {  // branch-free per block: empty blocks count as infinitely far
+        if (b > 0 && 8u * b >= in.B) break;  // blocks beyond the batch cap are never used
         const bool occ = ((uint32_t)(in.mask >> (8 * b)) & 0xFFu) != 0;
         const uint32_t d = occ ? ((half_of(bm, b) - K16) & 0xFFFFu) : 0x10000u;
         hit_blocks |= (d == 0 ? 1u : 0u) << b;
