@@ -249,6 +249,20 @@ MAASO_API int maaso_ins_deploy(maaso_ctx *ctx, const maaso_trace *trace, uint32_
                                uint32_t class_mask, const maaso_score_params *score, uint32_t flags,
                                double *phi_star, uint32_t *istar_len, uint32_t *istar_inst);
 
+/* getPrunedConfigs of Alg. 1: the configuration tree (Sec. III-C) after the two pruning rules of
+ * Sec. IV-D.  (1) On the tables: a strategy is dropped if another one needs no more devices, hosts
+ * every model it hosts and is at least as fast for those models at every decode level and in
+ * prefill (identical rows keep the lower index), or if no model fits on it.  (2) By simulation on the trace (class_mask as in
+ * maaso_ins_deploy): for each remaining strategy and each batch cap of `batches`, a probe placement
+ * with one instance of every model that fits is scored (all probes in one batch); a cap is kept
+ * iff no other cap of the strategy has >= SLO hits and <= mean time to first token with one of
+ * them strictly better (exact comparison; equal outcomes keep the smaller cap).
+ * Result in tree order (strategies by increasing level-1 decode step of model 0, caps ascending):
+ * out_configs (host, capacity n_strategies * n_batches), *out_n.  Synchronous. */
+MAASO_API int maaso_prune_configs(maaso_ctx *ctx, const maaso_trace *trace, int use_mask, uint32_t class_mask,
+                                  const uint32_t *batches, uint32_t n_batches, uint32_t flags,
+                                  maaso_config *out_configs, uint32_t *out_n);
+
 /* Alg. 2, "Dynamic Resource Partition", for two sub-clusters: R_t / R_l are the requests whose
  * class bit is set in mask_t / mask_l.  G'_l = floor(|R_l| * gpus / (|R_t| + |R_l|));
  * maaso_ins_deploy on (R_l, G'_l) and on (R_t, gpus); Phi_opt starts at the best score of

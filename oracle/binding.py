@@ -54,6 +54,7 @@ def _load():
         _lib.orc_rejected_by_model.restype = C.c_int
         _lib.orc_ins_deploy.restype = C.c_int
         _lib.orc_partition.restype = C.c_int
+        _lib.orc_prune_configs.restype = C.c_int
     return _lib
 
 
@@ -233,6 +234,25 @@ def partition(profile, trace, classes, mask_t, mask_l, gpus, configs, alpha, bet
     del keep
     return {"g_t": int(g[0]), "g_l": int(g[1]), "phi": phi.value, "inst_t": it[:lt.value].copy(),
             "inst_l": il[:ll.value].copy()}
+
+
+def prune_configs(profile, trace, classes, batches, class_mask=None, flags=0):
+    """getPrunedConfigs (see orc_prune_configs): list of (strategy, batch) in tree order."""
+    lib = _load()
+    p, keep = _profile_struct(profile)
+    trace = np.ascontiguousarray(trace, dtype=_REQ)
+    classes = np.ascontiguousarray(classes, dtype=_SLO)
+    b = np.ascontiguousarray(batches, dtype=np.uint32)
+    out = np.zeros((int(profile["n_strategies"]) * len(b), 2), dtype=np.uint32)
+    n_out = C.c_uint32(0)
+    rc = lib.orc_prune_configs(C.byref(p), _ptr(trace), C.c_uint64(len(trace)), _ptr(classes),
+                               C.c_uint32(len(classes)), C.c_int(0 if class_mask is None else 1),
+                               C.c_uint32(class_mask or 0), _ptr(b), C.c_uint32(len(b)), C.c_uint32(flags),
+                               _ptr(out), C.byref(n_out))
+    if rc != 0:
+        raise RuntimeError(f"oracle prune_configs failed with code {rc}")
+    del keep
+    return [tuple(int(x) for x in row) for row in out[:n_out.value]]
 
 
 def topk_scores(scores, k):

@@ -395,6 +395,8 @@ int orc_score(const orc_result *res, uint64_t n, const orc_score_params *p, doub
     return 0;
 }
 
+typedef struct { uint32_t strategy, batch; } orc_config;
+
 /* Requests of each model left unserved (rejected) by every candidate: counted from the
  * per-request outcome, out[c][16]. */
 int orc_rejected_by_model(const orc_profile *p, const orc_request *reqs, uint64_t n, const orc_slo *classes,
@@ -430,8 +432,6 @@ int orc_rejected_by_model(const orc_profile *p, const orc_request *reqs, uint64_
  * R_x = requests whose class bit is set in class_mask (all if has_mask == 0).
  * Outputs: phi_star[gpus + 1], istar_len[gpus + 1], istar_inst[gpus + 1][128] (packed words).
  */
-typedef struct { uint32_t strategy, batch; } orc_config;
-
 int orc_ins_deploy(const orc_profile *p, const orc_request *reqs, uint64_t n, const orc_slo *classes,
                    uint32_t n_classes, int has_mask, uint32_t class_mask, uint32_t gpus,
                    const orc_config *configs, uint32_t n_configs, const orc_score_params *sp, uint32_t flags,
@@ -481,6 +481,108 @@ int orc_ins_deploy(const orc_profile *p, const orc_request *reqs, uint64_t n, co
     }
     free(where);
     return 0;
+}
+
+/*
+ * getPrunedConfigs of Alg. 1: the configuration tree of Sec. III-C with the two pruning rules
+ * of Sec. IV-D.
+ *  (1) Parallelism-strategy pruning, on the tables: strategy P is dropped if some other strategy Q
+ *      needs no more devices, hosts every model that P hosts, and is at least as fast for those
+ *      models (every decode level, prefill base and slope), i.e. P "fails to outperform" Q "while
+ *      consuming" at least as many resources; identical rows on equal devices keep the lower
+ *      index.  A strategy on which no model fits is dropped as well.
+ *  (2) Batch-size pruning, by simulation on R_x: for each remaining strategy and each batch cap of
+ *      the caller's list, a probe placement with one instance (m, P, B) of every model that fits is
+ *      replayed; a batch cap is kept iff no other cap of the same strategy has at least as many SLO
+ *      hits and at most the same mean response latency (time to first token, exact rational
+ *      compare; nothing served = infinite latency) with one of the two strictly better: the
+ *      Pareto front between latency and SLO satisfaction.  Equal outcomes keep the smaller cap.
+ * Order of the result (in-order traversal of the tree = decreasing decode throughput): strategies
+ * by increasing level-1 decode step of model 0 (ties: lower index), batch caps ascending.
+ * out: (strategy, batch) pairs, *out_n of them; capacity n_strategies * n_batches.
+ */
+/* Q can stand in for S: every model that fits on S also fits on Q, and for those models Q is at
+ * least as fast at every decode level and in prefill. */
+static int orc_faster_or_equal(const orc_profile *p, uint32_t q, uint32_t s, int *strict) {
+    for (uint32_t m = 0; m < p->n_models; m++) {
+        if (p->devices[s] < p->min_devices[m]) continue;   /* S cannot host this model anyway */
+        if (p->devices[q] < p->min_devices[m]) return 0;   /* Q cannot replace S for it */
+        size_t rq = (size_t)m * p->n_strategies + q, rs = (size_t)m * p->n_strategies + s;
+        if (p->prefill_base_us[rq] > p->prefill_base_us[rs]) return 0;
+        if ((uint32_t)p->prefill_q16[rq] > (uint32_t)p->prefill_q16[rs]) return 0;
+        if (p->prefill_base_us[rq] < p->prefill_base_us[rs] ||
+            (uint32_t)p->prefill_q16[rq] < (uint32_t)p->prefill_q16[rs]) *strict = 1;
+        for (uint32_t w = 0; w < p->wmax; w++) {
+            if (p->step_us[rq * p->wmax + w] > p->step_us[rs * p->wmax + w]) return 0;
+            if (p->step_us[rq * p->wmax + w] < p->step_us[rs * p->wmax + w]) *strict = 1;
+        }
+    }
+    return 1;
+}
+
+int orc_prune_configs(const orc_profile *p, const orc_request *reqs, uint64_t n, const orc_slo *classes,
+                      uint32_t n_classes, int has_mask, uint32_t class_mask, const uint32_t *batches,
+                      uint32_t n_batches, uint32_t flags, orc_config *out, uint32_t *out_n) {
+    uint32_t S = p->n_strategies;
+    int *keep = (int *)calloc(S, sizeof(int));
+    uint32_t *order = (uint32_t *)malloc(S * sizeof(uint32_t));
+    orc_result *res = (orc_result *)malloc((size_t)(n_batches ? n_batches : 1) * sizeof(orc_result));
+    if (!keep || !order || !res) { free(keep); free(order); free(res); return -1; }
+    /* (1) strategy pruning */
+    for (uint32_t s = 0; s < S; s++) {
+        int fits = 0;
+        for (uint32_t m = 0; m < p->n_models; m++) if (p->devices[s] >= p->min_devices[m]) fits = 1;
+        keep[s] = fits;
+        for (uint32_t q = 0; q < S && keep[s]; q++) {
+            if (q == s || p->devices[q] > p->devices[s]) continue;
+            int strict = 0;
+            if (!orc_faster_or_equal(p, q, s, &strict)) continue;
+            if (strict || p->devices[q] < p->devices[s] || q < s) keep[s] = 0;
+        }
+    }
+    /* tree order: decreasing decode throughput = increasing level-1 step of model 0 */
+    uint32_t ns = 0;
+    for (uint32_t s = 0; s < S; s++) if (keep[s]) order[ns++] = s;
+    for (uint32_t i = 1; i < ns; i++)
+        for (uint32_t j = i; j > 0; j--) {
+            uint32_t a = order[j - 1], b = order[j];
+            int32_t sa = p->step_us[(size_t)a * p->wmax], sb = p->step_us[(size_t)b * p->wmax];
+            if (sa > sb || (sa == sb && a > b)) { order[j - 1] = b; order[j] = a; } else break;
+        }
+    /* (2) batch pruning per strategy */
+    *out_n = 0;
+    int rc = 0;
+    for (uint32_t i = 0; i < ns && !rc; i++) {
+        uint32_t s = order[i];
+        for (uint32_t b = 0; b < n_batches && !rc; b++) {
+            uint32_t inst[16], ni = 0;
+            for (uint32_t m = 0; m < p->n_models; m++)
+                if (p->devices[s] >= p->min_devices[m]) inst[ni++] = (m & 0xF) | ((s & 0xFF) << 4) | ((batches[b] & 0xFF) << 12);
+            rc = orc_eval_candidate(p, reqs, n, classes, n_classes, inst, ni, has_mask, class_mask, 0xFFFFFFFFu,
+                                    flags, &res[b], NULL, NULL, NULL);
+        }
+        for (uint32_t b = 0; b < n_batches && !rc; b++) {
+            int dominated = res[b].status != 0;
+            for (uint32_t c = 0; c < n_batches && !dominated; c++) {
+                if (c == b || res[c].status != 0) continue;
+                /* latency compare: sum_b / served_b vs sum_c / served_c, nothing served = infinite */
+                int lat_c_le, lat_c_lt;
+                if (res[c].n_served == 0) { lat_c_le = res[b].n_served == 0; lat_c_lt = 0; }
+                else if (res[b].n_served == 0) { lat_c_le = 1; lat_c_lt = 1; }
+                else {
+                    unsigned __int128 l = (unsigned __int128)(uint64_t)res[c].sum_ttft_us * res[b].n_served;
+                    unsigned __int128 r = (unsigned __int128)(uint64_t)res[b].sum_ttft_us * res[c].n_served;
+                    lat_c_le = l <= r; lat_c_lt = l < r;
+                }
+                int hit_c_ge = res[c].n_hit >= res[b].n_hit, hit_c_gt = res[c].n_hit > res[b].n_hit;
+                if (hit_c_ge && lat_c_le && (hit_c_gt || lat_c_lt)) dominated = 1;
+                else if (hit_c_ge && lat_c_le && !hit_c_gt && !lat_c_lt && batches[c] < batches[b]) dominated = 1;
+            }
+            if (!dominated) { out[*out_n].strategy = s; out[*out_n].batch = batches[b]; (*out_n)++; }
+        }
+    }
+    free(keep); free(order); free(res);
+    return rc;
 }
 
 /*

@@ -85,6 +85,8 @@ def _load():
     lib.maaso_topk_scores.argtypes = [vp, vp, vp, u64, u32, vp, vp, vp]
     lib.maaso_ins_deploy.argtypes = [vp, vp, u32, vp, u32, C.c_int, u32, C.POINTER(_ScoreParams), u32, vp, vp, vp]
     lib.maaso_ins_deploy.restype = C.c_int
+    lib.maaso_prune_configs.argtypes = [vp, vp, C.c_int, u32, vp, u32, u32, vp, C.POINTER(u32)]
+    lib.maaso_prune_configs.restype = C.c_int
     lib.maaso_partition.argtypes = [vp, vp, u32, u32, u32, vp, u32, C.POINTER(_ScoreParams), u32, C.c_int, vp,
                                     C.POINTER(C.c_double), C.POINTER(u32), vp, C.POINTER(u32), vp]
     lib.maaso_partition.restype = C.c_int
@@ -243,6 +245,17 @@ def maaso_ins_deploy(ctx, trace, gpus, configs, alpha, beta, gamma_t, gamma_l, c
     return phi, [iinst[k, :ilen[k]].copy() for k in range(gpus + 1)]
 
 
+def maaso_prune_configs(ctx, trace, n_strategies, batches, class_mask=None, flags=0):
+    """getPrunedConfigs: list of (strategy, batch) in configuration-tree order."""
+    b = np.ascontiguousarray(batches, dtype=np.uint32)
+    out = np.zeros((int(n_strategies) * len(b), 2), dtype=np.uint32)
+    n_out = C.c_uint32(0)
+    _check(_lib.maaso_prune_configs(ctx, trace, 0 if class_mask is None else 1, int(class_mask or 0),
+                                    b.ctypes.data, len(b), int(flags), out.ctypes.data, C.byref(n_out)),
+           "maaso_prune_configs", ctx)
+    return [tuple(int(x) for x in row) for row in out[:n_out.value]]
+
+
 def maaso_partition(ctx, trace, mask_t, mask_l, gpus, configs, alpha, beta, gamma_t, gamma_l, flags=0,
                     baseline=False):
     """Alg. 2 for two sub-clusters.  Returns dict(g_t, g_l, phi, inst_t, inst_l)."""
@@ -328,6 +341,9 @@ class Context:
         """uint32 numpy words -> int32 CUDA tensor with the same bits"""
         t = self.torch.from_numpy(np.ascontiguousarray(words, dtype=np.uint32).view(np.int32))
         return t.to(self.device)
+
+    def prune_configs(self, trace, n_strategies, batches, class_mask=None, flags=0):
+        return maaso_prune_configs(self.handle, trace.handle, n_strategies, batches, class_mask, flags)
 
     def partition(self, trace, mask_t, mask_l, gpus, configs, alpha, beta, gamma_t, gamma_l, flags=0,
                   baseline=False):

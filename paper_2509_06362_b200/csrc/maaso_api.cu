@@ -45,7 +45,9 @@ struct maaso_ctx {
     int32_t* d_rows;
     int32_t* d_devices;
     int32_t* d_min_devices;
-    std::vector<int32_t> h_devices;  // host copy for the Alg. 1 driver
+    std::vector<int32_t> h_devices;  // host copies for the Alg. 1 driver and the pruning rules
+    std::vector<int32_t> h_min_devices;
+    std::vector<int32_t> h_rows;
     std::vector<maaso_trace*> traces;
     void* scratch;
     size_t scratch_bytes;
@@ -237,6 +239,8 @@ MAASO_API int maaso_load_profile(maaso_ctx* ctx, const maaso_profile_desc* d) {
         (e = cudaMemcpy(ctx->d_min_devices, d->min_devices, M * 4, cudaMemcpyHostToDevice)) != cudaSuccess)
         return cuda_fail(ctx, e, "profile copy");
     ctx->h_devices.assign(d->devices, d->devices + S);
+    ctx->h_min_devices.assign(d->min_devices, d->min_devices + M);
+    ctx->h_rows = rows;
     ctx->n_models = M;
     ctx->n_strategies = S;
     ctx->n_rows = R;
@@ -677,6 +681,124 @@ MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_
                 for (uint32_t i = 0; i < sp.len && i < MAASO_MAX_INSTANCES; i++)
                     istar_inst[(size_t)sp.k * MAASO_MAX_INSTANCES + i] = chains[c].inst[i];
             }
+    return MAASO_OK;
+}
+
+// getPrunedConfigs: strategy dominance on the host copy of the tables, batch-cap Pareto front from
+// one batch of probe placements.
+MAASO_API int maaso_prune_configs(maaso_ctx* ctx, const maaso_trace* trace, int use_mask, uint32_t class_mask,
+                                  const uint32_t* batches, uint32_t n_batches, uint32_t flags,
+                                  maaso_config* out_configs, uint32_t* out_n) {
+    if (!ctx || !trace || !out_configs || !out_n || (n_batches && !batches) || n_batches > MAASO_WMAX)
+        return MAASO_EINVAL;
+    *out_n = 0;
+    if (!ctx->has_profile) return fail(ctx, MAASO_ESTATE, "prune: no profile loaded");
+    for (uint32_t b = 0; b < n_batches; b++)
+        if (batches[b] < 1 || batches[b] > MAASO_WMAX) return fail(ctx, MAASO_EINVAL, "prune: batch cap out of range");
+    const uint32_t S = ctx->n_strategies, M = ctx->n_models;
+    const int32_t* rows = ctx->h_rows.data();
+    auto faster_or_equal = [&](uint32_t q, uint32_t s, bool& strict) {
+        for (uint32_t m = 0; m < M; m++) {
+            if (ctx->h_devices[s] < ctx->h_min_devices[m]) continue;    // s cannot host this model anyway
+            if (ctx->h_devices[q] < ctx->h_min_devices[m]) return false;  // q cannot replace s for it
+            const int32_t* rq = rows + (size_t)(m * S + q) * kRowStride;
+            const int32_t* rs = rows + (size_t)(m * S + s) * kRowStride;
+            if (rq[0] > rs[0] || (uint32_t)rq[1] > (uint32_t)rs[1]) return false;
+            if (rq[0] < rs[0] || (uint32_t)rq[1] < (uint32_t)rs[1]) strict = true;
+            for (int w = 0; w < MAASO_WMAX; w++) {
+                if (rq[2 + w] > rs[2 + w]) return false;
+                if (rq[2 + w] < rs[2 + w]) strict = true;
+            }
+        }
+        return true;
+    };
+    std::vector<uint32_t> order;
+    for (uint32_t s = 0; s < S; s++) {
+        bool keep = false;
+        for (uint32_t m = 0; m < M; m++) keep = keep || ctx->h_devices[s] >= ctx->h_min_devices[m];
+        for (uint32_t q = 0; q < S && keep; q++) {
+            if (q == s || ctx->h_devices[q] > ctx->h_devices[s]) continue;
+            bool strict = false;
+            if (!faster_or_equal(q, s, strict)) continue;
+            if (strict || ctx->h_devices[q] < ctx->h_devices[s] || q < s) keep = false;
+        }
+        if (keep) order.push_back(s);
+    }
+    for (size_t i = 1; i < order.size(); i++)  // tree order: increasing level-1 step of model 0
+        for (size_t j = i; j > 0; j--) {
+            const uint32_t a = order[j - 1], b = order[j];
+            const int32_t sa = rows[(size_t)a * kRowStride + 2], sb = rows[(size_t)b * kRowStride + 2];
+            if (sa > sb || (sa == sb && a > b)) { order[j - 1] = b; order[j] = a; } else break;
+        }
+    if (order.empty() || n_batches == 0) return MAASO_OK;
+
+    // one batch of probe placements: (strategy, cap) -> one instance of every model that fits
+    const size_t C = order.size() * n_batches;
+    std::vector<uint32_t> h_off(C + 1), h_inst, h_mask(C, class_mask);
+    for (size_t i = 0; i < order.size(); i++)
+        for (uint32_t b = 0; b < n_batches; b++) {
+            h_off[i * n_batches + b] = (uint32_t)h_inst.size();
+            for (uint32_t m = 0; m < M; m++)
+                if (ctx->h_devices[order[i]] >= ctx->h_min_devices[m])
+                    h_inst.push_back((m & 0xFu) | ((order[i] & 0xFFu) << 4) | ((batches[b] & 0xFFu) << 12));
+        }
+    h_off[C] = (uint32_t)h_inst.size();
+    DeviceGuard g(ctx->device);
+    size_t off = 0;
+    const size_t o_off = off;  off = align_up(off + (C + 1) * 4, 256);
+    const size_t o_inst = off; off = align_up(off + h_inst.size() * 4 + 4, 256);
+    const size_t o_mask = off; off = align_up(off + C * 4, 256);
+    const size_t o_res = off;  off = align_up(off + C * sizeof(maaso_result), 256);
+    int rc = grow(ctx, &ctx->deploy, &ctx->deploy_bytes, off);
+    if (rc != MAASO_OK) return rc;
+    unsigned char* sb = static_cast<unsigned char*>(ctx->deploy);
+    cudaStream_t st = ctx->own_stream;
+    cudaError_t e = cudaMemcpyAsync(sb + o_off, h_off.data(), (C + 1) * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sb + o_inst, h_inst.data(), h_inst.size() * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && use_mask) e = cudaMemcpyAsync(sb + o_mask, h_mask.data(), C * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "prune: upload");
+    maaso_cand_batch bt;
+    memset(&bt, 0, sizeof(bt));
+    bt.offsets = reinterpret_cast<const uint32_t*>(sb + o_off);
+    bt.inst = reinterpret_cast<const uint32_t*>(sb + o_inst);
+    bt.class_mask = use_mask ? reinterpret_cast<const uint32_t*>(sb + o_mask) : nullptr;
+    bt.n_cand = C;
+    bt.n_inst = h_inst.size();
+    bt.budget = 0xFFFFFFFFu;  // a probe, not a deployment
+    maaso_eval_opts o;
+    memset(&o, 0, sizeof(o));
+    o.flags = flags;
+    rc = maaso_eval_placements(ctx, trace, &bt, &o, reinterpret_cast<maaso_result*>(sb + o_res), st);
+    if (rc != MAASO_OK) return rc;
+    std::vector<maaso_result> res(C);
+    e = cudaMemcpyAsync(res.data(), sb + o_res, C * sizeof(maaso_result), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "prune: download");
+    for (size_t i = 0; i < order.size(); i++) {
+        const maaso_result* r = res.data() + i * n_batches;
+        for (uint32_t b = 0; b < n_batches; b++) {
+            bool dominated = r[b].status != 0;
+            for (uint32_t c = 0; c < n_batches && !dominated; c++) {
+                if (c == b || r[c].status != 0) continue;
+                bool lat_le, lat_lt;  // mean time to first token of c vs b; nothing served = infinite
+                if (r[c].n_served == 0) { lat_le = r[b].n_served == 0; lat_lt = false; }
+                else if (r[b].n_served == 0) { lat_le = true; lat_lt = true; }
+                else {
+                    const unsigned __int128 l = (unsigned __int128)(uint64_t)r[c].sum_ttft_us * r[b].n_served;
+                    const unsigned __int128 rr = (unsigned __int128)(uint64_t)r[b].sum_ttft_us * r[c].n_served;
+                    lat_le = l <= rr; lat_lt = l < rr;
+                }
+                const bool hit_ge = r[c].n_hit >= r[b].n_hit, hit_gt = r[c].n_hit > r[b].n_hit;
+                if (hit_ge && lat_le && (hit_gt || lat_lt)) dominated = true;
+                else if (hit_ge && lat_le && batches[c] < batches[b]) dominated = true;  // equal outcome
+            }
+            if (!dominated) {
+                out_configs[*out_n].strategy = order[i];
+                out_configs[*out_n].batch = batches[b];
+                (*out_n)++;
+            }
+        }
+    }
     return MAASO_OK;
 }
 

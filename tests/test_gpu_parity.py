@@ -434,6 +434,21 @@ def test_table1_workload(ctx, oracle_mod, trace_no):
         assert (gd[k] == wd[k]).all(), k
 
 
+def test_prune_configs_matches_oracle(ctx, oracle_mod):
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 180_000_000)])
+    batches = [1, 2, 4, 8, 16, 32, 64]
+    for prof, mix in ((gen.profile_multimodel(0), (0.6, 0.3, 0.1)), (gen.profile_decay(), (1, 1, 1)),
+                      (gen.profile_node(3), (1.0,))):
+        ctx.load_profile(prof)
+        for rate, mask in ((8.0, None), (40.0, 0b011), (150.0, 0b100)):
+            tr = gen.make_trace(2500, rate, 7, cv=2.0, model_mix=mix)
+            t = ctx.load_trace(tr, classes)
+            got = ctx.prune_configs(t, prof["n_strategies"], batches, class_mask=mask)
+            want = oracle_mod.prune_configs(prof, tr, classes, batches, class_mask=mask)
+            assert got == want and len(got) > 0
+            ctx.free_trace(t)
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")

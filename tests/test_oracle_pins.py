@@ -484,3 +484,75 @@ def test_table1_generator_shapes():
     # gamma arrivals with CV 2: squared CV of the gaps near 4
     gaps = np.diff(tr["arrival_us"].astype(np.float64))
     assert 2.5 < gaps.var() / gaps.mean() ** 2 < 6.0
+
+
+# ---- configuration tree and pruning (Sec. III-C, IV-D) ---------------------------------------
+def test_prune_configs_strategy_rule_and_order(oracle_mod):
+    """Hand-made tables: strategy 1 is slower than 0 on more devices (dropped), 2 is faster on more
+    devices (kept), 3 copies 2 (the copy is dropped), 4 is faster than 0 at low levels but slower at
+    high ones (kept: no dominance), 5 fits no model (dropped)."""
+    W = gen.WMAX
+    w = np.arange(1, W + 1)
+    step = np.stack([9000 + 100 * w, 9500 + 100 * w, 5000 + 100 * w, 5000 + 100 * w,
+                     6000 + 400 * w, 3000 + 50 * w])[None].astype(np.int32)
+    prof = {"n_models": 1, "n_strategies": 6, "wmax": W,
+            "devices": np.array([1, 2, 2, 2, 1, 1], dtype=np.int32), "min_devices": np.array([1], dtype=np.int32),
+            "prefill_base_us": np.array([[2000, 2000, 1000, 1000, 2000, 500]], dtype=np.int32),
+            "prefill_q16": np.array([[7000, 7000, 3500, 3500, 7000, 100]], dtype=np.int32), "step_us": step}
+    prof["min_devices"] = np.array([1], dtype=np.int32)
+    tr = gen.make_trace(300, 10.0, 1, doc_class=None)
+    classes = gen.make_classes(NONE3 * 3)
+    got = oracle_mod.prune_configs(prof, tr, classes, [4])
+    # strategy 5 needs one device and is faster than every other row everywhere: it alone survives
+    assert [s for s, _ in got] == [5]
+    prof["min_devices"] = np.array([2], dtype=np.int32)      # now nothing fits on one device
+    got = oracle_mod.prune_configs(prof, tr, classes, [4])
+    assert [s for s, _ in got] == [2]                         # a strategy that hosts nothing dominates nothing
+    prof["min_devices"] = np.array([1], dtype=np.int32)
+    prof["step_us"] = step.copy()
+    prof["step_us"][0, 5] = 20000                             # strategy 5 no longer dominates anybody
+    got = oracle_mod.prune_configs(prof, tr, classes, [4])
+    # order: increasing level-1 step: 2 (5100), 4 (6400), 0 (9100), 5 (20000); 1 and 3 dropped
+    assert [s for s, _ in got] == [2, 4, 0, 5]
+
+
+def test_prune_configs_batch_pareto(oracle_mod):
+    from fractions import Fraction
+    prof = gen.profile_multimodel(0)
+    tr = gen.make_trace(1500, 25.0, 3, model_mix=(0.6, 0.3, 0.1))
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 180_000_000)])
+    batches = [1, 2, 4, 8, 16, 32, 64]
+    for mask in (None, 0b011):
+        got = oracle_mod.prune_configs(prof, tr, classes, batches, class_mask=mask)
+        strategies = []
+        for s, _ in got:
+            if s not in strategies:
+                strategies.append(s)
+        assert all(gen.STRATEGIES_NODE[s][1] == 1 for s in strategies)      # pipeline strategies lose to tp / dp
+        lvl1 = [int(prof["step_us"][0, s, 0]) for s in strategies]
+        assert lvl1 == sorted(lvl1)
+        want = []
+        for s in strategies:                                                 # brute-force Pareto front
+            outcome = []
+            for b in batches:
+                lst = [(m, s, b) for m in range(3) if prof["devices"][s] >= prof["min_devices"][m]]
+                off, inst = gen.candidates_from_lists([lst])
+                cm = None if mask is None else np.array([mask], dtype=np.uint32)
+                r = oracle_mod.eval_placements(prof, tr, classes, off, inst, 10 ** 9, cm)[0]
+                lat = Fraction(int(r["sum_ttft_us"]), int(r["n_served"])) if r["n_served"] else None
+                outcome.append((int(r["n_hit"]), lat))
+            def le(x, y):
+                return y is None or (x is not None and x <= y)
+            for i, b in enumerate(batches):
+                dom = False
+                for j in range(len(batches)):
+                    if i == j:
+                        continue
+                    hit_ge, hit_gt = outcome[j][0] >= outcome[i][0], outcome[j][0] > outcome[i][0]
+                    lat_le = le(outcome[j][1], outcome[i][1])
+                    lat_lt = lat_le and outcome[j][1] != outcome[i][1]
+                    if hit_ge and lat_le and (hit_gt or lat_lt or batches[j] < b):
+                        dom = True
+                if not dom:
+                    want.append((s, b))
+        assert got == want
