@@ -449,6 +449,27 @@ def test_prune_configs_matches_oracle(ctx, oracle_mod):
             ctx.free_trace(t)
 
 
+def test_placer_end_to_end(ctx, oracle_mod):
+    """The placer as the paper runs it: getPrunedConfigs, then Alg. 2 over Alg. 1, on a Table-I
+    shaped hour of traffic; library and oracle must name the same partition and placements."""
+    cfg = gen.make_config("table1-4", n_cand=1, n_req=6000)
+    prof, tr, classes = cfg["profile"], cfg["traces"][0], cfg["classes"][:32].copy()
+    tr = tr.copy()
+    tr["cls"] = np.minimum(tr["cls"] // 3, 31)           # 24 classes so that the class masks apply
+    strict = sum(1 << k for k in range(0, 8))             # SLO factors up to about 1.0
+    relaxed = sum(1 << k for k in range(8, 32))
+    ctx.load_profile(prof)
+    t = ctx.load_trace(tr, classes)
+    batches = [1, 4, 16, 64]
+    configs = ctx.prune_configs(t, prof["n_strategies"], batches)
+    assert configs == oracle_mod.prune_configs(prof, tr, classes, batches) and len(configs) >= 2
+    got = ctx.partition(t, strict, relaxed, 24, configs, 4.0, 0.3, 20000.0, 10.0, baseline=True)
+    want = oracle_mod.partition(prof, tr, classes, strict, relaxed, 24, configs, 4.0, 0.3, 20000.0, 10.0, baseline=True)
+    assert (got["g_t"], got["g_l"], got["phi"]) == (want["g_t"], want["g_l"], want["phi"])
+    assert got["inst_t"].tolist() == want["inst_t"].tolist() and got["inst_l"].tolist() == want["inst_l"].tolist()
+    ctx.free_trace(t)
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")

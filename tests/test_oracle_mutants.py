@@ -1,0 +1,102 @@
+"""Are the oracle's pins sharp?  Each case plants one plausible mistake in a COPY of the oracle's
+source (a dropped term, an off-by-one, a swapped comparison, a wrong table index), builds it on the
+CPU, and requires that at least one pin fails for the mutant.  The unmodified copy must pass all of
+them.  Nothing here touches the CUDA path."""
+import importlib.util
+import os
+import shutil
+
+import numpy as np
+import pytest
+
+import gen
+import test_oracle_pins as pins
+from golden_cases import all_cases
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+MUTANTS = [
+    ("prefill rounding term dropped", "* in_tokens + 32768u) >> 16", "* in_tokens + 0u) >> 16"),
+    ("predicted finish counts one token too many", "fin = first + (S - 1) * sB;", "fin = first + S * sB;"),
+    ("worst-case step taken at the current level", "int64_t sB = in->step[in->B - 1];",
+     "int64_t sB = in->step[in->w > 0 ? in->w - 1 : 0];"),
+    ("next free time one step early", "t0 = in->T + (min_fin(in) - in->K) *", "t0 = in->T + (min_fin(in) - in->K - 1) *"),
+    ("clock jump overshoots when the gap is a whole number of steps", "int64_t need = (t - in->T + s - 1) / s;",
+     "int64_t need = (t - in->T + s) / s;"),
+    ("ties go to the higher index", "(tier == best_tier && first < best_first)", "(tier == best_tier && first <= best_first)"),
+    ("free slot not preferred", "!have || tier < best_tier || (tier == best_tier && first < best_first)",
+     "!have || first < best_first"),
+    ("TBT budget counts one gap too many", "span <= (int64_t)(S - 1) * k->tbt_us", "span <= (int64_t)S * k->tbt_us"),
+    ("idle instance does not start at once", "if (!drain && in->w == 0 && in->T < t) in->T = t;", ""),
+    ("completion index one step late", "sl->fin_idx = in->K + S - 1;", "sl->fin_idx = in->K + S;"),
+    ("decode step taken one level too low", "int64_t s = in->step[in->w - 1];", "int64_t s = in->step[in->w > 1 ? in->w - 2 : 0];"),
+    ("wait overshoots by a microsecond", "now = best_t0;  ", "now = best_t0 + 1;"),
+    ("class mask inverted", "if (has_mask && !((class_mask >> q->cls) & 1u)) continue;",
+     "if (has_mask && ((class_mask >> q->cls) & 1u)) continue;"),
+    ("ranking prefers higher mean latency", "if (l != r) return l < r;", "if (l != r) return l > r;"),
+    ("ranking prefers fewer hits", "return x->n_hit > y->n_hit;", "return x->n_hit < y->n_hit;"),
+    ("latency weight is beta instead of 1 - beta", "double c = (1.0 - p->beta) * phil;", "double c = p->beta * phil;"),
+    ("prefill does not stall the running batch", "in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {",
+     "int64_t t_keep = in->T; in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {"),
+]
+
+
+def load_variant(tmp_path, tag, old=None, new=None):
+    d = tmp_path / tag
+    d.mkdir()
+    for name in ("binding.py", "maaso_oracle.c"):
+        shutil.copy(os.path.join(ROOT, "oracle", name), d / name)
+    if old is not None:
+        src = (d / "maaso_oracle.c").read_text()
+        assert src.count(old) == 1, f"mutation target not unique or missing: {old!r}"
+        (d / "maaso_oracle.c").write_text(src.replace(old, new))
+    spec = importlib.util.spec_from_file_location(f"oracle_variant_{tag}", d / "binding.py")
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.build(force=True)
+    return mod
+
+
+def run_pins(mod):
+    """Run a compact selection of the pins against `mod`; returns the names of those that fail."""
+    failed = []
+
+    def attempt(name, fn, *args):
+        try:
+            fn(mod, *args)
+        except AssertionError:
+            failed.append(name)
+
+    for case in all_cases():
+        attempt("hand:" + case["name"], pins.test_hand_timelines, case)
+    attempt("lindley", pins.test_single_server_closed_form)
+    attempt("no contention", pins.test_no_contention_closed_form)
+    for seed in (0, 3, 4, 7):
+        attempt(f"token by token {seed}", pins.test_against_token_by_token, seed)
+    attempt("invariants", pins.test_invariants_on_tiny_config)
+    attempt("no cascade", pins.test_no_cascade_without_prefill, 0)
+    attempt("mask algebra", pins.test_mask_algebra)
+    attempt("ranking", pins.test_topk_brute_force)
+    attempt("score", pins.test_score_worked_values)
+    return failed
+
+
+def test_unmodified_copy_passes_every_pin(tmp_path):
+    assert run_pins(load_variant(tmp_path, "clean")) == []
+
+
+@pytest.mark.parametrize("what,old,new", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_planted_mistake_is_caught(tmp_path, what, old, new):
+    if what == "prefill does not stall the running batch":
+        # second half of the mutation: the first token is still stamped, but the clock is put back
+        mod = load_variant(tmp_path, "m", old, new)
+        src = (tmp_path / "m" / "maaso_oracle.c").read_text()
+        tgt = "sl->cls = q->cls;\n                    in->w++;"
+        assert src.count(tgt) == 1
+        (tmp_path / "m" / "maaso_oracle.c").write_text(src.replace(tgt, tgt + "\n                    if (in->w > 1) in->T = t_keep;"))
+        mod.build(force=True)
+        mod._lib = None
+    else:
+        mod = load_variant(tmp_path, "m", old, new)
+    failed = run_pins(mod)
+    assert failed, f"no pin noticed: {what}"
