@@ -177,7 +177,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     }
     return true;
 }
-// Plain (no multicast) bulk copy global -> this CTA's shared memory; 16-byte aligned, size % 16 == 0.
+// Plain bulk copy global -> this CTA's own shared memory (one destination CTA); 16-byte aligned, size % 16 == 0.
 __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes,
                                           uint64_t* bar) {
     asm volatile(

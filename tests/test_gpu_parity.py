@@ -470,6 +470,62 @@ def test_placer_end_to_end(ctx, oracle_mod):
     ctx.free_trace(t)
 
 
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_extreme_values(ctx, oracle_mod, mapping):
+    """Corners of the integer ranges: 65535-token outputs (16-bit completion keys at their limit and
+    wrapping many times), decode steps of 2^30 us, 4-billion-token inputs, arrivals near 2^50 us with
+    gaps far above 2^32 us (the wide division path), single-token requests, full 64-slot instances."""
+    W = gen.WMAX
+    rng = np.random.default_rng(17)
+    step = np.zeros((2, 3, W), dtype=np.int32)
+    step[:, 0] = 1 + np.arange(W)                      # microsecond steps
+    step[:, 1] = (1 << 30) - np.arange(W)              # the largest allowed steps, decreasing with the level
+    step[:, 2] = rng.integers(1, 1 << 20, size=(2, W))
+    prof = {"n_models": 2, "n_strategies": 3, "wmax": W,
+            "devices": np.array([1, 1, 2], dtype=np.int32), "min_devices": np.array([1, 1], dtype=np.int32),
+            "prefill_base_us": np.array([[0, 1 << 30, 7], [3, 0, 1 << 20]], dtype=np.int32),
+            "prefill_q16": np.array([[0, (1 << 31) - 1, 65536], [1, 0, 123456]], dtype=np.int32), "step_us": step}
+    n = 1200
+    tr = np.zeros(n, dtype=gen.REQUEST_DTYPE)
+    gaps = rng.choice([0, 1, 1000, 10 ** 7, 5 * 10 ** 9, 3 * 10 ** 11], size=n, p=[0.2, 0.2, 0.3, 0.2, 0.07, 0.03])
+    tr["arrival_us"] = np.minimum(np.cumsum(gaps), (1 << 50) - 1)
+    tr["in_tokens"] = rng.choice([0, 1, 4096, 2 ** 32 - 1], size=n)
+    tr["out_tokens"] = rng.choice([1, 2, 300, 40000, 65535], size=n)
+    tr["cls"] = rng.integers(0, 3, size=n)
+    tr["model"] = rng.integers(0, 2, size=n)
+    classes = gen.make_classes([(None, None, None), (1 << 40, 1 << 40, 1 << 40), (10 ** 9, 10 ** 6, None)])
+    lists = [[(0, 0, 64), (1, 0, 64)], [(0, 1, 1), (1, 1, 2)], [(0, 2, 64), (1, 2, 3), (0, 0, 1), (1, 1, 64)],
+             [(m, s, b) for m in (0, 1) for s in (0, 1, 2) for b in (1, 7, 64)],
+             [(0, 0, 1)], [(1, 2, 64)] * 40]
+    off, inst = gen.candidates_from_lists(lists)
+    idx = np.arange(len(lists), dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(prof, tr, classes, off, inst, 10 ** 6, dump_idx=idx)
+    got, gd = gpu_eval(ctx, prof, tr, classes, off, inst, 10 ** 6, mapping=mapping, dump_idx=idx)
+    assert (want["status"] == 0).all() and want["n_served"].sum() > 0
+    assert_records_equal(got, want, "extreme values")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+
+
+def test_step_counter_wraps_32_bits(ctx, oracle_mod):
+    """70,000 requests of 65535 tokens through one single-slot instance: the instance's step counter
+    passes 2^32 (the kernels keep it modulo 2^32 and compare only 16-bit distances; the oracle counts
+    in 64 bits).  No limits, so everything is served in order (single-server queue)."""
+    prof = gen.profile_tiny()
+    prof["step_us"][:] = 3
+    n = 70_000
+    tr = np.zeros(n, dtype=gen.REQUEST_DTYPE)
+    tr["arrival_us"] = np.arange(n, dtype=np.int64) * 150_000
+    tr["in_tokens"] = 16
+    tr["out_tokens"] = 65535
+    classes = gen.make_classes([(None, None, None)])
+    off, inst = gen.candidates_from_lists([[(0, 0, 1)], [(0, 1, 2)]])
+    want = oracle_mod.eval_placements(prof, tr, classes, off, inst, 4)
+    got, _ = gpu_eval(ctx, prof, tr, classes, off, inst, 4)
+    assert int(want["n_served"][0]) == n and int(want["tokens_out"][0]) == n * 65535 > 2 ** 32
+    assert_records_equal(got, want, "counter wrap")
+
+
 def test_api_errors(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny")
