@@ -14,8 +14,10 @@ constexpr long long kWaitCycles = 4000000000ll;  // bound on any device-side wai
 
 // Buckets the validation kernel sorts candidates into.
 // 0..5: lane groups of 1,2,4,8,16,32 lanes (one lane per instance)
-// 6..8: block layout with 2, 8, 32 warps (one warp per instance, strided above 32)
-constexpr int kNumBuckets = 9;
+// 6..8: block layout with 2, 4, 8 warps, one warp per instance, state in registers
+// 9:    block layout with 16 warps striding over up to 128 instances, state in shared memory
+constexpr int kNumBuckets = 10;
+constexpr int kGenericBlockBucket = 9;
 constexpr int kCostBins = 256;   // bin 0 = most expensive (largest total batch cap)
 constexpr int kCounterWords = 8192;  // counters | work counters | histograms + cursors, cleared per call
 constexpr int kGroupThreads = 128;

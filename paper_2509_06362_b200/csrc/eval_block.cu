@@ -379,20 +379,14 @@ static int occupancy_one(const EvalParams& P, int tile_recs) {
     return n < 1 ? 1 : n;
 }
 
-// bucket 6: <= 2 instances (2 warps), 7: <= 8 (8 warps), 8: the rest (16 warps, strided)
+// the generic kernel: 16 warps striding over up to 128 instances (buckets with at most 8 instances
+// use the register-resident kernel of eval_block_reg.cu)
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream) {
-    if (bucket == 6) return launch_one<2>(P, grid, tile_recs, bucket, stream);
-    if (bucket == 7) return launch_one<8>(P, grid, tile_recs, bucket, stream);
     return launch_one<16>(P, grid, tile_recs, bucket, stream);
 }
-int occupancy_eval_block(const EvalParams& P, int bucket, int tile_recs) {
-    if (bucket == 6) return occupancy_one<2>(P, tile_recs);
-    if (bucket == 7) return occupancy_one<8>(P, tile_recs);
-    return occupancy_one<16>(P, tile_recs);
-}
-size_t block_payload_per_cta(int bucket) {
-    const int smem_inst = bucket == 6 ? 2 : (bucket == 7 ? 8 : 32);
-    return (size_t)(MAASO_MAX_INSTANCES - smem_inst) * MAASO_WMAX;  // Payload entries
+int occupancy_eval_block(const EvalParams& P, int, int tile_recs) { return occupancy_one<16>(P, tile_recs); }
+size_t block_payload_per_cta(int) {
+    return (size_t)(MAASO_MAX_INSTANCES - BlockCfg<16>::kSmemPay) * MAASO_WMAX;  // Payload entries
 }
 
 }  // namespace maaso

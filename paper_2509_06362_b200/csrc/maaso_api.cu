@@ -15,6 +15,8 @@ cudaError_t launch_rej_hash(uint64_t* out, uint32_t n);
 cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, cudaStream_t stream);
 int occupancy_eval_group(const EvalParams& P, int tile_recs);
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
+cudaError_t launch_eval_block_reg(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
+int occupancy_eval_block_reg(const EvalParams& P, int bucket, int tile_recs);
 int occupancy_eval_block(const EvalParams& P, int bucket, int tile_recs);
 size_t block_payload_per_cta(int bucket);
 size_t topk_scratch_bytes(uint64_t n_cand, uint32_t k);
@@ -382,17 +384,19 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     int grid_g = ctx->sm_count * occ_g;
     const uint64_t max_items_g = (uint64_t)C / 4 + 6;  // at most one work item per 4 candidates + bucket tails
     if ((uint64_t)grid_g > max_items_g) grid_g = (int)max_items_g;
-    int grid_b[3];
+    int grid_b[4];
     size_t pay_entries = (size_t)grid_g * kGroupThreads * MAASO_WMAX;
-    for (int b = 6; b <= 8; b++) {
+    for (int b = 6; b <= kGenericBlockBucket; b++) {
         // without the block mapping only candidates with more than 32 instances go to a block kernel
-        const bool used = o.mapping == MAASO_MAP_BLOCK || (b == 8 && cands->n_inst > 32);
+        const bool used = o.mapping == MAASO_MAP_BLOCK || (b == kGenericBlockBucket && cands->n_inst > 32);
         grid_b[b - 6] = 0;
         if (!used) continue;
-        int gb = ctx->sm_count * occupancy_eval_block(P, b, tile);
+        // placements with at most 8 instances: one warp per instance with register-resident state
+        int gb = ctx->sm_count * (b < kGenericBlockBucket ? occupancy_eval_block_reg(P, b, tile)
+                                                        : occupancy_eval_block(P, b, tile));
         if ((uint64_t)gb > C) gb = (int)C;
         grid_b[b - 6] = gb;
-        const size_t need = (size_t)gb * block_payload_per_cta(b);
+        const size_t need = b < kGenericBlockBucket ? 0 : (size_t)gb * block_payload_per_cta(b);
         if (need > pay_entries) pay_entries = need;
     }
 
@@ -432,9 +436,10 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
         if (e != cudaSuccess) return cuda_fail(ctx, e, "group kernel launch");
     }
     if (ctx->timing) cudaEventRecord(ctx->ev[2], stream);
-    for (int b = 6; b <= 8; b++) {
+    for (int b = 6; b <= kGenericBlockBucket; b++) {
         if (grid_b[b - 6] == 0) continue;
-        e = launch_eval_block(P, b, grid_b[b - 6], tile, stream);
+        e = b < kGenericBlockBucket ? launch_eval_block_reg(P, b, grid_b[b - 6], tile, stream)
+                  : launch_eval_block(P, b, grid_b[b - 6], tile, stream);
         launches++;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "block kernel launch");
     }

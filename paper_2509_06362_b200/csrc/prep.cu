@@ -47,9 +47,9 @@ __global__ void prep_kernel(const EvalParams P) {
         return;
     }
     int b;
-    if (P.mapping == MAASO_MAP_BLOCK) b = n <= 2 ? 6 : (n <= 8 ? 7 : 8);
+    if (P.mapping == MAASO_MAP_BLOCK) b = n <= 2 ? 6 : (n <= 4 ? 7 : (n <= 8 ? 8 : kGenericBlockBucket));
     else if (n <= 32) b = n <= 1 ? 0 : 32 - __clz((int)(n - 1));
-    else b = 8;
+    else b = kGenericBlockBucket;
     // Cost estimate: the total batch cap (how many requests the placement can have in flight;
     // it tracks the number of served requests and so the number of simulation events).
     const uint32_t bin = (kCostBins - 1) - min((uint32_t)(kCostBins - 1), sum_b / 8u);
