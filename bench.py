@@ -27,8 +27,8 @@ TOPK = 64
 # ncu counters of eval_group_kernel on the default workload (profiles/eval_group_kernel_node_sweep.md).
 # They describe the kernel as committed with that summary; set to None when the kernel changes.
 PROFILED = {"workload": "node", "mapping": 0,
-            "dram_bytes_per_launch": 11_255_040 + 3_470_336,
-            "warp_inst_per_launch": 6_513_415_397}
+            "dram_bytes_per_launch": 11_290_112 + 3_329_792,
+            "warp_inst_per_launch": 6_453_245_806}
 SM_COUNT, ISSUE_PER_SM = 148, 4   # B200: 148 SMs x 4 warp schedulers, one warp instruction per cycle each
 
 
