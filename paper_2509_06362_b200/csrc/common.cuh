@@ -40,6 +40,14 @@ __device__ __forceinline__ Request decode_request(uint4 v) {
     return q;
 }
 
+// A trace record prepared once per trace for the lane-group kernel (48 bytes, three 16-byte
+// words): everything about a request that does not depend on the candidate.
+//   word 0: arrival time, latest first-token time (arrival + TTFT limit, INT64_MAX if none)
+//   word 1: latest finish time (arrival + end-to-end limit, INT64_MAX if none), input tokens,
+//           TBT limit clamped to 32 bits (0xFFFFFFFF = none; step times are below 2^31)
+//   word 2: checksum term of "this request was rejected", S - 1 | cls << 16 | model << 24, 0
+constexpr int kCookedWords = 3;
+
 // What a running request must remember until it completes (32 bytes, two 16-byte words).
 struct Payload {
     int64_t first_tok;
@@ -127,8 +135,9 @@ __device__ __forceinline__ uint32_t ceil_div_steps(int64_t dt, uint32_t s) {
     return (uint32_t)(((uint64_t)dt - 1ull) / s) + 1u;
 }
 
-// ceil(dt / s) when the quotient is known to be below 2^16 and rs = 1/s rounded to float:
-// the float estimate is then within one of the true quotient and is fixed up exactly.
+// ceil(dt / s) when the quotient is known to be below 2^16 and rs = 1/s in float, exact to a
+// few units in the last place: the float estimate is then within one of the true quotient
+// and is fixed up exactly.
 __device__ __forceinline__ uint32_t ceil_div_small(int64_t dt, uint32_t s, float rs) {
     if (((uint64_t)dt >> 32) != 0) return (uint32_t)(((uint64_t)dt - 1ull) / s) + 1u;
     uint32_t q = (uint32_t)(__uint2float_rz((uint32_t)dt) * rs);
@@ -136,6 +145,12 @@ __device__ __forceinline__ uint32_t ceil_div_small(int64_t dt, uint32_t s, float
     if (r < 0) { q--; r += s; }
     else if (r >= (int64_t)s) { q++; r -= s; }
     return q + (r > 0 ? 1u : 0u);
+}
+
+__device__ __forceinline__ float rcp_approx(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
 }
 
 __device__ __forceinline__ int64_t prefill_us(uint32_t base, uint32_t q16, uint32_t in_tokens) {
@@ -195,6 +210,7 @@ struct EvalParams {
     uint32_t n_req;
     uint32_t n_classes;
     const int64_t* classes;  // [n_classes][3]
+    const uint4* cooked;     // [n_req][kCookedWords] prepared records (lane-group kernel)
     const uint64_t* rej_hash;  // [n_req] checksum term of "request r was rejected" (same for every candidate)
     const int32_t* rows;     // [n_rows][kRowStride]
     const int32_t* devices;

@@ -1,13 +1,16 @@
 // Scoring kernel, lane-group mapping: a candidate with I <= 32 instances is replayed by a
 // group of G = 2^ceil(log2 I) lanes of one warp, one lane per simulated instance.  All
-// instance state lives in registers; slot keys in shared memory; the distributor's argmin
-// is a shuffle butterfly inside the group.  The trace is staged once per thread block in
-// shared-memory tiles by 1-D bulk copies (TMA) and shared by every candidate of the block.
+// instance state lives in registers; slot keys and the data of running requests in a
+// shared-memory pool; the distributor's argmin is a shuffle butterfly inside the group.
+// The trace (and the per-request checksum term of a rejection) is staged once per thread
+// block in shared-memory tiles by 1-D bulk copies (TMA) and shared by every candidate of
+// the block.  No global memory access sits on the per-request path.
 #include "lane_sim.cuh"
 
 namespace maaso {
 
 constexpr int kStages = 3;
+constexpr uint32_t kFullMask = 0xFFFFFFFFu;
 
 __device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t v, int off, uint32_t mask) {
     uint32_t lo = __shfl_xor_sync(mask, (uint32_t)v, off);
@@ -27,56 +30,72 @@ struct ArgMin {
 };
 
 // Distributor's choice inside a lane group: smallest (tier, predicted first token), lowest lane
-// among equals.  Called by all 32 lanes; every operation uses the full mask and stays inside
-// the group because xor offsets are below G.  G may be smaller than the group when only its
-// first G lanes hold instances: the other lanes then see "nothing found", which is harmless
-// because only lanes with instances and the group's first lane act on the result.
-__device__ __forceinline__ ArgMin group_argmin(uint64_t key, uint32_t gmask, uint32_t G) {
+// among equals.  Called by all 32 lanes.  The comparison runs on the 32-bit keys of lane_predict;
+// only if the group's minimum is a clamped key (a first token 2^31 us or more ahead: rare) the
+// group repeats the reduction on (tier, first token) in 64 bits, with its own lane mask.
+// `own`: the warp holds a single candidate, so one full-warp reduction replaces the butterfly.
+__device__ __forceinline__ ArgMin group_argmin(uint32_t k32, int64_t first, uint32_t gmask, uint32_t G, bool own) {
     ArgMin r;
-    uint64_t best = key;
-    for (uint32_t off = 1; off < G; off <<= 1) best = min(best, shfl_xor_u64(best, (int)off, 0xFFFFFFFFu));
-    r.found = best != kKeyInf;
-    r.tier = (uint32_t)(best >> 63);
-    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, key == best) & gmask;
+    uint32_t best = k32;
+    if (own) {
+        best = __reduce_min_sync(kFullMask, k32);
+    } else {
+        for (uint32_t o = 1; o < G; o <<= 1) best = min(best, __shfl_xor_sync(kFullMask, best, (int)o));
+    }
+    bool eq = k32 == best;
+    if ((best & 0x7FFFFFFFu) == kOffSat) {
+        const uint64_t key = k32 == kKey32Inf ? kKeyInf : (((uint64_t)(k32 >> 31) << 63) | (uint64_t)first);
+        uint64_t b64 = key;
+        for (uint32_t o = 1; o < G; o <<= 1) b64 = min(b64, shfl_xor_u64(b64, (int)o, gmask));
+        eq = key == b64;
+    }
+    __syncwarp();
+    r.found = best != kKey32Inf;
+    r.tier = best >> 31;
+    const uint32_t votes = __ballot_sync(kFullMask, eq) & gmask;
     r.winner = r.found ? __ffs((int)votes) - 1 : (int)(threadIdx.x & 31u);
     return r;
 }
 
 struct GroupSmem {
-    uint4* tiles;        // [kStages][tile_recs]
-    int32_t* steps;      // [n_rows][64]
+    uint4* tiles;        // [kStages][tile_recs][kCookedWords] prepared request records
+    unsigned char* pool; // slot keys + block minima, carved per work item in 32-byte units
+    uint4* qa;           // [kQueue][kGroupThreads] queued completions: first-token time, arrival time
+    uint2* qb;           // [kQueue][kGroupThreads] request index, S | cls << 16
+    int64_t* qf;         // [kQueue][kGroupThreads] finish time
     int64_t* classes;    // [n_classes][3], negative = no limit (completion accounting)
-    int64_t* plimits;    // [n_classes][3], INT64_MAX = no limit (distributor prediction)
-    uint16_t* keys;      // [kGroupThreads][kKeyStride]
-    uint32_t* hbc;       // [kGroupThreads][8]
     uint64_t* full_bar;  // [kStages]
+    int32_t* steps;      // [n_rows][64]
     uint32_t* empty_cnt; // [kStages]
     uint32_t* work;      // [2]
+    uint32_t* wsum;      // [warps] pool units each warp asks for
 };
 
-__host__ __device__ inline size_t group_smem_bytes(uint32_t n_rows, uint32_t n_classes, int tile_recs) {
-    size_t b = (size_t)kStages * tile_recs * 16;
+__host__ __device__ inline size_t group_smem_static(uint32_t n_rows, uint32_t n_classes, int tile_recs) {
+    size_t b = (size_t)kStages * (tile_recs + 1) * 16 * kCookedWords;  // one spare record per stage (look-ahead read)
+    b += (size_t)kQueue * kGroupThreads * (16 + 8 + 8);
+    b += (size_t)n_classes * 24;
+    b += kStages * 8;
     b += (size_t)n_rows * 64 * 4;
-    b += (size_t)n_classes * 48;
-    b += (size_t)kGroupThreads * kKeyStride * 2;
-    b += (size_t)kGroupThreads * 8 * 4;
-    b += kStages * 8 + kStages * 4 + 8 + 32;
-    return (b + 15) & ~(size_t)15;
+    b += kStages * 4 + 8 + 16 + 32;
+    return (b + 31) & ~(size_t)31;
 }
 
 __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows, uint32_t n_classes,
-                                           int tile_recs) {
+                                           int tile_recs, uint32_t pool_bytes) {
     GroupSmem s;
-    // 16-byte aligned parts first (tiles, slot keys are read as 16-byte words)
+    // every part that is read in 16-byte words first (all sizes are multiples of 16 bytes)
+    s.pool = base;
+    base += pool_bytes;
     s.tiles = reinterpret_cast<uint4*>(base);
-    base += (size_t)kStages * tile_recs * 16;
-    s.keys = reinterpret_cast<uint16_t*>(base);
-    base += (size_t)kGroupThreads * kKeyStride * 2;
-    s.hbc = reinterpret_cast<uint32_t*>(base);
-    base += (size_t)kGroupThreads * 8 * 4;
+    base += (size_t)kStages * (tile_recs + 1) * 16 * kCookedWords;
+    s.qa = reinterpret_cast<uint4*>(base);
+    base += (size_t)kQueue * kGroupThreads * 16;
+    s.qb = reinterpret_cast<uint2*>(base);
+    base += (size_t)kQueue * kGroupThreads * 8;
+    s.qf = reinterpret_cast<int64_t*>(base);
+    base += (size_t)kQueue * kGroupThreads * 8;
     s.classes = reinterpret_cast<int64_t*>(base);
-    base += (size_t)n_classes * 24;
-    s.plimits = reinterpret_cast<int64_t*>(base);
     base += (size_t)n_classes * 24;
     s.full_bar = reinterpret_cast<uint64_t*>(base);
     base += kStages * 8;
@@ -85,25 +104,36 @@ __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows,
     s.empty_cnt = reinterpret_cast<uint32_t*>(base);
     base += kStages * 4;
     s.work = reinterpret_cast<uint32_t*>(base);
+    base += 8;
+    s.wsum = reinterpret_cast<uint32_t*>(base);
     return s;
+}
+
+// One tile of prepared records (48 bytes each, so every copy is a multiple of 16 bytes and
+// starts on a 16-byte boundary).
+__device__ __forceinline__ void issue_tile(const GroupSmem& sm, const EvalParams& P, uint32_t stage, uint32_t tile,
+                                           int tile_recs) {
+    const uint32_t recs = min((uint32_t)tile_recs, P.n_req - tile * tile_recs);
+    const uint32_t bytes = recs * 16u * kCookedWords;
+    mbar_expect_tx(&sm.full_bar[stage], bytes);
+    bulk_load(sm.tiles + (size_t)stage * (tile_recs + 1) * kCookedWords, P.cooked + (size_t)tile * tile_recs * kCookedWords,
+              bytes, &sm.full_bar[stage]);
 }
 
 // OPT: the distributor predicts with the step time right after admission (optimistic estimate)
 template <bool OPT>
-__global__ void __launch_bounds__(kGroupThreads)
-eval_group_kernel(const EvalParams P, const int tile_recs) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const GroupSmem sm = carve(smem_raw, P.n_rows, P.n_classes, tile_recs);
-    const uint32_t tid = threadIdx.x, lane = tid & 31u;
+__global__ void __launch_bounds__(kGroupThreads, 4)
+eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_bytes) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const GroupSmem sm = carve(smem_raw, P.n_rows, P.n_classes, tile_recs, pool_bytes);
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     constexpr uint32_t kWarps = kGroupThreads / 32;
 
     // profile residency: decode-step tables and SLO classes into shared memory
     for (uint32_t i = tid; i < P.n_rows * 64u; i += kGroupThreads)
         sm.steps[i] = P.rows[(i >> 6) * kRowStride + 2 + (i & 63u)];
     for (uint32_t i = tid; i < P.n_classes * 3u; i += kGroupThreads) {
-        const int64_t v = P.classes[i];
-        sm.classes[i] = v;
-        sm.plimits[i] = v < 0 ? INT64_MAX : v;
+        sm.classes[i] = P.classes[i];
     }
     if (tid == 0) {
         for (int s = 0; s < kStages; s++) {
@@ -115,12 +145,15 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
     }
     __syncthreads();
 
+    unsigned char* const lane_scratch =
+        reinterpret_cast<unsigned char*>(P.payload) + ((size_t)blockIdx.x * kGroupThreads + tid) * kLaneScratchBytes;
     LaneEnv env;
-    env.keys = sm.keys + tid * kKeyStride;
-    env.hbc = sm.hbc + tid * 8;
-    env.pay = P.payload + ((size_t)blockIdx.x * kGroupThreads + tid) * MAASO_WMAX;
-    env.classes = sm.classes;
-    uint32_t* const hbc = env.hbc;
+    env.qf = sm.qf + tid;
+    env.qa = sm.qa + tid;
+    env.qb = sm.qb + tid;
+    env.pay_a = reinterpret_cast<uint4*>(lane_scratch + kLaneScratchA);
+    env.pay_b = reinterpret_cast<uint2*>(lane_scratch + kLaneScratchB);
+    env.ovf = lane_scratch + kLaneScratchOvf;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
     const uint32_t n_tiles = (P.n_req + tile_recs - 1) / tile_recs;
     uint32_t tile_seq = 0;  // tiles consumed so far by this warp (same in every warp)
@@ -163,6 +196,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
         int b = 5;
         while (wi >= items[b]) { wi -= items[b]; b--; }
         const uint32_t G = 1u << b;
+        const bool own = b == 5;  // the warp holds one candidate
         const uint32_t sub = tid & (G - 1u);
         // The bucket list is sorted by decreasing cost estimate.  Group slot j of warp x takes
         // position j * n_warps + x: every warp gets one candidate of each cost quantile, so the
@@ -171,17 +205,18 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
         const uint32_t cnt = P.bucket_count[b];
         const uint32_t gpw = 32u >> b;
         const uint32_t n_warps = (cnt + gpw - 1) / gpw;
-        const uint32_t warp_x = wi * kWarps + (tid >> 5);
+        const uint32_t warp_x = wi * kWarps + warp;
         const uint32_t pos = (lane >> b) * n_warps + warp_x;
         const bool valid = warp_x < n_warps && pos < cnt;
         const uint32_t cand = valid ? P.bucket_list[(size_t)b * P.n_cand + pos] : 0u;
-        const uint32_t gmask = (G == 32u) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(G - 1u)));
+        const uint32_t gmask = (G == 32u) ? kFullMask : (((1u << G) - 1u) << (lane & ~(G - 1u)));
 
         uint32_t n_i = 0, lo = 0;
         if (valid) { lo = P.offsets[cand]; n_i = P.offsets[cand + 1] - lo; }
         const bool has = valid && sub < n_i;
         LaneInst in;
-        in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = 0; in.sw = 1; in.rsw = 1.0f; in.bslots = 0; in.mask = 0;
+        in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = kKeyEmpty; in.sw = 1; in.rsw = 1.0f; in.qn = 0;
+        in.mask = ~0ull; in.gen = 0;
         in.B = 1; in.model = 0xFFFFFFFFu; in.step = sm.steps; in.stepB = 1; in.pre_base = 0; in.pre_q16 = 0;
         if (has) {
             const uint32_t word = P.inst[lo + sub];
@@ -192,52 +227,83 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
             in.stepB = (uint32_t)in.step[in.B - 1];
             in.pre_base = (uint32_t)P.rows[row * kRowStride + 0];
             in.pre_q16 = (uint32_t)P.rows[row * kRowStride + 1];
+            in.mask = in.B >= 64u ? 0ull : (~0ull << in.B);
         }
-        // A warp that holds a single candidate (bucket 5, possibly promoted there with few
-        // instances) only needs as many butterfly rounds as it has instances.
-        const uint32_t n_i_warp = __shfl_sync(0xFFFFFFFFu, n_i, 0);
-        const uint32_t Geff = b == 5 ? (n_i_warp <= 1 ? 1u : 1u << (32 - __clz((int)(n_i_warp - 1)))) : G;
+        // key storage: every lane takes one 32-byte unit per block of 8 slots of its batch cap,
+        // plus one for the block minima, from the thread block's pool, in thread order; lanes the
+        // pool cannot hold use their global scratch instead
+        {
+            const uint32_t nblk = has ? (in.B + 7u) >> 3 : 0u;
+            const uint32_t units = has ? nblk + 1u : 0u;
+            uint32_t incl = units;
+            for (uint32_t o = 1; o < 32u; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(kFullMask, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31u) sm.wsum[warp] = incl;
+            __syncthreads();
+            uint32_t start = incl - units;
+            for (uint32_t i = 0; i < warp; i++) start += sm.wsum[i];
+            unsigned char* region = ((size_t)(start + units) * kKeyUnitBytes <= pool_bytes)
+                                        ? sm.pool + (size_t)start * kKeyUnitBytes
+                                        : lane_scratch + kLaneScratchKeys;
+            env.keys_shared = region != lane_scratch + kLaneScratchKeys;
+            env.keys = reinterpret_cast<uint32_t*>(region);
+            env.bm_lo = reinterpret_cast<uint4*>(region + (size_t)nblk * kKeyUnitBytes);
+            env.bm_hi = env.bm_lo + 1;
+            const uint4 e4 = make_uint4(kKeyEmpty, kKeyEmpty, kKeyEmpty, kKeyEmpty);
+            for (uint32_t i = 0; i < 2u * units; i++) reinterpret_cast<uint4*>(region)[i] = e4;
+        }
+        const bool warp_has_work = __any_sync(kFullMask, valid);
         const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
         Dump dump{nullptr, nullptr, nullptr};
         if (valid) dump = dump_for(P, cand);
-        env.dump = dump;
-        env.inst_idx = sub;
-        Stats st; st.clear();
-        for (int i = 0; i < 8; i++) hbc[i] = 0;
+        // per-request side outputs (dump rows, per-model rejection counts) are rare: one flag guards them
+        const bool side = dump.finish || dump.first || dump.inst || P.rej_by_model;
+        LaneStats ls;
+        ls.st.clear();
+        for (int i = 0; i < 8; i++) ls.hbc[i] = 0;
+        uint64_t rej_sum = 0;  // checksum terms of rejected requests
         int64_t now = 0;
         uint32_t n_counted = 0, n_rejected = 0, status = 0;
-        uint64_t attempts = 0;
+        uint64_t attempts = 0;   // distributor rounds beyond the first of each counted request
 
         // trace staging: first tiles of this batch
         if (tid == 0 && !P.stall_test) {
-            for (uint32_t j = 0; j < (uint32_t)kStages && j < n_tiles; j++) {
-                const uint32_t s = (tile_seq + j) % kStages;
-                const uint32_t recs = min((uint32_t)tile_recs, P.n_req - j * tile_recs);
-                mbar_expect_tx(&sm.full_bar[s], recs * 16u);
-                bulk_load(sm.tiles + (size_t)s * tile_recs, P.reqs + (size_t)j * tile_recs, recs * 16u,
-                          &sm.full_bar[s]);
-            }
+            for (uint32_t j = 0; j < (uint32_t)kStages && j < n_tiles; j++)
+                issue_tile(sm, P, (tile_seq + j) % kStages, j, tile_recs);
         }
 
         for (uint32_t t = 0; t < n_tiles; t++) {
             const uint32_t s = tile_seq % kStages, parity = (tile_seq / kStages) & 1u;
             const bool arrived = mbar_wait_bounded(&sm.full_bar[s], parity, P.wait_cycles);
-            if (!__all_sync(0xFFFFFFFFu, arrived)) {
+            if (!__all_sync(kFullMask, arrived)) {
                 mbar_wait_bounded(&sm.full_bar[s], parity, P.wait_cycles);  // give copies in flight one more bounded chance
                 status = MAASO_CAND_ETIMEOUT;
                 sm.work[1] = 1;
                 break;
             }
-            const uint4* tile = sm.tiles + (size_t)s * tile_recs;
+            const uint4* tile = sm.tiles + (size_t)s * (tile_recs + 1) * kCookedWords;
             const uint32_t recs = min((uint32_t)tile_recs, P.n_req - t * tile_recs);
-            uint4 raw_next = tile[0];
-            for (uint32_t ri = 0; ri < recs; ri++) {
-                const uint4 raw = raw_next;
-                raw_next = tile[min(ri + 1, recs - 1)];  // read the next record ahead of its use
+            uint4 nx0 = tile[0], nx1 = tile[1], nx2 = tile[2];
+            // a warp without a candidate only keeps the tile pipeline going
+            for (uint32_t ri = warp_has_work ? 0u : recs; ri < recs; ri++) {
+                const uint4 r0 = nx0, r1 = nx1, r2 = nx2;
+                {
+                    // next record, ahead of its use (after the last one: the stage's spare record, never used)
+                    const uint4* nx = tile + (size_t)(ri + 1) * kCookedWords;
+                    nx0 = nx[0]; nx1 = nx[1]; nx2 = nx[2];
+                }
+                // statistics of completed requests: every fourth request, if some lane's queue is half full
+                if ((ri & 3u) == 3u && __any_sync(kFullMask, in.qn >= (uint32_t)(kQueue / 2))) {
+                    flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first,
+                                dump.inst);
+                    in.qn = 0;
+                }
                 // All 32 lanes walk the trace together and every warp-level operation below uses
                 // the full mask (segmented by the group width), so the groups of a warp share one
                 // instruction stream; only events (retire, admit) diverge.
-                const Request q = decode_request(raw);
+                const CookedReq q = decode_cooked(r0, r1, r2);
                 const uint32_t req = t * tile_recs + ri;
                 bool pending = valid && status == 0 && ((cmask >> (q.cls & 31u)) & 1u);
                 if (pending) {
@@ -246,38 +312,37 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                 }
                 const int64_t pre = prefill_us(in.pre_base, in.pre_q16, q.in_tokens);
                 const bool elig = has && in.model == q.model;
-                const int64_t lim_ttft = sm.plimits[q.cls * 3 + 0];
-                const int64_t lim_tbt = sm.plimits[q.cls * 3 + 1];
-                const int64_t lim_e2e = sm.plimits[q.cls * 3 + 2];
                 uint32_t tries = 0;
                 do {
-                    uint64_t key = kKeyInf;
-                    int64_t t0 = 0;
-                    if (pending) {
+                    uint32_t key = kKey32Inf;
+                    int64_t t0 = 0, first = 0;
+                    if (OPT && pending) {
                         attempts++;
                         tries++;
                     }
                     if (pending && elig) {
-                        lane_advance(in, now, false, env, st);
-                        key = lane_predict(in, q, pre, lim_ttft, lim_tbt, lim_e2e, OPT, t0);
+                        lane_advance(in, now, false, env, status);
+                        key = lane_predict(in, q, pre, now, OPT, t0, first);
                     }
-                    const ArgMin am = group_argmin(key, gmask, Geff);
-                    const int64_t t0w = (int64_t)shfl_u64((uint64_t)t0, am.winner, 0xFFFFFFFFu);
+                    const ArgMin am = group_argmin(key, first, gmask, G, own);
+                    const int64_t t0w = (int64_t)shfl_u64((uint64_t)t0, am.winner, kFullMask);
                     if (pending) {
                         if (!am.found) {
                             // overflow protection: nobody can meet the deadline -> rejected
                             n_rejected++;
                             if (sub == 0) {
-                                st.checksum += __ldg(P.rej_hash + req);
-                                if (P.rej_by_model)
-                                    atomicAdd(&P.rej_by_model[(size_t)cand * MAASO_MAX_MODELS + q.model], 1u);
-                                if (dump.finish) dump.finish[req] = -1;
-                                if (dump.first) dump.first[req] = -1;
-                                if (dump.inst) dump.inst[req] = -1;
+                                rej_sum += q.rej;
+                                if (side) {
+                                    if (P.rej_by_model)
+                                        atomicAdd(&P.rej_by_model[(size_t)cand * MAASO_MAX_MODELS + q.model], 1u);
+                                    if (dump.finish) dump.finish[req] = -1;
+                                    if (dump.first) dump.first[req] = -1;
+                                    if (dump.inst) dump.inst[req] = -1;
+                                }
                             }
                             pending = false;
                         } else if (am.tier == 0) {
-                            if ((int)lane == am.winner) lane_admit(in, q, req, pre, env, st);
+                            if ((int)lane == am.winner) lane_admit(in, q, req, pre, env, status);
                             pending = false;
                         } else {
                             // every capable instance is full: wait until the chosen slot frees
@@ -287,10 +352,10 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                                 // at that time the winner has a free slot with the same predicted first
                                 // token, and no other instance's prediction can have become earlier or
                                 // feasible.  The second round is only counted; other clocks catch up lazily.
-                                attempts++;
+                                attempts++;  // the second round, counted only
                                 if ((int)lane == am.winner) {
-                                    lane_advance(in, now, false, env, st);
-                                    lane_admit(in, q, req, pre, env, st);
+                                    lane_advance(in, now, false, env, status);
+                                    lane_admit(in, q, req, pre, env, status);
                                 }
                                 pending = false;
                             } else if (tries >= kAttemptCap) {
@@ -299,7 +364,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                             }
                         }
                     }
-                } while (OPT && __any_sync(0xFFFFFFFFu, pending));
+                } while (OPT && __any_sync(kFullMask, pending));
             }
             // release the stage; the warp that arrives last refills it
             __syncwarp();
@@ -310,55 +375,81 @@ eval_group_kernel(const EvalParams P, const int tile_recs) {
                     sm.empty_cnt[s] = 0;
                     const uint32_t nt = t + kStages;
                     if (nt < n_tiles) {
-                        const uint32_t nrecs = min((uint32_t)tile_recs, P.n_req - nt * tile_recs);
                         fence_proxy_async();
-                        mbar_expect_tx(&sm.full_bar[s], nrecs * 16u);
-                        bulk_load(sm.tiles + (size_t)s * tile_recs, P.reqs + (size_t)nt * tile_recs,
-                                  nrecs * 16u, &sm.full_bar[s]);
+                        issue_tile(sm, P, s, nt, tile_recs);
                     }
                 }
             }
             tile_seq++;
         }
 
-        // drain, reduce over the group, write the record
-        if (has && status == 0) lane_advance(in, 0, true, env, st);
+        // drain, account what is still queued, reduce over the group, write the record
         __syncwarp();
-        constexpr uint32_t kFull = 0xFFFFFFFFu;
+        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first, dump.inst);
+        in.qn = 0;
+        if (has && status == 0) lane_advance(in, 0, true, env, status);
+        __syncwarp();
+        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first, dump.inst);
+        in.qn = 0;
+        Stats st = ls.st;
+        st.checksum += rej_sum;
+        uint32_t h[8];
+        for (int i = 0; i < 8; i++) h[i] = ls.hbc[i];
         for (uint32_t off = 1; off < G; off <<= 1) {
-            st.served += __shfl_xor_sync(kFull, st.served, (int)off);
-            st.hit += __shfl_xor_sync(kFull, st.hit, (int)off);
-            st.sum_ttft += (int64_t)shfl_xor_u64((uint64_t)st.sum_ttft, (int)off, kFull);
-            st.sum_e2e += (int64_t)shfl_xor_u64((uint64_t)st.sum_e2e, (int)off, kFull);
-            st.tokens += shfl_xor_u64(st.tokens, (int)off, kFull);
-            st.checksum += shfl_xor_u64(st.checksum, (int)off, kFull);
-            st.max_ttft = max(st.max_ttft, (int64_t)shfl_xor_u64((uint64_t)st.max_ttft, (int)off, kFull));
-            st.max_e2e = max(st.max_e2e, (int64_t)shfl_xor_u64((uint64_t)st.max_e2e, (int)off, kFull));
-            st.makespan = max(st.makespan, (int64_t)shfl_xor_u64((uint64_t)st.makespan, (int)off, kFull));
+            for (int i = 0; i < 8; i++) h[i] += __shfl_xor_sync(kFullMask, h[i], (int)off);
+            status |= __shfl_xor_sync(kFullMask, status, (int)off);
+            st.served += __shfl_xor_sync(kFullMask, st.served, (int)off);
+            st.hit += __shfl_xor_sync(kFullMask, st.hit, (int)off);
+            st.sum_ttft += (int64_t)shfl_xor_u64((uint64_t)st.sum_ttft, (int)off, kFullMask);
+            st.sum_e2e += (int64_t)shfl_xor_u64((uint64_t)st.sum_e2e, (int)off, kFullMask);
+            st.tokens += shfl_xor_u64(st.tokens, (int)off, kFullMask);
+            st.checksum += shfl_xor_u64(st.checksum, (int)off, kFullMask);
+            st.max_ttft = max(st.max_ttft, (int64_t)shfl_xor_u64((uint64_t)st.max_ttft, (int)off, kFullMask));
+            st.max_e2e = max(st.max_e2e, (int64_t)shfl_xor_u64((uint64_t)st.max_e2e, (int)off, kFullMask));
+            st.makespan = max(st.makespan, (int64_t)shfl_xor_u64((uint64_t)st.makespan, (int)off, kFullMask));
         }
         __syncwarp();
         if (valid && sub == 0) {
-            uint32_t h[8];
-            for (int i = 0; i < 8; i++) h[i] = 0;
-            for (uint32_t g = 0; g < G; g++)
-                for (int i = 0; i < 8; i++) h[i] += sm.hbc[(tid + g) * 8 + i];
-            write_result(P.out + cand, status, n_counted, n_rejected, attempts, st, h);
+            // worst-case mode: one round per counted request plus the counted second rounds
+            write_result(P.out + cand, status, n_counted, n_rejected, OPT ? attempts : attempts + n_counted, st, h);
         }
     }
 }
 
-cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, cudaStream_t stream) {
-    const size_t smem = group_smem_bytes(P.n_rows, P.n_classes, tile_recs);
+// Shared memory of one block: the fixed parts plus a key pool that fills what is left when
+// `blocks_per_sm` blocks share an SM (1 KB per block is reserved by the system), at most what
+// 128 lanes with 64 slots each can use.
+static size_t group_smem_bytes(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm,
+                               uint32_t* pool_bytes) {
+    const size_t fixed = group_smem_static(P.n_rows, P.n_classes, tile_recs);
+    size_t budget = (size_t)smem_per_sm / (size_t)blocks_per_sm;
+    budget = budget > 1024 ? budget - 1024 : 0;
+    if (budget > 227u * 1024u) budget = 227u * 1024u;
+    size_t pool = budget > fixed ? budget - fixed : 0;
+    pool -= pool % 128;
+    const size_t all = (size_t)kGroupThreads * 9 * kKeyUnitBytes;
+    if (pool > all) pool = all;
+    *pool_bytes = (uint32_t)pool;
+    return fixed + pool;
+}
+
+cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, int blocks_per_sm, int smem_per_sm,
+                              cudaStream_t stream) {
+    uint32_t pool = 0;
+    const size_t smem = group_smem_bytes(P, tile_recs, blocks_per_sm, smem_per_sm, &pool);
     const bool opt = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
     auto kernel = opt ? eval_group_kernel<true> : eval_group_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kernel<<<grid, kGroupThreads, smem, stream>>>(P, tile_recs);
+    kernel<<<grid, kGroupThreads, smem, stream>>>(P, tile_recs, pool);
     return cudaGetLastError();
 }
 
-int occupancy_eval_group(const EvalParams& P, int tile_recs) {
-    const size_t smem = group_smem_bytes(P.n_rows, P.n_classes, tile_recs);
+size_t group_scratch_per_lane() { return kLaneScratchBytes; }
+
+int occupancy_eval_group(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm) {
+    uint32_t pool = 0;
+    const size_t smem = group_smem_bytes(P, tile_recs, blocks_per_sm, smem_per_sm, &pool);
     const bool opt = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
     auto kernel = opt ? eval_group_kernel<true> : eval_group_kernel<false>;
     cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

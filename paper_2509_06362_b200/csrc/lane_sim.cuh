@@ -3,30 +3,56 @@
 // from the latency table row of the instance (Eq. 1 as a table).
 //
 // Slot bookkeeping.  A running request is identified by the value of the instance's step
-// counter at which it ends; only the low 16 bits are kept (a request has at most 65535
-// output tokens, so distances to the counter are below 2^16 and order is preserved).
-// The 64 slot keys of a lane sit in shared memory in 8 blocks of 8, followed by the key of
-// each block's nearest completion, so a completion re-scans one block of 8 keys instead of
-// all 64.  The time of the instance's next completion is cached (`tc`): between events it
-// does not change, which lets a full instance skip its clock update entirely.
+// counter at which it ends.  Its slot key is one 32-bit word, `end index << 6 | slot`, so
+// the minimum over keys names the next completion and the slot that holds it at once; an
+// empty slot is all ones.  The keys of a lane sit in shared memory in blocks of 8 (one
+// 32-byte read) followed by one minimum per block, so a completion re-reads one block and
+// the 8 block minima; a lane takes as many blocks from its thread block's key pool as its
+// batch cap needs (lanes the pool cannot hold use global scratch through the same pointers).
+// The step counter is relative: it restarts at 0 whenever the instance is idle, and all
+// live keys are rebased when an end index would not fit 26 bits.
+//
+// No load from global memory sits on the per-request path (an L2 hit costs several hundred
+// cycles, and every step of a candidate's replay depends on the previous one).  What a
+// running request must remember (first-token time, arrival, request index, length, class:
+// 24 bytes) is written to global scratch at admission and never read back by a load: when
+// the request completes, asynchronous copies (cp.async) move it into a small per-lane queue
+// in shared memory together with the finish time.  The statistics are accumulated later,
+// by all lanes of the warp together (flush_queue), into per-lane sums that live in local
+// memory so that they cost no registers in the replay loop.  Each slot has two scratch entries used
+// alternately, and a lane lets at most one group of copies be in flight, so an entry is
+// never overwritten while a copy may still read it.
 #pragma once
 #include "common.cuh"
 
 namespace maaso {
 
-constexpr int kKeyStride = 72;  // uint16 per lane: 64 slot keys + 8 block minima (144 bytes)
+constexpr uint32_t kKeyEmpty = 0xFFFFFFFFu;
+constexpr uint32_t kRelMax = (1u << 26) - 2u;  // largest end index a key can hold
+constexpr int kKeyUnitBytes = 32;              // pool unit: one block of 8 keys (or the 8 block minima)
+constexpr int kQueue = 4;                      // queued completions per lane in shared memory
+constexpr int kQueueOvf = 72;                  // further entries per lane in global scratch
+// Per-lane global scratch: payload A [64 slots][2] x 16 B, payload B [64][2] x 8 B, queue
+// overflow x 32 B, and room for 64 keys + 8 block minima if the shared-memory pool is full.
+constexpr size_t kLaneScratchA = 0;
+constexpr size_t kLaneScratchB = 64 * 2 * 16;
+constexpr size_t kLaneScratchOvf = kLaneScratchB + 64 * 2 * 8;
+constexpr size_t kLaneScratchKeys = kLaneScratchOvf + (size_t)kQueueOvf * 32;
+constexpr size_t kLaneScratchBytes = kLaneScratchKeys + 9 * kKeyUnitBytes + 32;
+static_assert(kLaneScratchBytes % 32 == 0 && kLaneScratchKeys % 16 == 0, "lane scratch layout");
 
 struct LaneInst {
     int64_t T;        // clock, always a decode-step boundary (may lag `now` while the instance is full)
     int64_t tc;       // time of the next completion if nobody is admitted (valid while w > 0)
-    uint32_t K;       // decode steps done at T (only differences modulo 2^16 are used)
+    uint32_t K;       // decode steps done at T since the counter last restarted
     uint32_t w;       // running requests
     uint32_t B;       // batch cap = number of virtual slots
-    uint32_t kmin;    // low 16 bits of the smallest completion index among running requests
+    uint32_t kmin;    // smallest slot key (next completion), kKeyEmpty when idle
     uint32_t sw;      // step[w-1]: length of one decode step at the current level (valid while w > 0)
     float rsw;        // 1 / sw
-    uint32_t bslots;  // 3 bits per block: which of its 8 slots holds the block minimum
-    uint64_t mask;    // occupied slots
+    uint32_t qn;      // completions waiting in this lane's queue
+    uint64_t mask;    // occupied slots; bits at and above B are always set
+    uint64_t gen;     // per slot: which of its two scratch entries the current occupant uses
     const int32_t* step;  // shared-memory row: step[w-1] = one decode step with w running
     uint32_t stepB;   // step[B-1]
     uint32_t pre_base, pre_q16;
@@ -34,80 +60,165 @@ struct LaneInst {
 };
 
 struct LaneEnv {
-    uint16_t* keys;          // this lane's kKeyStride shared-memory halfwords
-    Payload* pay;            // this lane's 64 payload entries (global scratch)
-    uint32_t* hbc;           // this lane's 8 hit-by-class counters (shared memory)
-    const int64_t* classes;  // shared memory
-    uint32_t inst_idx;
-    Dump dump;
+    uint32_t* keys;          // this lane's slot keys, 8 per block of its batch cap (pool or global scratch)
+    uint4* bm_lo;            // this lane's block minima, blocks 0..3 (right after the keys)
+    uint4* bm_hi;            // blocks 4..7
+    bool keys_shared;        // keys and block minima are in the shared-memory pool (the usual case)
+    int64_t* qf;             // this lane's queue column: entry j at qf[j * kGroupThreads] = finish time
+    uint4* qa;               // entry j at qa[j * kGroupThreads] = first-token time, arrival time
+    uint2* qb;               // entry j at qb[j * kGroupThreads] = request index, S | cls << 16
+    uint4* pay_a;            // global scratch [64][2]: first-token time, arrival time
+    uint2* pay_b;            // global scratch [64][2]: request index, S | cls << 16
+    unsigned char* ovf;      // this lane's queue overflow (global scratch, 32-byte entries)
 };
 
-// Bring the payload of the request that will complete next into L1 ahead of its use.
-__device__ __forceinline__ void prefetch_l1(const void* p) {
-    asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
+// Per-lane sums of completed requests; only flush_queue touches them.
+struct LaneStats {
+    Stats st;
+    uint32_t hbc[8];  // hits by class
+};
+
+// Asynchronous copies global -> shared: no register, nothing waits for them until a wait.
+__device__ __forceinline__ void async_copy16(void* dst_smem, const void* src_gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst_smem)), "l"(src_gmem) : "memory");
+}
+__device__ __forceinline__ void async_copy8(void* dst_smem, const void* src_gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_addr(dst_smem)), "l"(src_gmem) : "memory");
+}
+// Close the group of copies just issued and wait until only that group may still be in flight.
+__device__ __forceinline__ void async_commit_keep_one() {
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 1;" ::: "memory");
+}
+__device__ __forceinline__ void async_copies_done() {
+    asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
-__device__ __forceinline__ uint32_t half_of(const uint4& v, int j) {  // j static after unrolling
-    const uint32_t word = (j >> 1) == 0 ? v.x : ((j >> 1) == 1 ? v.y : ((j >> 1) == 2 ? v.z : v.w));
-    return (j & 1) ? (word >> 16) : (word & 0xFFFFu);
+__device__ __forceinline__ uint32_t min8(const uint32_t (&v)[8]) {
+    return min(min(__vimin3_u32(v[0], v[1], v[2]), __vimin3_u32(v[3], v[4], v[5])), min(v[6], v[7]));
 }
 
-// The counter K has just reached the smallest completion index (clock = in.T).  Retire every
-// request that ends here, fix the block minima, the level and the cached next completion.
-__device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, Stats& st) {
-    const uint32_t K16 = in.K & 0xFFFFu;
-    const uint4 bm = *reinterpret_cast<const uint4*>(env.keys + 64);
-    uint32_t hit_blocks = 0, nd = 0x10000u, nb = 0;
-#pragma unroll
-    for (int b = 0; b < 8; b++) {  // branch-free per block: empty blocks count as infinitely far
-        if (b > 0 && 8u * b >= in.B) break;  // blocks beyond the batch cap are never used
-        const bool occ = ((uint32_t)(in.mask >> (8 * b)) & 0xFFu) != 0;
-        const uint32_t d = occ ? ((half_of(bm, b) - K16) & 0xFFFFu) : 0x10000u;
-        hit_blocks |= (d == 0 ? 1u : 0u) << b;
-        const uint32_t dd = d == 0 ? 0x10000u : d;
-        nb = dd < nd ? (uint32_t)b : nb;
-        nd = min(nd, dd);
+// *p = min(*p, v) without waiting for the old value (a reduction, not an atomic with a result).
+__device__ __forceinline__ void block_min_update(uint32_t* p, uint32_t v, bool shared) {
+    if (shared)
+        asm volatile("red.shared.min.u32 [%0], %1;" ::"r"(smem_addr(p)), "r"(v) : "memory");
+    else
+        asm volatile("red.global.min.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ uint32_t* bm_entry(const LaneEnv& env, uint32_t b) {
+    return reinterpret_cast<uint32_t*>(b < 4u ? env.bm_lo : env.bm_hi) + (b & 3u);
+}
+
+// A running request has left the instance at t_fin: queue the finish time and start the
+// copies of what it remembered (scratch entry `idx` = 2 * slot + generation).
+__device__ __forceinline__ void lane_push_slot(LaneInst& in, const LaneEnv& env, int64_t t_fin, uint32_t idx,
+                                               uint32_t& status) {
+    const uint32_t j = in.qn;
+    if (j < (uint32_t)kQueue) {
+        env.qf[j * kGroupThreads] = t_fin;
+        async_copy16(env.qa + j * kGroupThreads, env.pay_a + idx);
+        async_copy8(env.qb + j * kGroupThreads, env.pay_b + idx);
+        async_commit_keep_one();
+    } else if (j < (uint32_t)(kQueue + kQueueOvf)) {
+        const uint4 a = env.pay_a[idx];
+        const uint2 b = env.pay_b[idx];
+        uint4* o = reinterpret_cast<uint4*>(env.ovf + (size_t)(j - kQueue) * 32);
+        o[0] = make_uint4((uint32_t)t_fin, (uint32_t)((uint64_t)t_fin >> 32), b.x, b.y);
+        o[1] = a;
+    } else {
+        status = MAASO_CAND_ELOOP;  // cannot happen: at most 64 completions per lane between flushes
+        return;
     }
-    while (hit_blocks) {
-        const int b = __ffs((int)hit_blocks) - 1;
-        hit_blocks &= hit_blocks - 1;
-        const uint32_t occ = (uint32_t)(in.mask >> (8 * b)) & 0xFFu;
-        const uint4 kv = *reinterpret_cast<const uint4*>(env.keys + 8 * b);
-        uint32_t done = 0, bd = 0x10000u, bj = 0;
-#pragma unroll
-        for (int j = 0; j < 8; j++) {
-            const uint32_t d = ((occ >> j) & 1u) ? ((half_of(kv, j) - K16) & 0xFFFFu) : 0x10000u;
-            done |= (d == 0 ? 1u : 0u) << j;
-            const uint32_t dd = d == 0 ? 0x10000u : d;
-            bj = dd < bd ? (uint32_t)j : bj;
-            bd = min(bd, dd);
+    in.qn = j + 1;
+}
+
+// Same for a request that completes at admission (one output token): everything is in registers.
+__device__ __forceinline__ void lane_push_now(LaneInst& in, const LaneEnv& env, int64_t t_fin, uint4 a, uint2 b,
+                                              uint32_t& status) {
+    const uint32_t j = in.qn;
+    if (j < (uint32_t)kQueue) {
+        env.qf[j * kGroupThreads] = t_fin;
+        env.qa[j * kGroupThreads] = a;
+        env.qb[j * kGroupThreads] = b;
+    } else if (j < (uint32_t)(kQueue + kQueueOvf)) {
+        uint4* o = reinterpret_cast<uint4*>(env.ovf + (size_t)(j - kQueue) * 32);
+        o[0] = make_uint4((uint32_t)t_fin, (uint32_t)((uint64_t)t_fin >> 32), b.x, b.y);
+        o[1] = a;
+    } else {
+        status = MAASO_CAND_ELOOP;
+        return;
+    }
+    in.qn = j + 1;
+}
+
+// Statistics of the queued completions (Phi_S indicator, latency and throughput sums), by
+// all lanes of the warp together; every lane handles its own `n` entries.  Out of line on
+// purpose: the sums stay in local memory and the replay loop stays small.
+__device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
+                                         const unsigned char* ovf, uint32_t n, const int64_t* classes,
+                                         uint32_t inst_idx, int64_t* dump_finish, int64_t* dump_first,
+                                         int32_t* dump_inst) {
+    async_copies_done();
+    Stats st = ls->st;
+    const Dump no_dump{nullptr, nullptr, nullptr};
+    const bool dumping = dump_finish || dump_first || dump_inst;
+    for (uint32_t j = 0; j < n; j++) {
+        int64_t t_fin;
+        uint4 a;
+        uint2 b;
+        if (j < (uint32_t)kQueue) {
+            t_fin = qf[j * kGroupThreads];
+            a = qa[j * kGroupThreads];
+            b = qb[j * kGroupThreads];
+        } else {
+            const uint4* o = reinterpret_cast<const uint4*>(ovf + (size_t)(j - kQueue) * 32);
+            const uint4 h = o[0];
+            t_fin = (int64_t)(((uint64_t)h.y << 32) | h.x);
+            a = o[1];
+            b = make_uint2(h.z, h.w);
         }
-        in.bslots = (in.bslots & ~(7u << (3 * b))) | (bj << (3 * b));
-        nb = bd < nd ? (uint32_t)b : nb;
-        in.mask &= ~((uint64_t)done << (8 * b));
-        in.w -= __popc(done);
-        env.keys[64 + b] = (uint16_t)(K16 + bd);
-        nd = min(nd, bd);
-        while (done) {
-            const int j = __ffs((int)done) - 1;
-            done &= done - 1;
-            const Payload* p = env.pay + 8 * b + j;
-            const uint4 a = reinterpret_cast<const uint4*>(p)[0];
-            const uint4 c = reinterpret_cast<const uint4*>(p)[1];
-            const int64_t first_tok = (int64_t)(((uint64_t)a.y << 32) | a.x);
-            const int64_t arrival = (int64_t)(((uint64_t)a.w << 32) | a.z);
-            const uint32_t cls = c.y >> 16;
-            if (account_completion(st, env.classes, env.inst_idx, c.x, arrival, first_tok, in.T, c.y & 0xFFFFu,
-                                   cls, env.dump))
-                env.hbc[cls < 7 ? cls : 7]++;
+        const int64_t first = (int64_t)(((uint64_t)a.y << 32) | a.x);
+        const int64_t arrival = (int64_t)(((uint64_t)a.w << 32) | a.z);
+        const uint32_t cls = b.y >> 16;
+        if (account_completion(st, classes, inst_idx, b.x, arrival, first, t_fin, b.y & 0xFFFFu, cls, no_dump))
+            ls->hbc[cls < 7 ? cls : 7]++;
+        if (dumping) {
+            if (dump_finish) dump_finish[b.x] = t_fin;
+            if (dump_first) dump_first[b.x] = first;
+            if (dump_inst) dump_inst[b.x] = (int32_t)inst_idx;
         }
     }
-    in.kmin = (K16 + nd) & 0xFFFFu;
+    ls->st = st;
+}
+
+// The counter K has just reached the smallest end index (clock = in.T).  Retire every
+// request that ends here, one per round (the smallest key names its slot), fix the block
+// minima, the level and the cached next completion.
+__device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, uint32_t& status) {
+    const uint32_t Kc = in.K;
+    do {
+        const uint32_t slot = in.kmin & 63u, b = slot >> 3, sj = slot & 7u;
+        const uint4* kp = reinterpret_cast<const uint4*>(env.keys + 8u * b);
+        const uint4 k0 = kp[0], k1 = kp[1];
+        const uint4 m0 = *env.bm_lo, m1 = *env.bm_hi;
+        env.keys[slot] = kKeyEmpty;
+        uint32_t kv[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
+#pragma unroll
+        for (int j = 0; j < 8; j++) kv[j] = (uint32_t)j == sj ? kKeyEmpty : kv[j];
+        const uint32_t bmin = min8(kv);
+        *bm_entry(env, b) = bmin;
+        uint32_t mv[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+#pragma unroll
+        for (int i = 0; i < 8; i++) mv[i] = (uint32_t)i == b ? bmin : mv[i];
+        in.kmin = min8(mv);
+        in.mask &= ~(1ull << slot);
+        in.w--;
+        lane_push_slot(in, env, in.T, 2u * slot + (uint32_t)((in.gen >> slot) & 1ull), status);
+    } while ((in.kmin >> 6) == Kc);
     if (in.w > 0) {
         in.sw = (uint32_t)in.step[in.w - 1];
-        in.rsw = __frcp_rn((float)in.sw);
-        in.tc = in.T + (int64_t)nd * (int64_t)in.sw;
-        prefetch_l1(env.pay + 8 * nb + ((in.bslots >> (3 * nb)) & 7u));
+        in.rsw = rcp_approx((float)in.sw);
+        in.tc = in.T + (int64_t)((in.kmin >> 6) - Kc) * (int64_t)in.sw;
     }
 }
 
@@ -116,78 +227,125 @@ __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, St
 // observable depends on its clock until a slot frees, and later updates land on the same
 // step boundaries.
 __device__ __forceinline__ void lane_advance(LaneInst& in, int64_t now, bool drain, const LaneEnv& env,
-                                             Stats& st) {
+                                             uint32_t& status) {
     while (in.w > 0 && (drain || in.T < now)) {
         if (!drain && now <= in.tc - (int64_t)in.sw) {
             // the clock reaches `now` before anything completes
             if (in.w < in.B) {
-                // fewer than kfin <= 65535 steps: the quotient fits the fast exact division
+                // fewer steps than the longest request has tokens: the quotient fits the fast exact division
                 const uint32_t k = ceil_div_small(now - in.T, in.sw, in.rsw);
                 in.T += (int64_t)k * (int64_t)in.sw;
                 in.K += k;
             }
             break;
         }
-        in.K += (in.kmin - in.K) & 0xFFFFu;
+        in.K = in.kmin >> 6;
         in.T = in.tc;
-        lane_retire(in, env, st);
+        lane_retire(in, env, status);
     }
     if (!drain && in.w == 0 && in.T < now) in.T = now;  // an idle instance starts at once
 }
 
-// Distributor prediction for one instance (Sec. IV-F steps 2-3).  Returns the 64-bit
-// choice key (tier << 63 | predicted first-token time) or kKeyInf if the request cannot
-// meet its SLO there; t0 = time the request could start its prefill.  Limits: "no limit" is
-// passed as INT64_MAX here (all compared quantities are far below it).
-__device__ __forceinline__ uint64_t lane_predict(const LaneInst& in, const Request& q, int64_t pre,
-                                                 int64_t lim_ttft, int64_t lim_tbt, int64_t lim_e2e,
-                                                 bool optimistic, int64_t& t0) {
-    uint64_t tier;
-    int64_t sB = (int64_t)in.stepB;  // worst case F(M,P,B_I)
+// One request as the replay loop sees it (decoded from a prepared trace record).
+struct CookedReq {
+    int64_t arrival;
+    int64_t dl_ttft;   // latest first-token time that meets the TTFT limit
+    int64_t dl_e2e;    // latest finish time that meets the end-to-end limit
+    uint64_t rej;      // checksum term if it is rejected
+    uint32_t in_tokens;
+    uint32_t tbt32;    // TBT limit, 0xFFFFFFFF = none
+    uint32_t Sm1;      // output tokens - 1
+    uint32_t cls, model;
+};
+
+__device__ __forceinline__ CookedReq decode_cooked(const uint4& a, const uint4& b, const uint4& c) {
+    CookedReq q;
+    q.arrival = (int64_t)(((uint64_t)a.y << 32) | a.x);
+    q.dl_ttft = (int64_t)(((uint64_t)a.w << 32) | a.z);
+    q.dl_e2e = (int64_t)(((uint64_t)b.y << 32) | b.x);
+    q.in_tokens = b.z;
+    q.tbt32 = b.w;
+    q.rej = ((uint64_t)c.y << 32) | c.x;
+    q.Sm1 = c.z & 0xFFFFu;
+    q.cls = (c.z >> 16) & 0xFFu;
+    q.model = c.z >> 24;
+    return q;
+}
+
+constexpr uint32_t kOffSat = 0x7FFFFFFEu;  // predicted first token this far after `now` or further
+constexpr uint32_t kKey32Inf = 0xFFFFFFFFu;
+
+// Distributor prediction for one instance (Sec. IV-F steps 2-3).  Returns the 32-bit choice
+// key, tier << 31 | (predicted first-token time - now) clamped to kOffSat, or kKey32Inf if the
+// request cannot meet its SLO there; t0 = time the request could start its prefill, first =
+// predicted first-token time (never before `now`).
+__device__ __forceinline__ uint32_t lane_predict(const LaneInst& in, const CookedReq& q, int64_t pre, int64_t now,
+                                                 bool optimistic, int64_t& t0, int64_t& first) {
+    uint32_t tier;
+    uint32_t sB = in.stepB;  // worst case F(M,P,B_I)
     if (in.w < in.B) {
         tier = 0;
         t0 = in.T;
-        if (optimistic) sB = (int64_t)in.step[min(in.w + 1, in.B) - 1];
+        if (optimistic) sB = (uint32_t)in.step[min(in.w + 1, in.B) - 1];
     } else {
         tier = 1;
         t0 = in.tc;  // exact time its next slot frees
     }
-    const int64_t first = t0 + pre;
-    const int64_t fin = first + (int64_t)(q.S - 1) * sB;
-    const bool ok = first - q.arrival <= lim_ttft && (q.S == 1 || sB <= lim_tbt) && fin - q.arrival <= lim_e2e;
-    return ok ? ((tier << 63) | (uint64_t)first) : kKeyInf;
+    first = t0 + pre;
+    const int64_t fin = first + (int64_t)((uint64_t)q.Sm1 * sB);
+    const bool ok = first <= q.dl_ttft && (q.Sm1 == 0 || sB <= q.tbt32) && fin <= q.dl_e2e;
+    const uint64_t off = (uint64_t)(first - now);
+    const uint32_t o31 = off >= (uint64_t)kOffSat ? kOffSat : (uint32_t)off;
+    return ok ? ((tier << 31) | o31) : kKey32Inf;
+}
+
+// All live end indices move down by the current counter value `K` (the caller restarts the
+// counter at 0).  Returns the rebased smallest key.  Rare: kept out of line, arguments by value.
+__device__ __noinline__ uint32_t lane_rebase(uint32_t* keys, uint32_t nslots, uint4* bm_lo, uint4* bm_hi,
+                                             uint32_t K, uint32_t kmin) {
+    const uint32_t d = K << 6;
+    for (uint32_t s = 0; s < nslots; s++) {
+        const uint32_t k = keys[s];
+        if (k != kKeyEmpty) keys[s] = k - d;
+    }
+    for (uint32_t b = 0; b < 8; b++) {
+        uint32_t* e = reinterpret_cast<uint32_t*>(b < 4u ? bm_lo : bm_hi) + (b & 3u);
+        if (*e != kKeyEmpty) *e -= d;
+    }
+    return kmin != kKeyEmpty ? kmin - d : kmin;
 }
 
 // "map": prefill at the step boundary (running decodes stall), then occupy a free slot.
-__device__ __forceinline__ void lane_admit(LaneInst& in, const Request& q, uint32_t req, int64_t pre,
-                                           const LaneEnv& env, Stats& st) {
+__device__ __forceinline__ void lane_admit(LaneInst& in, const CookedReq& q, uint32_t req, int64_t pre,
+                                           const LaneEnv& env, uint32_t& status) {
     in.T += pre;
-    if (q.S == 1) {  // done at the end of its prefill, never occupies a slot
+    const uint4 pa = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)q.arrival,
+                                (uint32_t)((uint64_t)q.arrival >> 32));
+    const uint2 pb = make_uint2(req, (q.Sm1 + 1u) | (q.cls << 16));
+    if (q.Sm1 == 0) {  // done at the end of its prefill, never occupies a slot
         in.tc += pre;
-        if (account_completion(st, env.classes, env.inst_idx, req, q.arrival, in.T, in.T, 1, q.cls, env.dump))
-            env.hbc[q.cls < 7 ? q.cls : 7]++;
+        lane_push_now(in, env, in.T, pa, pb, status);
         return;
     }
-    const int slot = __ffsll((long long)~in.mask) - 1;
-    const int b = slot >> 3;
-    const uint32_t key = (in.K + q.S - 1) & 0xFFFFu;
-    const uint32_t dist = (key - in.K) & 0xFFFFu;
-    env.keys[slot] = (uint16_t)key;
-    store_payload(env.pay + slot, in.T, q.arrival, req, q.S, q.cls);
-    const uint32_t occ = (uint32_t)(in.mask >> (8 * b)) & 0xFFu;
-    if (occ == 0 || dist < (((uint32_t)env.keys[64 + b] - in.K) & 0xFFFFu)) {
-        env.keys[64 + b] = (uint16_t)key;
-        in.bslots = (in.bslots & ~(7u << (3 * b))) | ((uint32_t)(slot & 7) << (3 * b));
+    if (in.w == 0) in.K = 0;  // no live end index: the counter restarts
+    if (in.K + q.Sm1 > kRelMax) {
+        in.kmin = lane_rebase(env.keys, 8u * ((in.B + 7u) >> 3), env.bm_lo, env.bm_hi, in.K, in.kmin);
+        in.K = 0;
     }
-    if (in.w == 0 || dist < ((in.kmin - in.K) & 0xFFFFu)) {
-        in.kmin = key;
-        prefetch_l1(env.pay + slot);
-    }
+    const uint32_t slot = (uint32_t)(__ffsll((long long)~in.mask) - 1);
+    const uint32_t key = ((in.K + q.Sm1) << 6) | slot;
+    env.keys[slot] = key;
+    in.gen ^= 1ull << slot;
+    const uint32_t idx = 2u * slot + (uint32_t)((in.gen >> slot) & 1ull);
+    env.pay_a[idx] = pa;
+    env.pay_b[idx] = pb;
+    block_min_update(bm_entry(env, slot >> 3), key, env.keys_shared);
+    in.kmin = min(in.kmin, key);
     in.mask |= 1ull << slot;
     in.w++;
     in.sw = (uint32_t)in.step[in.w - 1];
-    in.rsw = __frcp_rn((float)in.sw);
-    in.tc = in.T + (int64_t)((in.kmin - in.K) & 0xFFFFu) * (int64_t)in.sw;
+    in.rsw = rcp_approx((float)in.sw);
+    in.tc = in.T + (int64_t)((in.kmin >> 6) - in.K) * (int64_t)in.sw;
 }
 
 }  // namespace maaso

@@ -12,8 +12,11 @@
 namespace maaso {
 cudaError_t launch_prep(const EvalParams& P, const uint32_t* dump_idx, cudaStream_t stream, int* launches);
 cudaError_t launch_rej_hash(uint64_t* out, uint32_t n);
-cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, cudaStream_t stream);
-int occupancy_eval_group(const EvalParams& P, int tile_recs);
+cudaError_t launch_cook_trace(const uint4* reqs, const int64_t* classes, uint4* out, uint32_t n);
+cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, int blocks_per_sm, int smem_per_sm,
+                              cudaStream_t stream);
+int occupancy_eval_group(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm);
+size_t group_scratch_per_lane();
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 cudaError_t launch_eval_block_reg(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 int occupancy_eval_block_reg(const EvalParams& P, int bucket, int tile_recs);
@@ -34,6 +37,7 @@ struct maaso_trace {
     uint4* d_reqs;
     int64_t* d_classes;
     uint64_t* d_rej_hash;
+    uint4* d_cooked;  // prepared records for the lane-group kernel
     uint64_t n;
     uint32_t n_classes;
     uint32_t max_model;
@@ -63,6 +67,8 @@ struct maaso_ctx {
     cudaStream_t own_stream;
     uint64_t launches;
     int tile_recs;
+    int group_blocks;  // blocks of the lane-group kernel per SM its key pool is sized for; 0 = by batch size
+    int smem_per_sm;
     int promote_pct;  // share of the spare resident warps the planner may use for promotions
     bool timing;
     cudaEvent_t ev[6];   // eval: start, after prep, after group, after block; topk: start, end
@@ -130,7 +136,8 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
     ctx->scratch = ctx->topk_scratch = ctx->stage = ctx->deploy = nullptr;
     ctx->scratch_bytes = ctx->topk_scratch_bytes = ctx->stage_bytes = ctx->deploy_bytes = 0;
     ctx->launches = 0;
-    ctx->tile_recs = 256;
+    ctx->tile_recs = 64;
+    ctx->group_blocks = 0;
     ctx->own_stream = nullptr;
     ctx->timing = false;
     ctx->ev_eval = ctx->ev_topk = false;
@@ -147,6 +154,7 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
         return MAASO_ESTATE;
     }
     ctx->sm_count = prop.multiProcessorCount;
+    ctx->smem_per_sm = (int)prop.sharedMemPerMultiprocessor;
     e = cudaStreamCreateWithFlags(&ctx->own_stream, cudaStreamNonBlocking);
     if (e != cudaSuccess) {
         delete ctx;
@@ -161,7 +169,13 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
     const char* env = getenv("MAASO_TILE_RECS");
     if (env) {
         int v = atoi(env);
-        if (v >= 16 && v <= 2048) ctx->tile_recs = v;
+        if (v >= 16 && v <= 2048) ctx->tile_recs = v & ~1;  // even: tiles of 8-byte terms stay 16-byte aligned
+    }
+
+    const char* gb = getenv("MAASO_GROUP_BLOCKS");
+    if (gb) {
+        int v = atoi(gb);
+        if (v >= 0 && v <= 8) ctx->group_blocks = v;
     }
     *out = ctx;
     return MAASO_OK;
@@ -179,6 +193,7 @@ MAASO_API void maaso_free_trace(maaso_ctx* ctx, maaso_trace* trace) {
     if (trace->d_reqs) cudaFree(trace->d_reqs);
     if (trace->d_classes) cudaFree(trace->d_classes);
     if (trace->d_rej_hash) cudaFree(trace->d_rej_hash);
+    if (trace->d_cooked) cudaFree(trace->d_cooked);
     delete trace;
 }
 
@@ -302,19 +317,24 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     t->d_reqs = nullptr;
     t->d_classes = nullptr;
     t->d_rej_hash = nullptr;
+    t->d_cooked = nullptr;
     t->n = n;
     t->n_classes = n_classes;
     t->max_model = max_model;
     cudaError_t e = cudaMalloc(&t->d_reqs, (n ? n : 1) * sizeof(maaso_request));
     if (e == cudaSuccess) e = cudaMalloc(&t->d_classes, cls.size() * 8);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_rej_hash, (n ? n : 1) * 8);
+    if (e == cudaSuccess) e = cudaMalloc(&t->d_cooked, (n ? n : 1) * 16 * kCookedWords);
     if (e == cudaSuccess) e = launch_rej_hash(t->d_rej_hash, (uint32_t)n);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e == cudaSuccess && n)
         e = cudaMemcpy(t->d_reqs, reqs, n * sizeof(maaso_request),
                        on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(t->d_classes, cls.data(), cls.size() * 8, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = launch_cook_trace(t->d_reqs, t->d_classes, t->d_cooked, (uint32_t)n);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
+        if (t->d_cooked) cudaFree(t->d_cooked);
         if (t->d_reqs) cudaFree(t->d_reqs);
         if (t->d_classes) cudaFree(t->d_classes);
         if (t->d_rej_hash) cudaFree(t->d_rej_hash);
@@ -356,6 +376,7 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.n_classes = trace->n_classes;
     P.classes = trace->d_classes;
     P.rej_hash = trace->d_rej_hash;
+    P.cooked = trace->d_cooked;
     P.rows = ctx->d_rows;
     P.devices = ctx->d_devices;
     P.min_devices = ctx->d_min_devices;
@@ -380,12 +401,22 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.rej_by_model = o.rejected_by_model;
 
     // launch shapes: persistent grids bounded by what the batch can use
-    const int occ_g = occupancy_eval_group(P, tile);
+    // Blocks per SM of the lane-group kernel.  A batch that three blocks per SM can hold in one
+    // wave is bound by its longest dependent chains, which run faster with fewer warps sharing a
+    // scheduler; a larger batch is bound by instruction issue and wants all four.  Lanes needed
+    // ~ instances x 1.3 (group widths are powers of two).
+    int group_blocks = ctx->group_blocks;
+    if (group_blocks == 0) {
+        const uint64_t est_warps = (cands->n_inst * 13 / 10 + 31) / 32 + 6;
+        group_blocks = est_warps <= (uint64_t)ctx->sm_count * 3 * (kGroupThreads / 32) ? 3 : 4;
+    }
+    const int occ_g = occupancy_eval_group(P, tile, group_blocks, ctx->smem_per_sm);
     int grid_g = ctx->sm_count * occ_g;
     const uint64_t max_items_g = (uint64_t)C / 4 + 6;  // at most one work item per 4 candidates + bucket tails
     if ((uint64_t)grid_g > max_items_g) grid_g = (int)max_items_g;
     int grid_b[4];
-    size_t pay_entries = (size_t)grid_g * kGroupThreads * MAASO_WMAX;
+    size_t pay_entries = (size_t)grid_g * kGroupThreads * (group_scratch_per_lane() / sizeof(Payload));
+    static_assert(sizeof(Payload) == 32, "scratch is counted in 32-byte entries");
     for (int b = 6; b <= kGenericBlockBucket; b++) {
         // without the block mapping only candidates with more than 32 instances go to a block kernel
         const bool used = o.mapping == MAASO_MAP_BLOCK || (b == kGenericBlockBucket && cands->n_inst > 32);
@@ -431,7 +462,7 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     if (e != cudaSuccess) return cuda_fail(ctx, e, "prep launch");
     if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
     if (o.mapping != MAASO_MAP_BLOCK) {
-        e = launch_eval_group(P, grid_g, tile, stream);
+        e = launch_eval_group(P, grid_g, tile, group_blocks, ctx->smem_per_sm, stream);
         launches++;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "group kernel launch");
     }

@@ -134,6 +134,28 @@ __global__ void rej_hash_kernel(uint64_t* out, uint32_t n) {
     const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r < n) out[r] = rejected_hash(r);
 }
+// Prepared trace records for the lane-group kernel (layout: common.cuh).
+__global__ void cook_trace_kernel(const uint4* reqs, const int64_t* classes, uint4* out, uint32_t n) {
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n) return;
+    const Request q = decode_request(reqs[r]);
+    const int64_t l_ttft = classes[q.cls * 3 + 0], l_tbt = classes[q.cls * 3 + 1], l_e2e = classes[q.cls * 3 + 2];
+    const int64_t dl_ttft = l_ttft < 0 ? INT64_MAX : q.arrival + l_ttft;
+    const int64_t dl_e2e = l_e2e < 0 ? INT64_MAX : q.arrival + l_e2e;
+    const uint32_t tbt32 = (l_tbt < 0 || l_tbt > 0xFFFFFFFFll) ? 0xFFFFFFFFu : (uint32_t)l_tbt;
+    const uint64_t h = rejected_hash(r);
+    auto lo = [](uint64_t v) { return (uint32_t)v; };
+    auto hi = [](uint64_t v) { return (uint32_t)(v >> 32); };
+    uint4* o = out + (size_t)r * kCookedWords;
+    o[0] = make_uint4(lo((uint64_t)q.arrival), hi((uint64_t)q.arrival), lo((uint64_t)dl_ttft), hi((uint64_t)dl_ttft));
+    o[1] = make_uint4(lo((uint64_t)dl_e2e), hi((uint64_t)dl_e2e), q.in_tokens, tbt32);
+    o[2] = make_uint4(lo(h), hi(h), (q.S - 1u) | (q.cls << 16) | (q.model << 24), 0u);
+}
+cudaError_t launch_cook_trace(const uint4* reqs, const int64_t* classes, uint4* out, uint32_t n) {
+    if (n) cook_trace_kernel<<<(n + 255) / 256, 256>>>(reqs, classes, out, n);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_rej_hash(uint64_t* out, uint32_t n) {
     if (n) rej_hash_kernel<<<(n + 255) / 256, 256>>>(out, n);
     return cudaGetLastError();
