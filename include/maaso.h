@@ -44,6 +44,7 @@ extern "C" {
 #define MAASO_MAX_CLASSES 256
 #define MAASO_MAX_STEP_US (1 << 30)
 #define MAASO_MAX_TOPK 1024
+#define MAASO_TTFT_BINS 64     /* bins of the optional time-to-first-token histogram */
 
 /* return codes */
 #define MAASO_OK 0
@@ -141,6 +142,12 @@ typedef struct {
     int32_t *dump_inst;
     uint32_t *rejected_by_model; /* device, [n_cand][MAASO_MAX_MODELS] or NULL: requests of each model
                                     the placement left unserved (R_res of Alg. 1); zero for invalid ones */
+    uint32_t *ttft_hist;         /* device, [n_cand][MAASO_TTFT_BINS] or NULL: histogram of the time to
+                                    first token of the served requests (the "response latency" of
+                                    Sec. V-A), overwritten by the call.  Bin 0 holds t < 1024 us; for
+                                    t >= 1024 with e = floor(log2 t) and h = the bit below the leading
+                                    one, bin = min(63, 1 + 2 (e - 10) + h): two bins per octave.
+                                    All zero for an invalid candidate. */
 } maaso_eval_opts;
 
 /* Per-candidate result (128 bytes).  Statistics are over served requests unless noted. */
@@ -191,7 +198,8 @@ MAASO_API int maaso_eval_placements(maaso_ctx *ctx, const maaso_trace *trace, co
 
 /* Same scoring with HOST buffers: copies the candidate batch to the device, scores it,
  * copies the records back into out_results (host, [n_cand]) and synchronises.  Dump
- * buffers are not supported here (opts->dump_n must be 0). */
+ * buffers, per-model counts and histograms are not supported here (opts->dump_n must be 0,
+ * opts->rejected_by_model and opts->ttft_hist NULL). */
 MAASO_API int maaso_eval_placements_host(maaso_ctx *ctx, const maaso_trace *trace, const maaso_cand_batch *cands,
                                const maaso_eval_opts *opts, maaso_result *out_results);
 
@@ -217,6 +225,16 @@ MAASO_API int maaso_topk(maaso_ctx *ctx, const maaso_result *results, uint64_t n
 typedef struct {
     double alpha, beta, gamma_t, gamma_l;
 } maaso_score_params;
+
+/* Latency percentiles from the histograms maaso_eval_placements filled (opts.ttft_hist): for
+ * every candidate c and every requested rank permille[j] (1..1000, host array, n_p <= 16),
+ * out[c * n_p + j] (device, int64) = the upper edge in microseconds of the first bin at which the
+ * cumulative count reaches ceil(permille[j] * served / 1000), i.e. an upper bound of that
+ * percentile that is tight to a factor 1.5; INT64_MAX if it falls in the open last bin, -1 if
+ * the candidate served nothing.  The paper reports the mean response latency only (Sec. V-A);
+ * tail percentiles are an addition for comparing placements.  Enqueued on cuda_stream. */
+MAASO_API int maaso_ttft_percentiles(maaso_ctx *ctx, const uint32_t *ttft_hist, uint64_t n_cand,
+                                     const uint32_t *permille, uint32_t n_p, int64_t *out, void *cuda_stream);
 MAASO_API int maaso_score(maaso_ctx *ctx, const maaso_result *results, uint64_t n_cand,
                           const maaso_score_params *params, double *out_scores, void *cuda_stream);
 

@@ -4,8 +4,8 @@ Only tests, the smoke check and the benchmark's CPU-baseline leg import this pac
 It compiles oracle/maaso_oracle.c with gcc on first use and calls it through ctypes;
 it imports nothing from the CUDA package.
 """
-from .binding import (build, eval_placements, eval_placements_parallel, topk, score, topk_scores, rejected_by_model, ins_deploy, partition, prune_configs,
+from .binding import (build, eval_placements, eval_placements_parallel, topk, score, topk_scores, rejected_by_model, ins_deploy, partition, prune_configs, ttft_hist, ttft_percentiles,
                       FLAG_PRED_OPTIMISTIC, STATUS)
 
-__all__ = ["build", "eval_placements", "eval_placements_parallel", "topk", "score", "topk_scores", "rejected_by_model", "ins_deploy", "partition", "prune_configs",
+__all__ = ["build", "eval_placements", "eval_placements_parallel", "topk", "score", "topk_scores", "rejected_by_model", "ins_deploy", "partition", "prune_configs", "ttft_hist", "ttft_percentiles",
            "FLAG_PRED_OPTIMISTIC", "STATUS"]

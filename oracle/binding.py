@@ -55,6 +55,8 @@ def _load():
         _lib.orc_ins_deploy.restype = C.c_int
         _lib.orc_partition.restype = C.c_int
         _lib.orc_prune_configs.restype = C.c_int
+        _lib.orc_ttft_hist.restype = C.c_int
+        _lib.orc_ttft_percentile.restype = C.c_int64
     return _lib
 
 
@@ -187,6 +189,38 @@ def rejected_by_model(profile, trace, classes, offsets, inst, budget, class_mask
     if rc != 0:
         raise RuntimeError(f"oracle rejected_by_model failed with code {rc}")
     del keep
+    return out
+
+
+def ttft_hist(profile, trace, classes, offsets, inst, budget, class_mask=None, flags=0):
+    """[n_cand][64] histogram of the time to first token of the served requests (see orc_ttft_hist)."""
+    lib = _load()
+    p, keep = _profile_struct(profile)
+    trace = np.ascontiguousarray(trace, dtype=_REQ)
+    classes = np.ascontiguousarray(classes, dtype=_SLO)
+    offsets = np.ascontiguousarray(offsets, dtype=np.uint32)
+    inst = np.ascontiguousarray(inst, dtype=np.uint32)
+    if inst.size == 0:
+        inst = np.zeros(1, dtype=np.uint32)
+    mask = None if class_mask is None else np.ascontiguousarray(class_mask, dtype=np.uint32)
+    out = np.zeros((len(offsets) - 1, 64), dtype=np.uint32)
+    rc = lib.orc_ttft_hist(C.byref(p), _ptr(trace), C.c_uint64(len(trace)), _ptr(classes),
+                           C.c_uint32(len(classes)), _ptr(offsets), _ptr(inst), _ptr(mask),
+                           C.c_uint64(len(offsets) - 1), C.c_uint32(budget), C.c_uint32(flags), _ptr(out))
+    if rc != 0:
+        raise RuntimeError(f"oracle ttft_hist failed with code {rc}")
+    del keep
+    return out
+
+
+def ttft_percentiles(hist, permille):
+    """[n_cand][len(permille)] upper bounds in microseconds (see orc_ttft_percentile)."""
+    lib = _load()
+    hist = np.ascontiguousarray(hist, dtype=np.uint32).reshape(-1, 64)
+    out = np.zeros((len(hist), len(permille)), dtype=np.int64)
+    for c in range(len(hist)):
+        for j, pm in enumerate(permille):
+            out[c, j] = lib.orc_ttft_percentile(_ptr(hist[c]), C.c_uint32(int(pm)))
     return out
 
 

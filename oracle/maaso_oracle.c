@@ -420,6 +420,67 @@ int orc_rejected_by_model(const orc_profile *p, const orc_request *reqs, uint64_
 }
 
 /*
+ * Histogram of the time to first token ("response latency", Sec. V-A "Evaluation Metrics")
+ * of the requests a candidate served, for tail percentiles.  The paper reports the mean
+ * only; the bins are this library's definition: bin 0 holds t < 1024 us; for t >= 1024,
+ * with e = floor(log2 t) and h = the bit of t just below its leading one, the bin is
+ * 1 + 2 (e - 10) + h, capped at 63 (two bins per octave, the last one open).
+ * Computed from the per-request first-token times, out[c][64].
+ */
+static uint32_t orc_ttft_bin(int64_t t) {
+    if (t < 1024) return 0;
+    int e = 0;
+    while ((t >> (e + 1)) != 0) e++;   /* floor(log2 t) */
+    uint32_t h = (uint32_t)((t >> (e - 1)) & 1);
+    uint32_t b = 1u + 2u * (uint32_t)(e - 10) + h;
+    return b > 63u ? 63u : b;
+}
+
+int orc_ttft_hist(const orc_profile *p, const orc_request *reqs, uint64_t n, const orc_slo *classes,
+                  uint32_t n_classes, const uint32_t *offsets, const uint32_t *inst,
+                  const uint32_t *class_mask, uint64_t n_cand, uint32_t budget, uint32_t flags,
+                  uint32_t *out) {
+    int64_t *first = (int64_t *)malloc((n ? n : 1) * sizeof(int64_t));
+    if (!first) return -1;
+    for (uint64_t c = 0; c < n_cand; c++) {
+        orc_result r;
+        int rc = orc_eval_candidate(p, reqs, n, classes, n_classes, inst + offsets[c], offsets[c + 1] - offsets[c],
+                                    class_mask != NULL, class_mask ? class_mask[c] : 0, budget, flags, &r, NULL,
+                                    first, NULL);
+        if (rc) { free(first); return rc; }
+        for (int b = 0; b < 64; b++) out[c * 64 + b] = 0;
+        if (r.status != 0) continue;
+        for (uint64_t q = 0; q < n; q++)
+            if (first[q] >= 0) out[c * 64 + orc_ttft_bin(first[q] - reqs[q].arrival_us)]++;
+    }
+    free(first);
+    return 0;
+}
+
+/* Upper bound of the `permille`-th rank (1..1000) of one 64-bin histogram: the largest value
+ * of the first bin at which the cumulative count reaches ceil(permille * total / 1000);
+ * INT64_MAX in the open last bin, -1 for an empty histogram. */
+int64_t orc_ttft_percentile(const uint32_t *hist, uint32_t permille) {
+    uint64_t total = 0;
+    for (int b = 0; b < 64; b++) total += hist[b];
+    if (total == 0) return -1;
+    uint64_t target = ((uint64_t)permille * total + 999) / 1000;
+    if (target < 1) target = 1;
+    uint64_t cum = 0;
+    for (int b = 0; b < 64; b++) {
+        cum += hist[b];
+        if (cum >= target) {
+            if (b == 0) return 1023;
+            if (b == 63) return INT64_MAX;
+            int e = 10 + (b - 1) / 2, h = (b - 1) & 1;
+            /* bin b covers [2^e + h 2^(e-1), 2^e + (h+1) 2^(e-1) - 1] */
+            return ((int64_t)1 << e) + (int64_t)(h + 1) * ((int64_t)1 << (e - 1)) - 1;
+        }
+    }
+    return INT64_MAX;
+}
+
+/*
  * Alg. 1, "Simulator-Based Instance Configuration", taken literally.  For every configuration
  * (P, B) of the (already pruned) list: start from the empty placement; while GPUs remain and
  * some model is not saturated, add an instance (m', P, B) of the model m' with the most

@@ -49,7 +49,8 @@ class _CandBatch(C.Structure):
 class _EvalOpts(C.Structure):
     _fields_ = [("flags", C.c_uint32), ("mapping", C.c_uint32), ("dump_n", C.c_uint32),
                 ("reserved", C.c_uint32), ("dump_cand_idx", C.c_void_p), ("dump_finish_us", C.c_void_p),
-                ("dump_first_us", C.c_void_p), ("dump_inst", C.c_void_p), ("rejected_by_model", C.c_void_p)]
+                ("dump_first_us", C.c_void_p), ("dump_inst", C.c_void_p), ("rejected_by_model", C.c_void_p),
+                ("ttft_hist", C.c_void_p)]
 
 
 class _ScoreParams(C.Structure):
@@ -83,6 +84,8 @@ def _load():
     lib.maaso_topk.argtypes = [vp, vp, u64, u32, u32, vp, vp, vp]
     lib.maaso_score.argtypes = [vp, vp, u64, C.POINTER(_ScoreParams), vp, vp]
     lib.maaso_topk_scores.argtypes = [vp, vp, vp, u64, u32, vp, vp, vp]
+    lib.maaso_ttft_percentiles.argtypes = [vp, vp, u64, vp, u32, vp, vp]
+    lib.maaso_ttft_percentiles.restype = C.c_int
     lib.maaso_ins_deploy.argtypes = [vp, vp, u32, vp, u32, C.c_int, u32, C.POINTER(_ScoreParams), u32, vp, vp, vp]
     lib.maaso_ins_deploy.restype = C.c_int
     lib.maaso_prune_configs.argtypes = [vp, vp, C.c_int, u32, vp, u32, u32, vp, C.POINTER(u32)]
@@ -195,13 +198,13 @@ def _batch(offsets, inst, class_mask, budget):
 
 def maaso_eval_placements(ctx, trace, offsets, inst, budget, out_results, class_mask=None, flags=0,
                           mapping=MAP_AUTO, dump_cand_idx=None, dump_finish_us=None, dump_first_us=None,
-                          dump_inst=None, rejected_by_model=None, stream=None):
+                          dump_inst=None, rejected_by_model=None, ttft_hist=None, stream=None):
     """All array arguments are CUDA tensors (int32 views of the uint32 words; out_results a
     uint8 tensor of n_cand*128 bytes).  Work is enqueued on `stream` (default: torch's current)."""
     b = _batch(offsets, inst, class_mask, budget)
     o = _EvalOpts(int(flags), int(mapping), 0 if dump_cand_idx is None else int(dump_cand_idx.shape[0]), 0,
                   _ptr(dump_cand_idx), _ptr(dump_finish_us), _ptr(dump_first_us), _ptr(dump_inst),
-                  _ptr(rejected_by_model))
+                  _ptr(rejected_by_model), _ptr(ttft_hist))
     _check(_lib.maaso_eval_placements(ctx, trace, C.byref(b), C.byref(o), _ptr(out_results),
                                       _stream_ptr(stream)), "maaso_eval_placements", ctx)
 
@@ -210,7 +213,7 @@ def maaso_eval_placements_host(ctx, trace, offsets, inst, budget, out_results, c
                                mapping=MAP_AUTO):
     """Host (numpy) buffers in and out; copies happen inside the call, which synchronises."""
     b = _batch(offsets, inst, class_mask, budget)
-    o = _EvalOpts(int(flags), int(mapping), 0, 0, None, None, None, None, None)
+    o = _EvalOpts(int(flags), int(mapping), 0, 0, None, None, None, None, None, None)
     _check(_lib.maaso_eval_placements_host(ctx, trace, C.byref(b), C.byref(o), _ptr(out_results)),
            "maaso_eval_placements_host", ctx)
 
@@ -224,6 +227,12 @@ def maaso_score(ctx, results, n_cand, alpha, beta, gamma_t, gamma_l, out_scores,
     p = _ScoreParams(float(alpha), float(beta), float(gamma_t), float(gamma_l))
     _check(_lib.maaso_score(ctx, _ptr(results), int(n_cand), C.byref(p), _ptr(out_scores), _stream_ptr(stream)),
            "maaso_score", ctx)
+
+
+def maaso_ttft_percentiles(ctx, ttft_hist, n_cand, permille, out, stream=None):
+    pm = np.ascontiguousarray(permille, dtype=np.uint32)
+    _check(_lib.maaso_ttft_percentiles(ctx, _ptr(ttft_hist), int(n_cand), pm.ctypes.data, len(pm), _ptr(out),
+                                       _stream_ptr(stream)), "maaso_ttft_percentiles", ctx)
 
 
 def maaso_topk_scores(ctx, results, scores, n_cand, k, out_idx, out_res=None, stream=None):
@@ -355,7 +364,7 @@ class Context:
                                 class_mask, flags)
 
     def eval_placements(self, trace, offsets, inst, budget, class_mask=None, flags=0, mapping=MAP_AUTO,
-                        dump_idx=None, out=None, stream=None, rejected_by_model=None):
+                        dump_idx=None, out=None, stream=None, rejected_by_model=None, ttft_hist=None):
         """offsets / inst / class_mask: CUDA int32 tensors (see to_device).  Returns the uint8
         result tensor [n_cand, 128] and, if dump_idx is given, a dict of dump tensors."""
         torch = self.torch
@@ -372,7 +381,8 @@ class Context:
             kw = dict(dump_cand_idx=d, dump_finish_us=dumps["finish_us"], dump_first_us=dumps["first_us"],
                       dump_inst=dumps["inst"])
         maaso_eval_placements(self.handle, trace.handle, offsets, inst, budget, out, class_mask, flags,
-                              mapping, stream=stream, rejected_by_model=rejected_by_model, **kw)
+                              mapping, stream=stream, rejected_by_model=rejected_by_model, ttft_hist=ttft_hist,
+                              **kw)
         return (out, dumps) if dump_idx is not None else out
 
     def eval_placements_host(self, trace, offsets, inst, budget, class_mask=None, flags=0,
@@ -398,6 +408,14 @@ class Context:
     def score(self, results, alpha, beta, gamma_t, gamma_l, stream=None):
         out = self.torch.empty(int(results.shape[0]), dtype=self.torch.float64, device=self.device)
         maaso_score(self.handle, results, int(results.shape[0]), alpha, beta, gamma_t, gamma_l, out, stream)
+        return out
+
+    def ttft_percentiles(self, ttft_hist, permille, stream=None):
+        """ttft_hist: int32 CUDA tensor [n_cand, 64] filled by eval_placements(ttft_hist=...).
+        Returns an int64 tensor [n_cand, len(permille)] of bin upper edges in microseconds."""
+        n_cand = int(ttft_hist.shape[0])
+        out = self.torch.empty((n_cand, len(permille)), dtype=self.torch.int64, device=self.device)
+        maaso_ttft_percentiles(self.handle, ttft_hist, n_cand, permille, out, stream)
         return out
 
     def topk_scores(self, results, scores, k, with_records=True, stream=None):

@@ -101,7 +101,16 @@ struct Dump {
     int64_t* finish;
     int64_t* first;
     int32_t* inst;
+    uint32_t* hist;  // this candidate's time-to-first-token histogram, or null
 };
+
+// Histogram bin of a time to first token: bin 0 below 1024 us, then two bins per octave.
+__device__ __forceinline__ uint32_t ttft_bin(int64_t t) {
+    if (t < 1024) return 0;
+    const int e = 63 - __clzll(t);
+    const uint32_t b = 1u + 2u * (uint32_t)(e - 10) + (uint32_t)((t >> (e - 1)) & 1);
+    return b > (uint32_t)(MAASO_TTFT_BINS - 1) ? (uint32_t)(MAASO_TTFT_BINS - 1) : b;
+}
 
 // A request leaves the system served at t_fin (Phi_S indicator and the latency / throughput sums).
 // `classes` holds (ttft, tbt, e2e) per class, negative = no limit.  Returns whether it was a hit.
@@ -126,6 +135,7 @@ __device__ __forceinline__ bool account_completion(Stats& st, const int64_t* cla
     if (dump.finish) dump.finish[req] = t_fin;
     if (dump.first) dump.first[req] = first_tok;
     if (dump.inst) dump.inst[req] = (int32_t)inst;
+    if (dump.hist) atomicAdd(dump.hist + ttft_bin(ttft), 1u);
     return hit;
 }
 
@@ -243,10 +253,12 @@ struct EvalParams {
     int32_t* dump_inst;
     Payload* payload;        // scratch for running requests
     uint32_t* rej_by_model;  // [n_cand][MAASO_MAX_MODELS] or null
+    uint32_t* ttft_hist;     // [n_cand][MAASO_TTFT_BINS] or null (zeroed before the kernels run)
 };
 
 __device__ __forceinline__ Dump dump_for(const EvalParams& P, uint32_t cand) {
-    Dump d{nullptr, nullptr, nullptr};
+    Dump d{nullptr, nullptr, nullptr, nullptr};
+    if (P.ttft_hist) d.hist = P.ttft_hist + (size_t)cand * MAASO_TTFT_BINS;
     if (P.dump_row) {
         int32_t row = P.dump_row[cand];
         if (row >= 0) {

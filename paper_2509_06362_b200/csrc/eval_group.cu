@@ -256,7 +256,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         }
         const bool warp_has_work = __any_sync(kFullMask, valid);
         const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
-        Dump dump{nullptr, nullptr, nullptr};
+        Dump dump{nullptr, nullptr, nullptr, nullptr};
         if (valid) dump = dump_for(P, cand);
         // per-request side outputs (dump rows, per-model rejection counts) are rare: one flag guards them
         const bool side = dump.finish || dump.first || dump.inst || P.rej_by_model;
@@ -295,9 +295,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                     nx0 = nx[0]; nx1 = nx[1]; nx2 = nx[2];
                 }
                 // statistics of completed requests: every fourth request, if some lane's queue is half full
-                if ((ri & 3u) == 3u && __any_sync(kFullMask, in.qn >= (uint32_t)(kQueue / 2))) {
+                if ((ri & 3u) == 3u && __any_sync(kFullMask, in.qn >= (uint32_t)kFlushAt)) {
                     flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first,
-                                dump.inst);
+                                dump.inst, dump.hist);
                     in.qn = 0;
                 }
                 // All 32 lanes walk the trace together and every warp-level operation below uses
@@ -385,11 +385,13 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
 
         // drain, account what is still queued, reduce over the group, write the record
         __syncwarp();
-        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first, dump.inst);
+        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first, dump.inst,
+                    dump.hist);
         in.qn = 0;
         if (has && status == 0) lane_advance(in, 0, true, env, status);
         __syncwarp();
-        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first, dump.inst);
+        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first, dump.inst,
+                    dump.hist);
         in.qn = 0;
         Stats st = ls.st;
         st.checksum += rej_sum;

@@ -30,7 +30,14 @@ namespace maaso {
 constexpr uint32_t kKeyEmpty = 0xFFFFFFFFu;
 constexpr uint32_t kRelMax = (1u << 26) - 2u;  // largest end index a key can hold
 constexpr int kKeyUnitBytes = 32;              // pool unit: one block of 8 keys (or the 8 block minima)
-constexpr int kQueue = 4;                      // queued completions per lane in shared memory
+#ifndef MAASO_QUEUE
+#define MAASO_QUEUE 4
+#endif
+#ifndef MAASO_FLUSH_AT
+#define MAASO_FLUSH_AT 3
+#endif
+constexpr int kQueue = MAASO_QUEUE;            // queued completions per lane in shared memory
+constexpr int kFlushAt = MAASO_FLUSH_AT;       // the warp accounts its queues once some lane holds this many
 constexpr int kQueueOvf = 72;                  // further entries per lane in global scratch
 // Per-lane global scratch: payload A [64 slots][2] x 16 B, payload B [64][2] x 8 B, queue
 // overflow x 32 B, and room for 64 keys + 8 block minima if the shared-memory pool is full.
@@ -157,11 +164,11 @@ __device__ __forceinline__ void lane_push_now(LaneInst& in, const LaneEnv& env, 
 __device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
                                          const unsigned char* ovf, uint32_t n, const int64_t* classes,
                                          uint32_t inst_idx, int64_t* dump_finish, int64_t* dump_first,
-                                         int32_t* dump_inst) {
+                                         int32_t* dump_inst, uint32_t* hist) {
     async_copies_done();
     Stats st = ls->st;
-    const Dump no_dump{nullptr, nullptr, nullptr};
-    const bool dumping = dump_finish || dump_first || dump_inst;
+    const Dump no_dump{nullptr, nullptr, nullptr, nullptr};
+    const bool dumping = dump_finish || dump_first || dump_inst || hist;
     for (uint32_t j = 0; j < n; j++) {
         int64_t t_fin;
         uint4 a;
@@ -186,6 +193,7 @@ __device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const
             if (dump_finish) dump_finish[b.x] = t_fin;
             if (dump_first) dump_first[b.x] = first;
             if (dump_inst) dump_inst[b.x] = (int32_t)inst_idx;
+            if (hist) atomicAdd(hist + ttft_bin(first - arrival), 1u);
         }
     }
     ls->st = st;

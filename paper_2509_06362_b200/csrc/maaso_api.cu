@@ -28,6 +28,8 @@ cudaError_t launch_topk(const maaso_result* results, uint64_t n_cand, uint32_t k
                         const double* scores);
 cudaError_t launch_score(const maaso_result* res, uint64_t n, const maaso_score_params& p, double* out,
                          cudaStream_t stream);
+cudaError_t launch_ttft_percentiles(const uint32_t* hist, uint64_t n, const uint32_t* permille, uint32_t n_p,
+                                    int64_t* out, cudaStream_t stream);
 }  // namespace maaso
 
 using namespace maaso;
@@ -399,6 +401,7 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.dump_first = o.dump_first_us;
     P.dump_inst = o.dump_inst;
     P.rej_by_model = o.rejected_by_model;
+    P.ttft_hist = o.ttft_hist;
 
     // launch shapes: persistent grids bounded by what the batch can use
     // Blocks per SM of the lane-group kernel.  A batch that three blocks per SM can hold in one
@@ -455,6 +458,7 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.group_warps = (uint32_t)grid_g * (kGroupThreads / 32);
     P.promote_pct = (uint32_t)ctx->promote_pct;
     cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, kCounterWords * 4, stream);
+    if (e == cudaSuccess && o.ttft_hist) e = cudaMemsetAsync(o.ttft_hist, 0, (size_t)C * MAASO_TTFT_BINS * 4, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "memset");
     int launches = 0;
     if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
@@ -485,7 +489,8 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
 MAASO_API int maaso_eval_placements_host(maaso_ctx* ctx, const maaso_trace* trace, const maaso_cand_batch* cands,
                                const maaso_eval_opts* opts, maaso_result* out_results) {
     if (!ctx || !trace || !cands) return MAASO_EINVAL;
-    if (opts && opts->dump_n) return fail(ctx, MAASO_EINVAL, "eval_host: dump buffers are not supported");
+    if (opts && (opts->dump_n || opts->rejected_by_model || opts->ttft_hist))
+        return fail(ctx, MAASO_EINVAL, "eval_host: dump buffers, per-model counts and histograms are not supported");
     if (cands->n_cand == 0) return MAASO_OK;
     if (!cands->offsets || !out_results || (cands->n_inst && !cands->inst) || cands->n_cand >= 0xFFFFFFFFull ||
         cands->n_inst >= 0xFFFFFFFFull)
@@ -551,6 +556,20 @@ MAASO_API int maaso_score(maaso_ctx* ctx, const maaso_result* results, uint64_t 
     cudaError_t e = launch_score(results, n_cand, *params, out_scores, (cudaStream_t)cuda_stream);
     ctx->launches++;
     if (e != cudaSuccess) return cuda_fail(ctx, e, "score launch");
+    return MAASO_OK;
+}
+
+MAASO_API int maaso_ttft_percentiles(maaso_ctx* ctx, const uint32_t* ttft_hist, uint64_t n_cand,
+                                     const uint32_t* permille, uint32_t n_p, int64_t* out, void* cuda_stream) {
+    if (!ctx) return MAASO_EINVAL;
+    if (n_cand == 0 || n_p == 0) return MAASO_OK;
+    if (!ttft_hist || !permille || !out || n_p > 16) return fail(ctx, MAASO_EINVAL, "percentiles: null pointer or more than 16 ranks");
+    for (uint32_t j = 0; j < n_p; j++)
+        if (permille[j] < 1 || permille[j] > 1000) return fail(ctx, MAASO_EINVAL, "percentiles: rank outside 1..1000");
+    DeviceGuard g(ctx->device);
+    cudaError_t e = launch_ttft_percentiles(ttft_hist, n_cand, permille, n_p, out, (cudaStream_t)cuda_stream);
+    ctx->launches++;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "percentile launch");
     return MAASO_OK;
 }
 

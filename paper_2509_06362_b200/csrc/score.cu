@@ -41,4 +41,46 @@ cudaError_t launch_score(const maaso_result* res, uint64_t n, const maaso_score_
     return cudaGetLastError();
 }
 
+// Upper edge (microseconds) of a histogram bin of ttft_bin; the last bin is open.
+__device__ __forceinline__ int64_t ttft_bin_upper(uint32_t b) {
+    if (b == 0) return 1023;
+    if (b >= (uint32_t)(MAASO_TTFT_BINS - 1)) return INT64_MAX;
+    const uint32_t e = 10u + (b - 1u) / 2u, h = (b - 1u) & 1u;
+    return ((int64_t)1 << e) + (int64_t)(h + 1u) * ((int64_t)1 << (e - 1)) - 1;
+}
+
+struct PermilleList {
+    uint32_t v[16];
+};
+
+// One thread per candidate: cumulative counts over the 64 bins, one pass per requested rank.
+__global__ void ttft_percentile_kernel(const uint32_t* hist, uint64_t n, PermilleList pm, uint32_t n_p, int64_t* out) {
+    const uint64_t c = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= n) return;
+    const uint32_t* h = hist + c * MAASO_TTFT_BINS;
+    uint64_t total = 0;
+    for (int b = 0; b < MAASO_TTFT_BINS; b++) total += h[b];
+    for (uint32_t j = 0; j < n_p; j++) {
+        int64_t r = -1;
+        if (total > 0) {
+            uint64_t target = ((uint64_t)pm.v[j] * total + 999u) / 1000u;
+            if (target < 1) target = 1;
+            uint64_t cum = 0;
+            for (int b = 0; b < MAASO_TTFT_BINS; b++) {
+                cum += h[b];
+                if (cum >= target) { r = ttft_bin_upper((uint32_t)b); break; }
+            }
+        }
+        out[c * n_p + j] = r;
+    }
+}
+
+cudaError_t launch_ttft_percentiles(const uint32_t* hist, uint64_t n, const uint32_t* permille, uint32_t n_p,
+                                    int64_t* out, cudaStream_t stream) {
+    PermilleList pm;
+    for (uint32_t j = 0; j < 16; j++) pm.v[j] = j < n_p ? permille[j] : 0;
+    if (n) ttft_percentile_kernel<<<(unsigned)((n + 127) / 128), 128, 0, stream>>>(hist, n, pm, n_p, out);
+    return cudaGetLastError();
+}
+
 }  // namespace maaso

@@ -562,3 +562,48 @@ def test_api_errors(ctx):
     t = ctx.load_trace(dev, cfg["classes"])
     assert t.n == 500
     ctx.free_trace(t)
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_ttft_histogram_and_percentiles(ctx, oracle_mod, mapping):
+    import torch
+    cfg = gen.make_config("multimodel", n_cand=400, n_req=3000)
+    tr = cfg["traces"][0]
+    lists = [[(2, 0, 4)], []]                       # an invalid candidate and the empty placement
+    off2, inst2 = gen.candidates_from_lists(lists)
+    off = np.concatenate([cfg["offsets"], cfg["offsets"][-1] + off2[1:]]).astype(np.uint32)
+    inst = np.concatenate([cfg["inst"], inst2]).astype(np.uint32)
+    ctx.load_profile(cfg["profile"])
+    t = ctx.load_trace(tr, cfg["classes"])
+    n_cand = len(off) - 1
+    hist = torch.full((n_cand, 64), 77, dtype=torch.int32, device="cuda")
+    out = ctx.eval_placements(t, ctx.to_device(off), ctx.to_device(inst), 32, mapping=mapping, ttft_hist=hist)
+    pct = ctx.ttft_percentiles(hist, [500, 950, 990, 1000])
+    torch.cuda.synchronize()
+    want = oracle_mod.ttft_hist(cfg["profile"], tr, cfg["classes"], off, inst, 32)
+    got = hist.cpu().numpy().view(np.uint32)
+    assert (got == want).all(), np.nonzero((got != want).any(axis=1))[0][:5]
+    rec = ctx.results_to_numpy(out)
+    assert (got.sum(axis=1) == rec["n_served"]).all()
+    assert (pct.cpu().numpy() == oracle_mod.ttft_percentiles(want, [500, 950, 990, 1000])).all()
+    ctx.free_trace(t)
+
+
+def test_ttft_histogram_bin_edges_on_gpu(ctx, oracle_mod):
+    """The hand-worked bin edges of the oracle's pin, through the CUDA path."""
+    import torch
+    from test_oracle_pins import TTFT_BIN_EDGES, _prefill_only_profile, NONE3
+    prof = _prefill_only_profile([b for b, _ in TTFT_BIN_EDGES])
+    trace = np.zeros(1, dtype=gen.REQUEST_DTYPE)
+    trace["arrival_us"], trace["in_tokens"], trace["out_tokens"] = 5, 100, 2
+    offsets, inst = gen.candidates_from_lists([[(0, s, 1)] for s in range(len(TTFT_BIN_EDGES))])
+    for mapping in MAPPINGS:
+        ctx.load_profile(prof)
+        t = ctx.load_trace(trace, gen.make_classes(NONE3))
+        hist = torch.zeros((len(TTFT_BIN_EDGES), 64), dtype=torch.int32, device="cuda")
+        ctx.eval_placements(t, ctx.to_device(offsets), ctx.to_device(inst), 4, mapping=mapping, ttft_hist=hist)
+        torch.cuda.synchronize()
+        got = hist.cpu().numpy()
+        for c, (_, want_bin) in enumerate(TTFT_BIN_EDGES):
+            assert np.nonzero(got[c])[0].tolist() == [want_bin] and got[c, want_bin] == 1, (mapping, c)
+        ctx.free_trace(t)

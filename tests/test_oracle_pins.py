@@ -556,3 +556,75 @@ def test_prune_configs_batch_pareto(oracle_mod):
                 if not dom:
                     want.append((s, b))
         assert got == want
+
+
+# ---- time-to-first-token histogram and percentiles (Sec. V-A "response latency") -----------
+def _prefill_only_profile(bases):
+    """One model; strategy s = an instance whose prefill takes exactly bases[s] us (no per-token part)."""
+    n = len(bases)
+    return {"n_models": 1, "n_strategies": n, "wmax": gen.WMAX,
+            "devices": np.ones(n, dtype=np.int32), "min_devices": np.array([1], dtype=np.int32),
+            "prefill_base_us": np.array([bases], dtype=np.int32),
+            "prefill_q16": np.zeros((1, n), dtype=np.int32),
+            "step_us": np.full((1, n, gen.WMAX), 5000, dtype=np.int32)}
+
+
+# time to first token -> bin, worked out by hand from the definition in include/maaso.h:
+# below 1024 -> 0; 1024..1535 -> 1; 1536..2047 -> 2; 2048..3071 -> 3; 3072..4095 -> 4; 2^20 -> 21;
+# 1.5 * 2^20 -> 22; 2^30 -> 41; 2^30 + 2^29 -> 42
+TTFT_BIN_EDGES = [(0, 0), (1, 0), (1023, 0), (1024, 1), (1535, 1), (1536, 2), (2047, 2), (2048, 3), (3071, 3),
+                  (3072, 4), (4095, 4), (4096, 5), (1 << 20, 21), ((1 << 20) + (1 << 19), 22),
+                  ((1 << 21) - 1, 22), (1 << 30, 41), ((1 << 30) + (1 << 29), 42), ((1 << 31) - 1, 42)]
+
+
+def test_ttft_histogram_bin_edges(oracle_mod):
+    """One idle instance, one request: the time to first token is exactly the prefill time."""
+    bases = [b for b, _ in TTFT_BIN_EDGES]
+    prof = _prefill_only_profile(bases)
+    trace = np.zeros(1, dtype=gen.REQUEST_DTYPE)
+    trace["arrival_us"] = 5
+    trace["in_tokens"] = 100
+    trace["out_tokens"] = 2
+    classes = gen.make_classes(NONE3)
+    offsets, inst = gen.candidates_from_lists([[(0, s, 1)] for s in range(len(bases))])
+    hist = oracle_mod.ttft_hist(prof, trace, classes, offsets, inst, 4)
+    for c, (_, want_bin) in enumerate(TTFT_BIN_EDGES):
+        row = np.zeros(64, dtype=np.uint32)
+        row[want_bin] = 1
+        assert hist[c].tolist() == row.tolist(), (c, TTFT_BIN_EDGES[c], np.nonzero(hist[c])[0])
+
+
+def test_ttft_histogram_counts_served_requests_only(oracle_mod):
+    cfg = gen.make_config("tiny")
+    tr = cfg["traces"][0]
+    res, dumps = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"],
+                                            cfg["budget"], dump_idx=np.arange(len(cfg["offsets"]) - 1))
+    hist = oracle_mod.ttft_hist(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], cfg["budget"])
+    assert (hist.sum(axis=1) == res["n_served"]).all()
+    assert int(res["n_rejected"].sum()) > 0
+    # every percentile bound brackets the exact order statistic of the dumped first-token times
+    arr = tr["arrival_us"].astype(np.int64)
+    pct = oracle_mod.ttft_percentiles(hist, [500, 900, 990, 1000])
+    for c in range(0, len(hist), 7):
+        first = dumps["first_us"][c]
+        t = np.sort((first - arr)[first >= 0])
+        if len(t) == 0:
+            assert (pct[c] == -1).all()
+            continue
+        for j, pm in enumerate([500, 900, 990, 1000]):
+            exact = int(t[(pm * len(t) + 999) // 1000 - 1])      # the ceil(pm * n / 1000)-th smallest
+            upper = int(pct[c, j])
+            assert exact <= upper, (c, pm, exact, upper)
+            assert upper < max(1024, exact + exact // 2 + 1), (c, pm, exact, upper)   # two bins per octave
+
+
+def test_ttft_percentiles_by_hand(oracle_mod):
+    h = np.zeros((4, 64), dtype=np.uint32)
+    h[0, 0], h[0, 3] = 10, 10        # ten below 1024 us, ten in 2048..3071
+    h[1, 63] = 5                     # open last bin
+    h[2, 21] = 1                     # a single value in [2^20, 1.5 * 2^20)
+    pct = oracle_mod.ttft_percentiles(h, [1, 500, 501, 1000])
+    assert pct[0].tolist() == [1023, 1023, 3071, 3071]    # ranks 1, 10, 11, 20 of 20
+    assert pct[1].tolist() == [np.iinfo(np.int64).max] * 4
+    assert pct[2].tolist() == [(1 << 20) + (1 << 19) - 1] * 4
+    assert pct[3].tolist() == [-1] * 4                    # nothing served
