@@ -36,6 +36,14 @@ MUTANTS = [
     ("ranking prefers higher mean latency", "if (l != r) return l < r;", "if (l != r) return l > r;"),
     ("ranking prefers fewer hits", "return x->n_hit > y->n_hit;", "return x->n_hit < y->n_hit;"),
     ("latency weight is beta instead of 1 - beta", "double c = (1.0 - p->beta) * phil;", "double c = p->beta * phil;"),
+    ("histogram half-octave bit taken one position too low", "uint32_t h = (uint32_t)((t >> (e - 1)) & 1);",
+     "uint32_t h = (uint32_t)((t >> (e - 2)) & 1);"),
+    ("histogram counts rejected requests too", "if (first[q] >= 0) out[c * 64 + orc_ttft_bin(first[q] - reqs[q].arrival_us)]++;",
+     "if (first[q] >= -1) out[c * 64 + orc_ttft_bin(first[q] - reqs[q].arrival_us)]++;"),
+    ("percentile rank rounded down", "uint64_t target = ((uint64_t)permille * total + 999) / 1000;",
+     "uint64_t target = ((uint64_t)permille * total) / 1000;"),
+    ("percentile reports the lower bin edge", "return ((int64_t)1 << e) + (int64_t)(h + 1) * ((int64_t)1 << (e - 1)) - 1;",
+     "return ((int64_t)1 << e) + (int64_t)h * ((int64_t)1 << (e - 1));"),
     ("prefill does not stall the running batch", "in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {",
      "int64_t t_keep = in->T; in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {"),
 ]
@@ -78,6 +86,9 @@ def run_pins(mod):
     attempt("mask algebra", pins.test_mask_algebra)
     attempt("ranking", pins.test_topk_brute_force)
     attempt("score", pins.test_score_worked_values)
+    attempt("histogram edges", pins.test_ttft_histogram_bin_edges)
+    attempt("histogram counts", pins.test_ttft_histogram_counts_served_requests_only)
+    attempt("percentiles", pins.test_ttft_percentiles_by_hand)
     return failed
 
 
