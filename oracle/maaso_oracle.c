@@ -65,6 +65,7 @@
 #define ORC_EINVARIANT 0x80000000u /* an internal invariant failed: the oracle is wrong */
 
 #define ORC_FLAG_PRED_OPTIMISTIC 1u
+#define ORC_FLAG_ENGINE_FROZEN 2u /* the paper-literal engine: decode speed fixed at admission (below) */
 
 typedef struct {
     int64_t arrival_us;
@@ -213,6 +214,106 @@ static uint32_t validate(const orc_profile *p, const uint32_t *inst, uint32_t n_
 }
 
 /*
+ * The paper-literal engine ("frozen virtual slots").  Sec. IV-C writes the decode latency
+ * of request r as S_r / F(M, P, B, W_i) with W_i "the number of concurrent requests when
+ * request r arrives", and the simulator of Sec. V-A only keeps, per instance, B virtual
+ * slots and when each becomes free.  Read literally: the decode speed of a request is fixed
+ * when it is admitted, later admissions do not slow it down and prefills stall nobody.
+ *   - a slot is busy from the admission of its request until that request's finish time;
+ *     the running count w of an instance at time `now` = slots whose finish time is > now;
+ *   - admission at time t into an instance with w running: first token at t + prefill,
+ *     one token every step[w + 1] afterwards, finish = first + (S - 1) * step[w + 1];
+ *     the slot is held until the finish time (also when S = 1);
+ *   - the distributor is the one of the default engine: free slot first (start now), else the
+ *     time the earliest slot frees; feasibility with the worst case step[B], or, with the
+ *     optimistic flag and a free slot, with the step the request will really get; a wait moves
+ *     `now` to that time and the choice is made again;
+ *   - everything about a request is known at admission, so it is accounted there.
+ * With B = 1 everywhere the two engines coincide (nobody runs beside anybody).
+ */
+typedef struct {
+    uint32_t model, B;
+    const int32_t *step;
+    int64_t pre_base, pre_q16;
+    int busy[ORC_WMAX];
+    int64_t until[ORC_WMAX]; /* finish time of the request in the slot */
+} frozen_inst_t;
+
+static void frozen_replay(ctx_t *c, const orc_profile *p, const uint32_t *inst, uint32_t n_inst,
+                          const orc_request *reqs, uint64_t n, const orc_slo *classes, int has_mask,
+                          uint32_t class_mask, uint32_t flags, orc_result *out) {
+    frozen_inst_t *F = (frozen_inst_t *)calloc(n_inst ? n_inst : 1, sizeof(frozen_inst_t));
+    if (!F) { c->bad = 1; return; }
+    for (uint32_t i = 0; i < n_inst; i++) {
+        uint32_t word = inst[i];
+        F[i].model = word & 0xF; F[i].B = (word >> 12) & 0xFF;
+        size_t row = (size_t)F[i].model * p->n_strategies + ((word >> 4) & 0xFF);
+        F[i].step = p->step_us + row * p->wmax;
+        F[i].pre_base = p->prefill_base_us[row];
+        F[i].pre_q16 = (int64_t)(uint32_t)p->prefill_q16[row];
+    }
+    int64_t clock = 0;
+    for (uint64_t r = 0; r < n && !out->status; r++) {
+        const orc_request *q = &reqs[r];
+        if (has_mask && ((class_mask >> q->cls) & 1u) == 0) continue; /* not in R_x */
+        const orc_slo *k = &classes[q->cls];
+        int64_t len = q->out_tokens;
+        out->n_counted++;
+        if (q->arrival_us > clock) clock = q->arrival_us;
+        for (uint32_t round = 0;; round++) {
+            if (round >= ORC_ATTEMPT_CAP) { out->status = ORC_ELOOP; break; }
+            out->attempts++;
+            int found = 0, pick_tier = 0; int64_t pick_first = 0, pick_start = 0; uint32_t pick = 0;
+            for (uint32_t i = 0; i < n_inst; i++) {
+                frozen_inst_t *f = &F[i];
+                if (f->model != q->model) continue;
+                uint32_t running = 0; int64_t earliest = INT64_MAX;
+                for (uint32_t j = 0; j < f->B; j++) {
+                    if (f->busy[j] && f->until[j] <= clock) f->busy[j] = 0; /* the slot is free again */
+                    if (f->busy[j]) { running++; if (f->until[j] < earliest) earliest = f->until[j]; }
+                }
+                int tier_i = running < f->B ? 0 : 1;
+                int64_t start = tier_i == 0 ? clock : earliest;
+                int64_t prefill = f->pre_base + (int64_t)(((uint64_t)f->pre_q16 * q->in_tokens + 32768u) >> 16);
+                int64_t s_pred = f->step[f->B - 1];
+                if ((flags & ORC_FLAG_PRED_OPTIMISTIC) && tier_i == 0) s_pred = f->step[running];
+                int64_t p_first = start + prefill, p_fin = p_first + (len - 1) * s_pred;
+                int ok = (k->ttft_us < 0 || p_first - q->arrival_us <= k->ttft_us) &&
+                         (k->tbt_us < 0 || len == 1 || s_pred <= k->tbt_us) &&
+                         (k->e2e_us < 0 || p_fin - q->arrival_us <= k->e2e_us);
+                if (!ok) continue;
+                if (!found || tier_i < pick_tier || (tier_i == pick_tier && p_first < pick_first)) {
+                    found = 1; pick_tier = tier_i; pick_first = p_first; pick_start = start; pick = i;
+                }
+            }
+            if (!found) {
+                out->n_rejected++;
+                out->checksum += mix64((uint64_t)r * 0x9E3779B97F4A7C15ull ^ ~0ull);
+                if (c->dump_finish) c->dump_finish[r] = -1;
+                if (c->dump_first) c->dump_first[r] = -1;
+                if (c->dump_inst) c->dump_inst[r] = -1;
+                break;
+            }
+            if (pick_tier == 0) {
+                frozen_inst_t *f = &F[pick];
+                uint32_t running = 0, j = f->B;
+                for (uint32_t x = 0; x < f->B; x++) { if (f->busy[x]) running++; else if (j == f->B) j = x; }
+                if (j >= f->B) { c->bad = 1; break; }
+                int64_t speed = f->step[running];        /* level running + 1, fixed from now on */
+                int64_t first_tok = clock + f->pre_base + (int64_t)(((uint64_t)f->pre_q16 * q->in_tokens + 32768u) >> 16);
+                int64_t t_end = first_tok + (len - 1) * speed;
+                f->busy[j] = 1; f->until[j] = t_end;
+                complete(c, pick, (uint32_t)r, q->arrival_us, first_tok, t_end, (uint32_t)len, q->cls);
+                break;
+            }
+            if (pick_start <= clock) c->bad = 1;
+            clock = pick_start; /* wait for that slot, then choose again */
+        }
+    }
+    free(F);
+}
+
+/*
  * Score one candidate.  inst[n_inst]: packed words (model bits 0-3, strategy 4-11, batch
  * cap 12-19).  has_mask/class_mask: requests whose class bit is clear are not part of the
  * request subset R_x this placement is scored on (ignored when n_classes > 32).
@@ -249,6 +350,10 @@ int orc_eval_candidate(const orc_profile *p, const orc_request *reqs, uint64_t n
         I[i].pre_q16 = (int64_t)(uint32_t)p->prefill_q16[row];
     }
 
+    if (flags & ORC_FLAG_ENGINE_FROZEN) {
+        frozen_replay(&c, p, inst, n_inst, reqs, n, classes, has_mask, class_mask, flags, out);
+        goto replay_done;
+    }
     int64_t now = 0;
     for (uint64_t r = 0; r < n && !out->status; r++) {
         const orc_request *q = &reqs[r];
@@ -318,6 +423,7 @@ int orc_eval_candidate(const orc_profile *p, const orc_request *reqs, uint64_t n
     }
     if (!out->status)
         for (uint32_t i = 0; i < n_inst; i++) advance(&c, &I[i], i, -1); /* drain */
+replay_done:
     free(I);
 
     if (!out->status) {

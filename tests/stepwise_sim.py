@@ -130,3 +130,89 @@ def simulate(profile, trace, classes, instances, class_mask=None, optimistic=Fal
             ins.one_step(done_on(idx))
     st.update(finish_us=finish, first_us=first, inst=where)
     return st
+
+
+def simulate_frozen(profile, trace, classes, instances, class_mask=None, optimistic=False):
+    """The engine that fixes a request's decode speed at admission, in a formulation that
+    shares nothing with the C oracle's: no slots at all.  Every instance keeps the list of
+    token timestamps of the requests admitted to it (one list per request, built token by
+    token); the running count at time t is the number of lists whose last entry is after t."""
+    insts = []
+    for (m, s, b) in instances:
+        insts.append(dict(model=m, step=[int(x) for x in profile["step_us"][m][s]],
+                          base=int(profile["prefill_base_us"][m][s]),
+                          q16=int(profile["prefill_q16"][m][s]) & 0xFFFFFFFF, cap=b, tokens=[]))
+    n = len(trace)
+    finish, first, where = [-2] * n, [-2] * n, [-2] * n
+    st = dict(n_counted=0, n_served=0, n_hit=0, n_rejected=0, n_cascade=0, sum_ttft_us=0,
+              max_ttft_us=0, sum_e2e_us=0, max_e2e_us=0, makespan_us=0, tokens_out=0, attempts=0)
+
+    def lim(v):
+        return None if v < 0 else int(v)
+
+    def ends_after(ins, t):
+        return [tok[-1] for tok in ins["tokens"] if tok[-1] > t]
+
+    t_now = 0
+    for k in range(n):
+        q = trace[k]
+        cls, S, arrival, n_in = int(q["cls"]), int(q["out_tokens"]), int(q["arrival_us"]), int(q["in_tokens"])
+        if class_mask is not None and len(classes) <= 32 and not (class_mask >> cls) & 1:
+            continue
+        st["n_counted"] += 1
+        t_now = max(t_now, arrival)
+        c = classes[cls]
+        while True:
+            st["attempts"] += 1
+            options = []
+            for idx, ins in enumerate(insts):
+                if ins["model"] != int(q["model"]):
+                    continue
+                alive = ends_after(ins, t_now)
+                free = len(alive) < ins["cap"]
+                start = t_now if free else min(alive)
+                per_tok = ins["step"][ins["cap"] - 1]
+                if optimistic and free:
+                    per_tok = ins["step"][len(alive)]          # level len(alive) + 1
+                t_first = start + ins["base"] + ((ins["q16"] * n_in + 32768) >> 16)
+                t_end = t_first + (S - 1) * per_tok
+                if lim(c["ttft_us"]) is not None and t_first - arrival > lim(c["ttft_us"]):
+                    continue
+                if lim(c["tbt_us"]) is not None and S > 1 and per_tok > lim(c["tbt_us"]):
+                    continue
+                if lim(c["e2e_us"]) is not None and t_end - arrival > lim(c["e2e_us"]):
+                    continue
+                options.append((0 if free else 1, t_first, idx, start))
+            if not options:
+                st["n_rejected"] += 1
+                finish[k] = first[k] = where[k] = -1
+                break
+            tier, _, idx, start = min(options)
+            if tier == 1:
+                t_now = start
+                continue
+            ins = insts[idx]
+            gap = ins["step"][len(ends_after(ins, t_now))]      # fixed for the whole request
+            stamps = [t_now + ins["base"] + ((ins["q16"] * n_in + 32768) >> 16)]
+            for _ in range(S - 1):
+                stamps.append(stamps[-1] + gap)
+            ins["tokens"].append(stamps)
+            t_first, t_end = stamps[0], stamps[-1]
+            ttft, e2e = t_first - arrival, t_end - arrival
+            ok = ((lim(c["ttft_us"]) is None or ttft <= lim(c["ttft_us"])) and
+                  (lim(c["tbt_us"]) is None or S == 1 or
+                   Fraction(t_end - t_first, S - 1) <= lim(c["tbt_us"])) and
+                  (lim(c["e2e_us"]) is None or e2e <= lim(c["e2e_us"])))
+            st["n_served"] += 1
+            st["n_hit"] += ok
+            st["n_cascade"] += (not ok)
+            st["sum_ttft_us"] += ttft
+            st["max_ttft_us"] = max(st["max_ttft_us"], ttft)
+            st["sum_e2e_us"] += e2e
+            st["max_e2e_us"] = max(st["max_e2e_us"], e2e)
+            st["makespan_us"] = max(st["makespan_us"], t_end)
+            st["tokens_out"] += S
+            finish[k], first[k], where[k] = t_end, t_first, idx
+            break
+    st.update(finish_us=finish, first_us=first, inst=where)
+    return st

@@ -44,6 +44,16 @@ MUTANTS = [
      "uint64_t target = ((uint64_t)permille * total) / 1000;"),
     ("percentile reports the lower bin edge", "return ((int64_t)1 << e) + (int64_t)(h + 1) * ((int64_t)1 << (e - 1)) - 1;",
      "return ((int64_t)1 << e) + (int64_t)h * ((int64_t)1 << (e - 1));"),
+    ("frozen engine: slot freed one microsecond late", "if (f->busy[j] && f->until[j] <= clock) f->busy[j] = 0;",
+     "if (f->busy[j] && f->until[j] < clock) f->busy[j] = 0;"),
+    ("frozen engine: speed of one level too low", "int64_t speed = f->step[running];",
+     "int64_t speed = f->step[running > 0 ? running - 1 : 0];"),
+    ("frozen engine: wait overshoots", "int64_t start = tier_i == 0 ? clock : earliest;",
+     "int64_t start = tier_i == 0 ? clock : earliest + 1;"),
+    ("frozen engine: finish counts one token too many", "int64_t t_end = first_tok + (len - 1) * speed;",
+     "int64_t t_end = first_tok + len * speed;"),
+    ("frozen engine: optimistic estimate uses the current level", "tier_i == 0) s_pred = f->step[running];",
+     "tier_i == 0) s_pred = f->step[running > 0 ? running - 1 : 0];"),
     ("prefill does not stall the running batch", "in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {",
      "int64_t t_keep = in->T; in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {"),
 ]
@@ -86,6 +96,10 @@ def run_pins(mod):
     attempt("mask algebra", pins.test_mask_algebra)
     attempt("ranking", pins.test_topk_brute_force)
     attempt("score", pins.test_score_worked_values)
+    for seed in (0, 1, 2, 3):
+        attempt(f"frozen token lists {seed}", pins.test_frozen_engine_against_token_lists, seed)
+    attempt("frozen levels", pins.test_frozen_engine_levels_recomputed_from_the_dumps)
+    attempt("frozen cap one", pins.test_frozen_engine_equals_default_engine_for_one_instance_with_cap_one)
     attempt("histogram edges", pins.test_ttft_histogram_bin_edges)
     attempt("histogram counts", pins.test_ttft_histogram_counts_served_requests_only)
     attempt("percentiles", pins.test_ttft_percentiles_by_hand)

@@ -5,7 +5,7 @@ import pytest
 
 import gen
 from golden_cases import all_cases, check_against_expect, SCALAR_KEYS
-from stepwise_sim import simulate
+from stepwise_sim import simulate, simulate_frozen
 
 NONE3 = [(None, None, None)]
 
@@ -115,6 +115,91 @@ def test_against_token_by_token(oracle_mod, seed):
     assert d["finish_us"].tolist() == ref["finish_us"]
     assert d["first_us"].tolist() == ref["first_us"]
     assert d["inst"].tolist() == ref["inst"]
+
+
+# ---- the engine that fixes the decode speed at admission (flags = 2) -------------------------
+FROZEN = 2
+
+
+def _random_small_case(seed):
+    rng = np.random.default_rng(2000 + seed)
+    if seed % 3 == 2:
+        prof, model_mix = gen.profile_multimodel(seed), (0.5, 0.3, 0.2)
+    else:
+        prof, model_mix = gen.profile_node(seed), (1.0,)
+    trace = gen.make_trace(150, float(rng.choice([4.0, 20.0, 80.0])), seed, cv=float(rng.choice([1.0, 3.0])),
+                           model_mix=model_mix, out_dist=("lognormal", 3.0, 1.0, 1, 300), doc_out=(200, 400))
+    classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 8_000_000)])
+    instances = []
+    for _ in range(int(rng.integers(1, 7))):
+        m = int(rng.integers(prof["n_models"]))
+        ok = np.nonzero(prof["devices"] >= prof["min_devices"][m])[0]
+        instances.append((m, int(rng.choice(ok)), int(rng.choice([1, 2, 3, 4, 8, 16, 64]))))
+    return prof, trace, classes, instances
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_frozen_engine_against_token_lists(oracle_mod, seed):
+    prof, trace, classes, instances = _random_small_case(seed)
+    mask = None if seed % 4 else 0b110
+    opt = seed % 2
+    res, d = run_one(oracle_mod, prof, trace, classes, instances, mask=mask, flags=FROZEN | opt)
+    ref = simulate_frozen(prof, trace, classes, instances, class_mask=mask, optimistic=bool(opt))
+    for key in SCALAR_KEYS:
+        assert int(res[key]) == ref[key], key
+    assert d["finish_us"].tolist() == ref["finish_us"]
+    assert d["first_us"].tolist() == ref["first_us"]
+    assert d["inst"].tolist() == ref["inst"]
+
+
+def test_frozen_engine_equals_default_engine_for_one_instance_with_cap_one(oracle_mod):
+    """One instance with B = 1: nobody runs beside anybody, so there is no slowdown and no stall
+    and both engines must give every request the same times (single-server FIFO) and the same
+    record.  Only the number of distributor rounds may differ: the default engine's clock sits
+    on a decode-step boundary, so it can see the slot free one round earlier.  Requests of one
+    token are left out: they hold a slot during their prefill in this engine, none in the other."""
+    for seed in range(6):
+        prof, trace, classes, instances = _random_small_case(seed)
+        trace["out_tokens"] = np.maximum(trace["out_tokens"], 2)
+        trace["model"] = instances[0][0]
+        instances = [(instances[0][0], instances[0][1], 1)]
+        for opt in (0, 1):
+            a, da = run_one(oracle_mod, prof, trace, classes, instances, flags=opt)
+            b, db = run_one(oracle_mod, prof, trace, classes, instances, flags=FROZEN | opt)
+            a, b = a.copy(), b.copy()
+            a["attempts"] = b["attempts"] = 0
+            assert a.tobytes() == b.tobytes()
+            for key in da:
+                assert (da[key] == db[key]).all()
+
+
+def test_frozen_engine_levels_recomputed_from_the_dumps(oracle_mod):
+    """From the per-request times alone: a request holds its slot from (first token - prefill) to
+    its finish; at its admission the instance must have had a free slot, and its tokens must be
+    exactly one table step of the level (running + 1) apart.  No request may miss its SLO."""
+    cfg = gen.make_config("tiny", n_req=300)
+    prof, tr = cfg["profile"], cfg["traces"][0]
+    off, inst = cfg["offsets"], cfg["inst"]
+    pick = np.arange(0, len(off) - 1, 9)
+    for opt in (0, 1):
+        res, d = oracle_mod.eval_placements(prof, tr, cfg["classes"], off, inst, cfg["budget"], flags=FROZEN | opt,
+                                            dump_idx=pick)
+        for row, c in enumerate(pick):
+            words = inst[off[c]:off[c + 1]]
+            assert int(res[c]["n_cascade"]) == 0 and int(res[c]["n_served"]) == int(res[c]["n_hit"])
+            for i, word in enumerate(words):
+                m, s, B = int(word & 15), int((word >> 4) & 255), int((word >> 12) & 255)
+                mine = np.nonzero(d["inst"][row] == i)[0]
+                spans = []
+                for r in mine:
+                    pre = int(prof["prefill_base_us"][m, s]) + ((int(prof["prefill_q16"][m, s]) * int(tr["in_tokens"][r]) + 32768) >> 16)
+                    spans.append((int(d["first_us"][row][r]) - pre, int(d["finish_us"][row][r]), r))
+                for (t_adm, t_fin, r) in spans:
+                    running = sum(1 for (a, f, o) in spans if o != r and a <= t_adm < f and (a, o) < (t_adm, r))
+                    assert running < B
+                    S = int(tr["out_tokens"][r])
+                    if S > 1:
+                        assert t_fin - int(d["first_us"][row][r]) == (S - 1) * int(prof["step_us"][m, s, running])
 
 
 # ---- P4: invariants -----------------------------------------------------------------------
