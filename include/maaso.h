@@ -66,6 +66,16 @@ extern "C" {
 #define MAASO_FLAG_PRED_OPTIMISTIC 1u /* distributor predicts with the step time right after admission
                                          instead of the worst case F(M,P,B_I) of Sec. IV-F step 3 */
 
+#define MAASO_FLAG_ENGINE_FROZEN 2u /* replay with the engine that fixes a request's decode speed at its
+                                      admission (Sec. IV-C read literally: the concurrency W_i "when
+                                      request r arrives"; virtual slots of Sec. V-A): a slot is busy from
+                                      admission to the request's finish time, first token = admission +
+                                      prefill, one token every step[running + 1] afterwards; later
+                                      admissions slow nobody down and prefills stall nobody.  Same
+                                      distributor.  Lane-group mapping only: MAASO_MAP_BLOCK is refused and
+                                      a placement with more than 32 instances gets MAASO_CAND_ETOOMANY;
+                                      finish times must stay below 2^57 us (else MAASO_CAND_ELOOP). */
+
 #define MAASO_FLAG_TEST_STALL 0x80000000u /* test hook for the bounded device-side waits: the trace copies
                                              are never issued and every wait is limited to about 0.1 s, so
                                              each valid candidate must come back with MAASO_CAND_ETIMEOUT

@@ -5,7 +5,7 @@
 // The trace (and the per-request checksum term of a rejection) is staged once per thread
 // block in shared-memory tiles by 1-D bulk copies (TMA) and shared by every candidate of
 // the block.  No global memory access sits on the per-request path.
-#include "lane_sim.cuh"
+#include "lane_frozen.cuh"
 
 namespace maaso {
 
@@ -120,14 +120,18 @@ __device__ __forceinline__ void issue_tile(const GroupSmem& sm, const EvalParams
               bytes, &sm.full_bar[stage]);
 }
 
-// OPT: the distributor predicts with the step time right after admission (optimistic estimate)
-template <bool OPT>
+// OPT: the distributor predicts with the step time right after admission (optimistic estimate).
+// Inst: LaneInst (default engine: decode speed follows the running count) or FrozenInst (speed
+// fixed at admission).
+template <bool OPT, class Inst>
 __global__ void __launch_bounds__(kGroupThreads, 4)
 eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_bytes) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const GroupSmem sm = carve(smem_raw, P.n_rows, P.n_classes, tile_recs, pool_bytes);
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     constexpr uint32_t kWarps = kGroupThreads / 32;
+    // a wait is followed by a new choice, unless the engine and the estimate make that round redundant
+    constexpr bool LOOP = OPT || Inst::kAlwaysLoop;
 
     // profile residency: decode-step tables and SLO classes into shared memory
     for (uint32_t i = tid; i < P.n_rows * 64u; i += kGroupThreads)
@@ -214,10 +218,8 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         uint32_t n_i = 0, lo = 0;
         if (valid) { lo = P.offsets[cand]; n_i = P.offsets[cand + 1] - lo; }
         const bool has = valid && sub < n_i;
-        LaneInst in;
-        in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = kKeyEmpty; in.sw = 1; in.rsw = 1.0f; in.qn = 0;
-        in.mask = ~0ull; in.gen = 0;
-        in.B = 1; in.model = 0xFFFFFFFFu; in.step = sm.steps; in.stepB = 1; in.pre_base = 0; in.pre_q16 = 0;
+        Inst in;
+        lane_reset(in, sm.steps);
         if (has) {
             const uint32_t word = P.inst[lo + sub];
             in.model = word & 0xFu;
@@ -234,7 +236,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         // pool cannot hold use their global scratch instead
         {
             const uint32_t nblk = has ? (in.B + 7u) >> 3 : 0u;
-            const uint32_t units = has ? nblk + 1u : 0u;
+            const uint32_t units = has ? (nblk + 1u) * Inst::kKeyWords : 0u;
             uint32_t incl = units;
             for (uint32_t o = 1; o < 32u; o <<= 1) {
                 const uint32_t v = __shfl_up_sync(kFullMask, incl, o);
@@ -249,7 +251,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                                         : lane_scratch + kLaneScratchKeys;
             env.keys_shared = region != lane_scratch + kLaneScratchKeys;
             env.keys = reinterpret_cast<uint32_t*>(region);
-            env.bm_lo = reinterpret_cast<uint4*>(region + (size_t)nblk * kKeyUnitBytes);
+            env.bm_lo = reinterpret_cast<uint4*>(region + (size_t)nblk * kKeyUnitBytes * Inst::kKeyWords);
             env.bm_hi = env.bm_lo + 1;
             const uint4 e4 = make_uint4(kKeyEmpty, kKeyEmpty, kKeyEmpty, kKeyEmpty);
             for (uint32_t i = 0; i < 2u * units; i++) reinterpret_cast<uint4*>(region)[i] = e4;
@@ -316,7 +318,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                 do {
                     uint32_t key = kKey32Inf;
                     int64_t t0 = 0, first = 0;
-                    if (OPT && pending) {
+                    if (LOOP && pending) {
                         attempts++;
                         tries++;
                     }
@@ -342,12 +344,12 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                             }
                             pending = false;
                         } else if (am.tier == 0) {
-                            if ((int)lane == am.winner) lane_admit(in, q, req, pre, env, status);
+                            if ((int)lane == am.winner) lane_admit(in, q, req, pre, now, env, status);
                             pending = false;
                         } else {
                             // every capable instance is full: wait until the chosen slot frees
                             now = t0w;
-                            if (!OPT) {
+                            if (!LOOP) {
                                 // With the worst-case estimate the next round cannot choose differently:
                                 // at that time the winner has a free slot with the same predicted first
                                 // token, and no other instance's prediction can have become earlier or
@@ -355,7 +357,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                                 attempts++;  // the second round, counted only
                                 if ((int)lane == am.winner) {
                                     lane_advance(in, now, false, env, status);
-                                    lane_admit(in, q, req, pre, env, status);
+                                    lane_admit(in, q, req, pre, now, env, status);
                                 }
                                 pending = false;
                             } else if (tries >= kAttemptCap) {
@@ -364,7 +366,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                             }
                         }
                     }
-                } while (OPT && __any_sync(kFullMask, pending));
+                } while (LOOP && __any_sync(kFullMask, pending));
             }
             // release the stage; the warp that arrives last refills it
             __syncwarp();
@@ -413,9 +415,16 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         __syncwarp();
         if (valid && sub == 0) {
             // worst-case mode: one round per counted request plus the counted second rounds
-            write_result(P.out + cand, status, n_counted, n_rejected, OPT ? attempts : attempts + n_counted, st, h);
+            write_result(P.out + cand, status, n_counted, n_rejected, LOOP ? attempts : attempts + n_counted, st, h);
         }
     }
+}
+
+using GroupKernel = void (*)(const EvalParams, const int, const uint32_t);
+static GroupKernel group_kernel_for(uint32_t flags) {
+    const bool opt = (flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
+    if (flags & MAASO_FLAG_ENGINE_FROZEN) return opt ? eval_group_kernel<true, FrozenInst> : eval_group_kernel<false, FrozenInst>;
+    return opt ? eval_group_kernel<true, LaneInst> : eval_group_kernel<false, LaneInst>;
 }
 
 // Shared memory of one block: the fixed parts plus a key pool that fills what is left when
@@ -429,7 +438,7 @@ static size_t group_smem_bytes(const EvalParams& P, int tile_recs, int blocks_pe
     if (budget > 227u * 1024u) budget = 227u * 1024u;
     size_t pool = budget > fixed ? budget - fixed : 0;
     pool -= pool % 128;
-    const size_t all = (size_t)kGroupThreads * 9 * kKeyUnitBytes;
+    const size_t all = (size_t)kGroupThreads * 9 * kKeyUnitBytes * ((P.flags & MAASO_FLAG_ENGINE_FROZEN) ? 2 : 1);
     if (pool > all) pool = all;
     *pool_bytes = (uint32_t)pool;
     return fixed + pool;
@@ -439,8 +448,7 @@ cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, int 
                               cudaStream_t stream) {
     uint32_t pool = 0;
     const size_t smem = group_smem_bytes(P, tile_recs, blocks_per_sm, smem_per_sm, &pool);
-    const bool opt = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
-    auto kernel = opt ? eval_group_kernel<true> : eval_group_kernel<false>;
+    auto kernel = group_kernel_for(P.flags);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kernel<<<grid, kGroupThreads, smem, stream>>>(P, tile_recs, pool);
@@ -452,8 +460,7 @@ size_t group_scratch_per_lane() { return kLaneScratchBytes; }
 int occupancy_eval_group(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm) {
     uint32_t pool = 0;
     const size_t smem = group_smem_bytes(P, tile_recs, blocks_per_sm, smem_per_sm, &pool);
-    const bool opt = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
-    auto kernel = opt ? eval_group_kernel<true> : eval_group_kernel<false>;
+    auto kernel = group_kernel_for(P.flags);
     cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kGroupThreads, smem) != cudaSuccess) return 1;

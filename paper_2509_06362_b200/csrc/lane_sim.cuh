@@ -45,10 +45,12 @@ constexpr size_t kLaneScratchA = 0;
 constexpr size_t kLaneScratchB = 64 * 2 * 16;
 constexpr size_t kLaneScratchOvf = kLaneScratchB + 64 * 2 * 8;
 constexpr size_t kLaneScratchKeys = kLaneScratchOvf + (size_t)kQueueOvf * 32;
-constexpr size_t kLaneScratchBytes = kLaneScratchKeys + 9 * kKeyUnitBytes + 32;
+constexpr size_t kLaneScratchBytes = kLaneScratchKeys + 2 * 9 * kKeyUnitBytes + 32;  // keys of either engine
 static_assert(kLaneScratchBytes % 32 == 0 && kLaneScratchKeys % 16 == 0, "lane scratch layout");
 
 struct LaneInst {
+    static constexpr bool kAlwaysLoop = false;  // a wait is resolved in one round under the worst-case estimate
+    static constexpr uint32_t kKeyWords = 1;    // 32-bit words per slot key
     int64_t T;        // clock, always a decode-step boundary (may lag `now` while the instance is full)
     int64_t tc;       // time of the next completion if nobody is admitted (valid while w > 0)
     uint32_t K;       // decode steps done at T since the counter last restarted
@@ -104,12 +106,15 @@ __device__ __forceinline__ uint32_t min8(const uint32_t (&v)[8]) {
     return min(min(__vimin3_u32(v[0], v[1], v[2]), __vimin3_u32(v[3], v[4], v[5])), min(v[6], v[7]));
 }
 
-// *p = min(*p, v) without waiting for the old value (a reduction, not an atomic with a result).
+// *p = min(*p, v).  In shared memory as a reduction (nothing waits for the old value).  A lane
+// whose keys live in global scratch reads and writes them with plain loads and stores only: a
+// reduction would be carried out in L2 and a later load of the same lane could still be served
+// a stale line from L1.
 __device__ __forceinline__ void block_min_update(uint32_t* p, uint32_t v, bool shared) {
     if (shared)
         asm volatile("red.shared.min.u32 [%0], %1;" ::"r"(smem_addr(p)), "r"(v) : "memory");
     else
-        asm volatile("red.global.min.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+        *p = min(*p, v);
 }
 
 __device__ __forceinline__ uint32_t* bm_entry(const LaneEnv& env, uint32_t b) {
@@ -140,7 +145,8 @@ __device__ __forceinline__ void lane_push_slot(LaneInst& in, const LaneEnv& env,
 }
 
 // Same for a request that completes at admission (one output token): everything is in registers.
-__device__ __forceinline__ void lane_push_now(LaneInst& in, const LaneEnv& env, int64_t t_fin, uint4 a, uint2 b,
+template <class Inst>
+__device__ __forceinline__ void lane_push_now(Inst& in, const LaneEnv& env, int64_t t_fin, uint4 a, uint2 b,
                                               uint32_t& status) {
     const uint32_t j = in.qn;
     if (j < (uint32_t)kQueue) {
@@ -197,6 +203,12 @@ __device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const
         }
     }
     ls->st = st;
+}
+
+__device__ __forceinline__ void lane_reset(LaneInst& in, const int32_t* steps) {
+    in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = kKeyEmpty; in.sw = 1; in.rsw = 1.0f; in.qn = 0;
+    in.mask = ~0ull; in.gen = 0;
+    in.B = 1; in.model = 0xFFFFFFFFu; in.step = steps; in.stepB = 1; in.pre_base = 0; in.pre_q16 = 0;
 }
 
 // The counter K has just reached the smallest end index (clock = in.T).  Retire every
@@ -324,8 +336,9 @@ __device__ __noinline__ uint32_t lane_rebase(uint32_t* keys, uint32_t nslots, ui
 }
 
 // "map": prefill at the step boundary (running decodes stall), then occupy a free slot.
-__device__ __forceinline__ void lane_admit(LaneInst& in, const CookedReq& q, uint32_t req, int64_t pre,
+__device__ __forceinline__ void lane_admit(LaneInst& in, const CookedReq& q, uint32_t req, int64_t pre, int64_t now,
                                            const LaneEnv& env, uint32_t& status) {
+    (void)now;  // the instance's own clock is at or after `now`
     in.T += pre;
     const uint4 pa = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)q.arrival,
                                 (uint32_t)((uint64_t)q.arrival >> 32));

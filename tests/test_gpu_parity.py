@@ -24,6 +24,8 @@ def ctx():
 @pytest.mark.parametrize("case", all_cases(), ids=lambda c: c["name"])
 def test_hand_timelines_on_gpu(ctx, case, mapping):
     for flags, expect in case["runs"]:
+        if (flags & 2) and mapping == 1:
+            continue      # the fixed-speed engine exists in the lane-group mapping only
         res, dumps = gpu_eval(ctx, case["profile"], case["trace"], case["classes"], case["offsets"],
                               case["inst"], case["budget"], None, flags, mapping, dump_idx=[0])
         check_against_expect(res[0], {k: v[0] for k, v in dumps.items()}, expect)
@@ -607,3 +609,104 @@ def test_ttft_histogram_bin_edges_on_gpu(ctx, oracle_mod):
         for c, (_, want_bin) in enumerate(TTFT_BIN_EDGES):
             assert np.nonzero(got[c])[0].tolist() == [want_bin] and got[c, want_bin] == 1, (mapping, c)
         ctx.free_trace(t)
+
+
+# ---- the engine that fixes the decode speed at admission (flag 2) ----------------------------
+@pytest.mark.parametrize("flags", [2, 3])
+def test_frozen_engine_tiny_config_full(ctx, oracle_mod, flags):
+    cfg = gen.make_config("tiny")
+    tr = cfg["traces"][0]
+    idx = np.arange(0, 143, 5, dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"],
+                                          cfg["budget"], None, flags, dump_idx=idx)
+    got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], cfg["budget"],
+                       None, flags, 0, dump_idx=idx)
+    assert_records_equal(got, want, "tiny, fixed-speed engine")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+    assert int(want["n_served"].sum()) > 0 and int(want["n_rejected"].sum()) > 0
+
+
+@pytest.mark.parametrize("flags", [2, 3])
+def test_frozen_engine_node_and_multimodel_subsets(ctx, oracle_mod, flags):
+    # ragged trace length (tiles of 64 + a tail), every group width up to 32 lanes, class masks, dumps
+    cfg = gen.make_config("node", n_req=1777)
+    sel = np.arange(0, 10864, 29)
+    off = np.zeros(len(sel) + 1, dtype=np.uint32)
+    parts = []
+    for k, c in enumerate(sel):
+        parts.append(cfg["inst"][cfg["offsets"][c]:cfg["offsets"][c + 1]])
+        off[k + 1] = off[k] + len(parts[-1])
+    inst = np.concatenate(parts).astype(np.uint32)
+    tr = cfg["traces"][0]
+    idx = np.arange(0, len(sel), 41, dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 8, None, flags, dump_idx=idx)
+    got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 8, None, flags, 0, dump_idx=idx)
+    assert_records_equal(got, want, "node subset, fixed-speed engine")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+
+    cfg = gen.make_config("multimodel", n_cand=500, n_req=3000)
+    n_i = np.diff(cfg["offsets"])
+    keep = np.nonzero(n_i <= 32)[0]
+    off = np.zeros(len(keep) + 1, dtype=np.uint32)
+    parts = []
+    for k, c in enumerate(keep):
+        parts.append(cfg["inst"][cfg["offsets"][c]:cfg["offsets"][c + 1]])
+        off[k + 1] = off[k] + len(parts[-1])
+    inst = np.concatenate(parts).astype(np.uint32)
+    mask = np.random.default_rng(5).integers(1, 8, size=len(keep)).astype(np.uint32)
+    tr = cfg["traces"][0]
+    want = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 32, mask, flags)
+    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 32, mask, flags, 0)
+    assert_records_equal(got, want, "multimodel subset, fixed-speed engine")
+
+
+def test_frozen_engine_limits(ctx):
+    """No block mapping for this engine; placements with more than 32 instances are refused one by one."""
+    import paper_2509_06362_b200 as m
+    cfg = gen.make_config("tiny", n_req=50)
+    ctx.load_profile(cfg["profile"])
+    t = ctx.load_trace(cfg["traces"][0], cfg["classes"])
+    d_off, d_inst = ctx.to_device(cfg["offsets"]), ctx.to_device(cfg["inst"])
+    with pytest.raises(m.MaasoError):
+        ctx.eval_placements(t, d_off, d_inst, 4, flags=2, mapping=1)
+    off, inst = gen.candidates_from_lists([[(0, 0, 1)] * 33, [(0, 0, 1)] * 32])
+    import torch
+    out = ctx.eval_placements(t, ctx.to_device(off), ctx.to_device(inst), 64, flags=2)
+    torch.cuda.synchronize()
+    rec = ctx.results_to_numpy(out)
+    assert int(rec["status"][0]) == m.CAND_STATUS["ETOOMANY"] and int(rec["status"][1]) == 0
+    ctx.free_trace(t)
+
+
+@pytest.mark.parametrize("flags", [0, 1, 2, 3])
+def test_slot_keys_in_global_scratch_when_the_pool_is_too_small(oracle_mod, flags):
+    """A context created with MAASO_GROUP_BLOCKS=8 leaves no shared memory for the key pool, so
+    every lane keeps its slot keys in global scratch: same results."""
+    import os
+    import paper_2509_06362_b200 as m
+    old = os.environ.get("MAASO_GROUP_BLOCKS")
+    os.environ["MAASO_GROUP_BLOCKS"] = "8"
+    try:
+        c = m.Context(0)
+    finally:
+        if old is None:
+            del os.environ["MAASO_GROUP_BLOCKS"]
+        else:
+            os.environ["MAASO_GROUP_BLOCKS"] = old
+    try:
+        cfg = gen.make_config("multimodel", n_cand=300, n_req=2000)
+        keep = np.nonzero(np.diff(cfg["offsets"]) <= 32)[0]
+        off = np.zeros(len(keep) + 1, dtype=np.uint32)
+        parts = []
+        for k, cand in enumerate(keep):
+            parts.append(cfg["inst"][cfg["offsets"][cand]:cfg["offsets"][cand + 1]])
+            off[k + 1] = off[k] + len(parts[-1])
+        inst = np.concatenate(parts).astype(np.uint32)
+        tr = cfg["traces"][0]
+        want = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 32, None, flags)
+        got, _ = gpu_eval(c, cfg["profile"], tr, cfg["classes"], off, inst, 32, None, flags, 0)
+        assert_records_equal(got, want, "keys in global scratch")
+    finally:
+        c.close()
