@@ -27,8 +27,8 @@ TOPK = 64
 # ncu counters of eval_group_kernel on the default workload (profiles/eval_group_kernel_node_sweep.md).
 # They describe the kernel as committed with that summary; set to None when the kernel changes.
 PROFILED = {"workload": "node", "mapping": 0,
-            "dram_bytes_per_launch": 41_212_416 + 33_419_264,
-            "warp_inst_per_launch": 5_016_497_062}
+            "dram_bytes_per_launch": 43_010_048 + 37_484_288,
+            "warp_inst_per_launch": 4_999_789_912}
 SM_COUNT, ISSUE_PER_SM = 148, 4   # B200: 148 SMs x 4 warp schedulers, one warp instruction per cycle each
 
 
