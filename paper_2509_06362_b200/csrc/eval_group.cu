@@ -72,7 +72,7 @@ struct GroupSmem {
 };
 
 __host__ __device__ inline size_t group_smem_static(uint32_t n_rows, uint32_t n_classes, int tile_recs) {
-    size_t b = (size_t)kStages * (tile_recs + 1) * 16 * kCookedWords;  // one spare record per stage (look-ahead read)
+    size_t b = (size_t)kStages * tile_recs * 16 * kCookedWords;
     b += (size_t)kQueue * kGroupThreads * (16 + 8 + 8);
     b += (size_t)n_classes * 24;
     b += kStages * 8;
@@ -88,7 +88,7 @@ __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows,
     s.pool = base;
     base += pool_bytes;
     s.tiles = reinterpret_cast<uint4*>(base);
-    base += (size_t)kStages * (tile_recs + 1) * 16 * kCookedWords;
+    base += (size_t)kStages * tile_recs * 16 * kCookedWords;
     s.qa = reinterpret_cast<uint4*>(base);
     base += (size_t)kQueue * kGroupThreads * 16;
     s.qb = reinterpret_cast<uint2*>(base);
@@ -116,15 +116,27 @@ __device__ __forceinline__ void issue_tile(const GroupSmem& sm, const EvalParams
     const uint32_t recs = min((uint32_t)tile_recs, P.n_req - tile * tile_recs);
     const uint32_t bytes = recs * 16u * kCookedWords;
     mbar_expect_tx(&sm.full_bar[stage], bytes);
-    bulk_load(sm.tiles + (size_t)stage * (tile_recs + 1) * kCookedWords, P.cooked + (size_t)tile * tile_recs * kCookedWords,
+    bulk_load(sm.tiles + (size_t)stage * tile_recs * kCookedWords, P.cooked + (size_t)tile * tile_recs * kCookedWords,
               bytes, &sm.full_bar[stage]);
+}
+
+// Account the queued completions of the whole warp once some lane holds kFlushAt of them.
+__device__ __forceinline__ void flush_if_due(uint32_t& qn, LaneStats& ls, const LaneEnv& env, const int64_t* classes,
+                                             uint32_t sub, const Dump& dump) {
+    if (__any_sync(kFullMask, qn >= (uint32_t)kFlushAt)) {
+        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, qn, classes, sub, dump.finish, dump.first, dump.inst,
+                    dump.hist);
+        qn = 0;
+    }
 }
 
 // OPT: the distributor predicts with the step time right after admission (optimistic estimate).
 // Inst: LaneInst (default engine: decode speed follows the running count) or FrozenInst (speed
-// fixed at admission).
-template <bool OPT, class Inst>
-__global__ void __launch_bounds__(kGroupThreads, 4)
+// fixed at admission).  MINB: blocks per SM the register budget must allow: 4 for batches that
+// fill the GPU (128 registers), 3 for batches of one wave, which are bound by their longest
+// dependent chains and run a little faster without the spills of the tighter budget.
+template <bool OPT, class Inst, int MINB>
+__global__ void __launch_bounds__(kGroupThreads, MINB)
 eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_bytes) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const GroupSmem sm = carve(smem_raw, P.n_rows, P.n_classes, tile_recs, pool_bytes);
@@ -285,23 +297,14 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                 sm.work[1] = 1;
                 break;
             }
-            const uint4* tile = sm.tiles + (size_t)s * (tile_recs + 1) * kCookedWords;
+            const uint4* tile = sm.tiles + (size_t)s * tile_recs * kCookedWords;
             const uint32_t recs = min((uint32_t)tile_recs, P.n_req - t * tile_recs);
-            uint4 nx0 = tile[0], nx1 = tile[1], nx2 = tile[2];
             // a warp without a candidate only keeps the tile pipeline going
             for (uint32_t ri = warp_has_work ? 0u : recs; ri < recs; ri++) {
-                const uint4 r0 = nx0, r1 = nx1, r2 = nx2;
-                {
-                    // next record, ahead of its use (after the last one: the stage's spare record, never used)
-                    const uint4* nx = tile + (size_t)(ri + 1) * kCookedWords;
-                    nx0 = nx[0]; nx1 = nx[1]; nx2 = nx[2];
-                }
-                // statistics of completed requests: every fourth request, if some lane's queue is half full
-                if ((ri & 3u) == 3u && __any_sync(kFullMask, in.qn >= (uint32_t)kFlushAt)) {
-                    flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first,
-                                dump.inst, dump.hist);
-                    in.qn = 0;
-                }
+                // statistics of completed requests: every fourth request, if some lane's queue is nearly full
+                if ((ri & 3u) == 0u) flush_if_due(in.qn, ls, env, sm.classes, sub, dump);
+                const uint4* rec = tile + (size_t)ri * kCookedWords;
+                const uint4 r0 = rec[0], r1 = rec[1], r2 = rec[2];
                 // All 32 lanes walk the trace together and every warp-level operation below uses
                 // the full mask (segmented by the group width), so the groups of a warp share one
                 // instruction stream; only events (retire, admit) diverge.
@@ -327,7 +330,6 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                         key = lane_predict(in, q, pre, now, OPT, t0, first);
                     }
                     const ArgMin am = group_argmin(key, first, gmask, G, own);
-                    const int64_t t0w = (int64_t)shfl_u64((uint64_t)t0, am.winner, kFullMask);
                     if (pending) {
                         if (!am.found) {
                             // overflow protection: nobody can meet the deadline -> rejected
@@ -347,8 +349,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                             if ((int)lane == am.winner) lane_admit(in, q, req, pre, now, env, status);
                             pending = false;
                         } else {
-                            // every capable instance is full: wait until the chosen slot frees
-                            now = t0w;
+                            // every capable instance is full: wait until the chosen slot frees (the
+                            // outcome is the same for all lanes of the group, so they are all here)
+                            now = (int64_t)shfl_u64((uint64_t)t0, am.winner, gmask);
                             if (!LOOP) {
                                 // With the worst-case estimate the next round cannot choose differently:
                                 // at that time the winner has a free slot with the same predicted first
@@ -421,10 +424,15 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
 }
 
 using GroupKernel = void (*)(const EvalParams, const int, const uint32_t);
-static GroupKernel group_kernel_for(uint32_t flags) {
+template <int MINB>
+static GroupKernel group_kernel_of(uint32_t flags) {
     const bool opt = (flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
-    if (flags & MAASO_FLAG_ENGINE_FROZEN) return opt ? eval_group_kernel<true, FrozenInst> : eval_group_kernel<false, FrozenInst>;
-    return opt ? eval_group_kernel<true, LaneInst> : eval_group_kernel<false, LaneInst>;
+    if (flags & MAASO_FLAG_ENGINE_FROZEN)
+        return opt ? eval_group_kernel<true, FrozenInst, MINB> : eval_group_kernel<false, FrozenInst, MINB>;
+    return opt ? eval_group_kernel<true, LaneInst, MINB> : eval_group_kernel<false, LaneInst, MINB>;
+}
+static GroupKernel group_kernel_for(uint32_t flags, int blocks_per_sm) {
+    return blocks_per_sm >= 4 ? group_kernel_of<4>(flags) : group_kernel_of<3>(flags);
 }
 
 // Shared memory of one block: the fixed parts plus a key pool that fills what is left when
@@ -448,7 +456,7 @@ cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, int 
                               cudaStream_t stream) {
     uint32_t pool = 0;
     const size_t smem = group_smem_bytes(P, tile_recs, blocks_per_sm, smem_per_sm, &pool);
-    auto kernel = group_kernel_for(P.flags);
+    auto kernel = group_kernel_for(P.flags, blocks_per_sm);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kernel<<<grid, kGroupThreads, smem, stream>>>(P, tile_recs, pool);
@@ -460,7 +468,7 @@ size_t group_scratch_per_lane() { return kLaneScratchBytes; }
 int occupancy_eval_group(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm) {
     uint32_t pool = 0;
     const size_t smem = group_smem_bytes(P, tile_recs, blocks_per_sm, smem_per_sm, &pool);
-    auto kernel = group_kernel_for(P.flags);
+    auto kernel = group_kernel_for(P.flags, blocks_per_sm);
     cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kGroupThreads, smem) != cudaSuccess) return 1;
