@@ -596,52 +596,68 @@ MAASO_API int maaso_topk_scores(maaso_ctx* ctx, const maaso_result* results, con
 
 // Alg. 1 as a host driver: every configuration runs its own greedy chain; the tentative
 // placements of all chains in one greedy step are one candidate batch on the GPU.
-MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_t gpus,
-                               const maaso_config* configs, uint32_t n_configs, int use_mask,
-                               uint32_t class_mask, const maaso_score_params* score, uint32_t flags,
-                               double* phi_star, uint32_t* istar_len, uint32_t* istar_inst) {
-    if (!ctx || !trace || !score || !phi_star || !istar_len || !istar_inst || (n_configs && !configs) ||
-        gpus > 4096 || n_configs > (1u << 20))
-        return MAASO_EINVAL;
+// Alg. 1 for several independent problems at once (each with its own request subset and device
+// count): every greedy chain of every problem proposes its next tentative placement, and all of
+// them are scored in ONE batch, so a greedy step costs one trace replay however many problems
+// run side by side.  Problem p writes phi_star[p][0..gpus[p]], istar_len[p][..], istar_inst[p][..].
+struct DeployProblem {
+    uint32_t gpus;
+    int use_mask;
+    uint32_t class_mask;
+    double* phi_star;
+    uint32_t* istar_len;
+    uint32_t* istar_inst;
+};
+
+static int ins_deploy_multi(maaso_ctx* ctx, const maaso_trace* trace, const DeployProblem* prob, uint32_t n_prob,
+                            const maaso_config* configs, uint32_t n_configs, const maaso_score_params* score,
+                            uint32_t flags) {
     if (!ctx->has_profile) return fail(ctx, MAASO_ESTATE, "ins_deploy: no profile loaded");
     for (uint32_t c = 0; c < n_configs; c++)
         if (configs[c].strategy >= ctx->n_strategies || configs[c].batch < 1 || configs[c].batch > MAASO_WMAX)
             return fail(ctx, MAASO_EINVAL, "ins_deploy: configuration out of range");
-    for (uint32_t k = 0; k <= gpus; k++) { phi_star[k] = 0.0; istar_len[k] = 0; }
-    if (n_configs == 0) return MAASO_OK;
+    uint32_t max_gpus = 0;
+    bool any_mask = false;
+    for (uint32_t p = 0; p < n_prob; p++) {
+        for (uint32_t k = 0; k <= prob[p].gpus; k++) { prob[p].phi_star[k] = 0.0; prob[p].istar_len[k] = 0; }
+        if (prob[p].gpus > max_gpus) max_gpus = prob[p].gpus;
+        any_mask = any_mask || prob[p].use_mask;
+    }
+    if (n_configs == 0 || n_prob == 0) return MAASO_OK;
     DeviceGuard g(ctx->device);
 
     // device staging: offsets | inst | mask | results | scores | rejected-by-model
-    const size_t C = n_configs, cap_inst = C * (MAASO_MAX_INSTANCES + 1);
+    const size_t C = (size_t)n_configs * n_prob, cap_inst = C * (MAASO_MAX_INSTANCES + 1);
+    const size_t cap_cand = C > n_prob ? C : n_prob;
     size_t off = 0;
-    const size_t o_off = off;  off = align_up(off + (C + 1) * 4, 256);
+    const size_t o_off = off;  off = align_up(off + (cap_cand + 1) * 4, 256);
     const size_t o_inst = off; off = align_up(off + cap_inst * 4, 256);
-    const size_t o_mask = off; off = align_up(off + C * 4, 256);
-    const size_t o_res = off;  off = align_up(off + C * sizeof(maaso_result), 256);
-    const size_t o_sc = off;   off = align_up(off + C * 8, 256);
-    const size_t o_rbm = off;  off = align_up(off + C * MAASO_MAX_MODELS * 4, 256);
+    const size_t o_mask = off; off = align_up(off + cap_cand * 4, 256);
+    const size_t o_res = off;  off = align_up(off + cap_cand * sizeof(maaso_result), 256);
+    const size_t o_sc = off;   off = align_up(off + cap_cand * 8, 256);
+    const size_t o_rbm = off;  off = align_up(off + cap_cand * MAASO_MAX_MODELS * 4, 256);
     int rc = grow(ctx, &ctx->deploy, &ctx->deploy_bytes, off);
     if (rc != MAASO_OK) return rc;
     unsigned char* sb = static_cast<unsigned char*>(ctx->deploy);
     cudaStream_t st = ctx->own_stream;
 
-    std::vector<uint32_t> h_off(C + 1), h_inst, h_mask(C, class_mask), h_rbm(C * MAASO_MAX_MODELS);
-    std::vector<double> h_sc(C);
+    std::vector<uint32_t> h_off(cap_cand + 1), h_inst, h_mask(cap_cand), h_rbm(cap_cand * MAASO_MAX_MODELS);
+    std::vector<double> h_sc(cap_cand);
     auto run_batch = [&](uint32_t n_cand) -> int {
         cudaError_t e = cudaMemcpyAsync(sb + o_off, h_off.data(), (n_cand + 1) * 4, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess && !h_inst.empty())
             e = cudaMemcpyAsync(sb + o_inst, h_inst.data(), h_inst.size() * 4, cudaMemcpyHostToDevice, st);
-        if (e == cudaSuccess && use_mask)
+        if (e == cudaSuccess && any_mask)
             e = cudaMemcpyAsync(sb + o_mask, h_mask.data(), n_cand * 4, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) return cuda_fail(ctx, e, "ins_deploy: upload");
         maaso_cand_batch b;
         memset(&b, 0, sizeof(b));
         b.offsets = reinterpret_cast<const uint32_t*>(sb + o_off);
         b.inst = reinterpret_cast<const uint32_t*>(sb + o_inst);
-        b.class_mask = use_mask ? reinterpret_cast<const uint32_t*>(sb + o_mask) : nullptr;
+        b.class_mask = any_mask ? reinterpret_cast<const uint32_t*>(sb + o_mask) : nullptr;
         b.n_cand = n_cand;
         b.n_inst = h_inst.size();
-        b.budget = gpus;
+        b.budget = max_gpus;  // each chain's own device count is enforced below, on the host
         maaso_eval_opts o;
         memset(&o, 0, sizeof(o));
         o.flags = flags;
@@ -659,11 +675,14 @@ MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_
         if (e != cudaSuccess) return cuda_fail(ctx, e, "ins_deploy: download");
         return MAASO_OK;
     };
+    // a problem without a mask counts every class (masks are ignored anyway beyond 32 classes)
+    auto mask_of = [&](uint32_t p) { return prob[p].use_mask ? prob[p].class_mask : 0xFFFFFFFFu; };
 
     // R_res = R_x before anything is deployed: the empty placement rejects every request of R_x
-    h_off[0] = 0;
-    h_off[1] = 0;
-    rc = run_batch(1);
+    for (uint32_t p = 0; p <= n_prob; p++) h_off[p] = 0;
+    for (uint32_t p = 0; p < n_prob; p++) h_mask[p] = mask_of(p);
+    h_inst.clear();
+    rc = run_batch(n_prob);
     if (rc != MAASO_OK) return rc;
 
     struct Step {
@@ -678,36 +697,45 @@ MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_
         uint32_t unserved[MAASO_MAX_MODELS];
         double phi;
         uint32_t dev;
+        uint32_t gpus;  // device count of the chain's problem
+        uint32_t mask;
         int tentative;  // model of the tentative instance, -1 = chain finished
     };
-    std::vector<Chain> chains(C);
-    for (uint32_t c = 0; c < C; c++) {
-        Chain& ch = chains[c];
-        memset(ch.sat, 0, sizeof(ch.sat));
-        memcpy(ch.unserved, h_rbm.data(), sizeof(ch.unserved));
-        ch.phi = 0.0;
-        ch.dev = (uint32_t)ctx->h_devices[configs[c].strategy];
-        ch.tentative = 0;
-    }
+    std::vector<Chain> chains(C);  // chain p * n_configs + c
+    for (uint32_t p = 0; p < n_prob; p++)
+        for (uint32_t c = 0; c < n_configs; c++) {
+            Chain& ch = chains[(size_t)p * n_configs + c];
+            memset(ch.sat, 0, sizeof(ch.sat));
+            memcpy(ch.unserved, h_rbm.data() + (size_t)p * MAASO_MAX_MODELS, sizeof(ch.unserved));
+            ch.phi = 0.0;
+            ch.dev = (uint32_t)ctx->h_devices[configs[c].strategy];
+            ch.gpus = prob[p].gpus;
+            ch.mask = mask_of(p);
+            ch.tentative = 0;
+        }
     std::vector<uint32_t> batch_chain;
+    std::vector<char> batch_over;  // the tentative placement needs more devices than its problem has
     for (;;) {
         // every unfinished chain proposes its next tentative placement I' = I + (m', P, B)
         batch_chain.clear();
+        batch_over.clear();
         h_inst.clear();
-        for (uint32_t c = 0; c < C; c++) {
-            Chain& ch = chains[c];
+        for (size_t x = 0; x < C; x++) {
+            Chain& ch = chains[x];
+            const maaso_config& cf = configs[x % n_configs];
             if (ch.tentative < 0) continue;
             int mp = -1;  // model with the most unserved requests among the non-saturated ones
-            if ((uint64_t)ch.inst.size() * ch.dev < gpus && ch.inst.size() <= MAASO_MAX_INSTANCES)
+            if ((uint64_t)ch.inst.size() * ch.dev < ch.gpus && ch.inst.size() <= MAASO_MAX_INSTANCES)
                 for (uint32_t m = 0; m < ctx->n_models; m++)
                     if (!ch.sat[m] && (mp < 0 || ch.unserved[m] > ch.unserved[mp])) mp = (int)m;
             ch.tentative = mp;
             if (mp < 0) continue;
             h_off[batch_chain.size()] = (uint32_t)h_inst.size();
+            h_mask[batch_chain.size()] = ch.mask;
             h_inst.insert(h_inst.end(), ch.inst.begin(), ch.inst.end());
-            h_inst.push_back(((uint32_t)mp & 0xFu) | ((configs[c].strategy & 0xFFu) << 4) |
-                             ((configs[c].batch & 0xFFu) << 12));
-            batch_chain.push_back(c);
+            h_inst.push_back(((uint32_t)mp & 0xFu) | ((cf.strategy & 0xFFu) << 4) | ((cf.batch & 0xFFu) << 12));
+            batch_over.push_back(((uint64_t)ch.inst.size() + 1) * ch.dev > ch.gpus ? 1 : 0);
+            batch_chain.push_back((uint32_t)x);
         }
         if (batch_chain.empty()) break;
         h_off[batch_chain.size()] = (uint32_t)h_inst.size();
@@ -717,8 +745,11 @@ MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_
             Chain& ch = chains[batch_chain[j]];
             Step sp;
             sp.k = (uint32_t)ch.inst.size() * ch.dev;
-            if (h_sc[j] > ch.phi) {  // accept the new instance
-                ch.phi = h_sc[j];
+            // a placement beyond the problem's own device count is invalid (score -1), as it would be
+            // if the problem were scored alone with its device count as the budget
+            const double sc = batch_over[j] ? -1.0 : h_sc[j];
+            if (sc > ch.phi) {  // accept the new instance
+                ch.phi = sc;
                 ch.inst.push_back(h_inst[h_off[j + 1] - 1]);
                 memcpy(ch.unserved, h_rbm.data() + j * MAASO_MAX_MODELS, sizeof(ch.unserved));
             } else {
@@ -731,15 +762,29 @@ MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_
     }
     // Phi*[k] / I*[k]: replay the steps configuration by configuration, as the sequential algorithm
     // would have met them ("first strictly better wins")
-    for (uint32_t c = 0; c < C; c++)
-        for (const Step& sp : chains[c].steps)
-            if (sp.k <= gpus && sp.phi > phi_star[sp.k]) {
-                phi_star[sp.k] = sp.phi;
-                istar_len[sp.k] = sp.len;
-                for (uint32_t i = 0; i < sp.len && i < MAASO_MAX_INSTANCES; i++)
-                    istar_inst[(size_t)sp.k * MAASO_MAX_INSTANCES + i] = chains[c].inst[i];
-            }
+    for (uint32_t p = 0; p < n_prob; p++)
+        for (uint32_t c = 0; c < n_configs; c++) {
+            const Chain& ch = chains[(size_t)p * n_configs + c];
+            for (const Step& sp : ch.steps)
+                if (sp.k <= prob[p].gpus && sp.phi > prob[p].phi_star[sp.k]) {
+                    prob[p].phi_star[sp.k] = sp.phi;
+                    prob[p].istar_len[sp.k] = sp.len;
+                    for (uint32_t i = 0; i < sp.len && i < MAASO_MAX_INSTANCES; i++)
+                        prob[p].istar_inst[(size_t)sp.k * MAASO_MAX_INSTANCES + i] = ch.inst[i];
+                }
+        }
     return MAASO_OK;
+}
+
+MAASO_API int maaso_ins_deploy(maaso_ctx* ctx, const maaso_trace* trace, uint32_t gpus,
+                               const maaso_config* configs, uint32_t n_configs, int use_mask,
+                               uint32_t class_mask, const maaso_score_params* score, uint32_t flags,
+                               double* phi_star, uint32_t* istar_len, uint32_t* istar_inst) {
+    if (!ctx || !trace || !score || !phi_star || !istar_len || !istar_inst || (n_configs && !configs) ||
+        gpus > 4096 || n_configs > (1u << 20))
+        return MAASO_EINVAL;
+    const DeployProblem one{gpus, use_mask, class_mask, phi_star, istar_len, istar_inst};
+    return ins_deploy_multi(ctx, trace, &one, 1, configs, n_configs, score, flags);
 }
 
 // getPrunedConfigs: strategy dominance on the host copy of the tables, batch-cap Pareto front from
@@ -900,18 +945,19 @@ MAASO_API int maaso_partition(maaso_ctx* ctx, const maaso_trace* trace, uint32_t
     std::vector<uint32_t> ln_t(cells), ln_l(cells), ln_h(cells);
     std::vector<uint32_t> in_t(cells * MAASO_MAX_INSTANCES), in_l(cells * MAASO_MAX_INSTANCES),
         in_h(cells * MAASO_MAX_INSTANCES);
-    rc = maaso_ins_deploy(ctx, trace, gl_max, configs, n_configs, 1, mask_l, score, flags, phi_l.data(),
-                          ln_l.data(), in_l.data());
-    if (rc == MAASO_OK)
-        rc = maaso_ins_deploy(ctx, trace, gpus, configs, n_configs, 1, mask_t, score, flags, phi_t.data(),
-                              ln_t.data(), in_t.data());
+    // the loose, the tight and (if asked) the homogeneous problem are independent: their greedy
+    // chains advance side by side, one batch per step for all of them
+    if (!score || (n_configs && !configs) || n_configs > (1u << 20)) return MAASO_EINVAL;
+    DeployProblem probs[3] = {
+        {gl_max, 1, mask_l, phi_l.data(), ln_l.data(), in_l.data()},
+        {gpus, 1, mask_t, phi_t.data(), ln_t.data(), in_t.data()},
+        {gpus, 1, mask_t | mask_l, phi_h.data(), ln_h.data(), in_h.data()},
+    };
+    rc = ins_deploy_multi(ctx, trace, probs, baseline ? 3u : 2u, configs, n_configs, score, flags);
     double phi_opt = 0.0;
-    if (rc == MAASO_OK && baseline) {  // homogeneous deployment as the fallback
-        rc = maaso_ins_deploy(ctx, trace, gpus, configs, n_configs, 1, mask_t | mask_l, score, flags, phi_h.data(),
-                              ln_h.data(), in_h.data());
-        for (uint32_t k = 0; rc == MAASO_OK && k <= gpus; k++)
+    if (rc == MAASO_OK && baseline)  // homogeneous deployment as the fallback
+        for (uint32_t k = 0; k <= gpus; k++)
             if (phi_h[k] > phi_opt) phi_opt = phi_h[k];
-    }
     if (rc != MAASO_OK) return rc;
     out_g[0] = out_g[1] = 0;
     *len_t = *len_l = 0;
