@@ -65,6 +65,8 @@
 #define ORC_EINVARIANT 0x80000000u /* an internal invariant failed: the oracle is wrong */
 
 #define ORC_FLAG_PRED_OPTIMISTIC 1u
+#define ORC_FLAG_TBT_MAXGAP 4u    /* the TBT term of the hit test looks at the largest gap between two
+                                     consecutive tokens of the request instead of the mean gap */
 #define ORC_FLAG_ENGINE_FROZEN 2u /* the paper-literal engine: decode speed fixed at admission (below) */
 
 typedef struct {
@@ -100,6 +102,8 @@ typedef struct {
     uint32_t req;
     int64_t arrival, first_tok;
     int64_t fin_idx; /* value of the instance's step counter at which this request ends */
+    int64_t last_tok; /* time of its latest token */
+    int64_t max_gap;  /* largest gap between two consecutive tokens so far */
     uint32_t S;
     uint32_t cls;
 } slot_t;
@@ -122,6 +126,7 @@ typedef struct {
     int64_t *dump_first;
     int32_t *dump_inst;
     int bad; /* invariant violated */
+    int tbt_maxgap; /* hit test on the largest token gap (ORC_FLAG_TBT_MAXGAP) */
 } ctx_t;
 
 /* SplitMix64 output mixer (public domain, Steele/Lea/Flood) */
@@ -135,11 +140,13 @@ static uint64_t rotl64(uint64_t x, int r) { return (x << r) | (x >> (64 - r)); }
 
 /* A request leaves the system served: Phi_S indicator, latency and throughput sums. */
 static void complete(ctx_t *c, uint32_t inst_idx, uint32_t req, int64_t arrival, int64_t first_tok,
-                     int64_t t_fin, uint32_t S, uint32_t cls) {
+                     int64_t t_fin, uint32_t S, uint32_t cls, int64_t max_gap) {
     const orc_slo *k = &c->classes[cls];
     int64_t ttft = first_tok - arrival, e2e = t_fin - arrival, span = t_fin - first_tok;
-    int hit = (k->ttft_us < 0 || ttft <= k->ttft_us) &&
-              (k->tbt_us < 0 || span <= (int64_t)(S - 1) * k->tbt_us) &&
+    /* TBT term: mean gap (the normalised deadline of Sec. III-C as a per-token budget), or, as an
+     * option, the largest single gap (a request of one token has no gap) */
+    int tbt_ok = k->tbt_us < 0 || (c->tbt_maxgap ? max_gap <= k->tbt_us : span <= (int64_t)(S - 1) * k->tbt_us);
+    int hit = (k->ttft_us < 0 || ttft <= k->ttft_us) && tbt_ok &&
               (k->e2e_us < 0 || e2e <= k->e2e_us);
     orc_result *r = c->res;
     if (ttft < 0 || span < 0) c->bad = 1;
@@ -175,12 +182,21 @@ static void advance(ctx_t *c, inst_t *in, uint32_t inst_idx, int64_t t) {
             int64_t need = (t - in->T + s - 1) / s; /* ceil */
             if (need < k) k = need;
         }
+        for (uint32_t j = 0; j < in->B; j++) {
+            /* token gaps of this jump: the first one reaches back to the request's latest token (so it
+             * includes prefills that stalled the batch), the other k - 1 are s, which is not larger */
+            slot_t *sl = &in->slots[j];
+            if (!sl->used) continue;
+            int64_t gap = in->T + s - sl->last_tok;
+            if (gap > sl->max_gap) sl->max_gap = gap;
+            sl->last_tok = in->T + k * s;
+        }
         in->T += k * s;
         in->K += k;
         for (uint32_t j = 0; j < in->B; j++) {
             slot_t *sl = &in->slots[j];
             if (sl->used && sl->fin_idx == in->K) {
-                complete(c, inst_idx, sl->req, sl->arrival, sl->first_tok, in->T, sl->S, sl->cls);
+                complete(c, inst_idx, sl->req, sl->arrival, sl->first_tok, in->T, sl->S, sl->cls, sl->max_gap);
                 sl->used = 0;
                 in->w--;
             }
@@ -303,7 +319,8 @@ static void frozen_replay(ctx_t *c, const orc_profile *p, const uint32_t *inst, 
                 int64_t first_tok = clock + f->pre_base + (int64_t)(((uint64_t)f->pre_q16 * q->in_tokens + 32768u) >> 16);
                 int64_t t_end = first_tok + (len - 1) * speed;
                 f->busy[j] = 1; f->until[j] = t_end;
-                complete(c, pick, (uint32_t)r, q->arrival_us, first_tok, t_end, (uint32_t)len, q->cls);
+                complete(c, pick, (uint32_t)r, q->arrival_us, first_tok, t_end, (uint32_t)len, q->cls,
+                         len > 1 ? speed : 0); /* every gap of the request is `speed` */
                 break;
             }
             if (pick_start <= clock) c->bad = 1;
@@ -329,6 +346,7 @@ int orc_eval_candidate(const orc_profile *p, const orc_request *reqs, uint64_t n
     ctx_t c;
     memset(out, 0, sizeof(*out));
     c.classes = classes; c.res = out; c.bad = 0;
+    c.tbt_maxgap = (flags & ORC_FLAG_TBT_MAXGAP) != 0;
     c.dump_finish = dump_finish; c.dump_first = dump_first; c.dump_inst = dump_inst;
     for (uint64_t r = 0; r < n; r++) {
         if (dump_finish) dump_finish[r] = -2;
@@ -404,7 +422,7 @@ int orc_eval_candidate(const orc_profile *p, const orc_request *reqs, uint64_t n
                 inst_t *in = &I[best_i];
                 in->T += prefill_us(in, q->in_tokens);
                 if (S == 1) {
-                    complete(&c, best_i, (uint32_t)r, q->arrival_us, in->T, in->T, 1, q->cls);
+                    complete(&c, best_i, (uint32_t)r, q->arrival_us, in->T, in->T, 1, q->cls, 0);
                 } else {
                     uint32_t j = 0;
                     while (j < in->B && in->slots[j].used) j++;
@@ -412,6 +430,7 @@ int orc_eval_candidate(const orc_profile *p, const orc_request *reqs, uint64_t n
                     slot_t *sl = &in->slots[j];
                     sl->used = 1; sl->req = (uint32_t)r; sl->arrival = q->arrival_us;
                     sl->first_tok = in->T; sl->fin_idx = in->K + S - 1; sl->S = (uint32_t)S;
+                    sl->last_tok = in->T; sl->max_gap = 0;
                     sl->cls = q->cls;
                     in->w++;
                 }

@@ -33,6 +33,8 @@ def load_case(path):
     runs = [(raw["flags"], raw["expect"])]
     if "expect_flags0" in raw:
         runs.append((0, raw["expect_flags0"]))
+    if "expect_maxgap" in raw:                 # TBT term of the hit test on the largest token gap
+        runs.append((4, raw["expect_maxgap"]))
     if "expect_frozen" in raw:                 # the engine that fixes the decode speed at admission
         runs.append((2, raw["expect_frozen"]))
     return {"name": os.path.basename(path), "profile": prof, "classes": classes,

@@ -23,6 +23,7 @@ class _Inst:
         self.clock += int(self.step[len(self.running) - 1])
         keep = []
         for r in self.running:
+            r["stamps"].append(self.clock)    # every running request gets a token at the end of the step
             r["left"] -= 1
             if r["left"] == 0:
                 done(r, self.clock)
@@ -42,9 +43,10 @@ class _Inst:
         return self.clock + left * int(self.step[len(self.running) - 1])
 
 
-def simulate(profile, trace, classes, instances, class_mask=None, optimistic=False):
+def simulate(profile, trace, classes, instances, class_mask=None, optimistic=False, maxgap=False):
     """instances: list of (model, strategy, batch).  Returns a dict of statistics and
-    per-request lists finish / first / inst (-1 rejected, -2 not counted)."""
+    per-request lists finish / first / inst (-1 rejected, -2 not counted).
+    maxgap: the TBT term looks at the largest difference between consecutive token timestamps."""
     S_ = profile["n_strategies"]
     insts = []
     for (m, s, b) in instances:
@@ -62,9 +64,14 @@ def simulate(profile, trace, classes, instances, class_mask=None, optimistic=Fal
         def done(r, t):
             c = classes[r["cls"]]
             ttft, e2e, span = r["first"] - r["arrival"], t - r["arrival"], t - r["first"]
-            ok = ((lim(c["ttft_us"]) is None or ttft <= lim(c["ttft_us"])) and
-                  (lim(c["tbt_us"]) is None or r["S"] == 1 or
-                   Fraction(span, r["S"] - 1) <= lim(c["tbt_us"])) and
+            if maxgap:
+                ts = r["stamps"]
+                worst = max([b - a for a, b in zip(ts, ts[1:])], default=0)
+                tbt_ok = lim(c["tbt_us"]) is None or worst <= lim(c["tbt_us"])
+            else:
+                tbt_ok = (lim(c["tbt_us"]) is None or r["S"] == 1 or
+                          Fraction(span, r["S"] - 1) <= lim(c["tbt_us"]))
+            ok = ((lim(c["ttft_us"]) is None or ttft <= lim(c["ttft_us"])) and tbt_ok and
                   (lim(c["e2e_us"]) is None or e2e <= lim(c["e2e_us"])))
             st["n_served"] += 1
             st["n_hit"] += ok
@@ -118,7 +125,7 @@ def simulate(profile, trace, classes, instances, class_mask=None, optimistic=Fal
             if tier == 0:
                 ins = insts[idx]
                 ins.clock += ins.prefill(int(q["in_tokens"]))
-                rec = dict(req=k, arrival=arrival, first=ins.clock, left=S - 1, S=S, cls=cls)
+                rec = dict(req=k, arrival=arrival, first=ins.clock, left=S - 1, S=S, cls=cls, stamps=[ins.clock])
                 if S == 1:
                     done_on(idx)(rec, ins.clock)
                 else:
@@ -132,7 +139,7 @@ def simulate(profile, trace, classes, instances, class_mask=None, optimistic=Fal
     return st
 
 
-def simulate_frozen(profile, trace, classes, instances, class_mask=None, optimistic=False):
+def simulate_frozen(profile, trace, classes, instances, class_mask=None, optimistic=False, maxgap=False):
     """The engine that fixes a request's decode speed at admission, in a formulation that
     shares nothing with the C oracle's: no slots at all.  Every instance keeps the list of
     token timestamps of the requests admitted to it (one list per request, built token by
@@ -199,9 +206,12 @@ def simulate_frozen(profile, trace, classes, instances, class_mask=None, optimis
             ins["tokens"].append(stamps)
             t_first, t_end = stamps[0], stamps[-1]
             ttft, e2e = t_first - arrival, t_end - arrival
-            ok = ((lim(c["ttft_us"]) is None or ttft <= lim(c["ttft_us"])) and
-                  (lim(c["tbt_us"]) is None or S == 1 or
-                   Fraction(t_end - t_first, S - 1) <= lim(c["tbt_us"])) and
+            if maxgap:
+                worst = max([b - a for a, b in zip(stamps, stamps[1:])], default=0)
+                tbt_ok = lim(c["tbt_us"]) is None or worst <= lim(c["tbt_us"])
+            else:
+                tbt_ok = lim(c["tbt_us"]) is None or S == 1 or Fraction(t_end - t_first, S - 1) <= lim(c["tbt_us"])
+            ok = ((lim(c["ttft_us"]) is None or ttft <= lim(c["ttft_us"])) and tbt_ok and
                   (lim(c["e2e_us"]) is None or e2e <= lim(c["e2e_us"])))
             st["n_served"] += 1
             st["n_hit"] += ok

@@ -54,6 +54,10 @@ MUTANTS = [
      "int64_t t_end = first_tok + len * speed;"),
     ("frozen engine: optimistic estimate uses the current level", "tier_i == 0) s_pred = f->step[running];",
      "tier_i == 0) s_pred = f->step[running > 0 ? running - 1 : 0];"),
+    ("largest gap forgets the stall before the step", "int64_t gap = in->T + s - sl->last_tok;", "int64_t gap = s;"),
+    ("largest gap is not kept across jumps", "if (gap > sl->max_gap) sl->max_gap = gap;", "sl->max_gap = gap;"),
+    ("largest gap of a new request starts at the boundary", "sl->last_tok = in->T; sl->max_gap = 0;",
+     "sl->last_tok = in->T - prefill_us(in, q->in_tokens); sl->max_gap = 0;"),
     ("prefill does not stall the running batch", "in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {",
      "int64_t t_keep = in->T; in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {"),
 ]
@@ -100,6 +104,9 @@ def run_pins(mod):
         attempt(f"frozen token lists {seed}", pins.test_frozen_engine_against_token_lists, seed)
     attempt("frozen levels", pins.test_frozen_engine_levels_recomputed_from_the_dumps)
     attempt("frozen cap one", pins.test_frozen_engine_equals_default_engine_for_one_instance_with_cap_one)
+    for seed in (0, 1, 2, 3):
+        attempt(f"largest gap {seed}", pins.test_maxgap_against_token_timestamps, seed)
+    attempt("largest gap vs mean", pins.test_maxgap_only_changes_the_hit_test)
     attempt("histogram edges", pins.test_ttft_histogram_bin_edges)
     attempt("histogram counts", pins.test_ttft_histogram_counts_served_requests_only)
     attempt("percentiles", pins.test_ttft_percentiles_by_hand)

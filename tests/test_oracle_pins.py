@@ -202,6 +202,42 @@ def test_frozen_engine_levels_recomputed_from_the_dumps(oracle_mod):
                         assert t_fin - int(d["first_us"][row][r]) == (S - 1) * int(prof["step_us"][m, s, running])
 
 
+# ---- TBT term of the hit test on the largest token gap (flag 4) -------------------------------
+MAXGAP = 4
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_maxgap_against_token_timestamps(oracle_mod, seed):
+    """The token-by-token simulator keeps every token's timestamp; the largest difference between
+    neighbours decides the TBT term.  Tight limits so that stalls by prefills matter."""
+    prof, trace, classes, instances = _random_small_case(seed)
+    classes = gen.make_classes([(500_000, 14_000, None), (2_000_000, 30_000, None), (None, 60_000, 8_000_000)])
+    opt = seed % 2
+    res, d = run_one(oracle_mod, prof, trace, classes, instances, flags=MAXGAP | opt)
+    ref = simulate(prof, trace, classes, instances, optimistic=bool(opt), maxgap=True)
+    for key in SCALAR_KEYS:
+        assert int(res[key]) == ref[key], key
+    assert d["finish_us"].tolist() == ref["finish_us"]
+    res2, _ = run_one(oracle_mod, prof, trace, classes, instances, flags=MAXGAP | FROZEN | opt)
+    ref2 = simulate_frozen(prof, trace, classes, instances, optimistic=bool(opt), maxgap=True)
+    for key in SCALAR_KEYS:
+        assert int(res2[key]) == ref2[key], key
+
+
+def test_maxgap_only_changes_the_hit_test(oracle_mod):
+    """The largest gap is at least the mean gap: hits can only go down, nothing else moves."""
+    cfg = gen.make_config("tiny", n_req=400)
+    classes = gen.make_classes([(500_000, 12_000, None), (2_000_000, 20_000, None), (None, None, 180_000_000)])
+    a = oracle_mod.eval_placements(cfg["profile"], cfg["traces"][0], classes, cfg["offsets"], cfg["inst"], cfg["budget"], flags=1)
+    b = oracle_mod.eval_placements(cfg["profile"], cfg["traces"][0], classes, cfg["offsets"], cfg["inst"], cfg["budget"],
+                                   flags=1 | MAXGAP)
+    assert (b["n_hit"] <= a["n_hit"]).all() and int((a["n_hit"] - b["n_hit"]).sum()) > 0
+    for key in ("n_counted", "n_served", "n_rejected", "sum_ttft_us", "sum_e2e_us", "makespan_us", "tokens_out",
+                "checksum", "attempts"):
+        assert (a[key] == b[key]).all(), key
+    assert (b["n_cascade"] == b["n_served"] - b["n_hit"]).all()
+
+
 # ---- P4: invariants -----------------------------------------------------------------------
 def test_invariants_on_tiny_config(oracle_mod):
     cfg = gen.make_config("tiny")
