@@ -76,6 +76,12 @@ extern "C" {
                                       a placement with more than 32 instances gets MAASO_CAND_ETOOMANY;
                                       finish times must stay below 2^57 us (else MAASO_CAND_ELOOP). */
 
+#define MAASO_FLAG_TBT_MAXGAP 4u /* the TBT term of the hit test (Phi_S indicator) looks at the largest gap
+                                    between two consecutive tokens of a request, prefill stalls included,
+                                    instead of the mean gap; a request of one token has no gap.  The
+                                    distributor's prediction is unchanged.  Same limits as
+                                    MAASO_FLAG_ENGINE_FROZEN (lane-group mapping, at most 32 instances). */
+
 #define MAASO_FLAG_TEST_STALL 0x80000000u /* test hook for the bounded device-side waits: the trace copies
                                              are never issued and every wait is limited to about 0.1 s, so
                                              each valid candidate must come back with MAASO_CAND_ETIMEOUT

@@ -114,17 +114,19 @@ __device__ __forceinline__ uint32_t ttft_bin(int64_t t) {
 
 // A request leaves the system served at t_fin (Phi_S indicator and the latency / throughput sums).
 // `classes` holds (ttft, tbt, e2e) per class, negative = no limit.  Returns whether it was a hit.
+// max_gap: largest gap between two consecutive tokens of the request if the TBT term is to be
+// checked on it (MAASO_FLAG_TBT_MAXGAP), negative for the mean-gap form.
 __device__ __forceinline__ bool account_completion(Stats& st, const int64_t* classes, uint32_t inst,
                                                    uint32_t req, int64_t arrival, int64_t first_tok,
                                                    int64_t t_fin, uint32_t S, uint32_t cls,
-                                                   const Dump& dump) {
+                                                   const Dump& dump, int64_t max_gap) {
     const int64_t lim_ttft = classes[cls * 3 + 0];
     const int64_t lim_tbt = classes[cls * 3 + 1];
     const int64_t lim_e2e = classes[cls * 3 + 2];
     const int64_t ttft = first_tok - arrival, e2e = t_fin - arrival, span = t_fin - first_tok;
-    const bool hit = (lim_ttft < 0 || ttft <= lim_ttft) &&
-                     (lim_tbt < 0 || span <= (int64_t)(S - 1) * lim_tbt) &&
-                     (lim_e2e < 0 || e2e <= lim_e2e);
+    // TBT term: the mean gap between tokens, or (max_gap >= 0) the largest single gap
+    const bool tbt_ok = lim_tbt < 0 || (max_gap >= 0 ? max_gap <= lim_tbt : span <= (int64_t)(S - 1) * lim_tbt);
+    const bool hit = (lim_ttft < 0 || ttft <= lim_ttft) && tbt_ok && (lim_e2e < 0 || e2e <= lim_e2e);
     st.served++;
     st.hit += hit ? 1u : 0u;
     st.sum_ttft += ttft; st.max_ttft = max(st.max_ttft, ttft);
@@ -255,6 +257,14 @@ struct EvalParams {
     uint32_t* rej_by_model;  // [n_cand][MAASO_MAX_MODELS] or null
     uint32_t* ttft_hist;     // [n_cand][MAASO_TTFT_BINS] or null (zeroed before the kernels run)
 };
+
+// The usual form: TBT term on the mean gap.
+__device__ __forceinline__ bool account_completion(Stats& st, const int64_t* classes, uint32_t inst,
+                                                   uint32_t req, int64_t arrival, int64_t first_tok,
+                                                   int64_t t_fin, uint32_t S, uint32_t cls,
+                                                   const Dump& dump) {
+    return account_completion(st, classes, inst, req, arrival, first_tok, t_fin, S, cls, dump, (int64_t)-1);
+}
 
 __device__ __forceinline__ Dump dump_for(const EvalParams& P, uint32_t cand) {
     Dump d{nullptr, nullptr, nullptr, nullptr};

@@ -63,6 +63,7 @@ struct GroupSmem {
     uint4* qa;           // [kQueue][kGroupThreads] queued completions: first-token time, arrival time
     uint2* qb;           // [kQueue][kGroupThreads] request index, S | cls << 16
     int64_t* qf;         // [kQueue][kGroupThreads] finish time
+    int64_t* qg;         // [kQueue][kGroupThreads] largest token gap (largest-gap mode)
     int64_t* classes;    // [n_classes][3], negative = no limit (completion accounting)
     uint64_t* full_bar;  // [kStages]
     int32_t* steps;      // [n_rows][64]
@@ -71,9 +72,9 @@ struct GroupSmem {
     uint32_t* wsum;      // [warps] pool units each warp asks for
 };
 
-__host__ __device__ inline size_t group_smem_static(uint32_t n_rows, uint32_t n_classes, int tile_recs) {
+__host__ __device__ inline size_t group_smem_static(uint32_t n_rows, uint32_t n_classes, int tile_recs, bool maxgap) {
     size_t b = (size_t)kStages * tile_recs * 16 * kCookedWords;
-    b += (size_t)kQueue * kGroupThreads * (16 + 8 + 8);
+    b += (size_t)kQueue * kGroupThreads * (16 + 8 + 8 + (maxgap ? 8 : 0));
     b += (size_t)n_classes * 24;
     b += kStages * 8;
     b += (size_t)n_rows * 64 * 4;
@@ -82,7 +83,7 @@ __host__ __device__ inline size_t group_smem_static(uint32_t n_rows, uint32_t n_
 }
 
 __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows, uint32_t n_classes,
-                                           int tile_recs, uint32_t pool_bytes) {
+                                           int tile_recs, uint32_t pool_bytes, bool maxgap) {
     GroupSmem s;
     // every part that is read in 16-byte words first (all sizes are multiples of 16 bytes)
     s.pool = base;
@@ -95,6 +96,8 @@ __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows,
     base += (size_t)kQueue * kGroupThreads * 8;
     s.qf = reinterpret_cast<int64_t*>(base);
     base += (size_t)kQueue * kGroupThreads * 8;
+    s.qg = reinterpret_cast<int64_t*>(base);
+    if (maxgap) base += (size_t)kQueue * kGroupThreads * 8;
     s.classes = reinterpret_cast<int64_t*>(base);
     base += (size_t)n_classes * 24;
     s.full_bar = reinterpret_cast<uint64_t*>(base);
@@ -121,25 +124,33 @@ __device__ __forceinline__ void issue_tile(const GroupSmem& sm, const EvalParams
 }
 
 // Account the queued completions of the whole warp once some lane holds kFlushAt of them.
-__device__ __forceinline__ void flush_if_due(uint32_t& qn, LaneStats& ls, const LaneEnv& env, const int64_t* classes,
-                                             uint32_t sub, const Dump& dump) {
-    if (__any_sync(kFullMask, qn >= (uint32_t)kFlushAt)) {
+template <bool MAXGAP>
+__device__ __forceinline__ void flush_now(uint32_t& qn, LaneStats& ls, const LaneEnv& env, const int64_t* classes,
+                                          uint32_t sub, const Dump& dump) {
+    if (MAXGAP)
+        flush_queue_maxgap(&ls, env.qf, env.qa, env.qb, env.ovf, qn, classes, sub, dump.finish, dump.first, dump.inst,
+                           dump.hist);
+    else
         flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, qn, classes, sub, dump.finish, dump.first, dump.inst,
                     dump.hist);
-        qn = 0;
-    }
+    qn = 0;
+}
+template <bool MAXGAP>
+__device__ __forceinline__ void flush_if_due(uint32_t& qn, LaneStats& ls, const LaneEnv& env, const int64_t* classes,
+                                             uint32_t sub, const Dump& dump) {
+    if (__any_sync(kFullMask, qn >= (uint32_t)kFlushAt)) flush_now<MAXGAP>(qn, ls, env, classes, sub, dump);
 }
 
 // OPT: the distributor predicts with the step time right after admission (optimistic estimate).
 // Inst: LaneInst (default engine: decode speed follows the running count) or FrozenInst (speed
-// fixed at admission).  MINB: blocks per SM the register budget must allow: 4 for batches that
+// fixed at admission).  MAXGAP: the TBT term of the hit test looks at the largest token gap.  MINB: blocks per SM the register budget must allow: 4 for batches that
 // fill the GPU (128 registers), 3 for batches of one wave, which are bound by their longest
 // dependent chains and run a little faster without the spills of the tighter budget.
-template <bool OPT, class Inst, int MINB>
+template <bool OPT, class Inst, int MINB, bool MAXGAP>
 __global__ void __launch_bounds__(kGroupThreads, MINB)
 eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_bytes) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    const GroupSmem sm = carve(smem_raw, P.n_rows, P.n_classes, tile_recs, pool_bytes);
+    const GroupSmem sm = carve(smem_raw, P.n_rows, P.n_classes, tile_recs, pool_bytes, MAXGAP);
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     constexpr uint32_t kWarps = kGroupThreads / 32;
     // a wait is followed by a new choice, unless the engine and the estimate make that round redundant
@@ -170,6 +181,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
     env.pay_a = reinterpret_cast<uint4*>(lane_scratch + kLaneScratchA);
     env.pay_b = reinterpret_cast<uint2*>(lane_scratch + kLaneScratchB);
     env.ovf = lane_scratch + kLaneScratchOvf;
+    env.qg = MAXGAP ? sm.qg + tid : nullptr;
+    env.mg = nullptr;
+    env.dl = nullptr;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
     const uint32_t n_tiles = (P.n_req + tile_recs - 1) / tile_recs;
     uint32_t tile_seq = 0;  // tiles consumed so far by this warp (same in every warp)
@@ -248,7 +262,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         // pool cannot hold use their global scratch instead
         {
             const uint32_t nblk = has ? (in.B + 7u) >> 3 : 0u;
-            const uint32_t units = has ? (nblk + 1u) * Inst::kKeyWords : 0u;
+            // largest-gap mode of the default engine: two more 8-byte words per slot after the minima
+            const uint32_t gap_units = MAXGAP ? nblk * 2u * Inst::kGapWords : 0u;  // 8 slots x words x 4 B / 32 B
+            const uint32_t units = has ? (nblk + 1u) * Inst::kKeyWords + gap_units : 0u;
             uint32_t incl = units;
             for (uint32_t o = 1; o < 32u; o <<= 1) {
                 const uint32_t v = __shfl_up_sync(kFullMask, incl, o);
@@ -265,6 +281,10 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
             env.keys = reinterpret_cast<uint32_t*>(region);
             env.bm_lo = reinterpret_cast<uint4*>(region + (size_t)nblk * kKeyUnitBytes * Inst::kKeyWords);
             env.bm_hi = env.bm_lo + 1;
+            if (MAXGAP && Inst::kGapWords) {
+                env.mg = reinterpret_cast<uint64_t*>(region + (size_t)(nblk + 1u) * kKeyUnitBytes * Inst::kKeyWords);
+                env.dl = env.mg + 8u * nblk;
+            }
             const uint4 e4 = make_uint4(kKeyEmpty, kKeyEmpty, kKeyEmpty, kKeyEmpty);
             for (uint32_t i = 0; i < 2u * units; i++) reinterpret_cast<uint4*>(region)[i] = e4;
         }
@@ -277,6 +297,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         LaneStats ls;
         ls.st.clear();
         for (int i = 0; i < 8; i++) ls.hbc[i] = 0;
+        ls.qg = env.qg;  // read by the largest-gap form of the flush only
         uint64_t rej_sum = 0;  // checksum terms of rejected requests
         int64_t now = 0;
         uint32_t n_counted = 0, n_rejected = 0, status = 0;
@@ -302,7 +323,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
             // a warp without a candidate only keeps the tile pipeline going
             for (uint32_t ri = warp_has_work ? 0u : recs; ri < recs; ri++) {
                 // statistics of completed requests: every fourth request, if some lane's queue is nearly full
-                if ((ri & 3u) == 0u) flush_if_due(in.qn, ls, env, sm.classes, sub, dump);
+                if ((ri & 3u) == 0u) flush_if_due<MAXGAP>(in.qn, ls, env, sm.classes, sub, dump);
                 const uint4* rec = tile + (size_t)ri * kCookedWords;
                 const uint4 r0 = rec[0], r1 = rec[1], r2 = rec[2];
                 // All 32 lanes walk the trace together and every warp-level operation below uses
@@ -326,7 +347,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                         tries++;
                     }
                     if (pending && elig) {
-                        lane_advance(in, now, false, env, status);
+                        lane_advance<MAXGAP>(in, now, false, env, status);
                         key = lane_predict(in, q, pre, now, OPT, t0, first);
                     }
                     const ArgMin am = group_argmin(key, first, gmask, G, own);
@@ -346,7 +367,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                             }
                             pending = false;
                         } else if (am.tier == 0) {
-                            if ((int)lane == am.winner) lane_admit(in, q, req, pre, now, env, status);
+                            if ((int)lane == am.winner) lane_admit<MAXGAP>(in, q, req, pre, now, env, status);
                             pending = false;
                         } else {
                             // every capable instance is full: wait until the chosen slot frees (the
@@ -359,8 +380,8 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                                 // feasible.  The second round is only counted; other clocks catch up lazily.
                                 attempts++;  // the second round, counted only
                                 if ((int)lane == am.winner) {
-                                    lane_advance(in, now, false, env, status);
-                                    lane_admit(in, q, req, pre, now, env, status);
+                                    lane_advance<MAXGAP>(in, now, false, env, status);
+                                    lane_admit<MAXGAP>(in, q, req, pre, now, env, status);
                                 }
                                 pending = false;
                             } else if (tries >= kAttemptCap) {
@@ -390,14 +411,10 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
 
         // drain, account what is still queued, reduce over the group, write the record
         __syncwarp();
-        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first, dump.inst,
-                    dump.hist);
-        in.qn = 0;
-        if (has && status == 0) lane_advance(in, 0, true, env, status);
+        flush_now<MAXGAP>(in.qn, ls, env, sm.classes, sub, dump);
+        if (has && status == 0) lane_advance<MAXGAP>(in, 0, true, env, status);
         __syncwarp();
-        flush_queue(&ls, env.qf, env.qa, env.qb, env.ovf, in.qn, sm.classes, sub, dump.finish, dump.first, dump.inst,
-                    dump.hist);
-        in.qn = 0;
+        flush_now<MAXGAP>(in.qn, ls, env, sm.classes, sub, dump);
         Stats st = ls.st;
         st.checksum += rej_sum;
         uint32_t h[8];
@@ -424,15 +441,16 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
 }
 
 using GroupKernel = void (*)(const EvalParams, const int, const uint32_t);
-template <int MINB>
+template <int MINB, bool MAXGAP>
 static GroupKernel group_kernel_of(uint32_t flags) {
     const bool opt = (flags & MAASO_FLAG_PRED_OPTIMISTIC) != 0;
     if (flags & MAASO_FLAG_ENGINE_FROZEN)
-        return opt ? eval_group_kernel<true, FrozenInst, MINB> : eval_group_kernel<false, FrozenInst, MINB>;
-    return opt ? eval_group_kernel<true, LaneInst, MINB> : eval_group_kernel<false, LaneInst, MINB>;
+        return opt ? eval_group_kernel<true, FrozenInst, MINB, MAXGAP> : eval_group_kernel<false, FrozenInst, MINB, MAXGAP>;
+    return opt ? eval_group_kernel<true, LaneInst, MINB, MAXGAP> : eval_group_kernel<false, LaneInst, MINB, MAXGAP>;
 }
 static GroupKernel group_kernel_for(uint32_t flags, int blocks_per_sm) {
-    return blocks_per_sm >= 4 ? group_kernel_of<4>(flags) : group_kernel_of<3>(flags);
+    if (flags & MAASO_FLAG_TBT_MAXGAP) return group_kernel_of<4, true>(flags);  // one register budget for this mode
+    return blocks_per_sm >= 4 ? group_kernel_of<4, false>(flags) : group_kernel_of<3, false>(flags);
 }
 
 // Shared memory of one block: the fixed parts plus a key pool that fills what is left when
@@ -440,13 +458,16 @@ static GroupKernel group_kernel_for(uint32_t flags, int blocks_per_sm) {
 // 128 lanes with 64 slots each can use.
 static size_t group_smem_bytes(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm,
                                uint32_t* pool_bytes) {
-    const size_t fixed = group_smem_static(P.n_rows, P.n_classes, tile_recs);
+    const size_t fixed = group_smem_static(P.n_rows, P.n_classes, tile_recs, (P.flags & MAASO_FLAG_TBT_MAXGAP) != 0);
     size_t budget = (size_t)smem_per_sm / (size_t)blocks_per_sm;
     budget = budget > 1024 ? budget - 1024 : 0;
     if (budget > 227u * 1024u) budget = 227u * 1024u;
     size_t pool = budget > fixed ? budget - fixed : 0;
     pool -= pool % 128;
-    const size_t all = (size_t)kGroupThreads * 9 * kKeyUnitBytes * ((P.flags & MAASO_FLAG_ENGINE_FROZEN) ? 2 : 1);
+    size_t lane_units = 9;  // 8 key blocks + the block minima
+    if (P.flags & MAASO_FLAG_ENGINE_FROZEN) lane_units = 18;
+    else if (P.flags & MAASO_FLAG_TBT_MAXGAP) lane_units = 9 + 4 * 8;
+    const size_t all = (size_t)kGroupThreads * lane_units * kKeyUnitBytes;
     if (pool > all) pool = all;
     *pool_bytes = (uint32_t)pool;
     return fixed + pool;

@@ -18,6 +18,7 @@ constexpr uint64_t kKey64Empty = ~0ull;
 struct FrozenInst {
     static constexpr bool kAlwaysLoop = true;   // the single-round shortcut of the default engine does not hold here
     static constexpr uint32_t kKeyWords = 2;    // 32-bit words per slot key
+    static constexpr uint32_t kGapWords = 0;    // every gap of a request is its fixed speed: nothing to track
     uint64_t kmin;    // smallest slot key (the slot that frees next), kKey64Empty when idle
     uint64_t mask;    // busy slots; bits at and above B are always set
     uint32_t w;       // busy slots (requests running at the time of the last release)
@@ -62,6 +63,7 @@ __device__ __forceinline__ void frozen_release(FrozenInst& in, const LaneEnv& en
 
 // Free every slot whose request has finished by `now`.  Nothing to drain at the end of the
 // trace: every admitted request was accounted at its admission.
+template <bool MAXGAP>
 __device__ __forceinline__ void lane_advance(FrozenInst& in, int64_t now, bool drain, const LaneEnv& env,
                                              uint32_t& status) {
     (void)status;
@@ -95,10 +97,12 @@ __device__ __forceinline__ uint32_t lane_predict(const FrozenInst& in, const Coo
 
 // Admission at `now` into a free slot: the speed is the table step of the level running + 1 and
 // stays; the slot is held until the finish time (also for a request of one token).
+template <bool MAXGAP>
 __device__ __forceinline__ void lane_admit(FrozenInst& in, const CookedReq& q, uint32_t req, int64_t pre, int64_t now,
                                            const LaneEnv& env, uint32_t& status) {
     const int64_t first_tok = now + pre;
-    const int64_t t_end = first_tok + (int64_t)((uint64_t)q.Sm1 * (uint32_t)in.step[in.w]);
+    const uint32_t speed = (uint32_t)in.step[in.w];
+    const int64_t t_end = first_tok + (int64_t)((uint64_t)q.Sm1 * speed);
     if (((uint64_t)t_end >> 57) != 0) {  // beyond what a slot key can hold
         status = MAASO_CAND_ELOOP;
         return;
@@ -117,7 +121,7 @@ __device__ __forceinline__ void lane_admit(FrozenInst& in, const CookedReq& q, u
     const uint4 pa = make_uint4((uint32_t)first_tok, (uint32_t)((uint64_t)first_tok >> 32), (uint32_t)q.arrival,
                                 (uint32_t)((uint64_t)q.arrival >> 32));
     const uint2 pb = make_uint2(req, (q.Sm1 + 1u) | (q.cls << 16));
-    lane_push_now(in, env, t_end, pa, pb, status);
+    lane_push_now<MAXGAP>(in, env, t_end, pa, pb, MAXGAP ? (q.Sm1 ? (int64_t)speed : 0) : -1, status);
 }
 
 }  // namespace maaso

@@ -39,18 +39,21 @@ constexpr int kKeyUnitBytes = 32;              // pool unit: one block of 8 keys
 constexpr int kQueue = MAASO_QUEUE;            // queued completions per lane in shared memory
 constexpr int kFlushAt = MAASO_FLUSH_AT;       // the warp accounts its queues once some lane holds this many
 constexpr int kQueueOvf = 72;                  // further entries per lane in global scratch
+constexpr int kOvfEntryBytes = 48;             // overflow entry: finish, req, S|cls; first token, arrival; largest gap
 // Per-lane global scratch: payload A [64 slots][2] x 16 B, payload B [64][2] x 8 B, queue
-// overflow x 32 B, and room for 64 keys + 8 block minima if the shared-memory pool is full.
+// overflow x 48 B, and room for a lane's pool slice if the shared-memory pool is full (at most
+// 64 keys + 8 block minima of 8 bytes, or 64 keys + 8 minima of 4 bytes + 64 x 16 bytes of gap data).
 constexpr size_t kLaneScratchA = 0;
 constexpr size_t kLaneScratchB = 64 * 2 * 16;
 constexpr size_t kLaneScratchOvf = kLaneScratchB + 64 * 2 * 8;
-constexpr size_t kLaneScratchKeys = kLaneScratchOvf + (size_t)kQueueOvf * 32;
-constexpr size_t kLaneScratchBytes = kLaneScratchKeys + 2 * 9 * kKeyUnitBytes + 32;  // keys of either engine
+constexpr size_t kLaneScratchKeys = kLaneScratchOvf + (size_t)kQueueOvf * kOvfEntryBytes;
+constexpr size_t kLaneScratchBytes = kLaneScratchKeys + (9 + 4 * 8) * kKeyUnitBytes + 32;
 static_assert(kLaneScratchBytes % 32 == 0 && kLaneScratchKeys % 16 == 0, "lane scratch layout");
 
 struct LaneInst {
     static constexpr bool kAlwaysLoop = false;  // a wait is resolved in one round under the worst-case estimate
     static constexpr uint32_t kKeyWords = 1;    // 32-bit words per slot key
+    static constexpr uint32_t kGapWords = 4;    // 32-bit words per slot of gap data (largest-gap mode only)
     int64_t T;        // clock, always a decode-step boundary (may lag `now` while the instance is full)
     int64_t tc;       // time of the next completion if nobody is admitted (valid while w > 0)
     uint32_t K;       // decode steps done at T since the counter last restarted
@@ -62,6 +65,8 @@ struct LaneInst {
     uint32_t qn;      // completions waiting in this lane's queue
     uint64_t mask;    // occupied slots; bits at and above B are always set
     uint64_t gen;     // per slot: which of its two scratch entries the current occupant uses
+    uint64_t stall;   // largest-gap mode: prefill time since the instance's latest decode-step end
+    bool dirty;       // largest-gap mode: an admission or a retirement happened since the gaps were last folded in
     const int32_t* step;  // shared-memory row: step[w-1] = one decode step with w running
     uint32_t stepB;   // step[B-1]
     uint32_t pre_base, pre_q16;
@@ -78,13 +83,17 @@ struct LaneEnv {
     uint2* qb;               // entry j at qb[j * kGroupThreads] = request index, S | cls << 16
     uint4* pay_a;            // global scratch [64][2]: first-token time, arrival time
     uint2* pay_b;            // global scratch [64][2]: request index, S | cls << 16
-    unsigned char* ovf;      // this lane's queue overflow (global scratch, 32-byte entries)
+    unsigned char* ovf;      // this lane's queue overflow (global scratch, kOvfEntryBytes each)
+    int64_t* qg;             // largest-gap mode: entry j at qg[j * kGroupThreads] = largest token gap; else null
+    uint64_t* mg;            // largest-gap mode: per slot, largest token gap so far (pool slice, after the minima)
+    uint64_t* dl;            // largest-gap mode: per slot, time from the latest step end to the slot's latest token
 };
 
 // Per-lane sums of completed requests; only flush_queue touches them.
 struct LaneStats {
     Stats st;
-    uint32_t hbc[8];  // hits by class
+    uint32_t hbc[8];    // hits by class
+    const int64_t* qg;  // the lane's queue column of largest token gaps, null outside the largest-gap mode
 };
 
 // Asynchronous copies global -> shared: no register, nothing waits for them until a wait.
@@ -123,20 +132,23 @@ __device__ __forceinline__ uint32_t* bm_entry(const LaneEnv& env, uint32_t b) {
 
 // A running request has left the instance at t_fin: queue the finish time and start the
 // copies of what it remembered (scratch entry `idx` = 2 * slot + generation).
+template <bool MAXGAP>
 __device__ __forceinline__ void lane_push_slot(LaneInst& in, const LaneEnv& env, int64_t t_fin, uint32_t idx,
-                                               uint32_t& status) {
+                                               int64_t gap, uint32_t& status) {
     const uint32_t j = in.qn;
     if (j < (uint32_t)kQueue) {
         env.qf[j * kGroupThreads] = t_fin;
+        if (MAXGAP) env.qg[j * kGroupThreads] = gap;
         async_copy16(env.qa + j * kGroupThreads, env.pay_a + idx);
         async_copy8(env.qb + j * kGroupThreads, env.pay_b + idx);
         async_commit_keep_one();
     } else if (j < (uint32_t)(kQueue + kQueueOvf)) {
         const uint4 a = env.pay_a[idx];
         const uint2 b = env.pay_b[idx];
-        uint4* o = reinterpret_cast<uint4*>(env.ovf + (size_t)(j - kQueue) * 32);
+        uint4* o = reinterpret_cast<uint4*>(env.ovf + (size_t)(j - kQueue) * kOvfEntryBytes);
         o[0] = make_uint4((uint32_t)t_fin, (uint32_t)((uint64_t)t_fin >> 32), b.x, b.y);
         o[1] = a;
+        if (MAXGAP) o[2] = make_uint4((uint32_t)gap, (uint32_t)((uint64_t)gap >> 32), 0u, 0u);
     } else {
         status = MAASO_CAND_ELOOP;  // cannot happen: at most 64 completions per lane between flushes
         return;
@@ -145,18 +157,20 @@ __device__ __forceinline__ void lane_push_slot(LaneInst& in, const LaneEnv& env,
 }
 
 // Same for a request that completes at admission (one output token): everything is in registers.
-template <class Inst>
+template <bool MAXGAP, class Inst>
 __device__ __forceinline__ void lane_push_now(Inst& in, const LaneEnv& env, int64_t t_fin, uint4 a, uint2 b,
-                                              uint32_t& status) {
+                                              int64_t gap, uint32_t& status) {
     const uint32_t j = in.qn;
     if (j < (uint32_t)kQueue) {
         env.qf[j * kGroupThreads] = t_fin;
+        if (MAXGAP) env.qg[j * kGroupThreads] = gap;
         env.qa[j * kGroupThreads] = a;
         env.qb[j * kGroupThreads] = b;
     } else if (j < (uint32_t)(kQueue + kQueueOvf)) {
-        uint4* o = reinterpret_cast<uint4*>(env.ovf + (size_t)(j - kQueue) * 32);
+        uint4* o = reinterpret_cast<uint4*>(env.ovf + (size_t)(j - kQueue) * kOvfEntryBytes);
         o[0] = make_uint4((uint32_t)t_fin, (uint32_t)((uint64_t)t_fin >> 32), b.x, b.y);
         o[1] = a;
+        if (MAXGAP) o[2] = make_uint4((uint32_t)gap, (uint32_t)((uint64_t)gap >> 32), 0u, 0u);
     } else {
         status = MAASO_CAND_ELOOP;
         return;
@@ -165,36 +179,40 @@ __device__ __forceinline__ void lane_push_now(Inst& in, const LaneEnv& env, int6
 }
 
 // Statistics of the queued completions (Phi_S indicator, latency and throughput sums), by
-// all lanes of the warp together; every lane handles its own `n` entries.  Out of line on
-// purpose: the sums stay in local memory and the replay loop stays small.
-__device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
-                                         const unsigned char* ovf, uint32_t n, const int64_t* classes,
-                                         uint32_t inst_idx, int64_t* dump_finish, int64_t* dump_first,
-                                         int32_t* dump_inst, uint32_t* hist) {
+// all lanes of the warp together; every lane handles its own `n` entries.
+template <bool MAXGAP>
+__device__ __forceinline__ void flush_queue_body(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
+                                                 const unsigned char* ovf, uint32_t n, const int64_t* classes,
+                                                 uint32_t inst_idx, int64_t* dump_finish, int64_t* dump_first,
+                                                 int32_t* dump_inst, uint32_t* hist) {
     async_copies_done();
     Stats st = ls->st;
     const Dump no_dump{nullptr, nullptr, nullptr, nullptr};
     const bool dumping = dump_finish || dump_first || dump_inst || hist;
     for (uint32_t j = 0; j < n; j++) {
-        int64_t t_fin;
+        int64_t t_fin, gap = -1;  // gap stays negative unless the TBT term is checked on the largest gap
         uint4 a;
         uint2 b;
         if (j < (uint32_t)kQueue) {
             t_fin = qf[j * kGroupThreads];
             a = qa[j * kGroupThreads];
             b = qb[j * kGroupThreads];
+            if (MAXGAP) gap = ls->qg[j * kGroupThreads];
         } else {
-            const uint4* o = reinterpret_cast<const uint4*>(ovf + (size_t)(j - kQueue) * 32);
+            const uint4* o = reinterpret_cast<const uint4*>(ovf + (size_t)(j - kQueue) * kOvfEntryBytes);
             const uint4 h = o[0];
             t_fin = (int64_t)(((uint64_t)h.y << 32) | h.x);
             a = o[1];
             b = make_uint2(h.z, h.w);
+            if (MAXGAP) { const uint4 x = o[2]; gap = (int64_t)(((uint64_t)x.y << 32) | x.x); }
         }
         const int64_t first = (int64_t)(((uint64_t)a.y << 32) | a.x);
         const int64_t arrival = (int64_t)(((uint64_t)a.w << 32) | a.z);
         const uint32_t cls = b.y >> 16;
-        if (account_completion(st, classes, inst_idx, b.x, arrival, first, t_fin, b.y & 0xFFFFu, cls, no_dump))
-            ls->hbc[cls < 7 ? cls : 7]++;
+        bool hit;
+        if (MAXGAP) hit = account_completion(st, classes, inst_idx, b.x, arrival, first, t_fin, b.y & 0xFFFFu, cls, no_dump, gap);
+        else hit = account_completion(st, classes, inst_idx, b.x, arrival, first, t_fin, b.y & 0xFFFFu, cls, no_dump);
+        if (hit) ls->hbc[cls < 7 ? cls : 7]++;
         if (dumping) {
             if (dump_finish) dump_finish[b.x] = t_fin;
             if (dump_first) dump_first[b.x] = first;
@@ -205,15 +223,49 @@ __device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const
     ls->st = st;
 }
 
+// Out of line on purpose: the sums stay in local memory and the replay loop stays small.  One
+// copy per form of the TBT term, so that the usual one carries nothing of the other.
+__device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
+                                         const unsigned char* ovf, uint32_t n, const int64_t* classes,
+                                         uint32_t inst_idx, int64_t* dump_finish, int64_t* dump_first,
+                                         int32_t* dump_inst, uint32_t* hist) {
+    flush_queue_body<false>(ls, qf, qa, qb, ovf, n, classes, inst_idx, dump_finish, dump_first, dump_inst, hist);
+}
+__device__ __noinline__ void flush_queue_maxgap(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
+                                                const unsigned char* ovf, uint32_t n, const int64_t* classes,
+                                                uint32_t inst_idx, int64_t* dump_finish, int64_t* dump_first,
+                                                int32_t* dump_inst, uint32_t* hist) {
+    flush_queue_body<true>(ls, qf, qa, qb, ovf, n, classes, inst_idx, dump_finish, dump_first, dump_inst, hist);
+}
+
 __device__ __forceinline__ void lane_reset(LaneInst& in, const int32_t* steps) {
     in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = kKeyEmpty; in.sw = 1; in.rsw = 1.0f; in.qn = 0;
-    in.mask = ~0ull; in.gen = 0;
+    in.mask = ~0ull; in.gen = 0; in.stall = 0; in.dirty = false;
     in.B = 1; in.model = 0xFFFFFFFFu; in.step = steps; in.stepB = 1; in.pre_base = 0; in.pre_q16 = 0;
 }
 
 // The counter K has just reached the smallest end index (clock = in.T).  Retire every
 // request that ends here, one per round (the smallest key names its slot), fix the block
 // minima, the level and the cached next completion.
+// Largest-gap mode.  The instance is about to take its first decode step(s) since an admission or a
+// retirement: every running request's next token comes `stall` (prefills since the latest step
+// end) plus one step after that step end, minus what the request itself has already waited there
+// (a request admitted at this boundary got its first token part-way through the stall).  Further
+// steps of the same stretch are not longer.  Folded into every slot of the lane's blocks; slots
+// that are empty hold garbage until an admission resets them.
+__device__ __forceinline__ void gaps_fold(LaneInst& in, const LaneEnv& env) {
+    const uint64_t g = in.stall + in.sw;
+    const uint32_t n = 8u * ((in.B + 7u) >> 3);
+    for (uint32_t i = 0; i < n; i++) {
+        const uint64_t cand = g - env.dl[i];
+        env.mg[i] = max(env.mg[i], cand);
+        env.dl[i] = 0;
+    }
+    in.stall = 0;
+    in.dirty = false;
+}
+
+template <bool MAXGAP>
 __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, uint32_t& status) {
     const uint32_t Kc = in.K;
     do {
@@ -233,8 +285,10 @@ __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, ui
         in.kmin = min8(mv);
         in.mask &= ~(1ull << slot);
         in.w--;
-        lane_push_slot(in, env, in.T, 2u * slot + (uint32_t)((in.gen >> slot) & 1ull), status);
+        lane_push_slot<MAXGAP>(in, env, in.T, 2u * slot + (uint32_t)((in.gen >> slot) & 1ull),
+                               MAXGAP ? (int64_t)env.mg[slot] : -1, status);
     } while ((in.kmin >> 6) == Kc);
+    if (MAXGAP) in.dirty = true;  // the level changes: the next step has another length
     if (in.w > 0) {
         in.sw = (uint32_t)in.step[in.w - 1];
         in.rsw = rcp_approx((float)in.sw);
@@ -246,12 +300,14 @@ __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, ui
 // A full instance whose next completion lies beyond `now` is left untouched: nothing
 // observable depends on its clock until a slot frees, and later updates land on the same
 // step boundaries.
+template <bool MAXGAP>
 __device__ __forceinline__ void lane_advance(LaneInst& in, int64_t now, bool drain, const LaneEnv& env,
                                              uint32_t& status) {
     while (in.w > 0 && (drain || in.T < now)) {
         if (!drain && now <= in.tc - (int64_t)in.sw) {
             // the clock reaches `now` before anything completes
             if (in.w < in.B) {
+                if (MAXGAP && in.dirty) gaps_fold(in, env);
                 // fewer steps than the longest request has tokens: the quotient fits the fast exact division
                 const uint32_t k = ceil_div_small(now - in.T, in.sw, in.rsw);
                 in.T += (int64_t)k * (int64_t)in.sw;
@@ -259,11 +315,15 @@ __device__ __forceinline__ void lane_advance(LaneInst& in, int64_t now, bool dra
             }
             break;
         }
+        if (MAXGAP && in.dirty) gaps_fold(in, env);
         in.K = in.kmin >> 6;
         in.T = in.tc;
-        lane_retire(in, env, status);
+        lane_retire<MAXGAP>(in, env, status);
     }
-    if (!drain && in.w == 0 && in.T < now) in.T = now;  // an idle instance starts at once
+    if (!drain && in.w == 0 && in.T < now) {  // an idle instance starts at once
+        in.T = now;
+        if (MAXGAP) in.stall = 0;
+    }
 }
 
 // One request as the replay loop sees it (decoded from a prepared trace record).
@@ -336,16 +396,21 @@ __device__ __noinline__ uint32_t lane_rebase(uint32_t* keys, uint32_t nslots, ui
 }
 
 // "map": prefill at the step boundary (running decodes stall), then occupy a free slot.
+template <bool MAXGAP>
 __device__ __forceinline__ void lane_admit(LaneInst& in, const CookedReq& q, uint32_t req, int64_t pre, int64_t now,
                                            const LaneEnv& env, uint32_t& status) {
     (void)now;  // the instance's own clock is at or after `now`
     in.T += pre;
+    if (MAXGAP) {  // the prefill delays the next token of everybody who is running here
+        in.stall += (uint64_t)pre;
+        in.dirty = true;
+    }
     const uint4 pa = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)q.arrival,
                                 (uint32_t)((uint64_t)q.arrival >> 32));
     const uint2 pb = make_uint2(req, (q.Sm1 + 1u) | (q.cls << 16));
     if (q.Sm1 == 0) {  // done at the end of its prefill, never occupies a slot
         in.tc += pre;
-        lane_push_now(in, env, in.T, pa, pb, status);
+        lane_push_now<MAXGAP>(in, env, in.T, pa, pb, MAXGAP ? 0 : -1, status);
         return;
     }
     if (in.w == 0) in.K = 0;  // no live end index: the counter restarts
@@ -356,6 +421,10 @@ __device__ __forceinline__ void lane_admit(LaneInst& in, const CookedReq& q, uin
     const uint32_t slot = (uint32_t)(__ffsll((long long)~in.mask) - 1);
     const uint32_t key = ((in.K + q.Sm1) << 6) | slot;
     env.keys[slot] = key;
+    if (MAXGAP) {  // no gap yet; its first token came `stall` after the latest step end
+        env.mg[slot] = 0;
+        env.dl[slot] = in.stall;
+    }
     in.gen ^= 1ull << slot;
     const uint32_t idx = 2u * slot + (uint32_t)((in.gen >> slot) & 1ull);
     env.pay_a[idx] = pa;

@@ -364,10 +364,10 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     if (opts) o = *opts;
     if (o.mapping > MAASO_MAP_GROUP) return fail(ctx, MAASO_EINVAL, "eval: unknown mapping");
     if (o.dump_n && !o.dump_cand_idx) return fail(ctx, MAASO_EINVAL, "eval: dump_n without dump_cand_idx");
-    if (o.flags & ~(MAASO_FLAG_PRED_OPTIMISTIC | MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TEST_STALL))
+    if (o.flags & ~(MAASO_FLAG_PRED_OPTIMISTIC | MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_TEST_STALL))
         return fail(ctx, MAASO_EINVAL, "eval: unknown flag");
-    if ((o.flags & MAASO_FLAG_ENGINE_FROZEN) && o.mapping == MAASO_MAP_BLOCK)
-        return fail(ctx, MAASO_EINVAL, "eval: the fixed-speed engine has no block mapping");
+    if ((o.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP)) && o.mapping == MAASO_MAP_BLOCK)
+        return fail(ctx, MAASO_EINVAL, "eval: the fixed-speed engine and the largest-gap test have no block mapping");
 
     DeviceGuard g(ctx->device);
     cudaStream_t stream = (cudaStream_t)cuda_stream;

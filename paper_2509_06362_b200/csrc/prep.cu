@@ -13,8 +13,8 @@ __global__ void prep_kernel(const EvalParams P) {
         status = MAASO_CAND_EBADINST;  // malformed CSR row
     } else {
         n = hi - lo;
-        if (n > MAASO_MAX_INSTANCES || ((P.flags & MAASO_FLAG_ENGINE_FROZEN) && n > 32)) {
-            status = MAASO_CAND_ETOOMANY;  // the fixed-speed engine exists in the lane-group kernel only
+        if (n > MAASO_MAX_INSTANCES || ((P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP)) && n > 32)) {
+            status = MAASO_CAND_ETOOMANY;  // these options exist in the lane-group kernel only
         } else {
             uint64_t devsum = 0;
             for (uint32_t i = 0; i < n; i++) {

@@ -24,8 +24,8 @@ def ctx():
 @pytest.mark.parametrize("case", all_cases(), ids=lambda c: c["name"])
 def test_hand_timelines_on_gpu(ctx, case, mapping):
     for flags, expect in case["runs"]:
-        if (flags & 2) and mapping == 1:
-            continue      # the fixed-speed engine exists in the lane-group mapping only
+        if (flags & 6) and mapping == 1:
+            continue      # the fixed-speed engine and the largest-gap test exist in the lane-group mapping only
         res, dumps = gpu_eval(ctx, case["profile"], case["trace"], case["classes"], case["offsets"],
                               case["inst"], case["budget"], None, flags, mapping, dump_idx=[0])
         check_against_expect(res[0], {k: v[0] for k, v in dumps.items()}, expect)
@@ -680,7 +680,7 @@ def test_frozen_engine_limits(ctx):
     ctx.free_trace(t)
 
 
-@pytest.mark.parametrize("flags", [0, 1, 2, 3])
+@pytest.mark.parametrize("flags", [0, 1, 2, 3, 4, 5])
 def test_slot_keys_in_global_scratch_when_the_pool_is_too_small(oracle_mod, flags):
     """A context created with MAASO_GROUP_BLOCKS=8 leaves no shared memory for the key pool, so
     every lane keeps its slot keys in global scratch: same results."""
@@ -710,3 +710,44 @@ def test_slot_keys_in_global_scratch_when_the_pool_is_too_small(oracle_mod, flag
         assert_records_equal(got, want, "keys in global scratch")
     finally:
         c.close()
+
+
+# ---- TBT term of the hit test on the largest token gap (flag 4) -------------------------------
+@pytest.mark.parametrize("flags", [4, 5, 6, 7])
+def test_largest_gap_hit_test(ctx, oracle_mod, flags):
+    """Default and fixed-speed engine, with and without the optimistic estimate; limits tight
+    enough for prefill stalls to matter; every group width; ragged trace; dumps."""
+    tight = gen.make_classes([(500_000, 14_000, None), (2_000_000, 30_000, None), (None, 60_000, 180_000_000)])
+    cfg = gen.make_config("node", n_req=1777)
+    sel = np.arange(0, 10864, 31)
+    off = np.zeros(len(sel) + 1, dtype=np.uint32)
+    parts = []
+    for k, c in enumerate(sel):
+        parts.append(cfg["inst"][cfg["offsets"][c]:cfg["offsets"][c + 1]])
+        off[k + 1] = off[k] + len(parts[-1])
+    inst = np.concatenate(parts).astype(np.uint32)
+    tr = cfg["traces"][0]
+    idx = np.arange(0, len(sel), 43, dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(cfg["profile"], tr, tight, off, inst, 8, None, flags, dump_idx=idx)
+    got, gd = gpu_eval(ctx, cfg["profile"], tr, tight, off, inst, 8, None, flags, 0, dump_idx=idx)
+    assert_records_equal(got, want, "node subset, largest-gap test")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+    mean_form = oracle_mod.eval_placements(cfg["profile"], tr, tight, off, inst, 8, None, flags & ~4)
+    if not flags & 2:
+        assert int((mean_form["n_hit"] - want["n_hit"]).sum()) > 0     # the option changes something here
+
+    cfg = gen.make_config("multimodel", n_cand=400, n_req=2500)
+    keep = np.nonzero(np.diff(cfg["offsets"]) <= 32)[0]
+    off = np.zeros(len(keep) + 1, dtype=np.uint32)
+    parts = []
+    for k, c in enumerate(keep):
+        parts.append(cfg["inst"][cfg["offsets"][c]:cfg["offsets"][c + 1]])
+        off[k + 1] = off[k] + len(parts[-1])
+    inst = np.concatenate(parts).astype(np.uint32)
+    mask = np.random.default_rng(6).integers(1, 8, size=len(keep)).astype(np.uint32)
+    tight3 = gen.make_classes([(500_000, 60_000, None), (2_000_000, 150_000, None), (None, 300_000, 180_000_000)])
+    tr = cfg["traces"][0]
+    want = oracle_mod.eval_placements(cfg["profile"], tr, tight3, off, inst, 32, mask, flags)
+    got, _ = gpu_eval(ctx, cfg["profile"], tr, tight3, off, inst, 32, mask, flags, 0)
+    assert_records_equal(got, want, "multimodel subset, largest-gap test")
