@@ -212,6 +212,19 @@ MAASO_API void maaso_free_trace(maaso_ctx *ctx, maaso_trace *trace);
 MAASO_API int maaso_eval_placements(maaso_ctx *ctx, const maaso_trace *trace, const maaso_cand_batch *cands,
                           const maaso_eval_opts *opts, maaso_result *out_results, void *cuda_stream);
 
+/* The same batch of candidates scored against several traces in ONE pass (the load sweep of a
+ * placement study: the same candidate space under different arrival rates or burstiness).  traces:
+ * host array of n_traces <= 16 handles of this context, all loaded with the same SLO class table;
+ * out_results (device): n_traces blocks of n_cand records, record c of trace t at
+ * out_results[t * n_cand + c]; opts->rejected_by_model and opts->ttft_hist, if given, are laid out
+ * the same way ([n_traces * n_cand][...]).  Each record equals what maaso_eval_placements returns
+ * for that trace alone; scoring them together lets small candidate sets fill the GPU.  Lane-group
+ * mapping only: dump buffers and MAASO_MAP_BLOCK are refused, a placement with more than 32
+ * instances gets MAASO_CAND_ETOOMANY.  Enqueued on cuda_stream. */
+MAASO_API int maaso_eval_placements_multi(maaso_ctx *ctx, const maaso_trace *const *traces, uint32_t n_traces,
+                                          const maaso_cand_batch *cands, const maaso_eval_opts *opts,
+                                          maaso_result *out_results, void *cuda_stream);
+
 /* Same scoring with HOST buffers: copies the candidate batch to the device, scores it,
  * copies the records back into out_results (host, [n_cand]) and synchronises.  Dump
  * buffers, per-model counts and histograms are not supported here (opts->dump_n must be 0,

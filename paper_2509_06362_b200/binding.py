@@ -83,6 +83,8 @@ def _load():
     lib.maaso_free_trace.restype = None
     lib.maaso_eval_placements.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp, vp]
     lib.maaso_eval_placements_host.argtypes = [vp, vp, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp]
+    lib.maaso_eval_placements_multi.argtypes = [vp, C.POINTER(vp), u32, C.POINTER(_CandBatch), C.POINTER(_EvalOpts), vp, vp]
+    lib.maaso_eval_placements_multi.restype = C.c_int
     lib.maaso_topk.argtypes = [vp, vp, u64, u32, u32, vp, vp, vp]
     lib.maaso_score.argtypes = [vp, vp, u64, C.POINTER(_ScoreParams), vp, vp]
     lib.maaso_topk_scores.argtypes = [vp, vp, vp, u64, u32, vp, vp, vp]
@@ -209,6 +211,16 @@ def maaso_eval_placements(ctx, trace, offsets, inst, budget, out_results, class_
                   _ptr(rejected_by_model), _ptr(ttft_hist))
     _check(_lib.maaso_eval_placements(ctx, trace, C.byref(b), C.byref(o), _ptr(out_results),
                                       _stream_ptr(stream)), "maaso_eval_placements", ctx)
+
+
+def maaso_eval_placements_multi(ctx, traces, offsets, inst, budget, out_results, class_mask=None, flags=0,
+                                rejected_by_model=None, ttft_hist=None, stream=None):
+    """traces: sequence of trace handles; out_results: uint8 CUDA tensor of len(traces)*n_cand*128 bytes."""
+    b = _batch(offsets, inst, class_mask, budget)
+    o = _EvalOpts(int(flags), MAP_AUTO, 0, 0, None, None, None, None, _ptr(rejected_by_model), _ptr(ttft_hist))
+    arr = (C.c_void_p * len(traces))(*[t if isinstance(t, int) else (t.value if hasattr(t, "value") else t) for t in traces])
+    _check(_lib.maaso_eval_placements_multi(ctx, arr, len(traces), C.byref(b), C.byref(o), _ptr(out_results),
+                                            _stream_ptr(stream)), "maaso_eval_placements_multi", ctx)
 
 
 def maaso_eval_placements_host(ctx, trace, offsets, inst, budget, out_results, class_mask=None, flags=0,
@@ -386,6 +398,18 @@ class Context:
                               mapping, stream=stream, rejected_by_model=rejected_by_model, ttft_hist=ttft_hist,
                               **kw)
         return (out, dumps) if dump_idx is not None else out
+
+    def eval_placements_multi(self, traces, offsets, inst, budget, class_mask=None, flags=0, out=None, stream=None,
+                              rejected_by_model=None, ttft_hist=None):
+        """One pass over several traces (at most 16, same SLO classes).  Returns a uint8 tensor
+        [len(traces), n_cand, 128]: block t holds the records for traces[t]."""
+        torch = self.torch
+        n_cand = int(offsets.shape[0]) - 1
+        if out is None:
+            out = torch.empty((len(traces), n_cand, 128), dtype=torch.uint8, device=self.device)
+        maaso_eval_placements_multi(self.handle, [t.handle for t in traces], offsets, inst, budget, out, class_mask,
+                                    flags, rejected_by_model, ttft_hist, stream)
+        return out
 
     def eval_placements_host(self, trace, offsets, inst, budget, class_mask=None, flags=0,
                              mapping=MAP_AUTO, out=None):

@@ -21,6 +21,7 @@ constexpr int kGenericBlockBucket = 9;
 constexpr int kCostBins = 256;   // bin 0 = most expensive (largest total batch cap)
 constexpr int kCounterWords = 8192;  // counters | work counters | histograms + cursors, cleared per call
 constexpr int kGroupThreads = 128;
+constexpr int kMaxTraces = 16;  // traces one call of the lane-group kernel can replay side by side
 
 struct Request {
     int64_t arrival;
@@ -223,6 +224,12 @@ struct EvalParams {
     uint32_t n_classes;
     const int64_t* classes;  // [n_classes][3]
     const uint4* cooked;     // [n_req][kCookedWords] prepared records (lane-group kernel)
+    // several traces in one launch (lane-group kernel only): trace t of n_traces > 1 has
+    // trace_n[t] prepared records at trace_cooked[t]; record c of trace t goes to out[t * n_cand + c]
+    // (and likewise for the per-model counts and the histograms).  n_traces = 1: cooked / n_req.
+    uint32_t n_traces;
+    const uint4* trace_cooked[kMaxTraces];
+    uint32_t trace_n[kMaxTraces];
     const uint64_t* rej_hash;  // [n_req] checksum term of "request r was rejected" (same for every candidate)
     const int32_t* rows;     // [n_rows][kRowStride]
     const int32_t* devices;
@@ -266,9 +273,12 @@ __device__ __forceinline__ bool account_completion(Stats& st, const int64_t* cla
     return account_completion(st, classes, inst, req, arrival, first_tok, t_fin, S, cls, dump, (int64_t)-1);
 }
 
+// `cand`: index of the candidate's record in the output (trace index * n_cand + candidate index
+// when several traces are replayed in one launch; dump rows exist for one trace only).
 __device__ __forceinline__ Dump dump_for(const EvalParams& P, uint32_t cand) {
     Dump d{nullptr, nullptr, nullptr, nullptr};
     if (P.ttft_hist) d.hist = P.ttft_hist + (size_t)cand * MAASO_TTFT_BINS;
+    if (P.n_traces > 1) return d;
     if (P.dump_row) {
         int32_t row = P.dump_row[cand];
         if (row >= 0) {

@@ -114,12 +114,12 @@ __device__ __forceinline__ GroupSmem carve(unsigned char* base, uint32_t n_rows,
 
 // One tile of prepared records (48 bytes each, so every copy is a multiple of 16 bytes and
 // starts on a 16-byte boundary).
-__device__ __forceinline__ void issue_tile(const GroupSmem& sm, const EvalParams& P, uint32_t stage, uint32_t tile,
-                                           int tile_recs) {
-    const uint32_t recs = min((uint32_t)tile_recs, P.n_req - tile * tile_recs);
+__device__ __forceinline__ void issue_tile(const GroupSmem& sm, const uint4* cooked, uint32_t n_req, uint32_t stage,
+                                           uint32_t tile, int tile_recs) {
+    const uint32_t recs = min((uint32_t)tile_recs, n_req - tile * tile_recs);
     const uint32_t bytes = recs * 16u * kCookedWords;
     mbar_expect_tx(&sm.full_bar[stage], bytes);
-    bulk_load(sm.tiles + (size_t)stage * tile_recs * kCookedWords, P.cooked + (size_t)tile * tile_recs * kCookedWords,
+    bulk_load(sm.tiles + (size_t)stage * tile_recs * kCookedWords, cooked + (size_t)tile * tile_recs * kCookedWords,
               bytes, &sm.full_bar[stage]);
 }
 
@@ -185,7 +185,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
     env.mg = nullptr;
     env.dl = nullptr;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
-    const uint32_t n_tiles = (P.n_req + tile_recs - 1) / tile_recs;
+    const uint32_t n_traces = P.n_traces > 1 ? P.n_traces : 1u;
     uint32_t tile_seq = 0;  // tiles consumed so far by this warp (same in every warp)
 
     // how many work items (4 warps each) every bucket contributes (largest groups first)
@@ -197,6 +197,8 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         items[b] = (n_warps + kWarps - 1) / kWarps;
         total_items += items[b];
     }
+    // with several traces every work item exists once per trace: item index = item * n_traces + trace
+    const uint32_t total_all = total_items * n_traces;
 
     for (;;) {
         __syncthreads();  // everyone is done with the previous batch (tiles, work slot)
@@ -210,19 +212,25 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                 asm volatile("mov.u32 %0, %%smid;" : "=r"(my_sm));
                 for (uint32_t k = 0; k < P.n_sm && item == 0xFFFFFFFFu; k++) {
                     const uint32_t s = (my_sm + k) % P.n_sm;
-                    if (*(volatile uint32_t*)&P.sm_ctr[s] * P.n_sm >= total_items) continue;  // exhausted
+                    if (*(volatile uint32_t*)&P.sm_ctr[s] * P.n_sm >= total_all) continue;  // exhausted
                     // snake order: odd rounds run backwards, so the SM that got the most expensive
                     // item of one round gets the cheapest of the next
                     const uint32_t j = atomicAdd(&P.sm_ctr[s], 1u);
                     const uint32_t it = j * P.n_sm + ((j & 1u) ? P.n_sm - 1u - s : s);
-                    if (it < total_items) item = it;
+                    if (it < total_all) item = it;
                 }
             }
             sm.work[0] = item;
         }
         __syncthreads();
         uint32_t wi = sm.work[0];
-        if (wi >= total_items) break;
+        if (wi >= total_all) break;
+        const uint32_t tr = wi % n_traces;  // which trace this item replays
+        wi /= n_traces;
+        const uint4* const cooked = P.n_traces > 1 ? P.trace_cooked[tr] : P.cooked;
+        const uint32_t n_req = P.n_traces > 1 ? P.trace_n[tr] : P.n_req;
+        const uint32_t n_tiles = (n_req + tile_recs - 1) / tile_recs;
+        const uint32_t out_base = tr * P.n_cand;  // this trace's block of records
         int b = 5;
         while (wi >= items[b]) { wi -= items[b]; b--; }
         const uint32_t G = 1u << b;
@@ -291,7 +299,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         const bool warp_has_work = __any_sync(kFullMask, valid);
         const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
         Dump dump{nullptr, nullptr, nullptr, nullptr};
-        if (valid) dump = dump_for(P, cand);
+        if (valid) dump = dump_for(P, out_base + cand);
         // per-request side outputs (dump rows, per-model rejection counts) are rare: one flag guards them
         const bool side = dump.finish || dump.first || dump.inst || P.rej_by_model;
         LaneStats ls;
@@ -306,7 +314,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         // trace staging: first tiles of this batch
         if (tid == 0 && !P.stall_test) {
             for (uint32_t j = 0; j < (uint32_t)kStages && j < n_tiles; j++)
-                issue_tile(sm, P, (tile_seq + j) % kStages, j, tile_recs);
+                issue_tile(sm, cooked, n_req, (tile_seq + j) % kStages, j, tile_recs);
         }
 
         for (uint32_t t = 0; t < n_tiles; t++) {
@@ -319,7 +327,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                 break;
             }
             const uint4* tile = sm.tiles + (size_t)s * tile_recs * kCookedWords;
-            const uint32_t recs = min((uint32_t)tile_recs, P.n_req - t * tile_recs);
+            const uint32_t recs = min((uint32_t)tile_recs, n_req - t * tile_recs);
             // a warp without a candidate only keeps the tile pipeline going
             for (uint32_t ri = warp_has_work ? 0u : recs; ri < recs; ri++) {
                 // statistics of completed requests: every fourth request, if some lane's queue is nearly full
@@ -359,7 +367,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                                 rej_sum += q.rej;
                                 if (side) {
                                     if (P.rej_by_model)
-                                        atomicAdd(&P.rej_by_model[(size_t)cand * MAASO_MAX_MODELS + q.model], 1u);
+                                        atomicAdd(&P.rej_by_model[(size_t)(out_base + cand) * MAASO_MAX_MODELS + q.model], 1u);
                                     if (dump.finish) dump.finish[req] = -1;
                                     if (dump.first) dump.first[req] = -1;
                                     if (dump.inst) dump.inst[req] = -1;
@@ -402,7 +410,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                     const uint32_t nt = t + kStages;
                     if (nt < n_tiles) {
                         fence_proxy_async();
-                        issue_tile(sm, P, s, nt, tile_recs);
+                        issue_tile(sm, cooked, n_req, s, nt, tile_recs);
                     }
                 }
             }
@@ -435,7 +443,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         __syncwarp();
         if (valid && sub == 0) {
             // worst-case mode: one round per counted request plus the counted second rounds
-            write_result(P.out + cand, status, n_counted, n_rejected, LOOP ? attempts : attempts + n_counted, st, h);
+            write_result(P.out + out_base + cand, status, n_counted, n_rejected, LOOP ? attempts : attempts + n_counted, st, h);
         }
     }
 }

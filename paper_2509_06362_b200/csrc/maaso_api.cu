@@ -40,6 +40,7 @@ struct maaso_trace {
     int64_t* d_classes;
     uint64_t* d_rej_hash;
     uint4* d_cooked;  // prepared records for the lane-group kernel
+    std::vector<int64_t> h_classes;  // host copy of the class table (several traces in one call must agree on it)
     uint64_t n;
     uint32_t n_classes;
     uint32_t max_model;
@@ -323,6 +324,7 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     t->n = n;
     t->n_classes = n_classes;
     t->max_model = max_model;
+    t->h_classes = cls;
     cudaError_t e = cudaMalloc(&t->d_reqs, (n ? n : 1) * sizeof(maaso_request));
     if (e == cudaSuccess) e = cudaMalloc(&t->d_classes, cls.size() * 8);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_rej_hash, (n ? n : 1) * 8);
@@ -348,14 +350,27 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     return MAASO_OK;
 }
 
-MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, const maaso_cand_batch* cands,
-                          const maaso_eval_opts* opts, maaso_result* out_results, void* cuda_stream) {
-    if (!ctx || !trace || !cands) return MAASO_EINVAL;
+// Scoring of one candidate batch against n_traces traces (1 = the plain call).
+static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t n_traces,
+                     const maaso_cand_batch* cands, const maaso_eval_opts* opts, maaso_result* out_results,
+                     void* cuda_stream) {
+    if (!ctx || !traces || !cands || n_traces < 1 || n_traces > (uint32_t)kMaxTraces) return MAASO_EINVAL;
     if (!ctx->has_profile) return fail(ctx, MAASO_ESTATE, "eval: no profile loaded");
-    if (trace->owner != ctx) return fail(ctx, MAASO_ESTATE, "eval: trace belongs to another context");
-    if (trace->n && trace->max_model >= ctx->n_models)
-        return fail(ctx, MAASO_ESTATE, "eval: trace refers to a model the current profile lacks");
+    const maaso_trace* trace = traces[0];
+    uint64_t n_max = 0;
+    for (uint32_t t = 0; t < n_traces; t++) {
+        const maaso_trace* x = traces[t];
+        if (!x) return MAASO_EINVAL;
+        if (x->owner != ctx) return fail(ctx, MAASO_ESTATE, "eval: trace belongs to another context");
+        if (x->n && x->max_model >= ctx->n_models)
+            return fail(ctx, MAASO_ESTATE, "eval: trace refers to a model the current profile lacks");
+        if (x->h_classes != trace->h_classes)
+            return fail(ctx, MAASO_EINVAL, "eval: traces scored in one call must have the same SLO classes");
+        if (x->n > n_max) n_max = x->n;
+    }
     if (cands->n_cand == 0) return MAASO_OK;
+    if ((uint64_t)cands->n_cand * n_traces >= 0xFFFFFFFFull)
+        return fail(ctx, MAASO_EINVAL, "eval: candidates x traces out of range");
     if (!cands->offsets || !out_results || (cands->n_inst && !cands->inst) || cands->n_cand >= 0xFFFFFFFFull ||
         cands->n_inst >= 0xFFFFFFFFull)
         return fail(ctx, MAASO_EINVAL, "eval: null pointer or size out of range");
@@ -364,6 +379,8 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     if (opts) o = *opts;
     if (o.mapping > MAASO_MAP_GROUP) return fail(ctx, MAASO_EINVAL, "eval: unknown mapping");
     if (o.dump_n && !o.dump_cand_idx) return fail(ctx, MAASO_EINVAL, "eval: dump_n without dump_cand_idx");
+    if (n_traces > 1 && (o.dump_n || o.mapping == MAASO_MAP_BLOCK))
+        return fail(ctx, MAASO_EINVAL, "eval: several traces in one call allow no dump buffers and no block mapping");
     if (o.flags & ~(MAASO_FLAG_PRED_OPTIMISTIC | MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_TEST_STALL))
         return fail(ctx, MAASO_EINVAL, "eval: unknown flag");
     if ((o.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP)) && o.mapping == MAASO_MAP_BLOCK)
@@ -382,6 +399,11 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.classes = trace->d_classes;
     P.rej_hash = trace->d_rej_hash;
     P.cooked = trace->d_cooked;
+    P.n_traces = n_traces;
+    for (uint32_t t = 0; t < n_traces; t++) {
+        P.trace_cooked[t] = traces[t]->d_cooked;
+        P.trace_n[t] = (uint32_t)traces[t]->n;
+    }
     P.rows = ctx->d_rows;
     P.devices = ctx->d_devices;
     P.min_devices = ctx->d_min_devices;
@@ -413,19 +435,21 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     // ~ instances x 1.3 (group widths are powers of two).
     int group_blocks = ctx->group_blocks;
     if (group_blocks == 0) {
-        const uint64_t est_warps = (cands->n_inst * 13 / 10 + 31) / 32 + 6;
+        const uint64_t est_warps = ((cands->n_inst * 13 / 10 + 31) / 32 + 6) * n_traces;
         group_blocks = est_warps <= (uint64_t)ctx->sm_count * 3 * (kGroupThreads / 32) ? 3 : 4;
     }
     const int occ_g = occupancy_eval_group(P, tile, group_blocks, ctx->smem_per_sm);
     int grid_g = ctx->sm_count * occ_g;
-    const uint64_t max_items_g = (uint64_t)C / 4 + 6;  // at most one work item per 4 candidates + bucket tails
+    // at most one work item per 4 candidates + bucket tails, once per trace
+    const uint64_t max_items_g = ((uint64_t)C / 4 + 6) * n_traces;
     if ((uint64_t)grid_g > max_items_g) grid_g = (int)max_items_g;
     int grid_b[4];
     size_t pay_entries = (size_t)grid_g * kGroupThreads * (group_scratch_per_lane() / sizeof(Payload));
     static_assert(sizeof(Payload) == 32, "scratch is counted in 32-byte entries");
     for (int b = 6; b <= kGenericBlockBucket; b++) {
         // without the block mapping only candidates with more than 32 instances go to a block kernel
-        const bool used = o.mapping == MAASO_MAP_BLOCK || (b == kGenericBlockBucket && cands->n_inst > 32);
+        const bool used = n_traces == 1 &&
+                          (o.mapping == MAASO_MAP_BLOCK || (b == kGenericBlockBucket && cands->n_inst > 32));
         grid_b[b - 6] = 0;
         if (!used) continue;
         // placements with at most 8 instances: one warp per instance with register-resident state
@@ -461,7 +485,8 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     P.group_warps = (uint32_t)grid_g * (kGroupThreads / 32);
     P.promote_pct = (uint32_t)ctx->promote_pct;
     cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, kCounterWords * 4, stream);
-    if (e == cudaSuccess && o.ttft_hist) e = cudaMemsetAsync(o.ttft_hist, 0, (size_t)C * MAASO_TTFT_BINS * 4, stream);
+    if (e == cudaSuccess && o.ttft_hist)
+        e = cudaMemsetAsync(o.ttft_hist, 0, (size_t)C * n_traces * MAASO_TTFT_BINS * 4, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "memset");
     int launches = 0;
     if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
@@ -487,6 +512,18 @@ MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, co
     }
     ctx->launches += (uint64_t)launches;
     return MAASO_OK;
+}
+
+MAASO_API int maaso_eval_placements(maaso_ctx* ctx, const maaso_trace* trace, const maaso_cand_batch* cands,
+                                    const maaso_eval_opts* opts, maaso_result* out_results, void* cuda_stream) {
+    if (!trace) return MAASO_EINVAL;
+    return eval_impl(ctx, &trace, 1, cands, opts, out_results, cuda_stream);
+}
+
+MAASO_API int maaso_eval_placements_multi(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t n_traces,
+                                          const maaso_cand_batch* cands, const maaso_eval_opts* opts,
+                                          maaso_result* out_results, void* cuda_stream) {
+    return eval_impl(ctx, traces, n_traces, cands, opts, out_results, cuda_stream);
 }
 
 MAASO_API int maaso_eval_placements_host(maaso_ctx* ctx, const maaso_trace* trace, const maaso_cand_batch* cands,

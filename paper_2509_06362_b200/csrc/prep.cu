@@ -13,7 +13,7 @@ __global__ void prep_kernel(const EvalParams P) {
         status = MAASO_CAND_EBADINST;  // malformed CSR row
     } else {
         n = hi - lo;
-        if (n > MAASO_MAX_INSTANCES || ((P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP)) && n > 32)) {
+        if (n > MAASO_MAX_INSTANCES || (((P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP)) || P.n_traces > 1) && n > 32)) {
             status = MAASO_CAND_ETOOMANY;  // these options exist in the lane-group kernel only
         } else {
             uint64_t devsum = 0;
@@ -32,13 +32,15 @@ __global__ void prep_kernel(const EvalParams P) {
         }
     }
     if (P.dump_row) P.dump_row[c] = -1;
-    if (P.rej_by_model)
-        for (int m = 0; m < MAASO_MAX_MODELS; m++) P.rej_by_model[(size_t)c * MAASO_MAX_MODELS + m] = 0;
-    {
+    const uint32_t n_traces = P.n_traces > 1 ? P.n_traces : 1u;
+    for (uint32_t t = 0; t < n_traces; t++) {
+        const size_t oc = (size_t)t * P.n_cand + c;  // the candidate's record in trace t's block
+        if (P.rej_by_model)
+            for (int m = 0; m < MAASO_MAX_MODELS; m++) P.rej_by_model[oc * MAASO_MAX_MODELS + m] = 0;
         // Invalid candidates get their final record here.  Valid ones are pre-marked "not scored"
         // (ETIMEOUT); the scoring kernel overwrites the record when it finishes the candidate, so a
         // kernel that gave up on a bounded wait leaves no record undefined.
-        uint4* o = reinterpret_cast<uint4*>(P.out + c);
+        uint4* o = reinterpret_cast<uint4*>(P.out + oc);
         o[0] = make_uint4(status ? status : MAASO_CAND_ETIMEOUT, 0, 0, 0);
         for (int i = 1; i < 8; i++) o[i] = make_uint4(0, 0, 0, 0);
     }

@@ -751,3 +751,57 @@ def test_largest_gap_hit_test(ctx, oracle_mod, flags):
     want = oracle_mod.eval_placements(cfg["profile"], tr, tight3, off, inst, 32, mask, flags)
     got, _ = gpu_eval(ctx, cfg["profile"], tr, tight3, off, inst, 32, mask, flags, 0)
     assert_records_equal(got, want, "multimodel subset, largest-gap test")
+
+
+# ---- several traces in one pass ----------------------------------------------------------------
+@pytest.mark.parametrize("flags", [0, 1, 2, 4])
+def test_several_traces_in_one_pass(ctx, oracle_mod, flags):
+    """The bursty load sweep, cut down: the candidate set against 5 traces of different rates and
+    lengths in one call; every block of records must equal the oracle's for that trace, and so must
+    the per-model rejection counts and the histograms."""
+    import torch
+    cfg = gen.make_config("bursty", n_req=1500)
+    sel = np.arange(0, 10864, 37)
+    off = np.zeros(len(sel) + 1, dtype=np.uint32)
+    parts = []
+    for k, c in enumerate(sel):
+        parts.append(cfg["inst"][cfg["offsets"][c]:cfg["offsets"][c + 1]])
+        off[k + 1] = off[k] + len(parts[-1])
+    inst = np.concatenate(parts).astype(np.uint32)
+    traces_np = [cfg["traces"][j][: 1500 - 211 * i] for i, j in enumerate((0, 5, 9, 13, 15))]   # ragged lengths
+    ctx.load_profile(cfg["profile"])
+    handles = [ctx.load_trace(t, cfg["classes"]) for t in traces_np]
+    n_cand, n_tr = len(sel), len(handles)
+    mask = np.random.default_rng(9).integers(1, 8, size=n_cand).astype(np.uint32)
+    rbm = torch.full((n_tr * n_cand, 16), 77, dtype=torch.int32, device="cuda")
+    hist = torch.full((n_tr * n_cand, 64), 77, dtype=torch.int32, device="cuda")
+    out = ctx.eval_placements_multi(handles, ctx.to_device(off), ctx.to_device(inst), 8, ctx.to_device(mask), flags,
+                                    rejected_by_model=rbm, ttft_hist=hist)
+    torch.cuda.synchronize()
+    got = ctx.results_to_numpy(out).reshape(n_tr, n_cand)
+    rbm_h = rbm.cpu().numpy().view(np.uint32).reshape(n_tr, n_cand, 16)
+    hist_h = hist.cpu().numpy().view(np.uint32).reshape(n_tr, n_cand, 64)
+    for t, tr in enumerate(traces_np):
+        want = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 8, mask, flags)
+        assert_records_equal(got[t], want, f"trace {t} of the joint pass")
+        if flags == 0:
+            assert (rbm_h[t] == oracle_mod.rejected_by_model(cfg["profile"], tr, cfg["classes"], off, inst, 8, mask)).all()
+            assert (hist_h[t] == oracle_mod.ttft_hist(cfg["profile"], tr, cfg["classes"], off, inst, 8, mask)).all()
+    for h in handles:
+        ctx.free_trace(h)
+
+
+def test_several_traces_limits(ctx):
+    import paper_2509_06362_b200 as m
+    cfg = gen.make_config("tiny", n_req=60)
+    ctx.load_profile(cfg["profile"])
+    a = ctx.load_trace(cfg["traces"][0], cfg["classes"])
+    other = gen.make_classes([(1_000_000, None, None)] * 3)
+    b = ctx.load_trace(cfg["traces"][0], other)
+    d_off, d_inst = ctx.to_device(cfg["offsets"]), ctx.to_device(cfg["inst"])
+    with pytest.raises(m.MaasoError):          # different SLO class tables
+        ctx.eval_placements_multi([a, b], d_off, d_inst, 4)
+    with pytest.raises(m.MaasoError):          # more than 16 traces
+        ctx.eval_placements_multi([a] * 17, d_off, d_inst, 4)
+    ctx.free_trace(a)
+    ctx.free_trace(b)
