@@ -664,8 +664,11 @@ static int ins_deploy_multi(maaso_ctx* ctx, const maaso_trace* trace, const Depl
     DeviceGuard g(ctx->device);
 
     // device staging: offsets | inst | mask | results | scores | rejected-by-model
-    const size_t C = (size_t)n_configs * n_prob, cap_inst = C * (MAASO_MAX_INSTANCES + 1);
-    const size_t cap_cand = C > n_prob ? C : n_prob;
+    const size_t C = (size_t)n_configs * n_prob;
+    const size_t cap_spec = 1u << 16;  // speculative follow-ups only while the batch stays this small
+    const size_t per_chain = C * (2 + (size_t)ctx->n_models) <= cap_spec ? 2 + (size_t)ctx->n_models : 1;
+    const size_t cap_cand = C * per_chain > n_prob ? C * per_chain : n_prob;
+    const size_t cap_inst = cap_cand * (MAASO_MAX_INSTANCES + 2);
     size_t off = 0;
     const size_t o_off = off;  off = align_up(off + (cap_cand + 1) * 4, 256);
     const size_t o_inst = off; off = align_up(off + cap_inst * 4, 256);
@@ -750,51 +753,109 @@ static int ins_deploy_multi(maaso_ctx* ctx, const maaso_trace* trace, const Depl
             ch.mask = mask_of(p);
             ch.tentative = 0;
         }
-    std::vector<uint32_t> batch_chain;
-    std::vector<char> batch_over;  // the tentative placement needs more devices than its problem has
+    // Two greedy steps per batch.  Besides its tentative placement A = I + m' every chain also
+    // proposes what its NEXT step would score, for both outcomes of this one: if A is rejected the
+    // next tentative model is already known (m' becomes saturated, nothing else changes): B; if A is
+    // accepted the unserved counts change, so the next model is not known: I + m' + m for every model
+    // m still open.  After the batch the first step is taken with A's result and the second with the
+    // speculative result that matches the actual state.  The batches are a few times larger, the
+    // number of trace replays halves; the steps taken are those of the sequential algorithm.
+    const uint32_t n_models = ctx->n_models;
+    const bool speculate = C * (2 + (size_t)n_models) <= cap_spec;
+    auto next_model = [&](const Chain& ch, const bool* sat, size_t len) -> int {
+        int mp = -1;  // model with the most unserved requests among the non-saturated ones
+        if ((uint64_t)len * ch.dev < ch.gpus && len <= MAASO_MAX_INSTANCES)
+            for (uint32_t m = 0; m < n_models; m++)
+                if (!sat[m] && (mp < 0 || ch.unserved[m] > ch.unserved[mp])) mp = (int)m;
+        return mp;
+    };
+    uint32_t n_batch = 0;
+    std::vector<char> batch_over;  // the placement needs more devices than its problem has
+    auto propose = [&](const Chain& ch, const maaso_config& cf, int m1, int m2) -> int {
+        // candidate I + m1 (+ m2); returns its index in the batch
+        h_off[n_batch] = (uint32_t)h_inst.size();
+        h_mask[n_batch] = ch.mask;
+        h_inst.insert(h_inst.end(), ch.inst.begin(), ch.inst.end());
+        const uint32_t w = ((cf.strategy & 0xFFu) << 4) | ((cf.batch & 0xFFu) << 12);
+        h_inst.push_back(((uint32_t)m1 & 0xFu) | w);
+        if (m2 >= 0) h_inst.push_back(((uint32_t)m2 & 0xFu) | w);
+        batch_over.push_back(((uint64_t)ch.inst.size() + (m2 >= 0 ? 2 : 1)) * ch.dev > ch.gpus ? 1 : 0);
+        return (int)n_batch++;
+    };
+    auto take_step = [&](Chain& ch, int model, uint32_t word, int j) {
+        Step sp;
+        sp.k = (uint32_t)ch.inst.size() * ch.dev;
+        // a placement beyond the problem's own device count is invalid (score -1), as it would be
+        // if the problem were scored alone with its device count as the budget
+        const double sc = batch_over[j] ? -1.0 : h_sc[j];
+        bool accepted = false;
+        if (sc > ch.phi) {  // accept the new instance
+            ch.phi = sc;
+            ch.inst.push_back(word);
+            memcpy(ch.unserved, h_rbm.data() + (size_t)j * MAASO_MAX_MODELS, sizeof(ch.unserved));
+            accepted = true;
+        } else {
+            ch.sat[model] = true;  // stop deploying this model
+        }
+        sp.len = (uint32_t)ch.inst.size();
+        sp.phi = ch.phi;
+        ch.steps.push_back(sp);
+        return accepted;
+    };
+    struct Plan {
+        uint32_t chain;
+        int m1, a;           // tentative model, batch index of A
+        int mb, b;           // model and batch index of the "A rejected" follow-up (-1: none)
+        int c[MAASO_MAX_MODELS];  // batch index of the "A accepted, then model m" follow-up (-1: none)
+    };
+    std::vector<Plan> plans;
     for (;;) {
         // every unfinished chain proposes its next tentative placement I' = I + (m', P, B)
-        batch_chain.clear();
+        plans.clear();
         batch_over.clear();
         h_inst.clear();
+        n_batch = 0;
         for (size_t x = 0; x < C; x++) {
             Chain& ch = chains[x];
             const maaso_config& cf = configs[x % n_configs];
             if (ch.tentative < 0) continue;
-            int mp = -1;  // model with the most unserved requests among the non-saturated ones
-            if ((uint64_t)ch.inst.size() * ch.dev < ch.gpus && ch.inst.size() <= MAASO_MAX_INSTANCES)
-                for (uint32_t m = 0; m < ctx->n_models; m++)
-                    if (!ch.sat[m] && (mp < 0 || ch.unserved[m] > ch.unserved[mp])) mp = (int)m;
+            const int mp = next_model(ch, ch.sat, ch.inst.size());
             ch.tentative = mp;
             if (mp < 0) continue;
-            h_off[batch_chain.size()] = (uint32_t)h_inst.size();
-            h_mask[batch_chain.size()] = ch.mask;
-            h_inst.insert(h_inst.end(), ch.inst.begin(), ch.inst.end());
-            h_inst.push_back(((uint32_t)mp & 0xFu) | ((cf.strategy & 0xFFu) << 4) | ((cf.batch & 0xFFu) << 12));
-            batch_over.push_back(((uint64_t)ch.inst.size() + 1) * ch.dev > ch.gpus ? 1 : 0);
-            batch_chain.push_back((uint32_t)x);
-        }
-        if (batch_chain.empty()) break;
-        h_off[batch_chain.size()] = (uint32_t)h_inst.size();
-        rc = run_batch((uint32_t)batch_chain.size());
-        if (rc != MAASO_OK) return rc;
-        for (size_t j = 0; j < batch_chain.size(); j++) {
-            Chain& ch = chains[batch_chain[j]];
-            Step sp;
-            sp.k = (uint32_t)ch.inst.size() * ch.dev;
-            // a placement beyond the problem's own device count is invalid (score -1), as it would be
-            // if the problem were scored alone with its device count as the budget
-            const double sc = batch_over[j] ? -1.0 : h_sc[j];
-            if (sc > ch.phi) {  // accept the new instance
-                ch.phi = sc;
-                ch.inst.push_back(h_inst[h_off[j + 1] - 1]);
-                memcpy(ch.unserved, h_rbm.data() + j * MAASO_MAX_MODELS, sizeof(ch.unserved));
-            } else {
-                ch.sat[ch.tentative] = true;  // stop deploying this model
+            Plan pl;
+            pl.chain = (uint32_t)x;
+            pl.m1 = mp;
+            pl.a = propose(ch, cf, mp, -1);
+            pl.mb = -1;
+            pl.b = -1;
+            for (uint32_t m = 0; m < MAASO_MAX_MODELS; m++) pl.c[m] = -1;
+            if (speculate) {
+                bool sat2[MAASO_MAX_MODELS];
+                memcpy(sat2, ch.sat, sizeof(sat2));
+                sat2[mp] = true;
+                pl.mb = next_model(ch, sat2, ch.inst.size());
+                if (pl.mb >= 0) pl.b = propose(ch, cf, pl.mb, -1);
+                const size_t len2 = ch.inst.size() + 1;
+                if ((uint64_t)len2 * ch.dev < ch.gpus && len2 <= MAASO_MAX_INSTANCES)
+                    for (uint32_t m = 0; m < n_models; m++)
+                        if (!ch.sat[m]) pl.c[m] = propose(ch, cf, mp, (int)m);
             }
-            sp.len = (uint32_t)ch.inst.size();
-            sp.phi = ch.phi;
-            ch.steps.push_back(sp);
+            plans.push_back(pl);
+        }
+        if (plans.empty()) break;
+        h_off[n_batch] = (uint32_t)h_inst.size();
+        rc = run_batch(n_batch);
+        if (rc != MAASO_OK) return rc;
+        for (const Plan& pl : plans) {
+            Chain& ch = chains[pl.chain];
+            const maaso_config& cf = configs[pl.chain % n_configs];
+            const uint32_t w = ((cf.strategy & 0xFFu) << 4) | ((cf.batch & 0xFFu) << 12);
+            const bool accepted = take_step(ch, pl.m1, ((uint32_t)pl.m1 & 0xFu) | w, pl.a);
+            if (!speculate) continue;
+            const int m2 = next_model(ch, ch.sat, ch.inst.size());  // from the state the first step left
+            if (m2 < 0) continue;  // the chain ends; the next round marks it finished
+            const int j = accepted ? pl.c[m2] : (m2 == pl.mb ? pl.b : -1);
+            if (j >= 0) take_step(ch, m2, ((uint32_t)m2 & 0xFu) | w, j);
         }
     }
     // Phi*[k] / I*[k]: replay the steps configuration by configuration, as the sequential algorithm
