@@ -124,9 +124,14 @@ __device__ __forceinline__ void issue_tile(const GroupSmem& sm, const uint4* coo
 }
 
 // Account the queued completions of the whole warp once some lane holds kFlushAt of them.
+// The side-output pointers of the candidate (dump rows, histogram) are looked up here, when the
+// queues are accounted, instead of being carried through the replay loop in registers.
+// oc: index of the candidate's record in the output, or a negative value for a lane without one.
 template <bool MAXGAP>
 __device__ __forceinline__ void flush_now(uint32_t& qn, LaneStats& ls, const LaneEnv& env, const int64_t* classes,
-                                          uint32_t sub, const Dump& dump) {
+                                          uint32_t sub, const EvalParams& P, int64_t oc) {
+    Dump dump{nullptr, nullptr, nullptr, nullptr};
+    if (oc >= 0) dump = dump_for(P, (uint32_t)oc);
     if (MAXGAP)
         flush_queue_maxgap(&ls, env.qf, env.qa, env.qb, env.ovf, qn, classes, sub, dump.finish, dump.first, dump.inst,
                            dump.hist);
@@ -137,8 +142,8 @@ __device__ __forceinline__ void flush_now(uint32_t& qn, LaneStats& ls, const Lan
 }
 template <bool MAXGAP>
 __device__ __forceinline__ void flush_if_due(uint32_t& qn, LaneStats& ls, const LaneEnv& env, const int64_t* classes,
-                                             uint32_t sub, const Dump& dump) {
-    if (__any_sync(kFullMask, qn >= (uint32_t)kFlushAt)) flush_now<MAXGAP>(qn, ls, env, classes, sub, dump);
+                                             uint32_t sub, const EvalParams& P, int64_t oc) {
+    if (__any_sync(kFullMask, qn >= (uint32_t)kFlushAt)) flush_now<MAXGAP>(qn, ls, env, classes, sub, P, oc);
 }
 
 // OPT: the distributor predicts with the step time right after admission (optimistic estimate).
@@ -298,10 +303,11 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         }
         const bool warp_has_work = __any_sync(kFullMask, valid);
         const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
-        Dump dump{nullptr, nullptr, nullptr, nullptr};
-        if (valid) dump = dump_for(P, out_base + cand);
-        // per-request side outputs (dump rows, per-model rejection counts) are rare: one flag guards them
-        const bool side = dump.finish || dump.first || dump.inst || P.rej_by_model;
+        // index of the candidate's record; the side outputs hang on it (dump rows, histogram)
+        const int64_t oc = valid ? (int64_t)(out_base + cand) : -1;
+        // per-request side outputs of a rejection (dump rows, per-model counts) are rare: one flag guards them
+        bool side = P.rej_by_model != nullptr;
+        if (valid && P.dump_row) side = side || P.dump_row[cand] >= 0;
         LaneStats ls;
         ls.st.clear();
         for (int i = 0; i < 8; i++) ls.hbc[i] = 0;
@@ -331,7 +337,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
             // a warp without a candidate only keeps the tile pipeline going
             for (uint32_t ri = warp_has_work ? 0u : recs; ri < recs; ri++) {
                 // statistics of completed requests: every fourth request, if some lane's queue is nearly full
-                if ((ri & 3u) == 0u) flush_if_due<MAXGAP>(in.qn, ls, env, sm.classes, sub, dump);
+                if ((ri & 3u) == 0u) flush_if_due<MAXGAP>(in.qn, ls, env, sm.classes, sub, P, oc);
                 const uint4* rec = tile + (size_t)ri * kCookedWords;
                 const uint4 r0 = rec[0], r1 = rec[1], r2 = rec[2];
                 // All 32 lanes walk the trace together and every warp-level operation below uses
@@ -366,6 +372,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                             if (sub == 0) {
                                 rej_sum += q.rej;
                                 if (side) {
+                                    const Dump dump = dump_for(P, out_base + cand);
                                     if (P.rej_by_model)
                                         atomicAdd(&P.rej_by_model[(size_t)(out_base + cand) * MAASO_MAX_MODELS + q.model], 1u);
                                     if (dump.finish) dump.finish[req] = -1;
@@ -419,10 +426,10 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
 
         // drain, account what is still queued, reduce over the group, write the record
         __syncwarp();
-        flush_now<MAXGAP>(in.qn, ls, env, sm.classes, sub, dump);
+        flush_now<MAXGAP>(in.qn, ls, env, sm.classes, sub, P, oc);
         if (has && status == 0) lane_advance<MAXGAP>(in, 0, true, env, status);
         __syncwarp();
-        flush_now<MAXGAP>(in.qn, ls, env, sm.classes, sub, dump);
+        flush_now<MAXGAP>(in.qn, ls, env, sm.classes, sub, P, oc);
         Stats st = ls.st;
         st.checksum += rej_sum;
         uint32_t h[8];
