@@ -82,6 +82,15 @@ extern "C" {
                                     distributor's prediction is unchanged.  Same limits as
                                     MAASO_FLAG_ENGINE_FROZEN (lane-group mapping, at most 32 instances). */
 
+#define MAASO_FLAG_INSTANCE_QUEUES 8u /* a request whose chosen instance is full queues THERE (Sec. II-A: requests
+                                        beyond the batch cap wait in the instance's queue) instead of at the
+                                        dispatcher: it takes the slot that frees first (lowest slot among equal
+                                        finish times), starts at that time with the speed of the level then
+                                        (1 + the other slots still busy), and the dispatcher goes on to the
+                                        next request at once: one distributor round per request.  Implies the
+                                        engine of MAASO_FLAG_ENGINE_FROZEN (a queued request's times must be
+                                        known when it is handed over) and has its limits. */
+
 #define MAASO_FLAG_TEST_STALL 0x80000000u /* test hook for the bounded device-side waits: the trace copies
                                              are never issued and every wait is limited to about 0.1 s, so
                                              each valid candidate must come back with MAASO_CAND_ETIMEOUT

@@ -9,6 +9,7 @@ _SRC = os.path.join(_HERE, "maaso_oracle.c")
 _SO = os.path.join(_HERE, "libmaaso_oracle.so")
 
 FLAG_PRED_OPTIMISTIC = 1
+FLAG_INSTANCE_QUEUES = 8  # requests wait at their instance, not at the dispatcher (implies the fixed-speed engine)
 FLAG_TBT_MAXGAP = 4      # hit test on the largest token gap instead of the mean gap
 FLAG_ENGINE_FROZEN = 2   # decode speed fixed at admission (see frozen_replay in maaso_oracle.c)
 STATUS = {"EBUDGET": 1, "EMEMFIT": 2, "ETOOMANY": 4, "EBADINST": 8, "ETIMEOUT": 16, "ELOOP": 32,

@@ -67,6 +67,8 @@
 #define ORC_FLAG_PRED_OPTIMISTIC 1u
 #define ORC_FLAG_TBT_MAXGAP 4u    /* the TBT term of the hit test looks at the largest gap between two
                                      consecutive tokens of the request instead of the mean gap */
+#define ORC_FLAG_INSTANCE_QUEUES 8u /* requests wait at the instance they were given, not at the dispatcher
+                                       (implies the engine that fixes the decode speed at admission) */
 #define ORC_FLAG_ENGINE_FROZEN 2u /* the paper-literal engine: decode speed fixed at admission (below) */
 
 typedef struct {
@@ -246,6 +248,16 @@ static uint32_t validate(const orc_profile *p, const uint32_t *inst, uint32_t n_
  *     `now` to that time and the choice is made again;
  *   - everything about a request is known at admission, so it is accounted there.
  * With B = 1 everywhere the two engines coincide (nobody runs beside anybody).
+ *
+ * Per-instance queues (ORC_FLAG_INSTANCE_QUEUES).  Sec. II-A lets requests beyond the batch cap
+ * wait "in a waiting queue" of the instance, and Sec. IV-F step 2 sends a request to the instance
+ * with the shortest queue.  In this engine every finish time is known, so the queue of an
+ * instance can be measured in time: a request that finds every slot busy is given, at its
+ * arrival, to the feasible instance where it would get its first token earliest, takes the slot
+ * that frees first there (lowest index among equals), starts when that slot frees and runs at
+ * the step of the level it finds then (1 + the other slots still busy at that moment).  The
+ * dispatcher does not wait: the next request is handled at its own arrival time, so requests
+ * queue per instance, first come first served, and a request for another instance can overtake.
  */
 typedef struct {
     uint32_t model, B;
@@ -324,6 +336,23 @@ static void frozen_replay(ctx_t *c, const orc_profile *p, const uint32_t *inst, 
                 break;
             }
             if (pick_start <= clock) c->bad = 1;
+            if (flags & ORC_FLAG_INSTANCE_QUEUES) { /* queue at the chosen instance; the dispatcher moves on */
+                frozen_inst_t *f = &F[pick];
+                uint32_t j = f->B;
+                for (uint32_t x = 0; x < f->B; x++)
+                    if (j == f->B || f->until[x] < f->until[j]) j = x; /* the slot that frees first */
+                if (j >= f->B || !f->busy[j] || f->until[j] != pick_start) { c->bad = 1; break; }
+                uint32_t still = 0; /* other slots still busy when this one frees */
+                for (uint32_t x = 0; x < f->B; x++)
+                    if (x != j && f->until[x] > pick_start) still++;
+                int64_t q_speed = f->step[still];
+                int64_t q_first = pick_start + f->pre_base + (int64_t)(((uint64_t)f->pre_q16 * q->in_tokens + 32768u) >> 16);
+                int64_t q_end = q_first + (len - 1) * q_speed;
+                f->until[j] = q_end;
+                complete(c, pick, (uint32_t)r, q->arrival_us, q_first, q_end, (uint32_t)len, q->cls,
+                         len > 1 ? q_speed : 0);
+                break;
+            }
             clock = pick_start; /* wait for that slot, then choose again */
         }
     }
@@ -368,7 +397,7 @@ int orc_eval_candidate(const orc_profile *p, const orc_request *reqs, uint64_t n
         I[i].pre_q16 = (int64_t)(uint32_t)p->prefill_q16[row];
     }
 
-    if (flags & ORC_FLAG_ENGINE_FROZEN) {
+    if (flags & (ORC_FLAG_ENGINE_FROZEN | ORC_FLAG_INSTANCE_QUEUES)) {
         frozen_replay(&c, p, inst, n_inst, reqs, n, classes, has_mask, class_mask, flags, out);
         goto replay_done;
     }

@@ -25,6 +25,7 @@ assert REQUEST_DTYPE.itemsize == 16 and SLO_DTYPE.itemsize == 24 and RESULT_DTYP
 FLAG_PRED_OPTIMISTIC = 1
 FLAG_ENGINE_FROZEN = 2
 FLAG_TBT_MAXGAP = 4
+FLAG_INSTANCE_QUEUES = 8
 FLAG_TEST_STALL = 0x80000000
 MAP_AUTO, MAP_BLOCK, MAP_GROUP = 0, 1, 2
 CAND_STATUS = {"EBUDGET": 1, "EMEMFIT": 2, "ETOOMANY": 4, "EBADINST": 8, "ETIMEOUT": 16, "ELOOP": 32}

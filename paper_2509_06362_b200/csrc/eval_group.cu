@@ -384,6 +384,10 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                         } else if (am.tier == 0) {
                             if ((int)lane == am.winner) lane_admit<MAXGAP>(in, q, req, pre, now, env, status);
                             pending = false;
+                        } else if constexpr (Inst::kQueues) {
+                            // every capable instance is full: the request queues at the chosen one
+                            if ((int)lane == am.winner) lane_admit_queued<MAXGAP>(in, q, req, pre, env, status);
+                            pending = false;
                         } else {
                             // every capable instance is full: wait until the chosen slot frees (the
                             // outcome is the same for all lanes of the group, so they are all here)
@@ -463,7 +467,14 @@ static GroupKernel group_kernel_of(uint32_t flags) {
         return opt ? eval_group_kernel<true, FrozenInst, MINB, MAXGAP> : eval_group_kernel<false, FrozenInst, MINB, MAXGAP>;
     return opt ? eval_group_kernel<true, LaneInst, MINB, MAXGAP> : eval_group_kernel<false, LaneInst, MINB, MAXGAP>;
 }
+template <bool MAXGAP>
+static GroupKernel queue_kernel_of(uint32_t flags) {
+    return (flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_group_kernel<true, QueueInst, 4, MAXGAP>
+                                                : eval_group_kernel<false, QueueInst, 4, MAXGAP>;
+}
 static GroupKernel group_kernel_for(uint32_t flags, int blocks_per_sm) {
+    if (flags & MAASO_FLAG_INSTANCE_QUEUES)  // one register budget for this mode
+        return (flags & MAASO_FLAG_TBT_MAXGAP) ? queue_kernel_of<true>(flags) : queue_kernel_of<false>(flags);
     if (flags & MAASO_FLAG_TBT_MAXGAP) return group_kernel_of<4, true>(flags);  // one register budget for this mode
     return blocks_per_sm >= 4 ? group_kernel_of<4, false>(flags) : group_kernel_of<3, false>(flags);
 }
@@ -480,7 +491,7 @@ static size_t group_smem_bytes(const EvalParams& P, int tile_recs, int blocks_pe
     size_t pool = budget > fixed ? budget - fixed : 0;
     pool -= pool % 128;
     size_t lane_units = 9;  // 8 key blocks + the block minima
-    if (P.flags & MAASO_FLAG_ENGINE_FROZEN) lane_units = 18;
+    if (P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_INSTANCE_QUEUES)) lane_units = 18;
     else if (P.flags & MAASO_FLAG_TBT_MAXGAP) lane_units = 9 + 4 * 8;
     const size_t all = (size_t)kGroupThreads * lane_units * kKeyUnitBytes;
     if (pool > all) pool = all;

@@ -17,6 +17,7 @@ constexpr uint64_t kKey64Empty = ~0ull;
 
 struct FrozenInst {
     static constexpr bool kAlwaysLoop = true;   // the single-round shortcut of the default engine does not hold here
+    static constexpr bool kQueues = false;      // a request that finds every instance full waits at the dispatcher
     static constexpr uint32_t kKeyWords = 2;    // 32-bit words per slot key
     static constexpr uint32_t kGapWords = 0;    // every gap of a request is its fixed speed: nothing to track
     uint64_t kmin;    // smallest slot key (the slot that frees next), kKey64Empty when idle
@@ -118,6 +119,57 @@ __device__ __forceinline__ void lane_admit(FrozenInst& in, const CookedReq& q, u
     in.kmin = min(in.kmin, key);
     in.mask |= 1ull << slot;
     in.w++;
+    const uint4 pa = make_uint4((uint32_t)first_tok, (uint32_t)((uint64_t)first_tok >> 32), (uint32_t)q.arrival,
+                                (uint32_t)((uint64_t)q.arrival >> 32));
+    const uint2 pb = make_uint2(req, (q.Sm1 + 1u) | (q.cls << 16));
+    lane_push_now<MAXGAP>(in, env, t_end, pa, pb, MAXGAP ? (q.Sm1 ? (int64_t)speed : 0) : -1, status);
+}
+
+// The same engine with a queue in front of every instance (Sec. II-A: requests beyond the batch
+// cap wait in the instance's queue): a request whose chosen instance is full is handed over at
+// once and starts when the slot that frees first frees; the dispatcher does not wait.
+struct QueueInst : FrozenInst {
+    static constexpr bool kQueues = true;
+};
+
+// Queued admission: the request takes over the slot with the smallest key (earliest finish,
+// lowest slot among equals) at that slot's finish time.  Its level counts the other slots still
+// busy at that moment, i.e. all of them except those that end at exactly the same time.
+template <bool MAXGAP>
+__device__ __forceinline__ void lane_admit_queued(FrozenInst& in, const CookedReq& q, uint32_t req, int64_t pre,
+                                                  const LaneEnv& env, uint32_t& status) {
+    uint64_t* keys = reinterpret_cast<uint64_t*>(env.keys);
+    uint64_t* bm = reinterpret_cast<uint64_t*>(env.bm_lo);
+    const uint32_t slot = (uint32_t)in.kmin & 63u, b = slot >> 3, sj = slot & 7u;
+    const int64_t start = (int64_t)(in.kmin >> 6);
+    uint64_t kv[8], mv[8];
+#pragma unroll
+    for (int j = 0; j < 8; j++) kv[j] = keys[8u * b + j];
+#pragma unroll
+    for (int j = 0; j < 8; j++) mv[j] = bm[j];
+#pragma unroll
+    for (int j = 0; j < 8; j++) kv[j] = (uint32_t)j == sj ? kKey64Empty : kv[j];
+    uint64_t bmin = min8_u64(kv);
+#pragma unroll
+    for (int j = 0; j < 8; j++) mv[j] = (uint32_t)j == b ? bmin : mv[j];
+    uint32_t same = 0;
+    if ((int64_t)(min8_u64(mv) >> 6) == start) {  // rare: some other slot ends at the same time
+        for (uint32_t x = 0; x < in.B; x++) same += (x != slot && (int64_t)(keys[x] >> 6) == start) ? 1u : 0u;
+    }
+    const uint32_t speed = (uint32_t)in.step[in.B - 1u - same];
+    const int64_t first_tok = start + pre;
+    const int64_t t_end = first_tok + (int64_t)((uint64_t)q.Sm1 * speed);
+    if (((uint64_t)t_end >> 57) != 0) {
+        status = MAASO_CAND_ELOOP;
+        return;
+    }
+    const uint64_t key = ((uint64_t)t_end << 6) | slot;
+    keys[slot] = key;
+    bmin = min(bmin, key);
+    bm[b] = bmin;
+#pragma unroll
+    for (int j = 0; j < 8; j++) mv[j] = (uint32_t)j == b ? bmin : mv[j];
+    in.kmin = min8_u64(mv);
     const uint4 pa = make_uint4((uint32_t)first_tok, (uint32_t)((uint64_t)first_tok >> 32), (uint32_t)q.arrival,
                                 (uint32_t)((uint64_t)q.arrival >> 32));
     const uint2 pb = make_uint2(req, (q.Sm1 + 1u) | (q.cls << 16));

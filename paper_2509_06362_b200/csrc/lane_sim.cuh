@@ -51,7 +51,8 @@ constexpr size_t kLaneScratchBytes = kLaneScratchKeys + (9 + 4 * 8) * kKeyUnitBy
 static_assert(kLaneScratchBytes % 32 == 0 && kLaneScratchKeys % 16 == 0, "lane scratch layout");
 
 struct LaneInst {
-    static constexpr bool kAlwaysLoop = false;  // a wait is resolved in one round under the worst-case estimate
+    static constexpr bool kAlwaysLoop = false;
+    static constexpr bool kQueues = false;  // a wait is resolved in one round under the worst-case estimate
     static constexpr uint32_t kKeyWords = 1;    // 32-bit words per slot key
     static constexpr uint32_t kGapWords = 4;    // 32-bit words per slot of gap data (largest-gap mode only)
     int64_t T;        // clock, always a decode-step boundary (may lag `now` while the instance is full)

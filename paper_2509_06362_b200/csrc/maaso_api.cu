@@ -381,10 +381,13 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     if (o.dump_n && !o.dump_cand_idx) return fail(ctx, MAASO_EINVAL, "eval: dump_n without dump_cand_idx");
     if (n_traces > 1 && (o.dump_n || o.mapping == MAASO_MAP_BLOCK))
         return fail(ctx, MAASO_EINVAL, "eval: several traces in one call allow no dump buffers and no block mapping");
-    if (o.flags & ~(MAASO_FLAG_PRED_OPTIMISTIC | MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_TEST_STALL))
+    if (o.flags & ~(MAASO_FLAG_PRED_OPTIMISTIC | MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES |
+                    MAASO_FLAG_TEST_STALL))
         return fail(ctx, MAASO_EINVAL, "eval: unknown flag");
-    if ((o.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP)) && o.mapping == MAASO_MAP_BLOCK)
-        return fail(ctx, MAASO_EINVAL, "eval: the fixed-speed engine and the largest-gap test have no block mapping");
+    if ((o.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES)) &&
+        o.mapping == MAASO_MAP_BLOCK)
+        return fail(ctx, MAASO_EINVAL,
+                    "eval: the fixed-speed engine, per-instance queues and the largest-gap test have no block mapping");
 
     DeviceGuard g(ctx->device);
     cudaStream_t stream = (cudaStream_t)cuda_stream;

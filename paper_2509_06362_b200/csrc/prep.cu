@@ -13,7 +13,7 @@ __global__ void prep_kernel(const EvalParams P) {
         status = MAASO_CAND_EBADINST;  // malformed CSR row
     } else {
         n = hi - lo;
-        if (n > MAASO_MAX_INSTANCES || (((P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP)) || P.n_traces > 1) && n > 32)) {
+        if (n > MAASO_MAX_INSTANCES || (((P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES)) || P.n_traces > 1) && n > 32)) {
             status = MAASO_CAND_ETOOMANY;  // these options exist in the lane-group kernel only
         } else {
             uint64_t devsum = 0;

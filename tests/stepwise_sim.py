@@ -139,7 +139,8 @@ def simulate(profile, trace, classes, instances, class_mask=None, optimistic=Fal
     return st
 
 
-def simulate_frozen(profile, trace, classes, instances, class_mask=None, optimistic=False, maxgap=False):
+def simulate_frozen(profile, trace, classes, instances, class_mask=None, optimistic=False, maxgap=False,
+                    queues=False):
     """The engine that fixes a request's decode speed at admission, in a formulation that
     shares nothing with the C oracle's: no slots at all.  Every instance keeps the list of
     token timestamps of the requests admitted to it (one list per request, built token by
@@ -177,7 +178,9 @@ def simulate_frozen(profile, trace, classes, instances, class_mask=None, optimis
                     continue
                 alive = ends_after(ins, t_now)
                 free = len(alive) < ins["cap"]
-                start = t_now if free else min(alive)
+                # full: a place frees when fewer than cap of the requests sent here so far are unfinished
+                # (first come first served; with queues some of them have not even started yet)
+                start = t_now if free else sorted(alive)[-ins["cap"]]
                 per_tok = ins["step"][ins["cap"] - 1]
                 if optimistic and free:
                     per_tok = ins["step"][len(alive)]          # level len(alive) + 1
@@ -195,12 +198,13 @@ def simulate_frozen(profile, trace, classes, instances, class_mask=None, optimis
                 finish[k] = first[k] = where[k] = -1
                 break
             tier, _, idx, start = min(options)
-            if tier == 1:
+            if tier == 1 and not queues:
                 t_now = start
                 continue
             ins = insts[idx]
-            gap = ins["step"][len(ends_after(ins, t_now))]      # fixed for the whole request
-            stamps = [t_now + ins["base"] + ((ins["q16"] * n_in + 32768) >> 16)]
+            t_adm = t_now if tier == 0 else start               # queued: starts when that request ends
+            gap = ins["step"][len(ends_after(ins, t_adm))]      # fixed for the whole request
+            stamps = [t_adm + ins["base"] + ((ins["q16"] * n_in + 32768) >> 16)]
             for _ in range(S - 1):
                 stamps.append(stamps[-1] + gap)
             ins["tokens"].append(stamps)

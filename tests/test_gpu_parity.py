@@ -24,7 +24,7 @@ def ctx():
 @pytest.mark.parametrize("case", all_cases(), ids=lambda c: c["name"])
 def test_hand_timelines_on_gpu(ctx, case, mapping):
     for flags, expect in case["runs"]:
-        if (flags & 6) and mapping == 1:
+        if (flags & 14) and mapping == 1:
             continue      # the fixed-speed engine and the largest-gap test exist in the lane-group mapping only
         res, dumps = gpu_eval(ctx, case["profile"], case["trace"], case["classes"], case["offsets"],
                               case["inst"], case["budget"], None, flags, mapping, dump_idx=[0])
@@ -612,7 +612,7 @@ def test_ttft_histogram_bin_edges_on_gpu(ctx, oracle_mod):
 
 
 # ---- the engine that fixes the decode speed at admission (flag 2) ----------------------------
-@pytest.mark.parametrize("flags", [2, 3])
+@pytest.mark.parametrize("flags", [2, 3, 8, 9, 10])
 def test_frozen_engine_tiny_config_full(ctx, oracle_mod, flags):
     cfg = gen.make_config("tiny")
     tr = cfg["traces"][0]
@@ -625,9 +625,14 @@ def test_frozen_engine_tiny_config_full(ctx, oracle_mod, flags):
     for k in wd:
         assert (gd[k] == wd[k]).all(), k
     assert int(want["n_served"].sum()) > 0 and int(want["n_rejected"].sum()) > 0
+    if flags & 8:       # queues at the instances: one distributor round per request, and some requests did wait
+        assert (want["attempts"] == want["n_counted"]).all()
+        plain = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"],
+                                           cfg["budget"], None, (flags & 1) | 2)
+        assert int((plain["attempts"] > plain["n_counted"]).sum()) > 0
 
 
-@pytest.mark.parametrize("flags", [2, 3])
+@pytest.mark.parametrize("flags", [2, 3, 8, 9])
 def test_frozen_engine_node_and_multimodel_subsets(ctx, oracle_mod, flags):
     # ragged trace length (tiles of 64 + a tail), every group width up to 32 lanes, class masks, dumps
     cfg = gen.make_config("node", n_req=1777)
@@ -671,6 +676,8 @@ def test_frozen_engine_limits(ctx):
     d_off, d_inst = ctx.to_device(cfg["offsets"]), ctx.to_device(cfg["inst"])
     with pytest.raises(m.MaasoError):
         ctx.eval_placements(t, d_off, d_inst, 4, flags=2, mapping=1)
+    with pytest.raises(m.MaasoError):
+        ctx.eval_placements(t, d_off, d_inst, 4, flags=8, mapping=1)
     off, inst = gen.candidates_from_lists([[(0, 0, 1)] * 33, [(0, 0, 1)] * 32])
     import torch
     out = ctx.eval_placements(t, ctx.to_device(off), ctx.to_device(inst), 64, flags=2)
@@ -680,7 +687,7 @@ def test_frozen_engine_limits(ctx):
     ctx.free_trace(t)
 
 
-@pytest.mark.parametrize("flags", [0, 1, 2, 3, 4, 5])
+@pytest.mark.parametrize("flags", [0, 1, 2, 3, 4, 5, 8, 13])
 def test_slot_keys_in_global_scratch_when_the_pool_is_too_small(oracle_mod, flags):
     """A context created with MAASO_GROUP_BLOCKS=8 leaves no shared memory for the key pool, so
     every lane keeps its slot keys in global scratch: same results."""
@@ -713,7 +720,7 @@ def test_slot_keys_in_global_scratch_when_the_pool_is_too_small(oracle_mod, flag
 
 
 # ---- TBT term of the hit test on the largest token gap (flag 4) -------------------------------
-@pytest.mark.parametrize("flags", [4, 5, 6, 7])
+@pytest.mark.parametrize("flags", [4, 5, 6, 7, 12])
 def test_largest_gap_hit_test(ctx, oracle_mod, flags):
     """Default and fixed-speed engine, with and without the optimistic estimate; limits tight
     enough for prefill stalls to matter; every group width; ragged trace; dumps."""
@@ -734,7 +741,7 @@ def test_largest_gap_hit_test(ctx, oracle_mod, flags):
     for k in wd:
         assert (gd[k] == wd[k]).all(), k
     mean_form = oracle_mod.eval_placements(cfg["profile"], tr, tight, off, inst, 8, None, flags & ~4)
-    if not flags & 2:
+    if not flags & 10:
         assert int((mean_form["n_hit"] - want["n_hit"]).sum()) > 0     # the option changes something here
 
     cfg = gen.make_config("multimodel", n_cand=400, n_req=2500)
@@ -754,7 +761,7 @@ def test_largest_gap_hit_test(ctx, oracle_mod, flags):
 
 
 # ---- several traces in one pass ----------------------------------------------------------------
-@pytest.mark.parametrize("flags", [0, 1, 2, 4])
+@pytest.mark.parametrize("flags", [0, 1, 2, 4, 8])
 def test_several_traces_in_one_pass(ctx, oracle_mod, flags):
     """The bursty load sweep, cut down: the candidate set against 5 traces of different rates and
     lengths in one call; every block of records must equal the oracle's for that trace, and so must

@@ -58,6 +58,13 @@ MUTANTS = [
     ("largest gap is not kept across jumps", "if (gap > sl->max_gap) sl->max_gap = gap;", "sl->max_gap = gap;"),
     ("largest gap of a new request starts at the boundary", "sl->last_tok = in->T; sl->max_gap = 0;",
      "sl->last_tok = in->T - prefill_us(in, q->in_tokens); sl->max_gap = 0;"),
+    ("queued request takes the level of its arrival time", "if (x != j && f->until[x] > pick_start) still++;",
+     "if (x != j && f->until[x] > clock) still++;"),
+    ("queued request starts at its arrival", "int64_t q_first = pick_start + f->pre_base", "int64_t q_first = clock + f->pre_base"),
+    ("queued request: finish counts one token too many", "int64_t q_end = q_first + (len - 1) * q_speed;",
+     "int64_t q_end = q_first + len * q_speed;"),
+    ("queued request takes the last slot to free", "if (j == f->B || f->until[x] < f->until[j]) j = x; /* the slot that frees first */",
+     "if (j == f->B || f->until[x] > f->until[j]) j = x;"),
     ("prefill does not stall the running batch", "in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {",
      "int64_t t_keep = in->T; in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {"),
 ]
@@ -107,6 +114,9 @@ def run_pins(mod):
     for seed in (0, 1, 2, 3):
         attempt(f"largest gap {seed}", pins.test_maxgap_against_token_timestamps, seed)
     attempt("largest gap vs mean", pins.test_maxgap_only_changes_the_hit_test)
+    for seed in (0, 1, 2, 3):
+        attempt(f"instance queues {seed}", pins.test_instance_queues_against_token_lists, seed)
+    attempt("instance queues structure", pins.test_instance_queues_structure_from_the_dumps)
     attempt("histogram edges", pins.test_ttft_histogram_bin_edges)
     attempt("histogram counts", pins.test_ttft_histogram_counts_served_requests_only)
     attempt("percentiles", pins.test_ttft_percentiles_by_hand)

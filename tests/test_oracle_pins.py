@@ -202,6 +202,53 @@ def test_frozen_engine_levels_recomputed_from_the_dumps(oracle_mod):
                         assert t_fin - int(d["first_us"][row][r]) == (S - 1) * int(prof["step_us"][m, s, running])
 
 
+# ---- requests queue at their instance, not at the dispatcher (flag 8) --------------------------
+QUEUES = 8
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_instance_queues_against_token_lists(oracle_mod, seed):
+    prof, trace, classes, instances = _random_small_case(seed)
+    mask = None if seed % 4 else 0b011
+    opt = seed % 2
+    res, d = run_one(oracle_mod, prof, trace, classes, instances, mask=mask, flags=QUEUES | opt)
+    ref = simulate_frozen(prof, trace, classes, instances, class_mask=mask, optimistic=bool(opt), queues=True)
+    for key in SCALAR_KEYS:
+        assert int(res[key]) == ref[key], key
+    assert d["finish_us"].tolist() == ref["finish_us"]
+    assert d["first_us"].tolist() == ref["first_us"]
+    assert d["inst"].tolist() == ref["inst"]
+
+
+def test_instance_queues_structure_from_the_dumps(oracle_mod):
+    """From the per-request times alone: one distributor round per request; on every instance the
+    requests start in arrival order (first come first served), never more than B hold a slot at once,
+    and a request never starts before its arrival."""
+    cfg = gen.make_config("tiny", n_req=300)
+    prof, tr = cfg["profile"], cfg["traces"][0]
+    off, inst = cfg["offsets"], cfg["inst"]
+    pick = np.arange(0, len(off) - 1, 7)
+    res, d = oracle_mod.eval_placements(prof, tr, cfg["classes"], off, inst, cfg["budget"], flags=QUEUES, dump_idx=pick)
+    waited = 0
+    for row, c in enumerate(pick):
+        assert int(res[c]["attempts"]) == int(res[c]["n_counted"])
+        for i, word in enumerate(inst[off[c]:off[c + 1]]):
+            m, s, B = int(word & 15), int((word >> 4) & 255), int((word >> 12) & 255)
+            mine = np.nonzero(d["inst"][row] == i)[0]
+            starts, spans = [], []
+            for r in mine:
+                pre = int(prof["prefill_base_us"][m, s]) + ((int(prof["prefill_q16"][m, s]) * int(tr["in_tokens"][r]) + 32768) >> 16)
+                t_adm = int(d["first_us"][row][r]) - pre
+                assert t_adm >= int(tr["arrival_us"][r])
+                waited += t_adm > int(tr["arrival_us"][r])
+                starts.append(t_adm)
+                spans.append((t_adm, int(d["finish_us"][row][r])))
+            assert starts == sorted(starts)
+            for (a, f) in spans:
+                assert sum(1 for (a2, f2) in spans if a2 <= a < f2) <= B
+    assert waited > 0
+
+
 # ---- TBT term of the hit test on the largest token gap (flag 4) -------------------------------
 MAXGAP = 4
 
