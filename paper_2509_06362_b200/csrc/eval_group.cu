@@ -147,10 +147,12 @@ __device__ __forceinline__ void flush_if_due(uint32_t& qn, LaneStats& ls, const 
 }
 
 // OPT: the distributor predicts with the step time right after admission (optimistic estimate).
-// Inst: LaneInst (default engine: decode speed follows the running count) or FrozenInst (speed
-// fixed at admission).  MAXGAP: the TBT term of the hit test looks at the largest token gap.  MINB: blocks per SM the register budget must allow: 4 for batches that
-// fill the GPU (128 registers), 3 for batches of one wave, which are bound by their longest
-// dependent chains and run a little faster without the spills of the tighter budget.
+// Inst: LaneInst (default engine: decode speed follows the running count), FrozenInst (speed
+// fixed at admission) or QueueInst (FrozenInst with a queue in front of every instance).
+// MAXGAP: the TBT term of the hit test looks at the largest token gap.  MINB: blocks per SM the
+// register budget must allow: 4 for batches of many waves (127 registers), 3 for batches of one
+// wave, which are bound by their longest dependent chains and run a little faster with fewer
+// warps per scheduler and 144 registers.
 template <bool OPT, class Inst, int MINB, bool MAXGAP>
 __global__ void __launch_bounds__(kGroupThreads, MINB)
 eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_bytes) {
