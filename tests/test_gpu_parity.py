@@ -171,6 +171,19 @@ def test_node_config_full_size_as_benchmarked(ctx, oracle_mod):
     assert_records_equal(got, want, "node full, block mapping")
 
 
+@pytest.mark.parametrize("flags", [1, 2, 4, 8, 9])
+def test_node_config_full_size_variants_sampled(ctx, oracle_mod, flags):
+    """The other readings on the benchmark's workload, full size on the GPU (so that every placement sits
+    in the launch bucket, warp and lane it gets there); every 50th record checked against the oracle."""
+    cfg = gen.make_config("node")
+    tr = cfg["traces"][0]
+    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, None, flags, 0)
+    sel = list(range(0, 10864, 50)) + [10863]
+    off, inst = _subset(cfg, sel)
+    want = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 8, None, flags)
+    assert_records_equal(got[sel], want, f"node full, flags {flags}, sampled")
+
+
 def test_multimodel_full_trace_sampled_candidates(ctx, oracle_mod):
     cfg = gen.make_config("multimodel")
     tr = cfg["traces"][0]
