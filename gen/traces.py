@@ -49,3 +49,23 @@ def make_trace(n, rate, seed, *, cv=1.0, class_mix=(0.5, 0.3, 0.2), model_mix=(1
     t["cls"] = cls
     t["model"] = model
     return t
+
+
+def trace_from_rows(rows):
+    """rows: (arrival_us, in_tokens, out_tokens, cls, model) per request, in arrival order."""
+    t = np.zeros(len(rows), dtype=REQUEST_DTYPE)
+    for k, (a, n_in, n_out, c, m) in enumerate(rows):
+        t[k] = (a, n_in, n_out, c, m)
+    return t
+
+
+def shrinking_prompts_trace(n_followers=40, spacing_us=30_000, first_prompt=90_000, prompt_step=2_000,
+                            long_out=6_000, follower_out=(150, 900), n_classes=3):
+    """One long-running request, then followers whose prompts shrink from one to the next while all of
+    them keep running: with a prefill time that falls faster than the decode step grows, every
+    admission stalls the batch for a little less than the one before."""
+    rows = [(0, 100, long_out, n_classes - 1, 0)]
+    for k in range(n_followers):
+        rows.append(((k + 1) * spacing_us, first_prompt - k * prompt_step,
+                     follower_out[0] + (k * 37) % (follower_out[1] - follower_out[0]), k % n_classes, 0))
+    return trace_from_rows(rows)

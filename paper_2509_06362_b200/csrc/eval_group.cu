@@ -191,6 +191,8 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
     env.qg = MAXGAP ? sm.qg + tid : nullptr;
     env.mg = nullptr;
     env.dl = nullptr;
+    env.first = nullptr;
+    env.stk = nullptr;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
     const uint32_t n_traces = P.n_traces > 1 ? P.n_traces : 1u;
     uint32_t tile_seq = 0;  // tiles consumed so far by this warp (same in every warp)
@@ -277,8 +279,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
         // pool cannot hold use their global scratch instead
         {
             const uint32_t nblk = has ? (in.B + 7u) >> 3 : 0u;
-            // largest-gap mode of the default engine: two more 8-byte words per slot after the minima
-            const uint32_t gap_units = MAXGAP ? nblk * 2u * Inst::kGapWords : 0u;  // 8 slots x words x 4 B / 32 B
+            // largest-gap mode of the default engine: per slot two 8-byte words and one 4-byte word after the
+            // minima (8 slots x words x 4 B = `words` units per block), then the lane's list of stretch gaps
+            const uint32_t gap_units = (MAXGAP && Inst::kGapWords) ? nblk * Inst::kGapWords + Inst::kGapListUnits : 0u;
             const uint32_t units = has ? (nblk + 1u) * Inst::kKeyWords + gap_units : 0u;
             uint32_t incl = units;
             for (uint32_t o = 1; o < 32u; o <<= 1) {
@@ -299,6 +302,8 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
             if (MAXGAP && Inst::kGapWords) {
                 env.mg = reinterpret_cast<uint64_t*>(region + (size_t)(nblk + 1u) * kKeyUnitBytes * Inst::kKeyWords);
                 env.dl = env.mg + 8u * nblk;
+                env.first = reinterpret_cast<uint32_t*>(env.dl + 8u * nblk);
+                env.stk = reinterpret_cast<uint4*>(env.first + 8u * nblk);
             }
             const uint4 e4 = make_uint4(kKeyEmpty, kKeyEmpty, kKeyEmpty, kKeyEmpty);
             for (uint32_t i = 0; i < 2u * units; i++) reinterpret_cast<uint4*>(region)[i] = e4;
@@ -494,7 +499,7 @@ static size_t group_smem_bytes(const EvalParams& P, int tile_recs, int blocks_pe
     pool -= pool % 128;
     size_t lane_units = 9;  // 8 key blocks + the block minima
     if (P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_INSTANCE_QUEUES)) lane_units = 18;
-    else if (P.flags & MAASO_FLAG_TBT_MAXGAP) lane_units = 9 + 4 * 8;
+    else if (P.flags & MAASO_FLAG_TBT_MAXGAP) lane_units = 9 + 5 * 8 + 8;
     const size_t all = (size_t)kGroupThreads * lane_units * kKeyUnitBytes;
     if (pool > all) pool = all;
     *pool_bytes = (uint32_t)pool;

@@ -20,6 +20,7 @@ struct FrozenInst {
     static constexpr bool kQueues = false;      // a request that finds every instance full waits at the dispatcher
     static constexpr uint32_t kKeyWords = 2;    // 32-bit words per slot key
     static constexpr uint32_t kGapWords = 0;    // every gap of a request is its fixed speed: nothing to track
+    static constexpr uint32_t kGapListUnits = 0;
     uint64_t kmin;    // smallest slot key (the slot that frees next), kKey64Empty when idle
     uint64_t mask;    // busy slots; bits at and above B are always set
     uint32_t w;       // busy slots (requests running at the time of the last release)

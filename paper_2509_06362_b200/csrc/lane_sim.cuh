@@ -47,14 +47,15 @@ constexpr size_t kLaneScratchA = 0;
 constexpr size_t kLaneScratchB = 64 * 2 * 16;
 constexpr size_t kLaneScratchOvf = kLaneScratchB + 64 * 2 * 8;
 constexpr size_t kLaneScratchKeys = kLaneScratchOvf + (size_t)kQueueOvf * kOvfEntryBytes;
-constexpr size_t kLaneScratchBytes = kLaneScratchKeys + (9 + 4 * 8) * kKeyUnitBytes + 32;
+constexpr size_t kLaneScratchBytes = kLaneScratchKeys + (9 + 5 * 8 + 8) * kKeyUnitBytes + 32;
 static_assert(kLaneScratchBytes % 32 == 0 && kLaneScratchKeys % 16 == 0, "lane scratch layout");
 
 struct LaneInst {
     static constexpr bool kAlwaysLoop = false;
     static constexpr bool kQueues = false;  // a wait is resolved in one round under the worst-case estimate
     static constexpr uint32_t kKeyWords = 1;    // 32-bit words per slot key
-    static constexpr uint32_t kGapWords = 4;    // 32-bit words per slot of gap data (largest-gap mode only)
+    static constexpr uint32_t kGapWords = 5;    // 32-bit words per slot of gap data (largest-gap mode only)
+    static constexpr uint32_t kGapListUnits = 8; // 32-byte units of the lane's list of stretch gaps (16 entries)
     int64_t T;        // clock, always a decode-step boundary (may lag `now` while the instance is full)
     int64_t tc;       // time of the next completion if nobody is admitted (valid while w > 0)
     uint32_t K;       // decode steps done at T since the counter last restarted
@@ -67,7 +68,9 @@ struct LaneInst {
     uint64_t mask;    // occupied slots; bits at and above B are always set
     uint64_t gen;     // per slot: which of its two scratch entries the current occupant uses
     uint64_t stall;   // largest-gap mode: prefill time since the instance's latest decode-step end
-    bool dirty;       // largest-gap mode: an admission or a retirement happened since the gaps were last folded in
+    bool dirty;       // largest-gap mode: an admission or a retirement happened since the latest stretch was recorded
+    uint32_t sidx;    // largest-gap mode: index of the next stretch (decode steps at one level, after one stall)
+    uint32_t sdepth;  // largest-gap mode: entries in the lane's list of stretch gaps
     const int32_t* step;  // shared-memory row: step[w-1] = one decode step with w running
     uint32_t stepB;   // step[B-1]
     uint32_t pre_base, pre_q16;
@@ -86,8 +89,10 @@ struct LaneEnv {
     uint2* pay_b;            // global scratch [64][2]: request index, S | cls << 16
     unsigned char* ovf;      // this lane's queue overflow (global scratch, kOvfEntryBytes each)
     int64_t* qg;             // largest-gap mode: entry j at qg[j * kGroupThreads] = largest token gap; else null
-    uint64_t* mg;            // largest-gap mode: per slot, largest token gap so far (pool slice, after the minima)
-    uint64_t* dl;            // largest-gap mode: per slot, time from the latest step end to the slot's latest token
+    uint64_t* mg;            // largest-gap mode: per slot, largest gap among stretches that left the list (after the minima)
+    uint64_t* dl;            // largest-gap mode: per slot, part of its first stretch's stall that ended with its first token
+    uint32_t* first;         // largest-gap mode: per slot, index of the first stretch its request takes part in
+    uint4* stk;              // largest-gap mode: list of stretch gaps {gap lo, gap hi, stretch index, -}, decreasing gaps
 };
 
 // Per-lane sums of completed requests; only flush_queue touches them.
@@ -241,7 +246,7 @@ __device__ __noinline__ void flush_queue_maxgap(LaneStats* ls, const int64_t* qf
 
 __device__ __forceinline__ void lane_reset(LaneInst& in, const int32_t* steps) {
     in.T = 0; in.tc = 0; in.K = 0; in.w = 0; in.kmin = kKeyEmpty; in.sw = 1; in.rsw = 1.0f; in.qn = 0;
-    in.mask = ~0ull; in.gen = 0; in.stall = 0; in.dirty = false;
+    in.mask = ~0ull; in.gen = 0; in.stall = 0; in.dirty = false; in.sidx = 0; in.sdepth = 0;
     in.B = 1; in.model = 0xFFFFFFFFu; in.step = steps; in.stepB = 1; in.pre_base = 0; in.pre_q16 = 0;
 }
 
@@ -249,21 +254,64 @@ __device__ __forceinline__ void lane_reset(LaneInst& in, const int32_t* steps) {
 // request that ends here, one per round (the smallest key names its slot), fix the block
 // minima, the level and the cached next completion.
 // Largest-gap mode.  The instance is about to take its first decode step(s) since an admission or a
-// retirement: every running request's next token comes `stall` (prefills since the latest step
-// end) plus one step after that step end, minus what the request itself has already waited there
-// (a request admitted at this boundary got its first token part-way through the stall).  Further
-// steps of the same stretch are not longer.  Folded into every slot of the lane's blocks; slots
-// that are empty hold garbage until an admission resets them.
+// retirement: a new stretch.  Every running request's next token comes `stall` (prefills since the
+// latest step end) plus one step after that step end; a request admitted at this boundary got its
+// first token part-way through the stall and waits that much less.  Further steps of the stretch
+// are not longer.  A request's largest gap is therefore the maximum of the stretch gaps over the
+// stretches it lives through, minus its own part of the stall in the first one.  The lane keeps
+// the suffix maxima of the stretch gaps (a list with decreasing gaps and increasing stretch
+// indices: the largest gap of stretches a..now is the oldest entry with index >= a), so a new
+// stretch costs a few pops and one push and a completion one look-up.
+constexpr uint32_t kGapList = 16;
+
+__device__ __forceinline__ uint64_t gap_of(const uint4& e) { return ((uint64_t)e.y << 32) | e.x; }
+
+// The list is full of strictly decreasing gaps: fold its oldest entry into the slots it concerns
+// (exactly what the look-up would have found there) and drop it.  Rare, kept out of line.
+__device__ __noinline__ void gaps_drop_oldest(uint64_t* mg, uint64_t* dl, uint32_t* first, uint4* stk, uint32_t nslots) {
+    const uint4 e = stk[0];
+    const uint64_t v = gap_of(e);
+    for (uint32_t i = 0; i < nslots; i++) {
+        const uint32_t f = first[i];
+        if (f > e.z) continue;
+        mg[i] = max(mg[i], f == e.z ? v - dl[i] : v);
+        first[i] = e.z + 1u;  // later stretches are still in the list, without a share of a stall
+        dl[i] = 0;
+    }
+    for (uint32_t j = 0; j + 1u < kGapList; j++) stk[j] = stk[j + 1u];
+}
+
 __device__ __forceinline__ void gaps_fold(LaneInst& in, const LaneEnv& env) {
     const uint64_t g = in.stall + in.sw;
-    const uint32_t n = 8u * ((in.B + 7u) >> 3);
-    for (uint32_t i = 0; i < n; i++) {
-        const uint64_t cand = g - env.dl[i];
-        env.mg[i] = max(env.mg[i], cand);
-        env.dl[i] = 0;
+    uint32_t d = in.sdepth;
+    while (d > 0 && gap_of(env.stk[d - 1u]) <= g) d--;  // dominated by this stretch from now on
+    if (d == kGapList) {
+        gaps_drop_oldest(env.mg, env.dl, env.first, env.stk, 8u * ((in.B + 7u) >> 3));
+        d--;
     }
+    env.stk[d] = make_uint4((uint32_t)g, (uint32_t)(g >> 32), in.sidx, 0u);
+    in.sdepth = d + 1u;
+    in.sidx++;
     in.stall = 0;
     in.dirty = false;
+}
+
+// Largest token gap of the request in `slot`, which completes now (its last stretch is in the list).
+__device__ __forceinline__ uint64_t gaps_of_slot(const LaneInst& in, const LaneEnv& env, uint32_t slot) {
+    const uint32_t a = env.first[slot];
+    uint64_t r = env.mg[slot];
+    for (uint32_t j = 0; j < in.sdepth; j++) {
+        const uint4 e = env.stk[j];
+        if (e.z < a) continue;
+        uint64_t v = gap_of(e);
+        if (e.z == a) {  // its first stretch: it had waited part of the stall already
+            v -= env.dl[slot];
+            if (j + 1u < in.sdepth) v = max(v, gap_of(env.stk[j + 1u]));
+        }
+        r = max(r, v);
+        break;
+    }
+    return r;
 }
 
 template <bool MAXGAP>
@@ -287,7 +335,7 @@ __device__ __forceinline__ void lane_retire(LaneInst& in, const LaneEnv& env, ui
         in.mask &= ~(1ull << slot);
         in.w--;
         lane_push_slot<MAXGAP>(in, env, in.T, 2u * slot + (uint32_t)((in.gen >> slot) & 1ull),
-                               MAXGAP ? (int64_t)env.mg[slot] : -1, status);
+                               MAXGAP ? (int64_t)gaps_of_slot(in, env, slot) : -1, status);
     } while ((in.kmin >> 6) == Kc);
     if (MAXGAP) in.dirty = true;  // the level changes: the next step has another length
     if (in.w > 0) {
@@ -425,6 +473,7 @@ __device__ __forceinline__ void lane_admit(LaneInst& in, const CookedReq& q, uin
     if (MAXGAP) {  // no gap yet; its first token came `stall` after the latest step end
         env.mg[slot] = 0;
         env.dl[slot] = in.stall;
+        env.first[slot] = in.sidx;  // the stretch that the next clock movement opens
     }
     in.gen ^= 1ull << slot;
     const uint32_t idx = 2u * slot + (uint32_t)((in.gen >> slot) & 1ull);

@@ -773,6 +773,25 @@ def test_largest_gap_hit_test(ctx, oracle_mod, flags):
     assert_records_equal(got, want, "multimodel subset, largest-gap test")
 
 
+@pytest.mark.parametrize("flags", [4, 5])
+def test_largest_gap_when_the_list_of_stretch_gaps_overflows(ctx, oracle_mod, flags):
+    """Forty admissions whose stalls shrink one after the other while everybody keeps running: the lane's
+    list of stretch gaps (16 entries, decreasing) fills up and its oldest entries must be folded into
+    the slots.  Limits chosen so that the hit counts depend on each request's exact largest gap.  Also
+    with other placements in the same warp and with a second, smaller instance."""
+    prof = gen.make_config("tiny")["profile"]
+    trace = gen.shrinking_prompts_trace(n_classes=24)
+    classes = gen.make_classes([(None, 18_600 + 150 * c, None) for c in range(24)])   # a limit every 150 us
+    off, inst = gen.candidates_from_lists([[(0, 0, 64)], [(0, 0, 64), (0, 0, 8)], [(0, 0, 48)], [(0, 0, 40), (0, 0, 24)]])
+    idx = np.arange(4, dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(prof, trace, classes, off, inst, 4, None, flags, dump_idx=idx)
+    got, gd = gpu_eval(ctx, prof, trace, classes, off, inst, 4, None, flags, 0, dump_idx=idx)
+    assert_records_equal(got, want, "shrinking stalls")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+    assert int(want["n_served"][0]) == 41 and 5 < int(want["n_hit"][0]) < 36
+
+
 # ---- several traces in one pass ----------------------------------------------------------------
 @pytest.mark.parametrize("flags", [0, 1, 2, 4, 8])
 def test_several_traces_in_one_pass(ctx, oracle_mod, flags):

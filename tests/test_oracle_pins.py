@@ -202,6 +202,24 @@ def test_frozen_engine_levels_recomputed_from_the_dumps(oracle_mod):
                         assert t_fin - int(d["first_us"][row][r]) == (S - 1) * int(prof["step_us"][m, s, running])
 
 
+def test_largest_gap_with_stalls_that_shrink_from_one_admission_to_the_next(oracle_mod):
+    """Forty admissions in a row, each stalling the running batch a little less than the one before, none
+    of them finished yet: every request's largest gap is the stall right after its own admission, so
+    the hit counts step through the classes' limits.  Token timestamps of the step-by-step simulator."""
+    prof = gen.make_config("tiny")["profile"]
+    trace = gen.shrinking_prompts_trace(n_classes=24)
+    classes = gen.make_classes([(None, 18_600 + 150 * c, None) for c in range(24)])   # a limit every 150 us
+    for opt in (0, 1):
+        res, d = run_one(oracle_mod, prof, trace, classes, [(0, 0, 64)], flags=MAXGAP | opt)
+        ref = simulate(prof, trace, classes, [(0, 0, 64)], optimistic=bool(opt), maxgap=True)
+        for key in SCALAR_KEYS:
+            assert int(res[key]) == ref[key], key
+        assert d["finish_us"].tolist() == ref["finish_us"]
+        assert int(res["n_served"]) == 41 and 5 < int(res["n_hit"]) < 36
+        mean_form, _ = run_one(oracle_mod, prof, trace, classes, [(0, 0, 64)], flags=opt)
+        assert int(mean_form["n_hit"]) == 41
+
+
 # ---- requests queue at their instance, not at the dispatcher (flag 8) --------------------------
 QUEUES = 8
 
