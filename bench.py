@@ -27,8 +27,8 @@ TOPK = 64
 # ncu counters of eval_group_kernel on the default workload (profiles/eval_group_kernel_node_sweep.md).
 # They describe the kernel as committed with that summary; set to None when the kernel changes.
 PROFILED = {"workload": "node", "mapping": 0,
-            "dram_bytes_per_launch": 49_367_040 + 36_413_952,
-            "warp_inst_per_launch": 4_297_052_336}
+            "dram_bytes_per_launch": 49_585_664 + 36_903_424,
+            "warp_inst_per_launch": 4_299_223_620}
 SM_COUNT, ISSUE_PER_SM = 148, 4   # B200: 148 SMs x 4 warp schedulers, one warp instruction per cycle each
 
 
