@@ -117,6 +117,7 @@ def run_pins(mod):
     for seed in (0, 1, 2, 3):
         attempt(f"instance queues {seed}", pins.test_instance_queues_against_token_lists, seed)
     attempt("instance queues structure", pins.test_instance_queues_structure_from_the_dumps)
+    attempt("instance queues, one server", pins.test_instance_queues_single_server_is_the_lindley_recursion)
     attempt("histogram edges", pins.test_ttft_histogram_bin_edges)
     attempt("histogram counts", pins.test_ttft_histogram_counts_served_requests_only)
     attempt("percentiles", pins.test_ttft_percentiles_by_hand)

@@ -238,6 +238,27 @@ def test_instance_queues_against_token_lists(oracle_mod, seed):
     assert d["inst"].tolist() == ref["inst"]
 
 
+def test_instance_queues_single_server_is_the_lindley_recursion(oracle_mod):
+    """One instance with one slot, no limits: a first-come-first-served single-server queue, whose
+    departure times obey D_k = max(A_k, D_{k-1}) + service_k (textbook recursion); the service time
+    is prefill + (S - 1) steps at level 1."""
+    for seed in range(4):
+        prof, trace, _, instances = _random_small_case(seed)
+        m, s, _ = instances[0]
+        trace["model"] = m
+        classes = gen.make_classes([(None, None, None)] * 3)
+        res, d = run_one(oracle_mod, prof, trace, classes, [(m, s, 1)], flags=QUEUES)
+        step1 = int(prof["step_us"][m][s][0])
+        base, q16 = int(prof["prefill_base_us"][m][s]), int(prof["prefill_q16"][m][s]) & 0xFFFFFFFF
+        depart = 0
+        for k in range(len(trace)):
+            start = max(int(trace["arrival_us"][k]), depart)
+            first = start + base + ((q16 * int(trace["in_tokens"][k]) + 32768) >> 16)
+            depart = first + (int(trace["out_tokens"][k]) - 1) * step1
+            assert int(d["first_us"][k]) == first and int(d["finish_us"][k]) == depart, (seed, k)
+        assert int(res["n_served"]) == len(trace) and int(res["attempts"]) == len(trace)
+
+
 def test_instance_queues_structure_from_the_dumps(oracle_mod):
     """From the per-request times alone: one distributor round per request; on every instance the
     requests start in arrival order (first come first served), never more than B hold a slot at once,
