@@ -349,7 +349,9 @@ def main():
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": int(cfg["offsets"].nbytes + cfg["inst"].nbytes),
-                "d2h_bytes_per_step": int(n_tr * n_cand * 128)},
+                "d2h_bytes_per_step": int(n_tr * n_cand * 128),
+                "note": "host-buffer entry point: candidates copied in, all records copied out, every step; "
+                        "no top-k pass and no L2 flush between steps, hence a little above the device-timed value"},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "eval_group_kernel" if args.mapping == 0 else "eval_block_kernel",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
