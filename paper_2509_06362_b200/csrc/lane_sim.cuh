@@ -69,7 +69,8 @@ struct LaneInst {
     uint64_t gen;     // per slot: which of its two scratch entries the current occupant uses
     uint64_t stall;   // largest-gap mode: prefill time since the instance's latest decode-step end
     bool dirty;       // largest-gap mode: an admission or a retirement happened since the latest stretch was recorded
-    uint32_t sidx;    // largest-gap mode: index of the next stretch (decode steps at one level, after one stall)
+    uint32_t sidx;    // largest-gap mode: index of the next stretch (decode steps at one level, after one stall);
+                      // at most two per request of the lane, so 32 bits outlast any trace that fits the device
     uint32_t sdepth;  // largest-gap mode: entries in the lane's list of stretch gaps
     const int32_t* step;  // shared-memory row: step[w-1] = one decode step with w running
     uint32_t stepB;   // step[B-1]
