@@ -28,7 +28,8 @@ TOPK = 64
 # They describe the kernel as committed with that summary; set to None when the kernel changes.
 PROFILED = {"workload": "node", "mapping": 0,
             "dram_bytes_per_launch": 49_585_664 + 36_903_424,
-            "warp_inst_per_launch": 4_299_223_620}
+            "warp_inst_per_launch": 4_299_223_620,
+            "alu_pipe_busy": 0.412}   # sm__inst_executed_pipe_alu, share of its peak while an SM is active
 SM_COUNT, ISSUE_PER_SM = 148, 4   # B200: 148 SMs x 4 warp schedulers, one warp instruction per cycle each
 
 
@@ -338,7 +339,8 @@ def main():
         alu = {"bound": "alu", "kernel": "eval_group_kernel", "achieved": ach / 1e9, "peak": alu_peak / 1e9,
                "unit": "G warp-instructions/s", "frac": ach / alu_peak,
                "peak_kind": f"{SM_COUNT} SMs x {ISSUE_PER_SM} issue slots x {sm_mhz:.0f} MHz sampled during the run",
-               "warp_inst_per_eval": profiled["warp_inst_per_launch"] / evals_per_step}
+               "warp_inst_per_eval": profiled["warp_inst_per_launch"] / evals_per_step,
+               "alu_pipe_busy_profiled": profiled["alu_pipe_busy"]}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
