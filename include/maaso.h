@@ -97,9 +97,12 @@ extern "C" {
                                              and the call must return normally */
 
 /* maaso_eval_opts.mapping */
-#define MAASO_MAP_AUTO 0u  /* lanes-per-instance groups for <= 32 instances, one block otherwise */
-#define MAASO_MAP_BLOCK 1u /* one thread block per candidate, one warp per instance, lanes = slots */
-#define MAASO_MAP_GROUP 2u /* same as AUTO */
+#define MAASO_MAP_AUTO 0u   /* the library chooses: MAASO_MAP_THREAD where it exists, else MAASO_MAP_GROUP */
+#define MAASO_MAP_BLOCK 1u  /* one thread block per candidate, one warp per instance, lanes = slots */
+#define MAASO_MAP_GROUP 2u  /* one lane per instance, groups of lanes per candidate (<= 32 instances; one block
+                               per candidate beyond that) */
+#define MAASO_MAP_THREAD 3u /* one thread per candidate, looping over the instances of the request's model;
+                               default engine only (flags 0 or MAASO_FLAG_PRED_OPTIMISTIC), any instance count */
 
 typedef struct maaso_ctx maaso_ctx;
 typedef struct maaso_trace maaso_trace;
@@ -362,6 +365,7 @@ typedef struct {
     float group_ms; /* lane-group scoring kernel */
     float block_ms; /* block-layout scoring kernels */
     float topk_ms;  /* all passes of the last maaso_topk */
+    float thread_ms; /* thread-mapping scoring kernel */
 } maaso_timing;
 MAASO_API int maaso_set_timing(maaso_ctx *ctx, int enabled);
 MAASO_API int maaso_get_timing(maaso_ctx *ctx, maaso_timing *out);

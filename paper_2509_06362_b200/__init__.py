@@ -10,7 +10,7 @@ from .binding import (
     maaso_eval_placements, maaso_eval_placements_multi, maaso_eval_placements_host, maaso_topk, maaso_ins_deploy, maaso_partition, maaso_prune_configs, maaso_score, maaso_topk_scores, maaso_ttft_percentiles, maaso_topk_noalloc, NOALLOC_MAX_CAND, NOALLOC_MAX_K, maaso_launch_count, maaso_set_timing, maaso_get_timing,
     maaso_strerror, maaso_last_error, lib_path,
     REQUEST_DTYPE, SLO_DTYPE, RESULT_DTYPE,
-    FLAG_PRED_OPTIMISTIC, FLAG_ENGINE_FROZEN, FLAG_TBT_MAXGAP, FLAG_INSTANCE_QUEUES, FLAG_TEST_STALL, MAP_AUTO, MAP_BLOCK, MAP_GROUP, CAND_STATUS,
+    FLAG_PRED_OPTIMISTIC, FLAG_ENGINE_FROZEN, FLAG_TBT_MAXGAP, FLAG_INSTANCE_QUEUES, FLAG_TEST_STALL, MAP_AUTO, MAP_BLOCK, MAP_GROUP, MAP_THREAD, CAND_STATUS,
 )
 
 __all__ = [
@@ -18,5 +18,5 @@ __all__ = [
     "maaso_load_trace", "maaso_free_trace", "maaso_eval_placements", "maaso_eval_placements_multi", "maaso_eval_placements_host",
     "maaso_topk", "maaso_ins_deploy", "maaso_partition", "maaso_prune_configs", "maaso_score", "maaso_topk_scores", "maaso_ttft_percentiles", "maaso_topk_noalloc", "NOALLOC_MAX_CAND", "NOALLOC_MAX_K", "maaso_launch_count", "maaso_set_timing", "maaso_get_timing", "maaso_strerror", "maaso_last_error", "lib_path",
     "REQUEST_DTYPE", "SLO_DTYPE", "RESULT_DTYPE", "FLAG_PRED_OPTIMISTIC", "FLAG_ENGINE_FROZEN", "FLAG_TBT_MAXGAP", "FLAG_INSTANCE_QUEUES", "MAP_AUTO", "MAP_BLOCK",
-    "MAP_GROUP", "CAND_STATUS",
+    "MAP_GROUP", "MAP_THREAD", "CAND_STATUS",
 ]

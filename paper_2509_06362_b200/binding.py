@@ -27,7 +27,7 @@ FLAG_ENGINE_FROZEN = 2
 FLAG_TBT_MAXGAP = 4
 FLAG_INSTANCE_QUEUES = 8
 FLAG_TEST_STALL = 0x80000000
-MAP_AUTO, MAP_BLOCK, MAP_GROUP = 0, 1, 2
+MAP_AUTO, MAP_BLOCK, MAP_GROUP, MAP_THREAD = 0, 1, 2, 3
 CAND_STATUS = {"EBUDGET": 1, "EMEMFIT": 2, "ETOOMANY": 4, "EBADINST": 8, "ETIMEOUT": 16, "ELOOP": 32}
 
 
@@ -62,7 +62,7 @@ class _ScoreParams(C.Structure):
 
 class _Timing(C.Structure):
     _fields_ = [("prep_ms", C.c_float), ("group_ms", C.c_float), ("block_ms", C.c_float),
-                ("topk_ms", C.c_float)]
+                ("topk_ms", C.c_float), ("thread_ms", C.c_float)]
 
 
 def lib_path():
@@ -317,7 +317,8 @@ def maaso_get_timing(ctx):
     """milliseconds per kernel family of the most recent eval / topk calls (waits for them)"""
     t = _Timing()
     _check(_lib.maaso_get_timing(ctx, C.byref(t)), "maaso_get_timing", ctx)
-    return {"prep_ms": t.prep_ms, "group_ms": t.group_ms, "block_ms": t.block_ms, "topk_ms": t.topk_ms}
+    return {"prep_ms": t.prep_ms, "group_ms": t.group_ms, "block_ms": t.block_ms, "topk_ms": t.topk_ms,
+            "thread_ms": t.thread_ms}
 
 
 def maaso_launch_count(ctx):

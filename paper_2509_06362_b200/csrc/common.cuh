@@ -16,11 +16,15 @@ constexpr long long kWaitCycles = 4000000000ll;  // bound on any device-side wai
 // 0..5: lane groups of 1,2,4,8,16,32 lanes (one lane per instance)
 // 6..8: block layout with 2, 4, 8 warps, one warp per instance, state in registers
 // 9:    block layout with 16 warps striding over up to 128 instances, state in shared memory
+// With the thread mapping buckets 0..8 mean something else: how many lanes of a warp work on an
+// item (32, 24, 16, 12, 8, 6, 4, 2, 1: the larger the placements, the fewer fit the warp's pool).
 constexpr int kNumBuckets = 10;
 constexpr int kGenericBlockBucket = 9;
 constexpr int kCostBins = 256;   // bin 0 = most expensive (largest total batch cap)
 constexpr int kCounterWords = 8192;  // counters | work counters | histograms + cursors, cleared per call
 constexpr int kGroupThreads = 128;
+constexpr int kScanTile = 256;       // requests per scan tile of the thread mapping
+constexpr int kScanHdrUnits = 4;     // 16-byte units of a scan tile's header (8 int64)
 constexpr int kMaxTraces = 16;  // traces one call of the lane-group kernel can replay side by side
 
 struct Request {
@@ -229,6 +233,10 @@ struct EvalParams {
     // (and likewise for the per-model counts and the histograms).  n_traces = 1: cooked / n_req.
     uint32_t n_traces;
     const uint4* trace_cooked[kMaxTraces];
+    // thread mapping: scan tiles (header + 16-byte records, see scan_trace_kernel) and per-class totals
+    // {requests, sum of the checksum terms of "rejected"} of each trace (index 0 when there is only one)
+    const uint4* trace_scan[kMaxTraces];
+    const uint64_t* trace_class_tot[kMaxTraces];  // [n_classes][2]: count, checksum sum
     uint32_t trace_n[kMaxTraces];
     const uint64_t* rej_hash;  // [n_req] checksum term of "request r was rejected" (same for every candidate)
     const int32_t* rows;     // [n_rows][kRowStride]
@@ -253,6 +261,7 @@ struct EvalParams {
     uint32_t* sm_ctr;        // [n_sm] next work item of each SM's share (lane-group kernel)
     uint32_t n_sm;
     uint32_t promote_pct;
+    uint32_t thread_pool_units;  // thread mapping: 16-byte units of shared memory one warp has for its placements
     long long wait_cycles;   // bound of every device-side wait
     uint32_t stall_test;     // test hook: never issue the trace copies
     int32_t* dump_row;       // [n_cand] or null

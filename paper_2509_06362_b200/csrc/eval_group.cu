@@ -57,6 +57,15 @@ __device__ __forceinline__ ArgMin group_argmin(uint32_t k32, int64_t first, uint
     return r;
 }
 
+// Per-request side outputs of a rejection (dump rows, per-model counts); rare.
+__device__ __forceinline__ void reject_side(const EvalParams& P, uint32_t oc, uint32_t req, uint32_t model) {
+    const Dump dump = dump_for(P, oc);
+    if (P.rej_by_model) atomicAdd(&P.rej_by_model[(size_t)oc * MAASO_MAX_MODELS + model], 1u);
+    if (dump.finish) dump.finish[req] = -1;
+    if (dump.first) dump.first[req] = -1;
+    if (dump.inst) dump.inst[req] = -1;
+}
+
 struct GroupSmem {
     uint4* tiles;        // [kStages][tile_recs][kCookedWords] prepared request records
     unsigned char* pool; // slot keys + block minima, carved per work item in 32-byte units
@@ -309,6 +318,9 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
             for (uint32_t i = 0; i < 2u * units; i++) reinterpret_cast<uint4*>(region)[i] = e4;
         }
         const bool warp_has_work = __any_sync(kFullMask, valid);
+        // models the group's placement has an instance of
+        uint32_t gmodels = has ? (1u << in.model) : 0u;
+        for (uint32_t o = 1; o < G; o <<= 1) gmodels |= __shfl_xor_sync(kFullMask, gmodels, (int)o);
         const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
         // index of the candidate's record; the side outputs hang on it (dump rows, histogram)
         const int64_t oc = valid ? (int64_t)(out_base + cand) : -1;
@@ -356,7 +368,21 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                 if (pending) {
                     n_counted++;
                     now = max(now, q.arrival);  // pending time: the dispatcher never goes back
+                    // The plain rejections need no look at any instance: the placement has no instance
+                    // of the model, or the dispatcher's clock has already passed the request's
+                    // first-token or end-to-end deadline (every predicted first token lies at or after
+                    // `now`).  The instances are not advanced either: their clocks catch up lazily.
+                    if (!((gmodels >> q.model) & 1u) || q.dl_ttft < now || q.dl_e2e < now) {
+                        if (LOOP) attempts++;
+                        n_rejected++;
+                        if (sub == 0) {
+                            rej_sum += q.rej;
+                            if (side) reject_side(P, out_base + cand, req, q.model);
+                        }
+                        pending = false;
+                    }
                 }
+                if (!__any_sync(kFullMask, pending)) continue;  // nothing for the distributor in this warp
                 const int64_t pre = prefill_us(in.pre_base, in.pre_q16, q.in_tokens);
                 const bool elig = has && in.model == q.model;
                 uint32_t tries = 0;
@@ -378,14 +404,7 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                             n_rejected++;
                             if (sub == 0) {
                                 rej_sum += q.rej;
-                                if (side) {
-                                    const Dump dump = dump_for(P, out_base + cand);
-                                    if (P.rej_by_model)
-                                        atomicAdd(&P.rej_by_model[(size_t)(out_base + cand) * MAASO_MAX_MODELS + q.model], 1u);
-                                    if (dump.finish) dump.finish[req] = -1;
-                                    if (dump.first) dump.first[req] = -1;
-                                    if (dump.inst) dump.inst[req] = -1;
-                                }
+                                if (side) reject_side(P, out_base + cand, req, q.model);
                             }
                             pending = false;
                         } else if (am.tier == 0) {

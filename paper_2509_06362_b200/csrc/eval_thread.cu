@@ -1,0 +1,712 @@
+// Scoring kernel, thread mapping: ONE THREAD replays one candidate and walks over the instances
+// that can serve the request's model; the 32 candidates of a warp share the staged trace.
+//
+// Why: a request concerns only the instances of its model, and under load most instances are
+// full and far from their next completion, so the work per (candidate, request) is a few
+// loads and compares per capable instance.  With a lane per instance (lane-group mapping)
+// every warp instruction serves one to four candidates and most lanes idle; here it serves 32.
+//
+// Where the state lives.  All instance state is in shared memory, in 16-byte units laid out
+// unit-major: unit u of lane l sits at (u * lanes + l) * 16 bytes, so whatever unit each lane
+// touches, the eight lanes of a quarter warp hit eight different 16-byte bank groups and a
+// 128-bit access never conflicts.  A lane needs 2 units for its per-model instance ranges, 4
+// per instance (clock and next completion; level, step and prefill terms; step counter and
+// smallest key; slot mask and offsets) and, per instance, one 32-byte block per 8 virtual slots
+// for the slot keys plus one block for the block minima.  A warp takes candidates of similar
+// size (sorted by the validation kernels); how many lanes work on an item is what fits the
+// block's pool: large placements run with fewer lanes instead of not at all.
+//
+// Slot keys: `end index << 7 | generation << 6 | slot` (an empty slot keeps its generation and
+// slot bits under an all-ones end index).  The generation bit says which of the slot's two
+// scratch entries in global memory holds the data of the running request (first-token time,
+// arrival, request index, length, class, instance); entries are written at admission and come
+// back through asynchronous copies into a per-lane queue when the request completes, so no
+// load from global memory sits on the replay path.  The queue is accounted by all lanes
+// together every few requests (or by a lane alone when its queue is full).
+//
+// Clocks are lazy: an instance that nothing happens to is not written back; its clock is
+// recomputed from the last stored step boundary when it is looked at, which lands on the same
+// boundaries as long as its level (and so its step time) has not changed.
+//
+// Each thread block is one warp with its own two-stage trace pipeline (1-D bulk copies + mbarrier,
+// no multicast) and takes work items from one global counter; there is no block barrier.
+#include "lane_sim.cuh"
+
+namespace maaso {
+
+constexpr uint32_t kFullMaskT = 0xFFFFFFFFu;
+constexpr int kTStages = 2;
+constexpr int kTTile = kScanTile;               // requests per staged scan tile
+constexpr int kTStageUnits = kScanHdrUnits + kTTile + 4;  // header, records, padding for the 4-record look-ahead
+constexpr uint32_t kTEndEmpty = 0x1FFFFFFu;    // end-index field of an empty key
+constexpr uint32_t kTRelMax = (1u << 25) - 2u; // largest end index a key can hold
+constexpr int kTQueue = 4;                     // queued completions per lane
+constexpr uint32_t kTFixedBytes = kTStages * kTStageUnits * 16 + kTQueue * 32 * (16 + 8 + 8) + 64;
+
+// Lanes that work on one item, by launch bucket (bucket 9 = placements the pool cannot hold at all).
+__host__ __device__ inline uint32_t thread_lanes_of(int bucket) {
+    const uint32_t l[9] = {32, 24, 16, 12, 8, 6, 4, 2, 1};
+    return l[bucket];
+}
+
+// Pool units one placement needs: ranges + per instance 4 state units, 2 per block of 8 slots, 2 for the minima.
+__host__ __device__ inline uint32_t thread_units_of_instance(uint32_t B) { return 4u + 2u * ((B + 7u) >> 3) + 2u; }
+
+struct TPool {
+    unsigned char* base;  // pool + lane * 16
+    uint32_t stride;      // bytes from one unit of this lane to the next (= lanes * 16)
+    __device__ __forceinline__ uint4* unit(uint32_t u) const {
+        return reinterpret_cast<uint4*>(base + (size_t)u * stride);
+    }
+    __device__ __forceinline__ uint32_t* word(uint32_t u, uint32_t w) const {
+        return reinterpret_cast<uint32_t*>(base + (size_t)u * stride) + w;
+    }
+};
+
+// Working copy of one instance (units 0..2 of its state).
+struct TInst {
+    int64_t T;    // clock at the last stored step boundary
+    int64_t tc;   // time of the next completion if nobody is admitted (valid while w > 0)
+    uint32_t w, B, model, row;
+    uint32_t sw;  // one decode step at the current level (valid while w > 0)
+    uint32_t pre_base, pre_q16;
+    uint32_t K;     // decode steps done at T since the counter last restarted
+    uint32_t kmin;  // smallest slot key
+    uint32_t stepB; // step at the batch cap: the worst case F(M,P,B_I)
+    uint32_t swn;   // step at the level right after one more admission (optimistic estimate)
+};
+
+__device__ __forceinline__ void t_load(const TPool& pl, uint32_t ru, uint32_t j, TInst& in) {
+    const uint4 a = *pl.unit(ru + 4u * j), b = *pl.unit(ru + 4u * j + 1u), c = *pl.unit(ru + 4u * j + 2u);
+    in.T = (int64_t)(((uint64_t)a.y << 32) | a.x);
+    in.tc = (int64_t)(((uint64_t)a.w << 32) | a.z);
+    in.w = b.x & 0xFFu; in.B = (b.x >> 8) & 0xFFu; in.model = (b.x >> 16) & 0xFFu; in.row = b.x >> 24;
+    in.sw = b.y; in.pre_base = b.z; in.pre_q16 = b.w;
+    in.K = c.x; in.kmin = c.y; in.stepB = c.z; in.swn = c.w;
+}
+__device__ __forceinline__ void t_store(const TPool& pl, uint32_t ru, uint32_t j, const TInst& in) {
+    *pl.unit(ru + 4u * j) = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)in.tc,
+                                                 (uint32_t)((uint64_t)in.tc >> 32));
+    *pl.unit(ru + 4u * j + 1u) =
+        make_uint4(in.w | (in.B << 8) | (in.model << 16) | (in.row << 24), in.sw, in.pre_base, in.pre_q16);
+    *pl.unit(ru + 4u * j + 2u) = make_uint4(in.K, in.kmin, in.stepB, in.swn);
+}
+
+struct TStats {
+    Stats st;
+    uint32_t hbc[8];
+};
+
+// What a thread needs besides the instance at hand.
+struct TEnv {
+    TPool pl;
+    int64_t* qf;          // this lane's queue column: entry j at qf[j * 32] = finish time
+    uint4* qa;            // entry j at qa[j * 32] = first-token time, arrival time
+    uint2* qb;            // entry j at qb[j * 32] = request index, S | cls << 16 | instance << 24
+    uint4* pay_a;         // global scratch of this lane, entry 2 * slot number + generation
+    uint2* pay_b;
+    const int32_t* rows;  // latency tables (global, read through the read-only path at events only)
+    TStats* ls;
+    const EvalParams* P;
+    int64_t oc;           // index of the candidate's record, negative for a lane without one
+    uint32_t qn;          // completions waiting in the queue
+    uint32_t ru;          // units of the per-model instance ranges at the start of the lane's pool share
+};
+
+// Statistics of this lane's queued completions (Phi_S indicator, latency and throughput sums).
+static __device__ __noinline__ void t_flush(TStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb, uint32_t n,
+                                     const int64_t* classes, int64_t* dump_finish, int64_t* dump_first,
+                                     int32_t* dump_inst, uint32_t* hist) {
+    async_copies_done();
+    Stats st = ls->st;
+    const Dump no_dump{nullptr, nullptr, nullptr, nullptr};
+    const bool dumping = dump_finish || dump_first || dump_inst || hist;
+    for (uint32_t j = 0; j < n; j++) {
+        const int64_t t_fin = qf[j * 32];
+        const uint4 a = qa[j * 32];
+        const uint2 b = qb[j * 32];
+        const int64_t first = (int64_t)(((uint64_t)a.y << 32) | a.x);
+        const int64_t arrival = (int64_t)(((uint64_t)a.w << 32) | a.z);
+        const uint32_t cls = (b.y >> 16) & 0xFFu, inst = b.y >> 24;
+        const bool hit = account_completion(st, classes, inst, b.x, arrival, first, t_fin, b.y & 0xFFFFu, cls, no_dump);
+        if (hit) ls->hbc[cls < 7 ? cls : 7]++;
+        if (dumping) {
+            if (dump_finish) dump_finish[b.x] = t_fin;
+            if (dump_first) dump_first[b.x] = first;
+            if (dump_inst) dump_inst[b.x] = (int32_t)inst;
+            if (hist) atomicAdd(hist + ttft_bin(first - arrival), 1u);
+        }
+    }
+    ls->st = st;
+}
+
+__device__ __forceinline__ void t_flush_now(TEnv& e) {
+    Dump dump{nullptr, nullptr, nullptr, nullptr};
+    if (e.oc >= 0) dump = dump_for(*e.P, (uint32_t)e.oc);
+    t_flush(e.ls, e.qf, e.qa, e.qb, e.qn, e.P->classes, dump.finish, dump.first, dump.inst, dump.hist);
+    e.qn = 0;
+}
+
+// A running request has left its instance at t_fin: queue the finish time and start the copies
+// of what it remembered.  A full queue is accounted by this lane alone first.
+__device__ __forceinline__ void t_push_slot(TEnv& e, int64_t t_fin, uint32_t pidx) {
+    if (e.qn == (uint32_t)kTQueue) t_flush_now(e);
+    const uint32_t j = e.qn;
+    e.qf[j * 32] = t_fin;
+    async_copy16(e.qa + j * 32, e.pay_a + pidx);
+    async_copy8(e.qb + j * 32, e.pay_b + pidx);
+    async_commit_keep_one();
+    e.qn = j + 1;
+}
+// Same for a request of one output token, which completes at admission: everything is in registers.
+__device__ __forceinline__ void t_push_now(TEnv& e, int64_t t_fin, uint4 a, uint2 b) {
+    if (e.qn == (uint32_t)kTQueue) t_flush_now(e);
+    const uint32_t j = e.qn;
+    e.qf[j * 32] = t_fin;
+    e.qa[j * 32] = a;
+    e.qb[j * 32] = b;
+    e.qn = j + 1;
+}
+
+__device__ __forceinline__ uint32_t t_step(const TEnv& e, uint32_t row, uint32_t level) {  // level >= 1
+    return (uint32_t)__ldg(e.rows + row * kRowStride + 1u + level);
+}
+
+// Key storage of instance j: blocks of 8 keys from unit ko, then the 8 block minima.
+struct TKeys {
+    uint32_t ko;    // first key unit
+    uint32_t so;    // number of this instance's slot 0 among the lane's slots (scratch entries)
+    uint64_t mask;  // occupied slots; bits at and above B are always set
+};
+__device__ __forceinline__ TKeys t_load_keys(const TPool& pl, uint32_t ru, uint32_t j) {
+    const uint4 d = *pl.unit(ru + 4u * j + 3u);
+    TKeys k;
+    k.mask = ((uint64_t)d.y << 32) | d.x;
+    k.ko = d.z & 0xFFFFu;
+    k.so = d.z >> 16;
+    return k;
+}
+__device__ __forceinline__ void t_store_mask(const TPool& pl, uint32_t ru, uint32_t j, uint64_t mask) {
+    *reinterpret_cast<uint2*>(pl.unit(ru + 4u * j + 3u)) = make_uint2((uint32_t)mask, (uint32_t)(mask >> 32));
+}
+
+// The counter has just reached the smallest end index (clock = in.T): retire every request that
+// ends here, one per round, fix the block minima, the level and the cached next completion.
+__device__ __forceinline__ void t_retire(TInst& in, TKeys& ks, TEnv& e) {
+    const uint32_t Kc = in.K, nblk = (in.B + 7u) >> 3;
+    uint4* const bm_lo = e.pl.unit(ks.ko + 2u * nblk);
+    uint4* const bm_hi = e.pl.unit(ks.ko + 2u * nblk + 1u);
+    do {
+        const uint32_t slot = in.kmin & 63u, b = slot >> 3, sj = slot & 7u, gen = (in.kmin >> 6) & 1u;
+        const uint4 k0 = *e.pl.unit(ks.ko + 2u * b), k1 = *e.pl.unit(ks.ko + 2u * b + 1u);
+        const uint4 m0 = *bm_lo, m1 = *bm_hi;
+        const uint32_t cleared = (kTEndEmpty << 7) | (in.kmin & 127u);
+        *e.pl.word(ks.ko + 2u * b + (sj >> 2), sj & 3u) = cleared;
+        uint32_t kv[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
+#pragma unroll
+        for (int i = 0; i < 8; i++) kv[i] = (uint32_t)i == sj ? cleared : kv[i];
+        const uint32_t bmin = min8(kv);
+        *(reinterpret_cast<uint32_t*>(b < 4u ? bm_lo : bm_hi) + (b & 3u)) = bmin;
+        uint32_t mv[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+#pragma unroll
+        for (int i = 0; i < 8; i++) mv[i] = (uint32_t)i == b ? bmin : mv[i];
+        in.kmin = min8(mv);
+        ks.mask &= ~(1ull << slot);
+        in.w--;
+        t_push_slot(e, in.T, 2u * (ks.so + slot) + gen);
+    } while ((in.kmin >> 7) == Kc);
+    if (in.w > 0) {
+        in.sw = t_step(e, in.row, in.w);
+        in.tc = in.T + (int64_t)((in.kmin >> 7) - Kc) * (int64_t)in.sw;
+    }
+    in.swn = t_step(e, in.row, min(in.w + 1u, in.B));
+}
+
+// "reduce" with events: run whole decode steps until the clock reaches `now` (drain: until the
+// instance is empty), retiring what completes on the way; the instance is written back.
+__device__ __forceinline__ void t_advance_events(TInst& in, uint32_t j, int64_t now, bool drain, TEnv& e) {
+    TKeys ks = t_load_keys(e.pl, e.ru, j);
+    while (in.w > 0 && (drain || in.T < now)) {
+        if (!drain && now <= in.tc - (int64_t)in.sw) {
+            // the clock reaches `now` before anything completes (fewer steps than the longest request has tokens)
+            const uint32_t k = ceil_div_small(now - in.T, in.sw, rcp_approx((float)in.sw));
+            in.T += (int64_t)k * (int64_t)in.sw;
+            in.K += k;
+            break;
+        }
+        in.K = in.kmin >> 7;
+        in.T = in.tc;
+        t_retire(in, ks, e);
+    }
+    if (!drain && in.w == 0 && in.T < now) in.T = now;  // an idle instance starts at once
+    t_store(e.pl, e.ru, j, in);
+    t_store_mask(e.pl, e.ru, j, ks.mask);
+}
+
+// All live end indices move down by the counter value K (which restarts at 0).  Rare.
+static __device__ __noinline__ uint32_t t_rebase(unsigned char* base, uint32_t stride, uint32_t ko, uint32_t nblk, uint32_t K,
+                                         uint32_t kmin) {
+    const TPool pl{base, stride};
+    const uint32_t d = K << 7;
+    for (uint32_t u = 0; u < 2u * nblk + 2u; u++)
+        for (uint32_t w = 0; w < 4u; w++) {
+            uint32_t* p = pl.word(ko + u, w);
+            if ((*p >> 7) != kTEndEmpty) *p -= d;
+        }
+    return (kmin >> 7) != kTEndEmpty ? kmin - d : kmin;
+}
+
+// "map": prefill at the step boundary in.T (running decodes stall), then occupy a free slot.
+__device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& q, uint32_t req, int64_t pre, TEnv& e) {
+    in.T += pre;
+    const uint4 pa = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)q.arrival,
+                                (uint32_t)((uint64_t)q.arrival >> 32));
+    const uint2 pb = make_uint2(req, (q.Sm1 + 1u) | (q.cls << 16) | (j << 24));
+    if (q.Sm1 == 0) {  // done at the end of its prefill, never occupies a slot
+        in.tc += pre;
+        t_push_now(e, in.T, pa, pb);
+        t_store(e.pl, e.ru, j, in);
+        return;
+    }
+    TKeys ks = t_load_keys(e.pl, e.ru, j);
+    const uint32_t nblk = (in.B + 7u) >> 3;
+    if (in.w == 0) in.K = 0;  // no live end index: the counter restarts
+    if (in.K + q.Sm1 > kTRelMax) {
+        in.kmin = t_rebase(e.pl.base, e.pl.stride, ks.ko, nblk, in.K, in.kmin);
+        in.K = 0;
+    }
+    const uint32_t slot = (uint32_t)(__ffsll((long long)~ks.mask) - 1);
+    uint32_t* const kw = e.pl.word(ks.ko + (slot >> 2), slot & 3u);
+    const uint32_t gen = ((*kw >> 6) & 1u) ^ 1u;  // the other scratch entry than the previous occupant's
+    const uint32_t key = ((in.K + q.Sm1) << 7) | (gen << 6) | slot;
+    *kw = key;
+    const uint32_t pidx = 2u * (ks.so + slot) + gen;
+    e.pay_a[pidx] = pa;
+    e.pay_b[pidx] = pb;
+    const uint32_t b = slot >> 3;
+    uint32_t* const bm = e.pl.word(ks.ko + 2u * nblk + (b >> 2), b & 3u);
+    *bm = min(*bm, key);
+    in.kmin = min(in.kmin, key);
+    ks.mask |= 1ull << slot;
+    in.w++;
+    in.sw = t_step(e, in.row, in.w);
+    in.swn = t_step(e, in.row, min(in.w + 1u, in.B));
+    in.tc = in.T + (int64_t)((in.kmin >> 7) - in.K) * (int64_t)in.sw;
+    t_store(e.pl, e.ru, j, in);
+    t_store_mask(e.pl, e.ru, j, ks.mask);
+}
+
+// Per-request side outputs of a rejection (dump rows, per-model counts); rare.
+__device__ __forceinline__ void t_reject_side(const EvalParams& P, uint32_t oc, uint32_t req, uint32_t model) {
+    const Dump dump = dump_for(P, oc);
+    if (P.rej_by_model) atomicAdd(&P.rej_by_model[(size_t)oc * MAASO_MAX_MODELS + model], 1u);
+    if (dump.finish) dump.finish[req] = -1;
+    if (dump.first) dump.first[req] = -1;
+    if (dump.inst) dump.inst[req] = -1;
+}
+
+struct ThreadSmem {
+    unsigned char* pool;
+    uint4* tiles;       // [kTStages][kTStageUnits] scan tiles: header, records
+    uint4* qa;          // [kTQueue][32]
+    uint2* qb;
+    int64_t* qf;
+    uint64_t* full_bar; // [kTStages]
+};
+__device__ __forceinline__ ThreadSmem t_carve(unsigned char* base, uint32_t pool_bytes) {
+    ThreadSmem s;
+    s.pool = base;
+    base += pool_bytes;
+    s.tiles = reinterpret_cast<uint4*>(base);
+    base += (size_t)kTStages * kTStageUnits * 16;
+    s.qa = reinterpret_cast<uint4*>(base);
+    base += (size_t)kTQueue * 32 * 16;
+    s.qb = reinterpret_cast<uint2*>(base);
+    base += (size_t)kTQueue * 32 * 8;
+    s.qf = reinterpret_cast<int64_t*>(base);
+    base += (size_t)kTQueue * 32 * 8;
+    s.full_bar = reinterpret_cast<uint64_t*>(base);
+    return s;
+}
+
+__device__ __forceinline__ void t_issue_tile(const ThreadSmem& sm, const uint4* scan, uint32_t n_req, uint32_t stage,
+                                             uint32_t tile) {
+    const uint32_t recs = min((uint32_t)kTTile, n_req - tile * kTTile);
+    const uint32_t bytes = (recs + kScanHdrUnits) * 16u;
+    mbar_expect_tx(&sm.full_bar[stage], bytes);
+    bulk_load(sm.tiles + (size_t)stage * kTStageUnits, scan + (size_t)tile * (kScanTile + kScanHdrUnits), bytes,
+              &sm.full_bar[stage]);
+}
+
+__device__ __forceinline__ uint4 ldg_nc(const uint4* p) { return __ldg(p); }
+
+// OPT: the distributor predicts with the step time right after admission (optimistic estimate);
+// a wait is then followed by a new choice.  Under the worst-case estimate the choice after a
+// wait is known beforehand (same argument as in the lane-group kernel) and is only counted.
+//
+// How a warp walks a tile.  Most requests of a loaded placement are rejected for a reason that
+// needs no look at any instance: the placement has no instance of the model, or the
+// dispatcher's clock has already passed the request's first-token or end-to-end deadline
+// (every predicted first token lies at or after `now`).  Such a request costs its lane one
+// 16-byte scan record and a compare, and touches no instance (their clocks catch up lazily).
+// The lanes therefore run through the tile independently, each at its own request index;
+// a lane that meets a request which needs the distributor stops there, fetches the request's
+// full record, and waits.  Once `theta` lanes wait (or nobody can go on), the waiting lanes
+// handle their requests together, each its own.  Nothing is counted per request on the way:
+// a placement's request count and the checksum of "all of them rejected" come from per-class
+// totals of the trace, and an admission takes its request out again.
+template <bool OPT>
+__global__ void __launch_bounds__(32, 1)
+eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_bytes, const uint32_t theta) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const ThreadSmem sm = t_carve(smem_raw, pool_bytes);
+    const uint32_t lane = threadIdx.x;
+    if (lane == 0) {
+        for (int s = 0; s < kTStages; s++) mbar_init(&sm.full_bar[s], 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+
+    const uint32_t pool_units = pool_bytes / 16u;
+    const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
+    const uint32_t n_traces = P.n_traces > 1 ? P.n_traces : 1u;
+    const uint32_t ru = (P.n_models + 7u) >> 3;  // units of the per-model instance ranges
+    // items per bucket, buckets with the fewest lanes (the largest placements) first
+    uint32_t items[9];
+    uint32_t total_items = 0;
+    for (int b = 8; b >= 0; b--) {
+        const uint32_t L = thread_lanes_of(b);
+        items[b] = (P.bucket_count[b] + L - 1u) / L;
+        total_items += items[b];
+    }
+    const uint32_t total_all = total_items * n_traces;
+    uint32_t tile_seq = 0;  // tiles this warp has consumed so far (stage and parity of the next one)
+    bool dead = false;      // a bounded wait ran out: take no more work
+
+    TStats ls;
+    TEnv e;
+    e.qf = sm.qf + lane;
+    e.qa = sm.qa + lane;
+    e.qb = sm.qb + lane;
+    e.rows = P.rows;
+    e.ls = &ls;
+    e.P = &P;
+
+    while (!dead) {
+        uint32_t wi = 0;
+        if (lane == 0) wi = atomicAdd(&P.work_ctr[0], 1u);
+        wi = __shfl_sync(kFullMaskT, wi, 0);
+        if (wi >= total_all) break;
+        const uint32_t tr = wi % n_traces;
+        wi /= n_traces;
+        const uint4* const cooked = P.trace_cooked[tr];
+        const uint4* const scan = P.trace_scan[tr];
+        const uint32_t n_req = P.trace_n[tr];
+        const uint32_t n_tiles = (n_req + kTTile - 1) / kTTile;
+        const uint32_t out_base = tr * P.n_cand;
+        int b = 8;
+        while (wi >= items[b]) { wi -= items[b]; b--; }
+        const uint32_t L = thread_lanes_of(b);
+        const uint32_t cnt = P.bucket_count[b];
+        const uint32_t pos = wi * L + lane;
+        const bool valid = lane < L && pos < cnt;
+        const uint32_t cand = valid ? P.bucket_list[(size_t)b * P.n_cand + pos] : 0u;
+        const uint32_t cap_units = pool_units / L;  // what one lane of this item may use
+
+        e.pl.base = sm.pool + lane * 16u;
+        e.pl.stride = L * 16u;
+        e.ru = ru;
+        // scratch entries of this lane: two per slot, at most 4 slots per pool unit
+        {
+            unsigned char* const wbase = reinterpret_cast<unsigned char*>(P.payload) + (size_t)blockIdx.x * pool_units * 8u * 24u;
+            e.pay_a = reinterpret_cast<uint4*>(wbase) + (size_t)lane * cap_units * 8u;
+            e.pay_b = reinterpret_cast<uint2*>(wbase + (size_t)pool_units * 8u * 16u) + (size_t)lane * cap_units * 8u;
+        }
+        e.oc = valid ? (int64_t)(out_base + cand) : -1;
+        e.qn = 0;
+        ls.st.clear();
+        for (int i = 0; i < 8; i++) ls.hbc[i] = 0;
+
+        // ---- set up this lane's instances -----------------------------------------------------
+        uint32_t n_i = 0, status = 0;
+        uint32_t hasmodel = 0;  // models the placement has an instance of
+        if (valid) {
+            const uint32_t lo = P.offsets[cand];
+            n_i = P.offsets[cand + 1] - lo;
+            uint32_t rng_lo[MAASO_MAX_MODELS], rng_hi[MAASO_MAX_MODELS];
+            for (int m = 0; m < MAASO_MAX_MODELS; m++) { rng_lo[m] = 0xFFu; rng_hi[m] = 0u; }
+            uint32_t ko = ru + 4u * n_i, so = 0;
+            for (uint32_t j = 0; j < n_i; j++) {
+                const uint32_t word = P.inst[lo + j];
+                const uint32_t m = word & 0xFu, B = (word >> 12) & 0xFFu;
+                const uint32_t row = m * P.n_strategies + ((word >> 4) & 0xFFu);
+                const uint32_t nblk = (B + 7u) >> 3;
+                TInst in;
+                in.T = 0; in.tc = 0; in.w = 0; in.B = B; in.model = m; in.row = row; in.sw = 1;
+                in.pre_base = (uint32_t)P.rows[row * kRowStride + 0];
+                in.pre_q16 = (uint32_t)P.rows[row * kRowStride + 1];
+                in.K = 0; in.kmin = 0xFFFFFFFFu;
+                in.stepB = (uint32_t)P.rows[row * kRowStride + 1 + B];
+                in.swn = (uint32_t)P.rows[row * kRowStride + 2];
+                if (ko + 2u * nblk + 2u > cap_units) { status = MAASO_CAND_ETIMEOUT; break; }  // cannot happen: sized by the validation kernel
+                t_store(e.pl, ru, j, in);
+                const uint64_t mask = B >= 64u ? 0ull : (~0ull << B);
+                *e.pl.unit(ru + 4u * j + 3u) = make_uint4((uint32_t)mask, (uint32_t)(mask >> 32), ko | (so << 16), 0u);
+                for (uint32_t u = 0; u < 2u * nblk; u++) {
+                    const uint32_t s0 = (kTEndEmpty << 7) | (4u * u);
+                    *e.pl.unit(ko + u) = make_uint4(s0, s0 + 1u, s0 + 2u, s0 + 3u);
+                }
+                const uint4 ones = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+                *e.pl.unit(ko + 2u * nblk) = ones;
+                *e.pl.unit(ko + 2u * nblk + 1u) = ones;
+                ko += 2u * nblk + 2u;
+                so += 8u * nblk;
+                rng_lo[m] = min(rng_lo[m], j);
+                rng_hi[m] = j + 1u;
+                hasmodel |= 1u << m;
+            }
+            // per-model instance ranges: halfword m = first index | (last index + 1) << 8
+            for (uint32_t u = 0; u < ru; u++) {
+                uint32_t rw[4];
+                for (int i = 0; i < 4; i++) {
+                    const uint32_t m0 = 8u * u + 2u * i, m1 = m0 + 1u;
+                    const uint32_t a = rng_lo[m0] >= rng_hi[m0] ? 0u : (rng_lo[m0] | (rng_hi[m0] << 8));
+                    const uint32_t c = rng_lo[m1] >= rng_hi[m1] ? 0u : (rng_lo[m1] | (rng_hi[m1] << 8));
+                    rw[i] = a | (c << 16);
+                }
+                *e.pl.unit(u) = make_uint4(rw[0], rw[1], rw[2], rw[3]);
+            }
+        }
+        const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
+        // header entries of a scan tile this lane has to look at (classes 7 and up share entry 7)
+        const uint32_t hmask = (cmask & 0x7Fu) | ((cmask >> 7) ? 0x80u : 0u);
+        bool side = P.rej_by_model != nullptr;
+        if (valid && P.dump_row) side = side || P.dump_row[cand] >= 0;
+        // every request of the subset counted as rejected; admissions take theirs out
+        uint32_t n_counted = 0;
+        uint64_t rej_sum = 0;
+        if (valid) {
+            const uint64_t* ct = P.trace_class_tot[tr];
+            for (uint32_t c = 0; c < P.n_classes; c++)
+                if (!use_mask || ((cmask >> c) & 1u)) {
+                    n_counted += (uint32_t)ct[2u * c];
+                    rej_sum += ct[2u * c + 1u];
+                }
+        }
+        int64_t now = 0;
+        uint64_t extra = 0;  // distributor rounds beyond the first of a request
+        __syncwarp();
+
+        // ---- trace staging: first tiles of this item --------------------------------------------
+        if (lane == 0 && !P.stall_test) {
+            for (uint32_t s = 0; s < (uint32_t)kTStages && s < n_tiles; s++)
+                t_issue_tile(sm, scan, n_req, (tile_seq + s) % kTStages, s);
+        }
+        uint32_t in_flight = min((uint32_t)kTStages, n_tiles);
+
+        for (uint32_t t = 0; t < n_tiles; t++) {
+            const uint32_t s = tile_seq % kTStages, parity = (tile_seq / kTStages) & 1u;
+            const bool arrived = mbar_wait_bounded(&sm.full_bar[s], parity, P.wait_cycles);
+            if (!__all_sync(kFullMaskT, arrived)) {
+                // give up: wait (bounded) for every copy still in flight, then stop taking work
+                if (!P.stall_test)
+                    for (uint32_t x = 0; x < in_flight; x++) {
+                        const uint32_t ts = tile_seq + x;
+                        mbar_wait_bounded(&sm.full_bar[ts % kTStages], (ts / kTStages) & 1u, P.wait_cycles);
+                    }
+                status = MAASO_CAND_ETIMEOUT;
+                dead = true;
+                break;
+            }
+            in_flight--;
+            const uint4* const tile = sm.tiles + (size_t)s * kTStageUnits;
+            const uint4* const rp = tile + kScanHdrUnits;  // the tile's scan records
+            const uint32_t recs = min((uint32_t)kTTile, n_req - t * kTTile);
+            uint32_t ri = (valid && status == 0) ? 0u : recs;
+            // the whole tile is late for this lane if its clock has passed the header entry of every class it counts
+            if (ri < recs && !side) {
+                bool all_late = true;
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const uint4 h = tile[k];
+                    const int64_t a = (int64_t)(((uint64_t)h.y << 32) | h.x), c = (int64_t)(((uint64_t)h.w << 32) | h.z);
+                    if (((hmask >> (2 * k)) & 1u) && a >= now) all_late = false;
+                    if (((hmask >> (2 * k + 1)) & 1u) && c >= now) all_late = false;
+                }
+                if (all_late) ri = recs;
+            }
+            bool waiting = false;  // this lane stands at a request that needs the distributor
+            uint4 f0, f1, f2;      // that request's full record
+            f0 = f1 = f2 = make_uint4(0u, 0u, 0u, 0u);
+            for (;;) {
+                uint32_t wl;
+                for (;;) {
+#pragma unroll 1
+                    for (int c = 0; c < 2; c++) {
+                        if (waiting || ri >= recs) continue;
+                        // four records at a time: the first one that needs the distributor stops the lane
+                        uint4 r[4];
+#pragma unroll
+                        for (int k = 0; k < 4; k++) r[k] = rp[ri + k];
+                        uint32_t first = 4;
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            if (first != 4u || ri + k >= recs) continue;
+                            if (!((cmask >> ((r[k].w >> 8) & 31u)) & 1u)) continue;  // not in the request subset
+                            const int64_t arrival = (int64_t)(((uint64_t)r[k].y << 32) | r[k].x);
+                            now = max(now, arrival);  // pending time: the dispatcher never goes back
+                            const bool late = r[k].z != 0xFFFFFFFFu && arrival + (int64_t)r[k].z < now;
+                            if (((hasmodel >> (r[k].w & 0xFFu)) & 1u) && !late) first = k;
+                            // else overflow protection, the plain case: nobody can meet the deadline -> rejected
+                            else if (side) t_reject_side(P, out_base + cand, t * kTTile + ri + k, r[k].w & 0xFFu);
+                        }
+                        if (first != 4u) {
+                            ri += first;
+                            waiting = true;
+                            const uint4* full = cooked + (size_t)(t * kTTile + ri) * kCookedWords;
+                            f0 = ldg_nc(full); f1 = ldg_nc(full + 1); f2 = ldg_nc(full + 2);
+                        } else {
+                            ri = min(ri + 4u, recs);
+                        }
+                    }
+                    wl = __ballot_sync(kFullMaskT, waiting);
+                    const uint32_t act = __ballot_sync(kFullMaskT, !waiting && ri < recs);
+                    if (act == 0u || (uint32_t)__popc(wl) >= theta) break;
+                }
+                if (wl == 0u) break;  // everybody is through the tile
+                // statistics of completed requests, all lanes together
+                if (__any_sync(kFullMaskT, e.qn >= 3u)) t_flush_now(e);
+                if (!waiting) continue;
+                waiting = false;
+                const CookedReq q = decode_cooked(f0, f1, f2);
+                const uint32_t req = t * kTTile + ri;
+                ri++;
+                // instances of the request's model
+                const uint4 rg = *e.pl.unit(q.model >> 3);
+                const uint32_t rgw = (q.model & 4u) ? ((q.model & 2u) ? rg.w : rg.z) : ((q.model & 2u) ? rg.y : rg.x);
+                const uint32_t rh = (q.model & 1u) ? (rgw >> 16) : (rgw & 0xFFFFu);
+                const uint32_t j_lo = rh & 0xFFu, j_hi = rh >> 8;
+                bool pending = true;
+                uint32_t tries = 0;
+                do {
+                    tries++;
+                    uint64_t best = kKeyInf;
+                    uint32_t bj = 0, bk = 0;
+                    int64_t bT = 0, bpre = 0;
+                    for (uint32_t j = j_lo; j < j_hi; j++) {
+                        TInst in;
+                        t_load(e.pl, ru, j, in);
+                        if (in.model != q.model) continue;
+                        // "reduce": where the instance's clock stands once it has reached `now`
+                        int64_t T = in.T;
+                        uint32_t kadd = 0;
+                        if (in.w > 0) {
+                            if (T < now) {
+                                if (now > in.tc - (int64_t)in.sw) {  // something completes on the way
+                                    t_advance_events(in, j, now, false, e);
+                                    T = in.T;
+                                } else if (in.w < in.B) {
+                                    kadd = ceil_div_small(now - T, in.sw, rcp_approx((float)in.sw));
+                                    T += (int64_t)kadd * (int64_t)in.sw;
+                                }
+                            }
+                        } else if (T < now) {
+                            T = now;
+                        }
+                        // distributor prediction (Sec. IV-F steps 2-3)
+                        const int64_t pre = prefill_us(in.pre_base, in.pre_q16, q.in_tokens);
+                        const bool free_slot = in.w < in.B;
+                        const int64_t t0 = free_slot ? T : in.tc;
+                        const uint32_t sB = (OPT && free_slot) ? in.swn : in.stepB;
+                        const int64_t first = t0 + pre;
+                        const int64_t fin = first + (int64_t)((uint64_t)q.Sm1 * sB);
+                        const bool ok = first <= q.dl_ttft && (q.Sm1 == 0 || sB <= q.tbt32) && fin <= q.dl_e2e;
+                        const uint64_t key = ((uint64_t)(free_slot ? 0u : 1u) << 63) | (uint64_t)first;
+                        if (ok && key < best) { best = key; bj = j; bk = kadd; bT = T; bpre = pre; }
+                    }
+                    if (best == kKeyInf) {
+                        // overflow protection: nobody can meet the deadline -> rejected
+                        if (side) t_reject_side(P, out_base + cand, req, q.model);
+                        pending = false;
+                    } else {
+                        TInst in;
+                        t_load(e.pl, ru, bj, in);
+                        if ((best >> 63) == 0) {
+                            in.T = bT;  // the clock as the prediction saw it
+                            in.K += bk;
+                            t_admit(in, bj, q, req, bpre, e);
+                            rej_sum -= q.rej;
+                            pending = false;
+                        } else {
+                            // every capable instance is full: wait until the chosen slot frees
+                            now = in.tc;
+                            if (!OPT) {
+                                tries++;  // the second round, counted only
+                                t_advance_events(in, bj, now, false, e);
+                                t_admit(in, bj, q, req, bpre, e);
+                                rej_sum -= q.rej;
+                                pending = false;
+                            } else if (tries >= kAttemptCap) {
+                                status = MAASO_CAND_ELOOP;
+                                pending = false;
+                            }
+                        }
+                    }
+                } while (OPT && pending);
+                extra += tries - 1u;
+                if (status) ri = recs;  // given up on this candidate
+            }
+            // this warp is done with the stage: refill it
+            __syncwarp();
+            if (lane == 0 && t + kTStages < n_tiles) {
+                fence_proxy_async();
+                t_issue_tile(sm, scan, n_req, s, t + kTStages);
+            }
+            if (t + kTStages < n_tiles) in_flight++;
+            tile_seq++;
+        }
+
+        // ---- drain, account what is still queued, write the record ------------------------------
+        __syncwarp();
+        if (valid && status == 0) {
+            for (uint32_t j = 0; j < n_i; j++) {
+                TInst in;
+                t_load(e.pl, ru, j, in);
+                if (in.w > 0) t_advance_events(in, j, 0, true, e);
+            }
+        }
+        t_flush_now(e);
+        if (valid) {
+            Stats st = ls.st;
+            st.checksum += rej_sum;
+            write_result(P.out + out_base + cand, status, n_counted, n_counted - st.served, (uint64_t)n_counted + extra, st,
+                         ls.hbc);
+        }
+        __syncwarp();
+    }
+}
+
+cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t theta, cudaStream_t stream) {
+    auto kernel = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_thread_kernel<true> : eval_thread_kernel<false>;
+    const size_t smem = (size_t)pool_bytes + kTFixedBytes;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, 32, smem, stream>>>(P, pool_bytes, theta);
+    return cudaGetLastError();
+}
+
+int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes) {
+    auto kernel = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_thread_kernel<true> : eval_thread_kernel<false>;
+    const size_t smem = (size_t)pool_bytes + kTFixedBytes;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, 32, smem) != cudaSuccess) return 1;
+    return n < 1 ? 1 : n;
+}
+
+uint32_t thread_fixed_smem() { return kTFixedBytes; }
+
+// Global scratch one warp of the thread mapping needs: two entries of 24 bytes per slot, 4 slots per pool unit.
+size_t thread_scratch_per_warp(uint32_t pool_bytes) { return (size_t)(pool_bytes / 16u) * 8u * 24u; }
+
+}  // namespace maaso

@@ -232,13 +232,13 @@ __device__ __forceinline__ void flush_queue_body(LaneStats* ls, const int64_t* q
 
 // Out of line on purpose: the sums stay in local memory and the replay loop stays small.  One
 // copy per form of the TBT term, so that the usual one carries nothing of the other.
-__device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
+static __device__ __noinline__ void flush_queue(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
                                          const unsigned char* ovf, uint32_t n, const int64_t* classes,
                                          uint32_t inst_idx, int64_t* dump_finish, int64_t* dump_first,
                                          int32_t* dump_inst, uint32_t* hist) {
     flush_queue_body<false>(ls, qf, qa, qb, ovf, n, classes, inst_idx, dump_finish, dump_first, dump_inst, hist);
 }
-__device__ __noinline__ void flush_queue_maxgap(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
+static __device__ __noinline__ void flush_queue_maxgap(LaneStats* ls, const int64_t* qf, const uint4* qa, const uint2* qb,
                                                 const unsigned char* ovf, uint32_t n, const int64_t* classes,
                                                 uint32_t inst_idx, int64_t* dump_finish, int64_t* dump_first,
                                                 int32_t* dump_inst, uint32_t* hist) {
@@ -269,7 +269,7 @@ __device__ __forceinline__ uint64_t gap_of(const uint4& e) { return ((uint64_t)e
 
 // The list is full of strictly decreasing gaps: fold its oldest entry into the slots it concerns
 // (exactly what the look-up would have found there) and drop it.  Rare, kept out of line.
-__device__ __noinline__ void gaps_drop_oldest(uint64_t* mg, uint64_t* dl, uint32_t* first, uint4* stk, uint32_t nslots) {
+static __device__ __noinline__ void gaps_drop_oldest(uint64_t* mg, uint64_t* dl, uint32_t* first, uint4* stk, uint32_t nslots) {
     const uint4 e = stk[0];
     const uint64_t v = gap_of(e);
     for (uint32_t i = 0; i < nslots; i++) {
@@ -431,7 +431,7 @@ __device__ __forceinline__ uint32_t lane_predict(const LaneInst& in, const Cooke
 
 // All live end indices move down by the current counter value `K` (the caller restarts the
 // counter at 0).  Returns the rebased smallest key.  Rare: kept out of line, arguments by value.
-__device__ __noinline__ uint32_t lane_rebase(uint32_t* keys, uint32_t nslots, uint4* bm_lo, uint4* bm_hi,
+static __device__ __noinline__ uint32_t lane_rebase(uint32_t* keys, uint32_t nslots, uint4* bm_lo, uint4* bm_hi,
                                              uint32_t K, uint32_t kmin) {
     const uint32_t d = K << 6;
     for (uint32_t s = 0; s < nslots; s++) {

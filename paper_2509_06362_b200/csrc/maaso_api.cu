@@ -13,10 +13,16 @@ namespace maaso {
 cudaError_t launch_prep(const EvalParams& P, const uint32_t* dump_idx, cudaStream_t stream, int* launches);
 cudaError_t launch_rej_hash(uint64_t* out, uint32_t n);
 cudaError_t launch_cook_trace(const uint4* reqs, const int64_t* classes, uint4* out, uint32_t n);
+cudaError_t launch_scan_trace(const uint4* reqs, const int64_t* classes, uint4* scan, uint32_t n);
+size_t scan_trace_units(uint32_t n);
 cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, int blocks_per_sm, int smem_per_sm,
                               cudaStream_t stream);
 int occupancy_eval_group(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm);
 size_t group_scratch_per_lane();
+cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t theta, cudaStream_t stream);
+int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes);
+size_t thread_scratch_per_warp(uint32_t pool_bytes);
+uint32_t thread_fixed_smem();
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 cudaError_t launch_eval_block_reg(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 int occupancy_eval_block_reg(const EvalParams& P, int bucket, int tile_recs);
@@ -40,6 +46,8 @@ struct maaso_trace {
     int64_t* d_classes;
     uint64_t* d_rej_hash;
     uint4* d_cooked;  // prepared records for the lane-group kernel
+    uint4* d_scan;    // scan records for the thread mapping
+    uint64_t* d_class_tot;  // per class: number of requests, sum of their "rejected" checksum terms
     std::vector<int64_t> h_classes;  // host copy of the class table (several traces in one call must agree on it)
     uint64_t n;
     uint32_t n_classes;
@@ -73,6 +81,10 @@ struct maaso_ctx {
     int group_blocks;  // blocks of the lane-group kernel per SM its key pool is sized for; 0 = by batch size
     int smem_per_sm;
     int promote_pct;  // share of the spare resident warps the planner may use for promotions
+    int thread_blocks;   // one-warp blocks of the thread-mapping kernel per SM its pool is sized for
+    uint32_t thread_theta;     // waiting lanes of a warp that trigger a distributor round in the thread mapping
+    uint32_t thread_min_cand;  // MAASO_MAP_AUTO takes the thread mapping from this many candidates on
+    uint32_t last_mapping;     // mapping the most recent scoring call resolved to
     bool timing;
     cudaEvent_t ev[6];   // eval: start, after prep, after group, after block; topk: start, end
     bool ev_eval, ev_topk;
@@ -119,6 +131,16 @@ int grow(maaso_ctx* ctx, void** buf, size_t* have, size_t need) {
 }
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Checksum term of "request r was rejected": the SplitMix64 output mixer (public domain) of
+// r * 0x9E3779B97F4A7C15 ^ all-ones, as the kernels compute it.
+uint64_t host_rejected_hash(uint32_t r) {
+    uint64_t z = (uint64_t)r * 0x9E3779B97F4A7C15ull ^ ~0ull;
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+    z ^= z >> 27; z *= 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    return z;
+}
 
 }  // namespace
 
@@ -175,6 +197,25 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
         if (v >= 16 && v <= 2048) ctx->tile_recs = v & ~1;  // even: tiles of 8-byte terms stay 16-byte aligned
     }
 
+    ctx->thread_blocks = 6;
+    const char* tb = getenv("MAASO_THREAD_BLOCKS");
+    if (tb) {
+        int v = atoi(tb);
+        if (v >= 1 && v <= 16) ctx->thread_blocks = v;
+    }
+    ctx->thread_theta = 12;
+    const char* tt = getenv("MAASO_THREAD_THETA");
+    if (tt) {
+        int v = atoi(tt);
+        if (v >= 1 && v <= 32) ctx->thread_theta = (uint32_t)v;
+    }
+    ctx->thread_min_cand = 0xFFFFFFFFu;  // the lane groups unless asked otherwise
+    const char* tm = getenv("MAASO_THREAD_MIN_CAND");
+    if (tm) {
+        long v = atol(tm);
+        if (v >= 0) ctx->thread_min_cand = (uint32_t)v;
+    }
+    ctx->last_mapping = MAASO_MAP_GROUP;
     const char* gb = getenv("MAASO_GROUP_BLOCKS");
     if (gb) {
         int v = atoi(gb);
@@ -197,6 +238,8 @@ MAASO_API void maaso_free_trace(maaso_ctx* ctx, maaso_trace* trace) {
     if (trace->d_classes) cudaFree(trace->d_classes);
     if (trace->d_rej_hash) cudaFree(trace->d_rej_hash);
     if (trace->d_cooked) cudaFree(trace->d_cooked);
+    if (trace->d_scan) cudaFree(trace->d_scan);
+    if (trace->d_class_tot) cudaFree(trace->d_class_tot);
     delete trace;
 }
 
@@ -304,6 +347,9 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     int64_t prev = 0;
     uint32_t max_model = 0;
     const int64_t kArrMax = (int64_t)1 << 50;
+    // per class: how many requests, and the sum of their checksum terms as rejected requests (the thread
+    // mapping starts from "everything counted was rejected" and takes the served ones out)
+    std::vector<uint64_t> class_tot((size_t)n_classes * 2, 0);
     for (uint64_t r = 0; r < n; r++) {
         const maaso_request& q = host[r];
         if (q.arrival_us < prev || q.arrival_us > kArrMax)
@@ -313,6 +359,8 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
         if (q.cls >= n_classes) return fail(ctx, MAASO_EINVAL, "trace: unknown SLO class");
         if (q.model >= ctx->n_models) return fail(ctx, MAASO_EINVAL, "trace: unknown model");
         if (q.model > max_model) max_model = q.model;
+        class_tot[(size_t)q.cls * 2] += 1;
+        class_tot[(size_t)q.cls * 2 + 1] += host_rejected_hash((uint32_t)r);
     }
     maaso_trace* t = new (std::nothrow) maaso_trace();
     if (!t) return MAASO_ENOMEM;
@@ -321,6 +369,8 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     t->d_classes = nullptr;
     t->d_rej_hash = nullptr;
     t->d_cooked = nullptr;
+    t->d_scan = nullptr;
+    t->d_class_tot = nullptr;
     t->n = n;
     t->n_classes = n_classes;
     t->max_model = max_model;
@@ -329,6 +379,9 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     if (e == cudaSuccess) e = cudaMalloc(&t->d_classes, cls.size() * 8);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_rej_hash, (n ? n : 1) * 8);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_cooked, (n ? n : 1) * 16 * kCookedWords);
+    if (e == cudaSuccess) e = cudaMalloc(&t->d_scan, scan_trace_units((uint32_t)n) * 16);
+    if (e == cudaSuccess) e = cudaMalloc(&t->d_class_tot, (size_t)n_classes * 16);
+    if (e == cudaSuccess) e = cudaMemcpy(t->d_class_tot, class_tot.data(), (size_t)n_classes * 16, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = launch_rej_hash(t->d_rej_hash, (uint32_t)n);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e == cudaSuccess && n)
@@ -336,9 +389,12 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
                        on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(t->d_classes, cls.data(), cls.size() * 8, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = launch_cook_trace(t->d_reqs, t->d_classes, t->d_cooked, (uint32_t)n);
+    if (e == cudaSuccess) e = launch_scan_trace(t->d_reqs, t->d_classes, t->d_scan, (uint32_t)n);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         if (t->d_cooked) cudaFree(t->d_cooked);
+        if (t->d_scan) cudaFree(t->d_scan);
+        if (t->d_class_tot) cudaFree(t->d_class_tot);
         if (t->d_reqs) cudaFree(t->d_reqs);
         if (t->d_classes) cudaFree(t->d_classes);
         if (t->d_rej_hash) cudaFree(t->d_rej_hash);
@@ -377,7 +433,7 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     maaso_eval_opts o;
     memset(&o, 0, sizeof(o));
     if (opts) o = *opts;
-    if (o.mapping > MAASO_MAP_GROUP) return fail(ctx, MAASO_EINVAL, "eval: unknown mapping");
+    if (o.mapping > MAASO_MAP_THREAD) return fail(ctx, MAASO_EINVAL, "eval: unknown mapping");
     if (o.dump_n && !o.dump_cand_idx) return fail(ctx, MAASO_EINVAL, "eval: dump_n without dump_cand_idx");
     if (n_traces > 1 && (o.dump_n || o.mapping == MAASO_MAP_BLOCK))
         return fail(ctx, MAASO_EINVAL, "eval: several traces in one call allow no dump buffers and no block mapping");
@@ -388,6 +444,13 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
         o.mapping == MAASO_MAP_BLOCK)
         return fail(ctx, MAASO_EINVAL,
                     "eval: the fixed-speed engine, per-instance queues and the largest-gap test have no block mapping");
+    const bool variant = (o.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES)) != 0;
+    if (variant && o.mapping == MAASO_MAP_THREAD)
+        return fail(ctx, MAASO_EINVAL,
+                    "eval: the fixed-speed engine, per-instance queues and the largest-gap test have no thread mapping");
+    if (o.mapping == MAASO_MAP_AUTO)
+        o.mapping = (!variant && cands->n_cand >= ctx->thread_min_cand) ? MAASO_MAP_THREAD : MAASO_MAP_GROUP;
+    ctx->last_mapping = o.mapping;
 
     DeviceGuard g(ctx->device);
     cudaStream_t stream = (cudaStream_t)cuda_stream;
@@ -405,6 +468,8 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     P.n_traces = n_traces;
     for (uint32_t t = 0; t < n_traces; t++) {
         P.trace_cooked[t] = traces[t]->d_cooked;
+        P.trace_scan[t] = traces[t]->d_scan;
+        P.trace_class_tot[t] = traces[t]->d_class_tot;
         P.trace_n[t] = (uint32_t)traces[t]->n;
     }
     P.rows = ctx->d_rows;
@@ -436,23 +501,50 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     // wave is bound by its longest dependent chains, which run faster with fewer warps sharing a
     // scheduler; a larger batch is bound by instruction issue and wants all four.  Lanes needed
     // ~ instances x 1.3 (group widths are powers of two).
+    const bool threads = o.mapping == MAASO_MAP_THREAD;
     int group_blocks = ctx->group_blocks;
     if (group_blocks == 0) {
         const uint64_t est_warps = ((cands->n_inst * 13 / 10 + 31) / 32 + 6) * n_traces;
         group_blocks = est_warps <= (uint64_t)ctx->sm_count * 3 * (kGroupThreads / 32) ? 3 : 4;
     }
-    const int occ_g = occupancy_eval_group(P, tile, group_blocks, ctx->smem_per_sm);
-    int grid_g = ctx->sm_count * occ_g;
-    // at most one work item per 4 candidates + bucket tails, once per trace
-    const uint64_t max_items_g = ((uint64_t)C / 4 + 6) * n_traces;
-    if ((uint64_t)grid_g > max_items_g) grid_g = (int)max_items_g;
-    int grid_b[4];
-    size_t pay_entries = (size_t)grid_g * kGroupThreads * (group_scratch_per_lane() / sizeof(Payload));
+    int grid_g = 0, grid_t = 0;
+    uint32_t thread_pool = 0;
+    size_t pay_entries = 0;
     static_assert(sizeof(Payload) == 32, "scratch is counted in 32-byte entries");
+    if (threads) {
+        // thread mapping: one-warp blocks; the pool is what is left of an SM's shared memory when
+        // `thread_blocks` of them share it (1 KB per block is reserved by the system)
+        size_t per_block = (size_t)ctx->smem_per_sm / (size_t)ctx->thread_blocks;
+        per_block = per_block > 1024 ? per_block - 1024 : 0;
+        if (per_block > 227u * 1024u) per_block = 227u * 1024u;
+        const size_t fixed = thread_fixed_smem();
+        size_t pool = per_block > fixed ? per_block - fixed : 0;
+        pool -= pool % 512;
+        if (pool > 65535u * 16u) pool = 65535u * 16u - (65535u * 16u) % 512;  // unit offsets are 16-bit
+        if (pool < 4096) return fail(ctx, MAASO_ESTATE, "eval: no shared memory for the thread mapping");
+        thread_pool = (uint32_t)pool;
+        P.thread_pool_units = thread_pool / 16u;
+        grid_t = ctx->sm_count * occupancy_eval_thread(P, thread_pool);
+        const uint64_t max_items_t = ((uint64_t)C + 9) * n_traces;
+        if ((uint64_t)grid_t > max_items_t) grid_t = (int)max_items_t;
+        pay_entries = ((size_t)grid_t * thread_scratch_per_warp(thread_pool) + sizeof(Payload) - 1) / sizeof(Payload);
+    } else if (o.mapping != MAASO_MAP_BLOCK) {
+        const int occ_g = occupancy_eval_group(P, tile, group_blocks, ctx->smem_per_sm);
+        grid_g = ctx->sm_count * occ_g;
+        // at most one work item per 4 candidates + bucket tails, once per trace
+        const uint64_t max_items_g = ((uint64_t)C / 4 + 6) * n_traces;
+        if ((uint64_t)grid_g > max_items_g) grid_g = (int)max_items_g;
+        pay_entries = (size_t)grid_g * kGroupThreads * (group_scratch_per_lane() / sizeof(Payload));
+    }
+    int grid_b[4];
     for (int b = 6; b <= kGenericBlockBucket; b++) {
-        // without the block mapping only candidates with more than 32 instances go to a block kernel
-        const bool used = n_traces == 1 &&
-                          (o.mapping == MAASO_MAP_BLOCK || (b == kGenericBlockBucket && cands->n_inst > 32));
+        // without the block mapping only candidates the other kernel cannot take go to a block kernel:
+        // more than 32 instances (lane groups), or a state larger than a warp's pool (thread mapping)
+        bool used = n_traces == 1 && o.mapping == MAASO_MAP_BLOCK;
+        if (n_traces == 1 && b == kGenericBlockBucket) {
+            if (o.mapping == MAASO_MAP_GROUP) used = cands->n_inst > 32;
+            if (threads) used = cands->n_inst * 22ull + 2ull > P.thread_pool_units;  // 22 units: an instance with 64 slots
+        }
         grid_b[b - 6] = 0;
         if (!used) continue;
         // placements with at most 8 instances: one warp per instance with register-resident state
@@ -486,6 +578,7 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
 
     static_assert(64 + 2 * kNumBuckets * kCostBins + 1024 <= kCounterWords, "counter region");
     P.group_warps = (uint32_t)grid_g * (kGroupThreads / 32);
+    P.mapping = o.mapping;  // resolved: block, lane groups or threads
     P.promote_pct = (uint32_t)ctx->promote_pct;
     cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, kCounterWords * 4, stream);
     if (e == cudaSuccess && o.ttft_hist)
@@ -496,7 +589,11 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     e = launch_prep(P, o.dump_cand_idx, stream, &launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "prep launch");
     if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
-    if (o.mapping != MAASO_MAP_BLOCK) {
+    if (threads) {
+        e = launch_eval_thread(P, grid_t, thread_pool, ctx->thread_theta, stream);
+        launches++;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "thread kernel launch");
+    } else if (o.mapping != MAASO_MAP_BLOCK) {
         e = launch_eval_group(P, grid_g, tile, group_blocks, ctx->smem_per_sm, stream);
         launches++;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "group kernel launch");
@@ -1101,7 +1198,9 @@ MAASO_API int maaso_get_timing(maaso_ctx* ctx, maaso_timing* out) {
     if (ctx->ev_eval) {
         e = cudaEventSynchronize(ctx->ev[3]);
         if (e == cudaSuccess) e = cudaEventElapsedTime(&out->prep_ms, ctx->ev[0], ctx->ev[1]);
-        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->group_ms, ctx->ev[1], ctx->ev[2]);
+        if (e == cudaSuccess)
+            e = cudaEventElapsedTime(ctx->last_mapping == MAASO_MAP_THREAD ? &out->thread_ms : &out->group_ms,
+                                     ctx->ev[1], ctx->ev[2]);
         if (e == cudaSuccess) e = cudaEventElapsedTime(&out->block_ms, ctx->ev[2], ctx->ev[3]);
     }
     if (e == cudaSuccess && ctx->ev_topk) {

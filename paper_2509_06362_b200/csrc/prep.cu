@@ -9,11 +9,14 @@ __global__ void prep_kernel(const EvalParams P) {
     if (c >= P.n_cand) return;
     const uint32_t lo = P.offsets[c], hi = P.offsets[c + 1];
     uint32_t status = 0, n = 0, sum_b = 0;
+    uint32_t units = (P.n_models + 7u) >> 3;  // thread mapping: 16-byte units of state (model ranges, per instance 4 + key blocks + minima)
     if (hi < lo || hi > P.n_inst) {
         status = MAASO_CAND_EBADINST;  // malformed CSR row
     } else {
         n = hi - lo;
-        if (n > MAASO_MAX_INSTANCES || (((P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES)) || P.n_traces > 1) && n > 32)) {
+        const bool group_only = P.mapping != MAASO_MAP_THREAD &&
+                                ((P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES)) || P.n_traces > 1);
+        if (n > MAASO_MAX_INSTANCES || (group_only && n > 32)) {
             status = MAASO_CAND_ETOOMANY;  // these options exist in the lane-group kernel only
         } else {
             uint64_t devsum = 0;
@@ -25,10 +28,13 @@ __global__ void prep_kernel(const EvalParams P) {
                     continue;
                 }
                 sum_b += b;
+                units += 4u + 2u * ((b + 7u) >> 3) + 2u;
                 devsum += (uint64_t)P.devices[s];
                 if (P.devices[s] < P.min_devices[m]) status |= MAASO_CAND_EMEMFIT;
             }
             if (devsum > P.budget) status |= MAASO_CAND_EBUDGET;
+            // several traces in one pass exist in the lane-group and thread kernels only
+            if (P.mapping == MAASO_MAP_THREAD && P.n_traces > 1 && units > P.thread_pool_units) status |= MAASO_CAND_ETOOMANY;
         }
     }
     if (P.dump_row) P.dump_row[c] = -1;
@@ -50,6 +56,14 @@ __global__ void prep_kernel(const EvalParams P) {
     }
     int b;
     if (P.mapping == MAASO_MAP_BLOCK) b = n <= 2 ? 6 : (n <= 4 ? 7 : (n <= 8 ? 8 : kGenericBlockBucket));
+    else if (P.mapping == MAASO_MAP_THREAD) {
+        // as many lanes per item as placements of this size fit the warp's pool
+        const uint32_t fit = units ? P.thread_pool_units / units : 32u;
+        const uint32_t lanes[9] = {32, 24, 16, 12, 8, 6, 4, 2, 1};
+        b = kGenericBlockBucket;  // not even one: the block layout takes it
+        for (int i = 0; i < 9; i++)
+            if (fit >= lanes[i]) { b = i; break; }
+    }
     else if (n <= 32) b = n <= 1 ? 0 : 32 - __clz((int)(n - 1));
     else b = kGenericBlockBucket;
     // Cost estimate: the total batch cap (how many requests the placement can have in flight;
@@ -85,7 +99,7 @@ __global__ void __launch_bounds__(kCostBins) plan_kernel(const EvalParams P) {
     uint32_t cut = 0;  // bins below `cut` are promoted
     uint32_t narrow = 0;
     for (int b = 0; b < 5; b++) narrow += P.hist[b * kCostBins + bin];
-    if (P.mapping != MAASO_MAP_BLOCK) {
+    if (P.mapping == MAASO_MAP_GROUP) {
         uint32_t need = 0;
         for (int b = 0; b <= 5; b++) need += (P.bucket_count[b] + (32u >> b) - 1) / (32u >> b);
         const uint32_t spare = P.group_warps > need ? (uint32_t)((uint64_t)(P.group_warps - need) * P.promote_pct / 100) : 0;
@@ -152,6 +166,45 @@ __global__ void cook_trace_kernel(const uint4* reqs, const int64_t* classes, uin
     o[0] = make_uint4(lo((uint64_t)q.arrival), hi((uint64_t)q.arrival), lo((uint64_t)dl_ttft), hi((uint64_t)dl_ttft));
     o[1] = make_uint4(lo((uint64_t)dl_e2e), hi((uint64_t)dl_e2e), q.in_tokens, tbt32);
     o[2] = make_uint4(lo(h), hi(h), (q.S - 1u) | (q.cls << 16) | (q.model << 24), 0u);
+}
+
+// Scan tiles of the thread mapping.  Tile t (kScanTile requests) is a header of 8 int64 followed by
+// one 16-byte record per request: {arrival, lim32, model | cls << 8}, lim32 = the smaller of the
+// class's first-token and end-to-end limits clamped to 32 bits (all ones = none, or too large to
+// matter here).  Once the dispatcher's clock has passed arrival + lim32, no instance can serve the
+// request in time.  Header entry k (classes 7 and up share entry 7) is the largest arrival + lim32
+// over the tile's requests of that class: INT64_MAX if one of them has no limit, INT64_MIN if the
+// tile has none, so "clock beyond every entry of the classes I count" means the whole tile is late.
+__global__ void scan_trace_kernel(const uint4* reqs, const int64_t* classes, uint4* scan, uint32_t n) {
+    const uint32_t tile = blockIdx.x, t = threadIdx.x;  // kScanTile threads
+    __shared__ int64_t thr[8];
+    if (t < 8) thr[t] = INT64_MIN;
+    __syncthreads();
+    const uint32_t r = tile * kScanTile + t;
+    uint4* const base = scan + (size_t)tile * (kScanTile + kScanHdrUnits);
+    if (r < n) {
+        const Request q = decode_request(reqs[r]);
+        const int64_t l_ttft = classes[q.cls * 3 + 0], l_e2e = classes[q.cls * 3 + 2];
+        const int64_t lim = l_ttft < 0 ? l_e2e : (l_e2e < 0 ? l_ttft : min(l_ttft, l_e2e));
+        const uint32_t lim32 = (lim < 0 || lim >= 0xFFFFFFFFll) ? 0xFFFFFFFFu : (uint32_t)lim;
+        base[kScanHdrUnits + t] = make_uint4((uint32_t)q.arrival, (uint32_t)((uint64_t)q.arrival >> 32), lim32,
+                                             q.model | (q.cls << 8));
+        const int64_t v = lim32 == 0xFFFFFFFFu ? INT64_MAX : q.arrival + (int64_t)lim32;
+        atomicMax(reinterpret_cast<long long*>(&thr[q.cls < 7 ? q.cls : 7]), (long long)v);
+    }
+    __syncthreads();
+    if (t < 4) {
+        const uint64_t a = (uint64_t)thr[2 * t], b = (uint64_t)thr[2 * t + 1];
+        base[t] = make_uint4((uint32_t)a, (uint32_t)(a >> 32), (uint32_t)b, (uint32_t)(b >> 32));
+    }
+}
+size_t scan_trace_units(uint32_t n) {
+    const size_t tiles = ((size_t)n + kScanTile - 1) / kScanTile;
+    return (tiles ? tiles : 1) * (kScanTile + kScanHdrUnits);
+}
+cudaError_t launch_scan_trace(const uint4* reqs, const int64_t* classes, uint4* scan, uint32_t n) {
+    if (n) scan_trace_kernel<<<(n + kScanTile - 1) / kScanTile, kScanTile>>>(reqs, classes, scan, n);
+    return cudaGetLastError();
 }
 cudaError_t launch_cook_trace(const uint4* reqs, const int64_t* classes, uint4* out, uint32_t n) {
     if (n) cook_trace_kernel<<<(n + 255) / 256, 256>>>(reqs, classes, out, n);

@@ -9,7 +9,7 @@ from gpu_common import gpu_eval, assert_records_equal
 
 pytestmark = pytest.mark.gpu
 
-MAPPINGS = [0, 1]  # lane groups (auto), block layout
+MAPPINGS = [3, 2, 1]  # thread per placement, lane groups, block layout
 
 
 @pytest.fixture(scope="module")
@@ -24,7 +24,7 @@ def ctx():
 @pytest.mark.parametrize("case", all_cases(), ids=lambda c: c["name"])
 def test_hand_timelines_on_gpu(ctx, case, mapping):
     for flags, expect in case["runs"]:
-        if (flags & 14) and mapping == 1:
+        if (flags & 14) and mapping != 2:
             continue      # the fixed-speed engine and the largest-gap test exist in the lane-group mapping only
         res, dumps = gpu_eval(ctx, case["profile"], case["trace"], case["classes"], case["offsets"],
                               case["inst"], case["budget"], None, flags, mapping, dump_idx=[0])
