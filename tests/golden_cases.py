@@ -54,6 +54,7 @@ def check_against_expect(result, dumps, expect):
     assert int(result["status"]) == 0
     for key in SCALAR_KEYS:
         assert int(result[key]) == expect[key], (key, int(result[key]), expect[key])
+    assert list(map(int, result["hit_by_class"])) == expect["hit_by_class"], ("hit_by_class", result["hit_by_class"])
     assert list(map(int, dumps["finish_us"])) == expect["finish_us"]
     assert list(map(int, dumps["first_us"])) == expect["first_us"]
     assert list(map(int, dumps["inst"])) == expect["inst"]

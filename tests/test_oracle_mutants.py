@@ -65,6 +65,11 @@ MUTANTS = [
      "int64_t q_end = q_first + len * q_speed;"),
     ("queued request takes the last slot to free", "if (j == f->B || f->until[x] < f->until[j]) j = x; /* the slot that frees first */",
      "if (j == f->B || f->until[x] > f->until[j]) j = x;"),
+    ("hits booked under the class below", "r->hit_by_class[cls < 7 ? cls : 7]++;",
+     "r->hit_by_class[cls == 0 ? 0 : (cls < 8 ? cls - 1 : 7)]++;"),
+    ("last class bin starts one class early", "r->hit_by_class[cls < 7 ? cls : 7]++;", "r->hit_by_class[cls < 6 ? cls : 7]++;"),
+    ("classes above 7 wrap around instead of sharing the last bin", "r->hit_by_class[cls < 7 ? cls : 7]++;",
+     "r->hit_by_class[cls & 7]++;"),
     ("prefill does not stall the running batch", "in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {",
      "int64_t t_keep = in->T; in->T += prefill_us(in, q->in_tokens);\n                if (S == 1) {"),
 ]
