@@ -293,8 +293,10 @@ MAASO_API int maaso_topk_scores(maaso_ctx *ctx, const maaso_result *results, con
  * requests (ties: lowest index), evaluate the tentative placement (maaso_eval_placements +
  * maaso_score), accept it if the score improved, else mark the model saturated; the best score
  * and placement per device count are kept.  All configurations advance together, so each greedy
- * step is ONE batch of tentative placements on the GPU.  As printed in the paper, the device count
- * k that indexes the outputs is that of the placement before the tentative instance is added.
+ * step is ONE batch of tentative placements on the GPU.  The device count k that indexes the outputs
+ * is that of the placement stored there (Sec. IV-E: "solutions for all possible GPU allocations k"),
+ * so istar_inst[k] occupies exactly k devices; the listing's k, taken before the tentative instance
+ * is added, would file an accepted placement under fewer devices than it needs.
  * A tentative placement that violates a constraint scores -1 and is never accepted.
  * Host pointers: configs[n_configs]; outputs phi_star[gpus+1], istar_len[gpus+1],
  * istar_inst[(gpus+1) * MAASO_MAX_INSTANCES] (packed instance words).  Synchronous; uses the
@@ -346,8 +348,10 @@ MAASO_API int maaso_partition(maaso_ctx *ctx, const maaso_trace *trace, uint32_t
  * holds it until the process exits) instead of context scratch memory.
  * Limits: n_cand <= MAASO_NOALLOC_MAX_CAND and k <= MAASO_NOALLOC_MAX_K; anything larger
  * returns MAASO_ETOOBIG and does nothing.  The call uses the current CUDA device and calls
- * no cudaMalloc / cudaFree or other allocating routine.  The first call on a device looks
- * up the array's device address; make that first call before starting any stream capture.
+ * no cudaMalloc / cudaFree or other allocating routine.  Every call looks up the array's address
+ * on the current device (nothing is cached, so a re-created context or several host threads are
+ * fine); the first call on a device may make the runtime load the library's device code, so make
+ * that first call before starting any stream capture.
  * All calls on a device share the one array: two calls whose kernels may overlap on the
  * GPU (different streams, no ordering between them) race on it, so order them.  Nothing
  * in the array needs clearing between calls: each pass overwrites what the next one reads. */

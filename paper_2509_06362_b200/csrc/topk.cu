@@ -161,23 +161,14 @@ constexpr size_t kNoAllocBytes =
     ((((kNoAllocMaxCand + kChunk - 1) / kChunk) * kNoAllocMaxK * sizeof(Entry) * 2 + 64) + 255) / 256 * 256;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
-constexpr int kMaxDevices = 64;
-static void* g_noalloc_ptr[kMaxDevices];  // device address of the array, per device, once resolved
-
-// Resolves (once per device, with that device current) the device address of the array:
-// its name is only a host-side handle and must not be handed to a kernel.
+// The device address of the array on the current device: its name is only a host-side handle and
+// must not be handed to a kernel.  Looked up on every call (no allocation, no stream work), so no
+// cached pointer can go stale when a context is re-created, and host threads share nothing.
 static cudaError_t noalloc_scratch(void** out) {
-    int dev = -1;
-    cudaError_t e = cudaGetDevice(&dev);
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!g_noalloc_ptr[dev]) {
-        void* p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
-        if (e != cudaSuccess) return e;
-        g_noalloc_ptr[dev] = p;
-    }
-    *out = g_noalloc_ptr[dev];
+    *out = p;
     return cudaSuccess;
 }
 

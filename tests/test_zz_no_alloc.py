@@ -1,9 +1,10 @@
 """maaso_topk_noalloc: the top-k variant for callers that cannot allocate device memory
 (code running under a memory pool that owns the device, or a serving loop that must not
 synchronise on an allocation).  Its scratch is a fixed array inside the library, so this
-test checks, through the C ABI, that it returns exactly what maaso_topk returns, twice in a
-row on different inputs (the second call reuses whatever the first left in the array), and
-that sizes beyond the fixed capacity are refused.  Collected last on purpose."""
+test checks, through the C ABI, that it returns exactly what maaso_topk and the CPU oracle's
+ranking return, twice in a row on different inputs (the second call reuses whatever the first
+left in the array), at the full capacity it was sized for, without changing the amount of free
+device memory, and that sizes beyond the fixed capacity are refused.  Collected last on purpose."""
 import numpy as np
 import pytest
 
@@ -23,7 +24,7 @@ def _records(seed, n):
     return rec
 
 
-def test_no_alloc_topk_matches_topk_twice():
+def test_no_alloc_topk_matches_topk_twice(oracle_mod):
     import torch
     import paper_2509_06362_b200 as m
     ctx = m.Context(0)
@@ -38,7 +39,30 @@ def test_no_alloc_topk_matches_topk_twice():
         assert rc == 0, f"call {call}: {m.maaso_strerror(rc)}"
         assert torch.equal(got_idx, want_idx), f"call {call}: indices differ"
         assert torch.equal(got_rec, want_rec), f"call {call}: records differ"
+        want = oracle_mod.topk(rec, k)
+        assert got_idx.cpu().numpy().view(np.uint32).tolist() == want.tolist(), f"call {call}: oracle ranking differs"
     ctx.close()
+
+
+def test_no_alloc_topk_at_full_capacity_leaves_free_memory_alone(oracle_mod):
+    """The largest input the fixed array was sized for (three selection passes, both halves of the
+    array in use); the amount of free device memory is the same before and after the calls."""
+    import torch
+    import paper_2509_06362_b200 as m
+    n, k = m.NOALLOC_MAX_CAND, m.NOALLOC_MAX_K
+    rec = _records(3, n)
+    dev = torch.from_numpy(rec.view(np.uint8).reshape(n, 128)).cuda()
+    got_idx = torch.full((k,), -7, dtype=torch.int32, device="cuda")
+    got_rec = torch.empty((k, 128), dtype=torch.uint8, device="cuda")
+    assert m.maaso_topk_noalloc(dev, n, k, got_idx, got_rec) == 0    # first call: the device code is loaded by now
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    assert m.maaso_topk_noalloc(dev, n, k, got_idx, got_rec) == 0
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    want = oracle_mod.topk(rec, k)
+    assert got_idx.cpu().numpy().view(np.uint32).tolist() == want.tolist()
+    assert got_rec.cpu().numpy().tobytes() == rec[want].tobytes()
 
 
 def test_no_alloc_topk_refuses_sizes_beyond_its_capacity():
