@@ -671,7 +671,6 @@ int orc_ins_deploy(const orc_profile *p, const orc_request *reqs, uint64_t n, co
             if (mp < 0) break;                                /* M_sat == M */
             if (nI > ORC_MAX_INST) break;
             I[nI] = ((uint32_t)mp & 0xF) | ((configs[c].strategy & 0xFF) << 4) | ((configs[c].batch & 0xFF) << 12);
-            const uint32_t k = nI * dev;                      /* gpuCount(I), before the addition */
             orc_result r;
             int rc = orc_eval_candidate(p, reqs, n, classes, n_classes, I, nI + 1, has_mask, class_mask, gpus,
                                         flags, &r, NULL, NULL, where);
@@ -687,6 +686,11 @@ int orc_ins_deploy(const orc_profile *p, const orc_request *reqs, uint64_t n, co
             } else {
                 sat[mp] = 1;                                  /* stop deploying m' */
             }
+            /* Phi*[k], I*[k] hold "solutions for all possible GPU allocations k" (Sec. IV-E): k is the
+             * device count of the placement that is stored, i.e. gpuCount(I) after the decision above.
+             * (The listing takes k before the addition, which files an accepted placement under fewer
+             * devices than it occupies; Alg. 2 then pairs placements that overrun the cluster.) */
+            const uint32_t k = nI * dev;
             if (phi > phi_star[k]) {
                 phi_star[k] = phi;
                 istar_len[k] = nI;

@@ -436,6 +436,12 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
                         }
                     }
                 } while (LOOP && __any_sync(kFullMask, pending));
+                // An admission can flag its candidate on the winner's lane alone (a time or a queue
+                // beyond what the lane state can hold).  Every lane of the group must see the flag
+                // before the next request, or `pending` would differ inside the group and a group
+                // shuffle would name lanes that are not there.
+                if (__any_sync(kFullMask, status != 0u))
+                    for (uint32_t o = 1; o < G; o <<= 1) status |= __shfl_xor_sync(kFullMask, status, (int)o);
             }
             // release the stage; the warp that arrives last refills it
             __syncwarp();

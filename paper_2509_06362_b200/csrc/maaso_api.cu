@@ -826,7 +826,7 @@ static int ins_deploy_multi(maaso_ctx* ctx, const maaso_trace* trace, const Depl
     if (rc != MAASO_OK) return rc;
 
     struct Step {
-        uint32_t k;    // device count of the placement before the tentative instance was added
+        uint32_t k;    // device count of the placement the step leaves (the one stored under Phi*[k], I*[k])
         uint32_t len;  // instances of the accepted placement after the step
         double phi;    // its score after the step
     };
@@ -884,7 +884,6 @@ static int ins_deploy_multi(maaso_ctx* ctx, const maaso_trace* trace, const Depl
     };
     auto take_step = [&](Chain& ch, int model, uint32_t word, int j) {
         Step sp;
-        sp.k = (uint32_t)ch.inst.size() * ch.dev;
         // a placement beyond the problem's own device count is invalid (score -1), as it would be
         // if the problem were scored alone with its device count as the budget
         const double sc = batch_over[j] ? -1.0 : h_sc[j];
@@ -898,6 +897,7 @@ static int ins_deploy_multi(maaso_ctx* ctx, const maaso_trace* trace, const Depl
             ch.sat[model] = true;  // stop deploying this model
         }
         sp.len = (uint32_t)ch.inst.size();
+        sp.k = sp.len * ch.dev;  // "all possible GPU allocations k" (Sec. IV-E): the devices the stored placement occupies
         sp.phi = ch.phi;
         ch.steps.push_back(sp);
         return accepted;

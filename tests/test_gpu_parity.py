@@ -399,6 +399,10 @@ def test_partition_matches_oracle(ctx, oracle_mod):
         assert (got["g_t"], got["g_l"], got["phi"]) == (want["g_t"], want["g_l"], want["phi"])
         assert got["inst_t"].tolist() == want["inst_t"].tolist()
         assert got["inst_l"].tolist() == want["inst_l"].tolist()
+        # constraint (c) of Sec. IV-C: each sub-cluster's placement fits its share of the devices
+        for side, g in (("inst_t", got["g_t"]), ("inst_l", got["g_l"])):
+            if len(got[side]):
+                assert prof["devices"][gen.unpack_inst(got[side])[1]].sum() <= g
     ctx.free_trace(t)
 
 
@@ -698,6 +702,37 @@ def test_frozen_engine_limits(ctx):
     rec = ctx.results_to_numpy(out)
     assert int(rec["status"][0]) == m.CAND_STATUS["ETOOMANY"] and int(rec["status"][1]) == 0
     ctx.free_trace(t)
+
+
+@pytest.mark.parametrize("flags", [2, 8])
+def test_fixed_speed_engine_time_limit_flags_one_placement_only(ctx, oracle_mod, flags):
+    """Finish times of the fixed-speed engine must stay below 2^57 us.  A placement that passes the
+    limit (two one-slot instances, no SLO limits, a long run of requests of the largest cost the
+    tables allow, each starting when a slot frees) comes back with ELOOP and a zeroed record; the
+    flag is raised by one lane of its group in the middle of the trace, and the placements that share
+    its warp must be scored as if nothing had happened."""
+    import paper_2509_06362_b200 as m
+    prof = gen.profile_tiny()
+    prof["prefill_base_us"] = prof["prefill_base_us"].copy()
+    prof["prefill_q16"] = prof["prefill_q16"].copy()
+    prof["step_us"] = prof["step_us"].copy()
+    prof["prefill_base_us"][0, 2] = 2 ** 31 - 1      # strategy 2 is as slow as the tables allow
+    prof["prefill_q16"][0, 2] = 2 ** 31 - 1
+    prof["step_us"][0, 2, :] = 2 ** 30
+    classes = gen.make_classes([(None, None, None)])
+    n = 3000
+    tr = np.zeros(n, dtype=gen.REQUEST_DTYPE)
+    tr["arrival_us"] = np.arange(n)
+    tr["in_tokens"] = 2 ** 32 - 1
+    tr["out_tokens"] = 65535
+    lists = [[(0, 2, 1), (0, 2, 1)], [(0, 0, 4), (0, 1, 2)], [(0, 0, 1)], [(0, 1, 8), (0, 1, 8)], [(0, 2, 1), (0, 0, 2)]]
+    off, inst = gen.candidates_from_lists(lists)
+    got, _ = gpu_eval(ctx, prof, tr, classes, off, inst, 64, None, flags, 2)
+    want = oracle_mod.eval_placements(prof, tr, classes, off, inst, 64, None, flags)
+    assert int(got["status"][0]) == m.CAND_STATUS["ELOOP"]
+    assert got[0].tobytes()[4:] == bytes(124)                  # nothing but the status
+    assert (want["status"] == 0).all()                        # the oracle has no such limit
+    assert_records_equal(got[1:], want[1:], "placements beside the flagged one")
 
 
 @pytest.mark.parametrize("flags", [0, 1, 2, 3, 4, 5, 8, 13])

@@ -581,8 +581,9 @@ def test_score_properties_and_ranking(oracle_mod):
 def test_ins_deploy_worked_example(oracle_mod):
     """Requests 400 s apart on a one-model profile: one instance serves everything, a second one
     changes nothing, so the score does not improve, the model saturates and the search stops.
-    With k = device count before the addition (as printed), slot 0 gets the one-instance placement
-    in the first step and slot 1 gets the same placement in the second."""
+    Phi*[k] / I*[k] are indexed by the devices the stored placement occupies (Sec. IV-E: "solutions
+    for all possible GPU allocations k"): the one-instance placement sits in slot 1, slot 0 stays
+    empty, and with a one-device cluster the last slot, Phi*[|G_x|], is the one that is filled."""
     prof = gen.profile_tiny()
     tr = gen.make_trace(40, 1.0, 5, doc_class=None)
     tr["arrival_us"] = np.arange(40, dtype=np.int64) * 400_000_000
@@ -595,10 +596,15 @@ def test_ins_deploy_worked_example(oracle_mod):
     thr = tr["out_tokens"].astype(np.int64).sum() / (fin.max() * 1e-6)
     lat = pre.sum() / 40 * 1e-6
     want = 4.0 * 1.0 + 0.3 * min(thr, 1000.0) / 1000.0 + 0.7 * max(10.0 - lat, 0.0) / 10.0
-    assert phi[0] == pytest.approx(want, rel=1e-12) and phi[1] == phi[0]
-    assert phi[2] == 0.0 and phi[3] == 0.0
-    assert I[0].tolist() == [int(gen.pack_inst(0, 0, 4))] and I[1].tolist() == I[0].tolist()
-    assert len(I[2]) == 0 and len(I[3]) == 0
+    assert phi[1] == pytest.approx(want, rel=1e-12)
+    assert phi[0] == 0.0 and phi[2] == 0.0 and phi[3] == 0.0
+    assert I[1].tolist() == [int(gen.pack_inst(0, 0, 4))]
+    assert len(I[0]) == 0 and len(I[2]) == 0 and len(I[3]) == 0
+    phi1, I1 = oracle_mod.ins_deploy(prof, tr, classes, 1, [(0, 4)], 4.0, 0.3, 1000.0, 10.0)
+    assert phi1[1] == phi[1] and phi1[0] == 0.0 and I1[1].tolist() == I[1].tolist()
+    # a two-device strategy on three devices: one instance fits (slot 2), a second one would not
+    phi2, I2 = oracle_mod.ins_deploy(prof, tr, classes, 3, [(1, 4)], 4.0, 0.3, 1000.0, 10.0)
+    assert phi2[2] > 0.0 and phi2[0] == phi2[1] == phi2[3] == 0.0 and len(I2[2]) == 1
 
 
 def test_ins_deploy_properties(oracle_mod):
@@ -615,14 +621,16 @@ def test_ins_deploy_properties(oracle_mod):
             continue
         m, s, b = gen.unpack_inst(I[k])
         assert len(set(zip(s.tolist(), b.tolist()))) == 1 and (int(s[0]), int(b[0])) in configs  # one (P, B) per solution
-        assert prof["devices"][s].sum() <= gpus
+        assert prof["devices"][s].sum() == k          # slot k holds a placement of exactly k devices
         assert (prof["devices"][s] >= prof["min_devices"][m]).all()
         # the stored score is the score of the stored placement
         off = np.array([0, len(I[k])], dtype=np.uint32)
         rec = oracle_mod.eval_placements(prof, tr, classes, off, I[k], gpus)
         assert oracle_mod.score(rec, 4.0, 0.3, 2000.0, 5.0)[0] == phi[k]
     # the first instance of every chain serves the model with the most requests (model 1 here)
-    assert int(gen.unpack_inst(I[0])[0][0]) == 1
+    assert len(I[0]) == 0
+    first = next(k for k in range(gpus + 1) if len(I[k]))
+    assert int(gen.unpack_inst(I[first])[0][0]) == 1
     # a strategy that needs more devices than the sub-cluster has can never be deployed
     phi2, I2 = oracle_mod.ins_deploy(prof, tr, classes, 4, [(6, 16)], 4.0, 0.3, 2000.0, 5.0)
     assert (phi2 == 0).all() and all(len(x) == 0 for x in I2)
@@ -660,6 +668,10 @@ def test_partition_scan(oracle_mod):
             best, arg = phi_t[gpus - gl] + phi_l[gl], (gpus - gl, gl)
     assert (got["g_t"], got["g_l"]) == arg and got["phi"] == best
     assert got["g_t"] + got["g_l"] == gpus
+    # constraint (c) of Sec. IV-C: each sub-cluster's placement fits its share of the devices
+    for side, g in (("inst_t", got["g_t"]), ("inst_l", got["g_l"])):
+        if len(got[side]):
+            assert prof["devices"][gen.unpack_inst(got[side])[1]].sum() <= g
     assert got["inst_t"].tolist() == I_t[arg[0]].tolist() and got["inst_l"].tolist() == I_l[arg[1]].tolist()
     # homogeneous fallback: an unbeatable baseline leaves the cluster unpartitioned
     phi_h, _ = oracle_mod.ins_deploy(prof, tr, classes, gpus, configs, *args, class_mask=mt | ml)
