@@ -377,6 +377,13 @@ MAASO_API int maaso_get_timing(maaso_ctx *ctx, maaso_timing *out);
 /* Number of kernels this context has launched so far (for accounting in benchmarks). */
 MAASO_API uint64_t maaso_launch_count(const maaso_ctx *ctx);
 
+/* Test hook for the out-of-memory paths (no counterpart in the paper): the next `count` times the
+ * context would grow one of its scratch buffers, the growth is refused as if the device had no
+ * memory left.  The call that needed it returns MAASO_ENOMEM and enqueues nothing; the context
+ * keeps the buffers it had, stays usable, and the next call allocates normally.  count = 0
+ * switches the hook off. */
+MAASO_API int maaso_test_fail_allocs(maaso_ctx *ctx, int count);
+
 /* Text for a return code; for MAASO_ECUDA the context keeps the CUDA error string. */
 MAASO_API const char *maaso_strerror(int code);
 MAASO_API const char *maaso_last_error(const maaso_ctx *ctx);

@@ -103,6 +103,8 @@ def _load():
     lib.maaso_set_timing.argtypes = [vp, C.c_int]
     lib.maaso_get_timing.argtypes = [vp, C.POINTER(_Timing)]
     lib.maaso_launch_count.argtypes = [vp]
+    lib.maaso_test_fail_allocs.argtypes = [vp, C.c_int]
+    lib.maaso_test_fail_allocs.restype = C.c_int
     lib.maaso_launch_count.restype = u64
     lib.maaso_strerror.argtypes = [C.c_int]
     lib.maaso_strerror.restype = C.c_char_p
@@ -325,6 +327,11 @@ def maaso_launch_count(ctx):
     return int(_lib.maaso_launch_count(ctx))
 
 
+def maaso_test_fail_allocs(ctx, count):
+    """test hook: the next `count` growths of the context's scratch buffers are refused"""
+    _check(_lib.maaso_test_fail_allocs(ctx, int(count)), "maaso_test_fail_allocs", ctx)
+
+
 # ---- convenience wrappers (allocation of outputs only) -------------------------------------------
 class Trace:
     def __init__(self, ctx, handle, n):
@@ -461,6 +468,10 @@ class Context:
 
     def launch_count(self):
         return maaso_launch_count(self.handle)
+
+    def test_fail_allocs(self, count):
+        """test hook: refuse the next `count` growths of the context's scratch buffers"""
+        maaso_test_fail_allocs(self.handle, count)
 
     @staticmethod
     def results_to_numpy(t):

@@ -347,6 +347,13 @@ eval_group_kernel(const EvalParams P, const int tile_recs, const uint32_t pool_b
             const bool arrived = mbar_wait_bounded(&sm.full_bar[s], parity, P.wait_cycles);
             if (!__all_sync(kFullMask, arrived)) {
                 mbar_wait_bounded(&sm.full_bar[s], parity, P.wait_cycles);  // give copies in flight one more bounded chance
+                // and the later tiles of this item that may have been issued already: no bulk copy
+                // should land in this block's shared memory after the block has left
+                if (!P.stall_test)
+                    for (uint32_t x = 1; x < (uint32_t)kStages && t + x < n_tiles; x++) {
+                        const uint32_t ts = tile_seq + x;
+                        mbar_wait_bounded(&sm.full_bar[ts % kStages], (ts / kStages) & 1u, P.wait_cycles);
+                    }
                 status = MAASO_CAND_ETIMEOUT;
                 sm.work[1] = 1;
                 break;

@@ -85,6 +85,7 @@ struct maaso_ctx {
     uint32_t thread_theta;     // waiting lanes of a warp that trigger a distributor round in the thread mapping
     uint32_t thread_min_cand;  // MAASO_MAP_AUTO takes the thread mapping from this many candidates on
     uint32_t last_mapping;     // mapping the most recent scoring call resolved to
+    int fail_allocs;           // test hook: this many of the next scratch allocations are refused
     bool timing;
     cudaEvent_t ev[6];   // eval: start, after prep, after group, after block; topk: start, end
     bool ev_eval, ev_topk;
@@ -118,6 +119,10 @@ int fail(maaso_ctx* ctx, int code, const char* what) {
 
 int grow(maaso_ctx* ctx, void** buf, size_t* have, size_t need) {
     if (need <= *have) return MAASO_OK;
+    if (ctx && ctx->fail_allocs > 0) {  // test hook: behave as if the allocation had been refused
+        ctx->fail_allocs--;
+        return fail(ctx, MAASO_ENOMEM, "scratch allocation refused (test hook)");
+    }
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "synchronize before growing scratch");
     if (*buf) cudaFree(*buf);
@@ -216,6 +221,7 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
         if (v >= 0) ctx->thread_min_cand = (uint32_t)v;
     }
     ctx->last_mapping = MAASO_MAP_GROUP;
+    ctx->fail_allocs = 0;
     const char* gb = getenv("MAASO_GROUP_BLOCKS");
     if (gb) {
         int v = atoi(gb);
@@ -1212,6 +1218,12 @@ MAASO_API int maaso_get_timing(maaso_ctx* ctx, maaso_timing* out) {
 }
 
 MAASO_API uint64_t maaso_launch_count(const maaso_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+MAASO_API int maaso_test_fail_allocs(maaso_ctx* ctx, int count) {
+    if (!ctx || count < 0) return MAASO_EINVAL;
+    ctx->fail_allocs = count;
+    return MAASO_OK;
+}
 
 MAASO_API const char* maaso_strerror(int code) {
     switch (code) {

@@ -879,3 +879,48 @@ def test_several_traces_limits(ctx):
         ctx.eval_placements_multi([a] * 17, d_off, d_inst, 4)
     ctx.free_trace(a)
     ctx.free_trace(b)
+
+
+def test_refused_scratch_allocation_is_reported_and_survived(oracle_mod):
+    """Host-side failure path: the context's scratch growth is refused (test hook, as if the device
+    were out of memory).  The call returns MAASO_ENOMEM and enqueues nothing; the same context then
+    scores the same batch correctly, a larger one too, and holds no more device memory than a context
+    that never saw a failure."""
+    import torch
+    import paper_2509_06362_b200 as m
+    cfg = gen.make_config("node", n_cand=2000, n_req=600)
+    want = oracle_mod.eval_placements(cfg["profile"], cfg["traces"][0], cfg["classes"], cfg["offsets"], cfg["inst"], 8)
+
+    def used_by(fail_first):
+        torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info()[0]
+        c = m.Context(0)
+        c.load_profile(cfg["profile"])
+        t = c.load_trace(cfg["traces"][0], cfg["classes"])
+        d_off, d_inst = c.to_device(cfg["offsets"][:501]), c.to_device(cfg["inst"][:int(cfg["offsets"][500])])
+        out = torch.full((500, 128), 0xAB, dtype=torch.uint8, device="cuda")
+        if fail_first:
+            c.test_fail_allocs(1)
+            with pytest.raises(m.MaasoError) as err:
+                c.eval_placements(t, d_off, d_inst, 8, out=out)
+            assert err.value.code == -3
+            torch.cuda.synchronize()
+            assert bool((out == 0xAB).all())                      # nothing was enqueued
+            idx = torch.empty(8, dtype=torch.int32, device="cuda")
+            c.test_fail_allocs(1)
+            with pytest.raises(m.MaasoError) as err:
+                c.topk(out, 8)                                    # the ranking's scratch is refused as well
+            assert err.value.code == -3
+        got = c.eval_placements(t, d_off, d_inst, 8, out=out)
+        torch.cuda.synchronize()
+        assert c.results_to_numpy(got).tobytes() == want[:500].tobytes()
+        big = c.eval_placements(t, c.to_device(cfg["offsets"]), c.to_device(cfg["inst"]), 8)   # grows the scratch
+        c.topk(big, 8)
+        torch.cuda.synchronize()
+        assert c.results_to_numpy(big).tobytes() == want.tobytes()
+        used = free0 - torch.cuda.mem_get_info()[0]
+        c.close()
+        return used
+
+    clean = used_by(False)
+    assert used_by(True) <= clean
