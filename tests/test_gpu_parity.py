@@ -164,11 +164,10 @@ def test_node_config_full_size_as_benchmarked(ctx, oracle_mod):
     cfg = gen.make_config("node")
     tr = cfg["traces"][0]
     want = oracle_mod.eval_placements_parallel(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8)
-    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=0)
-    assert_records_equal(got, want, "node full")
     assert (want["status"] == 0).all() and (want["n_counted"] == 10000).all()
-    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=1)
-    assert_records_equal(got, want, "node full, block mapping")
+    for mapping in (0, 2, 3, 1):
+        got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=mapping)
+        assert_records_equal(got, want, f"node full, mapping {mapping}")
 
 
 @pytest.mark.parametrize("flags", [1, 2, 4, 8, 9])
@@ -192,24 +191,74 @@ def test_multimodel_full_trace_sampled_candidates(ctx, oracle_mod):
     off, inst = _subset(cfg, sel)
     idx = np.array([0, len(sel) - 1], dtype=np.uint32)
     want, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, 32, dump_idx=idx)
-    got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 32, dump_idx=idx)
-    assert_records_equal(got, want, "multimodel full trace")
-    for k in wd:
-        assert (gd[k] == wd[k]).all(), k
+    for mapping in (2, 3):
+        got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 32, mapping=mapping, dump_idx=idx)
+        assert_records_equal(got, want, f"multimodel full trace, mapping {mapping}")
+        for k in wd:
+            assert (gd[k] == wd[k]).all(), (k, mapping)
 
 
 def test_scale_full_trace_sampled_candidates(ctx, oracle_mod):
-    """10^6-request trace, four SLO classes, candidates sampled from the 10^6-candidate set
-    including the ones with the most instances (over 32: block path)."""
+    """10^6-request trace, four SLO classes, 272 placements of the 10^6-placement set: an even sample,
+    the ones with the most instances (over 32) and some of every lane-group width (1, 2, 3-4, 5-8,
+    9-16, 17-32 instances); per-request times compared for six of them."""
     cfg = gen.make_config("scale")
     tr = cfg["traces"][0]
     n_i = np.diff(cfg["offsets"].astype(np.int64))
-    sel = sorted(set(np.arange(0, 1_000_000, 40_000).tolist() + np.argsort(n_i)[-4:].tolist()))
+    pick = set(np.arange(0, 1_000_000, 5_000).tolist() + np.argsort(n_i)[-8:].tolist())
+    for lo_n, hi_n in ((1, 1), (2, 2), (3, 4), (5, 8), (9, 16), (17, 32), (33, 128)):
+        pick.update(np.nonzero((n_i >= lo_n) & (n_i <= hi_n))[0][:10].tolist())
+    sel = sorted(pick)
+    assert len(sel) >= 256 and (n_i[sel] > 32).sum() >= 4
     off, inst = _subset(cfg, sel)
+    big = [k for k, c in enumerate(sel) if n_i[c] > 32][:2]
+    idx = np.array(sorted(set([0, len(sel) // 3, len(sel) // 2, len(sel) - 1] + big)), dtype=np.uint32)
     want = oracle_mod.eval_placements_parallel(cfg["profile"], tr, cfg["classes"], off, inst, 128, workers=8)
-    got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 128)
+    _, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], *_subset(cfg, [sel[k] for k in idx]), 128,
+                                       dump_idx=np.arange(len(idx), dtype=np.uint32))
     assert (want["status"] == 0).all() and n_i.max() > 32
-    assert_records_equal(got, want, "scale full trace")
+    for mapping in (2, 3):
+        got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, 128, mapping=mapping, dump_idx=idx)
+        assert_records_equal(got, want, f"scale full trace, mapping {mapping}")
+        for k in wd:
+            assert (gd[k] == wd[k]).all(), (k, mapping)
+
+
+def test_multimodel_all_candidates_trace_prefix(ctx, oracle_mod):
+    """Every one of the 100,000 placements of the multi-model sweep in ONE call (the batch size the
+    benchmark launches: many waves of work items, cost-sorted buckets), against the first 200 requests."""
+    cfg = gen.make_config("multimodel", n_req=200)
+    tr = cfg["traces"][0]
+    want = oracle_mod.eval_placements_parallel(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 32,
+                                               workers=8)
+    assert len(want) == 100_000 and (want["status"] == 0).all()
+    for mapping in (2, 3):
+        got, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 32, mapping=mapping)
+        assert_records_equal(got, want, f"multimodel, all placements, mapping {mapping}")
+
+
+def test_scale_all_candidates_trace_prefix_and_topk(ctx, oracle_mod):
+    """All 10^6 placements of the scale-stress sweep in ONE call (placements of more than 32 instances
+    mixed in), against the first 100 requests; records byte for byte, and the top-64 of that run
+    against the CPU ranking."""
+    import torch
+    cfg = gen.make_config("scale", n_req=100)
+    tr = cfg["traces"][0]
+    want = oracle_mod.eval_placements_parallel(cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 128,
+                                               workers=8)
+    assert len(want) == 1_000_000 and (want["status"] == 0).all()
+    top = oracle_mod.topk(want, 64)
+    ctx.load_profile(cfg["profile"])
+    t = ctx.load_trace(tr, cfg["classes"])
+    d_off, d_inst = ctx.to_device(cfg["offsets"]), ctx.to_device(cfg["inst"])
+    for mapping in (2, 3):
+        out = ctx.eval_placements(t, d_off, d_inst, 128, mapping=mapping)
+        idx, rec = ctx.topk(out, 64)
+        torch.cuda.synchronize()
+        assert_records_equal(ctx.results_to_numpy(out), want, f"scale, all placements, mapping {mapping}")
+        assert idx.cpu().numpy().view(np.uint32).tolist() == top.tolist()
+        assert rec.cpu().numpy().tobytes() == want[top].tobytes()
+    ctx.free_trace(t)
 
 
 def test_bursty_all_traces_full_length(ctx, oracle_mod):
@@ -228,7 +277,9 @@ def test_determinism_and_mapping_independence(ctx):
     a, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=0)
     b, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=0)
     c, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=1)
-    assert a.tobytes() == b.tobytes() == c.tobytes()
+    d, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=2)
+    e, _ = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], cfg["offsets"], cfg["inst"], 8, mapping=3)
+    assert a.tobytes() == b.tobytes() == c.tobytes() == d.tobytes() == e.tobytes()
 
 
 def test_host_entry_point_matches_device_entry_point(ctx, oracle_mod):
