@@ -24,7 +24,10 @@ constexpr int kCostBins = 256;   // bin 0 = most expensive (largest total batch 
 constexpr int kCounterWords = 8192;  // counters | work counters | histograms + cursors, cleared per call
 constexpr int kGroupThreads = 128;
 constexpr int kScanTile = 256;       // requests per scan tile of the thread mapping
-constexpr int kScanHdrUnits = 4;     // 16-byte units of a scan tile's header (8 int64)
+constexpr int kScanHdrUnits = 40;    // 16-byte units of a scan tile's header (see scan_trace_kernel)
+constexpr int kScanHdrBase = 4;      // unit of the tile's base arrival time
+constexpr int kScanHdrClassBits = 5; // first unit of the 8 per-class bitmaps (2 units = 256 bits each)
+constexpr int kScanHdrModelBits = 21; // first unit of the 8 per-model bitmaps
 constexpr int kMaxTraces = 16;  // traces one call of the lane-group kernel can replay side by side
 
 struct Request {

@@ -357,9 +357,13 @@ __device__ __forceinline__ uint4 ldg_nc(const uint4* p) { return __ldg(p); }
 // totals of the trace, and an admission takes its request out again.
 template <bool OPT>
 __global__ void __launch_bounds__(32, 1)
-eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_bytes, const uint32_t theta) {
+eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_bytes, const uint32_t theta,
+                   unsigned char* const arena) {
+    // arena: the placements' state lives in global memory (one region of pool_bytes per warp, kept hot by
+    // L1/L2) instead of shared memory, which leaves room for many more resident warps; null = shared memory
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    const ThreadSmem sm = t_carve(smem_raw, pool_bytes);
+    ThreadSmem sm = t_carve(smem_raw, arena ? 0u : pool_bytes);
+    if (arena) sm.pool = arena + (size_t)blockIdx.x * pool_bytes;
     const uint32_t lane = threadIdx.x;
     if (lane == 0) {
         for (int s = 0; s < kTStages; s++) mbar_init(&sm.full_bar[s], 1);
@@ -370,7 +374,11 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
     const uint32_t pool_units = pool_bytes / 16u;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
     const uint32_t n_traces = P.n_traces > 1 ? P.n_traces : 1u;
-    const uint32_t ru = (P.n_models + 7u) >> 3;  // units of the per-model instance ranges
+    // a lane's share of the pool: units [0, rr) per-model instance ranges, [rr, rr + M) one entry per model
+    // (lower bound of any predicted first token, smallest prefill base, smallest prediction step),
+    // 2 units for the live map of the current tile, then the instances from unit ru on
+    const uint32_t rr = (P.n_models + 7u) >> 3;
+    const uint32_t ru = rr + P.n_models + 2u;
     // items per bucket, buckets with the fewest lanes (the largest placements) first
     uint32_t items[9];
     uint32_t total_items = 0;
@@ -433,8 +441,8 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
         if (valid) {
             const uint32_t lo = P.offsets[cand];
             n_i = P.offsets[cand + 1] - lo;
-            uint32_t rng_lo[MAASO_MAX_MODELS], rng_hi[MAASO_MAX_MODELS];
-            for (int m = 0; m < MAASO_MAX_MODELS; m++) { rng_lo[m] = 0xFFu; rng_hi[m] = 0u; }
+            uint32_t rng_lo[MAASO_MAX_MODELS], rng_hi[MAASO_MAX_MODELS], min_pre[MAASO_MAX_MODELS], min_step[MAASO_MAX_MODELS];
+            for (int m = 0; m < MAASO_MAX_MODELS; m++) { rng_lo[m] = 0xFFu; rng_hi[m] = 0u; min_pre[m] = 0xFFFFFFFFu; min_step[m] = 0xFFFFFFFFu; }
             uint32_t ko = ru + 4u * n_i, so = 0;
             for (uint32_t j = 0; j < n_i; j++) {
                 const uint32_t word = P.inst[lo + j];
@@ -464,9 +472,16 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                 rng_lo[m] = min(rng_lo[m], j);
                 rng_hi[m] = j + 1u;
                 hasmodel |= 1u << m;
+                // the smallest step a prediction for this model can use: the step at the batch cap, or
+                // (optimistic estimate) at any level up to it
+                uint32_t ms = in.stepB;
+                if (OPT)
+                    for (uint32_t w = 1; w < B; w++) ms = min(ms, (uint32_t)P.rows[row * kRowStride + 1 + w]);
+                min_step[m] = min(min_step[m], ms);
+                min_pre[m] = min(min_pre[m], in.pre_base);
             }
             // per-model instance ranges: halfword m = first index | (last index + 1) << 8
-            for (uint32_t u = 0; u < ru; u++) {
+            for (uint32_t u = 0; u < rr; u++) {
                 uint32_t rw[4];
                 for (int i = 0; i < 4; i++) {
                     const uint32_t m0 = 8u * u + 2u * i, m1 = m0 + 1u;
@@ -476,10 +491,13 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                 }
                 *e.pl.unit(u) = make_uint4(rw[0], rw[1], rw[2], rw[3]);
             }
+            // nothing runs yet: every predicted first token lies at or after the smallest prefill base
+            for (uint32_t m = 0; m < P.n_models; m++) *e.pl.unit(rr + m) = make_uint4(min_pre[m], 0u, min_pre[m], min_step[m]);
         }
         const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
         // header entries of a scan tile this lane has to look at (classes 7 and up share entry 7)
         const uint32_t hmask = (cmask & 0x7Fu) | ((cmask >> 7) ? 0x80u : 0u);
+        const uint32_t mmask = (hasmodel & 0x7Fu) | ((hasmodel >> 7) ? 0x80u : 0u);  // the same for the per-model maps
         bool side = P.rej_by_model != nullptr;
         if (valid && P.dump_row) side = side || P.dump_row[cand] >= 0;
         // every request of the subset counted as rejected; admissions take theirs out
@@ -523,18 +541,38 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
             const uint4* const rp = tile + kScanHdrUnits;  // the tile's scan records
             const uint32_t recs = min((uint32_t)kTTile, n_req - t * kTTile);
             uint32_t ri = (valid && status == 0) ? 0u : recs;
-            // the whole tile is late for this lane if its clock has passed the header entry of every class it counts
-            if (ri < recs && !side) {
-                bool all_late = true;
+            // The tile's live map of this lane: requests of a class that is not late as a whole (the
+            // dispatcher's clock has not passed the class's header entry) and of a model the placement
+            // has an instance of.  Everything else in the tile is rejected without being looked at.
+            if (ri < recs) {
+                uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
+                if (side) {
+                    lo = hi = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);  // every rejection is written out
+                } else {
+                    uint4 mlo = lo, mhi = lo;
 #pragma unroll
-                for (int k = 0; k < 4; k++) {
-                    const uint4 h = tile[k];
-                    const int64_t a = (int64_t)(((uint64_t)h.y << 32) | h.x), c = (int64_t)(((uint64_t)h.w << 32) | h.z);
-                    if (((hmask >> (2 * k)) & 1u) && a >= now) all_late = false;
-                    if (((hmask >> (2 * k + 1)) & 1u) && c >= now) all_late = false;
+                    for (int k = 0; k < 8; k++) {
+                        const uint4 h = tile[k >> 1];
+                        const int64_t thr = (k & 1) ? (int64_t)(((uint64_t)h.w << 32) | h.z) : (int64_t)(((uint64_t)h.y << 32) | h.x);
+                        if (((hmask >> k) & 1u) && thr >= now) {
+                            const uint4 a = tile[kScanHdrClassBits + 2 * k], c = tile[kScanHdrClassBits + 2 * k + 1];
+                            lo.x |= a.x; lo.y |= a.y; lo.z |= a.z; lo.w |= a.w;
+                            hi.x |= c.x; hi.y |= c.y; hi.z |= c.z; hi.w |= c.w;
+                        }
+                        if ((mmask >> k) & 1u) {
+                            const uint4 a = tile[kScanHdrModelBits + 2 * k], c = tile[kScanHdrModelBits + 2 * k + 1];
+                            mlo.x |= a.x; mlo.y |= a.y; mlo.z |= a.z; mlo.w |= a.w;
+                            mhi.x |= c.x; mhi.y |= c.y; mhi.z |= c.z; mhi.w |= c.w;
+                        }
+                    }
+                    lo.x &= mlo.x; lo.y &= mlo.y; lo.z &= mlo.z; lo.w &= mlo.w;
+                    hi.x &= mhi.x; hi.y &= mhi.y; hi.z &= mhi.z; hi.w &= mhi.w;
                 }
-                if (all_late) ri = recs;
+                *e.pl.unit(rr + P.n_models) = lo;
+                *e.pl.unit(rr + P.n_models + 1u) = hi;
+                if ((lo.x | lo.y | lo.z | lo.w | hi.x | hi.y | hi.z | hi.w) == 0u) ri = recs;
             }
+            const int64_t tile_base = (int64_t)(((uint64_t)tile[kScanHdrBase].y << 32) | tile[kScanHdrBase].x);
             bool waiting = false;  // this lane stands at a request that needs the distributor
             uint4 f0, f1, f2;      // that request's full record
             f0 = f1 = f2 = make_uint4(0u, 0u, 0u, 0u);
@@ -542,31 +580,37 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                 uint32_t wl;
                 for (;;) {
 #pragma unroll 1
-                    for (int c = 0; c < 2; c++) {
+                    for (int c = 0; c < 8; c++) {
                         if (waiting || ri >= recs) continue;
-                        // four records at a time: the first one that needs the distributor stops the lane
-                        uint4 r[4];
-#pragma unroll
-                        for (int k = 0; k < 4; k++) r[k] = rp[ri + k];
-                        uint32_t first = 4;
-#pragma unroll
-                        for (int k = 0; k < 4; k++) {
-                            if (first != 4u || ri + k >= recs) continue;
-                            if (!((cmask >> ((r[k].w >> 8) & 31u)) & 1u)) continue;  // not in the request subset
-                            const int64_t arrival = (int64_t)(((uint64_t)r[k].y << 32) | r[k].x);
-                            now = max(now, arrival);  // pending time: the dispatcher never goes back
-                            const bool late = r[k].z != 0xFFFFFFFFu && arrival + (int64_t)r[k].z < now;
-                            if (((hasmodel >> (r[k].w & 0xFFu)) & 1u) && !late) first = k;
-                            // else overflow protection, the plain case: nobody can meet the deadline -> rejected
-                            else if (side) t_reject_side(P, out_base + cand, t * kTTile + ri + k, r[k].w & 0xFFu);
+                        // the next live request at or after ri
+                        const uint32_t bits = *e.pl.word(rr + P.n_models + (ri >> 7), (ri >> 5) & 3u) >> (ri & 31u);
+                        if (bits == 0u) { ri = min((ri | 31u) + 1u, recs); continue; }
+                        ri += (uint32_t)__ffs((int)bits) - 1u;
+                        if (ri >= recs) { ri = recs; continue; }
+                        const uint4 sr = rp[ri];
+                        const uint32_t model = sr.w & 0xFFu;
+                        if (!((cmask >> ((sr.w >> 8) & 31u)) & 1u)) { ri++; continue; }  // not in the request subset
+                        bool real = ((hasmodel >> model) & 1u) != 0u;
+                        if (real && sr.x != 0xFFFFFFFFu) {
+                            // Too late whatever the instance?  Every predicted first token of this model lies at
+                            // or after flb: the dispatcher's clock plus the smallest prefill base, and the lower
+                            // bound kept from the latest look at the model's instances (times only move forward).
+                            const uint4 me = *e.pl.unit(rr + model);
+                            const int64_t arrival = tile_base + (int64_t)sr.x;
+                            const int64_t flb = max(max(now, arrival) + (int64_t)me.z, (int64_t)(((uint64_t)me.y << 32) | me.x));
+                            const bool late_first = sr.y != 0xFFFFFFFFu && arrival + (int64_t)sr.y < flb;
+                            const bool late_end = sr.z != 0xFFFFFFFFu &&
+                                                  arrival + (int64_t)sr.z < flb + (int64_t)((uint64_t)(sr.w >> 16) * me.w);
+                            real = !(late_first || late_end);
                         }
-                        if (first != 4u) {
-                            ri += first;
+                        if (real) {
                             waiting = true;
                             const uint4* full = cooked + (size_t)(t * kTTile + ri) * kCookedWords;
                             f0 = ldg_nc(full); f1 = ldg_nc(full + 1); f2 = ldg_nc(full + 2);
                         } else {
-                            ri = min(ri + 4u, recs);
+                            // overflow protection, the plain case: nobody can meet the deadline -> rejected
+                            if (side) t_reject_side(P, out_base + cand, t * kTTile + ri, model);
+                            ri++;
                         }
                     }
                     wl = __ballot_sync(kFullMaskT, waiting);
@@ -581,6 +625,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                 const CookedReq q = decode_cooked(f0, f1, f2);
                 const uint32_t req = t * kTTile + ri;
                 ri++;
+                now = max(now, q.arrival);  // pending time: the dispatcher never goes back
                 // instances of the request's model
                 const uint4 rg = *e.pl.unit(q.model >> 3);
                 const uint32_t rgw = (q.model & 4u) ? ((q.model & 2u) ? rg.w : rg.z) : ((q.model & 2u) ? rg.y : rg.x);
@@ -593,6 +638,9 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                     uint64_t best = kKeyInf;
                     uint32_t bj = 0, bk = 0;
                     int64_t bT = 0, bpre = 0;
+                    // smallest and second smallest (start time + prefill base) over the model's instances
+                    int64_t lb1 = INT64_MAX, lb2 = INT64_MAX;
+                    uint32_t lb1j = 0xFFFFFFFFu;
                     for (uint32_t j = j_lo; j < j_hi; j++) {
                         TInst in;
                         t_load(e.pl, ru, j, in);
@@ -620,10 +668,16 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                         const uint32_t sB = (OPT && free_slot) ? in.swn : in.stepB;
                         const int64_t first = t0 + pre;
                         const int64_t fin = first + (int64_t)((uint64_t)q.Sm1 * sB);
+                        {
+                            const int64_t lb = t0 + (int64_t)in.pre_base;
+                            if (lb < lb1) { lb2 = lb1; lb1 = lb; lb1j = j; }
+                            else if (lb < lb2) lb2 = lb;
+                        }
                         const bool ok = first <= q.dl_ttft && (q.Sm1 == 0 || sB <= q.tbt32) && fin <= q.dl_e2e;
                         const uint64_t key = ((uint64_t)(free_slot ? 0u : 1u) << 63) | (uint64_t)first;
                         if (ok && key < best) { best = key; bj = j; bk = kadd; bT = T; bpre = pre; }
                     }
+                    int64_t lb_new = lb1;  // the model's lower bound as this look at its instances leaves it
                     if (best == kKeyInf) {
                         // overflow protection: nobody can meet the deadline -> rejected
                         if (side) t_reject_side(P, out_base + cand, req, q.model);
@@ -637,6 +691,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                             t_admit(in, bj, q, req, bpre, e);
                             rej_sum -= q.rej;
                             pending = false;
+                            lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
                         } else {
                             // every capable instance is full: wait until the chosen slot frees
                             now = in.tc;
@@ -646,12 +701,15 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                                 t_admit(in, bj, q, req, bpre, e);
                                 rej_sum -= q.rej;
                                 pending = false;
+                                lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
                             } else if (tries >= kAttemptCap) {
                                 status = MAASO_CAND_ELOOP;
                                 pending = false;
                             }
                         }
                     }
+                    if (lb1 != INT64_MAX)
+                        *reinterpret_cast<uint2*>(e.pl.unit(rr + q.model)) = make_uint2((uint32_t)lb_new, (uint32_t)((uint64_t)lb_new >> 32));
                 } while (OPT && pending);
                 extra += tries - 1u;
                 if (status) ri = recs;  // given up on this candidate
@@ -686,18 +744,19 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
     }
 }
 
-cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t theta, cudaStream_t stream) {
+cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t theta, void* arena,
+                               cudaStream_t stream) {
     auto kernel = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_thread_kernel<true> : eval_thread_kernel<false>;
-    const size_t smem = (size_t)pool_bytes + kTFixedBytes;
+    const size_t smem = (arena ? 0 : (size_t)pool_bytes) + kTFixedBytes;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kernel<<<grid, 32, smem, stream>>>(P, pool_bytes, theta);
+    kernel<<<grid, 32, smem, stream>>>(P, pool_bytes, theta, static_cast<unsigned char*>(arena));
     return cudaGetLastError();
 }
 
-int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes) {
+int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, bool in_smem) {
     auto kernel = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_thread_kernel<true> : eval_thread_kernel<false>;
-    const size_t smem = (size_t)pool_bytes + kTFixedBytes;
+    const size_t smem = (in_smem ? (size_t)pool_bytes : 0) + kTFixedBytes;
     cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, 32, smem) != cudaSuccess) return 1;

@@ -19,8 +19,9 @@ cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, int 
                               cudaStream_t stream);
 int occupancy_eval_group(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm);
 size_t group_scratch_per_lane();
-cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t theta, cudaStream_t stream);
-int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes);
+cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t theta, void* arena,
+                               cudaStream_t stream);
+int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, bool in_smem);
 size_t thread_scratch_per_warp(uint32_t pool_bytes);
 uint32_t thread_fixed_smem();
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
@@ -81,6 +82,7 @@ struct maaso_ctx {
     int group_blocks;  // blocks of the lane-group kernel per SM its key pool is sized for; 0 = by batch size
     int smem_per_sm;
     int promote_pct;  // share of the spare resident warps the planner may use for promotions
+    int thread_arena_kb;  // thread mapping: KB of global memory per warp for the placements' state, 0 = shared memory
     int thread_blocks;   // one-warp blocks of the thread-mapping kernel per SM its pool is sized for
     uint32_t thread_theta;     // waiting lanes of a warp that trigger a distributor round in the thread mapping
     uint32_t thread_min_cand;  // MAASO_MAP_AUTO takes the thread mapping from this many candidates on
@@ -202,6 +204,12 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
         if (v >= 16 && v <= 2048) ctx->tile_recs = v & ~1;  // even: tiles of 8-byte terms stay 16-byte aligned
     }
 
+    ctx->thread_arena_kb = 0;
+    const char* ta = getenv("MAASO_THREAD_ARENA_KB");
+    if (ta) {
+        int v = atoi(ta);
+        if (v >= 0 && v <= 1023) ctx->thread_arena_kb = v;
+    }
     ctx->thread_blocks = 6;
     const char* tb = getenv("MAASO_THREAD_BLOCKS");
     if (tb) {
@@ -520,20 +528,26 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     if (threads) {
         // thread mapping: one-warp blocks; the pool is what is left of an SM's shared memory when
         // `thread_blocks` of them share it (1 KB per block is reserved by the system)
-        size_t per_block = (size_t)ctx->smem_per_sm / (size_t)ctx->thread_blocks;
-        per_block = per_block > 1024 ? per_block - 1024 : 0;
-        if (per_block > 227u * 1024u) per_block = 227u * 1024u;
-        const size_t fixed = thread_fixed_smem();
-        size_t pool = per_block > fixed ? per_block - fixed : 0;
-        pool -= pool % 512;
+        size_t pool;
+        if (ctx->thread_arena_kb > 0) {
+            pool = (size_t)ctx->thread_arena_kb * 1024;
+        } else {
+            size_t per_block = (size_t)ctx->smem_per_sm / (size_t)ctx->thread_blocks;
+            per_block = per_block > 1024 ? per_block - 1024 : 0;
+            if (per_block > 227u * 1024u) per_block = 227u * 1024u;
+            const size_t fixed = thread_fixed_smem();
+            pool = per_block > fixed ? per_block - fixed : 0;
+            pool -= pool % 512;
+        }
         if (pool > 65535u * 16u) pool = 65535u * 16u - (65535u * 16u) % 512;  // unit offsets are 16-bit
         if (pool < 4096) return fail(ctx, MAASO_ESTATE, "eval: no shared memory for the thread mapping");
         thread_pool = (uint32_t)pool;
         P.thread_pool_units = thread_pool / 16u;
-        grid_t = ctx->sm_count * occupancy_eval_thread(P, thread_pool);
+        grid_t = ctx->sm_count * occupancy_eval_thread(P, thread_pool, ctx->thread_arena_kb == 0);
         const uint64_t max_items_t = ((uint64_t)C + 9) * n_traces;
         if ((uint64_t)grid_t > max_items_t) grid_t = (int)max_items_t;
-        pay_entries = ((size_t)grid_t * thread_scratch_per_warp(thread_pool) + sizeof(Payload) - 1) / sizeof(Payload);
+        pay_entries = ((size_t)grid_t * (thread_scratch_per_warp(thread_pool) + (ctx->thread_arena_kb > 0 ? thread_pool : 0)) +
+                       sizeof(Payload) - 1) / sizeof(Payload);
     } else if (o.mapping != MAASO_MAP_BLOCK) {
         const int occ_g = occupancy_eval_group(P, tile, group_blocks, ctx->smem_per_sm);
         grid_g = ctx->sm_count * occ_g;
@@ -549,7 +563,7 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
         bool used = n_traces == 1 && o.mapping == MAASO_MAP_BLOCK;
         if (n_traces == 1 && b == kGenericBlockBucket) {
             if (o.mapping == MAASO_MAP_GROUP) used = cands->n_inst > 32;
-            if (threads) used = cands->n_inst * 22ull + 2ull > P.thread_pool_units;  // 22 units: an instance with 64 slots
+            if (threads) used = cands->n_inst * 22ull + 20ull > P.thread_pool_units;  // 22 units: an instance with 64 slots
         }
         grid_b[b - 6] = 0;
         if (!used) continue;
@@ -596,7 +610,11 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     if (e != cudaSuccess) return cuda_fail(ctx, e, "prep launch");
     if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
     if (threads) {
-        e = launch_eval_thread(P, grid_t, thread_pool, ctx->thread_theta, stream);
+        // the arena (if any) follows the scratch entries of the running requests
+        void* arena = ctx->thread_arena_kb > 0
+                          ? static_cast<void*>(reinterpret_cast<unsigned char*>(P.payload) + (size_t)grid_t * thread_scratch_per_warp(thread_pool))
+                          : nullptr;
+        e = launch_eval_thread(P, grid_t, thread_pool, ctx->thread_theta, arena, stream);
         launches++;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "thread kernel launch");
     } else if (o.mapping != MAASO_MAP_BLOCK) {

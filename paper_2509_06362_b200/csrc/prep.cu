@@ -9,7 +9,9 @@ __global__ void prep_kernel(const EvalParams P) {
     if (c >= P.n_cand) return;
     const uint32_t lo = P.offsets[c], hi = P.offsets[c + 1];
     uint32_t status = 0, n = 0, sum_b = 0;
-    uint32_t units = (P.n_models + 7u) >> 3;  // thread mapping: 16-byte units of state (model ranges, per instance 4 + key blocks + minima)
+    // thread mapping: 16-byte units of state (model ranges, one entry per model, the tile's live map, per
+    // instance 4 + key blocks + minima)
+    uint32_t units = ((P.n_models + 7u) >> 3) + P.n_models + 2u;
     if (hi < lo || hi > P.n_inst) {
         status = MAASO_CAND_EBADINST;  // malformed CSR row
     } else {
@@ -168,13 +170,19 @@ __global__ void cook_trace_kernel(const uint4* reqs, const int64_t* classes, uin
     o[2] = make_uint4(lo(h), hi(h), (q.S - 1u) | (q.cls << 16) | (q.model << 24), 0u);
 }
 
-// Scan tiles of the thread mapping.  Tile t (kScanTile requests) is a header of 8 int64 followed by
-// one 16-byte record per request: {arrival, lim32, model | cls << 8}, lim32 = the smaller of the
-// class's first-token and end-to-end limits clamped to 32 bits (all ones = none, or too large to
-// matter here).  Once the dispatcher's clock has passed arrival + lim32, no instance can serve the
-// request in time.  Header entry k (classes 7 and up share entry 7) is the largest arrival + lim32
-// over the tile's requests of that class: INT64_MAX if one of them has no limit, INT64_MIN if the
-// tile has none, so "clock beyond every entry of the classes I count" means the whole tile is late.
+// Scan tiles of the thread mapping.  Tile t (kScanTile requests) is a header followed by one
+// 16-byte record per request.
+//   record: {arrival - the tile's base arrival (all ones: does not fit 32 bits, look at the full record),
+//            TTFT limit, end-to-end limit (each clamped to 32 bits; all ones = none, or too large to
+//            matter here), model | cls << 8 | (output tokens - 1) << 16}.  Once the dispatcher's clock has
+//            passed arrival + limit, no instance can serve the request in time.
+//   header units 0..3: eight int64, entry k (classes 7 and up share entry 7) = the largest arrival +
+//            min(TTFT, end-to-end limit) over the tile's requests of that class: INT64_MAX if one of
+//            them has no limit, INT64_MIN if the tile has none, so "clock beyond the entries of the
+//            classes I count" means the whole tile is late;
+//   unit 4: base arrival (int64) = arrival of the tile's first request;
+//   units 5..20: per class slot a 256-bit map of the tile's requests of that class;
+//   units 21..36: the same per model (models 7 and up share slot 7).
 __global__ void scan_trace_kernel(const uint4* reqs, const int64_t* classes, uint4* scan, uint32_t n) {
     const uint32_t tile = blockIdx.x, t = threadIdx.x;  // kScanTile threads
     __shared__ int64_t thr[8];
@@ -182,21 +190,37 @@ __global__ void scan_trace_kernel(const uint4* reqs, const int64_t* classes, uin
     __syncthreads();
     const uint32_t r = tile * kScanTile + t;
     uint4* const base = scan + (size_t)tile * (kScanTile + kScanHdrUnits);
+    const int64_t base_arrival = decode_request(reqs[tile * kScanTile]).arrival;
+    uint32_t cslot = 0xFFu, mslot = 0xFFu;
     if (r < n) {
         const Request q = decode_request(reqs[r]);
         const int64_t l_ttft = classes[q.cls * 3 + 0], l_e2e = classes[q.cls * 3 + 2];
-        const int64_t lim = l_ttft < 0 ? l_e2e : (l_e2e < 0 ? l_ttft : min(l_ttft, l_e2e));
-        const uint32_t lim32 = (lim < 0 || lim >= 0xFFFFFFFFll) ? 0xFFFFFFFFu : (uint32_t)lim;
-        base[kScanHdrUnits + t] = make_uint4((uint32_t)q.arrival, (uint32_t)((uint64_t)q.arrival >> 32), lim32,
-                                             q.model | (q.cls << 8));
+        const uint32_t t32 = (l_ttft < 0 || l_ttft >= 0xFFFFFFFFll) ? 0xFFFFFFFFu : (uint32_t)l_ttft;
+        const uint32_t e32 = (l_e2e < 0 || l_e2e >= 0xFFFFFFFFll) ? 0xFFFFFFFFu : (uint32_t)l_e2e;
+        const int64_t rel = q.arrival - base_arrival;
+        const uint32_t rel32 = rel >= 0xFFFFFFFFll ? 0xFFFFFFFFu : (uint32_t)rel;
+        base[kScanHdrUnits + t] = make_uint4(rel32, t32, e32, q.model | (q.cls << 8) | ((q.S - 1u) << 16));
+        const uint32_t lim32 = min(t32, e32);
         const int64_t v = lim32 == 0xFFFFFFFFu ? INT64_MAX : q.arrival + (int64_t)lim32;
-        atomicMax(reinterpret_cast<long long*>(&thr[q.cls < 7 ? q.cls : 7]), (long long)v);
+        cslot = q.cls < 7 ? q.cls : 7;
+        mslot = q.model < 7 ? q.model : 7;
+        atomicMax(reinterpret_cast<long long*>(&thr[cslot]), (long long)v);
+    }
+    uint32_t* const words = reinterpret_cast<uint32_t*>(base);
+    for (uint32_t k = 0; k < 8; k++) {
+        const uint32_t cb = __ballot_sync(0xFFFFFFFFu, cslot == k), mb = __ballot_sync(0xFFFFFFFFu, mslot == k);
+        if ((t & 31u) == 0) {
+            words[(kScanHdrClassBits + 2 * k) * 4 + (t >> 5)] = cb;
+            words[(kScanHdrModelBits + 2 * k) * 4 + (t >> 5)] = mb;
+        }
     }
     __syncthreads();
     if (t < 4) {
         const uint64_t a = (uint64_t)thr[2 * t], b = (uint64_t)thr[2 * t + 1];
         base[t] = make_uint4((uint32_t)a, (uint32_t)(a >> 32), (uint32_t)b, (uint32_t)(b >> 32));
     }
+    if (t == 4) base[kScanHdrBase] = make_uint4((uint32_t)base_arrival, (uint32_t)((uint64_t)base_arrival >> 32), 0u, 0u);
+    if (t >= 5 && t < 8) base[kScanHdrUnits - 3 + (t - 5)] = make_uint4(0u, 0u, 0u, 0u);  // padding units 37..39
 }
 size_t scan_trace_units(uint32_t n) {
     const size_t tiles = ((size_t)n + kScanTile - 1) / kScanTile;
