@@ -16,12 +16,19 @@ constexpr long long kWaitCycles = 4000000000ll;  // bound on any device-side wai
 // 0..5: lane groups of 1,2,4,8,16,32 lanes (one lane per instance)
 // 6..8: block layout with 2, 4, 8 warps, one warp per instance, state in registers
 // 9:    block layout with 16 warps striding over up to 128 instances, state in shared memory
-// With the thread mapping buckets 0..8 mean something else: how many lanes of a warp work on an
-// item (32, 24, 16, 12, 8, 6, 4, 2, 1: the larger the placements, the fewer fit the warp's pool).
-constexpr int kNumBuckets = 10;
+// 10..18: thread mapping, by how many lanes of a warp work at a time (32, 24, 16, 12, 8, 6, 4, 2, 1:
+//        the larger the placements, the fewer fit the warp's pools)
+constexpr int kNumBuckets = 19;
 constexpr int kGenericBlockBucket = 9;
+constexpr int kThreadBucket0 = 10;  // buckets 10..18: the thread mapping, by lanes per warp
 constexpr int kCostBins = 256;   // bin 0 = most expensive (largest total batch cap)
-constexpr int kCounterWords = 8192;  // counters | work counters | histograms + cursors, cleared per call
+constexpr int kCounterWords = 16384;  // counters | work counters | histograms + cursors, cleared per call
+// histogram sets (rows of kCostBins words in EvalParams::hist): candidates that can only go to a lane-group
+// or block bucket, only to a thread bucket, or either way (counted once per side); then the write cursors
+constexpr int kHistOnlyG = 0, kHistBothG = 10, kHistOnlyT = 20, kHistBothT = 29, kHistCursor = 38;
+constexpr int kHistRows = kHistCursor + kNumBuckets;
+// counters beside the bucket counts (EvalParams::bucket_count[0..31])
+constexpr int kCtrBoth = 24, kCtrLoaded = 25, kCtrCut = 26, kCtrUseThreads = 27;
 constexpr int kGroupThreads = 128;
 constexpr int kScanTile = 256;       // requests per scan tile of the thread mapping
 constexpr int kScanHdrUnits = 40;    // 16-byte units of a scan tile's header (see scan_trace_kernel)
@@ -255,16 +262,20 @@ struct EvalParams {
     uint32_t flags;
     uint32_t mapping;
     maaso_result* out;
-    uint32_t* bucket_count;  // [kNumBuckets]
+    uint32_t* bucket_count;  // [32]: candidates per bucket after planning, and the kCtr* counters
     uint32_t* bucket_list;   // [kNumBuckets][n_cand], each bucket sorted by decreasing cost estimate
-    uint32_t* work_ctr;      // [4]
-    uint32_t* hist;          // [2][kNumBuckets][kCostBins]: candidates per cost bin, then write cursors
-    uint32_t* code;          // [n_cand] bucket << 8 | cost bin, 0xFFFFFFFF for invalid candidates
+    uint32_t* work_ctr;      // [16]: next work item of the block kernels [1..4] and of the thread buckets [bucket - 10]... see the kernels
+    uint32_t* hist;          // [kHistRows][kCostBins]: candidates per cost bin by set, then write cursors
+    uint32_t* code;          // [n_cand] lane-group / block bucket << 8 | cost bin, 0xFFFFFFFF if none
+    uint32_t* code2;         // [n_cand] thread bucket << 8 | cost bin, 0xFFFFFFFF if none
+    uint32_t demand_tok_s;   // output tokens per second the trace(s) ask for
+    uint32_t thread_min_cand; // MAASO_MAP_AUTO: fewest loaded candidates for which the thread mapping is chosen
     uint32_t group_warps;    // warps the lane-group grid keeps resident (capacity for promotions)
     uint32_t* sm_ctr;        // [n_sm] next work item of each SM's share (lane-group kernel)
     uint32_t n_sm;
     uint32_t promote_pct;
-    uint32_t thread_pool_units;  // thread mapping: 16-byte units of shared memory one warp has for its placements
+    uint32_t thread_pool_units;  // thread mapping: 16-byte units one warp has for the cold part of its placements' state
+    uint32_t thread_hot_units;   // and for the hot part (3 units per instance, shared memory)
     long long wait_cycles;   // bound of every device-side wait
     uint32_t stall_test;     // test hook: never issue the trace copies
     int32_t* dump_row;       // [n_cand] or null

@@ -35,13 +35,10 @@
 namespace maaso {
 
 constexpr uint32_t kFullMaskT = 0xFFFFFFFFu;
-constexpr int kTStages = 2;
-constexpr int kTTile = kScanTile;               // requests per staged scan tile
-constexpr int kTStageUnits = kScanHdrUnits + kTTile + 4;  // header, records, padding for the 4-record look-ahead
+constexpr int kTTile = kScanTile;               // requests per scan tile
 constexpr uint32_t kTEndEmpty = 0x1FFFFFFu;    // end-index field of an empty key
 constexpr uint32_t kTRelMax = (1u << 25) - 2u; // largest end index a key can hold
 constexpr int kTQueue = 4;                     // queued completions per lane
-constexpr uint32_t kTFixedBytes = kTStages * kTStageUnits * 16 + kTQueue * 32 * (16 + 8 + 8) + 64;
 
 // Lanes that work on one item, by launch bucket (bucket 9 = placements the pool cannot hold at all).
 __host__ __device__ inline uint32_t thread_lanes_of(int bucket) {
@@ -76,20 +73,20 @@ struct TInst {
     uint32_t swn;   // step at the level right after one more admission (optimistic estimate)
 };
 
-__device__ __forceinline__ void t_load(const TPool& pl, uint32_t ru, uint32_t j, TInst& in) {
-    const uint4 a = *pl.unit(ru + 4u * j), b = *pl.unit(ru + 4u * j + 1u), c = *pl.unit(ru + 4u * j + 2u);
+__device__ __forceinline__ void t_load(const TPool& hp, uint32_t j, TInst& in) {
+    const uint4 a = *hp.unit(3u * j), b = *hp.unit(3u * j + 1u), c = *hp.unit(3u * j + 2u);
     in.T = (int64_t)(((uint64_t)a.y << 32) | a.x);
     in.tc = (int64_t)(((uint64_t)a.w << 32) | a.z);
     in.w = b.x & 0xFFu; in.B = (b.x >> 8) & 0xFFu; in.model = (b.x >> 16) & 0xFFu; in.row = b.x >> 24;
     in.sw = b.y; in.pre_base = b.z; in.pre_q16 = b.w;
     in.K = c.x; in.kmin = c.y; in.stepB = c.z; in.swn = c.w;
 }
-__device__ __forceinline__ void t_store(const TPool& pl, uint32_t ru, uint32_t j, const TInst& in) {
-    *pl.unit(ru + 4u * j) = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)in.tc,
+__device__ __forceinline__ void t_store(const TPool& hp, uint32_t j, const TInst& in) {
+    *hp.unit(3u * j) = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)in.tc,
                                                  (uint32_t)((uint64_t)in.tc >> 32));
-    *pl.unit(ru + 4u * j + 1u) =
+    *hp.unit(3u * j + 1u) =
         make_uint4(in.w | (in.B << 8) | (in.model << 16) | (in.row << 24), in.sw, in.pre_base, in.pre_q16);
-    *pl.unit(ru + 4u * j + 2u) = make_uint4(in.K, in.kmin, in.stepB, in.swn);
+    *hp.unit(3u * j + 2u) = make_uint4(in.K, in.kmin, in.stepB, in.swn);
 }
 
 struct TStats {
@@ -99,7 +96,8 @@ struct TStats {
 
 // What a thread needs besides the instance at hand.
 struct TEnv {
-    TPool pl;
+    TPool hp;             // hot part of the instances (3 units each: what a prediction reads), shared memory
+    TPool pl;             // cold part: one unit per instance (slot mask, offsets), then the slot keys; shared or global memory
     int64_t* qf;          // this lane's queue column: entry j at qf[j * 32] = finish time
     uint4* qa;            // entry j at qa[j * 32] = first-token time, arrival time
     uint2* qb;            // entry j at qb[j * 32] = request index, S | cls << 16 | instance << 24
@@ -110,7 +108,6 @@ struct TEnv {
     const EvalParams* P;
     int64_t oc;           // index of the candidate's record, negative for a lane without one
     uint32_t qn;          // completions waiting in the queue
-    uint32_t ru;          // units of the per-model instance ranges at the start of the lane's pool share
 };
 
 // Statistics of this lane's queued completions (Phi_S indicator, latency and throughput sums).
@@ -178,16 +175,16 @@ struct TKeys {
     uint32_t so;    // number of this instance's slot 0 among the lane's slots (scratch entries)
     uint64_t mask;  // occupied slots; bits at and above B are always set
 };
-__device__ __forceinline__ TKeys t_load_keys(const TPool& pl, uint32_t ru, uint32_t j) {
-    const uint4 d = *pl.unit(ru + 4u * j + 3u);
+__device__ __forceinline__ TKeys t_load_keys(const TPool& pl, uint32_t j) {
+    const uint4 d = *pl.unit(j);
     TKeys k;
     k.mask = ((uint64_t)d.y << 32) | d.x;
     k.ko = d.z & 0xFFFFu;
     k.so = d.z >> 16;
     return k;
 }
-__device__ __forceinline__ void t_store_mask(const TPool& pl, uint32_t ru, uint32_t j, uint64_t mask) {
-    *reinterpret_cast<uint2*>(pl.unit(ru + 4u * j + 3u)) = make_uint2((uint32_t)mask, (uint32_t)(mask >> 32));
+__device__ __forceinline__ void t_store_mask(const TPool& pl, uint32_t j, uint64_t mask) {
+    *reinterpret_cast<uint2*>(pl.unit(j)) = make_uint2((uint32_t)mask, (uint32_t)(mask >> 32));
 }
 
 // The counter has just reached the smallest end index (clock = in.T): retire every request that
@@ -225,7 +222,7 @@ __device__ __forceinline__ void t_retire(TInst& in, TKeys& ks, TEnv& e) {
 // "reduce" with events: run whole decode steps until the clock reaches `now` (drain: until the
 // instance is empty), retiring what completes on the way; the instance is written back.
 __device__ __forceinline__ void t_advance_events(TInst& in, uint32_t j, int64_t now, bool drain, TEnv& e) {
-    TKeys ks = t_load_keys(e.pl, e.ru, j);
+    TKeys ks = t_load_keys(e.pl, j);
     while (in.w > 0 && (drain || in.T < now)) {
         if (!drain && now <= in.tc - (int64_t)in.sw) {
             // the clock reaches `now` before anything completes (fewer steps than the longest request has tokens)
@@ -239,8 +236,8 @@ __device__ __forceinline__ void t_advance_events(TInst& in, uint32_t j, int64_t 
         t_retire(in, ks, e);
     }
     if (!drain && in.w == 0 && in.T < now) in.T = now;  // an idle instance starts at once
-    t_store(e.pl, e.ru, j, in);
-    t_store_mask(e.pl, e.ru, j, ks.mask);
+    t_store(e.hp, j, in);
+    t_store_mask(e.pl, j, ks.mask);
 }
 
 // All live end indices move down by the counter value K (which restarts at 0).  Rare.
@@ -265,10 +262,10 @@ __device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& 
     if (q.Sm1 == 0) {  // done at the end of its prefill, never occupies a slot
         in.tc += pre;
         t_push_now(e, in.T, pa, pb);
-        t_store(e.pl, e.ru, j, in);
+        t_store(e.hp, j, in);
         return;
     }
-    TKeys ks = t_load_keys(e.pl, e.ru, j);
+    TKeys ks = t_load_keys(e.pl, j);
     const uint32_t nblk = (in.B + 7u) >> 3;
     if (in.w == 0) in.K = 0;  // no live end index: the counter restarts
     if (in.K + q.Sm1 > kTRelMax) {
@@ -292,8 +289,8 @@ __device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& 
     in.sw = t_step(e, in.row, in.w);
     in.swn = t_step(e, in.row, min(in.w + 1u, in.B));
     in.tc = in.T + (int64_t)((in.kmin >> 7) - in.K) * (int64_t)in.sw;
-    t_store(e.pl, e.ru, j, in);
-    t_store_mask(e.pl, e.ru, j, ks.mask);
+    t_store(e.hp, j, in);
+    t_store_mask(e.pl, j, ks.mask);
 }
 
 // Per-request side outputs of a rejection (dump rows, per-model counts); rare.
@@ -306,90 +303,79 @@ __device__ __forceinline__ void t_reject_side(const EvalParams& P, uint32_t oc, 
 }
 
 struct ThreadSmem {
-    unsigned char* pool;
-    uint4* tiles;       // [kTStages][kTStageUnits] scan tiles: header, records
-    uint4* qa;          // [kTQueue][32]
+    unsigned char* hot;  // per lane: model ranges, one entry per model, the live map of the lane's current tile
+    uint4* qa;           // [kTQueue][32]
     uint2* qb;
     int64_t* qf;
-    uint64_t* full_bar; // [kTStages]
+    unsigned char* hpool; // hot part of the instances
+    unsigned char* pool;  // cold part (shared-memory mode)
 };
-__device__ __forceinline__ ThreadSmem t_carve(unsigned char* base, uint32_t pool_bytes) {
+__host__ __device__ inline uint32_t t_hot_units(uint32_t n_models) { return ((n_models + 7u) >> 3) + n_models + 2u; }
+__host__ __device__ inline size_t t_fixed_smem(uint32_t n_models) {
+    return (size_t)t_hot_units(n_models) * 512u + (size_t)kTQueue * 32 * (16 + 8 + 8);
+}
+__device__ __forceinline__ ThreadSmem t_carve(unsigned char* base, uint32_t n_models, uint32_t hot_bytes) {
     ThreadSmem s;
-    s.pool = base;
-    base += pool_bytes;
-    s.tiles = reinterpret_cast<uint4*>(base);
-    base += (size_t)kTStages * kTStageUnits * 16;
+    s.hot = base;
+    base += (size_t)t_hot_units(n_models) * 512u;
     s.qa = reinterpret_cast<uint4*>(base);
     base += (size_t)kTQueue * 32 * 16;
     s.qb = reinterpret_cast<uint2*>(base);
     base += (size_t)kTQueue * 32 * 8;
     s.qf = reinterpret_cast<int64_t*>(base);
     base += (size_t)kTQueue * 32 * 8;
-    s.full_bar = reinterpret_cast<uint64_t*>(base);
+    s.hpool = base;
+    base += hot_bytes;
+    s.pool = base;
     return s;
 }
 
-__device__ __forceinline__ void t_issue_tile(const ThreadSmem& sm, const uint4* scan, uint32_t n_req, uint32_t stage,
-                                             uint32_t tile) {
-    const uint32_t recs = min((uint32_t)kTTile, n_req - tile * kTTile);
-    const uint32_t bytes = (recs + kScanHdrUnits) * 16u;
-    mbar_expect_tx(&sm.full_bar[stage], bytes);
-    bulk_load(sm.tiles + (size_t)stage * kTStageUnits, scan + (size_t)tile * (kScanTile + kScanHdrUnits), bytes,
-              &sm.full_bar[stage]);
-}
-
 __device__ __forceinline__ uint4 ldg_nc(const uint4* p) { return __ldg(p); }
+__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+
+enum : uint32_t { kLaneIdle = 0, kLaneScan = 1, kLaneWait = 2, kLaneDone = 3 };
 
 // OPT: the distributor predicts with the step time right after admission (optimistic estimate);
 // a wait is then followed by a new choice.  Under the worst-case estimate the choice after a
 // wait is known beforehand (same argument as in the lane-group kernel) and is only counted.
 //
-// How a warp walks a tile.  Most requests of a loaded placement are rejected for a reason that
-// needs no look at any instance: the placement has no instance of the model, or the
-// dispatcher's clock has already passed the request's first-token or end-to-end deadline
-// (every predicted first token lies at or after `now`).  Such a request costs its lane one
-// 16-byte scan record and a compare, and touches no instance (their clocks catch up lazily).
-// The lanes therefore run through the tile independently, each at its own request index;
-// a lane that meets a request which needs the distributor stops there, fetches the request's
-// full record, and waits.  Once `theta` lanes wait (or nobody can go on), the waiting lanes
-// handle their requests together, each its own.  Nothing is counted per request on the way:
-// a placement's request count and the checksum of "all of them rejected" come from per-class
-// totals of the trace, and an admission takes its request out again.
+// How a lane walks its trace.  Most requests of a loaded placement are rejected for a reason that
+// needs no look at the instances' state: the placement has no instance of the model, or the
+// dispatcher's clock (and the earliest time any instance of the model could start a prefill) has
+// passed the request's first-token or end-to-end deadline.  The trace is therefore kept as scan
+// tiles (prep.cu): 256 requests with, per class, the latest deadline in the tile and a bit map of
+// the class's requests, and per model a bit map.  A lane entering a tile builds its live map:
+// requests of classes that are not late as a whole and of models the placement serves.  A tile
+// without live requests costs five loads; a live request costs a 16-byte record and a compare
+// against the model's lower bound; only what survives goes to the distributor.  Nothing is counted
+// per request on the way: a placement's request count and the checksum of "all of them rejected"
+// come from per-class totals of the trace, and an admission takes its request out again.
+//
+// The lanes of a warp are independent: each has its own placement and its own position in the
+// trace, and takes the next placement of the bucket when it is through.  What they share is the
+// instruction stream, so the warp alternates between scan iterations (for the lanes that can go
+// on) and distributor rounds (for the lanes that stand at a request which needs one), and starts a
+// round when `theta` lanes wait or nobody can scan.
 template <bool OPT>
 __global__ void __launch_bounds__(32, 1)
-eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_bytes, const uint32_t theta,
-                   unsigned char* const arena) {
-    // arena: the placements' state lives in global memory (one region of pool_bytes per warp, kept hot by
+eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_bytes, const uint32_t hot_bytes,
+                   const uint32_t theta, unsigned char* const arena) {
+    // arena: the instances' state lives in global memory (one region of pool_bytes per warp, kept hot by
     // L1/L2) instead of shared memory, which leaves room for many more resident warps; null = shared memory
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    ThreadSmem sm = t_carve(smem_raw, arena ? 0u : pool_bytes);
-    if (arena) sm.pool = arena + (size_t)blockIdx.x * pool_bytes;
+    const ThreadSmem sm = t_carve(smem_raw, P.n_models, hot_bytes);
+    unsigned char* const pool = arena ? arena + (size_t)blockIdx.x * pool_bytes : sm.pool;
     const uint32_t lane = threadIdx.x;
-    if (lane == 0) {
-        for (int s = 0; s < kTStages; s++) mbar_init(&sm.full_bar[s], 1);
-        fence_barrier_init();
-    }
-    __syncwarp();
+    if (P.stall_test) return;  // test hook: nothing is scored, every valid candidate keeps its "not scored" mark
 
     const uint32_t pool_units = pool_bytes / 16u;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
     const uint32_t n_traces = P.n_traces > 1 ? P.n_traces : 1u;
-    // a lane's share of the pool: units [0, rr) per-model instance ranges, [rr, rr + M) one entry per model
-    // (lower bound of any predicted first token, smallest prefill base, smallest prediction step),
-    // 2 units for the live map of the current tile, then the instances from unit ru on
+    // a lane's hot units: [0, rr) per-model instance ranges, [rr, rr + M) one entry per model (lower bound
+    // of any predicted first token, smallest prefill base, smallest prediction step), then the live map
     const uint32_t rr = (P.n_models + 7u) >> 3;
-    const uint32_t ru = rr + P.n_models + 2u;
-    // items per bucket, buckets with the fewest lanes (the largest placements) first
-    uint32_t items[9];
-    uint32_t total_items = 0;
-    for (int b = 8; b >= 0; b--) {
-        const uint32_t L = thread_lanes_of(b);
-        items[b] = (P.bucket_count[b] + L - 1u) / L;
-        total_items += items[b];
-    }
-    const uint32_t total_all = total_items * n_traces;
-    uint32_t tile_seq = 0;  // tiles this warp has consumed so far (stage and parity of the next one)
-    bool dead = false;      // a bounded wait ran out: take no more work
+    const uint32_t lm = rr + P.n_models;  // first unit of the live map
+    const TPool hot{sm.hot + lane * 16u, 512u};
 
     TStats ls;
     TEnv e;
@@ -399,371 +385,406 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
     e.rows = P.rows;
     e.ls = &ls;
     e.P = &P;
+    e.qn = 0;
+    e.oc = -1;
 
-    while (!dead) {
-        uint32_t wi = 0;
-        if (lane == 0) wi = atomicAdd(&P.work_ctr[0], 1u);
-        wi = __shfl_sync(kFullMaskT, wi, 0);
-        if (wi >= total_all) break;
-        const uint32_t tr = wi % n_traces;
-        wi /= n_traces;
-        const uint4* const cooked = P.trace_cooked[tr];
-        const uint4* const scan = P.trace_scan[tr];
-        const uint32_t n_req = P.trace_n[tr];
-        const uint32_t n_tiles = (n_req + kTTile - 1) / kTTile;
-        const uint32_t out_base = tr * P.n_cand;
-        int b = 8;
-        while (wi >= items[b]) { wi -= items[b]; b--; }
+    // buckets with the fewest lanes per warp (the largest placements) first
+    for (int b = 8; b >= 0; b--) {
         const uint32_t L = thread_lanes_of(b);
-        const uint32_t cnt = P.bucket_count[b];
-        const uint32_t pos = wi * L + lane;
-        const bool valid = lane < L && pos < cnt;
-        const uint32_t cand = valid ? P.bucket_list[(size_t)b * P.n_cand + pos] : 0u;
-        const uint32_t cap_units = pool_units / L;  // what one lane of this item may use
-
-        e.pl.base = sm.pool + lane * 16u;
+        const uint32_t cnt = P.bucket_count[kThreadBucket0 + b];
+        const uint64_t total = (uint64_t)cnt * n_traces;
+        if (total == 0 || *(volatile uint32_t*)&P.work_ctr[5 + b] >= total) continue;
+        const uint32_t cap_units = pool_units / L;  // what one lane may use
+        const uint32_t hot_cap = hot_bytes / 16u / L;
+        e.pl.base = pool + lane * 16u;
         e.pl.stride = L * 16u;
-        e.ru = ru;
-        // scratch entries of this lane: two per slot, at most 4 slots per pool unit
-        {
+        e.hp.base = sm.hpool + lane * 16u;
+        e.hp.stride = L * 16u;
+        {   // scratch entries of this lane: two per slot, at most 4 slots per pool unit
             unsigned char* const wbase = reinterpret_cast<unsigned char*>(P.payload) + (size_t)blockIdx.x * pool_units * 8u * 24u;
             e.pay_a = reinterpret_cast<uint4*>(wbase) + (size_t)lane * cap_units * 8u;
             e.pay_b = reinterpret_cast<uint2*>(wbase + (size_t)pool_units * 8u * 16u) + (size_t)lane * cap_units * 8u;
         }
-        e.oc = valid ? (int64_t)(out_base + cand) : -1;
-        e.qn = 0;
-        ls.st.clear();
-        for (int i = 0; i < 8; i++) ls.hbc[i] = 0;
+        bool open = lane < L;         // this lane may still find a placement in the bucket
+        uint32_t state = kLaneIdle;
+        // the lane's placement and where it stands
+        uint32_t cand = 0, n_i = 0, status = 0, hasmodel = 0, cmask = 0, hmask = 0, mmask = 0, n_counted = 0;
+        uint32_t n_req = 0, pos = 0, cur_tile = 0xFFFFFFFFu, out_base = 0;
+        const uint4* cooked = nullptr;
+        const uint4* scan = nullptr;
+        uint64_t rej_sum = 0, extra = 0;
+        int64_t now = 0, tile_base = 0;
+        bool side = false;
 
-        // ---- set up this lane's instances -----------------------------------------------------
-        uint32_t n_i = 0, status = 0;
-        uint32_t hasmodel = 0;  // models the placement has an instance of
-        if (valid) {
-            const uint32_t lo = P.offsets[cand];
-            n_i = P.offsets[cand + 1] - lo;
-            uint32_t rng_lo[MAASO_MAX_MODELS], rng_hi[MAASO_MAX_MODELS], min_pre[MAASO_MAX_MODELS], min_step[MAASO_MAX_MODELS];
-            for (int m = 0; m < MAASO_MAX_MODELS; m++) { rng_lo[m] = 0xFFu; rng_hi[m] = 0u; min_pre[m] = 0xFFFFFFFFu; min_step[m] = 0xFFFFFFFFu; }
-            uint32_t ko = ru + 4u * n_i, so = 0;
-            for (uint32_t j = 0; j < n_i; j++) {
-                const uint32_t word = P.inst[lo + j];
-                const uint32_t m = word & 0xFu, B = (word >> 12) & 0xFFu;
-                const uint32_t row = m * P.n_strategies + ((word >> 4) & 0xFFu);
-                const uint32_t nblk = (B + 7u) >> 3;
-                TInst in;
-                in.T = 0; in.tc = 0; in.w = 0; in.B = B; in.model = m; in.row = row; in.sw = 1;
-                in.pre_base = (uint32_t)P.rows[row * kRowStride + 0];
-                in.pre_q16 = (uint32_t)P.rows[row * kRowStride + 1];
-                in.K = 0; in.kmin = 0xFFFFFFFFu;
-                in.stepB = (uint32_t)P.rows[row * kRowStride + 1 + B];
-                in.swn = (uint32_t)P.rows[row * kRowStride + 2];
-                if (ko + 2u * nblk + 2u > cap_units) { status = MAASO_CAND_ETIMEOUT; break; }  // cannot happen: sized by the validation kernel
-                t_store(e.pl, ru, j, in);
-                const uint64_t mask = B >= 64u ? 0ull : (~0ull << B);
-                *e.pl.unit(ru + 4u * j + 3u) = make_uint4((uint32_t)mask, (uint32_t)(mask >> 32), ko | (so << 16), 0u);
-                for (uint32_t u = 0; u < 2u * nblk; u++) {
-                    const uint32_t s0 = (kTEndEmpty << 7) | (4u * u);
-                    *e.pl.unit(ko + u) = make_uint4(s0, s0 + 1u, s0 + 2u, s0 + 3u);
-                }
-                const uint4 ones = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
-                *e.pl.unit(ko + 2u * nblk) = ones;
-                *e.pl.unit(ko + 2u * nblk + 1u) = ones;
-                ko += 2u * nblk + 2u;
-                so += 8u * nblk;
-                rng_lo[m] = min(rng_lo[m], j);
-                rng_hi[m] = j + 1u;
-                hasmodel |= 1u << m;
-                // the smallest step a prediction for this model can use: the step at the batch cap, or
-                // (optimistic estimate) at any level up to it
-                uint32_t ms = in.stepB;
-                if (OPT)
-                    for (uint32_t w = 1; w < B; w++) ms = min(ms, (uint32_t)P.rows[row * kRowStride + 1 + w]);
-                min_step[m] = min(min_step[m], ms);
-                min_pre[m] = min(min_pre[m], in.pre_base);
-            }
-            // per-model instance ranges: halfword m = first index | (last index + 1) << 8
-            for (uint32_t u = 0; u < rr; u++) {
-                uint32_t rw[4];
-                for (int i = 0; i < 4; i++) {
-                    const uint32_t m0 = 8u * u + 2u * i, m1 = m0 + 1u;
-                    const uint32_t a = rng_lo[m0] >= rng_hi[m0] ? 0u : (rng_lo[m0] | (rng_hi[m0] << 8));
-                    const uint32_t c = rng_lo[m1] >= rng_hi[m1] ? 0u : (rng_lo[m1] | (rng_hi[m1] << 8));
-                    rw[i] = a | (c << 16);
-                }
-                *e.pl.unit(u) = make_uint4(rw[0], rw[1], rw[2], rw[3]);
-            }
-            // nothing runs yet: every predicted first token lies at or after the smallest prefill base
-            for (uint32_t m = 0; m < P.n_models; m++) *e.pl.unit(rr + m) = make_uint4(min_pre[m], 0u, min_pre[m], min_step[m]);
-        }
-        const uint32_t cmask = (valid && use_mask) ? P.class_mask[cand] : 0xFFFFFFFFu;
-        // header entries of a scan tile this lane has to look at (classes 7 and up share entry 7)
-        const uint32_t hmask = (cmask & 0x7Fu) | ((cmask >> 7) ? 0x80u : 0u);
-        const uint32_t mmask = (hasmodel & 0x7Fu) | ((hasmodel >> 7) ? 0x80u : 0u);  // the same for the per-model maps
-        bool side = P.rej_by_model != nullptr;
-        if (valid && P.dump_row) side = side || P.dump_row[cand] >= 0;
-        // every request of the subset counted as rejected; admissions take theirs out
-        uint32_t n_counted = 0;
-        uint64_t rej_sum = 0;
-        if (valid) {
-            const uint64_t* ct = P.trace_class_tot[tr];
-            for (uint32_t c = 0; c < P.n_classes; c++)
-                if (!use_mask || ((cmask >> c) & 1u)) {
-                    n_counted += (uint32_t)ct[2u * c];
-                    rej_sum += ct[2u * c + 1u];
-                }
-        }
-        int64_t now = 0;
-        uint64_t extra = 0;  // distributor rounds beyond the first of a request
-        __syncwarp();
-
-        // ---- trace staging: first tiles of this item --------------------------------------------
-        if (lane == 0 && !P.stall_test) {
-            for (uint32_t s = 0; s < (uint32_t)kTStages && s < n_tiles; s++)
-                t_issue_tile(sm, scan, n_req, (tile_seq + s) % kTStages, s);
-        }
-        uint32_t in_flight = min((uint32_t)kTStages, n_tiles);
-
-        for (uint32_t t = 0; t < n_tiles; t++) {
-            const uint32_t s = tile_seq % kTStages, parity = (tile_seq / kTStages) & 1u;
-            const bool arrived = mbar_wait_bounded(&sm.full_bar[s], parity, P.wait_cycles);
-            if (!__all_sync(kFullMaskT, arrived)) {
-                // give up: wait (bounded) for every copy still in flight, then stop taking work
-                if (!P.stall_test)
-                    for (uint32_t x = 0; x < in_flight; x++) {
-                        const uint32_t ts = tile_seq + x;
-                        mbar_wait_bounded(&sm.full_bar[ts % kTStages], (ts / kTStages) & 1u, P.wait_cycles);
-                    }
-                status = MAASO_CAND_ETIMEOUT;
-                dead = true;
-                break;
-            }
-            in_flight--;
-            const uint4* const tile = sm.tiles + (size_t)s * kTStageUnits;
-            const uint4* const rp = tile + kScanHdrUnits;  // the tile's scan records
-            const uint32_t recs = min((uint32_t)kTTile, n_req - t * kTTile);
-            uint32_t ri = (valid && status == 0) ? 0u : recs;
-            // The tile's live map of this lane: requests of a class that is not late as a whole (the
-            // dispatcher's clock has not passed the class's header entry) and of a model the placement
-            // has an instance of.  Everything else in the tile is rejected without being looked at.
-            if (ri < recs) {
-                uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
-                if (side) {
-                    lo = hi = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);  // every rejection is written out
+        for (;;) {
+            // ---- lanes without a placement take the next one of the bucket --------------------------------
+            if (open && state == kLaneIdle) {
+                const uint64_t idx = atomicAdd(&P.work_ctr[5 + b], 1u);
+                if (idx >= total) {
+                    open = false;
                 } else {
-                    uint4 mlo = lo, mhi = lo;
-#pragma unroll
-                    for (int k = 0; k < 8; k++) {
-                        const uint4 h = tile[k >> 1];
-                        const int64_t thr = (k & 1) ? (int64_t)(((uint64_t)h.w << 32) | h.z) : (int64_t)(((uint64_t)h.y << 32) | h.x);
-                        if (((hmask >> k) & 1u) && thr >= now) {
-                            const uint4 a = tile[kScanHdrClassBits + 2 * k], c = tile[kScanHdrClassBits + 2 * k + 1];
-                            lo.x |= a.x; lo.y |= a.y; lo.z |= a.z; lo.w |= a.w;
-                            hi.x |= c.x; hi.y |= c.y; hi.z |= c.z; hi.w |= c.w;
-                        }
-                        if ((mmask >> k) & 1u) {
-                            const uint4 a = tile[kScanHdrModelBits + 2 * k], c = tile[kScanHdrModelBits + 2 * k + 1];
-                            mlo.x |= a.x; mlo.y |= a.y; mlo.z |= a.z; mlo.w |= a.w;
-                            mhi.x |= c.x; mhi.y |= c.y; mhi.z |= c.z; mhi.w |= c.w;
-                        }
-                    }
-                    lo.x &= mlo.x; lo.y &= mlo.y; lo.z &= mlo.z; lo.w &= mlo.w;
-                    hi.x &= mhi.x; hi.y &= mhi.y; hi.z &= mhi.z; hi.w &= mhi.w;
-                }
-                *e.pl.unit(rr + P.n_models) = lo;
-                *e.pl.unit(rr + P.n_models + 1u) = hi;
-                if ((lo.x | lo.y | lo.z | lo.w | hi.x | hi.y | hi.z | hi.w) == 0u) ri = recs;
-            }
-            const int64_t tile_base = (int64_t)(((uint64_t)tile[kScanHdrBase].y << 32) | tile[kScanHdrBase].x);
-            bool waiting = false;  // this lane stands at a request that needs the distributor
-            uint4 f0, f1, f2;      // that request's full record
-            f0 = f1 = f2 = make_uint4(0u, 0u, 0u, 0u);
-            for (;;) {
-                uint32_t wl;
-                for (;;) {
-#pragma unroll 1
-                    for (int c = 0; c < 8; c++) {
-                        if (waiting || ri >= recs) continue;
-                        // the next live request at or after ri
-                        const uint32_t bits = *e.pl.word(rr + P.n_models + (ri >> 7), (ri >> 5) & 3u) >> (ri & 31u);
-                        if (bits == 0u) { ri = min((ri | 31u) + 1u, recs); continue; }
-                        ri += (uint32_t)__ffs((int)bits) - 1u;
-                        if (ri >= recs) { ri = recs; continue; }
-                        const uint4 sr = rp[ri];
-                        const uint32_t model = sr.w & 0xFFu;
-                        if (!((cmask >> ((sr.w >> 8) & 31u)) & 1u)) { ri++; continue; }  // not in the request subset
-                        bool real = ((hasmodel >> model) & 1u) != 0u;
-                        if (real && sr.x != 0xFFFFFFFFu) {
-                            // Too late whatever the instance?  Every predicted first token of this model lies at
-                            // or after flb: the dispatcher's clock plus the smallest prefill base, and the lower
-                            // bound kept from the latest look at the model's instances (times only move forward).
-                            const uint4 me = *e.pl.unit(rr + model);
-                            const int64_t arrival = tile_base + (int64_t)sr.x;
-                            const int64_t flb = max(max(now, arrival) + (int64_t)me.z, (int64_t)(((uint64_t)me.y << 32) | me.x));
-                            const bool late_first = sr.y != 0xFFFFFFFFu && arrival + (int64_t)sr.y < flb;
-                            const bool late_end = sr.z != 0xFFFFFFFFu &&
-                                                  arrival + (int64_t)sr.z < flb + (int64_t)((uint64_t)(sr.w >> 16) * me.w);
-                            real = !(late_first || late_end);
-                        }
-                        if (real) {
-                            waiting = true;
-                            const uint4* full = cooked + (size_t)(t * kTTile + ri) * kCookedWords;
-                            f0 = ldg_nc(full); f1 = ldg_nc(full + 1); f2 = ldg_nc(full + 2);
-                        } else {
-                            // overflow protection, the plain case: nobody can meet the deadline -> rejected
-                            if (side) t_reject_side(P, out_base + cand, t * kTTile + ri, model);
-                            ri++;
-                        }
-                    }
-                    wl = __ballot_sync(kFullMaskT, waiting);
-                    const uint32_t act = __ballot_sync(kFullMaskT, !waiting && ri < recs);
-                    if (act == 0u || (uint32_t)__popc(wl) >= theta) break;
-                }
-                if (wl == 0u) break;  // everybody is through the tile
-                // statistics of completed requests, all lanes together
-                if (__any_sync(kFullMaskT, e.qn >= 3u)) t_flush_now(e);
-                if (!waiting) continue;
-                waiting = false;
-                const CookedReq q = decode_cooked(f0, f1, f2);
-                const uint32_t req = t * kTTile + ri;
-                ri++;
-                now = max(now, q.arrival);  // pending time: the dispatcher never goes back
-                // instances of the request's model
-                const uint4 rg = *e.pl.unit(q.model >> 3);
-                const uint32_t rgw = (q.model & 4u) ? ((q.model & 2u) ? rg.w : rg.z) : ((q.model & 2u) ? rg.y : rg.x);
-                const uint32_t rh = (q.model & 1u) ? (rgw >> 16) : (rgw & 0xFFFFu);
-                const uint32_t j_lo = rh & 0xFFu, j_hi = rh >> 8;
-                bool pending = true;
-                uint32_t tries = 0;
-                do {
-                    tries++;
-                    uint64_t best = kKeyInf;
-                    uint32_t bj = 0, bk = 0;
-                    int64_t bT = 0, bpre = 0;
-                    // smallest and second smallest (start time + prefill base) over the model's instances
-                    int64_t lb1 = INT64_MAX, lb2 = INT64_MAX;
-                    uint32_t lb1j = 0xFFFFFFFFu;
-                    for (uint32_t j = j_lo; j < j_hi; j++) {
+                    const uint32_t tr = (uint32_t)(idx % n_traces);
+                    cand = P.bucket_list[(size_t)(kThreadBucket0 + b) * P.n_cand + (uint32_t)(idx / n_traces)];
+                    cooked = P.trace_cooked[tr];
+                    scan = P.trace_scan[tr];
+                    n_req = P.trace_n[tr];
+                    out_base = tr * P.n_cand;
+                    e.oc = (int64_t)(out_base + cand);
+                    e.qn = 0;
+                    ls.st.clear();
+                    for (int i = 0; i < 8; i++) ls.hbc[i] = 0;
+                    status = 0;
+                    hasmodel = 0;
+                    const uint32_t lo = P.offsets[cand];
+                    n_i = P.offsets[cand + 1] - lo;
+                    uint32_t rng_lo[MAASO_MAX_MODELS], rng_hi[MAASO_MAX_MODELS], min_pre[MAASO_MAX_MODELS], min_step[MAASO_MAX_MODELS];
+                    for (int m = 0; m < MAASO_MAX_MODELS; m++) { rng_lo[m] = 0xFFu; rng_hi[m] = 0u; min_pre[m] = 0xFFFFFFFFu; min_step[m] = 0xFFFFFFFFu; }
+                    uint32_t ko = n_i, so = 0;  // cold units: one per instance, then the key blocks
+                    for (uint32_t j = 0; j < n_i; j++) {
+                        const uint32_t word = P.inst[lo + j];
+                        const uint32_t m = word & 0xFu, B = (word >> 12) & 0xFFu;
+                        const uint32_t row = m * P.n_strategies + ((word >> 4) & 0xFFu);
+                        const uint32_t nblk = (B + 7u) >> 3;
                         TInst in;
-                        t_load(e.pl, ru, j, in);
-                        if (in.model != q.model) continue;
-                        // "reduce": where the instance's clock stands once it has reached `now`
-                        int64_t T = in.T;
-                        uint32_t kadd = 0;
-                        if (in.w > 0) {
-                            if (T < now) {
-                                if (now > in.tc - (int64_t)in.sw) {  // something completes on the way
-                                    t_advance_events(in, j, now, false, e);
-                                    T = in.T;
-                                } else if (in.w < in.B) {
-                                    kadd = ceil_div_small(now - T, in.sw, rcp_approx((float)in.sw));
-                                    T += (int64_t)kadd * (int64_t)in.sw;
+                        in.T = 0; in.tc = 0; in.w = 0; in.B = B; in.model = m; in.row = row; in.sw = 1;
+                        in.pre_base = (uint32_t)P.rows[row * kRowStride + 0];
+                        in.pre_q16 = (uint32_t)P.rows[row * kRowStride + 1];
+                        in.K = 0; in.kmin = 0xFFFFFFFFu;
+                        in.stepB = (uint32_t)P.rows[row * kRowStride + 1 + B];
+                        in.swn = (uint32_t)P.rows[row * kRowStride + 2];
+                        if (ko + 2u * nblk + 2u > cap_units || 3u * (j + 1u) > hot_cap) { status = MAASO_CAND_ETIMEOUT; break; }  // cannot happen: sized by the validation kernel
+                        t_store(e.hp, j, in);
+                        const uint64_t mask = B >= 64u ? 0ull : (~0ull << B);
+                        *e.pl.unit(j) = make_uint4((uint32_t)mask, (uint32_t)(mask >> 32), ko | (so << 16), 0u);
+                        for (uint32_t u = 0; u < 2u * nblk; u++) {
+                            const uint32_t s0 = (kTEndEmpty << 7) | (4u * u);
+                            *e.pl.unit(ko + u) = make_uint4(s0, s0 + 1u, s0 + 2u, s0 + 3u);
+                        }
+                        const uint4 ones = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+                        *e.pl.unit(ko + 2u * nblk) = ones;
+                        *e.pl.unit(ko + 2u * nblk + 1u) = ones;
+                        ko += 2u * nblk + 2u;
+                        so += 8u * nblk;
+                        rng_lo[m] = min(rng_lo[m], j);
+                        rng_hi[m] = j + 1u;
+                        hasmodel |= 1u << m;
+                        // the smallest step a prediction for this model can use: the step at the batch cap, or
+                        // (optimistic estimate) at any level up to it
+                        uint32_t ms = in.stepB;
+                        if (OPT)
+                            for (uint32_t w = 1; w < B; w++) ms = min(ms, (uint32_t)P.rows[row * kRowStride + 1 + w]);
+                        min_step[m] = min(min_step[m], ms);
+                        min_pre[m] = min(min_pre[m], in.pre_base);
+                    }
+                    // per-model instance ranges: halfword m = first index | (last index + 1) << 8
+                    for (uint32_t u = 0; u < rr; u++) {
+                        uint32_t rw[4];
+                        for (int i = 0; i < 4; i++) {
+                            const uint32_t m0 = 8u * u + 2u * i, m1 = m0 + 1u;
+                            const uint32_t a = rng_lo[m0] >= rng_hi[m0] ? 0u : (rng_lo[m0] | (rng_hi[m0] << 8));
+                            const uint32_t c = rng_lo[m1] >= rng_hi[m1] ? 0u : (rng_lo[m1] | (rng_hi[m1] << 8));
+                            rw[i] = a | (c << 16);
+                        }
+                        *hot.unit(u) = make_uint4(rw[0], rw[1], rw[2], rw[3]);
+                    }
+                    // nothing runs yet: every predicted first token lies at or after the smallest prefill base
+                    for (uint32_t m = 0; m < P.n_models; m++) *hot.unit(rr + m) = make_uint4(min_pre[m], 0u, min_pre[m], min_step[m]);
+                    cmask = use_mask ? P.class_mask[cand] : 0xFFFFFFFFu;
+                    // header entries of a scan tile this lane has to look at (classes 7 and up share entry 7)
+                    hmask = (cmask & 0x7Fu) | ((cmask >> 7) ? 0x80u : 0u);
+                    mmask = (hasmodel & 0x7Fu) | ((hasmodel >> 7) ? 0x80u : 0u);  // the same for the per-model maps
+                    side = P.rej_by_model != nullptr;
+                    if (P.dump_row) side = side || P.dump_row[cand] >= 0;
+                    // every request of the subset counted as rejected; admissions take theirs out
+                    n_counted = 0;
+                    rej_sum = 0;
+                    const uint64_t* ct = P.trace_class_tot[tr];
+                    for (uint32_t c = 0; c < P.n_classes; c++)
+                        if (!use_mask || ((cmask >> c) & 1u)) {
+                            n_counted += (uint32_t)ct[2u * c];
+                            rej_sum += ct[2u * c + 1u];
+                        }
+                    now = 0;
+                    extra = 0;
+                    pos = 0;
+                    cur_tile = 0xFFFFFFFFu;
+                    state = (status == 0 && n_req > 0) ? kLaneScan : kLaneDone;
+                }
+            }
+            if (!__any_sync(kFullMaskT, state != kLaneIdle)) break;  // the bucket is done as far as this warp goes
+
+            // ---- scan iterations -------------------------------------------------------------------------------
+#pragma unroll 1
+            for (int c = 0; c < 4; c++) {
+                if (state != kLaneScan) continue;
+                const uint32_t tile = pos / (uint32_t)kTTile;
+                const uint4* const th = scan + (size_t)tile * (kScanTile + kScanHdrUnits);
+                const uint32_t recs = min((uint32_t)kTTile, n_req - tile * kTTile);
+                if (tile != cur_tile) {
+                    // A new tile: its live map for this lane = requests of a class that is not late as a whole
+                    // (the dispatcher's clock has not passed the class's header entry) and of a model the
+                    // placement has an instance of.  Everything else in the tile is rejected without a look.
+                    cur_tile = tile;
+                    uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo, hb = lo;
+                    if (side) {
+                        lo = hi = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);  // every rejection is written out
+                        hb = ldg_nc(th + kScanHdrBase);
+                    } else {
+                        // first the eight class entries: most tiles of a loaded placement end here, wholly late
+                        const uint4 h0 = ldg_nc(th), h1 = ldg_nc(th + 1), h2 = ldg_nc(th + 2), h3 = ldg_nc(th + 3);
+                        const uint32_t hw[16] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w, h2.x, h2.y, h2.z, h2.w, h3.x, h3.y, h3.z, h3.w};
+                        uint32_t livec = 0;
+#pragma unroll
+                        for (int k = 0; k < 8; k++) {
+                            const int64_t thr = (int64_t)(((uint64_t)hw[2 * k + 1] << 32) | hw[2 * k]);
+                            if (((hmask >> k) & 1u) && thr >= now) livec |= 1u << k;
+                        }
+                        if (livec) {
+                            hb = ldg_nc(th + kScanHdrBase);
+                            uint4 mlo = lo, mhi = lo;
+#pragma unroll 1
+                            for (uint32_t k = 0; k < 8u; k++) {
+                                if ((livec >> k) & 1u) {
+                                    const uint4 a = ldg_nc(th + kScanHdrClassBits + 2u * k), x = ldg_nc(th + kScanHdrClassBits + 2u * k + 1u);
+                                    lo.x |= a.x; lo.y |= a.y; lo.z |= a.z; lo.w |= a.w;
+                                    hi.x |= x.x; hi.y |= x.y; hi.z |= x.z; hi.w |= x.w;
+                                }
+                                if ((mmask >> k) & 1u) {
+                                    const uint4 a = ldg_nc(th + kScanHdrModelBits + 2u * k), x = ldg_nc(th + kScanHdrModelBits + 2u * k + 1u);
+                                    mlo.x |= a.x; mlo.y |= a.y; mlo.z |= a.z; mlo.w |= a.w;
+                                    mhi.x |= x.x; mhi.y |= x.y; mhi.z |= x.z; mhi.w |= x.w;
                                 }
                             }
-                        } else if (T < now) {
-                            T = now;
+                            lo.x &= mlo.x; lo.y &= mlo.y; lo.z &= mlo.z; lo.w &= mlo.w;
+                            hi.x &= mhi.x; hi.y &= mhi.y; hi.z &= mhi.z; hi.w &= mhi.w;
                         }
-                        // distributor prediction (Sec. IV-F steps 2-3)
-                        const int64_t pre = prefill_us(in.pre_base, in.pre_q16, q.in_tokens);
-                        const bool free_slot = in.w < in.B;
-                        const int64_t t0 = free_slot ? T : in.tc;
-                        const uint32_t sB = (OPT && free_slot) ? in.swn : in.stepB;
-                        const int64_t first = t0 + pre;
-                        const int64_t fin = first + (int64_t)((uint64_t)q.Sm1 * sB);
-                        {
-                            const int64_t lb = t0 + (int64_t)in.pre_base;
-                            if (lb < lb1) { lb2 = lb1; lb1 = lb; lb1j = j; }
-                            else if (lb < lb2) lb2 = lb;
-                        }
-                        const bool ok = first <= q.dl_ttft && (q.Sm1 == 0 || sB <= q.tbt32) && fin <= q.dl_e2e;
-                        const uint64_t key = ((uint64_t)(free_slot ? 0u : 1u) << 63) | (uint64_t)first;
-                        if (ok && key < best) { best = key; bj = j; bk = kadd; bT = T; bpre = pre; }
                     }
-                    int64_t lb_new = lb1;  // the model's lower bound as this look at its instances leaves it
-                    if (best == kKeyInf) {
-                        // overflow protection: nobody can meet the deadline -> rejected
-                        if (side) t_reject_side(P, out_base + cand, req, q.model);
-                        pending = false;
+                    if ((lo.x | lo.y | lo.z | lo.w | hi.x | hi.y | hi.z | hi.w) == 0u) {
+                        pos = tile * kTTile + recs;  // nothing to look at in this tile
                     } else {
-                        TInst in;
-                        t_load(e.pl, ru, bj, in);
-                        if ((best >> 63) == 0) {
-                            in.T = bT;  // the clock as the prediction saw it
-                            in.K += bk;
-                            t_admit(in, bj, q, req, bpre, e);
-                            rej_sum -= q.rej;
+                        *hot.unit(lm) = lo;
+                        *hot.unit(lm + 1u) = hi;
+                        tile_base = (int64_t)(((uint64_t)hb.y << 32) | hb.x);
+                    }
+                } else {
+                    // the next live requests at or after pos: up to four of one 32-request word of the map
+                    uint32_t ri = pos - tile * kTTile;
+                    uint32_t bits = *hot.word(lm + (ri >> 7), (ri >> 5) & 3u) >> (ri & 31u);
+                    while (bits == 0u) {
+                        ri = (ri | 31u) + 1u;
+                        if (ri >= recs) break;
+                        bits = *hot.word(lm + (ri >> 7), (ri >> 5) & 3u);
+                    }
+                    if (ri >= recs) {
+                        pos = tile * kTTile + recs;
+                    } else {
+                        const uint4* const rp = th + kScanHdrUnits;  // the tile's scan records
+                        uint32_t at[4];
+                        uint4 sr[4];
+                        bool have[4], real[4];
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            have[k] = bits != 0u;
+                            at[k] = ri + (uint32_t)__ffs((int)bits) - 1u;
+                            bits &= bits - 1u;
+                            have[k] = have[k] && at[k] < recs;
+                            sr[k] = ldg_nc(rp + (have[k] ? at[k] : ri));
+                        }
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            const uint32_t model = sr[k].w & 0xFFu;
+                            // in the request subset, and a model the placement serves
+                            bool r = have[k] && ((cmask >> ((sr[k].w >> 8) & 31u)) & 1u) && ((hasmodel >> model) & 1u);
+                            if (r && sr[k].x != 0xFFFFFFFFu) {
+                                // Too late whatever the instance?  Every predicted first token of this model lies at
+                                // or after flb: the dispatcher's clock plus the smallest prefill base, and the lower
+                                // bound kept from the latest look at the model's instances (times only move forward).
+                                const uint4 me = *hot.unit(rr + model);
+                                const int64_t arrival = tile_base + (int64_t)sr[k].x;
+                                const int64_t flb = max(max(now, arrival) + (int64_t)me.z, (int64_t)(((uint64_t)me.y << 32) | me.x));
+                                const bool late_first = sr[k].y != 0xFFFFFFFFu && arrival + (int64_t)sr[k].y < flb;
+                                const bool late_end = sr[k].z != 0xFFFFFFFFu &&
+                                                      arrival + (int64_t)sr[k].z < flb + (int64_t)((uint64_t)(sr[k].w >> 16) * me.w);
+                                r = !(late_first || late_end);
+                            }
+                            real[k] = r;
+                        }
+                        // the first of them that needs the distributor stops the lane; the ones before it are
+                        // rejected (overflow protection, the plain case: nobody can meet the deadline)
+                        uint32_t next = recs;
+                        bool stop = false;
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            if (stop || !have[k]) continue;
+                            if (real[k]) {
+                                stop = true;
+                                next = at[k];
+                            } else {
+                                if (side && ((cmask >> ((sr[k].w >> 8) & 31u)) & 1u))
+                                    t_reject_side(P, out_base + cand, tile * kTTile + at[k], sr[k].w & 0xFFu);
+                                next = at[k] + 1u;
+                            }
+                        }
+                        pos = tile * kTTile + next;
+                        if (stop) {
+                            // the request's full record is read when the waiting lanes are served; a load into
+                            // registers here would make the next iteration wait for it
+                            state = kLaneWait;
+                            const uint4* full = cooked + (size_t)pos * kCookedWords;
+                            prefetch_l1(full);
+                            prefetch_l1(full + 2);
+                        }
+                    }
+                }
+                if (state == kLaneScan && pos >= n_req) state = kLaneDone;
+            }
+
+            // ---- a distributor round for the waiting lanes, once enough of them wait --------------------------
+            const uint32_t wl = __ballot_sync(kFullMaskT, state == kLaneWait);
+            const uint32_t act = __ballot_sync(kFullMaskT, state == kLaneScan);
+            if (wl != 0u && ((uint32_t)__popc(wl) >= theta || act == 0u)) {
+                // statistics of completed requests, all lanes together
+                if (__any_sync(kFullMaskT, e.qn >= 3u)) t_flush_now(e);
+                if (state == kLaneWait) {
+                    const uint32_t req = pos;
+                    const uint4* const full = cooked + (size_t)req * kCookedWords;
+                    const CookedReq q = decode_cooked(ldg_nc(full), ldg_nc(full + 1), ldg_nc(full + 2));
+                    pos++;
+                    now = max(now, q.arrival);  // pending time: the dispatcher never goes back
+                    // instances of the request's model
+                    const uint4 rg = *hot.unit(q.model >> 3);
+                    const uint32_t rgw = (q.model & 4u) ? ((q.model & 2u) ? rg.w : rg.z) : ((q.model & 2u) ? rg.y : rg.x);
+                    const uint32_t rh = (q.model & 1u) ? (rgw >> 16) : (rgw & 0xFFFFu);
+                    const uint32_t j_lo = rh & 0xFFu, j_hi = rh >> 8;
+                    bool pending = true;
+                    uint32_t tries = 0;
+                    do {
+                        tries++;
+                        uint64_t best = kKeyInf;
+                        uint32_t bj = 0, bk = 0;
+                        int64_t bT = 0, bpre = 0;
+                        // smallest and second smallest (start time + prefill base) over the model's instances
+                        int64_t lb1 = INT64_MAX, lb2 = INT64_MAX;
+                        uint32_t lb1j = 0xFFFFFFFFu;
+                        for (uint32_t j = j_lo; j < j_hi; j++) {
+                            TInst in;
+                            t_load(e.hp, j, in);
+                            if (in.model != q.model) continue;
+                            // "reduce": where the instance's clock stands once it has reached `now`
+                            int64_t T = in.T;
+                            uint32_t kadd = 0;
+                            if (in.w > 0) {
+                                if (T < now) {
+                                    if (now > in.tc - (int64_t)in.sw) {  // something completes on the way
+                                        t_advance_events(in, j, now, false, e);
+                                        T = in.T;
+                                    } else if (in.w < in.B) {
+                                        kadd = ceil_div_small(now - T, in.sw, rcp_approx((float)in.sw));
+                                        T += (int64_t)kadd * (int64_t)in.sw;
+                                    }
+                                }
+                            } else if (T < now) {
+                                T = now;
+                            }
+                            // distributor prediction (Sec. IV-F steps 2-3)
+                            const int64_t pre = prefill_us(in.pre_base, in.pre_q16, q.in_tokens);
+                            const bool free_slot = in.w < in.B;
+                            const int64_t t0 = free_slot ? T : in.tc;
+                            const uint32_t sB = (OPT && free_slot) ? in.swn : in.stepB;
+                            const int64_t first = t0 + pre;
+                            const int64_t fin = first + (int64_t)((uint64_t)q.Sm1 * sB);
+                            {
+                                const int64_t lb = t0 + (int64_t)in.pre_base;
+                                if (lb < lb1) { lb2 = lb1; lb1 = lb; lb1j = j; }
+                                else if (lb < lb2) lb2 = lb;
+                            }
+                            const bool ok = first <= q.dl_ttft && (q.Sm1 == 0 || sB <= q.tbt32) && fin <= q.dl_e2e;
+                            const uint64_t key = ((uint64_t)(free_slot ? 0u : 1u) << 63) | (uint64_t)first;
+                            if (ok && key < best) { best = key; bj = j; bk = kadd; bT = T; bpre = pre; }
+                        }
+                        int64_t lb_new = lb1;  // the model's lower bound as this look at its instances leaves it
+                        if (best == kKeyInf) {
+                            // overflow protection: nobody can meet the deadline -> rejected
+                            if (side) t_reject_side(P, out_base + cand, req, q.model);
                             pending = false;
-                            lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
                         } else {
-                            // every capable instance is full: wait until the chosen slot frees
-                            now = in.tc;
-                            if (!OPT) {
-                                tries++;  // the second round, counted only
-                                t_advance_events(in, bj, now, false, e);
+                            TInst in;
+                            t_load(e.hp, bj, in);
+                            if ((best >> 63) == 0) {
+                                in.T = bT;  // the clock as the prediction saw it
+                                in.K += bk;
                                 t_admit(in, bj, q, req, bpre, e);
                                 rej_sum -= q.rej;
                                 pending = false;
                                 lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
-                            } else if (tries >= kAttemptCap) {
-                                status = MAASO_CAND_ELOOP;
-                                pending = false;
+                            } else {
+                                // every capable instance is full: wait until the chosen slot frees
+                                now = in.tc;
+                                if (!OPT) {
+                                    tries++;  // the second round, counted only
+                                    t_advance_events(in, bj, now, false, e);
+                                    t_admit(in, bj, q, req, bpre, e);
+                                    rej_sum -= q.rej;
+                                    pending = false;
+                                    lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
+                                } else if (tries >= kAttemptCap) {
+                                    status = MAASO_CAND_ELOOP;
+                                    pending = false;
+                                }
                             }
                         }
-                    }
-                    if (lb1 != INT64_MAX)
-                        *reinterpret_cast<uint2*>(e.pl.unit(rr + q.model)) = make_uint2((uint32_t)lb_new, (uint32_t)((uint64_t)lb_new >> 32));
-                } while (OPT && pending);
-                extra += tries - 1u;
-                if (status) ri = recs;  // given up on this candidate
+                        if (lb1 != INT64_MAX)
+                            *reinterpret_cast<uint2*>(hot.unit(rr + q.model)) = make_uint2((uint32_t)lb_new, (uint32_t)((uint64_t)lb_new >> 32));
+                    } while (OPT && pending);
+                    extra += tries - 1u;
+                    state = (status != 0u || pos >= n_req) ? kLaneDone : kLaneScan;  // a flagged candidate is given up
+                }
             }
-            // this warp is done with the stage: refill it
-            __syncwarp();
-            if (lane == 0 && t + kTStages < n_tiles) {
-                fence_proxy_async();
-                t_issue_tile(sm, scan, n_req, s, t + kTStages);
-            }
-            if (t + kTStages < n_tiles) in_flight++;
-            tile_seq++;
-        }
 
-        // ---- drain, account what is still queued, write the record ------------------------------
-        __syncwarp();
-        if (valid && status == 0) {
-            for (uint32_t j = 0; j < n_i; j++) {
-                TInst in;
-                t_load(e.pl, ru, j, in);
-                if (in.w > 0) t_advance_events(in, j, 0, true, e);
+            // ---- lanes that are through their trace: drain, account what is still queued, write the record -----
+            if (__any_sync(kFullMaskT, state == kLaneDone)) {
+                if (state == kLaneDone) {
+                    if (status == 0) {
+                        for (uint32_t j = 0; j < n_i; j++) {
+                            TInst in;
+                            t_load(e.hp, j, in);
+                            if (in.w > 0) t_advance_events(in, j, 0, true, e);
+                        }
+                    }
+                    t_flush_now(e);
+                    Stats st = ls.st;
+                    st.checksum += rej_sum;
+                    write_result(P.out + out_base + cand, status, n_counted, n_counted - st.served, (uint64_t)n_counted + extra, st,
+                                 ls.hbc);
+                    state = kLaneIdle;
+                    e.oc = -1;
+                }
             }
-        }
-        t_flush_now(e);
-        if (valid) {
-            Stats st = ls.st;
-            st.checksum += rej_sum;
-            write_result(P.out + out_base + cand, status, n_counted, n_counted - st.served, (uint64_t)n_counted + extra, st,
-                         ls.hbc);
         }
         __syncwarp();
     }
 }
 
-cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t theta, void* arena,
-                               cudaStream_t stream) {
+cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t hot_bytes, uint32_t theta,
+                               void* arena, cudaStream_t stream) {
     auto kernel = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_thread_kernel<true> : eval_thread_kernel<false>;
-    const size_t smem = (arena ? 0 : (size_t)pool_bytes) + kTFixedBytes;
+    const size_t smem = (arena ? 0 : (size_t)pool_bytes) + hot_bytes + t_fixed_smem(P.n_models);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kernel<<<grid, 32, smem, stream>>>(P, pool_bytes, theta, static_cast<unsigned char*>(arena));
+    kernel<<<grid, 32, smem, stream>>>(P, pool_bytes, hot_bytes, theta, static_cast<unsigned char*>(arena));
     return cudaGetLastError();
 }
 
-int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, bool in_smem) {
+int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, uint32_t hot_bytes, bool in_smem) {
     auto kernel = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_thread_kernel<true> : eval_thread_kernel<false>;
-    const size_t smem = (in_smem ? (size_t)pool_bytes : 0) + kTFixedBytes;
+    const size_t smem = (in_smem ? (size_t)pool_bytes : 0) + hot_bytes + t_fixed_smem(P.n_models);
     cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, 32, smem) != cudaSuccess) return 1;
     return n < 1 ? 1 : n;
 }
 
-uint32_t thread_fixed_smem() { return kTFixedBytes; }
+uint32_t thread_fixed_smem(uint32_t n_models) { return (uint32_t)t_fixed_smem(n_models); }
 
 // Global scratch one warp of the thread mapping needs: two entries of 24 bytes per slot, 4 slots per pool unit.
 size_t thread_scratch_per_warp(uint32_t pool_bytes) { return (size_t)(pool_bytes / 16u) * 8u * 24u; }

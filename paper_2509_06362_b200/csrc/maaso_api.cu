@@ -19,11 +19,11 @@ cudaError_t launch_eval_group(const EvalParams& P, int grid, int tile_recs, int 
                               cudaStream_t stream);
 int occupancy_eval_group(const EvalParams& P, int tile_recs, int blocks_per_sm, int smem_per_sm);
 size_t group_scratch_per_lane();
-cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t theta, void* arena,
-                               cudaStream_t stream);
-int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, bool in_smem);
+cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t hot_bytes, uint32_t theta,
+                               void* arena, cudaStream_t stream);
+int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, uint32_t hot_bytes, bool in_smem);
 size_t thread_scratch_per_warp(uint32_t pool_bytes);
-uint32_t thread_fixed_smem();
+uint32_t thread_fixed_smem(uint32_t n_models);
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 cudaError_t launch_eval_block_reg(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 int occupancy_eval_block_reg(const EvalParams& P, int bucket, int tile_recs);
@@ -53,6 +53,7 @@ struct maaso_trace {
     uint64_t n;
     uint32_t n_classes;
     uint32_t max_model;
+    double tok_rate;  // output tokens per second the trace asks for (routing hint of MAASO_MAP_AUTO)
 };
 
 struct maaso_ctx {
@@ -82,14 +83,15 @@ struct maaso_ctx {
     int group_blocks;  // blocks of the lane-group kernel per SM its key pool is sized for; 0 = by batch size
     int smem_per_sm;
     int promote_pct;  // share of the spare resident warps the planner may use for promotions
-    int thread_arena_kb;  // thread mapping: KB of global memory per warp for the placements' state, 0 = shared memory
+    int thread_arena_kb;  // thread mapping: KB of global memory per warp for the cold part of the placements' state, 0 = shared memory
+    int thread_hot_kb;    // with an arena: KB of shared memory per warp for the hot part
     int thread_blocks;   // one-warp blocks of the thread-mapping kernel per SM its pool is sized for
     uint32_t thread_theta;     // waiting lanes of a warp that trigger a distributor round in the thread mapping
     uint32_t thread_min_cand;  // MAASO_MAP_AUTO takes the thread mapping from this many candidates on
     uint32_t last_mapping;     // mapping the most recent scoring call resolved to
     int fail_allocs;           // test hook: this many of the next scratch allocations are refused
     bool timing;
-    cudaEvent_t ev[6];   // eval: start, after prep, after group, after block; topk: start, end
+    cudaEvent_t ev[7];   // eval: start, after prep, after group, after block; topk: start, end; eval: after thread
     bool ev_eval, ev_topk;
     std::string last_error;
 };
@@ -173,7 +175,7 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
     ctx->own_stream = nullptr;
     ctx->timing = false;
     ctx->ev_eval = ctx->ev_topk = false;
-    for (int i = 0; i < 6; i++) ctx->ev[i] = nullptr;
+    for (int i = 0; i < 7; i++) ctx->ev[i] = nullptr;
     DeviceGuard g(cuda_device);
     cudaDeviceProp prop;
     e = cudaGetDeviceProperties(&prop, cuda_device);
@@ -204,11 +206,17 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
         if (v >= 16 && v <= 2048) ctx->tile_recs = v & ~1;  // even: tiles of 8-byte terms stay 16-byte aligned
     }
 
-    ctx->thread_arena_kb = 0;
+    ctx->thread_arena_kb = 128;
     const char* ta = getenv("MAASO_THREAD_ARENA_KB");
     if (ta) {
         int v = atoi(ta);
         if (v >= 0 && v <= 1023) ctx->thread_arena_kb = v;
+    }
+    ctx->thread_hot_kb = 12;
+    const char* thk = getenv("MAASO_THREAD_HOT_KB");
+    if (thk) {
+        int v = atoi(thk);
+        if (v >= 2 && v <= 128) ctx->thread_hot_kb = v;
     }
     ctx->thread_blocks = 6;
     const char* tb = getenv("MAASO_THREAD_BLOCKS");
@@ -216,13 +224,13 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
         int v = atoi(tb);
         if (v >= 1 && v <= 16) ctx->thread_blocks = v;
     }
-    ctx->thread_theta = 12;
+    ctx->thread_theta = 8;
     const char* tt = getenv("MAASO_THREAD_THETA");
     if (tt) {
         int v = atoi(tt);
         if (v >= 1 && v <= 32) ctx->thread_theta = (uint32_t)v;
     }
-    ctx->thread_min_cand = 0xFFFFFFFFu;  // the lane groups unless asked otherwise
+    ctx->thread_min_cand = 16384;  // fewer loaded placements than this do not fill the GPU one per lane
     const char* tm = getenv("MAASO_THREAD_MIN_CAND");
     if (tm) {
         long v = atol(tm);
@@ -270,7 +278,7 @@ MAASO_API void maaso_destroy(maaso_ctx* ctx) {
     if (ctx->stage) cudaFree(ctx->stage);
     if (ctx->deploy) cudaFree(ctx->deploy);
     if (ctx->own_stream) cudaStreamDestroy(ctx->own_stream);
-    for (int i = 0; i < 6; i++)
+    for (int i = 0; i < 7; i++)
         if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
     delete ctx;
 }
@@ -364,6 +372,7 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     // per class: how many requests, and the sum of their checksum terms as rejected requests (the thread
     // mapping starts from "everything counted was rejected" and takes the served ones out)
     std::vector<uint64_t> class_tot((size_t)n_classes * 2, 0);
+    uint64_t tok_sum = 0;
     for (uint64_t r = 0; r < n; r++) {
         const maaso_request& q = host[r];
         if (q.arrival_us < prev || q.arrival_us > kArrMax)
@@ -373,6 +382,7 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
         if (q.cls >= n_classes) return fail(ctx, MAASO_EINVAL, "trace: unknown SLO class");
         if (q.model >= ctx->n_models) return fail(ctx, MAASO_EINVAL, "trace: unknown model");
         if (q.model > max_model) max_model = q.model;
+        tok_sum += q.out_tokens;
         class_tot[(size_t)q.cls * 2] += 1;
         class_tot[(size_t)q.cls * 2 + 1] += host_rejected_hash((uint32_t)r);
     }
@@ -388,6 +398,10 @@ MAASO_API int maaso_load_trace(maaso_ctx* ctx, const maaso_request* reqs, uint64
     t->n = n;
     t->n_classes = n_classes;
     t->max_model = max_model;
+    {
+        const double span_s = n > 1 ? (double)(host[n - 1].arrival_us - host[0].arrival_us) * 1e-6 : 0.0;
+        t->tok_rate = span_s > 0.0 ? (double)tok_sum / span_s : 0.0;
+    }
     t->h_classes = cls;
     cudaError_t e = cudaMalloc(&t->d_reqs, (n ? n : 1) * sizeof(maaso_request));
     if (e == cudaSuccess) e = cudaMalloc(&t->d_classes, cls.size() * 8);
@@ -462,8 +476,9 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     if (variant && o.mapping == MAASO_MAP_THREAD)
         return fail(ctx, MAASO_EINVAL,
                     "eval: the fixed-speed engine, per-instance queues and the largest-gap test have no thread mapping");
-    if (o.mapping == MAASO_MAP_AUTO)
-        o.mapping = (!variant && cands->n_cand >= ctx->thread_min_cand) ? MAASO_MAP_THREAD : MAASO_MAP_GROUP;
+    // MAASO_MAP_AUTO: the other engines exist in the lane-group kernel only; for the default engine both the
+    // lane-group and the thread kernel are launched and the validation kernels route the batch
+    if (o.mapping == MAASO_MAP_AUTO && variant) o.mapping = MAASO_MAP_GROUP;
     ctx->last_mapping = o.mapping;
 
     DeviceGuard g(ctx->device);
@@ -515,40 +530,51 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     // wave is bound by its longest dependent chains, which run faster with fewer warps sharing a
     // scheduler; a larger batch is bound by instruction issue and wants all four.  Lanes needed
     // ~ instances x 1.3 (group widths are powers of two).
-    const bool threads = o.mapping == MAASO_MAP_THREAD;
+    const bool threads = o.mapping == MAASO_MAP_THREAD || o.mapping == MAASO_MAP_AUTO;
+    const bool groups = o.mapping == MAASO_MAP_GROUP || o.mapping == MAASO_MAP_AUTO;
     int group_blocks = ctx->group_blocks;
     if (group_blocks == 0) {
         const uint64_t est_warps = ((cands->n_inst * 13 / 10 + 31) / 32 + 6) * n_traces;
         group_blocks = est_warps <= (uint64_t)ctx->sm_count * 3 * (kGroupThreads / 32) ? 3 : 4;
     }
     int grid_g = 0, grid_t = 0;
-    uint32_t thread_pool = 0;
-    size_t pay_entries = 0;
+    uint32_t thread_pool = 0, thread_hot = 0;
+    size_t pay_entries = 0, pay_thread = 0;  // scratch entries of the lane-group / block kernels, of the thread kernel
     static_assert(sizeof(Payload) == 32, "scratch is counted in 32-byte entries");
     if (threads) {
         // thread mapping: one-warp blocks; the pool is what is left of an SM's shared memory when
         // `thread_blocks` of them share it (1 KB per block is reserved by the system)
-        size_t pool;
+        // The hot part of the instances (what a prediction reads: 3 units each) is always in shared memory;
+        // the cold part (slot masks and keys) is in shared memory too, or in a per-warp arena in global memory,
+        // which leaves room for more resident warps.
+        size_t pool, hot;
         if (ctx->thread_arena_kb > 0) {
             pool = (size_t)ctx->thread_arena_kb * 1024;
+            hot = (size_t)ctx->thread_hot_kb * 1024;
         } else {
             size_t per_block = (size_t)ctx->smem_per_sm / (size_t)ctx->thread_blocks;
             per_block = per_block > 1024 ? per_block - 1024 : 0;
             if (per_block > 227u * 1024u) per_block = 227u * 1024u;
-            const size_t fixed = thread_fixed_smem();
-            pool = per_block > fixed ? per_block - fixed : 0;
+            const size_t fixed = thread_fixed_smem(ctx->n_models);
+            const size_t both = per_block > fixed ? per_block - fixed : 0;
+            hot = both / 4;  // an instance has 3 hot units and about 8 cold ones
+            hot -= hot % 512;
+            pool = both - hot;
             pool -= pool % 512;
         }
         if (pool > 65535u * 16u) pool = 65535u * 16u - (65535u * 16u) % 512;  // unit offsets are 16-bit
-        if (pool < 4096) return fail(ctx, MAASO_ESTATE, "eval: no shared memory for the thread mapping");
+        if (pool < 4096 || hot < 1536) return fail(ctx, MAASO_ESTATE, "eval: no shared memory for the thread mapping");
         thread_pool = (uint32_t)pool;
+        thread_hot = (uint32_t)hot;
         P.thread_pool_units = thread_pool / 16u;
-        grid_t = ctx->sm_count * occupancy_eval_thread(P, thread_pool, ctx->thread_arena_kb == 0);
+        P.thread_hot_units = thread_hot / 16u;
+        grid_t = ctx->sm_count * occupancy_eval_thread(P, thread_pool, thread_hot, ctx->thread_arena_kb == 0);
         const uint64_t max_items_t = ((uint64_t)C + 9) * n_traces;
         if ((uint64_t)grid_t > max_items_t) grid_t = (int)max_items_t;
-        pay_entries = ((size_t)grid_t * (thread_scratch_per_warp(thread_pool) + (ctx->thread_arena_kb > 0 ? thread_pool : 0)) +
-                       sizeof(Payload) - 1) / sizeof(Payload);
-    } else if (o.mapping != MAASO_MAP_BLOCK) {
+        pay_thread = ((size_t)grid_t * (thread_scratch_per_warp(thread_pool) + (ctx->thread_arena_kb > 0 ? thread_pool : 0)) +
+                      sizeof(Payload) - 1) / sizeof(Payload);
+    }
+    if (groups) {
         const int occ_g = occupancy_eval_group(P, tile, group_blocks, ctx->smem_per_sm);
         grid_g = ctx->sm_count * occ_g;
         // at most one work item per 4 candidates + bucket tails, once per trace
@@ -562,8 +588,9 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
         // more than 32 instances (lane groups), or a state larger than a warp's pool (thread mapping)
         bool used = n_traces == 1 && o.mapping == MAASO_MAP_BLOCK;
         if (n_traces == 1 && b == kGenericBlockBucket) {
+            // more than 32 instances: the thread kernel where it can run, else one block per placement
             if (o.mapping == MAASO_MAP_GROUP) used = cands->n_inst > 32;
-            if (threads) used = cands->n_inst * 22ull + 20ull > P.thread_pool_units;  // 22 units: an instance with 64 slots
+            if (threads) used = cands->n_inst * 19ull > P.thread_pool_units || cands->n_inst * 3ull > P.thread_hot_units;  // 22 units: an instance with 64 slots
         }
         grid_b[b - 6] = 0;
         if (!used) continue;
@@ -580,25 +607,35 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     size_t off = 0;
     const size_t off_counters = off; off = align_up(off + kCounterWords * 4, 256);
     const size_t off_code = off;     off = align_up(off + (size_t)C * 4, 256);
+    const size_t off_code2 = off;    off = align_up(off + (size_t)C * 4, 256);
     const size_t off_lists = off;    off = align_up(off + (size_t)kNumBuckets * C * 4, 256);
     const size_t off_dump = off;     off = align_up(off + (o.dump_n ? (size_t)C * 4 : 0), 256);
     const size_t off_pay = off;      off = align_up(off + pay_entries * sizeof(Payload), 256);
+    const size_t off_pay_t = off;    off = align_up(off + pay_thread * sizeof(Payload), 256);
     int rc = grow(ctx, &ctx->scratch, &ctx->scratch_bytes, off);
     if (rc != MAASO_OK) return rc;
     unsigned char* sb = static_cast<unsigned char*>(ctx->scratch);
     P.bucket_count = reinterpret_cast<uint32_t*>(sb + off_counters);
-    P.work_ctr = P.bucket_count + 16;
+    P.work_ctr = P.bucket_count + 32;
     P.hist = P.bucket_count + 64;
-    P.sm_ctr = P.hist + 2 * kNumBuckets * kCostBins;
+    P.sm_ctr = P.hist + kHistRows * kCostBins;
     P.n_sm = (uint32_t)(ctx->sm_count < 1024 ? ctx->sm_count : 1024);
     P.code = reinterpret_cast<uint32_t*>(sb + off_code);
+    P.code2 = reinterpret_cast<uint32_t*>(sb + off_code2);
     P.bucket_list = reinterpret_cast<uint32_t*>(sb + off_lists);
     P.dump_row = o.dump_n ? reinterpret_cast<int32_t*>(sb + off_dump) : nullptr;
     P.payload = reinterpret_cast<Payload*>(sb + off_pay);
 
-    static_assert(64 + 2 * kNumBuckets * kCostBins + 1024 <= kCounterWords, "counter region");
+    static_assert(64 + kHistRows * kCostBins + 1024 <= kCounterWords, "counter region");
     P.group_warps = (uint32_t)grid_g * (kGroupThreads / 32);
-    P.mapping = o.mapping;  // resolved: block, lane groups or threads
+    P.mapping = o.mapping;  // block, lane groups, threads, or auto (routed by the validation kernels)
+    P.thread_min_cand = ctx->thread_min_cand;
+    {   // output tokens per second the trace(s) ask for (mean over the traces of the call)
+        double d = 0.0;
+        for (uint32_t t = 0; t < n_traces; t++) d += traces[t]->tok_rate;
+        d /= n_traces;
+        P.demand_tok_s = d >= 4.0e9 ? 4000000000u : (uint32_t)d;
+    }
     P.promote_pct = (uint32_t)ctx->promote_pct;
     cudaError_t e = cudaMemsetAsync(sb + off_counters, 0, kCounterWords * 4, stream);
     if (e == cudaSuccess && o.ttft_hist)
@@ -609,20 +646,24 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     e = launch_prep(P, o.dump_cand_idx, stream, &launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "prep launch");
     if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
-    if (threads) {
-        // the arena (if any) follows the scratch entries of the running requests
-        void* arena = ctx->thread_arena_kb > 0
-                          ? static_cast<void*>(reinterpret_cast<unsigned char*>(P.payload) + (size_t)grid_t * thread_scratch_per_warp(thread_pool))
-                          : nullptr;
-        e = launch_eval_thread(P, grid_t, thread_pool, ctx->thread_theta, arena, stream);
-        launches++;
-        if (e != cudaSuccess) return cuda_fail(ctx, e, "thread kernel launch");
-    } else if (o.mapping != MAASO_MAP_BLOCK) {
+    if (groups) {
         e = launch_eval_group(P, grid_g, tile, group_blocks, ctx->smem_per_sm, stream);
         launches++;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "group kernel launch");
     }
     if (ctx->timing) cudaEventRecord(ctx->ev[2], stream);
+    if (threads) {
+        // the thread kernel has scratch of its own; its arena (if any) follows the entries of the running requests
+        EvalParams PT = P;
+        PT.payload = reinterpret_cast<Payload*>(sb + off_pay_t);
+        void* arena = ctx->thread_arena_kb > 0
+                          ? static_cast<void*>(sb + off_pay_t + (size_t)grid_t * thread_scratch_per_warp(thread_pool))
+                          : nullptr;
+        e = launch_eval_thread(PT, grid_t, thread_pool, thread_hot, ctx->thread_theta, arena, stream);
+        launches++;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "thread kernel launch");
+    }
+    if (ctx->timing) cudaEventRecord(ctx->ev[6], stream);
     for (int b = 6; b <= kGenericBlockBucket; b++) {
         if (grid_b[b - 6] == 0) continue;
         e = b < kGenericBlockBucket ? launch_eval_block_reg(P, b, grid_b[b - 6], tile, stream)
@@ -1203,7 +1244,7 @@ MAASO_API int maaso_set_timing(maaso_ctx* ctx, int enabled) {
     if (!ctx) return MAASO_EINVAL;
     DeviceGuard g(ctx->device);
     if (enabled)
-        for (int i = 0; i < 6; i++)
+        for (int i = 0; i < 7; i++)
             if (!ctx->ev[i]) {
                 cudaError_t e = cudaEventCreate(&ctx->ev[i]);
                 if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventCreate");
@@ -1222,10 +1263,9 @@ MAASO_API int maaso_get_timing(maaso_ctx* ctx, maaso_timing* out) {
     if (ctx->ev_eval) {
         e = cudaEventSynchronize(ctx->ev[3]);
         if (e == cudaSuccess) e = cudaEventElapsedTime(&out->prep_ms, ctx->ev[0], ctx->ev[1]);
-        if (e == cudaSuccess)
-            e = cudaEventElapsedTime(ctx->last_mapping == MAASO_MAP_THREAD ? &out->thread_ms : &out->group_ms,
-                                     ctx->ev[1], ctx->ev[2]);
-        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->block_ms, ctx->ev[2], ctx->ev[3]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->group_ms, ctx->ev[1], ctx->ev[2]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->thread_ms, ctx->ev[2], ctx->ev[6]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&out->block_ms, ctx->ev[6], ctx->ev[3]);
     }
     if (e == cudaSuccess && ctx->ev_topk) {
         e = cudaEventSynchronize(ctx->ev[5]);

@@ -4,22 +4,26 @@
 
 namespace maaso {
 
+// Where a valid candidate can be scored.  `code` = its bucket among the lane-group / block buckets
+// (0..9) and its cost bin, `code2` = its bucket among the thread-mapping buckets (10..18) and the
+// bin; 0xFFFFFFFF = it has no such place.  A candidate with both is placed by the batch-wide choice
+// plan_kernel makes (MAASO_MAP_AUTO).
 __global__ void prep_kernel(const EvalParams P) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= P.n_cand) return;
     const uint32_t lo = P.offsets[c], hi = P.offsets[c + 1];
     uint32_t status = 0, n = 0, sum_b = 0;
-    // thread mapping: 16-byte units of state (model ranges, one entry per model, the tile's live map, per
-    // instance 4 + key blocks + minima)
-    uint32_t units = ((P.n_models + 7u) >> 3) + P.n_models + 2u;
+    uint32_t units = 0;  // thread mapping: 16-byte units of cold instance state (per instance 1 + key blocks + minima)
+    uint64_t supply = 0; // decode tokens per second the placement can produce with every slot busy
+    const bool variant = (P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES)) != 0;
+    const bool threads_ok = !variant && (P.mapping == MAASO_MAP_THREAD || P.mapping == MAASO_MAP_AUTO);
+    const bool groups_ok = P.mapping != MAASO_MAP_THREAD;
     if (hi < lo || hi > P.n_inst) {
         status = MAASO_CAND_EBADINST;  // malformed CSR row
     } else {
         n = hi - lo;
-        const bool group_only = P.mapping != MAASO_MAP_THREAD &&
-                                ((P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES)) || P.n_traces > 1);
-        if (n > MAASO_MAX_INSTANCES || (group_only && n > 32)) {
-            status = MAASO_CAND_ETOOMANY;  // these options exist in the lane-group kernel only
+        if (n > MAASO_MAX_INSTANCES) {
+            status = MAASO_CAND_ETOOMANY;
         } else {
             uint64_t devsum = 0;
             for (uint32_t i = 0; i < n; i++) {
@@ -30,13 +34,33 @@ __global__ void prep_kernel(const EvalParams P) {
                     continue;
                 }
                 sum_b += b;
-                units += 4u + 2u * ((b + 7u) >> 3) + 2u;
+                units += 1u + 2u * ((b + 7u) >> 3) + 2u;
+                supply += (uint64_t)b * 1000000ull / (uint64_t)P.rows[(m * P.n_strategies + s) * kRowStride + 1 + b];
                 devsum += (uint64_t)P.devices[s];
                 if (P.devices[s] < P.min_devices[m]) status |= MAASO_CAND_EMEMFIT;
             }
             if (devsum > P.budget) status |= MAASO_CAND_EBUDGET;
-            // several traces in one pass exist in the lane-group and thread kernels only
-            if (P.mapping == MAASO_MAP_THREAD && P.n_traces > 1 && units > P.thread_pool_units) status |= MAASO_CAND_ETOOMANY;
+        }
+    }
+    // where it can go
+    int bg = -1, bt = -1;
+    if (!status) {
+        if (threads_ok) {
+            // as many lanes per item as placements of this size fit the warp's pools
+            const uint32_t fit = n ? min(P.thread_pool_units / units, P.thread_hot_units / (3u * n)) : 32u;
+            const uint32_t lanes[9] = {32, 24, 16, 12, 8, 6, 4, 2, 1};
+            for (int i = 0; i < 9; i++)
+                if (fit >= lanes[i]) { bt = kThreadBucket0 + i; break; }
+        }
+        if (P.mapping == MAASO_MAP_BLOCK) bg = n <= 2 ? 6 : (n <= 4 ? 7 : (n <= 8 ? 8 : kGenericBlockBucket));
+        else if (groups_ok && n <= 32) bg = n <= 1 ? 0 : 32 - __clz((int)(n - 1));
+        // More than 32 instances: the thread mapping if it can hold the placement, else one block per
+        // placement (default engine, one trace); the other engines and several traces in one pass
+        // exist in the lane-group and thread kernels only.
+        if (n > 32 && bt >= 0) bg = -1;
+        if (bg < 0 && bt < 0) {
+            if (!variant && P.n_traces <= 1) bg = kGenericBlockBucket;
+            else status = MAASO_CAND_ETOOMANY;
         }
     }
     if (P.dump_row) P.dump_row[c] = -1;
@@ -54,32 +78,35 @@ __global__ void prep_kernel(const EvalParams P) {
     }
     if (status) {
         P.code[c] = 0xFFFFFFFFu;
+        P.code2[c] = 0xFFFFFFFFu;
         return;
     }
-    int b;
-    if (P.mapping == MAASO_MAP_BLOCK) b = n <= 2 ? 6 : (n <= 4 ? 7 : (n <= 8 ? 8 : kGenericBlockBucket));
-    else if (P.mapping == MAASO_MAP_THREAD) {
-        // as many lanes per item as placements of this size fit the warp's pool
-        const uint32_t fit = units ? P.thread_pool_units / units : 32u;
-        const uint32_t lanes[9] = {32, 24, 16, 12, 8, 6, 4, 2, 1};
-        b = kGenericBlockBucket;  // not even one: the block layout takes it
-        for (int i = 0; i < 9; i++)
-            if (fit >= lanes[i]) { b = i; break; }
-    }
-    else if (n <= 32) b = n <= 1 ? 0 : 32 - __clz((int)(n - 1));
-    else b = kGenericBlockBucket;
     // Cost estimate: the total batch cap (how many requests the placement can have in flight;
     // it tracks the number of served requests and so the number of simulation events).
     const uint32_t bin = (kCostBins - 1) - min((uint32_t)(kCostBins - 1), sum_b / 8u);
-    atomicAdd(&P.bucket_count[b], 1u);
-    atomicAdd(&P.hist[b * kCostBins + bin], 1u);
-    P.code[c] = ((uint32_t)b << 8) | bin;
+    P.code[c] = bg >= 0 ? (((uint32_t)bg << 8) | bin) : 0xFFFFFFFFu;
+    P.code2[c] = bt >= 0 ? (((uint32_t)bt << 8) | bin) : 0xFFFFFFFFu;
+    if (bg >= 0 && bt >= 0) {
+        atomicAdd(&P.hist[(kHistBothG + bg) * kCostBins + bin], 1u);
+        atomicAdd(&P.hist[(kHistBothT + bt - kThreadBucket0) * kCostBins + bin], 1u);
+        // loaded beyond what it can decode: most of its requests will be turned away, which the
+        // thread mapping does for next to nothing
+        atomicAdd(&P.bucket_count[kCtrBoth], 1u);
+        if ((uint64_t)P.demand_tok_s >= 2ull * supply) atomicAdd(&P.bucket_count[kCtrLoaded], 1u);
+    } else if (bg >= 0) {
+        atomicAdd(&P.hist[(kHistOnlyG + bg) * kCostBins + bin], 1u);
+    } else {
+        atomicAdd(&P.hist[(kHistOnlyT + bt - kThreadBucket0) * kCostBins + bin], 1u);
+    }
 }
 
-// One block, one thread per cost bin: (1) if the resident grid has warps to spare, promote
-// the most expensive candidates of the narrower lane-group buckets to a warp of their own
-// (bucket 5) so that their event handling is not serialised with other candidates' in the
-// same warp; (2) turn the per-bin histograms into write cursors (bins in decreasing cost order).
+// One block, one thread per cost bin: (0) the batch-wide choice between lane groups and threads for
+// the candidates that can go either way (MAASO_MAP_AUTO): threads if most of them are loaded beyond
+// their decode capacity and there are enough of them to fill the GPU one placement per lane; (1) if the
+// resident lane-group grid has warps to spare, promote the most expensive candidates of the narrower
+// lane-group buckets to a warp of their own (bucket 5) so that their event handling is not
+// serialised with other candidates' in the same warp; (2) turn the per-bin histograms into write
+// cursors (bins in decreasing cost order).
 __device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t v, uint32_t* buf) {
     const int t = threadIdx.x;
     buf[t] = v;
@@ -97,38 +124,59 @@ __device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t v, uint32_t* b
 
 __global__ void __launch_bounds__(kCostBins) plan_kernel(const EvalParams P) {
     __shared__ uint32_t buf[kCostBins];
+    __shared__ uint32_t tot[6];
     const int bin = threadIdx.x;
+    const uint32_t n_both = P.bucket_count[kCtrBoth], n_loaded = P.bucket_count[kCtrLoaded];
+    const bool use_threads = n_loaded >= P.thread_min_cand && 2u * n_loaded >= n_both;
+    // final counts of this bin per bucket
+    uint32_t cnt[kNumBuckets];
+    for (int b = 0; b < kThreadBucket0; b++)
+        cnt[b] = P.hist[(kHistOnlyG + b) * kCostBins + bin] + (use_threads ? 0u : P.hist[(kHistBothG + b) * kCostBins + bin]);
+    for (int b = kThreadBucket0; b < kNumBuckets; b++)
+        cnt[b] = P.hist[(kHistOnlyT + b - kThreadBucket0) * kCostBins + bin] +
+                 (use_threads ? P.hist[(kHistBothT + b - kThreadBucket0) * kCostBins + bin] : 0u);
     uint32_t cut = 0;  // bins below `cut` are promoted
     uint32_t narrow = 0;
-    for (int b = 0; b < 5; b++) narrow += P.hist[b * kCostBins + bin];
-    if (P.mapping == MAASO_MAP_GROUP) {
+    for (int b = 0; b < 5; b++) narrow += cnt[b];
+    if (P.mapping != MAASO_MAP_BLOCK && P.mapping != MAASO_MAP_THREAD) {
+        // warps the lane-group buckets need: bucket totals = sums over the bins
         uint32_t need = 0;
-        for (int b = 0; b <= 5; b++) need += (P.bucket_count[b] + (32u >> b) - 1) / (32u >> b);
+        for (int b = 0; b <= 5; b++) {
+            const uint32_t incl = block_inclusive_scan(cnt[b], buf);
+            if (bin == kCostBins - 1) tot[b] = incl;
+        }
+        __syncthreads();
+        for (int b = 0; b <= 5; b++) need += (tot[b] + (32u >> b) - 1) / (32u >> b);
         const uint32_t spare = P.group_warps > need ? (uint32_t)((uint64_t)(P.group_warps - need) * P.promote_pct / 100) : 0;
         const uint32_t incl = block_inclusive_scan(narrow, buf);
         cut = (uint32_t)__syncthreads_count(incl <= spare);  // prefix sums are monotone
     }
     __syncthreads();
     for (int b = 0; b < kNumBuckets; b++) {
-        uint32_t v = P.hist[b * kCostBins + bin];
+        uint32_t v = cnt[b];
         if (b < 5 && (uint32_t)bin < cut) v = 0;
         if (b == 5 && (uint32_t)bin < cut) v += narrow;
         const uint32_t incl = block_inclusive_scan(v, buf);
-        P.hist[(kNumBuckets + b) * kCostBins + bin] = incl - v;
+        P.hist[(kHistCursor + b) * kCostBins + bin] = incl - v;
         if (bin == kCostBins - 1) P.bucket_count[b] = incl;
     }
-    if (bin == 0) P.bucket_count[15] = cut;
+    if (bin == 0) {
+        P.bucket_count[kCtrCut] = cut;
+        P.bucket_count[kCtrUseThreads] = use_threads ? 1u : 0u;
+    }
 }
 
 __global__ void scatter_kernel(const EvalParams P) {
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= P.n_cand) return;
-    const uint32_t code = P.code[c];
-    if (code == 0xFFFFFFFFu) return;
+    const uint32_t cg = P.code[c], ct = P.code2[c];
+    if (cg == 0xFFFFFFFFu && ct == 0xFFFFFFFFu) return;
+    const uint32_t code = (cg != 0xFFFFFFFFu && ct != 0xFFFFFFFFu) ? (P.bucket_count[kCtrUseThreads] ? ct : cg)
+                                                                    : (cg != 0xFFFFFFFFu ? cg : ct);
     uint32_t b = code >> 8;
     const uint32_t bin = code & 0xFFu;
-    if (b < 5 && bin < P.bucket_count[15]) b = 5;
-    const uint32_t pos = atomicAdd(&P.hist[(kNumBuckets + b) * kCostBins + bin], 1u);
+    if (b < 5 && bin < P.bucket_count[kCtrCut]) b = 5;
+    const uint32_t pos = atomicAdd(&P.hist[(kHistCursor + b) * kCostBins + bin], 1u);
     P.bucket_list[(size_t)b * P.n_cand + pos] = c;
 }
 
