@@ -38,7 +38,14 @@ constexpr uint32_t kFullMaskT = 0xFFFFFFFFu;
 constexpr int kTTile = kScanTile;               // requests per scan tile
 constexpr uint32_t kTEndEmpty = 0x1FFFFFFu;    // end-index field of an empty key
 constexpr uint32_t kTRelMax = (1u << 25) - 2u; // largest end index a key can hold
-constexpr int kTQueue = 4;                     // queued completions per lane
+#ifndef MAASO_TQUEUE
+#define MAASO_TQUEUE 4
+#endif
+constexpr int kTQueue = MAASO_TQUEUE;           // queued completions per lane
+#ifndef MAASO_THREAD_BPS
+#define MAASO_THREAD_BPS 12
+#endif
+constexpr int kTBlocksPerSM = MAASO_THREAD_BPS;    // one-warp blocks per SM the register budget allows (3 per scheduler)
 
 // Lanes that work on one item, by launch bucket (bucket 9 = placements the pool cannot hold at all).
 __host__ __device__ inline uint32_t thread_lanes_of(int bucket) {
@@ -73,20 +80,23 @@ struct TInst {
     uint32_t swn;   // step at the level right after one more admission (optimistic estimate)
 };
 
-__device__ __forceinline__ void t_load(const TPool& hp, uint32_t j, TInst& in) {
-    const uint4 a = *hp.unit(3u * j), b = *hp.unit(3u * j + 1u), c = *hp.unit(3u * j + 2u);
+// The hot part (what a prediction reads): unit 2j = clock and next completion, unit 2j+1 = level, batch cap,
+// model, table row | current step | step at the batch cap | step after one more admission.  The prefill
+// terms of the row come from the warp's row table.  K and kmin belong to the cold part (t_load_keys).
+__device__ __forceinline__ void t_load(const TPool& hp, const uint2* rowtab, uint32_t j, TInst& in) {
+    const uint4 a = *hp.unit(2u * j), b = *hp.unit(2u * j + 1u);
     in.T = (int64_t)(((uint64_t)a.y << 32) | a.x);
     in.tc = (int64_t)(((uint64_t)a.w << 32) | a.z);
     in.w = b.x & 0xFFu; in.B = (b.x >> 8) & 0xFFu; in.model = (b.x >> 16) & 0xFFu; in.row = b.x >> 24;
-    in.sw = b.y; in.pre_base = b.z; in.pre_q16 = b.w;
-    in.K = c.x; in.kmin = c.y; in.stepB = c.z; in.swn = c.w;
+    in.sw = b.y; in.stepB = b.z; in.swn = b.w;
+    const uint2 pr = rowtab[in.row];
+    in.pre_base = pr.x; in.pre_q16 = pr.y;
+    in.K = 0; in.kmin = 0;
 }
 __device__ __forceinline__ void t_store(const TPool& hp, uint32_t j, const TInst& in) {
-    *hp.unit(3u * j) = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)in.tc,
-                                                 (uint32_t)((uint64_t)in.tc >> 32));
-    *hp.unit(3u * j + 1u) =
-        make_uint4(in.w | (in.B << 8) | (in.model << 16) | (in.row << 24), in.sw, in.pre_base, in.pre_q16);
-    *hp.unit(3u * j + 2u) = make_uint4(in.K, in.kmin, in.stepB, in.swn);
+    *hp.unit(2u * j) = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)in.tc,
+                                  (uint32_t)((uint64_t)in.tc >> 32));
+    *hp.unit(2u * j + 1u) = make_uint4(in.w | (in.B << 8) | (in.model << 16) | (in.row << 24), in.sw, in.stepB, in.swn);
 }
 
 struct TStats {
@@ -96,7 +106,8 @@ struct TStats {
 
 // What a thread needs besides the instance at hand.
 struct TEnv {
-    TPool hp;             // hot part of the instances (3 units each: what a prediction reads), shared memory
+    TPool hp;             // hot part of the instances (2 units each: what a prediction reads), shared memory
+    const uint2* rowtab;  // per table row: prefill base, prefill slope (shared memory, one copy per warp)
     TPool pl;             // cold part: one unit per instance (slot mask, offsets), then the slot keys; shared or global memory
     int64_t* qf;          // this lane's queue column: entry j at qf[j * 32] = finish time
     uint4* qa;            // entry j at qa[j * 32] = first-token time, arrival time
@@ -175,16 +186,22 @@ struct TKeys {
     uint32_t so;    // number of this instance's slot 0 among the lane's slots (scratch entries)
     uint64_t mask;  // occupied slots; bits at and above B are always set
 };
-__device__ __forceinline__ TKeys t_load_keys(const TPool& pl, uint32_t j) {
-    const uint4 d = *pl.unit(j);
+// The cold part of instance j: unit 2j = slot mask, key offset | slot offset; unit 2j+1 = step counter K,
+// smallest key.  Read and written at events only.
+__device__ __forceinline__ TKeys t_load_keys(const TPool& pl, uint32_t j, TInst& in) {
+    const uint4 d = *pl.unit(2u * j);
+    const uint2 c = *reinterpret_cast<const uint2*>(pl.unit(2u * j + 1u));
     TKeys k;
     k.mask = ((uint64_t)d.y << 32) | d.x;
     k.ko = d.z & 0xFFFFu;
     k.so = d.z >> 16;
+    in.K = c.x;
+    in.kmin = c.y;
     return k;
 }
-__device__ __forceinline__ void t_store_mask(const TPool& pl, uint32_t j, uint64_t mask) {
-    *reinterpret_cast<uint2*>(pl.unit(j)) = make_uint2((uint32_t)mask, (uint32_t)(mask >> 32));
+__device__ __forceinline__ void t_store_cold(const TPool& pl, uint32_t j, uint64_t mask, const TInst& in) {
+    *reinterpret_cast<uint2*>(pl.unit(2u * j)) = make_uint2((uint32_t)mask, (uint32_t)(mask >> 32));
+    *reinterpret_cast<uint2*>(pl.unit(2u * j + 1u)) = make_uint2(in.K, in.kmin);
 }
 
 // The counter has just reached the smallest end index (clock = in.T): retire every request that
@@ -222,7 +239,7 @@ __device__ __forceinline__ void t_retire(TInst& in, TKeys& ks, TEnv& e) {
 // "reduce" with events: run whole decode steps until the clock reaches `now` (drain: until the
 // instance is empty), retiring what completes on the way; the instance is written back.
 __device__ __forceinline__ void t_advance_events(TInst& in, uint32_t j, int64_t now, bool drain, TEnv& e) {
-    TKeys ks = t_load_keys(e.pl, j);
+    TKeys ks = t_load_keys(e.pl, j, in);
     while (in.w > 0 && (drain || in.T < now)) {
         if (!drain && now <= in.tc - (int64_t)in.sw) {
             // the clock reaches `now` before anything completes (fewer steps than the longest request has tokens)
@@ -237,7 +254,7 @@ __device__ __forceinline__ void t_advance_events(TInst& in, uint32_t j, int64_t 
     }
     if (!drain && in.w == 0 && in.T < now) in.T = now;  // an idle instance starts at once
     t_store(e.hp, j, in);
-    t_store_mask(e.pl, j, ks.mask);
+    t_store_cold(e.pl, j, ks.mask, in);
 }
 
 // All live end indices move down by the counter value K (which restarts at 0).  Rare.
@@ -254,7 +271,11 @@ static __device__ __noinline__ uint32_t t_rebase(unsigned char* base, uint32_t s
 }
 
 // "map": prefill at the step boundary in.T (running decodes stall), then occupy a free slot.
-__device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& q, uint32_t req, int64_t pre, TEnv& e) {
+// `kadd`: decode steps the clock in.T is ahead of the stored step counter (a clock that was advanced lazily).
+__device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& q, uint32_t req, int64_t pre, uint32_t kadd,
+                                        TEnv& e) {
+    TKeys ks = t_load_keys(e.pl, j, in);
+    in.K += kadd;
     in.T += pre;
     const uint4 pa = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)q.arrival,
                                 (uint32_t)((uint64_t)q.arrival >> 32));
@@ -263,9 +284,9 @@ __device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& 
         in.tc += pre;
         t_push_now(e, in.T, pa, pb);
         t_store(e.hp, j, in);
+        t_store_cold(e.pl, j, ks.mask, in);
         return;
     }
-    TKeys ks = t_load_keys(e.pl, j);
     const uint32_t nblk = (in.B + 7u) >> 3;
     if (in.w == 0) in.K = 0;  // no live end index: the counter restarts
     if (in.K + q.Sm1 > kTRelMax) {
@@ -290,7 +311,7 @@ __device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& 
     in.swn = t_step(e, in.row, min(in.w + 1u, in.B));
     in.tc = in.T + (int64_t)((in.kmin >> 7) - in.K) * (int64_t)in.sw;
     t_store(e.hp, j, in);
-    t_store_mask(e.pl, j, ks.mask);
+    t_store_cold(e.pl, j, ks.mask, in);
 }
 
 // Per-request side outputs of a rejection (dump rows, per-model counts); rare.
@@ -307,14 +328,15 @@ struct ThreadSmem {
     uint4* qa;           // [kTQueue][32]
     uint2* qb;
     int64_t* qf;
+    uint2* rowtab;        // [n_rows] prefill base, prefill slope
     unsigned char* hpool; // hot part of the instances
     unsigned char* pool;  // cold part (shared-memory mode)
 };
 __host__ __device__ inline uint32_t t_hot_units(uint32_t n_models) { return ((n_models + 7u) >> 3) + n_models + 2u; }
-__host__ __device__ inline size_t t_fixed_smem(uint32_t n_models) {
-    return (size_t)t_hot_units(n_models) * 512u + (size_t)kTQueue * 32 * (16 + 8 + 8);
+__host__ __device__ inline size_t t_fixed_smem(uint32_t n_models, uint32_t n_rows) {
+    return (size_t)t_hot_units(n_models) * 512u + (size_t)kTQueue * 32 * (16 + 8 + 8) + (((size_t)n_rows * 8u + 15u) & ~(size_t)15u);
 }
-__device__ __forceinline__ ThreadSmem t_carve(unsigned char* base, uint32_t n_models, uint32_t hot_bytes) {
+__device__ __forceinline__ ThreadSmem t_carve(unsigned char* base, uint32_t n_models, uint32_t n_rows, uint32_t hot_bytes) {
     ThreadSmem s;
     s.hot = base;
     base += (size_t)t_hot_units(n_models) * 512u;
@@ -324,6 +346,8 @@ __device__ __forceinline__ ThreadSmem t_carve(unsigned char* base, uint32_t n_mo
     base += (size_t)kTQueue * 32 * 8;
     s.qf = reinterpret_cast<int64_t*>(base);
     base += (size_t)kTQueue * 32 * 8;
+    s.rowtab = reinterpret_cast<uint2*>(base);
+    base += ((size_t)n_rows * 8u + 15u) & ~(size_t)15u;
     s.hpool = base;
     base += hot_bytes;
     s.pool = base;
@@ -357,16 +381,19 @@ enum : uint32_t { kLaneIdle = 0, kLaneScan = 1, kLaneWait = 2, kLaneDone = 3 };
 // on) and distributor rounds (for the lanes that stand at a request which needs one), and starts a
 // round when `theta` lanes wait or nobody can scan.
 template <bool OPT>
-__global__ void __launch_bounds__(32, 1)
+__global__ void __launch_bounds__(32, kTBlocksPerSM)
 eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_bytes, const uint32_t hot_bytes,
                    const uint32_t theta, unsigned char* const arena) {
     // arena: the instances' state lives in global memory (one region of pool_bytes per warp, kept hot by
     // L1/L2) instead of shared memory, which leaves room for many more resident warps; null = shared memory
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    const ThreadSmem sm = t_carve(smem_raw, P.n_models, hot_bytes);
+    const ThreadSmem sm = t_carve(smem_raw, P.n_models, P.n_rows, hot_bytes);
     unsigned char* const pool = arena ? arena + (size_t)blockIdx.x * pool_bytes : sm.pool;
     const uint32_t lane = threadIdx.x;
     if (P.stall_test) return;  // test hook: nothing is scored, every valid candidate keeps its "not scored" mark
+    for (uint32_t r = lane; r < P.n_rows; r += 32u)
+        sm.rowtab[r] = make_uint2((uint32_t)P.rows[r * kRowStride + 0], (uint32_t)P.rows[r * kRowStride + 1]);
+    __syncwarp();
 
     const uint32_t pool_units = pool_bytes / 16u;
     const bool use_mask = P.class_mask != nullptr && P.n_classes <= 32;
@@ -383,6 +410,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
     e.qa = sm.qa + lane;
     e.qb = sm.qb + lane;
     e.rows = P.rows;
+    e.rowtab = sm.rowtab;
     e.ls = &ls;
     e.P = &P;
     e.qn = 0;
@@ -439,7 +467,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                     n_i = P.offsets[cand + 1] - lo;
                     uint32_t rng_lo[MAASO_MAX_MODELS], rng_hi[MAASO_MAX_MODELS], min_pre[MAASO_MAX_MODELS], min_step[MAASO_MAX_MODELS];
                     for (int m = 0; m < MAASO_MAX_MODELS; m++) { rng_lo[m] = 0xFFu; rng_hi[m] = 0u; min_pre[m] = 0xFFFFFFFFu; min_step[m] = 0xFFFFFFFFu; }
-                    uint32_t ko = n_i, so = 0;  // cold units: one per instance, then the key blocks
+                    uint32_t ko = 2u * n_i, so = 0;  // cold units: two per instance, then the key blocks
                     for (uint32_t j = 0; j < n_i; j++) {
                         const uint32_t word = P.inst[lo + j];
                         const uint32_t m = word & 0xFu, B = (word >> 12) & 0xFFu;
@@ -452,10 +480,11 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                         in.K = 0; in.kmin = 0xFFFFFFFFu;
                         in.stepB = (uint32_t)P.rows[row * kRowStride + 1 + B];
                         in.swn = (uint32_t)P.rows[row * kRowStride + 2];
-                        if (ko + 2u * nblk + 2u > cap_units || 3u * (j + 1u) > hot_cap) { status = MAASO_CAND_ETIMEOUT; break; }  // cannot happen: sized by the validation kernel
+                        if (ko + 2u * nblk + 2u > cap_units || 2u * (j + 1u) > hot_cap) { status = MAASO_CAND_ETIMEOUT; break; }  // cannot happen: sized by the validation kernel
                         t_store(e.hp, j, in);
                         const uint64_t mask = B >= 64u ? 0ull : (~0ull << B);
-                        *e.pl.unit(j) = make_uint4((uint32_t)mask, (uint32_t)(mask >> 32), ko | (so << 16), 0u);
+                        *e.pl.unit(2u * j) = make_uint4((uint32_t)mask, (uint32_t)(mask >> 32), ko | (so << 16), 0u);
+                        *e.pl.unit(2u * j + 1u) = make_uint4(0u, 0xFFFFFFFFu, 0u, 0u);
                         for (uint32_t u = 0; u < 2u * nblk; u++) {
                             const uint32_t s0 = (kTEndEmpty << 7) | (4u * u);
                             *e.pl.unit(ko + u) = make_uint4(s0, s0 + 1u, s0 + 2u, s0 + 3u);
@@ -644,7 +673,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
             const uint32_t act = __ballot_sync(kFullMaskT, state == kLaneScan);
             if (wl != 0u && ((uint32_t)__popc(wl) >= theta || act == 0u)) {
                 // statistics of completed requests, all lanes together
-                if (__any_sync(kFullMaskT, e.qn >= 3u)) t_flush_now(e);
+                if (__any_sync(kFullMaskT, e.qn >= (uint32_t)(kTQueue - 1))) t_flush_now(e);
                 if (state == kLaneWait) {
                     const uint32_t req = pos;
                     const uint4* const full = cooked + (size_t)req * kCookedWords;
@@ -668,7 +697,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                         uint32_t lb1j = 0xFFFFFFFFu;
                         for (uint32_t j = j_lo; j < j_hi; j++) {
                             TInst in;
-                            t_load(e.hp, j, in);
+                            t_load(e.hp, e.rowtab, j, in);
                             if (in.model != q.model) continue;
                             // "reduce": where the instance's clock stands once it has reached `now`
                             int64_t T = in.T;
@@ -709,28 +738,31 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                             pending = false;
                         } else {
                             TInst in;
-                            t_load(e.hp, bj, in);
+                            t_load(e.hp, e.rowtab, bj, in);
+                            bool admit = true;
+                            uint32_t kadd = 0;
                             if ((best >> 63) == 0) {
                                 in.T = bT;  // the clock as the prediction saw it
-                                in.K += bk;
-                                t_admit(in, bj, q, req, bpre, e);
-                                rej_sum -= q.rej;
-                                pending = false;
-                                lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
+                                kadd = bk;
                             } else {
                                 // every capable instance is full: wait until the chosen slot frees
                                 now = in.tc;
                                 if (!OPT) {
                                     tries++;  // the second round, counted only
                                     t_advance_events(in, bj, now, false, e);
-                                    t_admit(in, bj, q, req, bpre, e);
-                                    rej_sum -= q.rej;
-                                    pending = false;
-                                    lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
-                                } else if (tries >= kAttemptCap) {
-                                    status = MAASO_CAND_ELOOP;
-                                    pending = false;
+                                } else {
+                                    admit = false;
+                                    if (tries >= kAttemptCap) {
+                                        status = MAASO_CAND_ELOOP;
+                                        pending = false;
+                                    }
                                 }
+                            }
+                            if (admit) {
+                                t_admit(in, bj, q, req, bpre, kadd, e);
+                                rej_sum -= q.rej;
+                                pending = false;
+                                lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
                             }
                         }
                         if (lb1 != INT64_MAX)
@@ -747,7 +779,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                     if (status == 0) {
                         for (uint32_t j = 0; j < n_i; j++) {
                             TInst in;
-                            t_load(e.hp, j, in);
+                            t_load(e.hp, e.rowtab, j, in);
                             if (in.w > 0) t_advance_events(in, j, 0, true, e);
                         }
                     }
@@ -768,8 +800,9 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
 cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_bytes, uint32_t hot_bytes, uint32_t theta,
                                void* arena, cudaStream_t stream) {
     auto kernel = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_thread_kernel<true> : eval_thread_kernel<false>;
-    const size_t smem = (arena ? 0 : (size_t)pool_bytes) + hot_bytes + t_fixed_smem(P.n_models);
+    const size_t smem = (arena ? 0 : (size_t)pool_bytes) + hot_bytes + t_fixed_smem(P.n_models, P.n_rows);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
     kernel<<<grid, 32, smem, stream>>>(P, pool_bytes, hot_bytes, theta, static_cast<unsigned char*>(arena));
     return cudaGetLastError();
@@ -777,14 +810,15 @@ cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_byte
 
 int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, uint32_t hot_bytes, bool in_smem) {
     auto kernel = (P.flags & MAASO_FLAG_PRED_OPTIMISTIC) ? eval_thread_kernel<true> : eval_thread_kernel<false>;
-    const size_t smem = (in_smem ? (size_t)pool_bytes : 0) + hot_bytes + t_fixed_smem(P.n_models);
+    const size_t smem = (in_smem ? (size_t)pool_bytes : 0) + hot_bytes + t_fixed_smem(P.n_models, P.n_rows);
     cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, 32, smem) != cudaSuccess) return 1;
     return n < 1 ? 1 : n;
 }
 
-uint32_t thread_fixed_smem(uint32_t n_models) { return (uint32_t)t_fixed_smem(n_models); }
+uint32_t thread_fixed_smem(uint32_t n_models, uint32_t n_rows) { return (uint32_t)t_fixed_smem(n_models, n_rows); }
 
 // Global scratch one warp of the thread mapping needs: two entries of 24 bytes per slot, 4 slots per pool unit.
 size_t thread_scratch_per_warp(uint32_t pool_bytes) { return (size_t)(pool_bytes / 16u) * 8u * 24u; }

@@ -23,7 +23,7 @@ cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_byte
                                void* arena, cudaStream_t stream);
 int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, uint32_t hot_bytes, bool in_smem);
 size_t thread_scratch_per_warp(uint32_t pool_bytes);
-uint32_t thread_fixed_smem(uint32_t n_models);
+uint32_t thread_fixed_smem(uint32_t n_models, uint32_t n_rows);
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 cudaError_t launch_eval_block_reg(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 int occupancy_eval_block_reg(const EvalParams& P, int bucket, int tile_recs);
@@ -85,6 +85,7 @@ struct maaso_ctx {
     int promote_pct;  // share of the spare resident warps the planner may use for promotions
     int thread_arena_kb;  // thread mapping: KB of global memory per warp for the cold part of the placements' state, 0 = shared memory
     int thread_hot_kb;    // with an arena: KB of shared memory per warp for the hot part
+    bool thread_blocks_set;  // MAASO_THREAD_BLOCKS was given: also caps the resident warps per SM in arena mode
     int thread_blocks;   // one-warp blocks of the thread-mapping kernel per SM its pool is sized for
     uint32_t thread_theta;     // waiting lanes of a warp that trigger a distributor round in the thread mapping
     uint32_t thread_min_cand;  // MAASO_MAP_AUTO takes the thread mapping from this many candidates on
@@ -212,17 +213,18 @@ MAASO_API int maaso_create(maaso_ctx** out, int cuda_device) {
         int v = atoi(ta);
         if (v >= 0 && v <= 1023) ctx->thread_arena_kb = v;
     }
-    ctx->thread_hot_kb = 12;
+    ctx->thread_hot_kb = 10;
     const char* thk = getenv("MAASO_THREAD_HOT_KB");
     if (thk) {
         int v = atoi(thk);
         if (v >= 2 && v <= 128) ctx->thread_hot_kb = v;
     }
     ctx->thread_blocks = 6;
+    ctx->thread_blocks_set = false;
     const char* tb = getenv("MAASO_THREAD_BLOCKS");
     if (tb) {
         int v = atoi(tb);
-        if (v >= 1 && v <= 16) ctx->thread_blocks = v;
+        if (v >= 1 && v <= 16) { ctx->thread_blocks = v; ctx->thread_blocks_set = true; }
     }
     ctx->thread_theta = 8;
     const char* tt = getenv("MAASO_THREAD_THETA");
@@ -555,9 +557,9 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
             size_t per_block = (size_t)ctx->smem_per_sm / (size_t)ctx->thread_blocks;
             per_block = per_block > 1024 ? per_block - 1024 : 0;
             if (per_block > 227u * 1024u) per_block = 227u * 1024u;
-            const size_t fixed = thread_fixed_smem(ctx->n_models);
+            const size_t fixed = thread_fixed_smem(ctx->n_models, ctx->n_rows);
             const size_t both = per_block > fixed ? per_block - fixed : 0;
-            hot = both / 4;  // an instance has 3 hot units and about 8 cold ones
+            hot = both / 5;  // an instance has 2 hot units and about 9 cold ones
             hot -= hot % 512;
             pool = both - hot;
             pool -= pool % 512;
@@ -568,7 +570,9 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
         thread_hot = (uint32_t)hot;
         P.thread_pool_units = thread_pool / 16u;
         P.thread_hot_units = thread_hot / 16u;
-        grid_t = ctx->sm_count * occupancy_eval_thread(P, thread_pool, thread_hot, ctx->thread_arena_kb == 0);
+        int occ_t = occupancy_eval_thread(P, thread_pool, thread_hot, ctx->thread_arena_kb == 0);
+        if (ctx->thread_arena_kb > 0 && ctx->thread_blocks_set && occ_t > ctx->thread_blocks) occ_t = ctx->thread_blocks;
+        grid_t = ctx->sm_count * occ_t;
         const uint64_t max_items_t = ((uint64_t)C + 9) * n_traces;
         if ((uint64_t)grid_t > max_items_t) grid_t = (int)max_items_t;
         pay_thread = ((size_t)grid_t * (thread_scratch_per_warp(thread_pool) + (ctx->thread_arena_kb > 0 ? thread_pool : 0)) +
@@ -590,7 +594,7 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
         if (n_traces == 1 && b == kGenericBlockBucket) {
             // more than 32 instances: the thread kernel where it can run, else one block per placement
             if (o.mapping == MAASO_MAP_GROUP) used = cands->n_inst > 32;
-            if (threads) used = cands->n_inst * 19ull > P.thread_pool_units || cands->n_inst * 3ull > P.thread_hot_units;  // 22 units: an instance with 64 slots
+            if (threads) used = cands->n_inst * 20ull > P.thread_pool_units || cands->n_inst * 2ull > P.thread_hot_units;  // 22 units: an instance with 64 slots
         }
         grid_b[b - 6] = 0;
         if (!used) continue;

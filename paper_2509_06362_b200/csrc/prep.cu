@@ -13,7 +13,7 @@ __global__ void prep_kernel(const EvalParams P) {
     if (c >= P.n_cand) return;
     const uint32_t lo = P.offsets[c], hi = P.offsets[c + 1];
     uint32_t status = 0, n = 0, sum_b = 0;
-    uint32_t units = 0;  // thread mapping: 16-byte units of cold instance state (per instance 1 + key blocks + minima)
+    uint32_t units = 0;  // thread mapping: 16-byte units of cold instance state (per instance 2 + key blocks + minima)
     uint64_t supply = 0; // decode tokens per second the placement can produce with every slot busy
     const bool variant = (P.flags & (MAASO_FLAG_ENGINE_FROZEN | MAASO_FLAG_TBT_MAXGAP | MAASO_FLAG_INSTANCE_QUEUES)) != 0;
     const bool threads_ok = !variant && (P.mapping == MAASO_MAP_THREAD || P.mapping == MAASO_MAP_AUTO);
@@ -34,7 +34,7 @@ __global__ void prep_kernel(const EvalParams P) {
                     continue;
                 }
                 sum_b += b;
-                units += 1u + 2u * ((b + 7u) >> 3) + 2u;
+                units += 2u + 2u * ((b + 7u) >> 3) + 2u;
                 supply += (uint64_t)b * 1000000ull / (uint64_t)P.rows[(m * P.n_strategies + s) * kRowStride + 1 + b];
                 devsum += (uint64_t)P.devices[s];
                 if (P.devices[s] < P.min_devices[m]) status |= MAASO_CAND_EMEMFIT;
@@ -47,7 +47,7 @@ __global__ void prep_kernel(const EvalParams P) {
     if (!status) {
         if (threads_ok) {
             // as many lanes per item as placements of this size fit the warp's pools
-            const uint32_t fit = n ? min(P.thread_pool_units / units, P.thread_hot_units / (3u * n)) : 32u;
+            const uint32_t fit = n ? min(P.thread_pool_units / units, P.thread_hot_units / (2u * n)) : 32u;
             const uint32_t lanes[9] = {32, 24, 16, 12, 8, 6, 4, 2, 1};
             for (int i = 0; i < 9; i++)
                 if (fit >= lanes[i]) { bt = kThreadBucket0 + i; break; }
