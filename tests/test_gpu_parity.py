@@ -916,6 +916,52 @@ def test_several_traces_in_one_pass(ctx, oracle_mod, flags):
         ctx.free_trace(h)
 
 
+@pytest.mark.parametrize("flags", [0, 1])
+def test_several_traces_in_one_pass_on_the_thread_kernel(oracle_mod, monkeypatch, flags):
+    """Several traces in one pass where the thread kernel scores them: placements of more than 32
+    instances go there whatever the batch (no ETOOMANY below 129 instances), and with the routing
+    threshold at zero the loaded rest of the batch follows; records, per-model rejection counts and
+    histograms must equal the oracle's for every trace."""
+    import torch
+    import paper_2509_06362_b200 as m
+    prof = gen.profile_multimodel(0)
+    rng = np.random.default_rng(21)
+    lists = []
+    for n_i in (33, 40, 128, 5, 1, 64, 9, 2):
+        lists.append([(int(rng.integers(2)), 0, int(rng.choice([1, 2, 4, 8, 16, 32, 64]))) for _ in range(n_i)])
+    cfg = gen.make_config("multimodel", n_cand=300, n_req=10)
+    off, inst = gen.candidates_from_lists(lists)
+    off = np.concatenate([off, off[-1] + cfg["offsets"][1:]]).astype(np.uint32)
+    inst = np.concatenate([inst, cfg["inst"]]).astype(np.uint32)
+    classes = cfg["classes"]
+    traces_np = [gen.make_trace(900 - 150 * i, 40.0 * (i + 1), 30 + i, model_mix=(0.6, 0.3, 0.1)) for i in range(3)]
+    n_cand, n_tr = len(off) - 1, len(traces_np)
+    for min_cand in ("0", "1000000"):        # the whole batch on the thread kernel / only the large placements
+        monkeypatch.setenv("MAASO_THREAD_MIN_CAND", min_cand)
+        c = m.Context(0)
+        c.load_profile(prof)
+        handles = [c.load_trace(t, classes) for t in traces_np]
+        rbm = torch.full((n_tr * n_cand, 16), 77, dtype=torch.int32, device="cuda")
+        hist = torch.full((n_tr * n_cand, 64), 77, dtype=torch.int32, device="cuda")
+        c.set_timing(True)
+        out = c.eval_placements_multi(handles, c.to_device(off), c.to_device(inst), 1024, None, flags,
+                                      rejected_by_model=rbm, ttft_hist=hist)
+        torch.cuda.synchronize()
+        tm = c.get_timing()
+        got = c.results_to_numpy(out).reshape(n_tr, n_cand)
+        rbm_h = rbm.cpu().numpy().view(np.uint32).reshape(n_tr, n_cand, 16)
+        hist_h = hist.cpu().numpy().view(np.uint32).reshape(n_tr, n_cand, 64)
+        for t, tr in enumerate(traces_np):
+            want = oracle_mod.eval_placements(prof, tr, classes, off, inst, 1024, None, flags)
+            assert (want["status"] == 0).all()
+            assert_records_equal(got[t], want, f"trace {t}, routing threshold {min_cand}")
+            if flags == 0:
+                assert (rbm_h[t] == oracle_mod.rejected_by_model(prof, tr, classes, off, inst, 1024)).all()
+                assert (hist_h[t] == oracle_mod.ttft_hist(prof, tr, classes, off, inst, 1024)).all()
+        assert tm["thread_ms"] > 0.0 and tm["block_ms"] < 0.5
+        c.close()
+
+
 def test_several_traces_limits(ctx):
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny", n_req=60)
