@@ -219,6 +219,9 @@ MAASO_API void maaso_free_trace(maaso_ctx *ctx, maaso_trace *trace);
  * through the distributor (Sec. IV-F) and per-instance continuous batching with virtual
  * slots (Sec. V-A), and write one record per candidate to out_results (device,
  * [n_cand]).  Work is enqueued on `cuda_stream` (a cudaStream_t, NULL = default stream).
+ * opts->mapping chooses the kernel: MAASO_MAP_AUTO (default) lets the library route the batch (large
+ * batches of placements that the trace overloads go to the thread kernel, the rest to the lane groups;
+ * placements of more than 32 instances always to the thread kernel); the records do not depend on it.
  * The context's scratch memory grows on demand (this may allocate and synchronise on the
  * first call or when a batch is larger than any before). */
 MAASO_API int maaso_eval_placements(maaso_ctx *ctx, const maaso_trace *trace, const maaso_cand_batch *cands,
@@ -231,8 +234,9 @@ MAASO_API int maaso_eval_placements(maaso_ctx *ctx, const maaso_trace *trace, co
  * out_results[t * n_cand + c]; opts->rejected_by_model and opts->ttft_hist, if given, are laid out
  * the same way ([n_traces * n_cand][...]).  Each record equals what maaso_eval_placements returns
  * for that trace alone; scoring them together lets small candidate sets fill the GPU.  Lane-group
- * mapping only: dump buffers and MAASO_MAP_BLOCK are refused, a placement with more than 32
- * instances gets MAASO_CAND_ETOOMANY.  Enqueued on cuda_stream. */
+ * and thread mappings only: dump buffers and MAASO_MAP_BLOCK are refused.  With the default engine a
+ * placement of more than 32 instances is scored by the thread kernel; with MAASO_MAP_GROUP or one of
+ * the other engines it gets MAASO_CAND_ETOOMANY.  Enqueued on cuda_stream. */
 MAASO_API int maaso_eval_placements_multi(maaso_ctx *ctx, const maaso_trace *const *traces, uint32_t n_traces,
                                           const maaso_cand_batch *cands, const maaso_eval_opts *opts,
                                           maaso_result *out_results, void *cuda_stream);
@@ -365,7 +369,7 @@ MAASO_API int maaso_topk_noalloc(const maaso_result *results, uint64_t n_cand, u
  * events of the most recent calls and reports milliseconds (0 for a family that did not
  * run).  Off by default; costs a few event records per call when on. */
 typedef struct {
-    float prep_ms;  /* validation + bucket sort (+ dump buffer fill) */
+    float prep_ms;  /* validation, routing + bucket sort (+ dump buffer fill) */
     float group_ms; /* lane-group scoring kernel */
     float block_ms; /* block-layout scoring kernels */
     float topk_ms;  /* all passes of the last maaso_topk */
