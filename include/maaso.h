@@ -72,15 +72,18 @@ extern "C" {
                                       admission to the request's finish time, first token = admission +
                                       prefill, one token every step[running + 1] afterwards; later
                                       admissions slow nobody down and prefills stall nobody.  Same
-                                      distributor.  Lane-group mapping only: MAASO_MAP_BLOCK is refused and
-                                      a placement with more than 32 instances gets MAASO_CAND_ETOOMANY;
-                                      finish times must stay below 2^57 us (else MAASO_CAND_ELOOP). */
+                                      distributor.  Lane-group code only: MAASO_MAP_BLOCK and
+                                      MAASO_MAP_THREAD are refused; a placement with more than 32 instances
+                                      (up to MAASO_MAX_INSTANCES) is replayed by one warp, four instances
+                                      per lane; finish times must stay below 2^57 us (else
+                                      MAASO_CAND_ELOOP). */
 
 #define MAASO_FLAG_TBT_MAXGAP 4u /* the TBT term of the hit test (Phi_S indicator) looks at the largest gap
                                     between two consecutive tokens of a request, prefill stalls included,
                                     instead of the mean gap; a request of one token has no gap.  The
                                     distributor's prediction is unchanged.  Same limits as
-                                    MAASO_FLAG_ENGINE_FROZEN (lane-group mapping, at most 32 instances). */
+                                    MAASO_FLAG_ENGINE_FROZEN (lane-group code; one warp per placement
+                                    beyond 32 instances). */
 
 #define MAASO_FLAG_INSTANCE_QUEUES 8u /* a request whose chosen instance is full queues THERE (Sec. II-A: requests
                                         beyond the batch cap wait in the instance's queue) instead of at the
@@ -99,8 +102,9 @@ extern "C" {
 /* maaso_eval_opts.mapping */
 #define MAASO_MAP_AUTO 0u   /* the library chooses: MAASO_MAP_THREAD where it exists, else MAASO_MAP_GROUP */
 #define MAASO_MAP_BLOCK 1u  /* one thread block per candidate, one warp per instance, lanes = slots */
-#define MAASO_MAP_GROUP 2u  /* one lane per instance, groups of lanes per candidate (<= 32 instances; one block
-                               per candidate beyond that) */
+#define MAASO_MAP_GROUP 2u  /* one lane per instance, groups of lanes per candidate (<= 32 instances; beyond
+                               that one block per candidate, or, with several traces in one pass, one warp
+                               per candidate with four instances per lane) */
 #define MAASO_MAP_THREAD 3u /* one thread per candidate, looping over the instances of the request's model;
                                default engine only (flags 0 or MAASO_FLAG_PRED_OPTIMISTIC), any instance count */
 
@@ -236,7 +240,8 @@ MAASO_API int maaso_eval_placements(maaso_ctx *ctx, const maaso_trace *trace, co
  * for that trace alone; scoring them together lets small candidate sets fill the GPU.  Lane-group
  * and thread mappings only: dump buffers and MAASO_MAP_BLOCK are refused.  With the default engine a
  * placement of more than 32 instances is scored by the thread kernel; with MAASO_MAP_GROUP or one of
- * the other engines it gets MAASO_CAND_ETOOMANY.  Enqueued on cuda_stream. */
+ * the other engines one warp replays it with the lane-group code (four instances per lane).  No engine
+ * and no mapping refuses a placement of MAASO_MAX_INSTANCES instances or fewer.  Enqueued on cuda_stream. */
 MAASO_API int maaso_eval_placements_multi(maaso_ctx *ctx, const maaso_trace *const *traces, uint32_t n_traces,
                                           const maaso_cand_batch *cands, const maaso_eval_opts *opts,
                                           maaso_result *out_results, void *cuda_stream);
@@ -371,7 +376,7 @@ MAASO_API int maaso_topk_noalloc(const maaso_result *results, uint64_t n_cand, u
 typedef struct {
     float prep_ms;  /* validation, routing + bucket sort (+ dump buffer fill) */
     float group_ms; /* lane-group scoring kernel */
-    float block_ms; /* block-layout scoring kernels */
+    float block_ms; /* block-layout scoring kernels and the one-warp-per-placement kernel for more than 32 instances */
     float topk_ms;  /* all passes of the last maaso_topk */
     float thread_ms; /* thread-mapping scoring kernel */
 } maaso_timing;

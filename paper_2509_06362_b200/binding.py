@@ -217,10 +217,10 @@ def maaso_eval_placements(ctx, trace, offsets, inst, budget, out_results, class_
 
 
 def maaso_eval_placements_multi(ctx, traces, offsets, inst, budget, out_results, class_mask=None, flags=0,
-                                rejected_by_model=None, ttft_hist=None, stream=None):
+                                rejected_by_model=None, ttft_hist=None, stream=None, mapping=MAP_AUTO):
     """traces: sequence of trace handles; out_results: uint8 CUDA tensor of len(traces)*n_cand*128 bytes."""
     b = _batch(offsets, inst, class_mask, budget)
-    o = _EvalOpts(int(flags), MAP_AUTO, 0, 0, None, None, None, None, _ptr(rejected_by_model), _ptr(ttft_hist))
+    o = _EvalOpts(int(flags), int(mapping), 0, 0, None, None, None, None, _ptr(rejected_by_model), _ptr(ttft_hist))
     arr = (C.c_void_p * len(traces))(*[t if isinstance(t, int) else (t.value if hasattr(t, "value") else t) for t in traces])
     _check(_lib.maaso_eval_placements_multi(ctx, arr, len(traces), C.byref(b), C.byref(o), _ptr(out_results),
                                             _stream_ptr(stream)), "maaso_eval_placements_multi", ctx)
@@ -409,7 +409,7 @@ class Context:
         return (out, dumps) if dump_idx is not None else out
 
     def eval_placements_multi(self, traces, offsets, inst, budget, class_mask=None, flags=0, out=None, stream=None,
-                              rejected_by_model=None, ttft_hist=None):
+                              rejected_by_model=None, ttft_hist=None, mapping=MAP_AUTO):
         """One pass over several traces (at most 16, same SLO classes).  Returns a uint8 tensor
         [len(traces), n_cand, 128]: block t holds the records for traces[t]."""
         torch = self.torch
@@ -417,7 +417,7 @@ class Context:
         if out is None:
             out = torch.empty((len(traces), n_cand, 128), dtype=torch.uint8, device=self.device)
         maaso_eval_placements_multi(self.handle, [t.handle for t in traces], offsets, inst, budget, out, class_mask,
-                                    flags, rejected_by_model, ttft_hist, stream)
+                                    flags, rejected_by_model, ttft_hist, stream, mapping)
         return out
 
     def eval_placements_host(self, trace, offsets, inst, budget, class_mask=None, flags=0,

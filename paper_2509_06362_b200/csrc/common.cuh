@@ -18,14 +18,16 @@ constexpr long long kWaitCycles = 4000000000ll;  // bound on any device-side wai
 // 9:    block layout with 16 warps striding over up to 128 instances, state in shared memory
 // 10..18: thread mapping, by how many lanes of a warp work at a time (32, 24, 16, 12, 8, 6, 4, 2, 1:
 //        the larger the placements, the fewer fit the warp's pools)
-constexpr int kNumBuckets = 19;
+constexpr int kNumBuckets = 20;
 constexpr int kGenericBlockBucket = 9;
 constexpr int kThreadBucket0 = 10;  // buckets 10..18: the thread mapping, by lanes per warp
+constexpr int kThreadBuckets = 9;
+constexpr int kWideBucket = 19;     // 33..128 instances under the engines of the lane-group code: one warp per placement
 constexpr int kCostBins = 256;   // bin 0 = most expensive (largest total batch cap)
 constexpr int kCounterWords = 16384;  // counters | work counters | histograms + cursors, cleared per call
 // histogram sets (rows of kCostBins words in EvalParams::hist): candidates that can only go to a lane-group
 // or block bucket, only to a thread bucket, or either way (counted once per side); then the write cursors
-constexpr int kHistOnlyG = 0, kHistBothG = 10, kHistOnlyT = 20, kHistBothT = 29, kHistCursor = 38;
+constexpr int kHistOnlyG = 0, kHistBothG = 10, kHistOnlyT = 20, kHistBothT = 29, kHistWide = 38, kHistCursor = 39;
 constexpr int kHistRows = kHistCursor + kNumBuckets;
 // counters beside the bucket counts (EvalParams::bucket_count[0..31])
 constexpr int kCtrBoth = 24, kCtrLoaded = 25, kCtrCut = 26, kCtrUseThreads = 27;
@@ -264,7 +266,7 @@ struct EvalParams {
     maaso_result* out;
     uint32_t* bucket_count;  // [32]: candidates per bucket after planning, and the kCtr* counters
     uint32_t* bucket_list;   // [kNumBuckets][n_cand], each bucket sorted by decreasing cost estimate
-    uint32_t* work_ctr;      // [16]: next work item of the block kernels [1..4] and of the thread buckets [bucket - 10]... see the kernels
+    uint32_t* work_ctr;      // [16]: next work item of the block kernels [1..4], of the thread buckets [5..13], of the wide kernel [14]
     uint32_t* hist;          // [kHistRows][kCostBins]: candidates per cost bin by set, then write cursors
     uint32_t* code;          // [n_cand] lane-group / block bucket << 8 | cost bin, 0xFFFFFFFF if none
     uint32_t* code2;         // [n_cand] thread bucket << 8 | cost bin, 0xFFFFFFFF if none

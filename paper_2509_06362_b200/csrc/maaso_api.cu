@@ -24,6 +24,9 @@ cudaError_t launch_eval_thread(const EvalParams& P, int grid, uint32_t pool_byte
 int occupancy_eval_thread(const EvalParams& P, uint32_t pool_bytes, uint32_t hot_bytes, bool in_smem);
 size_t thread_scratch_per_warp(uint32_t pool_bytes);
 uint32_t thread_fixed_smem(uint32_t n_models, uint32_t n_rows);
+cudaError_t launch_eval_wide(const EvalParams& P, int grid, cudaStream_t stream);
+int occupancy_eval_wide(const EvalParams& P);
+size_t wide_scratch_per_warp();
 cudaError_t launch_eval_block(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 cudaError_t launch_eval_block_reg(const EvalParams& P, int bucket, int grid, int tile_recs, cudaStream_t stream);
 int occupancy_eval_block_reg(const EvalParams& P, int bucket, int tile_recs);
@@ -607,6 +610,20 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
         if (need > pay_entries) pay_entries = need;
     }
 
+    // placements of more than 32 instances under the other engines, or with several traces where the thread
+    // kernel is not used: one warp per placement with the lane-group code
+    int grid_w = 0;
+    if (o.mapping != MAASO_MAP_BLOCK && cands->n_inst > 32 && (variant || n_traces > 1)) {
+        // at most as many warps as the lane-group grid has blocks: a warp's scratch is a lane-group block's
+        int occ_w = occupancy_eval_wide(P);
+        if (occ_w > 4) occ_w = 4;
+        grid_w = ctx->sm_count * occ_w;
+        const uint64_t max_items_w = (uint64_t)C * n_traces;
+        if ((uint64_t)grid_w > max_items_w) grid_w = (int)max_items_w;
+        const size_t need = ((size_t)grid_w * wide_scratch_per_warp() + sizeof(Payload) - 1) / sizeof(Payload);
+        if (need > pay_entries) pay_entries = need;
+    }
+
     // scratch layout: counters | bucket lists | dump rows | payload
     size_t off = 0;
     const size_t off_counters = off; off = align_up(off + kCounterWords * 4, 256);
@@ -668,6 +685,11 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
         if (e != cudaSuccess) return cuda_fail(ctx, e, "thread kernel launch");
     }
     if (ctx->timing) cudaEventRecord(ctx->ev[6], stream);
+    if (grid_w > 0) {
+        e = launch_eval_wide(P, grid_w, stream);
+        launches++;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "wide kernel launch");
+    }
     for (int b = 6; b <= kGenericBlockBucket; b++) {
         if (grid_b[b - 6] == 0) continue;
         e = b < kGenericBlockBucket ? launch_eval_block_reg(P, b, grid_b[b - 6], tile, stream)

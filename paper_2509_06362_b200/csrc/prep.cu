@@ -55,13 +55,10 @@ __global__ void prep_kernel(const EvalParams P) {
         if (P.mapping == MAASO_MAP_BLOCK) bg = n <= 2 ? 6 : (n <= 4 ? 7 : (n <= 8 ? 8 : kGenericBlockBucket));
         else if (groups_ok && n <= 32) bg = n <= 1 ? 0 : 32 - __clz((int)(n - 1));
         // More than 32 instances: the thread mapping if it can hold the placement, else one block per
-        // placement (default engine, one trace); the other engines and several traces in one pass
-        // exist in the lane-group and thread kernels only.
+        // placement (default engine, one trace), else (the other engines, several traces in one pass)
+        // one warp per placement with the lane-group code.
         if (n > 32 && bt >= 0) bg = -1;
-        if (bg < 0 && bt < 0) {
-            if (!variant && P.n_traces <= 1) bg = kGenericBlockBucket;
-            else status = MAASO_CAND_ETOOMANY;
-        }
+        if (bg < 0 && bt < 0) bg = (!variant && P.n_traces <= 1) ? kGenericBlockBucket : kWideBucket;
     }
     if (P.dump_row) P.dump_row[c] = -1;
     const uint32_t n_traces = P.n_traces > 1 ? P.n_traces : 1u;
@@ -93,6 +90,8 @@ __global__ void prep_kernel(const EvalParams P) {
         // thread mapping does for next to nothing
         atomicAdd(&P.bucket_count[kCtrBoth], 1u);
         if ((uint64_t)P.demand_tok_s >= 2ull * supply) atomicAdd(&P.bucket_count[kCtrLoaded], 1u);
+    } else if (bg == kWideBucket) {
+        atomicAdd(&P.hist[kHistWide * kCostBins + bin], 1u);
     } else if (bg >= 0) {
         atomicAdd(&P.hist[(kHistOnlyG + bg) * kCostBins + bin], 1u);
     } else {
@@ -132,9 +131,10 @@ __global__ void __launch_bounds__(kCostBins) plan_kernel(const EvalParams P) {
     uint32_t cnt[kNumBuckets];
     for (int b = 0; b < kThreadBucket0; b++)
         cnt[b] = P.hist[(kHistOnlyG + b) * kCostBins + bin] + (use_threads ? 0u : P.hist[(kHistBothG + b) * kCostBins + bin]);
-    for (int b = kThreadBucket0; b < kNumBuckets; b++)
+    for (int b = kThreadBucket0; b < kThreadBucket0 + kThreadBuckets; b++)
         cnt[b] = P.hist[(kHistOnlyT + b - kThreadBucket0) * kCostBins + bin] +
                  (use_threads ? P.hist[(kHistBothT + b - kThreadBucket0) * kCostBins + bin] : 0u);
+    cnt[kWideBucket] = P.hist[kHistWide * kCostBins + bin];
     uint32_t cut = 0;  // bins below `cut` are promoted
     uint32_t narrow = 0;
     for (int b = 0; b < 5; b++) narrow += cnt[b];

@@ -99,9 +99,7 @@ def test_bursty_optimistic_shows_cascades(ctx, oracle_mod, mapping):
     assert total_cascade > 0
 
 
-@pytest.mark.parametrize("mapping", MAPPINGS)
-def test_large_placements_over_32_instances(ctx, oracle_mod, mapping):
-    """Candidates with up to 128 instances (budget 128): the strided block path."""
+def _large_placements():
     prof = gen.profile_multimodel(0)
     rng = np.random.default_rng(3)
     lists = []
@@ -116,6 +114,13 @@ def test_large_placements_over_32_instances(ctx, oracle_mod, mapping):
     tr = gen.make_trace(4000, 400.0, 9, model_mix=(0.6, 0.3, 0.1), class_mix=(0.45, 0.27, 0.18, 0.10))
     classes = gen.make_classes([(500_000, 50_000, None), (2_000_000, 150_000, None),
                                 (None, None, 180_000_000), (30_000_000, None, 600_000_000)])
+    return prof, off, inst, tr, classes
+
+
+@pytest.mark.parametrize("mapping", MAPPINGS)
+def test_large_placements_over_32_instances(ctx, oracle_mod, mapping):
+    """Candidates with up to 128 instances (budget 128): the thread kernel, the block path."""
+    prof, off, inst, tr, classes = _large_placements()
     idx = np.array([1, 4, 6], dtype=np.uint32)
     want, wd = oracle_mod.eval_placements(prof, tr, classes, off, inst, 1024, dump_idx=idx)
     got, gd = gpu_eval(ctx, prof, tr, classes, off, inst, 1024, mapping=mapping, dump_idx=idx)
@@ -123,6 +128,42 @@ def test_large_placements_over_32_instances(ctx, oracle_mod, mapping):
     assert_records_equal(got, want, "large placements")
     for k in wd:
         assert (gd[k] == wd[k]).all(), k
+
+
+@pytest.mark.parametrize("flags", [0, 1, 2, 3, 4, 5, 6, 8, 9, 12])
+def test_large_placements_over_32_instances_every_engine(ctx, oracle_mod, flags):
+    """No engine stops at 32 instances: the optimistic estimate, the fixed-speed engine, the largest-gap
+    test and per-instance queues (and combinations) on placements of 33 to 128 instances, records and
+    per-request times against the oracle; no ETOOMANY below 129 instances."""
+    prof, off, inst, tr, classes = _large_placements()
+    idx = np.array([0, 4, 6], dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(prof, tr, classes, off, inst, 1024, None, flags, dump_idx=idx)
+    got, gd = gpu_eval(ctx, prof, tr, classes, off, inst, 1024, None, flags, 0, dump_idx=idx)
+    assert (want["status"] == 0).all()
+    assert_records_equal(got, want, f"large placements, flags {flags}")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), (k, flags)
+
+
+@pytest.mark.parametrize("flags,mapping", [(0, 2), (2, 0), (8, 0), (4, 0)])
+def test_large_placements_several_traces_in_one_pass(ctx, oracle_mod, flags, mapping):
+    """The same placements against three traces in one call, where the thread kernel is not used (lane
+    groups forced, or one of the other engines): one warp per placement with the lane-group code."""
+    import torch
+    prof, off, inst, tr, classes = _large_placements()
+    traces_np = [tr[:1500], tr[1000:3100].copy(), tr[:700]]
+    traces_np[1]["arrival_us"] -= traces_np[1]["arrival_us"][0]
+    ctx.load_profile(prof)
+    handles = [ctx.load_trace(t, classes) for t in traces_np]
+    out = ctx.eval_placements_multi(handles, ctx.to_device(off), ctx.to_device(inst), 1024, None, flags, mapping=mapping)
+    torch.cuda.synchronize()
+    got = ctx.results_to_numpy(out).reshape(3, -1)
+    for t, trn in enumerate(traces_np):
+        want = oracle_mod.eval_placements(prof, trn, classes, off, inst, 1024, None, flags)
+        assert (want["status"] == 0).all()
+        assert_records_equal(got[t], want, f"trace {t}, flags {flags}")
+    for h in handles:
+        ctx.free_trace(h)
 
 
 @pytest.mark.parametrize("mapping", MAPPINGS)
@@ -736,7 +777,7 @@ def test_frozen_engine_node_and_multimodel_subsets(ctx, oracle_mod, flags):
 
 
 def test_frozen_engine_limits(ctx):
-    """No block mapping for this engine; placements with more than 32 instances are refused one by one."""
+    """No block mapping for this engine; more than 128 instances are refused, placement by placement."""
     import paper_2509_06362_b200 as m
     cfg = gen.make_config("tiny", n_req=50)
     ctx.load_profile(cfg["profile"])
@@ -746,12 +787,13 @@ def test_frozen_engine_limits(ctx):
         ctx.eval_placements(t, d_off, d_inst, 4, flags=2, mapping=1)
     with pytest.raises(m.MaasoError):
         ctx.eval_placements(t, d_off, d_inst, 4, flags=8, mapping=1)
-    off, inst = gen.candidates_from_lists([[(0, 0, 1)] * 33, [(0, 0, 1)] * 32])
+    off, inst = gen.candidates_from_lists([[(0, 0, 1)] * 129, [(0, 0, 1)] * 33, [(0, 0, 1)] * 32])
     import torch
-    out = ctx.eval_placements(t, ctx.to_device(off), ctx.to_device(inst), 64, flags=2)
+    out = ctx.eval_placements(t, ctx.to_device(off), ctx.to_device(inst), 256, flags=2)
     torch.cuda.synchronize()
     rec = ctx.results_to_numpy(out)
-    assert int(rec["status"][0]) == m.CAND_STATUS["ETOOMANY"] and int(rec["status"][1]) == 0
+    assert int(rec["status"][0]) == m.CAND_STATUS["ETOOMANY"]          # the limit is 128 instances, for every engine
+    assert int(rec["status"][1]) == 0 and int(rec["status"][2]) == 0
     ctx.free_trace(t)
 
 
