@@ -8,11 +8,16 @@ CSRC = os.path.join(_HERE, "csrc")
 LIB = os.environ.get("MAASO_LIB") or os.path.join(_HERE, "libmaaso.so")  # MAASO_LIB: use a prebuilt library
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-              "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--shared"]
+              "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
+OBJ_DIR = os.path.join(_HERE, "_build")
 
 
 def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
+
+
+def _headers():
+    return glob.glob(os.path.join(CSRC, "*.cuh")) + [os.path.join(os.path.dirname(_HERE), "include", "maaso.h")]
 
 
 def stale():
@@ -21,19 +26,33 @@ def stale():
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + \
-        [os.path.join(os.path.dirname(_HERE), "include", "maaso.h")]
-    return any(os.path.getmtime(d) > t for d in deps)
+    return any(os.path.getmtime(d) > t for d in sources() + _headers())
 
 
 def build(force=False, verbose=False):
-    """Compile csrc/*.cu into libmaaso.so next to this file; returns its path."""
+    """Compile csrc/*.cu into libmaaso.so next to this file; returns its path.  Every source is a
+    translation unit of its own: the objects are compiled side by side (and kept, so that a change
+    to one file recompiles that file only), then linked into one shared object."""
     if not force and not stale():
         return LIB
+    from concurrent.futures import ThreadPoolExecutor
     nvcc = os.environ.get("NVCC", "nvcc")
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    newest_header = max(os.path.getmtime(h) for h in _headers())
+
+    def compile_one(src):
+        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        if not force and os.path.exists(obj) and os.path.getmtime(obj) > max(os.path.getmtime(src), newest_header):
+            return obj
+        tmp = obj + f".{os.getpid()}.tmp"
+        subprocess.check_call([nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", tmp, src])
+        os.replace(tmp, obj)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        objs = list(pool.map(compile_one, sources()))
     tmp = LIB + f".{os.getpid()}.tmp"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + sources()
-    subprocess.check_call(cmd)
+    subprocess.check_call([nvcc, "--shared", "-o", tmp] + objs)
     os.replace(tmp, LIB)
     return LIB
 

@@ -157,13 +157,17 @@ __device__ __forceinline__ void t_flush_now(TEnv& e) {
 
 // A running request has left its instance at t_fin: queue the finish time and start the copies
 // of what it remembered.  A full queue is accounted by this lane alone first.
+// Nothing waits for the copies here, so the retirements of one visit overlap their reads.  No entry
+// is overwritten under a copy: a lane has no copy in flight when it starts a distributor round (it
+// waits for them there, long after they were issued), the only write of a round is the admission
+// at its end, and that goes to the other entry of its slot than the previous occupant's, the only
+// one of that slot a copy of the same round can read.
 __device__ __forceinline__ void t_push_slot(TEnv& e, int64_t t_fin, uint32_t pidx) {
     if (e.qn == (uint32_t)kTQueue) t_flush_now(e);
     const uint32_t j = e.qn;
     e.qf[j * 32] = t_fin;
     async_copy16(e.qa + j * 32, e.pay_a + pidx);
     async_copy8(e.qb + j * 32, e.pay_b + pidx);
-    async_commit_keep_one();
     e.qn = j + 1;
 }
 // Same for a request of one output token, which completes at admission: everything is in registers.
@@ -237,9 +241,8 @@ __device__ __forceinline__ void t_retire(TInst& in, TKeys& ks, TEnv& e) {
 }
 
 // "reduce" with events: run whole decode steps until the clock reaches `now` (drain: until the
-// instance is empty), retiring what completes on the way; the instance is written back.
-__device__ __forceinline__ void t_advance_events(TInst& in, uint32_t j, int64_t now, bool drain, TEnv& e) {
-    TKeys ks = t_load_keys(e.pl, j, in);
+// instance is empty), retiring what completes on the way.  `ks`: the instance's cold part, loaded by the caller.
+__device__ __forceinline__ void t_events(TInst& in, TKeys& ks, int64_t now, bool drain, TEnv& e) {
     while (in.w > 0 && (drain || in.T < now)) {
         if (!drain && now <= in.tc - (int64_t)in.sw) {
             // the clock reaches `now` before anything completes (fewer steps than the longest request has tokens)
@@ -253,6 +256,11 @@ __device__ __forceinline__ void t_advance_events(TInst& in, uint32_t j, int64_t 
         t_retire(in, ks, e);
     }
     if (!drain && in.w == 0 && in.T < now) in.T = now;  // an idle instance starts at once
+}
+// The same with the cold part read and everything written back.
+__device__ __forceinline__ void t_advance_events(TInst& in, uint32_t j, int64_t now, bool drain, TEnv& e) {
+    TKeys ks = t_load_keys(e.pl, j, in);
+    t_events(in, ks, now, drain, e);
     t_store(e.hp, j, in);
     t_store_cold(e.pl, j, ks.mask, in);
 }
@@ -272,9 +280,9 @@ static __device__ __noinline__ uint32_t t_rebase(unsigned char* base, uint32_t s
 
 // "map": prefill at the step boundary in.T (running decodes stall), then occupy a free slot.
 // `kadd`: decode steps the clock in.T is ahead of the stored step counter (a clock that was advanced lazily).
-__device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& q, uint32_t req, int64_t pre, uint32_t kadd,
-                                        TEnv& e) {
-    TKeys ks = t_load_keys(e.pl, j, in);
+// `ks`: the instance's cold part, loaded by the caller; everything is written back here.
+__device__ __forceinline__ void t_admit(TInst& in, TKeys& ks, uint32_t j, const CookedReq& q, uint32_t req, int64_t pre,
+                                        uint32_t kadd, TEnv& e) {
     in.K += kadd;
     in.T += pre;
     const uint4 pa = make_uint4((uint32_t)in.T, (uint32_t)((uint64_t)in.T >> 32), (uint32_t)q.arrival,
@@ -299,8 +307,9 @@ __device__ __forceinline__ void t_admit(TInst& in, uint32_t j, const CookedReq& 
     const uint32_t key = ((in.K + q.Sm1) << 7) | (gen << 6) | slot;
     *kw = key;
     const uint32_t pidx = 2u * (ks.so + slot) + gen;
-    e.pay_a[pidx] = pa;
-    e.pay_b[pidx] = pb;
+    // read once, much later, through an asynchronous copy: written past the caches' working set
+    __stcs(e.pay_a + pidx, pa);
+    __stcs(e.pay_b + pidx, pb);
     const uint32_t b = slot >> 3;
     uint32_t* const bm = e.pl.word(ks.ko + 2u * nblk + (b >> 2), b & 3u);
     *bm = min(*bm, key);
@@ -424,8 +433,10 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
         if (total == 0 || *(volatile uint32_t*)&P.work_ctr[5 + b] >= total) continue;
         const uint32_t cap_units = pool_units / L;  // what one lane may use
         const uint32_t hot_cap = hot_bytes / 16u / L;
-        e.pl.base = pool + lane * 16u;
-        e.pl.stride = L * 16u;
+        // The cold part: unit-major like the hot part in shared memory; in the arena every lane has a region
+        // of its own, so that an instance's mask, counters, keys and block minima share one or two cache lines.
+        e.pl.base = arena ? pool + (size_t)lane * cap_units * 16u : pool + lane * 16u;
+        e.pl.stride = arena ? 16u : L * 16u;
         e.hp.base = sm.hpool + lane * 16u;
         e.hp.stride = L * 16u;
         {   // scratch entries of this lane: two per slot, at most 4 slots per pool unit
@@ -559,8 +570,22 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                         lo = hi = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);  // every rejection is written out
                         hb = ldg_nc(th + kScanHdrBase);
                     } else {
-                        // first the eight class entries: most tiles of a loaded placement end here, wholly late
+                        // One round trip for the whole header: the eight class entries, the base arrival, and the
+                        // maps of class slots 0..3 and model slots 0..3 as far as this placement can need them
+                        // (which of the class maps count is known once the entries are here).  Slots 4..7 follow
+                        // in a second step for the placements that use them.
+                        const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
                         const uint4 h0 = ldg_nc(th), h1 = ldg_nc(th + 1), h2 = ldg_nc(th + 2), h3 = ldg_nc(th + 3);
+                        hb = ldg_nc(th + kScanHdrBase);
+                        uint4 ca[4], cx[4], ma[4], mx[4];
+#pragma unroll
+                        for (uint32_t k = 0; k < 4u; k++) {
+                            const bool hc = (hmask >> k) & 1u, hm = (mmask >> k) & 1u;
+                            ca[k] = hc ? ldg_nc(th + kScanHdrClassBits + 2u * k) : z4;
+                            cx[k] = hc ? ldg_nc(th + kScanHdrClassBits + 2u * k + 1u) : z4;
+                            ma[k] = hm ? ldg_nc(th + kScanHdrModelBits + 2u * k) : z4;
+                            mx[k] = hm ? ldg_nc(th + kScanHdrModelBits + 2u * k + 1u) : z4;
+                        }
                         const uint32_t hw[16] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w, h2.x, h2.y, h2.z, h2.w, h3.x, h3.y, h3.z, h3.w};
                         uint32_t livec = 0;
 #pragma unroll
@@ -568,11 +593,18 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                             const int64_t thr = (int64_t)(((uint64_t)hw[2 * k + 1] << 32) | hw[2 * k]);
                             if (((hmask >> k) & 1u) && thr >= now) livec |= 1u << k;
                         }
-                        if (livec) {
-                            hb = ldg_nc(th + kScanHdrBase);
-                            uint4 mlo = lo, mhi = lo;
+                        uint4 mlo = z4, mhi = z4;
+#pragma unroll
+                        for (uint32_t k = 0; k < 4u; k++) {
+                            const uint32_t s = 0u - ((livec >> k) & 1u);  // all ones for a live class
+                            lo.x |= ca[k].x & s; lo.y |= ca[k].y & s; lo.z |= ca[k].z & s; lo.w |= ca[k].w & s;
+                            hi.x |= cx[k].x & s; hi.y |= cx[k].y & s; hi.z |= cx[k].z & s; hi.w |= cx[k].w & s;
+                            mlo.x |= ma[k].x; mlo.y |= ma[k].y; mlo.z |= ma[k].z; mlo.w |= ma[k].w;
+                            mhi.x |= mx[k].x; mhi.y |= mx[k].y; mhi.z |= mx[k].z; mhi.w |= mx[k].w;
+                        }
+                        if (((livec | mmask) >> 4) != 0u) {
 #pragma unroll 1
-                            for (uint32_t k = 0; k < 8u; k++) {
+                            for (uint32_t k = 4; k < 8u; k++) {
                                 if ((livec >> k) & 1u) {
                                     const uint4 a = ldg_nc(th + kScanHdrClassBits + 2u * k), x = ldg_nc(th + kScanHdrClassBits + 2u * k + 1u);
                                     lo.x |= a.x; lo.y |= a.y; lo.z |= a.z; lo.w |= a.w;
@@ -584,9 +616,9 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                                     mhi.x |= x.x; mhi.y |= x.y; mhi.z |= x.z; mhi.w |= x.w;
                                 }
                             }
-                            lo.x &= mlo.x; lo.y &= mlo.y; lo.z &= mlo.z; lo.w &= mlo.w;
-                            hi.x &= mhi.x; hi.y &= mhi.y; hi.z &= mhi.z; hi.w &= mhi.w;
                         }
+                        lo.x &= mlo.x; lo.y &= mlo.y; lo.z &= mlo.z; lo.w &= mlo.w;
+                        hi.x &= mhi.x; hi.y &= mhi.y; hi.z &= mhi.z; hi.w &= mhi.w;
                     }
                     if ((lo.x | lo.y | lo.z | lo.w | hi.x | hi.y | hi.z | hi.w) == 0u) {
                         pos = tile * kTTile + recs;  // nothing to look at in this tile
@@ -675,6 +707,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                 // statistics of completed requests, all lanes together
                 if (__any_sync(kFullMaskT, e.qn >= (uint32_t)(kTQueue - 1))) t_flush_now(e);
                 if (state == kLaneWait) {
+                    async_copies_done();  // of earlier rounds: none in flight while this round admits
                     const uint32_t req = pos;
                     const uint4* const full = cooked + (size_t)req * kCookedWords;
                     const CookedReq q = decode_cooked(ldg_nc(full), ldg_nc(full + 1), ldg_nc(full + 2));
@@ -739,9 +772,11 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                         } else {
                             TInst in;
                             t_load(e.hp, e.rowtab, bj, in);
+                            TKeys ks{0u, 0u, 0ull};
                             bool admit = true;
                             uint32_t kadd = 0;
                             if ((best >> 63) == 0) {
+                                ks = t_load_keys(e.pl, bj, in);
                                 in.T = bT;  // the clock as the prediction saw it
                                 kadd = bk;
                             } else {
@@ -749,7 +784,8 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                                 now = in.tc;
                                 if (!OPT) {
                                     tries++;  // the second round, counted only
-                                    t_advance_events(in, bj, now, false, e);
+                                    ks = t_load_keys(e.pl, bj, in);
+                                    t_events(in, ks, now, false, e);
                                 } else {
                                     admit = false;
                                     if (tries >= kAttemptCap) {
@@ -759,7 +795,7 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                                 }
                             }
                             if (admit) {
-                                t_admit(in, bj, q, req, bpre, kadd, e);
+                                t_admit(in, ks, bj, q, req, bpre, kadd, e);
                                 rej_sum -= q.rej;
                                 pending = false;
                                 lb_new = min(lb1j == bj ? lb2 : lb1, (in.w < in.B ? in.T : in.tc) + (int64_t)in.pre_base);
