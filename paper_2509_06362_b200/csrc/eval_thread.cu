@@ -341,7 +341,11 @@ struct ThreadSmem {
     unsigned char* hpool; // hot part of the instances
     unsigned char* pool;  // cold part (shared-memory mode)
 };
-__host__ __device__ inline uint32_t t_hot_units(uint32_t n_models) { return ((n_models + 7u) >> 3) + n_models + 2u; }
+// per lane: model ranges (8 models per unit), one entry per model, the classes each model can serve at all
+// (one word per model), the live map of the current tile (2 units)
+__host__ __device__ inline uint32_t t_hot_units(uint32_t n_models) {
+    return ((n_models + 7u) >> 3) + n_models + ((n_models + 3u) >> 2) + 2u;
+}
 __host__ __device__ inline size_t t_fixed_smem(uint32_t n_models, uint32_t n_rows) {
     return (size_t)t_hot_units(n_models) * 512u + (size_t)kTQueue * 32 * (16 + 8 + 8) + (((size_t)n_rows * 8u + 15u) & ~(size_t)15u);
 }
@@ -410,7 +414,8 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
     // a lane's hot units: [0, rr) per-model instance ranges, [rr, rr + M) one entry per model (lower bound
     // of any predicted first token, smallest prefill base, smallest prediction step), then the live map
     const uint32_t rr = (P.n_models + 7u) >> 3;
-    const uint32_t lm = rr + P.n_models;  // first unit of the live map
+    const uint32_t cfu = rr + P.n_models;                  // per model: the classes whose TBT limit some instance can meet
+    const uint32_t lm = cfu + ((P.n_models + 3u) >> 2);    // first unit of the live map
     const TPool hot{sm.hot + lane * 16u, 512u};
 
     TStats ls;
@@ -529,6 +534,16 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                     }
                     // nothing runs yet: every predicted first token lies at or after the smallest prefill base
                     for (uint32_t m = 0; m < P.n_models; m++) *hot.unit(rr + m) = make_uint4(min_pre[m], 0u, min_pre[m], min_step[m]);
+                    // A request of more than one token is served only by an instance whose prediction step meets
+                    // the class's TBT limit (Sec. IV-F step 3).  Which classes a model's instances can serve at all
+                    // is fixed for the placement: bit c of the model's word (classes 32 and up are not filtered).
+                    for (uint32_t m = 0; m < P.n_models; m++) *hot.word(cfu + (m >> 2), m & 3u) = 0u;
+                    for (uint32_t c = 0; c < P.n_classes && c < 32u; c++) {
+                        const int64_t l_tbt = P.classes[c * 3u + 1u];
+                        const uint32_t t32 = (l_tbt < 0 || l_tbt > 0xFFFFFFFFll) ? 0xFFFFFFFFu : (uint32_t)l_tbt;
+                        for (uint32_t m = 0; m < P.n_models; m++)
+                            if (t32 == 0xFFFFFFFFu || min_step[m] <= t32) *hot.word(cfu + (m >> 2), m & 3u) |= 1u << c;
+                    }
                     cmask = use_mask ? P.class_mask[cand] : 0xFFFFFFFFu;
                     // header entries of a scan tile this lane has to look at (classes 7 and up share entry 7)
                     hmask = (cmask & 0x7Fu) | ((cmask >> 7) ? 0x80u : 0u);
@@ -655,18 +670,24 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
                         for (int k = 0; k < 4; k++) {
                             const uint32_t model = sr[k].w & 0xFFu;
                             // in the request subset, and a model the placement serves
-                            bool r = have[k] && ((cmask >> ((sr[k].w >> 8) & 31u)) & 1u) && ((hasmodel >> model) & 1u);
-                            if (r && sr[k].x != 0xFFFFFFFFu) {
+                            const uint32_t cls = (sr[k].w >> 8) & 0xFFu;
+                            bool r = have[k] && ((cmask >> (cls & 31u)) & 1u) && ((hasmodel >> model) & 1u);
+                            if (r) {
                                 // Too late whatever the instance?  Every predicted first token of this model lies at
                                 // or after flb: the dispatcher's clock plus the smallest prefill base, and the lower
                                 // bound kept from the latest look at the model's instances (times only move forward).
+                                // And no instance of the model may meet the class's TBT limit at all.  (One guarded block
+                                // with all its loads at the top: branches in this loop cost more than the work they skip.)
                                 const uint4 me = *hot.unit(rr + model);
+                                const uint32_t cf = *hot.word(cfu + (model >> 2), model & 3u);
+                                const uint32_t Sm1 = sr[k].w >> 16;
+                                const bool tbt_dead = Sm1 != 0u && cls < 32u && !((cf >> cls) & 1u);
                                 const int64_t arrival = tile_base + (int64_t)sr[k].x;
                                 const int64_t flb = max(max(now, arrival) + (int64_t)me.z, (int64_t)(((uint64_t)me.y << 32) | me.x));
                                 const bool late_first = sr[k].y != 0xFFFFFFFFu && arrival + (int64_t)sr[k].y < flb;
-                                const bool late_end = sr[k].z != 0xFFFFFFFFu &&
-                                                      arrival + (int64_t)sr[k].z < flb + (int64_t)((uint64_t)(sr[k].w >> 16) * me.w);
-                                r = !(late_first || late_end);
+                                const bool late_end = sr[k].z != 0xFFFFFFFFu && arrival + (int64_t)sr[k].z < flb + (int64_t)((uint64_t)Sm1 * me.w);
+                                // an arrival offset of all ones does not fit 32 bits: the distributor looks at the full record
+                                r = !(tbt_dead || (sr[k].x != 0xFFFFFFFFu && (late_first || late_end)));
                             }
                             real[k] = r;
                         }
@@ -703,7 +724,11 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
             // ---- a distributor round for the waiting lanes, once enough of them wait --------------------------
             const uint32_t wl = __ballot_sync(kFullMaskT, state == kLaneWait);
             const uint32_t act = __ballot_sync(kFullMaskT, state == kLaneScan);
-            if (wl != 0u && ((uint32_t)__popc(wl) >= theta || act == 0u)) {
+            // Once the bucket has run out of placements nothing is gained by collecting lanes for a round: what
+            // is left is a tail of placements whose own chains of rounds bound the launch, so a waiting lane
+            // is served at once.
+            const bool tail = __any_sync(kFullMaskT, lane < L && !open);
+            if (wl != 0u && ((uint32_t)__popc(wl) >= (tail ? 1u : theta) || act == 0u)) {
                 // statistics of completed requests, all lanes together
                 if (__any_sync(kFullMaskT, e.qn >= (uint32_t)(kTQueue - 1))) t_flush_now(e);
                 if (state == kLaneWait) {

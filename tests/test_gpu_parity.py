@@ -145,6 +145,44 @@ def test_large_placements_over_32_instances_every_engine(ctx, oracle_mod, flags)
         assert (gd[k] == wd[k]).all(), (k, flags)
 
 
+@pytest.mark.parametrize("flags", [0, 1])
+def test_thread_kernel_classes_no_instance_can_serve(ctx, oracle_mod, flags):
+    """The thread kernel turns a request away while scanning when no instance of its model can meet the
+    class's TBT limit (the prediction step of every instance is above it).  The cases around that rule:
+    such a request of ONE output token has no TBT term and must still be served; classes 32 and up are
+    never filtered there; a class without a TBT limit; the optimistic estimate, where the step of a lower
+    level may meet the limit although the step at the batch cap does not.  Records, per-request times and
+    per-model rejection counts against the oracle."""
+    import torch
+    prof = gen.profile_multimodel(0)
+    # model 1 / strategy 9 / cap 64: 71 ms per step at the cap, 35 ms at level 1; model 2 is slower still
+    lists = [[(1, 9, 64), (1, 9, 64)], [(1, 9, 64), (2, 5, 8), (0, 6, 4)], [(2, 9, 64)], [(1, 9, 2), (1, 5, 32)],
+             [(0, 0, 64), (1, 3, 64), (2, 6, 1)], [(2, 3, 1), (2, 4, 2), (1, 8, 64)]]
+    off, inst = gen.candidates_from_lists(lists)
+    rows = [(500_000, 50_000, None), (2_000_000, 150_000, None), (None, None, 180_000_000), (None, 40_000, None)]
+    rows += [(3_000_000, 60_000 + 5_000 * k, None) for k in range(36)]          # classes 4..39, some beyond bit 31
+    classes = gen.make_classes(rows)
+    tr = gen.make_trace(6000, 80.0, 17, model_mix=(0.3, 0.4, 0.3), class_mix=(0.25, 0.2, 0.1, 0.15) + (0.3 / 36,) * 36)
+    tr["out_tokens"][::5] = 1                                                   # no TBT term for these
+    tr["out_tokens"][1::9] = 2
+    idx = np.arange(len(lists), dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(prof, tr, classes, off, inst, 1024, None, flags, dump_idx=idx)
+    got, gd = gpu_eval(ctx, prof, tr, classes, off, inst, 1024, None, flags, 3, dump_idx=idx)
+    assert (want["status"] == 0).all()
+    assert_records_equal(got, want, f"classes no instance can serve, flags {flags}")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+    served_single = (wd["finish_us"][0] >= 0) & (tr["out_tokens"] == 1) & (tr["cls"] == 0) & (tr["model"] == 1)
+    assert served_single.any()        # the case exists: class 0 on the 71 ms instances, served because of one token
+    ctx.load_profile(prof)
+    t = ctx.load_trace(tr, classes)
+    rbm = torch.full((len(lists), 16), 77, dtype=torch.int32, device="cuda")
+    ctx.eval_placements(t, ctx.to_device(off), ctx.to_device(inst), 1024, None, flags, 3, rejected_by_model=rbm)
+    torch.cuda.synchronize()
+    assert (rbm.cpu().numpy().view(np.uint32) == oracle_mod.rejected_by_model(prof, tr, classes, off, inst, 1024, flags=flags)).all()
+    ctx.free_trace(t)
+
+
 @pytest.mark.parametrize("flags,mapping", [(0, 2), (2, 0), (8, 0), (4, 0)])
 def test_large_placements_several_traces_in_one_pass(ctx, oracle_mod, flags, mapping):
     """The same placements against three traces in one call, where the thread kernel is not used (lane
