@@ -45,6 +45,7 @@ constexpr int kTQueue = MAASO_TQUEUE;           // queued completions per lane
 #ifndef MAASO_THREAD_BPS
 #define MAASO_THREAD_BPS 12
 #endif
+constexpr int kTScanSteps = 2;                     // scan iterations between two looks at the waiting lanes
 constexpr int kTBlocksPerSM = MAASO_THREAD_BPS;    // one-warp blocks per SM the register budget allows (3 per scheduler)
 
 // Lanes that work on one item, by launch bucket (bucket 9 = placements the pool cannot hold at all).
@@ -569,8 +570,10 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
             if (!__any_sync(kFullMaskT, state != kLaneIdle)) break;  // the bucket is done as far as this warp goes
 
             // ---- scan iterations -------------------------------------------------------------------------------
+            // Two per pass (measured: 1, 2, 3, 4, 6): a lane that has found its request idles through the rest
+            // of them, a lane that still scans idles through the round that follows.
 #pragma unroll 1
-            for (int c = 0; c < 4; c++) {
+            for (int c = 0; c < kTScanSteps; c++) {
                 if (state != kLaneScan) continue;
                 const uint32_t tile = pos / (uint32_t)kTTile;
                 const uint4* const th = scan + (size_t)tile * (kScanTile + kScanHdrUnits);
