@@ -45,6 +45,7 @@ constexpr int kTQueue = MAASO_TQUEUE;           // queued completions per lane
 #ifndef MAASO_THREAD_BPS
 #define MAASO_THREAD_BPS 12
 #endif
+constexpr int kTDoneLanes = 2;                     // finished lanes that are handled together
 constexpr int kTScanSteps = 2;                     // scan iterations between two looks at the waiting lanes
 constexpr int kTBlocksPerSM = MAASO_THREAD_BPS;    // one-warp blocks per SM the register budget allows (3 per scheduler)
 
@@ -838,7 +839,12 @@ eval_thread_kernel(const __grid_constant__ EvalParams P, const uint32_t pool_byt
             }
 
             // ---- lanes that are through their trace: drain, account what is still queued, write the record -----
-            if (__any_sync(kFullMaskT, state == kLaneDone)) {
+            // Two of them together where it can be had (the drain, the record and the set-up of the next placement are long paths
+            // that a lane alone would walk with the other 31 idle), unless nobody else is at work or the bucket
+            // has run out.
+            const uint32_t dn = __ballot_sync(kFullMaskT, state == kLaneDone);
+            if (dn != 0u && ((uint32_t)__popc(dn) >= (uint32_t)kTDoneLanes || tail ||
+                             !__any_sync(kFullMaskT, state == kLaneScan || state == kLaneWait))) {
                 if (state == kLaneDone) {
                     if (status == 0) {
                         for (uint32_t j = 0; j < n_i; j++) {
