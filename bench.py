@@ -29,7 +29,13 @@ TOPK = 64
 
 # ncu counters of the dominant kernel on the default workload (see profiles/).  They describe the
 # kernels whose source hashes to `csrc_sha256`; with any other source they are not printed.
-PROFILED = None
+PROFILED = {
+    "workload": "multimodel", "mapping": 0, "kernel": "eval_thread_kernel",
+    # profiles/eval_thread_kernel_multimodel_sweep_counters.md: one launch of the default workload
+    "warp_inst_per_launch": 46563395435,                 # smsp__inst_executed.sum
+    "dram_bytes_per_launch": 8580613888 + 6594006784,    # dram__bytes_read.sum + dram__bytes_write.sum
+    "csrc_sha256": "2e1044a5122c150cc97bb4ec46fbcf4a226c4c27ab5065b7bd1d91467fe5f806",
+}
 SM_COUNT, ISSUE_PER_SM = 148, 4   # B200: 148 SMs x 4 warp schedulers, one warp instruction per cycle each
 
 
