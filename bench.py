@@ -303,6 +303,12 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    # the clock sampler starts (and settles) before the warm-up, so that the timed steps follow the warm-up
+    # steps directly and no idle gap lets the GPU leave its loaded state
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
     for _ in range(args.warmup):
         flush.fill_(1)
         step()
@@ -314,10 +320,6 @@ def main():
         dist.all_reduce(evals_t)
     evals_per_step = int(evals_t.item())      # of the whole sweep, all ranks
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
     launches0 = ctx.launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
           for _ in range(args.steps)]
