@@ -75,3 +75,35 @@ def test_random_case_every_engine_and_mapping(ctx, oracle_mod, seed):
             assert_records_equal(got, want, f"seed {seed}, flags {flags}, mapping {mapping}")
             for k in wd:
                 assert (gd[k] == wd[k]).all(), (seed, flags, mapping, k)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_case_several_traces_in_one_pass(oracle_mod, seed, monkeypatch):
+    """The same kind of workload against three traces in one call, under both routings of the default
+    mapping (the thread kernel takes the loaded part of the batch / only what the lane groups cannot)."""
+    import torch
+    import paper_2509_06362_b200 as m
+    prof, off, inst, classes, tr, mask = _case(100 + seed)
+    n = len(tr)
+    traces_np = [tr[: n // 2].copy(), tr[n // 3:].copy(), tr.copy()]
+    for t in traces_np:
+        t["arrival_us"] -= t["arrival_us"][0]
+    rng = np.random.default_rng(seed)
+    for min_cand in ("0", "1000000"):
+        monkeypatch.setenv("MAASO_THREAD_MIN_CAND", min_cand)
+        c = m.Context(0)
+        c.load_profile(prof)
+        handles = [c.load_trace(t, classes) for t in traces_np]
+        d_mask = None if mask is None else c.to_device(mask)
+        for flags in (0, int(rng.choice([1, 2, 4, 8]))):
+            mappings = [0, 2, 3] if flags < 2 else [0, 2]
+            want = [oracle_mod.eval_placements(prof, t, classes, off, inst, 1024, mask, flags) for t in traces_np]
+            for mapping in mappings:
+                out = c.eval_placements_multi(handles, c.to_device(off), c.to_device(inst), 1024, d_mask, flags,
+                                              mapping=mapping)
+                torch.cuda.synchronize()
+                got = c.results_to_numpy(out).reshape(len(traces_np), -1)
+                for k in range(len(traces_np)):
+                    assert_records_equal(got[k], want[k], f"seed {seed}, trace {k}, flags {flags}, mapping {mapping}, "
+                                                          f"routing threshold {min_cand}")
+        c.close()
