@@ -103,8 +103,7 @@ extern "C" {
 #define MAASO_MAP_AUTO 0u   /* the library chooses: MAASO_MAP_THREAD where it exists, else MAASO_MAP_GROUP */
 #define MAASO_MAP_BLOCK 1u  /* one thread block per candidate, one warp per instance, lanes = slots */
 #define MAASO_MAP_GROUP 2u  /* one lane per instance, groups of lanes per candidate (<= 32 instances; beyond
-                               that one block per candidate, or, with several traces in one pass, one warp
-                               per candidate with four instances per lane) */
+                               that one warp per candidate with four instances per lane) */
 #define MAASO_MAP_THREAD 3u /* one thread per candidate, looping over the instances of the request's model;
                                default engine only (flags 0 or MAASO_FLAG_PRED_OPTIMISTIC), any instance count */
 
@@ -224,8 +223,8 @@ MAASO_API void maaso_free_trace(maaso_ctx *ctx, maaso_trace *trace);
  * slots (Sec. V-A), and write one record per candidate to out_results (device,
  * [n_cand]).  Work is enqueued on `cuda_stream` (a cudaStream_t, NULL = default stream).
  * opts->mapping chooses the kernel: MAASO_MAP_AUTO (default) lets the library route the batch (large
- * batches of placements that the trace overloads go to the thread kernel, the rest to the lane groups;
- * placements of more than 32 instances always to the thread kernel); the records do not depend on it.
+ * batches of placements that the trace overloads go to the thread kernel, the rest to the lane groups,
+ * where a placement of more than 32 instances gets a warp of its own); the records do not depend on it.
  * The context's scratch memory grows on demand (this may allocate and synchronise on the
  * first call or when a batch is larger than any before). */
 MAASO_API int maaso_eval_placements(maaso_ctx *ctx, const maaso_trace *trace, const maaso_cand_batch *cands,
@@ -238,10 +237,10 @@ MAASO_API int maaso_eval_placements(maaso_ctx *ctx, const maaso_trace *trace, co
  * out_results[t * n_cand + c]; opts->rejected_by_model and opts->ttft_hist, if given, are laid out
  * the same way ([n_traces * n_cand][...]).  Each record equals what maaso_eval_placements returns
  * for that trace alone; scoring them together lets small candidate sets fill the GPU.  Lane-group
- * and thread mappings only: dump buffers and MAASO_MAP_BLOCK are refused.  With the default engine a
- * placement of more than 32 instances is scored by the thread kernel; with MAASO_MAP_GROUP or one of
- * the other engines one warp replays it with the lane-group code (four instances per lane).  No engine
- * and no mapping refuses a placement of MAASO_MAX_INSTANCES instances or fewer.  Enqueued on cuda_stream. */
+ * and thread mappings only: dump buffers and MAASO_MAP_BLOCK are refused.  A placement of more than 32
+ * instances is scored by the thread kernel where the batch goes there, else one warp replays it with the
+ * lane-group code (four instances per lane).  No engine and no mapping refuses a placement of
+ * MAASO_MAX_INSTANCES instances or fewer.  Enqueued on cuda_stream. */
 MAASO_API int maaso_eval_placements_multi(maaso_ctx *ctx, const maaso_trace *const *traces, uint32_t n_traces,
                                           const maaso_cand_batch *cands, const maaso_eval_opts *opts,
                                           maaso_result *out_results, void *cuda_stream);

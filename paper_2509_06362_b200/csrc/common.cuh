@@ -24,10 +24,10 @@ constexpr int kThreadBucket0 = 10;  // buckets 10..18: the thread mapping, by la
 constexpr int kThreadBuckets = 9;
 constexpr int kWideBucket = 19;     // 33..128 instances under the engines of the lane-group code: one warp per placement
 constexpr int kCostBins = 256;   // bin 0 = most expensive (largest total batch cap)
-constexpr int kCounterWords = 16384;  // counters | work counters | histograms + cursors, cleared per call
+constexpr int kCounterWords = 17408;  // counters | work counters | histograms + cursors, cleared per call
 // histogram sets (rows of kCostBins words in EvalParams::hist): candidates that can only go to a lane-group
 // or block bucket, only to a thread bucket, or either way (counted once per side); then the write cursors
-constexpr int kHistOnlyG = 0, kHistBothG = 10, kHistOnlyT = 20, kHistBothT = 29, kHistWide = 38, kHistCursor = 39;
+constexpr int kHistOnlyG = 0, kHistBothG = 10, kHistOnlyT = 20, kHistBothT = 29, kHistWide = 38, kHistBothW = 39, kHistCursor = 40;
 constexpr int kHistRows = kHistCursor + kNumBuckets;
 // counters beside the bucket counts (EvalParams::bucket_count[0..31])
 constexpr int kCtrBoth = 24, kCtrLoaded = 25, kCtrCut = 26, kCtrUseThreads = 27;

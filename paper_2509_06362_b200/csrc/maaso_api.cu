@@ -591,16 +591,9 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     }
     int grid_b[4];
     for (int b = 6; b <= kGenericBlockBucket; b++) {
-        // without the block mapping only candidates the other kernel cannot take go to a block kernel:
-        // more than 32 instances (lane groups), or a state larger than a warp's pool (thread mapping)
-        bool used = n_traces == 1 && o.mapping == MAASO_MAP_BLOCK;
-        if (n_traces == 1 && b == kGenericBlockBucket) {
-            // more than 32 instances: the thread kernel where it can run, else one block per placement
-            if (o.mapping == MAASO_MAP_GROUP) used = cands->n_inst > 32;
-            if (threads) used = cands->n_inst * 20ull > P.thread_pool_units || cands->n_inst * 2ull > P.thread_hot_units;  // 22 units: an instance with 64 slots
-        }
+        // the block kernels run only when the block mapping is asked for
         grid_b[b - 6] = 0;
-        if (!used) continue;
+        if (!(n_traces == 1 && o.mapping == MAASO_MAP_BLOCK)) continue;
         // placements with at most 8 instances: one warp per instance with register-resident state
         int gb = ctx->sm_count * (b < kGenericBlockBucket ? occupancy_eval_block_reg(P, b, tile)
                                                         : occupancy_eval_block(P, b, tile));
@@ -610,15 +603,19 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
         if (need > pay_entries) pay_entries = need;
     }
 
-    // placements of more than 32 instances under the other engines, or with several traces where the thread
-    // kernel is not used: one warp per placement with the lane-group code
+    // placements of more than 32 instances outside the thread kernel (the other engines; the default engine
+    // unless the batch goes to the threads; whatever the thread kernel's pools cannot hold): one warp per
+    // placement with the lane-group code
     int grid_w = 0;
-    if (o.mapping != MAASO_MAP_BLOCK && cands->n_inst > 32 && (variant || n_traces > 1)) {
+    if (o.mapping != MAASO_MAP_BLOCK && cands->n_inst > 32) {
         // at most as many warps as the lane-group grid has blocks: a warp's scratch is a lane-group block's
         int occ_w = occupancy_eval_wide(P);
         if (occ_w > 4) occ_w = 4;
         grid_w = ctx->sm_count * occ_w;
-        const uint64_t max_items_w = (uint64_t)C * n_traces;
+        // a placement that needs this kernel has more than 32 instances (or, thread mapping forced, more state
+        // than a warp's pools): the batch cannot hold more of them than instances / 33
+        uint64_t max_items_w = (o.mapping == MAASO_MAP_THREAD ? (uint64_t)C : cands->n_inst / 33u) * n_traces;
+        if (max_items_w < 1) max_items_w = 1;
         if ((uint64_t)grid_w > max_items_w) grid_w = (int)max_items_w;
         const size_t need = ((size_t)grid_w * wide_scratch_per_warp() + sizeof(Payload) - 1) / sizeof(Payload);
         if (need > pay_entries) pay_entries = need;

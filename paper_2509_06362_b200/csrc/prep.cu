@@ -54,11 +54,10 @@ __global__ void prep_kernel(const EvalParams P) {
         }
         if (P.mapping == MAASO_MAP_BLOCK) bg = n <= 2 ? 6 : (n <= 4 ? 7 : (n <= 8 ? 8 : kGenericBlockBucket));
         else if (groups_ok && n <= 32) bg = n <= 1 ? 0 : 32 - __clz((int)(n - 1));
-        // More than 32 instances: the thread mapping if it can hold the placement, else one block per
-        // placement (default engine, one trace), else (the other engines, several traces in one pass)
-        // one warp per placement with the lane-group code.
-        if (n > 32 && bt >= 0) bg = -1;
-        if (bg < 0 && bt < 0) bg = (!variant && P.n_traces <= 1) ? kGenericBlockBucket : kWideBucket;
+        // More than 32 instances: one warp per placement with the lane-group code (every engine), or the thread
+        // mapping where that exists and can hold the placement; the batch-wide choice of plan_kernel decides
+        // between the two.  (One block per placement only when the block mapping is asked for.)
+        if (bg < 0 && (groups_ok || bt < 0)) bg = kWideBucket;
     }
     if (P.dump_row) P.dump_row[c] = -1;
     const uint32_t n_traces = P.n_traces > 1 ? P.n_traces : 1u;
@@ -84,7 +83,7 @@ __global__ void prep_kernel(const EvalParams P) {
     P.code[c] = bg >= 0 ? (((uint32_t)bg << 8) | bin) : 0xFFFFFFFFu;
     P.code2[c] = bt >= 0 ? (((uint32_t)bt << 8) | bin) : 0xFFFFFFFFu;
     if (bg >= 0 && bt >= 0) {
-        atomicAdd(&P.hist[(kHistBothG + bg) * kCostBins + bin], 1u);
+        atomicAdd(&P.hist[(bg == kWideBucket ? kHistBothW : kHistBothG + bg) * kCostBins + bin], 1u);
         atomicAdd(&P.hist[(kHistBothT + bt - kThreadBucket0) * kCostBins + bin], 1u);
         // loaded beyond what it can decode: most of its requests will be turned away, which the
         // thread mapping does for next to nothing
@@ -134,7 +133,7 @@ __global__ void __launch_bounds__(kCostBins) plan_kernel(const EvalParams P) {
     for (int b = kThreadBucket0; b < kThreadBucket0 + kThreadBuckets; b++)
         cnt[b] = P.hist[(kHistOnlyT + b - kThreadBucket0) * kCostBins + bin] +
                  (use_threads ? P.hist[(kHistBothT + b - kThreadBucket0) * kCostBins + bin] : 0u);
-    cnt[kWideBucket] = P.hist[kHistWide * kCostBins + bin];
+    cnt[kWideBucket] = P.hist[kHistWide * kCostBins + bin] + (use_threads ? 0u : P.hist[kHistBothW * kCostBins + bin]);
     uint32_t cut = 0;  // bins below `cut` are promoted
     uint32_t narrow = 0;
     for (int b = 0; b < 5; b++) narrow += cnt[b];
