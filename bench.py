@@ -121,7 +121,7 @@ def algorithmic_bytes(cfg, evals):
     return evals * 16 + 4 * len(cfg["inst"]) + 8 * n_cand + 128 * n_cand + prof_bytes
 
 
-FULL_CANDIDATES = {"tiny": 143, "node": 10_864, "bursty": 10_864, "multimodel": 100_000, "scale": 1_000_000}
+FULL_CANDIDATES = {"tiny": 143, "node": 10_864, "bursty": 10_864, "multimodel": 100_000, "scale": 1_000_000, "large": 2_000}
 
 
 def workload_label(name, n_cand, n_req, n_tr, budget):
@@ -130,9 +130,9 @@ def workload_label(name, n_cand, n_req, n_tr, budget):
             f"{f' x {n_tr} traces in one pass' if n_tr > 1 else ''}, budget {budget}, top-{TOPK}")
 
 
-def oracle_pass(oracle, cfg):
+def oracle_pass(oracle, cfg, flags=0):
     res = oracle.eval_placements(cfg["profile"], cfg["traces"][0], cfg["classes"], cfg["offsets"],
-                                 cfg["inst"], cfg["budget"])
+                                 cfg["inst"], cfg["budget"], None, flags)
     oracle.topk(res, TOPK)
     return int(res["n_counted"][res["status"] == 0].astype(np.int64).sum())
 
@@ -166,7 +166,7 @@ def run_reference(args):
     times, evals = [], 0
     for step in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        ev = oracle_pass(oracle, cfg)
+        ev = oracle_pass(oracle, cfg, args.flags)
         dt = time.perf_counter() - t0
         if step >= args.warmup:
             times.append(dt)
@@ -195,7 +195,7 @@ def cpu_baseline(args):
     oracle.build()
     cfg, how = sample_of(gen, args.workload, args.n_cand, args.n_req, 4096 if args.workload != "scale" else 256)
     t0 = time.perf_counter()
-    evals = oracle_pass(oracle, cfg)
+    evals = oracle_pass(oracle, cfg, args.flags)
     dt = time.perf_counter() - t0
     return {"value": evals / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": f"{how} x all {len(cfg['traces'][0])} requests, {dt:.1f} s, 1 thread; the rate is that of "
@@ -243,6 +243,7 @@ def main():
     ap.add_argument("--workload", default="multimodel", help="multimodel (default) or another configuration name")
     ap.add_argument("--n-cand", type=int, default=None)
     ap.add_argument("--n-req", type=int, default=None)
+    ap.add_argument("--flags", type=int, default=0, help="engine flags of maaso_eval_placements (0: the default engine)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-scale-slice", action="store_true")
     args = ap.parse_args()
@@ -289,9 +290,9 @@ def main():
 
     def step():
         if n_tr > 1:
-            ctx.eval_placements_multi(traces, d_off, d_inst, cfg["budget"], out=results, stream=stream)
+            ctx.eval_placements_multi(traces, d_off, d_inst, cfg["budget"], flags=args.flags, out=results, stream=stream)
         else:
-            ctx.eval_placements(trace, d_off, d_inst, cfg["budget"], mapping=args.mapping, out=results,
+            ctx.eval_placements(trace, d_off, d_inst, cfg["budget"], flags=args.flags, mapping=args.mapping, out=results,
                                 stream=stream)
         if world == 1:
             return ctx.topk(results, TOPK, stream=stream)
@@ -358,9 +359,9 @@ def main():
         d_off2.copy_(off_pin, non_blocking=True)
         d_inst2.copy_(inst_pin, non_blocking=True)
         if n_tr > 1:
-            ctx.eval_placements_multi(traces, d_off2, d_inst2, cfg["budget"], out=results, stream=stream)
+            ctx.eval_placements_multi(traces, d_off2, d_inst2, cfg["budget"], flags=args.flags, out=results, stream=stream)
         else:
-            ctx.eval_placements(trace, d_off2, d_inst2, cfg["budget"], mapping=args.mapping, out=results, stream=stream)
+            ctx.eval_placements(trace, d_off2, d_inst2, cfg["budget"], flags=args.flags, mapping=args.mapping, out=results, stream=stream)
         if world == 1:
             idx, top = ctx.topk(results, TOPK, stream=stream)
             top_idx_pin.copy_(idx, non_blocking=True)
@@ -399,13 +400,15 @@ def main():
     peak, peak_kind = measured_peak()
     mean_ms = {k: statistics.mean(x[k] for x in kernel_ms) for k in kernel_ms[0]}
     dom = max(("thread_ms", "group_ms", "block_ms"), key=lambda k: mean_ms[k])
-    dom_kernel = {"thread_ms": "eval_thread_kernel", "group_ms": "eval_group_kernel", "block_ms": "eval_block_kernel"}[dom]
+    # block_ms covers the block kernels (block mapping) and the one-warp-per-placement kernel (other mappings)
+    dom_kernel = {"thread_ms": "eval_thread_kernel", "group_ms": "eval_group_kernel",
+                  "block_ms": "eval_block_kernel" if args.mapping == 1 else "eval_wide_kernel"}[dom]
     dom_ms = mean_ms[dom]
     # the dominant kernel's launch on rank 0 processes rank 0's shard
     abytes = algorithmic_bytes({"offsets": off_np, "inst": inst_np, "profile": cfg["profile"]}, evals_rank)
     achieved = abytes / (dom_ms * 1e-3) / 1e9
     profiled = None
-    if (PROFILED and args.workload == PROFILED["workload"] and args.mapping == PROFILED["mapping"] and world == 1
+    if (PROFILED and args.workload == PROFILED["workload"] and args.mapping == PROFILED["mapping"] and world == 1 and args.flags == 0
             and args.n_cand is None and args.n_req is None and PROFILED["kernel"] == dom_kernel
             and PROFILED["csrc_sha256"] == csrc_sha256()):
         profiled = PROFILED
@@ -426,6 +429,7 @@ def main():
         "scaling": "strong", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
         "config": {"workload": workload_label(cfg["name"], n_total, len(trace_np), n_tr, cfg["budget"]),
                    "evals_per_step": evals_per_step, "mapping": {0: "auto", 1: "block", 2: "lane groups", 3: "threads"}[args.mapping],
+                   "engine_flags": args.flags,
                    "l2": "flushed between timed steps (256 MB write)",
                    "per_gpu": "one sweep, contiguous candidate shards" if world > 1 else "the whole sweep"},
         "clocks": clocks,

@@ -98,6 +98,20 @@ def make_config(name, n_cand=None, n_req=None):
                              out_dist=("lognormal", 5.0, 1.2, 1, 8192))]
         offsets, inst = sample_candidates(1_000_000 if n_cand is None else n_cand, 2, 128, prof)
         budget = 128
+    elif name == "large":
+        # Not one of the five benchmark configurations: placements of 33 to 128 instances on a modelled
+        # cluster of 1,024 devices, the case the one-warp-per-placement kernel exists for.
+        prof = profile_multimodel(0)
+        classes = make_classes([_INTERACTIVE, _CHAT, _DOCUMENT, _BATCH])
+        traces = [make_trace(10_000 if n_req is None else n_req, 400.0, 9,
+                             class_mix=(0.45, 0.27, 0.18, 0.10), model_mix=(0.6, 0.3, 0.1))]
+        want = 2_000 if n_cand is None else n_cand
+        offsets, inst = sample_candidates(3 * want + 64, 3, 1024, prof, stop_p=0.015)
+        keep = np.nonzero(np.diff(offsets.astype(np.int64)) > 32)[0][:want]
+        parts = [inst[offsets[c]:offsets[c + 1]] for c in keep]
+        offsets = np.concatenate([[0], np.cumsum([len(x) for x in parts])]).astype(np.uint32)
+        inst = np.concatenate(parts).astype(np.uint32)
+        budget = 1024
     elif name.startswith("table1-"):
         return make_table1_config(int(name.split("-")[1]), n_cand=2000 if n_cand is None else n_cand,
                                   n_req=17_000 if n_req is None else n_req)

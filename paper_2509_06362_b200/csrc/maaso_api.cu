@@ -608,9 +608,10 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     // placement with the lane-group code
     int grid_w = 0;
     if (o.mapping != MAASO_MAP_BLOCK && cands->n_inst > 32) {
-        // at most as many warps as the lane-group grid has blocks: a warp's scratch is a lane-group block's
+        // as many warps per SM as the registers allow (8): the kernel waits on dependent chains, and four
+        // more warps per SM are worth a third of its time; a warp's scratch is a lane-group block's (1 MB)
         int occ_w = occupancy_eval_wide(P);
-        if (occ_w > 4) occ_w = 4;
+        if (occ_w > 8) occ_w = 8;
         grid_w = ctx->sm_count * occ_w;
         // a placement that needs this kernel has more than 32 instances (or, thread mapping forced, more state
         // than a warp's pools): the batch cannot hold more of them than instances / 33

@@ -145,6 +145,25 @@ def test_large_placements_over_32_instances_every_engine(ctx, oracle_mod, flags)
         assert (gd[k] == wd[k]).all(), (k, flags)
 
 
+@pytest.mark.parametrize("flags,mapping", [(0, 0), (0, 3), (1, 0), (2, 0), (8, 0), (4, 0)])
+def test_large_configuration_sample(ctx, oracle_mod, flags, mapping):
+    """The configuration of placements with 33 to 128 instances (2,000 of them in full): every 25th
+    against the whole trace, one warp per placement (and the thread kernel, forced)."""
+    cfg = gen.make_config("large")
+    sel = np.arange(0, len(cfg["offsets"]) - 1, 25)
+    parts = [cfg["inst"][cfg["offsets"][c]:cfg["offsets"][c + 1]] for c in sel]
+    off = np.concatenate([[0], np.cumsum([len(x) for x in parts])]).astype(np.uint32)
+    inst = np.concatenate(parts).astype(np.uint32)
+    tr = cfg["traces"][0]
+    idx = np.array([0, 40, 79], dtype=np.uint32)
+    want, wd = oracle_mod.eval_placements(cfg["profile"], tr, cfg["classes"], off, inst, cfg["budget"], None, flags, dump_idx=idx)
+    got, gd = gpu_eval(ctx, cfg["profile"], tr, cfg["classes"], off, inst, cfg["budget"], None, flags, mapping, dump_idx=idx)
+    assert (want["status"] == 0).all()
+    assert_records_equal(got, want, f"large configuration, flags {flags}, mapping {mapping}")
+    for k in wd:
+        assert (gd[k] == wd[k]).all(), k
+
+
 @pytest.mark.parametrize("flags", [0, 1])
 def test_thread_kernel_classes_no_instance_can_serve(ctx, oracle_mod, flags):
     """The thread kernel turns a request away while scanning when no instance of its model can meet the
