@@ -608,10 +608,13 @@ static int eval_impl(maaso_ctx* ctx, const maaso_trace* const* traces, uint32_t 
     // placement with the lane-group code
     int grid_w = 0;
     if (o.mapping != MAASO_MAP_BLOCK && cands->n_inst > 32) {
-        // as many warps per SM as the registers allow (8): the kernel waits on dependent chains, and four
-        // more warps per SM are worth a third of its time; a warp's scratch is a lane-group block's (1 MB)
+        // As many warps per SM as the registers allow (8) where the batch is made of large placements (more
+        // than 16 instances per placement on average): the kernel waits on dependent chains, and four more
+        // warps per SM are worth a third of its time.  Elsewhere 4 per SM, which needs no more scratch than
+        // the lane-group kernel has anyway (a warp's scratch is a lane-group block's, 1 MB).
         int occ_w = occupancy_eval_wide(P);
-        if (occ_w > 8) occ_w = 8;
+        const int occ_cap = cands->n_inst > 16ull * C ? 8 : 4;
+        if (occ_w > occ_cap) occ_w = occ_cap;
         grid_w = ctx->sm_count * occ_w;
         // a placement that needs this kernel has more than 32 instances (or, thread mapping forced, more state
         // than a warp's pools): the batch cannot hold more of them than instances / 33
