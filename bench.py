@@ -32,9 +32,9 @@ TOPK = 64
 PROFILED = {
     "workload": "multimodel", "mapping": 0, "kernel": "eval_thread_kernel",
     # profiles/eval_thread_kernel_multimodel_sweep_counters.md: one launch of the default workload
-    "warp_inst_per_launch": 46526339343,                 # smsp__inst_executed.sum
-    "dram_bytes_per_launch": 8570338560 + 6587270400,    # dram__bytes_read.sum + dram__bytes_write.sum
-    "csrc_sha256": "85668342bf3cefdaefa50be854ccfc0f314786f53727c4e0f4ae2c0440e75a24",
+    "warp_inst_per_launch": 46569990180,                 # smsp__inst_executed.sum
+    "dram_bytes_per_launch": 8544527616 + 6588603136,    # dram__bytes_read.sum + dram__bytes_write.sum
+    "csrc_sha256": "a0f7e33b28fbe2b47bfd948151d49416482dfd85dd16ebadee99caabcc78edd0",
 }
 SM_COUNT, ISSUE_PER_SM = 148, 4   # B200: 148 SMs x 4 warp schedulers, one warp instruction per cycle each
 
