@@ -146,7 +146,11 @@ __global__ void __launch_bounds__(kCostBins) plan_kernel(const EvalParams P) {
         }
         __syncthreads();
         for (int b = 0; b <= 5; b++) need += (tot[b] + (32u >> b) - 1) / (32u >> b);
-        const uint32_t spare = P.group_warps > need ? (uint32_t)((uint64_t)(P.group_warps - need) * P.promote_pct / 100) : 0;
+        // every work item exists once per trace, and a promoted candidate takes a warp in each of them
+        const uint32_t n_tr = P.n_traces > 1 ? P.n_traces : 1u;
+        const uint64_t need_all = (uint64_t)need * n_tr;
+        const uint32_t spare = P.group_warps > need_all
+                                   ? (uint32_t)((P.group_warps - need_all) / n_tr * P.promote_pct / 100) : 0;
         const uint32_t incl = block_inclusive_scan(narrow, buf);
         cut = (uint32_t)__syncthreads_count(incl <= spare);  // prefix sums are monotone
     }
