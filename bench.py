@@ -32,9 +32,9 @@ TOPK = 64
 PROFILED = {
     "workload": "multimodel", "mapping": 0, "kernel": "eval_thread_kernel",
     # profiles/eval_thread_kernel_multimodel_sweep_counters.md: one launch of the default workload
-    "warp_inst_per_launch": 46569990180,                 # smsp__inst_executed.sum
-    "dram_bytes_per_launch": 8544527616 + 6588603136,    # dram__bytes_read.sum + dram__bytes_write.sum
-    "csrc_sha256": "a0f7e33b28fbe2b47bfd948151d49416482dfd85dd16ebadee99caabcc78edd0",
+    "warp_inst_per_launch": 46573414946,                 # smsp__inst_executed.sum
+    "dram_bytes_per_launch": 8540173312 + 6593907712,    # dram__bytes_read.sum + dram__bytes_write.sum
+    "csrc_sha256": "38d6462581e8b3e93e08ae6faacbcde5536639edd825c4f14a4a1d54dd9372cb",
 }
 SM_COUNT, ISSUE_PER_SM = 148, 4   # B200: 148 SMs x 4 warp schedulers, one warp instruction per cycle each
 
