@@ -100,7 +100,8 @@ extern "C" {
                                              and the call must return normally */
 
 /* maaso_eval_opts.mapping */
-#define MAASO_MAP_AUTO 0u   /* the library chooses: MAASO_MAP_THREAD where it exists, else MAASO_MAP_GROUP */
+#define MAASO_MAP_AUTO 0u   /* the library routes the batch: threads for large batches of placements the trace
+                               overloads (default engine), else lane groups; see maaso_eval_placements */
 #define MAASO_MAP_BLOCK 1u  /* one thread block per candidate, one warp per instance, lanes = slots */
 #define MAASO_MAP_GROUP 2u  /* one lane per instance, groups of lanes per candidate (<= 32 instances; beyond
                                that one warp per candidate with four instances per lane) */
